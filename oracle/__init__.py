@@ -1,0 +1,17 @@
+"""CPU oracle for the tree-packed linear-attention path.  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline legs may import this
+package; the product (the CUDA library and its binding) never does, and this package
+never imports the product.
+
+Pins (see tests/test_oracle_*.py, tests/test_plan_oracle.py):
+  * la_oracle   -- token recurrence fwd/bwd: closed forms (cumulative sum, geometric
+                   series), the dense decay-masked matmul form, central finite differences,
+                   fp64 autograd of the dense form, equality with a depth-first compact
+                   evaluation of the tree, invariance to how dO is split over copies.
+  * plan_oracle -- Algorithm 1: brute-force minimum call counts on tiny trees, the worked
+                   examples of Figs. 1-3, the strict boundary cases, the replay total of
+                   Eq. 15, fp64 execution of the plan against la_oracle.
+  * Appendix planning cases I-III: parity unpinned (the trees' token counts were only in
+                   the figures); only the printed totals are checked for self-consistency.
+"""
