@@ -1,0 +1,205 @@
+/*
+ * harts_la -- tree-packed chunkwise linear attention for sm_100a (B200): C ABI.
+ *
+ * The operation (paper Section 3.3 "Minimum-Call Planning", Section 3.4 "Differentiable
+ * boundary states" / "Round-wise execution", Eq. 16): a forest of rollout trees is turned into
+ * compact token rows (each shared-prefix token stored once), grouped into the minimum number of
+ * sequential packed calls ("rounds", Algorithm 1).  Every sequence of a round starts from a zero
+ * state or from a chunk-boundary state that an earlier round exported ("slot"), replays the
+ * fewer-than-one-chunk ancestor interval between that boundary and its fork (Eq. 2), and then
+ * runs its own rows.  Gradients flow back through the state hand-off and through the replayed
+ * rows.  The recurrence is Eq. 1 specialised to a scalar gate:
+ *
+ *     S_t = exp(g_t) S_{t-1} + k_t^T v_t,     o_t = q_t S_t        (per head, S in R^{dk x dv})
+ *
+ * Conventions
+ *   - Every function returns an int32 status: HARTS_OK or a negative HARTS_E* code.  Nothing
+ *     throws, aborts or prints.  harts_la_strerror() gives text.
+ *   - The library allocates NO device memory.  Tensors, slots, workspaces and the uploaded index
+ *     tables are caller-owned device buffers; their sizes come from the query calls.
+ *   - "host" / "device" in a comment says where the pointer must point.
+ *   - Kernels are enqueued on the caller's stream (a cudaStream_t passed as void*) and the calls
+ *     return without synchronising.  Device-detected errors (a bounded wait that ran out) are
+ *     written to a caller-owned device status word and read back by harts_la_check().
+ *   - There is no CPU fallback: an unsupported (dtype, dk, dv, chunk) gives HARTS_EUNSUPPORTED.
+ *   - Tensor layout: row-major [rows, H, d] with physical compact rows outermost (plan order,
+ *     see row_of_token), heads next, the feature dimension contiguous.  Base pointers must be
+ *     16-byte aligned.  g and dg are fp32 [rows, H]; g is the log-decay (<= 0) itself.
+ */
+#ifndef HARTS_LA_H_
+#define HARTS_LA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HARTS_OK 0
+#define HARTS_EINVAL (-1)        /* bad argument: null/misaligned pointer, malformed tree, bad size */
+#define HARTS_ENOMEM (-2)        /* host allocation failed */
+#define HARTS_EUNSUPPORTED (-3)  /* no kernel for this (dtype, dk, dv, chunk) */
+#define HARTS_ETIMEOUT (-4)      /* a bounded device-side wait ran out (from harts_la_check) */
+#define HARTS_EINTERNAL (-5)
+#define HARTS_ECUDA (-6)         /* a CUDA runtime/driver call failed */
+
+#define HARTS_FP32 0
+#define HARTS_BF16 1
+
+/* flags */
+#define HARTS_FLAG_FMA_KERNELS 1u /* use the fp32-FMA (non tensor-core) kernels also for bf16 inputs */
+
+typedef struct harts_la_plan harts_la_plan_t; /* opaque, host memory, library-owned */
+
+/*
+ * Host view of a plan.  All pointers are const HOST arrays owned by the plan.
+ * Sequences are numbered globally in execution order: round-major, inside a round by the
+ * canonical index of their first own token (canonical = tree, node, offset order of the input).
+ * Physical rows follow the same order, the own rows of a sequence are contiguous, no padding rows.
+ */
+typedef struct harts_la_plan_view {
+    int32_t chunk;            /* B of Section 2.2 */
+    int32_t n_rounds;         /* minimum number of sequential packed calls (T_pre(root), max over trees) */
+    int32_t n_rows;           /* C: compact token rows */
+    int32_t n_replay;         /* R of Eq. 15 */
+    int32_t n_seq;
+    int32_t n_slots;          /* requested chunk-boundary states */
+    int32_t n_chunks;         /* sum over sequences of ceil((replay + own) / chunk) */
+    int32_t n_rg_rows;        /* compact rows that are replayed by at least one sequence */
+    const int32_t* row_of_token;   /* [n_rows]   canonical token index -> physical row */
+    const int32_t* round_seq_ptr;  /* [n_rounds+1] sequences of round r are [ptr[r], ptr[r+1]) */
+    const int32_t* seq_tree;       /* [n_seq] */
+    const int32_t* seq_own_begin;  /* [n_seq+1] first physical row of the own rows (cu_seqlens; last = n_rows) */
+    const int32_t* seq_own_len;    /* [n_seq] */
+    const int32_t* seq_start_pos;  /* [n_seq] absolute position of the start anchor (multiple of chunk) */
+    const int32_t* seq_init_slot;  /* [n_seq] slot holding the initial state, -1 = zero state */
+    const int32_t* seq_replay_ptr; /* [n_seq+1] CSR into replay_row */
+    const int32_t* replay_row;     /* [n_replay] physical rows replayed before the own rows, path order */
+    const int32_t* seq_req_ptr;    /* [n_seq+1] slots [ptr[i], ptr[i+1]) are produced by sequence i */
+    const int32_t* slot_chunk;     /* [n_slots] chunk index (>= 1) whose start state goes to the slot */
+    const int32_t* seq_chunk_ptr;  /* [n_seq+1] CSR of chunk counts (addresses the chunk-state workspace) */
+    const int32_t* slot_cons_ptr;  /* [n_slots+1] CSR: sequences whose initial state is that slot */
+    const int32_t* slot_cons_seq;
+    const int32_t* rg_row;         /* [n_rg_rows] replayed physical rows, ascending */
+    const int32_t* rg_ptr;         /* [n_rg_rows+1] CSR into rg_entry */
+    const int32_t* rg_entry;       /* [n_replay] indices into replay_row whose gradients land on rg_row */
+} harts_la_plan_view_t;
+
+/*
+ * Device-side index tables for one problem (all DEVICE pointers, int32, same meaning as in the
+ * view).  harts_la_plan_tables() fills it from an uploaded plan; a caller that wants to drive the
+ * per-call contract of Eq. 16 without the planner fills it by hand.
+ */
+typedef struct harts_la_tables {
+    int32_t chunk, n_rows, n_replay, n_seq, n_slots, n_chunks, n_rg_rows;
+    const int32_t* seq_own_begin;
+    const int32_t* seq_init_slot;
+    const int32_t* seq_replay_ptr;
+    const int32_t* replay_row;
+    const int32_t* seq_req_ptr;
+    const int32_t* slot_chunk;
+    const int32_t* seq_chunk_ptr;
+    const int32_t* slot_cons_ptr;
+    const int32_t* slot_cons_seq;
+    const int32_t* rg_row;
+    const int32_t* rg_ptr;
+    const int32_t* rg_entry;
+} harts_la_tables_t;
+
+const char* harts_la_strerror(int32_t code);
+
+/*
+ * Minimum-call planning (Section 3.3, Algorithm 1, Eqs. 11-15) plus the compact physical
+ * ordering of Section 4.2.  O(nodes + tokens) time.
+ *   tree_node_ptr [n_trees+1] host: CSR into the node arrays
+ *   node_parent   [n_nodes]   host: tree-local parent index (< own index), -1 for a root (node 0 of a tree)
+ *   node_fork_off [n_nodes]   host: offset inside the parent at which the node forks, 1..len(parent); 0 for roots
+ *   node_len      [n_nodes]   host: tokens in the node, >= 1
+ *   chunk: B.  *out is created by the library; free it with harts_la_plan_free().
+ * Errors: HARTS_EINVAL for a malformed forest (nothing is created), HARTS_ENOMEM.
+ */
+int32_t harts_la_plan(int32_t n_trees, const int32_t* tree_node_ptr, const int32_t* node_parent,
+                      const int32_t* node_fork_off, const int32_t* node_len, int32_t chunk,
+                      harts_la_plan_t** out);
+void harts_la_plan_free(harts_la_plan_t* plan);
+int32_t harts_la_plan_view(const harts_la_plan_t* plan, harts_la_plan_view_t* out);
+
+/* Size of the flat index blob, upload of it (one cudaMemcpyAsync on `stream`; dev_blob is a
+ * caller-owned DEVICE buffer of that size, 16-byte aligned), and the table of device pointers
+ * into an uploaded blob (pure pointer arithmetic, no CUDA call). */
+int32_t harts_la_plan_device_bytes(const harts_la_plan_t* plan, size_t* bytes);
+int32_t harts_la_plan_upload(const harts_la_plan_t* plan, void* dev_blob, void* stream);
+int32_t harts_la_plan_tables(const harts_la_plan_t* plan, const void* dev_blob, harts_la_tables_t* out);
+
+/*
+ * Workspace sizes (Section 3.4 "Full-layer activation recomputation": the forward keeps only
+ * chunk-boundary states, the backward recomputes everything inside a chunk from them).
+ *   chunk_state_bytes: [n_chunks, H, dk, dv] start-of-chunk states in the run dtype, written by the
+ *                      forward, read by the backward.
+ *   scratch_bytes:     backward scratch: per-sequence initial-state gradients [n_seq, H, dk, dv] fp32
+ *                      and replay-row gradients [n_replay, H, dk + dv + 1] fp32.
+ */
+int32_t harts_la_workspace_bytes(const harts_la_tables_t* tables, int32_t H, int32_t dk, int32_t dv,
+                                 int32_t dtype, uint32_t flags, size_t* chunk_state_bytes,
+                                 size_t* scratch_bytes);
+
+/*
+ * One packed call of Eq. 16 over sequences [seq_lo, seq_hi) (one round).  All tensors DEVICE.
+ *   q,k [n_rows,H,dk], v [n_rows,H,dv] in `dtype`; g [n_rows,H] fp32.  Never modified.
+ *   o   [n_rows,H,dv]: the own rows of the issued sequences are written exactly once; replay rows
+ *       produce no output (Section 3.4 "Round-wise execution").
+ *   slots [n_slots,H,dk,dv] fp32: read as initial states (seq_init_slot), written for the requested
+ *       boundaries of the issued sequences (no second state scan).  A slot read by this call must have
+ *       been written by an earlier call on the same stream.
+ *   chunk_states: workspace above (may be NULL: then no backward is possible).
+ * Errors: HARTS_EINVAL (null/misaligned pointers, bad range), HARTS_EUNSUPPORTED, HARTS_ECUDA.
+ */
+int32_t harts_la_fwd_seqs(const harts_la_tables_t* tables, int32_t seq_lo, int32_t seq_hi, const void* q,
+                          const void* k, const void* v, const float* g, void* o, float* slots,
+                          void* chunk_states, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                          uint32_t flags, int32_t* dev_status, void* stream);
+
+/*
+ * Backward of the same call.  Calls must be issued in the reverse order of the forward calls, on
+ * one stream: a sequence reads the initial-state gradients of the consumers of its slots
+ * (Section 3.4: several consumers of one boundary are summed) from `scratch`, where those
+ * consumers' calls left them.
+ *   dO [n_rows,H,dv]; dq,dk_ [n_rows,H,dk], dv_ [n_rows,H,dv] in `dtype`; dg [n_rows,H] fp32: own rows
+ *   of the issued sequences are overwritten.  Gradients of replayed rows go to `scratch` and are
+ *   folded into their ancestor rows by harts_la_bwd_finish().
+ */
+int32_t harts_la_bwd_seqs(const harts_la_tables_t* tables, int32_t seq_lo, int32_t seq_hi, const void* q,
+                          const void* k, const void* v, const float* g, const void* dO, void* dq, void* dk_,
+                          void* dv_, float* dg, const void* chunk_states, void* scratch, int32_t H,
+                          int32_t dk, int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status,
+                          void* stream);
+
+/* Adds the replay-row gradients (Section 4.2: the gather's backward sums every consumer into the
+ * unique producer row) into dk_, dv_, dg.  Call once, after the backward of the first round. */
+int32_t harts_la_bwd_finish(const harts_la_tables_t* tables, void* dk_, void* dv_, float* dg,
+                            const void* scratch, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                            void* stream);
+
+/*
+ * Plan-driven wrappers: round r in 1..n_rounds issues that round's packed call; round 0 issues all
+ * rounds in order (forward: 1..K; backward: K..1 followed by harts_la_bwd_finish).  With explicit
+ * rounds the backward of round 1 also runs harts_la_bwd_finish.  dev_blob is the uploaded blob.
+ */
+int32_t harts_la_fwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t round, const void* q,
+                     const void* k, const void* v, const float* g, void* o, float* slots, void* chunk_states,
+                     int32_t H, int32_t dk, int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status,
+                     void* stream);
+int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t round, const void* q,
+                     const void* k, const void* v, const float* g, const void* dO, void* dq, void* dk_,
+                     void* dv_, float* dg, const void* chunk_states, void* scratch, int32_t H, int32_t dk,
+                     int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream);
+
+/* Synchronises `stream`, reads the device status word and returns HARTS_OK, HARTS_ETIMEOUT or
+ * HARTS_ECUDA.  dev_status must be zeroed by the caller before the first launch. */
+int32_t harts_la_check(const int32_t* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HARTS_LA_H_ */

@@ -1,0 +1,12 @@
+"""Tree-packed chunkwise linear attention for B200 (sm_100a).
+
+Thin Python binding over the C-ABI library ``libharts_la.so`` (declared in
+``include/harts_la.h``).  Every step of the path runs in the library's CUDA kernels or its
+host planner; PyTorch only owns device memory and streams.  There is no CPU fallback: if the
+library cannot be loaded the import of :mod:`paper_2608_28158_b200.binding` fails.
+"""
+from .binding import (  # noqa: F401
+    HARTS_BF16, HARTS_FP32, HARTS_FLAG_FMA_KERNELS, HartsError, Plan, Workspace, harts_la_bwd, harts_la_bwd_finish,
+    harts_la_bwd_seqs, harts_la_check, harts_la_fwd, harts_la_fwd_seqs, harts_la_plan, harts_la_strerror,
+    harts_la_workspace_bytes, lib, run_fwd_bwd, run_fwd_bwd_host, expand_trajectories,
+)

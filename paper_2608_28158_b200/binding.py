@@ -1,0 +1,265 @@
+"""ctypes binding with the C ABI's names.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+HARTS_OK = 0
+HARTS_FP32, HARTS_BF16 = 0, 1
+HARTS_FLAG_FMA_KERNELS = 1
+_DTYPE_CODE = {torch.float32: HARTS_FP32, torch.bfloat16: HARTS_BF16}
+
+_I32P = C.POINTER(C.c_int32)
+
+
+class HartsError(RuntimeError):
+    def __init__(self, code, where):
+        super().__init__(f"{where}: {harts_la_strerror(code)} ({code})")
+        self.code = code
+
+
+class _View(C.Structure):
+    _counts = ("chunk", "n_rounds", "n_rows", "n_replay", "n_seq", "n_slots", "n_chunks", "n_rg_rows")
+    _arrays = ("row_of_token", "round_seq_ptr", "seq_tree", "seq_own_begin", "seq_own_len", "seq_start_pos",
+               "seq_init_slot", "seq_replay_ptr", "replay_row", "seq_req_ptr", "slot_chunk", "seq_chunk_ptr",
+               "slot_cons_ptr", "slot_cons_seq", "rg_row", "rg_ptr", "rg_entry")
+    _fields_ = [(n, C.c_int32) for n in _counts] + [(n, _I32P) for n in _arrays]
+
+
+class Tables(C.Structure):
+    _counts = ("chunk", "n_rows", "n_replay", "n_seq", "n_slots", "n_chunks", "n_rg_rows")
+    _arrays = ("seq_own_begin", "seq_init_slot", "seq_replay_ptr", "replay_row", "seq_req_ptr", "slot_chunk",
+               "seq_chunk_ptr", "slot_cons_ptr", "slot_cons_seq", "rg_row", "rg_ptr", "rg_entry")
+    _fields_ = [(n, C.c_int32) for n in _counts] + [(n, C.c_void_p) for n in _arrays]
+
+
+def _load():
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = C.CDLL(path)
+    vp, i32, u32, sz = C.c_void_p, C.c_int32, C.c_uint32, C.c_size_t
+    lib.harts_la_strerror.argtypes = [i32]
+    lib.harts_la_strerror.restype = C.c_char_p
+    lib.harts_la_plan.argtypes = [i32, _I32P, _I32P, _I32P, _I32P, i32, C.POINTER(vp)]
+    lib.harts_la_plan_free.argtypes = [vp]
+    lib.harts_la_plan_free.restype = None
+    lib.harts_la_plan_view.argtypes = [vp, C.POINTER(_View)]
+    lib.harts_la_plan_device_bytes.argtypes = [vp, C.POINTER(sz)]
+    lib.harts_la_plan_upload.argtypes = [vp, vp, vp]
+    lib.harts_la_plan_tables.argtypes = [vp, vp, C.POINTER(Tables)]
+    lib.harts_la_workspace_bytes.argtypes = [C.POINTER(Tables), i32, i32, i32, i32, u32, C.POINTER(sz), C.POINTER(sz)]
+    lib.harts_la_fwd_seqs.argtypes = [C.POINTER(Tables), i32, i32] + [vp] * 7 + [i32] * 4 + [u32, vp, vp]
+    lib.harts_la_bwd_seqs.argtypes = [C.POINTER(Tables), i32, i32] + [vp] * 11 + [i32] * 4 + [u32, vp, vp]
+    lib.harts_la_bwd_finish.argtypes = [C.POINTER(Tables)] + [vp] * 4 + [i32] * 4 + [vp]
+    lib.harts_la_fwd.argtypes = [vp, vp, i32] + [vp] * 7 + [i32] * 4 + [u32, vp, vp]
+    lib.harts_la_bwd.argtypes = [vp, vp, i32] + [vp] * 11 + [i32] * 4 + [u32, vp, vp]
+    lib.harts_la_check.argtypes = [vp, vp]
+    for name in ("harts_la_plan", "harts_la_plan_view", "harts_la_plan_device_bytes", "harts_la_plan_upload",
+                 "harts_la_plan_tables", "harts_la_workspace_bytes", "harts_la_fwd_seqs", "harts_la_bwd_seqs",
+                 "harts_la_bwd_finish", "harts_la_fwd", "harts_la_bwd", "harts_la_check"):
+        getattr(lib, name).restype = i32
+    return lib
+
+
+lib = _load()
+
+
+def harts_la_strerror(code: int) -> str:
+    return lib.harts_la_strerror(code).decode()
+
+
+def _check(code, where):
+    if code != HARTS_OK:
+        raise HartsError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+class Plan:
+    """Host plan (owned by the library) plus, after ``upload``, its device index blob."""
+
+    def __init__(self, handle):
+        self._h = handle
+        v = _View()
+        _check(lib.harts_la_plan_view(handle, C.byref(v)), "harts_la_plan_view")
+        for n in _View._counts:
+            setattr(self, n, int(getattr(v, n)))
+        sizes = dict(row_of_token=self.n_rows, round_seq_ptr=self.n_rounds + 1, seq_tree=self.n_seq,
+                     seq_own_begin=self.n_seq + 1, seq_own_len=self.n_seq, seq_start_pos=self.n_seq,
+                     seq_init_slot=self.n_seq, seq_replay_ptr=self.n_seq + 1, replay_row=self.n_replay,
+                     seq_req_ptr=self.n_seq + 1, slot_chunk=self.n_slots, seq_chunk_ptr=self.n_seq + 1,
+                     slot_cons_ptr=self.n_slots + 1, slot_cons_seq=None, rg_row=self.n_rg_rows,
+                     rg_ptr=self.n_rg_rows + 1 if self.n_rg_rows else 1, rg_entry=self.n_replay)
+        for n in _View._arrays:
+            size = sizes[n]
+            if n == "slot_cons_seq":
+                size = int(self.slot_cons_ptr[-1])
+            arr = np.ctypeslib.as_array(getattr(v, n), shape=(size,)).copy() if size else np.zeros(0, np.int32)
+            setattr(self, n, arr)
+        self.C, self.R = self.n_rows, self.n_replay
+        self.blob = None
+        self.tables = None
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            lib.harts_la_plan_free(h)
+
+    def upload(self, device="cuda", stream=None):
+        n = C.c_size_t(0)
+        _check(lib.harts_la_plan_device_bytes(self._h, C.byref(n)), "harts_la_plan_device_bytes")
+        self.blob = torch.empty(max(int(n.value), 16), dtype=torch.uint8, device=device)
+        _check(lib.harts_la_plan_upload(self._h, _ptr(self.blob), _stream(stream)), "harts_la_plan_upload")
+        self.tables = Tables()
+        _check(lib.harts_la_plan_tables(self._h, _ptr(self.blob), C.byref(self.tables)), "harts_la_plan_tables")
+        return self
+
+
+def harts_la_plan(tree_node_ptr, node_parent, node_fork_off, node_len, chunk=64) -> Plan:
+    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in (tree_node_ptr, node_parent, node_fork_off, node_len)]
+    handle = C.c_void_p()
+    code = lib.harts_la_plan(len(arrs[0]) - 1, *(a.ctypes.data_as(_I32P) for a in arrs), int(chunk), C.byref(handle))
+    _check(code, "harts_la_plan")
+    return Plan(handle)
+
+
+def harts_la_workspace_bytes(tables, H, dk, dv, dtype, flags=0):
+    a, b = C.c_size_t(0), C.c_size_t(0)
+    _check(lib.harts_la_workspace_bytes(C.byref(tables), H, dk, dv, dtype, flags, C.byref(a), C.byref(b)),
+           "harts_la_workspace_bytes")
+    return int(a.value), int(b.value)
+
+
+def _dims(q, v):
+    return q.shape[1], q.shape[2], v.shape[2], _DTYPE_CODE[q.dtype]
+
+
+def harts_la_fwd_seqs(tables, seq_lo, seq_hi, q, k, v, g, o, slots, chunk_states, flags=0, dev_status=None,
+                      stream=None):
+    H, dk, dv, dt = _dims(q, v)
+    _check(lib.harts_la_fwd_seqs(C.byref(tables), seq_lo, seq_hi, _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(o),
+                                 _ptr(slots), _ptr(chunk_states), H, dk, dv, dt, flags, _ptr(dev_status),
+                                 _stream(stream)), "harts_la_fwd_seqs")
+
+
+def harts_la_bwd_seqs(tables, seq_lo, seq_hi, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, scratch, flags=0,
+                      dev_status=None, stream=None):
+    H, dk, dv, dt = _dims(q, v)
+    _check(lib.harts_la_bwd_seqs(C.byref(tables), seq_lo, seq_hi, _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(dO),
+                                 _ptr(dq), _ptr(dk_), _ptr(dv_), _ptr(dg), _ptr(chunk_states), _ptr(scratch), H, dk,
+                                 dv, dt, flags, _ptr(dev_status), _stream(stream)), "harts_la_bwd_seqs")
+
+
+def harts_la_bwd_finish(tables, dk_, dv_, dg, scratch, stream=None):
+    H, dk, dv = dk_.shape[1], dk_.shape[2], dv_.shape[2]
+    _check(lib.harts_la_bwd_finish(C.byref(tables), _ptr(dk_), _ptr(dv_), _ptr(dg), _ptr(scratch), H, dk, dv,
+                                   _DTYPE_CODE[dk_.dtype], _stream(stream)), "harts_la_bwd_finish")
+
+
+def harts_la_fwd(plan, round, q, k, v, g, o, slots, chunk_states, flags=0, dev_status=None, stream=None):
+    H, dk, dv, dt = _dims(q, v)
+    _check(lib.harts_la_fwd(plan._h, _ptr(plan.blob), round, _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(o),
+                            _ptr(slots), _ptr(chunk_states), H, dk, dv, dt, flags, _ptr(dev_status),
+                            _stream(stream)), "harts_la_fwd")
+
+
+def harts_la_bwd(plan, round, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, scratch, flags=0, dev_status=None,
+                 stream=None):
+    H, dk, dv, dt = _dims(q, v)
+    _check(lib.harts_la_bwd(plan._h, _ptr(plan.blob), round, _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(dO), _ptr(dq),
+                            _ptr(dk_), _ptr(dv_), _ptr(dg), _ptr(chunk_states), _ptr(scratch), H, dk, dv, dt, flags,
+                            _ptr(dev_status), _stream(stream)), "harts_la_bwd")
+
+
+def harts_la_check(dev_status, stream=None):
+    _check(lib.harts_la_check(_ptr(dev_status), _stream(stream)), "harts_la_check")
+
+
+class Workspace:
+    """Caller-owned device buffers for one plan: slots, chunk states, backward scratch, status word."""
+
+    def __init__(self, plan: Plan, H, dk, dv, dtype, flags=0, device="cuda"):
+        if plan.tables is None:
+            plan.upload(device)
+        cs_bytes, sc_bytes = harts_la_workspace_bytes(plan.tables, H, dk, dv, _DTYPE_CODE[dtype], flags)
+        self.slots = torch.empty(max(plan.n_slots, 1) * H * dk * dv, dtype=torch.float32, device=device)
+        self.chunk_states = torch.empty(cs_bytes, dtype=torch.uint8, device=device)
+        self.scratch = torch.empty(sc_bytes, dtype=torch.uint8, device=device)
+        self.dev_status = torch.zeros(4, dtype=torch.int32, device=device)
+        self.flags = flags
+
+
+def run_fwd_bwd(plan: Plan, ws: Workspace, q, k, v, g, dO, out=None, backward=True, stream=None):
+    """All rounds forward (and backward) on device tensors in physical row order."""
+    if out is None:
+        out = {"o": torch.empty_like(v)}
+        if backward:
+            out.update(dq=torch.empty_like(q), dk=torch.empty_like(k), dv=torch.empty_like(v),
+                       dg=torch.empty_like(g))
+    harts_la_fwd(plan, 0, q, k, v, g, out["o"], ws.slots, ws.chunk_states, ws.flags, ws.dev_status, stream)
+    if backward:
+        harts_la_bwd(plan, 0, q, k, v, g, dO, out["dq"], out["dk"], out["dv"], out["dg"], ws.chunk_states,
+                     ws.scratch, ws.flags, ws.dev_status, stream)
+    return out
+
+
+def run_fwd_bwd_host(plan: Plan, ws: Workspace, host_in: dict, dev_in: dict, dev_out: dict, host_out: dict):
+    """End-to-end step on HOST buffers: pinned host inputs -> device, all rounds forward and backward,
+    outputs -> pinned host buffers.  Buffers are preallocated by the caller; returns after a sync."""
+    for n in ("q", "k", "v", "g", "dO"):
+        dev_in[n].copy_(host_in[n], non_blocking=True)
+    run_fwd_bwd(plan, ws, dev_in["q"], dev_in["k"], dev_in["v"], dev_in["g"], dev_in["dO"], out=dev_out)
+    for n in ("o", "dq", "dk", "dv", "dg"):
+        host_out[n].copy_(dev_out[n], non_blocking=True)
+    torch.cuda.current_stream().synchronize()
+    return host_out
+
+
+def expand_trajectories(tree_node_ptr, node_parent, node_fork_off, node_len):
+    """Trajectory-wise view of a forest (the conventional baseline of Section 5): every root-to-leaf
+    path becomes its own single-node tree.  Returns (forest arrays of the expanded problem,
+    canonical compact token index of every expanded token)."""
+    tree_node_ptr, node_parent, node_fork_off, node_len = (np.asarray(a) for a in
+                                                            (tree_node_ptr, node_parent, node_fork_off, node_len))
+    base = np.zeros(len(node_len) + 1, dtype=np.int64)
+    np.cumsum(node_len, out=base[1:])
+    lens, src = [], []
+    for t in range(len(tree_node_ptr) - 1):
+        lo, hi = int(tree_node_ptr[t]), int(tree_node_ptr[t + 1])
+        has_tail_child = np.zeros(hi - lo, dtype=bool)
+        for i in range(lo + 1, hi):
+            p = lo + int(node_parent[i])
+            if node_fork_off[i] == node_len[p]:
+                has_tail_child[p - lo] = True
+        for leaf in range(lo, hi):
+            if has_tail_child[leaf - lo]:
+                continue
+            parts, node, upto = [], leaf, int(node_len[leaf])
+            while True:
+                parts.append(np.arange(base[node], base[node] + upto, dtype=np.int64))
+                if node_parent[node] < 0:
+                    break
+                upto = int(node_fork_off[node])
+                node = lo + int(node_parent[node])
+            parts.reverse()
+            rows = np.concatenate(parts)
+            src.append(rows)
+            lens.append(len(rows))
+    n = len(lens)
+    forest = (np.arange(n + 1, dtype=np.int32), np.full(n, -1, np.int32), np.zeros(n, np.int32),
+              np.asarray(lens, np.int32))
+    return forest, np.concatenate(src)

@@ -1,0 +1,144 @@
+// C ABI: argument checks, kernel selection and launches.  No device memory is allocated here.
+#include "kernels.h"
+#include "plan.h"
+
+namespace {
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
+
+int32_t check_common(const harts_la_tables_t* tb, int32_t seq_lo, int32_t seq_hi, int32_t H, int32_t dk, int32_t dv,
+                     int32_t dtype) {
+    if (!tb) return HARTS_EINVAL;
+    if (seq_lo < 0 || seq_hi < seq_lo || seq_hi > tb->n_seq) return HARTS_EINVAL;
+    if (H < 1 || dk < 1 || dv < 1) return HARTS_EINVAL;
+    if (dtype != HARTS_FP32 && dtype != HARTS_BF16) return HARTS_EUNSUPPORTED;
+    if (tb->chunk != 64) return HARTS_EUNSUPPORTED;
+    if (!harts::fma_supported(dtype, dk, dv)) return HARTS_EUNSUPPORTED;
+    if (!tb->seq_own_begin || !tb->seq_init_slot || !tb->seq_replay_ptr || !tb->replay_row || !tb->seq_req_ptr ||
+        !tb->slot_chunk || !tb->seq_chunk_ptr || !tb->slot_cons_ptr || !tb->slot_cons_seq || !tb->rg_row ||
+        !tb->rg_ptr || !tb->rg_entry)
+        return HARTS_EINVAL;
+    return HARTS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* harts_la_strerror(int32_t code) {
+    switch (code) {
+        case HARTS_OK: return "ok";
+        case HARTS_EINVAL: return "invalid argument";
+        case HARTS_ENOMEM: return "out of host memory";
+        case HARTS_EUNSUPPORTED: return "unsupported dtype / head dimension / chunk size";
+        case HARTS_ETIMEOUT: return "a bounded device-side wait ran out";
+        case HARTS_EINTERNAL: return "internal error";
+        case HARTS_ECUDA: return "CUDA call failed";
+        default: return "unknown status";
+    }
+}
+
+int32_t harts_la_plan_upload(const harts_la_plan_t* plan, void* dev_blob, void* stream) {
+    const harts::Plan* p = harts_la_plan_internal(plan);
+    if (!p || !dev_blob || misaligned(dev_blob)) return HARTS_EINVAL;
+    cudaError_t e = cudaMemcpyAsync(dev_blob, p->blob.data(), p->blob.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
+                                    static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+int32_t harts_la_workspace_bytes(const harts_la_tables_t* tb, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                                 uint32_t /*flags*/, size_t* chunk_state_bytes, size_t* scratch_bytes) {
+    if (!tb || H < 1 || dk < 1 || dv < 1) return HARTS_EINVAL;
+    if (dtype != HARTS_FP32 && dtype != HARTS_BF16) return HARTS_EUNSUPPORTED;
+    size_t elem = dtype == HARTS_FP32 ? 4 : 2;
+    if (chunk_state_bytes) {
+        size_t b = (size_t)tb->n_chunks * H * dk * dv * elem;
+        *chunk_state_bytes = b < 256 ? 256 : b;
+    }
+    if (scratch_bytes) *scratch_bytes = harts::scratch_layout(*tb, H, dk, dv).total;
+    return HARTS_OK;
+}
+
+int32_t harts_la_fwd_seqs(const harts_la_tables_t* tb, int32_t seq_lo, int32_t seq_hi, const void* q, const void* k,
+                          const void* v, const float* g, void* o, float* slots, void* chunk_states, int32_t H,
+                          int32_t dk, int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream) {
+    int32_t rc = check_common(tb, seq_lo, seq_hi, H, dk, dv, dtype);
+    if (rc != HARTS_OK) return rc;
+    if (!q || !k || !v || !g || !o || (tb->n_slots > 0 && !slots)) return HARTS_EINVAL;
+    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(g) || misaligned(o) || misaligned(slots) ||
+        misaligned(chunk_states))
+        return HARTS_EINVAL;
+    harts::FwdArgs a{*tb, seq_lo, seq_hi, q, k, v, g, o, slots, chunk_states, H, dk, dv, dtype, flags, dev_status,
+                     static_cast<cudaStream_t>(stream)};
+    return harts::fma_fwd(a);
+}
+
+int32_t harts_la_bwd_seqs(const harts_la_tables_t* tb, int32_t seq_lo, int32_t seq_hi, const void* q, const void* k,
+                          const void* v, const float* g, const void* dO, void* dq, void* dk_, void* dv_, float* dg,
+                          const void* chunk_states, void* scratch, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                          uint32_t flags, int32_t* dev_status, void* stream) {
+    int32_t rc = check_common(tb, seq_lo, seq_hi, H, dk, dv, dtype);
+    if (rc != HARTS_OK) return rc;
+    if (!q || !k || !v || !g || !dO || !dq || !dk_ || !dv_ || !dg || !chunk_states || !scratch) return HARTS_EINVAL;
+    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(g) || misaligned(dO) || misaligned(dq) ||
+        misaligned(dk_) || misaligned(dv_) || misaligned(dg) || misaligned(chunk_states) || misaligned(scratch))
+        return HARTS_EINVAL;
+    harts::BwdArgs a{*tb, seq_lo, seq_hi, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, scratch, H, dk, dv, dtype,
+                     flags, dev_status, static_cast<cudaStream_t>(stream)};
+    return harts::fma_bwd(a);
+}
+
+int32_t harts_la_bwd_finish(const harts_la_tables_t* tb, void* dk_, void* dv_, float* dg, const void* scratch,
+                            int32_t H, int32_t dk, int32_t dv, int32_t dtype, void* stream) {
+    int32_t rc = check_common(tb, 0, 0, H, dk, dv, dtype);
+    if (rc != HARTS_OK) return rc;
+    if (!dk_ || !dv_ || !dg || !scratch) return HARTS_EINVAL;
+    return harts::replay_reduce(*tb, dk_, dv_, dg, scratch, H, dk, dv, dtype, static_cast<cudaStream_t>(stream));
+}
+
+int32_t harts_la_fwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t round, const void* q, const void* k,
+                     const void* v, const float* g, void* o, float* slots, void* chunk_states, int32_t H, int32_t dk,
+                     int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream) {
+    const harts::Plan* p = harts_la_plan_internal(plan);
+    if (!p || round < 0 || round > p->n_rounds) return HARTS_EINVAL;
+    harts_la_tables_t tb;
+    int32_t rc = harts_la_plan_tables(plan, dev_blob, &tb);
+    if (rc != HARTS_OK) return rc;
+    int32_t r0 = round == 0 ? 1 : round, r1 = round == 0 ? p->n_rounds : round;
+    for (int32_t r = r0; r <= r1; r++) {
+        rc = harts_la_fwd_seqs(&tb, p->round_seq_ptr[r - 1], p->round_seq_ptr[r], q, k, v, g, o, slots, chunk_states,
+                               H, dk, dv, dtype, flags, dev_status, stream);
+        if (rc != HARTS_OK) return rc;
+    }
+    return HARTS_OK;
+}
+
+int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t round, const void* q, const void* k,
+                     const void* v, const float* g, const void* dO, void* dq, void* dk_, void* dv_, float* dg,
+                     const void* chunk_states, void* scratch, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                     uint32_t flags, int32_t* dev_status, void* stream) {
+    const harts::Plan* p = harts_la_plan_internal(plan);
+    if (!p || round < 0 || round > p->n_rounds) return HARTS_EINVAL;
+    harts_la_tables_t tb;
+    int32_t rc = harts_la_plan_tables(plan, dev_blob, &tb);
+    if (rc != HARTS_OK) return rc;
+    int32_t r1 = round == 0 ? p->n_rounds : round, r0 = round == 0 ? 1 : round;
+    for (int32_t r = r1; r >= r0; r--) {
+        rc = harts_la_bwd_seqs(&tb, p->round_seq_ptr[r - 1], p->round_seq_ptr[r], q, k, v, g, dO, dq, dk_, dv_, dg,
+                               chunk_states, scratch, H, dk, dv, dtype, flags, dev_status, stream);
+        if (rc != HARTS_OK) return rc;
+    }
+    if (r0 == 1) return harts_la_bwd_finish(&tb, dk_, dv_, dg, scratch, H, dk, dv, dtype, stream);
+    return HARTS_OK;
+}
+
+int32_t harts_la_check(const int32_t* dev_status, void* stream) {
+    if (!dev_status) return HARTS_EINVAL;
+    int32_t host = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&host, dev_status, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess) return HARTS_ECUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return HARTS_ECUDA;
+    return host == 0 ? HARTS_OK : HARTS_ETIMEOUT;
+}
+
+}  // extern "C"

@@ -1,0 +1,75 @@
+// Internal launch interface between the C ABI (api.cu) and the kernel files.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstddef>
+#include <cstdint>
+
+#include "../../include/harts_la.h"
+
+namespace harts {
+
+struct FwdArgs {
+    harts_la_tables_t tb;
+    int32_t seq_lo, seq_hi;
+    const void *q, *k, *v;
+    const float* g;
+    void* o;
+    float* slots;
+    void* chunk_states;
+    int32_t H, dk, dv, dtype;
+    uint32_t flags;
+    int32_t* dev_status;
+    cudaStream_t stream;
+};
+
+struct BwdArgs {
+    harts_la_tables_t tb;
+    int32_t seq_lo, seq_hi;
+    const void *q, *k, *v;
+    const float* g;
+    const void* dO;
+    void *dq, *dk_, *dv_;
+    float* dg;
+    const void* chunk_states;
+    void* scratch;
+    int32_t H, dk, dv, dtype;
+    uint32_t flags;
+    int32_t* dev_status;
+    cudaStream_t stream;
+};
+
+// Byte offsets inside the backward scratch buffer (each region 256-byte aligned).
+struct ScratchLayout {
+    size_t ds0;    // [n_seq, H, dk, dv] fp32: gradient w.r.t. each sequence's initial state
+    size_t rk;     // [n_replay, H, dk] fp32: dk of replayed rows
+    size_t rv;     // [n_replay, H, dv] fp32
+    size_t rg;     // [n_replay, H] fp32
+    size_t total;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline ScratchLayout scratch_layout(const harts_la_tables_t& tb, int32_t H, int32_t dk, int32_t dv) {
+    ScratchLayout s;
+    size_t off = 0;
+    s.ds0 = off;
+    off = align_up(off + (size_t)tb.n_seq * H * dk * dv * sizeof(float), 256);
+    s.rk = off;
+    off = align_up(off + (size_t)tb.n_replay * H * dk * sizeof(float), 256);
+    s.rv = off;
+    off = align_up(off + (size_t)tb.n_replay * H * dv * sizeof(float), 256);
+    s.rg = off;
+    off = align_up(off + (size_t)tb.n_replay * H * sizeof(float), 256);
+    s.total = off < 256 ? 256 : off;
+    return s;
+}
+
+int32_t fma_supported(int32_t dtype, int32_t dk, int32_t dv);
+int32_t fma_fwd(const FwdArgs& a);
+int32_t fma_bwd(const BwdArgs& a);
+int32_t replay_reduce(const harts_la_tables_t& tb, void* dk_, void* dv_, float* dg, const void* scratch, int32_t H,
+                      int32_t dk, int32_t dv, int32_t dtype, cudaStream_t stream);
+
+}  // namespace harts

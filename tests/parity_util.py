@@ -1,0 +1,67 @@
+"""Shared helpers for the GPU parity tests: run a forest through the C ABI and through the oracle."""
+import numpy as np
+import torch
+
+import paper_2608_28158_b200 as H
+from oracle import la_oracle as lo
+from workloads import CONFIGS, config_forest, make_inputs
+
+TORCH_DTYPE = {"fp32": torch.float32, "bf16": torch.bfloat16}
+
+
+def rel_err(x, ref):
+    x = np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    return float(np.linalg.norm(x - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+def plan_of(fo, chunk=64):
+    return H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, chunk)
+
+
+def to_physical(plan, canon: dict, device="cuda"):
+    """canonical-order tensors -> physical-row-order device tensors"""
+    rows = torch.as_tensor(plan.row_of_token.astype(np.int64), device=canon["q"].device)
+    out = {}
+    for n, x in canon.items():
+        y = torch.empty_like(x)
+        y[rows] = x
+        out[n] = y.to(device)
+    return out
+
+
+def run_gpu(fo, inp_canon, flags=0, backward=True, chunk=64):
+    """Returns (plan, outputs in CANONICAL order as device tensors)."""
+    plan = plan_of(fo, chunk).upload()
+    phys = to_physical(plan, inp_canon)
+    H_, dk, dv = phys["q"].shape[1], phys["q"].shape[2], phys["v"].shape[2]
+    ws = H.Workspace(plan, H_, dk, dv, phys["q"].dtype, flags)
+    out = H.run_fwd_bwd(plan, ws, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"], backward=backward)
+    H.harts_la_check(ws.dev_status)
+    rows = torch.as_tensor(plan.row_of_token.astype(np.int64), device="cuda")
+    return plan, {n: x[rows] for n, x in out.items()}
+
+
+def oracle_subset(fo, inp_canon, tree_ids, heads, backward=True):
+    """Oracle on the given trees and heads.  Returns (canonical token indices of the subset, results)."""
+    base = fo.token_base()
+    tok = np.concatenate([np.arange(base[fo.tree_node_ptr[t]], base[fo.tree_node_ptr[t + 1]]) for t in tree_ids])
+    sub = fo.subset(tree_ids)
+    ti = torch.as_tensor(tok, device=inp_canon["q"].device)
+    hi = torch.as_tensor(heads, device=inp_canon["q"].device)
+    pick = {n: x[ti][:, hi].cpu() for n, x in inp_canon.items()}
+    res = lo.forest_eval(sub, pick["q"], pick["k"], pick["v"], pick["g"], pick["dO"] if backward else None)
+    return tok, res
+
+
+def compare(out_canon, tok, heads, ref, names=("o", "dq", "dk", "dv", "dg")):
+    ti = torch.as_tensor(tok, device="cuda")
+    hi = torch.as_tensor(heads, device="cuda")
+    return {n: rel_err(out_canon[n][ti][:, hi].float().cpu().numpy(), ref[n]) for n in names}
+
+
+def config_case(name, device="cpu"):
+    cfg = CONFIGS[name]
+    fo = config_forest(name)
+    inp = make_inputs(fo.n_tokens, cfg["H"], cfg["dk"], cfg["dv"], cfg["dtype"], cfg["seed"], device=device)
+    return cfg, fo, inp

@@ -1,0 +1,128 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 trajectory-wise oracle, element
+by element on the same seeded inputs.  Tolerances (relative Frobenius error per tensor): bf16
+inputs with fp32 accumulation 5e-3 for outputs and 1e-2 for gradients; the fp32 configuration is
+held to 1e-4 (fp32 accumulation over 64-row chunks plus the fast exponential)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_28158_b200 as H
+from workloads import make_forest, make_inputs
+from parity_util import compare, config_case, oracle_subset, plan_of, rel_err, run_gpu, to_physical
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"fp32": dict(o=1e-4, dq=1e-4, dk=1e-4, dv=1e-4, dg=1e-4),
+       "bf16": dict(o=5e-3, dq=1e-2, dk=1e-2, dv=1e-2, dg=1e-2)}
+
+
+def check(errs, dtype):
+    for n, e in errs.items():
+        assert e <= TOL[dtype][n], (n, e, errs)
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg0b", "cfg1"])
+def test_small_configs_full_parity(name):
+    cfg, fo, inp = config_case(name)
+    plan, out = run_gpu(fo, inp)
+    tok, ref = oracle_subset(fo, inp, list(range(fo.n_trees)), list(range(cfg["H"])))
+    assert ref["copy_gap"] < 1e-9
+    errs = compare(out, tok, list(range(cfg["H"])), ref)
+    print(name, errs)
+    check(errs, cfg["dtype"])
+
+
+@pytest.mark.parametrize("name,trees", [("cfg2", [0, 5]), ("cfg3", [3]), ("cfg4", [0, 63])])
+def test_large_configs_sampled_parity(name, trees):
+    # full-size launch on the GPU; the oracle evaluates whole trees for three heads
+    cfg, fo, inp = config_case(name, device="cuda")
+    plan, out = run_gpu(fo, inp)
+    heads = [0, cfg["H"] // 2, cfg["H"] - 1]
+    tok, ref = oracle_subset(fo, inp, trees, heads)
+    errs = compare(out, tok, heads, ref)
+    print(name, "C", plan.C, "R", plan.R, "rounds", plan.n_rounds, "seqs", plan.n_seq, errs)
+    check(errs, cfg["dtype"])
+    for x in out.values():
+        assert torch.isfinite(x.float()).all()
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg0b", "cfg1"])
+def test_compact_equals_trajectory_wise_on_gpu(name):
+    # same kernels on the expanded forest (one zero-state sequence per leaf): outputs at m(s) agree.
+    cfg, fo, inp = config_case(name)
+    _, out = run_gpu(fo, inp, backward=False)
+    (ptr, par, off, ln), src = H.expand_trajectories(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len)
+    src_t = torch.as_tensor(src)
+    exp_inp = {n: x[src_t] for n, x in inp.items()}
+    exp_fo = make_forest([([-1], [0], [int(l)]) for l in ln])
+    _, exp_out = run_gpu(exp_fo, exp_inp, backward=False)
+    a = exp_out["o"].float().cpu().numpy()
+    b = out["o"][src_t.cuda()].float().cpu().numpy()
+    # the chunk grid of a replay-started branch coincides with the trajectory's own grid
+    assert rel_err(a, b) < (1e-6 if cfg["dtype"] == "fp32" else 2e-3)
+
+
+def edge_forests():
+    return {
+        "one_token": make_forest([([-1], [0], [1])]),
+        "exact_chunk": make_forest([([-1, 0, 0], [0, 64, 64], [64, 64, 1])]),
+        "two_chunks_and_tail": make_forest([([-1, 0, 0, 1], [0, 128, 100, 63], [129, 5, 200, 64])]),
+        "many_tiny": make_forest([([-1] + [0] * 40, [0] + [1 + (7 * i) % 90 for i in range(40)],
+                                   [90] + [1 + i % 5 for i in range(40)])] * 3),
+        "nested_in_chunk": make_forest([([-1, 0, 1, 2, 3, 0], [0, 10, 5, 3, 2, 10], [10, 7, 6, 4, 70, 130])]),
+    }
+
+
+@pytest.mark.parametrize("case", list(edge_forests()))
+@pytest.mark.parametrize("dtype,d", [("fp32", 64), ("bf16", 128)])
+def test_edge_cases(case, dtype, d):
+    fo = edge_forests()[case]
+    inp = make_inputs(fo.n_tokens, 2, d, d, dtype, 17)
+    plan, out = run_gpu(fo, inp)
+    tok, ref = oracle_subset(fo, inp, list(range(fo.n_trees)), [0, 1])
+    errs = compare(out, tok, [0, 1], ref)
+    print(case, dtype, errs)
+    check(errs, dtype)
+
+
+def test_rounds_issued_one_by_one_match_round_zero():
+    cfg, fo, inp = config_case("cfg0b")
+    plan = plan_of(fo).upload()
+    phys = to_physical(plan, inp)
+    ws = H.Workspace(plan, 1, 64, 64, torch.float32)
+    ref = H.run_fwd_bwd(plan, ws, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"])
+    ref = {n: x.clone() for n, x in ref.items()}
+    ws2 = H.Workspace(plan, 1, 64, 64, torch.float32)
+    o = torch.zeros_like(phys["v"])
+    dq, dk, dv, dg = (torch.zeros_like(phys[n]) for n in ("q", "k", "v", "g"))
+    for r in range(1, plan.n_rounds + 1):
+        H.harts_la_fwd(plan, r, phys["q"], phys["k"], phys["v"], phys["g"], o, ws2.slots, ws2.chunk_states)
+    for r in range(plan.n_rounds, 0, -1):
+        H.harts_la_bwd(plan, r, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"], dq, dk, dv, dg,
+                       ws2.chunk_states, ws2.scratch)
+    torch.cuda.synchronize()
+    for n, x in (("o", o), ("dq", dq), ("dk", dk), ("dv", dv), ("dg", dg)):
+        assert torch.equal(x, ref[n]), n
+
+
+def test_errors_are_reported_without_launching():
+    cfg, fo, inp = config_case("cfg0")
+    plan = plan_of(fo).upload()
+    phys = to_physical(plan, inp)
+    ws = H.Workspace(plan, 1, 64, 64, torch.float32)
+    o = torch.empty_like(phys["v"])
+    # misaligned pointer
+    bad = torch.empty(phys["q"].numel() + 1, dtype=torch.float32, device="cuda")[1:].view_as(phys["q"])
+    with pytest.raises(H.HartsError) as e:
+        H.harts_la_fwd(plan, 0, bad, phys["k"], phys["v"], phys["g"], o, ws.slots, ws.chunk_states)
+    assert e.value.code == -1
+    # unsupported head dimension
+    q96 = torch.zeros(plan.C, 1, 96, device="cuda")
+    with pytest.raises(H.HartsError) as e:
+        H.harts_la_fwd(plan, 0, q96, q96, q96, phys["g"], torch.empty_like(q96), ws.slots, ws.chunk_states)
+    assert e.value.code == -3
+    # round out of range
+    with pytest.raises(H.HartsError) as e:
+        H.harts_la_fwd(plan, 9, phys["q"], phys["k"], phys["v"], phys["g"], o, ws.slots, ws.chunk_states)
+    assert e.value.code == -1
+    torch.cuda.synchronize()
