@@ -1,0 +1,353 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-packed linear-attention hot path (forward + backward over all rounds).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl ours|reference]
+
+One step = one pass of the whole path over one batch: every forward round, every backward round and
+the replay-gradient fold, on synthetic trees and tensors of the named configuration.  Prints ONE
+JSON line.  ``value`` is compact tokens per second with inputs resident in HBM; ``e2e`` is the same
+metric through the host-buffer call (pinned host inputs copied in, results copied out, inside the
+timed region).  With N > 1 (torchrun) every rank runs its own copy of the workload (weak scaling,
+no collective on the data path); time is the maximum over ranks.
+
+``--impl reference`` times the fp64 CPU oracle (oracle/), as it stands, on the host cores, on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tree-packed linear-attn fwd+bwd compact tokens/s"
+UNIT = "compact tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+
+
+# --------------------------------------------------------------------------------------------------
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, val in zip(names, r[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------------
+def oracle_sample(name, seconds_hint=15.0):
+    """The fp64 oracle on a bounded sample of the workload: whole trees, a few heads."""
+    import torch
+    from oracle import la_oracle
+    from workloads import CONFIGS, config_forest, make_inputs
+
+    cfg = CONFIGS[name]
+    fo = config_forest(name)
+    heads = sorted({0, cfg["H"] // 2, cfg["H"] - 1})
+    # about 40k semantic token-heads per second on 8 cores: take trees until the budget is used
+    budget = 40000.0 * seconds_hint * max(1, (os.cpu_count() or 8)) / 8
+    base = fo.token_base()
+    trees, sem = [], 0
+    from workloads.trees import tree_counts
+    for t in range(fo.n_trees):
+        c, s, _ = tree_counts(*(a.tolist() for a in fo.tree(t)))
+        if trees and (sem + s) * len(heads) > budget:
+            break
+        trees.append(t)
+        sem += s
+    sub = fo.subset(trees)
+    inp = make_inputs(sub.n_tokens, len(heads), cfg["dk"], cfg["dv"], cfg["dtype"], cfg["seed"])
+    t0 = time.perf_counter()
+    res = la_oracle.forest_eval(sub, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"])
+    dt = time.perf_counter() - t0
+    # compact tokens/s at the configuration's head count: the sample covered len(heads) of H heads
+    value = sub.n_tokens * len(heads) / cfg["H"] / dt
+    return {"value": value, "unit": UNIT, "cores": res["threads"], "kind": "oracle",
+            "sample": f"{name}: trees {trees[0]}..{trees[-1]} ({sub.n_tokens} compact / {res['S']} trajectory-wise "
+                      f"tokens), {len(heads)} of {cfg['H']} heads, fwd+bwd, {dt:.1f} s",
+            "semantic_token_heads_per_s": res["S"] * len(heads) / dt, "seconds": dt}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times, secs, last = [], [], None
+    for i in range(args.warmup + args.steps):
+        last = oracle_sample(args.workload, seconds_hint=8.0)
+        if i >= args.warmup:
+            times.append(last["value"])
+            secs.append(last["seconds"])
+    value = statistics.mean(times)
+    from workloads import CONFIGS
+    cfg = CONFIGS[args.workload]
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(secs) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "H": cfg["H"], "dk": cfg["dk"], "dv": cfg["dv"], "chunk": 64},
+            "cpu_baseline": {"kind": last["kind"], "cores": last["cores"], "sample": last["sample"], "value": value,
+                             "unit": UNIT},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2608_28158_b200 as H
+    from workloads import CONFIGS, config_forest, make_inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    cfg = CONFIGS[args.workload]
+    fo = config_forest(args.workload)
+    t0 = time.perf_counter()
+    plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, cfg["chunk"])
+    t_plan = time.perf_counter() - t0
+    plan.upload()
+    Hh, dk, dv = cfg["H"], cfg["dk"], cfg["dv"]
+    # every rank draws its own tensors (independent batches of the same shape)
+    inp = make_inputs(plan.C, Hh, dk, dv, cfg["dtype"], cfg["seed"] + 100 * rank, device="cuda")
+    flags = H.HARTS_FLAG_FMA_KERNELS if args.fma else 0
+    ws = H.Workspace(plan, Hh, dk, dv, inp["q"].dtype, flags)
+    out = {"o": torch.empty_like(inp["v"]), "dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]),
+           "dv": torch.empty_like(inp["v"]), "dg": torch.empty_like(inp["g"])}
+    elem = inp["q"].element_size()
+    in_bytes = sum(x.numel() * x.element_size() for x in inp.values())
+    out_bytes = sum(x.numel() * x.element_size() for x in out.values())
+    stream = torch.cuda.current_stream()
+    K = plan.n_rounds
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+    launch_times = {"fwd": [], "bwd": [], "fold": []}
+
+    def step(record):
+        marks = []
+        for r in range(1, K + 1):
+            a, b = ev(), ev()
+            a.record(stream)
+            H.harts_la_fwd(plan, r, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], ws.slots, ws.chunk_states,
+                           flags, ws.dev_status)
+            b.record(stream)
+            marks.append(("fwd", a, b))
+        for r in range(K, 0, -1):
+            a, b = ev(), ev()
+            a.record(stream)
+            H.harts_la_bwd_seqs(plan.tables, int(plan.round_seq_ptr[r - 1]), int(plan.round_seq_ptr[r]), inp["q"],
+                                inp["k"], inp["v"], inp["g"], inp["dO"], out["dq"], out["dk"], out["dv"], out["dg"],
+                                ws.chunk_states, ws.scratch, flags, ws.dev_status)
+            b.record(stream)
+            marks.append(("bwd", a, b))
+        a, b = ev(), ev()
+        a.record(stream)
+        H.harts_la_bwd_finish(plan.tables, out["dk"], out["dv"], out["dg"], ws.scratch)
+        b.record(stream)
+        marks.append(("fold", a, b))
+        if record:
+            return marks
+        return None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step(False)
+    H.harts_la_check(ws.dev_status)
+    barrier()
+    all_marks = []
+    t_begin, t_end = ev(), ev()
+    with ClockSampler(local) as clocks:
+        t_begin.record(stream)
+        for _ in range(args.steps):
+            all_marks.append(step(True))
+        t_end.record(stream)
+        barrier()
+    ms_total = t_begin.elapsed_time(t_end)
+    H.harts_la_check(ws.dev_status)
+    for marks in all_marks:
+        for kind, a, b in marks:
+            launch_times[kind].append(a.elapsed_time(b))
+
+    # ---- end to end through host buffers -----------------------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        pinned = True
+        try:
+            host_in = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in inp.items()}
+            host_out = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in out.items()}
+        except RuntimeError:
+            pinned = False
+            host_in = {n: torch.empty(x.shape, dtype=x.dtype) for n, x in inp.items()}
+            host_out = {n: torch.empty(x.shape, dtype=x.dtype) for n, x in out.items()}
+        for n in inp:
+            host_in[n].copy_(inp[n])
+        torch.cuda.synchronize()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        H.run_fwd_bwd_host(plan, ws, host_in, inp, out, host_out)       # warm-up
+        barrier()
+        t0 = time.perf_counter()
+        a, b = ev(), ev()
+        a.record(stream)
+        for _ in range(e2e_steps):
+            H.run_fwd_bwd_host(plan, ws, host_in, inp, out, host_out)
+        b.record(stream)
+        barrier()
+        e2e_ms = a.elapsed_time(b) / e2e_steps
+        e2e = {"ms_per_step": e2e_ms, "steps": e2e_steps, "pinned": pinned,
+               "wall_ms_per_step": (time.perf_counter() - t0) * 1e3 / e2e_steps}
+        del host_in, host_out
+
+    # ---- reduce over ranks ------------------------------------------------------------------------
+    ms_step = ms_total / args.steps
+    if world > 1:
+        t = torch.tensor([ms_step, e2e["ms_per_step"] if e2e else 0.0], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t[0])
+        if e2e:
+            e2e["ms_per_step"] = float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    tokens = plan.C * world
+    value = tokens / (ms_step * 1e-3)
+    th = plan.C * Hh                                  # token-heads per rank and step
+    # algorithmic (compulsory) bytes per token-head: fwd reads q,k,v,g and writes o; bwd reads q,k,v,dO,g
+    # and writes dq,dk,dv,dg
+    fwd_bytes = th * ((2 * dk + 2 * dv) * elem + 4)
+    bwd_bytes = th * ((4 * dk + 3 * dv) * elem + 8)
+    flops_fwd = th * (2 * 64 * dk + 2 * 64 * dv + 4 * dk * dv)
+    flops_bwd = th * (5 * 2 * 64 * (dk + dv) // 2 + 4 * 2 * dk * dv)
+    bwd_ms = sum(launch_times["bwd"]) / args.steps
+    fwd_ms = sum(launch_times["fwd"]) / args.steps
+    fold_ms = sum(launch_times["fold"]) / args.steps
+    hbm_peak = peaks["hbm_gbs"]
+    achieved = bwd_bytes / (bwd_ms * 1e-3) / 1e9
+    t_roof_bytes = (fwd_bytes + bwd_bytes) / (hbm_peak * 1e9)
+    t_roof_flops = (flops_fwd + flops_bwd) / (peaks["bf16_tflops_sustained"] * 1e12)
+    clock = clocks.summary()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": cfg["dtype"] if cfg["dtype"] != "fp32" else "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "H": Hh, "dk": dk, "dv": dv, "chunk": cfg["chunk"],
+                   "compact_tokens": plan.C, "replay_rows": plan.R, "rounds": plan.n_rounds,
+                   "sequences": plan.n_seq, "slots": plan.n_slots, "chunks": plan.n_chunks,
+                   "l2": f"inputs larger than L2 ({in_bytes / 2**30:.2f} GiB read per step)"
+                         if in_bytes > 2 * L2_BYTES else "inputs smaller than L2: no flush (small workload)",
+                   "kernels": "fma" if args.fma or cfg["dtype"] == "fp32" else "default",
+                   "plan_ms": t_plan * 1e3},
+        "roofline": {"bound": "hbm", "kernel": "backward packed call (all rounds)", "achieved": achieved,
+                     "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak, "traffic": None,
+                     "peak_source": peaks["source"],
+                     "whole_path": {"roof_ms": max(t_roof_bytes, t_roof_flops) * 1e3,
+                                    "frac_strict": max(t_roof_bytes, t_roof_flops) * 1e3 / ms_step,
+                                    "frac_strict_nominal": max((fwd_bytes + bwd_bytes) / 8e12,
+                                                               (flops_fwd + flops_bwd) / 2.25e15) * 1e3 / ms_step}},
+        "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms, "fold": fold_ms},
+        "gpu_launches": (2 * K + (1 if plan.n_rg_rows else 0)) * args.steps,
+        "clocks": clock,
+    }
+    if e2e:
+        line["e2e"] = {"value": tokens / (e2e["ms_per_step"] * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_bytes, "steps": e2e["steps"],
+                       "pinned_host_memory": e2e["pinned"]}
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = oracle_sample(args.workload)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--fma", action="store_true", help="force the fp32-FMA kernels")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -10,9 +10,12 @@ TORCH_DTYPE = {"fp32": torch.float32, "bf16": torch.bfloat16}
 
 
 def rel_err(x, ref):
+    """Relative Frobenius error.  Where the reference is (numerically) zero -- e.g. dg of a one-token
+    trajectory, which is exactly 0 -- the denominator falls back to 1e-3 per element, i.e. the
+    difference is held to an absolute bound instead."""
     x = np.asarray(x, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
-    return float(np.linalg.norm(x - ref) / max(np.linalg.norm(ref), 1e-300))
+    return float(np.linalg.norm(x - ref) / max(np.linalg.norm(ref), 1e-3 * np.sqrt(ref.size)))
 
 
 def plan_of(fo, chunk=64):

@@ -66,7 +66,7 @@ def edge_forests():
     return {
         "one_token": make_forest([([-1], [0], [1])]),
         "exact_chunk": make_forest([([-1, 0, 0], [0, 64, 64], [64, 64, 1])]),
-        "two_chunks_and_tail": make_forest([([-1, 0, 0, 1], [0, 128, 100, 63], [129, 5, 200, 64])]),
+        "two_chunks_and_tail": make_forest([([-1, 0, 0, 2], [0, 128, 100, 63], [129, 5, 200, 64])]),
         "many_tiny": make_forest([([-1] + [0] * 40, [0] + [1 + (7 * i) % 90 for i in range(40)],
                                    [90] + [1 + i % 5 for i in range(40)])] * 3),
         "nested_in_chunk": make_forest([([-1, 0, 1, 2, 3, 0], [0, 10, 5, 3, 2, 10], [10, 7, 6, 4, 70, 130])]),
