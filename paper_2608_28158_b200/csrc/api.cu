@@ -21,6 +21,11 @@ int32_t check_common(const harts_la_tables_t* tb, int32_t seq_lo, int32_t seq_hi
     return HARTS_OK;
 }
 
+// The tensor-core kernels serve bf16 with d_k = d_v = 128 unless the caller asks for the FMA kernels.
+inline bool use_tc(int32_t dtype, int32_t dk, int32_t dv, uint32_t flags) {
+    return !(flags & HARTS_FLAG_FMA_KERNELS) && harts::tc_supported(dtype, dk, dv);
+}
+
 }  // namespace
 
 extern "C" {
@@ -70,6 +75,7 @@ int32_t harts_la_fwd_seqs(const harts_la_tables_t* tb, int32_t seq_lo, int32_t s
         return HARTS_EINVAL;
     harts::FwdArgs a{*tb, seq_lo, seq_hi, q, k, v, g, o, slots, chunk_states, H, dk, dv, dtype, flags, dev_status,
                      static_cast<cudaStream_t>(stream)};
+    if (use_tc(dtype, dk, dv, flags)) return harts::tc_fwd(a);
     return harts::fma_fwd(a);
 }
 
@@ -84,7 +90,7 @@ int32_t harts_la_bwd_seqs(const harts_la_tables_t* tb, int32_t seq_lo, int32_t s
         misaligned(dk_) || misaligned(dv_) || misaligned(dg) || misaligned(chunk_states) || misaligned(scratch))
         return HARTS_EINVAL;
     harts::BwdArgs a{*tb, seq_lo, seq_hi, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, scratch, H, dk, dv, dtype,
-                     flags, dev_status, static_cast<cudaStream_t>(stream)};
+                     flags, dev_status, static_cast<cudaStream_t>(stream), use_tc(dtype, dk, dv, flags) ? 1 : 0};
     return harts::fma_bwd(a);
 }
 

@@ -38,6 +38,7 @@ struct BwdArgs {
     uint32_t flags;
     int32_t* dev_status;
     cudaStream_t stream;
+    int32_t cs_transposed;   // chunk states stored [dv][dk] (tensor-core forward) instead of [dk][dv]
 };
 
 // Byte offsets inside the backward scratch buffer (each region 256-byte aligned).
@@ -69,6 +70,8 @@ inline ScratchLayout scratch_layout(const harts_la_tables_t& tb, int32_t H, int3
 int32_t fma_supported(int32_t dtype, int32_t dk, int32_t dv);
 int32_t fma_fwd(const FwdArgs& a);
 int32_t fma_bwd(const BwdArgs& a);
+int32_t tc_supported(int32_t dtype, int32_t dk, int32_t dv);
+int32_t tc_fwd(const FwdArgs& a);
 int32_t replay_reduce(const harts_la_tables_t& tb, void* dk_, void* dv_, float* dg, const void* scratch, int32_t H,
                       int32_t dk, int32_t dv, int32_t dtype, cudaStream_t stream);
 

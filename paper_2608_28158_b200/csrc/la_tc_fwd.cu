@@ -1,0 +1,379 @@
+// Tensor-core forward of the packed chunkwise call (Eq. 16) for bf16, d_k = d_v = 128, chunk 64.
+//
+// One CTA per (sequence, head) walks the chunks in order.  The recurrent state lives in tensor
+// memory for the whole walk, TRANSPOSED: lane j' (0..127) holds row j' of S^T, i.e. S[i][j'] for all
+// i in its 128 fp32 columns.  Per chunk (b_t = running sum of g, n = last row, w_j = e^{b_n-b_j}):
+//     A     = Q K^T                      tcgen05, M=128 (rows 64..127 unused) N=64  K=128
+//     P     = A .* e^{b_t-b_j} [j<=t]    registers -> bf16 tile in shared memory
+//     O1^T  = V^T P^T                    tcgen05, M=128 (d_v) N=64 (t) K=64 (j)
+//     O2^T  = S_c^T Q^T                  tcgen05, M=128 N=64 K=128, S_c^T as bf16 tile
+//     o_t   = O1 + e^{b_t} O2            epilogue, own rows only
+//     S^T   = e^{b_n} S^T + V^T (w .* K) tcgen05 accumulate, M=128 N=128 K=64
+// q/k/v tiles arrive by TMA as 128-byte-swizzled panels; the first chunk of a replay-started
+// sequence is gathered row by row instead (replay rows come from arbitrary ancestor rows).  The
+// start-of-chunk state goes to the chunk-state workspace (bf16, [d_v][d_k] per chunk-head) by TMA
+// store, and to its slot (fp32, [d_k][d_v]) when the plan requests that boundary.
+// Every wait is bounded; a wait that runs out sets the status word and the walk carries on.
+#include "kernels.h"
+#include "tc_common.cuh"
+
+namespace harts {
+namespace {
+
+using namespace tc;
+
+constexpr int BT = 64, D = 128, NT = 128;
+constexpr int TILE = BT * D * 2;              // 16 KB: two panels of [64][64] bf16
+constexpr int PANEL = BT * 128;               // 8 KB
+constexpr int S_PANEL = D * 128;              // 16 KB: [128][64] bf16
+constexpr float LOG2E = 1.4426950408889634f;
+
+// tensor-memory columns
+constexpr int COL_S = 0, COL_A = 128, COL_O1 = 192, TMEM_COLS = 256;
+
+struct Smem {
+    static constexpr int q = 0, k = TILE, v = 2 * TILE, p = 3 * TILE, s = 3 * TILE + PANEL,
+                         misc = 3 * TILE + PANEL + 2 * S_PANEL;
+    static constexpr int bytes = misc + 2048;
+};
+struct Misc {
+    float part[BT];      // per-warp partial running sums of g
+    float b2[BT];        // running log-decay, in log2 units
+    float eb[BT];        // e^{b_t}
+    float w[BT];         // e^{b_n - b_t}
+    int code[BT];        // physical row (>= 0 own), -2 - row (replay), -1 (past the end)
+    float gamma;
+    uint32_t tmem;
+    uint64_t bar_tma, bar_a, bar_o;
+};
+
+struct SeqInfo {
+    int own_begin, n_replay, n_virtual, n_chunks, replay_base, init_slot, req_lo, req_hi, chunk_base;
+};
+__device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq) {
+    SeqInfo s;
+    s.own_begin = tb.seq_own_begin[seq];
+    int own_len = tb.seq_own_begin[seq + 1] - s.own_begin;
+    s.replay_base = tb.seq_replay_ptr[seq];
+    s.n_replay = tb.seq_replay_ptr[seq + 1] - s.replay_base;
+    s.n_virtual = s.n_replay + own_len;
+    s.n_chunks = (s.n_virtual + BT - 1) / BT;
+    s.init_slot = tb.seq_init_slot[seq];
+    s.req_lo = tb.seq_req_ptr[seq];
+    s.req_hi = tb.seq_req_ptr[seq + 1];
+    s.chunk_base = tb.seq_chunk_ptr[seq];
+    return s;
+}
+
+__global__ void __launch_bounds__(NT, 2)
+tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_constant__ CUtensorMap map_q,
+              const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+              const __grid_constant__ CUtensorMap map_cs, const __nv_bfloat16* __restrict__ q,
+              const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
+              __nv_bfloat16* __restrict__ o, float* __restrict__ slots, int store_states, int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    unsigned char* sQ = smem + Smem::q;
+    unsigned char* sK = smem + Smem::k;
+    unsigned char* sV = smem + Smem::v;
+    unsigned char* sP = smem + Smem::p;
+    unsigned char* sS = smem + Smem::s;
+    Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
+    const SeqInfo s = seq_info(tb, seq);
+    const size_t state_elems = (size_t)D * D;
+
+    if (tid == 0) {
+        mbar_init(&m.bar_tma, 1);
+        mbar_init(&m.bar_a, 1);
+        mbar_init(&m.bar_o, 1);
+        fence_barrier_init();
+    }
+    if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = m.tmem;
+    const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this thread's lane = tid
+
+    // initial state S^T into tensor memory: lane j' = tid, column i
+    {
+        const float* src = s.init_slot < 0 ? nullptr : slots + ((size_t)s.init_slot * H + h) * state_elems;
+        for (int blk = 0; blk < 4; blk++) {
+            uint32_t x[32];
+#pragma unroll
+            for (int i = 0; i < 32; i++) x[i] = src ? __float_as_uint(src[(size_t)(blk * 32 + i) * D + tid]) : 0u;
+            tmem_st32(tm_lane + COL_S + blk * 32, x);
+        }
+        tmem_st_wait();
+    }
+
+    const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV), aP = smem_u32(sP), aS = smem_u32(sS);
+    constexpr uint32_t IDESC_A = instr_desc(128, 64, 0, 0);    // Q (K-major) x K (K-major)
+    constexpr uint32_t IDESC_O1 = instr_desc(128, 64, 1, 0);   // V^T (MN-major) x P (K-major)
+    constexpr uint32_t IDESC_O2 = instr_desc(128, 64, 0, 0);   // S^T (K-major) x Q (K-major)
+    constexpr uint32_t IDESC_S = instr_desc(128, 128, 1, 1);   // V^T (MN-major) x K~ (MN-major)
+
+    auto issue_tma = [&](int c) {
+        int row0 = s.own_begin - s.n_replay + c * BT;
+        mbar_expect_tx(&m.bar_tma, 3 * TILE);
+        for (int p = 0; p < 2; p++) {
+            tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_tma);
+            tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tma);
+            tma_load_3d(sV + p * PANEL, &map_v, p * 64, h, row0, &m.bar_tma);
+        }
+    };
+
+    const bool gather_first = s.n_replay > 0;
+    uint32_t ph_tma = 0, ph_a = 0, ph_o = 0;
+    int next_req = s.req_lo;
+    if (!gather_first && tid == 0) issue_tma(0);
+
+    for (int c = 0; c < s.n_chunks; c++) {
+        // ---- row codes and g for this chunk (registers first: the previous epilogue still reads m.code) ----
+        float gval = 0.f;
+        int my_code = -1;
+        if (tid < BT) {
+            int vr = c * BT + tid;
+            if (vr < s.n_virtual) {
+                int r = vr < s.n_replay ? tb.replay_row[s.replay_base + vr] : s.own_begin + (vr - s.n_replay);
+                my_code = vr < s.n_replay ? -2 - r : r;
+                gval = g[(size_t)r * H + h];
+            }
+        }
+        if (tid == 0) tma_store_wait_read();      // the previous chunk's state store has left sS
+        tc_fence_before();
+        __syncthreads();                          // (1) epilogue of the previous chunk is over everywhere
+        tc_fence_after();
+        if (tid < BT) {
+            m.code[tid] = my_code;
+            float x = gval;                       // inclusive scan inside each of the two warps
+#pragma unroll
+            for (int o_ = 1; o_ < 32; o_ <<= 1) {
+                float y = __shfl_up_sync(0xffffffffu, x, o_);
+                if (lane >= o_) x += y;
+            }
+            m.part[tid] = x;
+        }
+        if (c == 0 && gather_first) {
+            __syncthreads();
+            for (int e = tid; e < BT * 16; e += NT) {
+                int row = e >> 4, ch = e & 15, code = m.code[row];
+                uint4 zero = make_uint4(0, 0, 0, 0), kq = zero, vq = zero, qq = zero;
+                if (code != -1) {
+                    int r = code >= 0 ? code : -2 - code;
+                    size_t off = ((size_t)r * H + h) * D + ch * 8;
+                    kq = *reinterpret_cast<const uint4*>(k + off);
+                    vq = *reinterpret_cast<const uint4*>(v + off);
+                    if (code >= 0) qq = *reinterpret_cast<const uint4*>(q + off);
+                }
+                uint32_t dst = (ch >> 3) * PANEL + sw128_chunk(row, ch & 7);
+                *reinterpret_cast<uint4*>(sQ + dst) = qq;
+                *reinterpret_cast<uint4*>(sK + dst) = kq;
+                *reinterpret_cast<uint4*>(sV + dst) = vq;
+            }
+            fence_async_smem();
+        }
+        __syncthreads();                          // (2) codes, gathered tiles, partial sums visible
+        if (tid < BT) {
+            float first_half_total = m.part[31];
+            float b = m.part[tid] + (tid >= 32 ? first_half_total : 0.f);
+            float bn = m.part[63] + first_half_total;
+            m.b2[tid] = b * LOG2E;
+            m.eb[tid] = ex2(b * LOG2E);
+            m.w[tid] = ex2((bn - b) * LOG2E);
+            if (tid == 0) m.gamma = ex2(bn * LOG2E);
+        }
+        if (!(c == 0 && gather_first)) {
+            mbar_wait(&m.bar_tma, ph_tma, status);
+            ph_tma ^= 1;
+        }
+        // ---- A = Q K^T ----------------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_A, desc_kmajor<BT>(aQ, ks), desc_kmajor<BT>(aK, ks), IDESC_A, ks > 0);
+            mma_commit(&m.bar_a);
+        }
+        __syncthreads();                          // (3) b2 / eb / w / gamma visible
+        // ---- state pass: S_c^T -> bf16 operand tile (+ slot), S^T <- gamma S^T ----------------------------
+        {
+            const bool export_slot = next_req < s.req_hi && tb.slot_chunk[next_req] == c;
+            float* slot_dst = export_slot ? slots + ((size_t)next_req * H + h) * state_elems : nullptr;
+            const float gamma = m.gamma;
+            for (int blk = 0; blk < 4; blk++) {
+                uint32_t x[32];
+                tmem_ld32(tm_lane + COL_S + blk * 32, x);
+                tmem_ld_wait();
+                if (slot_dst) {
+#pragma unroll
+                    for (int i = 0; i < 32; i++) slot_dst[(size_t)(blk * 32 + i) * D + tid] = __uint_as_float(x[i]);
+                }
+#pragma unroll
+                for (int v4 = 0; v4 < 4; v4++) {
+                    uint4 pk;
+                    pk.x = pack_bf16(__uint_as_float(x[v4 * 8 + 0]), __uint_as_float(x[v4 * 8 + 1]));
+                    pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
+                    pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
+                    pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
+                    int col = blk * 32 + v4 * 8;           // first of 8 consecutive i
+                    *reinterpret_cast<uint4*>(sS + (col >> 6) * S_PANEL + sw128_chunk(tid, (col & 63) >> 3)) = pk;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
+                tmem_st32(tm_lane + COL_S + blk * 32, x);
+            }
+            tmem_st_wait();
+            if (export_slot) next_req++;
+            fence_async_smem();
+        }
+        // ---- P = A .* decay (warps 0,1)  |  K <- w .* K (warps 2,3) ------------------------------------------
+        mbar_wait(&m.bar_a, ph_a, status);
+        ph_a ^= 1;
+        tc_fence_after();
+        if (warp < 2) {
+            const int t = tid;
+            const float bt = m.b2[t];
+            for (int half = 0; half < 2; half++) {
+                uint32_t x[32];
+                tmem_ld32(tm_lane + COL_A + half * 32, x);
+                tmem_ld_wait();
+#pragma unroll
+                for (int v4 = 0; v4 < 4; v4++) {
+                    float y[8];
+#pragma unroll
+                    for (int e = 0; e < 8; e++) {
+                        int j = half * 32 + v4 * 8 + e;
+                        y[e] = j <= t ? __uint_as_float(x[v4 * 8 + e]) * ex2(bt - m.b2[j]) : 0.f;
+                    }
+                    uint4 pk = make_uint4(pack_bf16(y[0], y[1]), pack_bf16(y[2], y[3]), pack_bf16(y[4], y[5]),
+                                          pack_bf16(y[6], y[7]));
+                    *reinterpret_cast<uint4*>(sP + sw128_chunk(t, half * 4 + v4)) = pk;
+                }
+            }
+        } else {
+            for (int e = tid - 64; e < BT * 16; e += 64) {
+                uint32_t off = e * 16;
+                float wj = m.w[(off % PANEL) >> 7];
+                uint4 raw = *reinterpret_cast<uint4*>(sK + off);
+                __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+                for (int e2 = 0; e2 < 4; e2++) {
+                    float2 f = __bfloat1622float2(h2[e2]);
+                    h2[e2] = __floats2bfloat162_rn(f.x * wj, f.y * wj);
+                }
+                *reinterpret_cast<uint4*>(sK + off) = raw;
+            }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();                          // (4) P, scaled K, S operand tile and scaled S^T are in place
+        tc_fence_after();
+        // ---- O1^T, O2^T, state update --------------------------------------------------------------------
+        if (tid == 0) {
+            if (store_states) {
+                int idx = (s.chunk_base + c) * H + h;
+                tma_store_3d(&map_cs, sS, 0, 0, idx);
+                tma_store_3d(&map_cs, sS + S_PANEL, 64, 0, idx);
+                tma_store_commit();
+            }
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_O1, desc_mnmajor<BT>(aV, ks), desc_kmajor<BT>(aP, ks), IDESC_O1, ks > 0);
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_A, desc_kmajor<D>(aS, ks), desc_kmajor<BT>(aQ, ks), IDESC_O2, ks > 0);
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_S, desc_mnmajor<BT>(aV, ks), desc_mnmajor<BT>(aK, ks), IDESC_S, true);
+            mma_commit(&m.bar_o);
+        }
+        mbar_wait(&m.bar_o, ph_o, status);
+        ph_o ^= 1;
+        tc_fence_after();
+        if (tid == 0 && c + 1 < s.n_chunks) issue_tma(c + 1);   // tiles are free: every MMA that read them is done
+        // ---- epilogue: o_t = O1 + e^{b_t} O2, lane = output column j' ---------------------------------------
+        for (int half = 0; half < 2; half++) {
+            uint32_t x1[32], x2[32];
+            tmem_ld32(tm_lane + COL_O1 + half * 32, x1);
+            tmem_ld32(tm_lane + COL_A + half * 32, x2);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; e++) {
+                int t = half * 32 + e, code = m.code[t];
+                if (code >= 0) {
+                    float val = __uint_as_float(x1[e]) + m.eb[t] * __uint_as_float(x2[e]);
+                    o[((size_t)code * H + h) * D + tid] = __float2bfloat16_rn(val);
+                }
+            }
+        }
+    }
+    if (tid == 0) tma_store_wait_all();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc<TMEM_COLS>(tmem);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+}  // namespace
+
+// [rows][H][128] bf16 tensor, box = 64 rows x 1 head x 64 columns
+int32_t make_row_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return HARTS_ECUDA;
+    cuuint64_t dims[3] = {128, (cuuint64_t)H, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {256, (cuuint64_t)H * 256};
+    cuuint32_t box[3] = {64, 1, 64}, es[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HARTS_OK : HARTS_ECUDA;
+}
+
+// [n][128][128] bf16 states, box = 1 state x 128 rows x 64 columns
+int32_t make_state_map(CUtensorMap* map, const void* base, int64_t n) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return HARTS_ECUDA;
+    cuuint64_t dims[3] = {128, 128, (cuuint64_t)(n < 1 ? 1 : n)};
+    cuuint64_t strides[2] = {256, 32768};
+    cuuint32_t box[3] = {64, 128, 1}, es[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HARTS_OK : HARTS_ECUDA;
+}
+
+int32_t tc_supported(int32_t dtype, int32_t dk, int32_t dv) { return dtype == HARTS_BF16 && dk == 128 && dv == 128; }
+
+int32_t tc_fwd(const FwdArgs& a) {
+    if (a.seq_hi == a.seq_lo) return HARTS_OK;
+    CUtensorMap mq, mk, mv, mcs;
+    int32_t rc;
+    if ((rc = make_row_map(&mq, a.q, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mk, a.k, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mv, a.v, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    const void* cs = a.chunk_states ? a.chunk_states : a.q;   // a valid address for the (unused) map
+    if ((rc = make_state_map(&mcs, cs, a.chunk_states ? (int64_t)a.tb.n_chunks * a.H : 1)) != HARTS_OK) return rc;
+    if (cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+        cudaSuccess)
+        return HARTS_ECUDA;
+    int n = (a.seq_hi - a.seq_lo) * a.H;
+    tc_fwd_kernel<<<n, NT, Smem::bytes + 1024, a.stream>>>(
+        a.tb, a.seq_lo, a.H, mq, mk, mv, mcs, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
+        (const __nv_bfloat16*)a.v, a.g, (__nv_bfloat16*)a.o, a.slots, a.chunk_states != nullptr, a.dev_status);
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+}  // namespace harts
