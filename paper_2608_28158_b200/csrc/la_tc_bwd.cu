@@ -1,0 +1,482 @@
+// Tensor-core backward of the packed chunkwise call for bf16, d_k = d_v = 128, chunk 64: one fused
+// kernel that walks a sequence's chunks in reverse and emits dq, dk, dv, dg and the gradient of the
+// sequence's initial state (the hand-off into the sequence that produced it, Section 3.4).
+//
+// One CTA per (sequence, head).  dS (gradient w.r.t. the state at the END of the current chunk) lives
+// in tensor memory for the whole walk, lane i (0..127) = row i of dS, columns = d_v.  Per chunk
+// (b_t running sum of g, n last row, w_j = e^{b_n-b_j}, D_tj = e^{b_t-b_j}[j<=t], dO~_t = e^{b_t} dO_t):
+//     A  = Q K^T,  dA = dO V^T                               (t on lanes 0..63)
+//     P  = A .* D, dP = dA .* D                              bf16 tiles, rows past the end zeroed
+//     dq^T = K^T dP^T + S_c dO~^T                            (lanes = d_k, columns = t)
+//     dk^T = Q^T dP   + w .* (dS V^T)                        two accumulators, combined in the epilogue
+//     dv^T = dO^T P   + w .* (dS^T K^T)                      two accumulators
+//     dg_t = sum_{tau>=t} (q.dq - k.dk) + e^{b_n} <S_c, dS> + sum_j k_j . (w_j dS v_j)
+//     dS  <- e^{b_n} dS + Q^T dO~                            accumulate in tensor memory
+// where dS includes, at an exported boundary, the initial-state gradients of every sequence that
+// started there (read from the scratch area, where those sequences' calls left them).
+// S_c comes from the chunk-state workspace written by the forward ([d_v][d_k] bf16 per chunk-head).
+// Gradients of replayed rows go to the scratch area (fp32) and are folded into their ancestor rows by
+// the replay-reduce kernel.  Every wait is bounded.
+#include "kernels.h"
+#include "tc_common.cuh"
+
+namespace harts {
+
+int32_t make_row_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H);
+int32_t make_state_map(CUtensorMap* map, const void* base, int64_t n);
+
+namespace {
+
+using namespace tc;
+
+constexpr int BT = 64, D = 128, NT = 128;
+constexpr int TILE = BT * D * 2;              // 16 KB
+constexpr int PANEL = BT * 128;               // 8 KB
+constexpr int S_PANEL = D * 128;              // 16 KB
+constexpr float LOG2E = 1.4426950408889634f;
+
+constexpr int COL_DS = 0, COL_A = 128, COL_DA = 192, COL_DQ = 256, COL_DK = 320, COL_DV = 384, TMEM_COLS = 512;
+
+struct Smem {
+    static constexpr int q = 0, k = TILE, v = 2 * TILE, dO = 3 * TILE, dOs = 4 * TILE, p = 5 * TILE,
+                         dp = 5 * TILE + PANEL, s = 5 * TILE + 2 * PANEL, ds = s + 2 * S_PANEL,
+                         misc = ds + 2 * S_PANEL;
+    static constexpr int bytes = misc + 4096;
+};
+struct Misc {
+    float part[BT];
+    float b2[BT];
+    float eb[BT];
+    float w[BT];
+    int code[BT];
+    float red[4][BT];     // per-warp partial sums of q.dq - k.dk
+    float gred[4];
+    float gamma;
+    uint32_t tmem;
+    uint64_t bar_tma, bar_a, bar_o;
+};
+
+struct SeqInfo {
+    int own_begin, n_replay, n_virtual, n_chunks, replay_base, init_slot, req_lo, req_hi, chunk_base;
+};
+__device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq) {
+    SeqInfo s;
+    s.own_begin = tb.seq_own_begin[seq];
+    int own_len = tb.seq_own_begin[seq + 1] - s.own_begin;
+    s.replay_base = tb.seq_replay_ptr[seq];
+    s.n_replay = tb.seq_replay_ptr[seq + 1] - s.replay_base;
+    s.n_virtual = s.n_replay + own_len;
+    s.n_chunks = (s.n_virtual + BT - 1) / BT;
+    s.init_slot = tb.seq_init_slot[seq];
+    s.req_lo = tb.seq_req_ptr[seq];
+    s.req_hi = tb.seq_req_ptr[seq + 1];
+    s.chunk_base = tb.seq_chunk_ptr[seq];
+    return s;
+}
+
+__device__ __forceinline__ float bf16_at(const unsigned char* tile, int row, int col) {
+    return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(tile + (col >> 6) * PANEL + sw128(row, col & 63)));
+}
+
+// Sum over the 32 lanes of a warp for each of 32 per-lane values; lane l returns the total of z[l].
+__device__ __forceinline__ float warp_transpose_reduce(float (&z)[32], int lane) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        const bool upper = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < s; i++) {
+            float send = upper ? z[i] : z[i + s];
+            float keep = upper ? z[i + s] : z[i];
+            z[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
+    }
+    return z[0];
+}
+
+__global__ void __launch_bounds__(NT, 1)
+tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_constant__ CUtensorMap map_q,
+              const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+              const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_cs,
+              const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+              const __nv_bfloat16* __restrict__ v, const float* __restrict__ g, const __nv_bfloat16* __restrict__ dO,
+              __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk_, __nv_bfloat16* __restrict__ dv_,
+              float* __restrict__ dg, float* __restrict__ ds0, float* __restrict__ rk, float* __restrict__ rv,
+              float* __restrict__ rg, int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    unsigned char* sQ = smem + Smem::q;
+    unsigned char* sK = smem + Smem::k;
+    unsigned char* sV = smem + Smem::v;
+    unsigned char* sDO = smem + Smem::dO;
+    unsigned char* sDOs = smem + Smem::dOs;
+    unsigned char* sP = smem + Smem::p;
+    unsigned char* sDP = smem + Smem::dp;
+    unsigned char* sS = smem + Smem::s;
+    unsigned char* sDS = smem + Smem::ds;
+    Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
+    const SeqInfo s = seq_info(tb, seq);
+    const size_t state_elems = (size_t)D * D;
+
+    if (tid == 0) {
+        mbar_init(&m.bar_tma, 1);
+        mbar_init(&m.bar_a, 1);
+        mbar_init(&m.bar_o, 1);
+        fence_barrier_init();
+    }
+    if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = m.tmem;
+    const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);
+
+    {   // dS = 0: nothing follows the last chunk
+        uint32_t zero[32];
+#pragma unroll
+        for (int i = 0; i < 32; i++) zero[i] = 0u;
+        for (int blk = 0; blk < 4; blk++) tmem_st32(tm_lane + COL_DS + blk * 32, zero);
+        tmem_st_wait();
+    }
+
+    const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV), aDO = smem_u32(sDO), aDOs = smem_u32(sDOs),
+                   aP = smem_u32(sP), aDP = smem_u32(sDP), aS = smem_u32(sS), aDS = smem_u32(sDS);
+    constexpr uint32_t I_KK64 = instr_desc(128, 64, 0, 0);
+    constexpr uint32_t I_MK64 = instr_desc(128, 64, 1, 0);
+    constexpr uint32_t I_MM64 = instr_desc(128, 64, 1, 1);
+    constexpr uint32_t I_MM128 = instr_desc(128, 128, 1, 1);
+
+    auto issue_tma = [&](int c, bool tiles) {
+        int row0 = s.own_begin - s.n_replay + c * BT;
+        int idx = (s.chunk_base + c) * H + h;
+        mbar_expect_tx(&m.bar_tma, (tiles ? 4 * TILE : 0) + 2 * S_PANEL);
+        tma_load_3d(sS, &map_cs, 0, 0, idx, &m.bar_tma);
+        tma_load_3d(sS + S_PANEL, &map_cs, 64, 0, idx, &m.bar_tma);
+        if (tiles)
+            for (int p = 0; p < 2; p++) {
+                tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_tma);
+                tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tma);
+                tma_load_3d(sV + p * PANEL, &map_v, p * 64, h, row0, &m.bar_tma);
+                tma_load_3d(sDO + p * PANEL, &map_do, p * 64, h, row0, &m.bar_tma);
+            }
+    };
+
+    const bool gather_first = s.n_replay > 0;
+    uint32_t ph_tma = 0, ph_a = 0, ph_o = 0;
+    int next_req = s.req_hi - 1;
+    if (tid == 0) issue_tma(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
+
+    for (int c = s.n_chunks - 1; c >= 0; c--) {
+        const bool gathered = c == 0 && gather_first;
+        // ---- row codes and g ---------------------------------------------------------------------------------
+        float gval = 0.f;
+        int my_code = -1;
+        if (tid < BT) {
+            int vr = c * BT + tid;
+            if (vr < s.n_virtual) {
+                int r = vr < s.n_replay ? tb.replay_row[s.replay_base + vr] : s.own_begin + (vr - s.n_replay);
+                my_code = vr < s.n_replay ? -2 - r : r;
+                gval = g[(size_t)r * H + h];
+            }
+        }
+        tc_fence_before();
+        __syncthreads();                          // (1) the previous chunk's epilogue is over everywhere
+        tc_fence_after();
+        if (tid < BT) {
+            m.code[tid] = my_code;
+            float x = gval;
+#pragma unroll
+            for (int o_ = 1; o_ < 32; o_ <<= 1) {
+                float y = __shfl_up_sync(0xffffffffu, x, o_);
+                if (lane >= o_) x += y;
+            }
+            m.part[tid] = x;
+        }
+        if (gathered) {
+            __syncthreads();
+            for (int e = tid; e < BT * 16; e += NT) {
+                int row = e >> 4, ch = e & 15, code = m.code[row];
+                uint4 zero = make_uint4(0, 0, 0, 0), kq = zero, vq = zero, qq = zero, dq4 = zero;
+                if (code != -1) {
+                    int r = code >= 0 ? code : -2 - code;
+                    size_t off = ((size_t)r * H + h) * D + ch * 8;
+                    kq = *reinterpret_cast<const uint4*>(k + off);
+                    vq = *reinterpret_cast<const uint4*>(v + off);
+                    if (code >= 0) {
+                        qq = *reinterpret_cast<const uint4*>(q + off);
+                        dq4 = *reinterpret_cast<const uint4*>(dO + off);
+                    }
+                }
+                uint32_t dst = (ch >> 3) * PANEL + sw128_chunk(row, ch & 7);
+                *reinterpret_cast<uint4*>(sQ + dst) = qq;
+                *reinterpret_cast<uint4*>(sK + dst) = kq;
+                *reinterpret_cast<uint4*>(sV + dst) = vq;
+                *reinterpret_cast<uint4*>(sDO + dst) = dq4;
+            }
+            fence_async_smem();
+        }
+        __syncthreads();                          // (2)
+        if (tid < BT) {
+            float first_half_total = m.part[31];
+            float b = m.part[tid] + (tid >= 32 ? first_half_total : 0.f);
+            float bn = m.part[63] + first_half_total;
+            m.b2[tid] = b * LOG2E;
+            m.eb[tid] = m.code[tid] >= 0 ? ex2(b * LOG2E) : 0.f;    // rows without an output carry no dO
+            m.w[tid] = ex2((bn - b) * LOG2E);
+            if (tid == 0) m.gamma = ex2(bn * LOG2E);
+        }
+        mbar_wait(&m.bar_tma, ph_tma, status);
+        ph_tma ^= 1;
+        // ---- A = Q K^T, dA = dO V^T -------------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_A, desc_kmajor<BT>(aQ, ks), desc_kmajor<BT>(aK, ks), I_KK64, ks > 0);
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_DA, desc_kmajor<BT>(aDO, ks), desc_kmajor<BT>(aV, ks), I_KK64, ks > 0);
+            mma_commit(&m.bar_a);
+        }
+        __syncthreads();                          // (3) b2 / eb / w / gamma visible
+        // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma ---------------------
+        float g_part = 0.f;                       // this thread's share of <S_{c+1}, dS_{c+1}>
+        {
+            const bool boundary = next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1;
+            const int cons_lo = boundary ? tb.slot_cons_ptr[next_req] : 0;
+            const int cons_hi = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
+            const float gamma = m.gamma;
+            float dot = 0.f;
+            for (int blk = 0; blk < 4; blk++) {
+                uint32_t x[32];
+                tmem_ld32(tm_lane + COL_DS + blk * 32, x);
+                tmem_ld_wait();
+                for (int u = cons_lo; u < cons_hi; u++) {
+                    const float4* src = reinterpret_cast<const float4*>(
+                        ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + (size_t)tid * D + blk * 32);
+#pragma unroll
+                    for (int i4 = 0; i4 < 8; i4++) {
+                        float4 a = src[i4];
+                        x[i4 * 4 + 0] = __float_as_uint(__uint_as_float(x[i4 * 4 + 0]) + a.x);
+                        x[i4 * 4 + 1] = __float_as_uint(__uint_as_float(x[i4 * 4 + 1]) + a.y);
+                        x[i4 * 4 + 2] = __float_as_uint(__uint_as_float(x[i4 * 4 + 2]) + a.z);
+                        x[i4 * 4 + 3] = __float_as_uint(__uint_as_float(x[i4 * 4 + 3]) + a.w);
+                    }
+                }
+#pragma unroll
+                for (int v4 = 0; v4 < 4; v4++) {
+                    uint4 pk;
+                    pk.x = pack_bf16(__uint_as_float(x[v4 * 8 + 0]), __uint_as_float(x[v4 * 8 + 1]));
+                    pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
+                    pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
+                    pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
+                    int col = blk * 32 + v4 * 8;
+                    *reinterpret_cast<uint4*>(sDS + (col >> 6) * S_PANEL + sw128_chunk(tid, (col & 63) >> 3)) = pk;
+                }
+                // S_c[i][j'] sits at row j', column i of the state tile (i = tid)
+#pragma unroll
+                for (int e = 0; e < 32; e++) {
+                    int jp = blk * 32 + e;
+                    float sv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(
+                        sS + (tid >> 6) * S_PANEL + sw128(jp, tid & 63)));
+                    dot += sv * __uint_as_float(x[e]);
+                }
+#pragma unroll
+                for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
+                tmem_st32(tm_lane + COL_DS + blk * 32, x);
+            }
+            tmem_st_wait();
+            if (boundary) next_req--;
+            g_part = gamma * dot;
+            fence_async_smem();
+        }
+        // ---- P, dP (warps 0,1) | dO~ = e^{b_t} dO (warps 2,3) ----------------------------------------------------
+        mbar_wait(&m.bar_a, ph_a, status);
+        ph_a ^= 1;
+        tc_fence_after();
+        if (warp < 2) {
+            const int t = tid;
+            const float bt = m.b2[t];
+            const bool live = m.code[t] >= 0;     // replay rows and rows past the end have no dO and no q
+            for (int half = 0; half < 2; half++) {
+                uint32_t xa[32], xd[32];
+                tmem_ld32(tm_lane + COL_A + half * 32, xa);
+                tmem_ld32(tm_lane + COL_DA + half * 32, xd);
+                tmem_ld_wait();
+#pragma unroll
+                for (int v4 = 0; v4 < 4; v4++) {
+                    float ya[8], yd[8];
+#pragma unroll
+                    for (int e = 0; e < 8; e++) {
+                        int j = half * 32 + v4 * 8 + e;
+                        float dec = (live && j <= t) ? ex2(bt - m.b2[j]) : 0.f;
+                        ya[e] = dec != 0.f ? __uint_as_float(xa[v4 * 8 + e]) * dec : 0.f;
+                        yd[e] = dec != 0.f ? __uint_as_float(xd[v4 * 8 + e]) * dec : 0.f;
+                    }
+                    uint32_t off = sw128_chunk(t, half * 4 + v4);
+                    *reinterpret_cast<uint4*>(sP + off) = make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]),
+                                                                     pack_bf16(ya[4], ya[5]), pack_bf16(ya[6], ya[7]));
+                    *reinterpret_cast<uint4*>(sDP + off) = make_uint4(pack_bf16(yd[0], yd[1]), pack_bf16(yd[2], yd[3]),
+                                                                      pack_bf16(yd[4], yd[5]), pack_bf16(yd[6], yd[7]));
+                }
+            }
+        } else {
+            for (int e = tid - 64; e < BT * 16; e += 64) {
+                uint32_t off = e * 16;
+                float sc = m.eb[(off % PANEL) >> 7];
+                uint4 raw = *reinterpret_cast<const uint4*>(sDO + off);
+                __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+                for (int e2 = 0; e2 < 4; e2++) {
+                    float2 f = __bfloat1622float2(h2[e2]);
+                    h2[e2] = sc != 0.f ? __floats2bfloat162_rn(f.x * sc, f.y * sc) : __floats2bfloat162_rn(0.f, 0.f);
+                }
+                *reinterpret_cast<uint4*>(sDOs + off) = raw;
+            }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();                          // (4) all operand tiles and the scaled dS are in place
+        tc_fence_after();
+        if (tid == 0) {
+            // dq^T = K^T dP^T + S_c dO~^T
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_DQ, desc_mnmajor<BT>(aK, ks), desc_kmajor<BT>(aDP, ks), I_MK64, ks > 0);
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_DQ, desc_mnmajor<D>(aS, ks), desc_kmajor<BT>(aDOs, ks), I_MK64, true);
+            // dk^T: Q^T dP   |   dS V^T (into the columns A occupied)
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_DK, desc_mnmajor<BT>(aQ, ks), desc_mnmajor<BT>(aDP, ks), I_MM64, ks > 0);
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_A, desc_kmajor<D>(aDS, ks), desc_kmajor<BT>(aV, ks), I_KK64, ks > 0);
+            // dv^T: dO^T P   |   dS^T K^T (into the columns dA occupied)
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_DV, desc_mnmajor<BT>(aDO, ks), desc_mnmajor<BT>(aP, ks), I_MM64, ks > 0);
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_DA, desc_mnmajor<D>(aDS, ks), desc_kmajor<BT>(aK, ks), I_MK64, ks > 0);
+            // dS += Q^T dO~   (dS was pre-scaled by e^{b_n})
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_DS, desc_mnmajor<BT>(aQ, ks), desc_mnmajor<BT>(aDOs, ks), I_MM128, true);
+            mma_commit(&m.bar_o);
+        }
+        mbar_wait(&m.bar_o, ph_o, status);
+        ph_o ^= 1;
+        tc_fence_after();
+        // ---- epilogue (lane = feature index) -------------------------------------------------------------------------
+        for (int half = 0; half < 2; half++) {
+            float z[32];
+            {
+                uint32_t xq[32], xi[32], xe[32];
+                tmem_ld32(tm_lane + COL_DQ + half * 32, xq);
+                tmem_ld32(tm_lane + COL_DK + half * 32, xi);
+                tmem_ld32(tm_lane + COL_A + half * 32, xe);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; e++) {
+                    int t = half * 32 + e, code = m.code[t];
+                    float dqv = __uint_as_float(xq[e]);
+                    float inter = m.w[t] * __uint_as_float(xe[e]);
+                    float dkv = __uint_as_float(xi[e]) + inter;
+                    float qv = bf16_at(sQ, t, tid), kv = bf16_at(sK, t, tid);
+                    z[e] = code == -1 ? 0.f : qv * dqv - kv * dkv;
+                    if (code != -1) g_part += kv * inter;
+                    if (code >= 0) {
+                        size_t off = ((size_t)code * H + h) * D + tid;
+                        dq[off] = __float2bfloat16_rn(dqv);
+                        dk_[off] = __float2bfloat16_rn(dkv);
+                    } else if (code < -1) {
+                        rk[((size_t)(s.replay_base + t) * H + h) * D + tid] = dkv;    // replay rows sit in chunk 0
+                    }
+                }
+            }
+            float tot = warp_transpose_reduce(z, lane);
+            m.red[warp][half * 32 + lane] = tot;
+            {
+                uint32_t xi[32], xe[32];
+                tmem_ld32(tm_lane + COL_DV + half * 32, xi);
+                tmem_ld32(tm_lane + COL_DA + half * 32, xe);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; e++) {
+                    int t = half * 32 + e, code = m.code[t];
+                    float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
+                    if (code >= 0) dv_[((size_t)code * H + h) * D + tid] = __float2bfloat16_rn(dvv);
+                    else if (code < -1) rv[((size_t)(s.replay_base + t) * H + h) * D + tid] = dvv;
+                }
+            }
+        }
+        // <S_{c+1}, dS_{c+1}> over the block
+#pragma unroll
+        for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
+        if (lane == 0) m.gred[warp] = g_part;
+        tc_fence_before();
+        __syncthreads();                          // (5) tiles are no longer read; partial sums visible
+        if (tid == 0 && c > 0) issue_tma(c - 1, !(c - 1 == 0 && gather_first));
+        if (tid < BT) {
+            float r = m.red[0][tid] + m.red[1][tid] + m.red[2][tid] + m.red[3][tid];
+            // inclusive suffix sum over the 64 rows (two warps)
+            float x = r;
+#pragma unroll
+            for (int o_ = 1; o_ < 32; o_ <<= 1) {
+                float y = __shfl_down_sync(0xffffffffu, x, o_);
+                if (lane + o_ < 32) x += y;
+            }
+            m.part[tid] = x;
+        }
+        __syncthreads();                          // (6)
+        if (tid < BT) {
+            float G = m.gred[0] + m.gred[1] + m.gred[2] + m.gred[3];
+            float val = m.part[tid] + (tid < 32 ? m.part[32] : 0.f) + G;
+            int code = m.code[tid];
+            if (code >= 0) dg[(size_t)code * H + h] = val;
+            else if (code < -1) rg[(size_t)(s.replay_base + tid) * H + h] = val;
+        }
+    }
+    // gradient w.r.t. the initial state: the hand-off into the producing sequence
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (s.init_slot >= 0) {
+        float* dst = ds0 + ((size_t)seq * H + h) * state_elems + (size_t)tid * D;
+        for (int blk = 0; blk < 4; blk++) {
+            uint32_t x[32];
+            tmem_ld32(tm_lane + COL_DS + blk * 32, x);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i4 = 0; i4 < 8; i4++)
+                reinterpret_cast<float4*>(dst + blk * 32)[i4] =
+                    make_float4(__uint_as_float(x[i4 * 4]), __uint_as_float(x[i4 * 4 + 1]),
+                                __uint_as_float(x[i4 * 4 + 2]), __uint_as_float(x[i4 * 4 + 3]));
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc<TMEM_COLS>(tmem);
+}
+
+}  // namespace
+
+int32_t tc_bwd(const BwdArgs& a) {
+    if (a.seq_hi == a.seq_lo) return HARTS_OK;
+    CUtensorMap mq, mk, mv, mdo, mcs;
+    int32_t rc;
+    if ((rc = make_row_map(&mq, a.q, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mk, a.k, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mv, a.v, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mdo, a.dO, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_state_map(&mcs, a.chunk_states, (int64_t)a.tb.n_chunks * a.H)) != HARTS_OK) return rc;
+    if (cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+        cudaSuccess)
+        return HARTS_ECUDA;
+    ScratchLayout sl = scratch_layout(a.tb, a.H, a.dk, a.dv);
+    char* base = static_cast<char*>(a.scratch);
+    int n = (a.seq_hi - a.seq_lo) * a.H;
+    tc_bwd_kernel<<<n, NT, Smem::bytes + 1024, a.stream>>>(
+        a.tb, a.seq_lo, a.H, mq, mk, mv, mdo, mcs, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
+        (const __nv_bfloat16*)a.v, a.g, (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_,
+        (__nv_bfloat16*)a.dv_, a.dg, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
+        (float*)(base + sl.rg), a.dev_status);
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+}  // namespace harts
