@@ -29,7 +29,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int BT = 64, D = 128, NT = 128;
+constexpr int BT = 64, D = 128, NT = 256;   // 8 warps: warps w and w+4 share tensor-memory lanes 32(w&3)..+31
 constexpr int TILE = BT * D * 2;              // 16 KB
 constexpr int PANEL = BT * 128;               // 8 KB
 constexpr int S_PANEL = D * 128;              // 16 KB
@@ -49,11 +49,11 @@ struct Misc {
     float eb[BT];
     float w[BT];
     int code[BT];
-    float red[4][BT];     // per-warp partial sums of q.dq - k.dk
-    float gred[4];
+    float red[8][32];     // per-warp partial sums of q.dq - k.dk (warp w covers rows 32(w>>2)..+31)
+    float gred[8];
     float gamma;
     uint32_t tmem;
-    uint64_t bar_tma, bar_a, bar_o;
+    uint64_t bar_vds, bar_qk, bar_a, bar_o;
 };
 
 struct SeqInfo {
@@ -116,12 +116,15 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int grp = warp >> 2;                    // which half of the columns this warp works on
+    const int L = (warp & 3) * 32 + lane;         // tensor-memory lane = feature index (or row t) of this thread
     const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
     const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)D * D;
 
     if (tid == 0) {
-        mbar_init(&m.bar_tma, 1);
+        mbar_init(&m.bar_vds, 1);
+        mbar_init(&m.bar_qk, 1);
         mbar_init(&m.bar_a, 1);
         mbar_init(&m.bar_o, 1);
         fence_barrier_init();
@@ -131,13 +134,13 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = m.tmem;
-    const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
     {   // dS = 0: nothing follows the last chunk
         uint32_t zero[32];
 #pragma unroll
         for (int i = 0; i < 32; i++) zero[i] = 0u;
-        for (int blk = 0; blk < 4; blk++) tmem_st32(tm_lane + COL_DS + blk * 32, zero);
+        for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) tmem_st32(tm_lane + COL_DS + blk * 32, zero);
         tmem_st_wait();
     }
 
@@ -148,39 +151,53 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     constexpr uint32_t I_MM64 = instr_desc(128, 64, 1, 1);
     constexpr uint32_t I_MM128 = instr_desc(128, 128, 1, 1);
 
-    auto issue_tma = [&](int c, bool tiles) {
+    // v, dO and the start-of-chunk state are free as soon as the chunk's MMAs are done; q and k are still
+    // read by the epilogue, so they travel on a barrier of their own.
+    auto issue_vds = [&](int c, bool tiles) {
         int row0 = s.own_begin - s.n_replay + c * BT;
         int idx = (s.chunk_base + c) * H + h;
-        mbar_expect_tx(&m.bar_tma, (tiles ? 4 * TILE : 0) + 2 * S_PANEL);
-        tma_load_3d(sS, &map_cs, 0, 0, idx, &m.bar_tma);
-        tma_load_3d(sS + S_PANEL, &map_cs, 64, 0, idx, &m.bar_tma);
+        mbar_expect_tx(&m.bar_vds, (tiles ? 2 * TILE : 0) + 2 * S_PANEL);
+        tma_load_3d(sS, &map_cs, 0, 0, idx, &m.bar_vds);
+        tma_load_3d(sS + S_PANEL, &map_cs, 64, 0, idx, &m.bar_vds);
         if (tiles)
             for (int p = 0; p < 2; p++) {
-                tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_tma);
-                tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tma);
-                tma_load_3d(sV + p * PANEL, &map_v, p * 64, h, row0, &m.bar_tma);
-                tma_load_3d(sDO + p * PANEL, &map_do, p * 64, h, row0, &m.bar_tma);
+                tma_load_3d(sV + p * PANEL, &map_v, p * 64, h, row0, &m.bar_vds);
+                tma_load_3d(sDO + p * PANEL, &map_do, p * 64, h, row0, &m.bar_vds);
             }
+    };
+    auto issue_qk = [&](int c) {
+        int row0 = s.own_begin - s.n_replay + c * BT;
+        mbar_expect_tx(&m.bar_qk, 2 * TILE);
+        for (int p = 0; p < 2; p++) {
+            tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_qk);
+            tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_qk);
+        }
+    };
+    auto row_code = [&](int c, int& code, float& gval) {
+        code = -1;
+        gval = 0.f;
+        int vr = c * BT + tid;
+        if (tid < BT && c >= 0 && vr < s.n_virtual) {
+            int r = vr < s.n_replay ? tb.replay_row[s.replay_base + vr] : s.own_begin + (vr - s.n_replay);
+            code = vr < s.n_replay ? -2 - r : r;
+            gval = g[(size_t)r * H + h];
+        }
     };
 
     const bool gather_first = s.n_replay > 0;
-    uint32_t ph_tma = 0, ph_a = 0, ph_o = 0;
+    uint32_t ph_vds = 0, ph_qk = 0, ph_a = 0, ph_o = 0;
     int next_req = s.req_hi - 1;
-    if (tid == 0) issue_tma(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
+    if (tid == 0) {
+        const bool tiles = !(gather_first && s.n_chunks == 1);
+        issue_vds(s.n_chunks - 1, tiles);
+        if (tiles) issue_qk(s.n_chunks - 1);
+    }
+    int my_code;
+    float gval;
+    row_code(s.n_chunks - 1, my_code, gval);
 
     for (int c = s.n_chunks - 1; c >= 0; c--) {
         const bool gathered = c == 0 && gather_first;
-        // ---- row codes and g ---------------------------------------------------------------------------------
-        float gval = 0.f;
-        int my_code = -1;
-        if (tid < BT) {
-            int vr = c * BT + tid;
-            if (vr < s.n_virtual) {
-                int r = vr < s.n_replay ? tb.replay_row[s.replay_base + vr] : s.own_begin + (vr - s.n_replay);
-                my_code = vr < s.n_replay ? -2 - r : r;
-                gval = g[(size_t)r * H + h];
-            }
-        }
         tc_fence_before();
         __syncthreads();                          // (1) the previous chunk's epilogue is over everywhere
         tc_fence_after();
@@ -227,16 +244,13 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             m.w[tid] = ex2((bn - b) * LOG2E);
             if (tid == 0) m.gamma = ex2(bn * LOG2E);
         }
-        mbar_wait(&m.bar_tma, ph_tma, status);
-        ph_tma ^= 1;
-        // ---- A = Q K^T, dA = dO V^T -------------------------------------------------------------------------------
+        mbar_wait(&m.bar_vds, ph_vds, status);
+        ph_vds ^= 1;
+        // ---- dA = dO V^T can start before q and k have landed -----------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
             for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_A, desc_kmajor<BT>(aQ, ks), desc_kmajor<BT>(aK, ks), I_KK64, ks > 0);
-            for (int ks = 0; ks < 8; ks++)
                 mma_ss(tmem + COL_DA, desc_kmajor<BT>(aDO, ks), desc_kmajor<BT>(aV, ks), I_KK64, ks > 0);
-            mma_commit(&m.bar_a);
         }
         __syncthreads();                          // (3) b2 / eb / w / gamma visible
         // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma ---------------------
@@ -247,13 +261,13 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             const int cons_hi = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
             const float gamma = m.gamma;
             float dot = 0.f;
-            for (int blk = 0; blk < 4; blk++) {
+            for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
                 uint32_t x[32];
                 tmem_ld32(tm_lane + COL_DS + blk * 32, x);
                 tmem_ld_wait();
                 for (int u = cons_lo; u < cons_hi; u++) {
                     const float4* src = reinterpret_cast<const float4*>(
-                        ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + (size_t)tid * D + blk * 32);
+                        ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + (size_t)L * D + blk * 32);
 #pragma unroll
                     for (int i4 = 0; i4 < 8; i4++) {
                         float4 a = src[i4];
@@ -271,14 +285,14 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                     pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
                     pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
                     int col = blk * 32 + v4 * 8;
-                    *reinterpret_cast<uint4*>(sDS + (col >> 6) * S_PANEL + sw128_chunk(tid, (col & 63) >> 3)) = pk;
+                    *reinterpret_cast<uint4*>(sDS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3)) = pk;
                 }
-                // S_c[i][j'] sits at row j', column i of the state tile (i = tid)
+                // S_c[i][j'] sits at row j', column i of the state tile (i = L)
 #pragma unroll
                 for (int e = 0; e < 32; e++) {
                     int jp = blk * 32 + e;
                     float sv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(
-                        sS + (tid >> 6) * S_PANEL + sw128(jp, tid & 63)));
+                        sS + (L >> 6) * S_PANEL + sw128(jp, L & 63)));
                     dot += sv * __uint_as_float(x[e]);
                 }
 #pragma unroll
@@ -290,15 +304,26 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             g_part = gamma * dot;
             fence_async_smem();
         }
-        // ---- P, dP (warps 0,1) | dO~ = e^{b_t} dO (warps 2,3) ----------------------------------------------------
+        // ---- A = Q K^T once q and k are here ---------------------------------------------------------------------
+        if (!gathered) {
+            mbar_wait(&m.bar_qk, ph_qk, status);
+            ph_qk ^= 1;
+        }
+        if (tid == 0) {
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_A, desc_kmajor<BT>(aQ, ks), desc_kmajor<BT>(aK, ks), I_KK64, ks > 0);
+            mma_commit(&m.bar_a);
+        }
+        // ---- P, dP (lanes 0..63 of both column groups) | dO~ = e^{b_t} dO (the other four warps) ----------------------
         mbar_wait(&m.bar_a, ph_a, status);
         ph_a ^= 1;
         tc_fence_after();
-        if (warp < 2) {
-            const int t = tid;
+        if ((warp & 3) < 2) {
+            const int t = L;
             const float bt = m.b2[t];
             const bool live = m.code[t] >= 0;     // replay rows and rows past the end have no dO and no q
-            for (int half = 0; half < 2; half++) {
+            {
+                const int half = grp;
                 uint32_t xa[32], xd[32];
                 tmem_ld32(tm_lane + COL_A + half * 32, xa);
                 tmem_ld32(tm_lane + COL_DA + half * 32, xd);
@@ -321,7 +346,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 }
             }
         } else {
-            for (int e = tid - 64; e < BT * 16; e += 64) {
+            for (int e = ((warp & 3) - 2) * 32 + lane + 64 * grp; e < BT * 16; e += 128) {
                 uint32_t off = e * 16;
                 float sc = m.eb[(off % PANEL) >> 7];
                 uint4 raw = *reinterpret_cast<const uint4*>(sDO + off);
@@ -362,8 +387,12 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         mbar_wait(&m.bar_o, ph_o, status);
         ph_o ^= 1;
         tc_fence_after();
+        const bool next_tiles = !(c - 1 == 0 && gather_first);
+        if (tid == 0 && c > 0) issue_vds(c - 1, next_tiles);
+        row_code(c - 1, my_code, gval);           // next chunk's rows and g, in flight during the epilogue
         // ---- epilogue (lane = feature index) -------------------------------------------------------------------------
-        for (int half = 0; half < 2; half++) {
+        {
+            const int half = grp;
             float z[32];
             {
                 uint32_t xq[32], xi[32], xe[32];
@@ -377,20 +406,20 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                     float dqv = __uint_as_float(xq[e]);
                     float inter = m.w[t] * __uint_as_float(xe[e]);
                     float dkv = __uint_as_float(xi[e]) + inter;
-                    float qv = bf16_at(sQ, t, tid), kv = bf16_at(sK, t, tid);
+                    float qv = bf16_at(sQ, t, L), kv = bf16_at(sK, t, L);
                     z[e] = code == -1 ? 0.f : qv * dqv - kv * dkv;
                     if (code != -1) g_part += kv * inter;
                     if (code >= 0) {
-                        size_t off = ((size_t)code * H + h) * D + tid;
+                        size_t off = ((size_t)code * H + h) * D + L;
                         dq[off] = __float2bfloat16_rn(dqv);
                         dk_[off] = __float2bfloat16_rn(dkv);
                     } else if (code < -1) {
-                        rk[((size_t)(s.replay_base + t) * H + h) * D + tid] = dkv;    // replay rows sit in chunk 0
+                        rk[((size_t)(s.replay_base + t) * H + h) * D + L] = dkv;    // replay rows sit in chunk 0
                     }
                 }
             }
             float tot = warp_transpose_reduce(z, lane);
-            m.red[warp][half * 32 + lane] = tot;
+            m.red[warp][lane] = tot;
             {
                 uint32_t xi[32], xe[32];
                 tmem_ld32(tm_lane + COL_DV + half * 32, xi);
@@ -400,8 +429,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 for (int e = 0; e < 32; e++) {
                     int t = half * 32 + e, code = m.code[t];
                     float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
-                    if (code >= 0) dv_[((size_t)code * H + h) * D + tid] = __float2bfloat16_rn(dvv);
-                    else if (code < -1) rv[((size_t)(s.replay_base + t) * H + h) * D + tid] = dvv;
+                    if (code >= 0) dv_[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dvv);
+                    else if (code < -1) rv[((size_t)(s.replay_base + t) * H + h) * D + L] = dvv;
                 }
             }
         }
@@ -411,9 +440,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         if (lane == 0) m.gred[warp] = g_part;
         tc_fence_before();
         __syncthreads();                          // (5) tiles are no longer read; partial sums visible
-        if (tid == 0 && c > 0) issue_tma(c - 1, !(c - 1 == 0 && gather_first));
+        if (tid == 0 && c > 0 && next_tiles) issue_qk(c - 1);
         if (tid < BT) {
-            float r = m.red[0][tid] + m.red[1][tid] + m.red[2][tid] + m.red[3][tid];
+            const int g4 = (tid >> 5) * 4;
+            float r = m.red[g4][lane] + m.red[g4 + 1][lane] + m.red[g4 + 2][lane] + m.red[g4 + 3][lane];
             // inclusive suffix sum over the 64 rows (two warps)
             float x = r;
 #pragma unroll
@@ -425,7 +455,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         }
         __syncthreads();                          // (6)
         if (tid < BT) {
-            float G = m.gred[0] + m.gred[1] + m.gred[2] + m.gred[3];
+            float G = m.gred[0] + m.gred[1] + m.gred[2] + m.gred[3] + m.gred[4] + m.gred[5] + m.gred[6] + m.gred[7];
             float val = m.part[tid] + (tid < 32 ? m.part[32] : 0.f) + G;
             int code = m.code[tid];
             if (code >= 0) dg[(size_t)code * H + h] = val;
@@ -437,8 +467,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     __syncthreads();
     tc_fence_after();
     if (s.init_slot >= 0) {
-        float* dst = ds0 + ((size_t)seq * H + h) * state_elems + (size_t)tid * D;
-        for (int blk = 0; blk < 4; blk++) {
+        float* dst = ds0 + ((size_t)seq * H + h) * state_elems + (size_t)L * D;
+        for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
             uint32_t x[32];
             tmem_ld32(tm_lane + COL_DS + blk * 32, x);
             tmem_ld_wait();
