@@ -24,12 +24,15 @@ namespace harts {
 
 int32_t make_row_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H);
 int32_t make_state_map(CUtensorMap* map, const void* base, int64_t n);
+int32_t make_out_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H);
 
 namespace {
 
 using namespace tc;
 
-constexpr int BT = 64, D = 128, NT = 256;   // 8 warps: warps w and w+4 share tensor-memory lanes 32(w&3)..+31
+constexpr int BT = 64, D = 128;
+constexpr int NT = 512;                       // 16 warps: warp w works on tensor-memory lanes 32(w&3)..+31 and on
+constexpr int NGRP = NT / 128;                //           column group w>>2 (a quarter of every accumulator)
 constexpr int TILE = BT * D * 2;              // 16 KB
 constexpr int PANEL = BT * 128;               // 8 KB
 constexpr int S_PANEL = D * 128;              // 16 KB
@@ -42,6 +45,8 @@ struct Smem {
                          dp = 5 * TILE + PANEL, s = 5 * TILE + 2 * PANEL, ds = s + 2 * S_PANEL,
                          misc = ds + 2 * S_PANEL;
     static constexpr int bytes = misc + 4096;
+    // after a chunk's MMAs are done these operand tiles are dead and stage the outputs for the TMA stores
+    static constexpr int stage_dq = dOs, stage_dk = p, stage_dv = ds;
 };
 struct Misc {
     float part[BT];
@@ -49,8 +54,8 @@ struct Misc {
     float eb[BT];
     float w[BT];
     int code[BT];
-    float red[8][32];     // per-warp partial sums of q.dq - k.dk (warp w covers rows 32(w>>2)..+31)
-    float gred[8];
+    float red[NT / 32][16];   // per-warp partial sums of q.dq - k.dk (warp w covers rows 16(w>>2)..+15)
+    float gred[NT / 32];
     float gamma;
     uint32_t tmem;
     uint64_t bar_vds, bar_qk, bar_a, bar_o;
@@ -74,14 +79,10 @@ __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq
     return s;
 }
 
-__device__ __forceinline__ float bf16_at(const unsigned char* tile, int row, int col) {
-    return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(tile + (col >> 6) * PANEL + sw128(row, col & 63)));
-}
-
-// Sum over the 32 lanes of a warp for each of 32 per-lane values; lane l returns the total of z[l].
-__device__ __forceinline__ float warp_transpose_reduce(float (&z)[32], int lane) {
+// Sum over the 32 lanes of a warp for each of 16 per-lane values; lane l returns the total of z[l & 15].
+__device__ __forceinline__ float warp_transpose_reduce16(float (&z)[16], int lane) {
 #pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) {
+    for (int s = 8; s >= 1; s >>= 1) {
         const bool upper = (lane & s) != 0;
 #pragma unroll
         for (int i = 0; i < s; i++) {
@@ -90,18 +91,89 @@ __device__ __forceinline__ float warp_transpose_reduce(float (&z)[32], int lane)
             z[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
         }
     }
-    return z[0];
+    return z[0] + __shfl_xor_sync(0xffffffffu, z[0], 16);
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(unsigned short b) { return __uint_as_float((uint32_t)b << 16); }
+
+// Epilogue of one chunk for this thread's feature index L and its 16 rows.  FULL: all 64 rows are own rows, so
+// the outputs are staged in shared memory ([row][feature], plain layout) for one TMA store per tensor; otherwise
+// every row is checked and written on its own (own rows to the outputs, replayed rows to the scratch area).
+template <bool FULL>
+__device__ __forceinline__ void epilogue(const Misc& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int lane,
+                                         int H, int h, int replay_base, __nv_bfloat16* dq, __nv_bfloat16* dk_,
+                                         __nv_bfloat16* dv_, float* rk, float* rv, float& g_part, float& row_total) {
+    const unsigned char* sQ = smem + Smem::q;
+    const unsigned char* sK = smem + Smem::k;
+    const int t0 = grp * 16;
+    const uint32_t qk_base = (L >> 6) * PANEL + (L & 7) * 2;
+    const uint32_t cL = (L & 63) >> 3;
+    float z[16];
+    {
+        uint32_t xq[16], xi[16], xe[16];
+        tmem_ld16(tm_lane + COL_DQ + t0, xq);
+        tmem_ld16(tm_lane + COL_DK + t0, xi);
+        tmem_ld16(tm_lane + COL_A + t0, xe);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 16; e++) {
+            const int t = t0 + e;
+            const uint32_t off = qk_base + t * 128 + ((cL ^ (uint32_t)(t & 7)) << 4);
+            const float qv = bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(sQ + off));
+            const float kv = bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(sK + off));
+            const float dqv = __uint_as_float(xq[e]);
+            const float inter = m.w[t] * __uint_as_float(xe[e]);
+            const float dkv = __uint_as_float(xi[e]) + inter;
+            if (FULL) {
+                z[e] = qv * dqv - kv * dkv;
+                g_part += kv * inter;
+                *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dq + t * 256 + L * 2) = __float2bfloat16_rn(dqv);
+                *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dk + t * 256 + L * 2) = __float2bfloat16_rn(dkv);
+            } else {
+                const int code = m.code[t];
+                z[e] = code == -1 ? 0.f : qv * dqv - kv * dkv;
+                if (code != -1) g_part += kv * inter;
+                if (code >= 0) {
+                    size_t o_ = ((size_t)code * H + h) * D + L;
+                    dq[o_] = __float2bfloat16_rn(dqv);
+                    dk_[o_] = __float2bfloat16_rn(dkv);
+                } else if (code < -1) {
+                    rk[((size_t)(replay_base + t) * H + h) * D + L] = dkv;     // replayed rows sit in chunk 0
+                }
+            }
+        }
+    }
+    row_total = warp_transpose_reduce16(z, lane);
+    {
+        uint32_t xi[16], xe[16];
+        tmem_ld16(tm_lane + COL_DV + t0, xi);
+        tmem_ld16(tm_lane + COL_DA + t0, xe);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 16; e++) {
+            const int t = t0 + e;
+            const float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
+            if (FULL) {
+                *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dv + t * 256 + L * 2) = __float2bfloat16_rn(dvv);
+            } else {
+                const int code = m.code[t];
+                if (code >= 0) dv_[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dvv);
+                else if (code < -1) rv[((size_t)(replay_base + t) * H + h) * D + L] = dvv;
+            }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(NT, 1)
 tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_constant__ CUtensorMap map_q,
               const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_cs,
-              const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
-              const __nv_bfloat16* __restrict__ v, const float* __restrict__ g, const __nv_bfloat16* __restrict__ dO,
-              __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk_, __nv_bfloat16* __restrict__ dv_,
-              float* __restrict__ dg, float* __restrict__ ds0, float* __restrict__ rk, float* __restrict__ rv,
-              float* __restrict__ rg, int* status) {
+              const __grid_constant__ CUtensorMap map_dq, const __grid_constant__ CUtensorMap map_dk,
+              const __grid_constant__ CUtensorMap map_dv, const __nv_bfloat16* __restrict__ q,
+              const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
+              const __nv_bfloat16* __restrict__ dO, __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk_,
+              __nv_bfloat16* __restrict__ dv_, float* __restrict__ dg, float* __restrict__ ds0, float* __restrict__ rk,
+              float* __restrict__ rv, float* __restrict__ rg, int* status) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     unsigned char* sQ = smem + Smem::q;
@@ -116,7 +188,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int grp = warp >> 2;                    // which half of the columns this warp works on
+    const int grp = warp >> 2;                    // column group
     const int L = (warp & 3) * 32 + lane;         // tensor-memory lane = feature index (or row t) of this thread
     const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
     const SeqInfo s = seq_info(tb, seq);
@@ -140,7 +212,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         uint32_t zero[32];
 #pragma unroll
         for (int i = 0; i < 32; i++) zero[i] = 0u;
-        for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) tmem_st32(tm_lane + COL_DS + blk * 32, zero);
+        tmem_st32(tm_lane + COL_DS + grp * 32, zero);
         tmem_st_wait();
     }
 
@@ -198,6 +270,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
 
     for (int c = s.n_chunks - 1; c >= 0; c--) {
         const bool gathered = c == 0 && gather_first;
+        // all 64 rows are own rows: outputs leave through staged TMA stores
+        const bool full = !gathered && (c + 1) * BT <= s.n_virtual;
         tc_fence_before();
         __syncthreads();                          // (1) the previous chunk's epilogue is over everywhere
         tc_fence_after();
@@ -251,8 +325,9 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             tc_fence_after();
             for (int ks = 0; ks < 8; ks++)
                 mma_ss(tmem + COL_DA, desc_kmajor<BT>(aDO, ks), desc_kmajor<BT>(aV, ks), I_KK64, ks > 0);
+            tma_store_wait_read();                // the previous chunk's output stores have left their staging tiles
         }
-        __syncthreads();                          // (3) b2 / eb / w / gamma visible
+        __syncthreads();                          // (3) b2 / eb / w / gamma visible; staging tiles reusable
         // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma ---------------------
         float g_part = 0.f;                       // this thread's share of <S_{c+1}, dS_{c+1}>
         {
@@ -261,44 +336,47 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             const int cons_hi = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
             const float gamma = m.gamma;
             float dot = 0.f;
-            for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
-                uint32_t x[32];
-                tmem_ld32(tm_lane + COL_DS + blk * 32, x);
-                tmem_ld_wait();
-                for (int u = cons_lo; u < cons_hi; u++) {
-                    const float4* src = reinterpret_cast<const float4*>(
-                        ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + (size_t)L * D + blk * 32);
+            const int blk = grp;
+            uint32_t x[32];
+            tmem_ld32(tm_lane + COL_DS + blk * 32, x);
+            tmem_ld_wait();
+            for (int u = cons_lo; u < cons_hi; u++) {
+                const float4* src = reinterpret_cast<const float4*>(
+                    ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + (size_t)L * D + blk * 32);
 #pragma unroll
-                    for (int i4 = 0; i4 < 8; i4++) {
-                        float4 a = src[i4];
-                        x[i4 * 4 + 0] = __float_as_uint(__uint_as_float(x[i4 * 4 + 0]) + a.x);
-                        x[i4 * 4 + 1] = __float_as_uint(__uint_as_float(x[i4 * 4 + 1]) + a.y);
-                        x[i4 * 4 + 2] = __float_as_uint(__uint_as_float(x[i4 * 4 + 2]) + a.z);
-                        x[i4 * 4 + 3] = __float_as_uint(__uint_as_float(x[i4 * 4 + 3]) + a.w);
-                    }
+                for (int i4 = 0; i4 < 8; i4++) {
+                    float4 a = src[i4];
+                    x[i4 * 4 + 0] = __float_as_uint(__uint_as_float(x[i4 * 4 + 0]) + a.x);
+                    x[i4 * 4 + 1] = __float_as_uint(__uint_as_float(x[i4 * 4 + 1]) + a.y);
+                    x[i4 * 4 + 2] = __float_as_uint(__uint_as_float(x[i4 * 4 + 2]) + a.z);
+                    x[i4 * 4 + 3] = __float_as_uint(__uint_as_float(x[i4 * 4 + 3]) + a.w);
                 }
+            }
 #pragma unroll
-                for (int v4 = 0; v4 < 4; v4++) {
-                    uint4 pk;
-                    pk.x = pack_bf16(__uint_as_float(x[v4 * 8 + 0]), __uint_as_float(x[v4 * 8 + 1]));
-                    pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
-                    pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
-                    pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
-                    int col = blk * 32 + v4 * 8;
-                    *reinterpret_cast<uint4*>(sDS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3)) = pk;
-                }
-                // S_c[i][j'] sits at row j', column i of the state tile (i = L)
+            for (int v4 = 0; v4 < 4; v4++) {
+                uint4 pk;
+                pk.x = pack_bf16(__uint_as_float(x[v4 * 8 + 0]), __uint_as_float(x[v4 * 8 + 1]));
+                pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
+                pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
+                pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
+                int col = blk * 32 + v4 * 8;
+                *reinterpret_cast<uint4*>(sDS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3)) = pk;
+            }
+            // S_c[i][j'] sits at row j', column i of the state tile (i = L)
+            {
+                const unsigned char* sbase = sS + (L >> 6) * S_PANEL + (L & 7) * 2;
+                const uint32_t cL = (L & 63) >> 3;
 #pragma unroll
                 for (int e = 0; e < 32; e++) {
-                    int jp = blk * 32 + e;
-                    float sv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(
-                        sS + (L >> 6) * S_PANEL + sw128(jp, L & 63)));
+                    const int jp = blk * 32 + e;
+                    float sv = bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(
+                        sbase + jp * 128 + ((cL ^ (uint32_t)(e & 7)) << 4)));
                     dot += sv * __uint_as_float(x[e]);
                 }
-#pragma unroll
-                for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
-                tmem_st32(tm_lane + COL_DS + blk * 32, x);
             }
+#pragma unroll
+            for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
+            tmem_st32(tm_lane + COL_DS + blk * 32, x);
             tmem_st_wait();
             if (boundary) next_req--;
             g_part = gamma * dot;
@@ -314,7 +392,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 mma_ss(tmem + COL_A, desc_kmajor<BT>(aQ, ks), desc_kmajor<BT>(aK, ks), I_KK64, ks > 0);
             mma_commit(&m.bar_a);
         }
-        // ---- P, dP (lanes 0..63 of both column groups) | dO~ = e^{b_t} dO (the other four warps) ----------------------
+        // ---- P, dP (lanes 0..63 of the four column groups) | dO~ = e^{b_t} dO (the other eight warps) ------------------
         mbar_wait(&m.bar_a, ph_a, status);
         ph_a ^= 1;
         tc_fence_after();
@@ -322,31 +400,28 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             const int t = L;
             const float bt = m.b2[t];
             const bool live = m.code[t] >= 0;     // replay rows and rows past the end have no dO and no q
-            {
-                const int half = grp;
-                uint32_t xa[32], xd[32];
-                tmem_ld32(tm_lane + COL_A + half * 32, xa);
-                tmem_ld32(tm_lane + COL_DA + half * 32, xd);
-                tmem_ld_wait();
+            uint32_t xa[16], xd[16];
+            tmem_ld16(tm_lane + COL_A + grp * 16, xa);
+            tmem_ld16(tm_lane + COL_DA + grp * 16, xd);
+            tmem_ld_wait();
 #pragma unroll
-                for (int v4 = 0; v4 < 4; v4++) {
-                    float ya[8], yd[8];
+            for (int v4 = 0; v4 < 2; v4++) {
+                float ya[8], yd[8];
 #pragma unroll
-                    for (int e = 0; e < 8; e++) {
-                        int j = half * 32 + v4 * 8 + e;
-                        float dec = (live && j <= t) ? ex2(bt - m.b2[j]) : 0.f;
-                        ya[e] = dec != 0.f ? __uint_as_float(xa[v4 * 8 + e]) * dec : 0.f;
-                        yd[e] = dec != 0.f ? __uint_as_float(xd[v4 * 8 + e]) * dec : 0.f;
-                    }
-                    uint32_t off = sw128_chunk(t, half * 4 + v4);
-                    *reinterpret_cast<uint4*>(sP + off) = make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]),
-                                                                     pack_bf16(ya[4], ya[5]), pack_bf16(ya[6], ya[7]));
-                    *reinterpret_cast<uint4*>(sDP + off) = make_uint4(pack_bf16(yd[0], yd[1]), pack_bf16(yd[2], yd[3]),
-                                                                      pack_bf16(yd[4], yd[5]), pack_bf16(yd[6], yd[7]));
+                for (int e = 0; e < 8; e++) {
+                    int j = grp * 16 + v4 * 8 + e;
+                    float dec = (live && j <= t) ? ex2(bt - m.b2[j]) : 0.f;
+                    ya[e] = dec != 0.f ? __uint_as_float(xa[v4 * 8 + e]) * dec : 0.f;
+                    yd[e] = dec != 0.f ? __uint_as_float(xd[v4 * 8 + e]) * dec : 0.f;
                 }
+                uint32_t off = sw128_chunk(t, grp * 2 + v4);
+                *reinterpret_cast<uint4*>(sP + off) = make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]),
+                                                                 pack_bf16(ya[4], ya[5]), pack_bf16(ya[6], ya[7]));
+                *reinterpret_cast<uint4*>(sDP + off) = make_uint4(pack_bf16(yd[0], yd[1]), pack_bf16(yd[2], yd[3]),
+                                                                  pack_bf16(yd[4], yd[5]), pack_bf16(yd[6], yd[7]));
             }
         } else {
-            for (int e = ((warp & 3) - 2) * 32 + lane + 64 * grp; e < BT * 16; e += 128) {
+            for (int e = ((warp & 3) - 2) * 32 + lane + 64 * grp; e < BT * 16; e += 64 * NGRP) {
                 uint32_t off = e * 16;
                 float sc = m.eb[(off % PANEL) >> 7];
                 uint4 raw = *reinterpret_cast<const uint4*>(sDO + off);
@@ -390,60 +465,33 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         const bool next_tiles = !(c - 1 == 0 && gather_first);
         if (tid == 0 && c > 0) issue_vds(c - 1, next_tiles);
         row_code(c - 1, my_code, gval);           // next chunk's rows and g, in flight during the epilogue
-        // ---- epilogue (lane = feature index) -------------------------------------------------------------------------
-        {
-            const int half = grp;
-            float z[32];
-            {
-                uint32_t xq[32], xi[32], xe[32];
-                tmem_ld32(tm_lane + COL_DQ + half * 32, xq);
-                tmem_ld32(tm_lane + COL_DK + half * 32, xi);
-                tmem_ld32(tm_lane + COL_A + half * 32, xe);
-                tmem_ld_wait();
-#pragma unroll
-                for (int e = 0; e < 32; e++) {
-                    int t = half * 32 + e, code = m.code[t];
-                    float dqv = __uint_as_float(xq[e]);
-                    float inter = m.w[t] * __uint_as_float(xe[e]);
-                    float dkv = __uint_as_float(xi[e]) + inter;
-                    float qv = bf16_at(sQ, t, L), kv = bf16_at(sK, t, L);
-                    z[e] = code == -1 ? 0.f : qv * dqv - kv * dkv;
-                    if (code != -1) g_part += kv * inter;
-                    if (code >= 0) {
-                        size_t off = ((size_t)code * H + h) * D + L;
-                        dq[off] = __float2bfloat16_rn(dqv);
-                        dk_[off] = __float2bfloat16_rn(dkv);
-                    } else if (code < -1) {
-                        rk[((size_t)(s.replay_base + t) * H + h) * D + L] = dkv;    // replay rows sit in chunk 0
-                    }
-                }
-            }
-            float tot = warp_transpose_reduce(z, lane);
-            m.red[warp][lane] = tot;
-            {
-                uint32_t xi[32], xe[32];
-                tmem_ld32(tm_lane + COL_DV + half * 32, xi);
-                tmem_ld32(tm_lane + COL_DA + half * 32, xe);
-                tmem_ld_wait();
-#pragma unroll
-                for (int e = 0; e < 32; e++) {
-                    int t = half * 32 + e, code = m.code[t];
-                    float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
-                    if (code >= 0) dv_[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dvv);
-                    else if (code < -1) rv[((size_t)(s.replay_base + t) * H + h) * D + L] = dvv;
-                }
-            }
-        }
-        // <S_{c+1}, dS_{c+1}> over the block
+        // ---- epilogue (lane = feature index, 16 rows per column group) ---------------------------------------------------
+        float row_total;
+        if (full)
+            epilogue<true>(m, smem, tm_lane, grp, L, lane, H, h, s.replay_base, dq, dk_, dv_, rk, rv, g_part, row_total);
+        else
+            epilogue<false>(m, smem, tm_lane, grp, L, lane, H, h, s.replay_base, dq, dk_, dv_, rk, rv, g_part, row_total);
+        if (lane < 16) m.red[warp][lane] = row_total;
 #pragma unroll
         for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
         if (lane == 0) m.gred[warp] = g_part;
+        if (full) fence_async_smem();
         tc_fence_before();
-        __syncthreads();                          // (5) tiles are no longer read; partial sums visible
-        if (tid == 0 && c > 0 && next_tiles) issue_qk(c - 1);
+        __syncthreads();                          // (5) tiles are no longer read; staged outputs and partial sums visible
+        if (tid == 0) {
+            if (full) {
+                int row0 = s.own_begin - s.n_replay + c * BT;
+                tma_store_3d(&map_dq, smem + Smem::stage_dq, 0, h, row0);
+                tma_store_3d(&map_dk, smem + Smem::stage_dk, 0, h, row0);
+                tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
+                tma_store_commit();
+            }
+            if (c > 0 && next_tiles) issue_qk(c - 1);
+        }
         if (tid < BT) {
-            const int g4 = (tid >> 5) * 4;
-            float r = m.red[g4][lane] + m.red[g4 + 1][lane] + m.red[g4 + 2][lane] + m.red[g4 + 3][lane];
+            const int g4 = (tid >> 4) * 4;
+            const int e = tid & 15;
+            float r = m.red[g4][e] + m.red[g4 + 1][e] + m.red[g4 + 2][e] + m.red[g4 + 3][e];
             // inclusive suffix sum over the 64 rows (two warps)
             float x = r;
 #pragma unroll
@@ -455,7 +503,9 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         }
         __syncthreads();                          // (6)
         if (tid < BT) {
-            float G = m.gred[0] + m.gred[1] + m.gred[2] + m.gred[3] + m.gred[4] + m.gred[5] + m.gred[6] + m.gred[7];
+            float G = 0.f;
+#pragma unroll
+            for (int w_ = 0; w_ < NT / 32; w_++) G += m.gred[w_];
             float val = m.part[tid] + (tid < 32 ? m.part[32] : 0.f) + G;
             int code = m.code[tid];
             if (code >= 0) dg[(size_t)code * H + h] = val;
@@ -468,17 +518,16 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     tc_fence_after();
     if (s.init_slot >= 0) {
         float* dst = ds0 + ((size_t)seq * H + h) * state_elems + (size_t)L * D;
-        for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
-            uint32_t x[32];
-            tmem_ld32(tm_lane + COL_DS + blk * 32, x);
-            tmem_ld_wait();
+        uint32_t x[32];
+        tmem_ld32(tm_lane + COL_DS + grp * 32, x);
+        tmem_ld_wait();
 #pragma unroll
-            for (int i4 = 0; i4 < 8; i4++)
-                reinterpret_cast<float4*>(dst + blk * 32)[i4] =
-                    make_float4(__uint_as_float(x[i4 * 4]), __uint_as_float(x[i4 * 4 + 1]),
-                                __uint_as_float(x[i4 * 4 + 2]), __uint_as_float(x[i4 * 4 + 3]));
-        }
+        for (int i4 = 0; i4 < 8; i4++)
+            reinterpret_cast<float4*>(dst + grp * 32)[i4] =
+                make_float4(__uint_as_float(x[i4 * 4]), __uint_as_float(x[i4 * 4 + 1]), __uint_as_float(x[i4 * 4 + 2]),
+                            __uint_as_float(x[i4 * 4 + 3]));
     }
+    if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc<TMEM_COLS>(tmem);
@@ -488,13 +537,16 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
 
 int32_t tc_bwd(const BwdArgs& a) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
-    CUtensorMap mq, mk, mv, mdo, mcs;
+    CUtensorMap mq, mk, mv, mdo, mcs, mdq, mdk, mdv;
     int32_t rc;
     if ((rc = make_row_map(&mq, a.q, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mk, a.k, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mv, a.v, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mdo, a.dO, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_state_map(&mcs, a.chunk_states, (int64_t)a.tb.n_chunks * a.H)) != HARTS_OK) return rc;
+    if ((rc = make_out_map(&mdq, a.dq, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_out_map(&mdk, a.dk_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_out_map(&mdv, a.dv_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if (cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
@@ -502,7 +554,7 @@ int32_t tc_bwd(const BwdArgs& a) {
     char* base = static_cast<char*>(a.scratch);
     int n = (a.seq_hi - a.seq_lo) * a.H;
     tc_bwd_kernel<<<n, NT, Smem::bytes + 1024, a.stream>>>(
-        a.tb, a.seq_lo, a.H, mq, mk, mv, mdo, mcs, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
+        a.tb, a.seq_lo, a.H, mq, mk, mv, mdo, mcs, mdq, mdk, mdv, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_,
         (__nv_bfloat16*)a.dv_, a.dg, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
         (float*)(base + sl.rg), a.dev_status);

@@ -355,6 +355,19 @@ int32_t make_state_map(CUtensorMap* map, const void* base, int64_t n) {
     return r == CUDA_SUCCESS ? HARTS_OK : HARTS_ECUDA;
 }
 
+// [rows][H][128] bf16 output tensor, box = 64 rows x 1 head x 128 columns, plain (unswizzled) rows
+int32_t make_out_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return HARTS_ECUDA;
+    cuuint64_t dims[3] = {128, (cuuint64_t)H, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {256, (cuuint64_t)H * 256};
+    cuuint32_t box[3] = {128, 1, 64}, es[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HARTS_OK : HARTS_ECUDA;
+}
+
 int32_t tc_supported(int32_t dtype, int32_t dk, int32_t dv) { return dtype == HARTS_BF16 && dk == 128 && dv == 128; }
 
 int32_t tc_fwd(const FwdArgs& a) {
