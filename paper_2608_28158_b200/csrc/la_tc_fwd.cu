@@ -22,7 +22,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int BT = 64, D = 128, NT = 128;
+constexpr int BT = 64, D = 128;
+constexpr int NT = 256;                       // 8 warps: warp w works on tensor-memory lanes 32(w&3)..+31, column half w>>2
 constexpr int TILE = BT * D * 2;              // 16 KB: two panels of [64][64] bf16
 constexpr int PANEL = BT * 128;               // 8 KB
 constexpr int S_PANEL = D * 128;              // 16 KB: [128][64] bf16
@@ -33,7 +34,8 @@ constexpr int COL_S = 0, COL_A = 128, COL_O1 = 192, TMEM_COLS = 256;
 
 struct Smem {
     static constexpr int q = 0, k = TILE, v = 2 * TILE, p = 3 * TILE, s = 3 * TILE + PANEL,
-                         misc = 3 * TILE + PANEL + 2 * S_PANEL;
+                         stage = 3 * TILE + PANEL + 2 * S_PANEL,       // outputs of a full chunk, [row][feature]
+                         misc = stage + TILE;
     static constexpr int bytes = misc + 2048;
 };
 struct Misc {
@@ -68,7 +70,8 @@ __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq
 __global__ void __launch_bounds__(NT, 2)
 tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_constant__ CUtensorMap map_q,
               const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-              const __grid_constant__ CUtensorMap map_cs, const __nv_bfloat16* __restrict__ q,
+              const __grid_constant__ CUtensorMap map_cs, const __grid_constant__ CUtensorMap map_o,
+              const __nv_bfloat16* __restrict__ q,
               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
               __nv_bfloat16* __restrict__ o, float* __restrict__ slots, int store_states, int* status) {
     extern __shared__ unsigned char smem_raw[];
@@ -78,9 +81,12 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     unsigned char* sV = smem + Smem::v;
     unsigned char* sP = smem + Smem::p;
     unsigned char* sS = smem + Smem::s;
+    unsigned char* sO = smem + Smem::stage;
     Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int grp = warp >> 2;                    // column half
+    const int L = (warp & 3) * 32 + lane;         // tensor-memory lane of this thread
     const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
     const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)D * D;
@@ -96,15 +102,15 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = m.tmem;
-    const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this thread's lane = tid
+    const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
-    // initial state S^T into tensor memory: lane j' = tid, column i
+    // initial state S^T into tensor memory: lane j' = L, column i
     {
         const float* src = s.init_slot < 0 ? nullptr : slots + ((size_t)s.init_slot * H + h) * state_elems;
-        for (int blk = 0; blk < 4; blk++) {
+        for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
             uint32_t x[32];
 #pragma unroll
-            for (int i = 0; i < 32; i++) x[i] = src ? __float_as_uint(src[(size_t)(blk * 32 + i) * D + tid]) : 0u;
+            for (int i = 0; i < 32; i++) x[i] = src ? __float_as_uint(src[(size_t)(blk * 32 + i) * D + L]) : 0u;
             tmem_st32(tm_lane + COL_S + blk * 32, x);
         }
         tmem_st_wait();
@@ -203,13 +209,13 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             const bool export_slot = next_req < s.req_hi && tb.slot_chunk[next_req] == c;
             float* slot_dst = export_slot ? slots + ((size_t)next_req * H + h) * state_elems : nullptr;
             const float gamma = m.gamma;
-            for (int blk = 0; blk < 4; blk++) {
+            for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
                 uint32_t x[32];
                 tmem_ld32(tm_lane + COL_S + blk * 32, x);
                 tmem_ld_wait();
                 if (slot_dst) {
 #pragma unroll
-                    for (int i = 0; i < 32; i++) slot_dst[(size_t)(blk * 32 + i) * D + tid] = __uint_as_float(x[i]);
+                    for (int i = 0; i < 32; i++) slot_dst[(size_t)(blk * 32 + i) * D + L] = __uint_as_float(x[i]);
                 }
 #pragma unroll
                 for (int v4 = 0; v4 < 4; v4++) {
@@ -219,7 +225,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                     pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
                     pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
                     int col = blk * 32 + v4 * 8;           // first of 8 consecutive i
-                    *reinterpret_cast<uint4*>(sS + (col >> 6) * S_PANEL + sw128_chunk(tid, (col & 63) >> 3)) = pk;
+                    *reinterpret_cast<uint4*>(sS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3)) = pk;
                 }
 #pragma unroll
                 for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
@@ -233,10 +239,11 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         mbar_wait(&m.bar_a, ph_a, status);
         ph_a ^= 1;
         tc_fence_after();
-        if (warp < 2) {
-            const int t = tid;
+        if ((warp & 3) < 2) {
+            const int t = L;
             const float bt = m.b2[t];
-            for (int half = 0; half < 2; half++) {
+            {
+                const int half = grp;
                 uint32_t x[32];
                 tmem_ld32(tm_lane + COL_A + half * 32, x);
                 tmem_ld_wait();
@@ -254,7 +261,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 }
             }
         } else {
-            for (int e = tid - 64; e < BT * 16; e += 64) {
+            for (int e = ((warp & 3) - 2) * 32 + lane + 64 * grp; e < BT * 16; e += 128) {
                 uint32_t off = e * 16;
                 float wj = m.w[(off % PANEL) >> 7];
                 uint4 raw = *reinterpret_cast<uint4*>(sK + off);
@@ -291,19 +298,39 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         ph_o ^= 1;
         tc_fence_after();
         if (tid == 0 && c + 1 < s.n_chunks) issue_tma(c + 1);   // tiles are free: every MMA that read them is done
-        // ---- epilogue: o_t = O1 + e^{b_t} O2, lane = output column j' ---------------------------------------
-        for (int half = 0; half < 2; half++) {
+        // ---- epilogue: o_t = O1 + e^{b_t} O2, lane = output column j', 32 rows per column half ---------------
+        const bool full = !(c == 0 && gather_first) && (c + 1) * BT <= s.n_virtual;
+        {
+            const int t0 = grp * 32;
             uint32_t x1[32], x2[32];
-            tmem_ld32(tm_lane + COL_O1 + half * 32, x1);
-            tmem_ld32(tm_lane + COL_A + half * 32, x2);
+            tmem_ld32(tm_lane + COL_O1 + t0, x1);
+            tmem_ld32(tm_lane + COL_A + t0, x2);
             tmem_ld_wait();
+            if (full) {            // all 64 rows are own rows: stage [row][feature] for one TMA store
 #pragma unroll
-            for (int e = 0; e < 32; e++) {
-                int t = half * 32 + e, code = m.code[t];
-                if (code >= 0) {
+                for (int e = 0; e < 32; e++) {
+                    int t = t0 + e;
                     float val = __uint_as_float(x1[e]) + m.eb[t] * __uint_as_float(x2[e]);
-                    o[((size_t)code * H + h) * D + tid] = __float2bfloat16_rn(val);
+                    *reinterpret_cast<__nv_bfloat16*>(sO + t * 256 + L * 2) = __float2bfloat16_rn(val);
                 }
+                fence_async_smem();
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; e++) {
+                    int t = t0 + e, code = m.code[t];
+                    if (code >= 0) {
+                        float val = __uint_as_float(x1[e]) + m.eb[t] * __uint_as_float(x2[e]);
+                        o[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(val);
+                    }
+                }
+            }
+        }
+        if (full) {
+            tc_fence_before();
+            __syncthreads();                      // (5) staged outputs complete
+            if (tid == 0) {
+                tma_store_3d(&map_o, sO, 0, h, s.own_begin - s.n_replay + c * BT);
+                tma_store_commit();
             }
         }
     }
@@ -372,19 +399,20 @@ int32_t tc_supported(int32_t dtype, int32_t dk, int32_t dv) { return dtype == HA
 
 int32_t tc_fwd(const FwdArgs& a) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
-    CUtensorMap mq, mk, mv, mcs;
+    CUtensorMap mq, mk, mv, mcs, mo;
     int32_t rc;
     if ((rc = make_row_map(&mq, a.q, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mk, a.k, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mv, a.v, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     const void* cs = a.chunk_states ? a.chunk_states : a.q;   // a valid address for the (unused) map
     if ((rc = make_state_map(&mcs, cs, a.chunk_states ? (int64_t)a.tb.n_chunks * a.H : 1)) != HARTS_OK) return rc;
+    if ((rc = make_out_map(&mo, a.o, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if (cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
     int n = (a.seq_hi - a.seq_lo) * a.H;
     tc_fwd_kernel<<<n, NT, Smem::bytes + 1024, a.stream>>>(
-        a.tb, a.seq_lo, a.H, mq, mk, mv, mcs, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
+        a.tb, a.seq_lo, a.H, mq, mk, mv, mcs, mo, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (__nv_bfloat16*)a.o, a.slots, a.chunk_states != nullptr, a.dev_status);
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
