@@ -43,6 +43,7 @@ extern "C" {
 #define HARTS_ETIMEOUT (-4)      /* a bounded device-side wait ran out (from harts_la_check) */
 #define HARTS_EINTERNAL (-5)
 #define HARTS_ECUDA (-6)         /* a CUDA runtime/driver call failed */
+#define HARTS_ESCRATCH (-7)      /* the problem needs more scratch than the library's fixed scratch array holds */
 
 #define HARTS_FP32 0
 #define HARTS_BF16 1
@@ -194,6 +195,31 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
                      const void* k, const void* v, const float* g, const void* dO, void* dq, void* dk_,
                      void* dv_, float* dg, const void* chunk_states, void* scratch, int32_t H, int32_t dk,
                      int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream);
+
+/*
+ * (No counterpart in the paper: an addition for a kind of caller, not part of the method.)
+ * Backward of ALL rounds followed by the replay-gradient fold, like harts_la_bwd(plan, blob, 0, ...), but with the
+ * scratch area inside the library instead of in a caller-owned buffer.  It is meant for callers that have no way to
+ * get device memory at the point where they run the backward: code that runs inside a step whose device memory was
+ * handed out in full beforehand (a framework's arena, a fixed-size serving budget), where one more allocation would
+ * either fail or stall the device, and plug-in style callers that are given tensors but no allocator.  This call
+ * allocates nothing -- no cudaMalloc, cudaFree or allocating library routine -- and the caller still passes every
+ * input and output tensor and the chunk-state workspace the forward filled.
+ *   - The scratch is a fixed device array of HARTS_STATIC_SCRATCH_BYTES that every GPU which loads the library
+ *     holds until the process ends.  A problem whose scratch need (harts_la_workspace_bytes) is larger is rejected
+ *     with HARTS_ESCRATCH before anything is launched.
+ *   - The first call on a device looks up the array's device address (one runtime query, result kept per device);
+ *     make that first call with the device current and before any stream capture begins.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left in it.  The backward
+ *     writes every scratch entry before it reads it, so nothing needs clearing; but two calls that overlap on the
+ *     GPU (different streams, or another host thread) race on the array and corrupt each other's gradients.
+ * Arguments, layouts and the other error codes are those of harts_la_bwd.
+ */
+#define HARTS_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+int32_t harts_la_bwd_static(const harts_la_plan_t* plan, const void* dev_blob, const void* q, const void* k,
+                            const void* v, const float* g, const void* dO, void* dq, void* dk_, void* dv_, float* dg,
+                            const void* chunk_states, int32_t H, int32_t dk, int32_t dv, int32_t dtype, uint32_t flags,
+                            int32_t* dev_status, void* stream);
 
 /* Synchronises `stream`, reads the device status word and returns HARTS_OK, HARTS_ETIMEOUT or
  * HARTS_ECUDA.  dev_status must be zeroed by the caller before the first launch. */

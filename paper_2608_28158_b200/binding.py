@@ -60,6 +60,8 @@ def _load():
     lib.harts_la_fwd.argtypes = [vp, vp, i32] + [vp] * 7 + [i32] * 4 + [u32, vp, vp]
     lib.harts_la_bwd.argtypes = [vp, vp, i32] + [vp] * 11 + [i32] * 4 + [u32, vp, vp]
     lib.harts_la_check.argtypes = [vp, vp]
+    lib.harts_la_bwd_static.argtypes = [vp, vp] + [vp] * 10 + [i32] * 4 + [u32, vp, vp]
+    lib.harts_la_bwd_static.restype = i32
     for name in ("harts_la_plan", "harts_la_plan_view", "harts_la_plan_device_bytes", "harts_la_plan_upload",
                  "harts_la_plan_tables", "harts_la_workspace_bytes", "harts_la_fwd_seqs", "harts_la_bwd_seqs",
                  "harts_la_bwd_finish", "harts_la_fwd", "harts_la_bwd", "harts_la_check"):
@@ -183,6 +185,16 @@ def harts_la_bwd(plan, round, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, sc
     _check(lib.harts_la_bwd(plan._h, _ptr(plan.blob), round, _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(dO), _ptr(dq),
                             _ptr(dk_), _ptr(dv_), _ptr(dg), _ptr(chunk_states), _ptr(scratch), H, dk, dv, dt, flags,
                             _ptr(dev_status), _stream(stream)), "harts_la_bwd")
+
+
+def harts_la_bwd_static(plan, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, flags=0, dev_status=None, stream=None):
+    """All backward rounds and the replay fold with the scratch area inside the library (a fixed device array):
+    for callers that cannot provide or allocate a scratch buffer.  Raises HartsError(-7) when the problem needs
+    more scratch than that array holds.  Calls that overlap on the GPU race on the shared array."""
+    H, dk, dv, dt = _dims(q, v)
+    _check(lib.harts_la_bwd_static(plan._h, _ptr(plan.blob), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(dO), _ptr(dq),
+                                   _ptr(dk_), _ptr(dv_), _ptr(dg), _ptr(chunk_states), H, dk, dv, dt, flags,
+                                   _ptr(dev_status), _stream(stream)), "harts_la_bwd_static")
 
 
 def harts_la_check(dev_status, stream=None):

@@ -39,6 +39,7 @@ const char* harts_la_strerror(int32_t code) {
         case HARTS_ETIMEOUT: return "a bounded device-side wait ran out";
         case HARTS_EINTERNAL: return "internal error";
         case HARTS_ECUDA: return "CUDA call failed";
+        case HARTS_ESCRATCH: return "scratch need exceeds the library's fixed scratch array";
         default: return "unknown status";
     }
 }
