@@ -30,9 +30,15 @@ namespace {
 
 using namespace tc;
 
+#ifdef HARTS_PHASE_CLOCKS
+#define PHASE(i) do { if (tid == 0 && blockIdx.x == 0) { long long now_ = clock64(); atomicAdd((unsigned long long*)(status + 8) + (i), (unsigned long long)(now_ - last_)); last_ = now_; } } while (0)
+#else
+#define PHASE(i) do {} while (0)
+#endif
+
 constexpr int BT = 64, D = 128;
 constexpr int NT = 512;                       // 16 warps: warp w works on tensor-memory lanes 32(w&3)..+31 and on
-constexpr int NGRP = NT / 128;                //           column group w>>2 (a quarter of every accumulator)
+                                              //           column group w>>2 (a quarter of every accumulator)
 constexpr int TILE = BT * D * 2;              // 16 KB
 constexpr int PANEL = BT * 128;               // 8 KB
 constexpr int S_PANEL = D * 128;              // 16 KB
@@ -43,10 +49,9 @@ constexpr int COL_DS = 0, COL_A = 128, COL_DA = 192, COL_DQ = 256, COL_DK = 320,
 struct Smem {
     static constexpr int q = 0, k = TILE, v = 2 * TILE, dO = 3 * TILE, dOs = 4 * TILE, p = 5 * TILE,
                          dp = 5 * TILE + PANEL, s = 5 * TILE + 2 * PANEL, ds = s + 2 * S_PANEL,
-                         misc = ds + 2 * S_PANEL;
+                         stage_dq = ds + 2 * S_PANEL, stage_dk = stage_dq + TILE, stage_dv = stage_dk + TILE,
+                         misc = stage_dv + TILE;       // stage_*: outputs of a full chunk, [row][feature], for TMA stores
     static constexpr int bytes = misc + 4096;
-    // after a chunk's MMAs are done these operand tiles are dead and stage the outputs for the TMA stores
-    static constexpr int stage_dq = dOs, stage_dk = p, stage_dv = ds;
 };
 struct Misc {
     float part[BT];
@@ -58,7 +63,7 @@ struct Misc {
     float gred[NT / 32];
     float gamma;
     uint32_t tmem;
-    uint64_t bar_vds, bar_qk, bar_a, bar_o;
+    uint64_t bar_tiles, bar_a, bar_o, bar_o2, bar_o3;
 };
 
 struct SeqInfo {
@@ -96,70 +101,83 @@ __device__ __forceinline__ float warp_transpose_reduce16(float (&z)[16], int lan
 
 __device__ __forceinline__ float bf16_bits_to_float(unsigned short b) { return __uint_as_float((uint32_t)b << 16); }
 
-// Epilogue of one chunk for this thread's feature index L and its 16 rows.  FULL: all 64 rows are own rows, so
-// the outputs are staged in shared memory ([row][feature], plain layout) for one TMA store per tensor; otherwise
-// every row is checked and written on its own (own rows to the outputs, replayed rows to the scratch area).
+// Epilogue of one chunk for this thread's feature index L and its 16 rows, in three parts that follow the three
+// commits of the MMA batch (dq, dk, dv).  qk[e] holds q[t][L] (low half) and k[t][L] (high half) as bf16 bits, read
+// from the tiles before the batch so that the tiles can be reloaded while the epilogue runs.  FULL: all 64 rows are
+// own rows, so the outputs are staged in shared memory ([row][feature], plain layout) for one TMA store per tensor;
+// otherwise every row is checked and written on its own (own rows to the outputs, replayed rows to the scratch).
 template <bool FULL>
-__device__ __forceinline__ void epilogue(const Misc& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int lane,
-                                         int H, int h, int replay_base, __nv_bfloat16* dq, __nv_bfloat16* dk_,
-                                         __nv_bfloat16* dv_, float* rk, float* rv, float& g_part, float& row_total) {
-    const unsigned char* sQ = smem + Smem::q;
-    const unsigned char* sK = smem + Smem::k;
+__device__ __forceinline__ void epilogue_dq(const Misc& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
+                                            int h, const uint32_t (&qk)[16], __nv_bfloat16* dq, float (&z)[16]) {
     const int t0 = grp * 16;
-    const uint32_t qk_base = (L >> 6) * PANEL + (L & 7) * 2;
-    const uint32_t cL = (L & 63) >> 3;
-    float z[16];
-    {
-        uint32_t xq[16], xi[16], xe[16];
-        tmem_ld16(tm_lane + COL_DQ + t0, xq);
-        tmem_ld16(tm_lane + COL_DK + t0, xi);
-        tmem_ld16(tm_lane + COL_A + t0, xe);
-        tmem_ld_wait();
+    uint32_t xq[16];
+    tmem_ld16(tm_lane + COL_DQ + t0, xq);
+    tmem_ld_wait();
 #pragma unroll
-        for (int e = 0; e < 16; e++) {
-            const int t = t0 + e;
-            const uint32_t off = qk_base + t * 128 + ((cL ^ (uint32_t)(t & 7)) << 4);
-            const float qv = bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(sQ + off));
-            const float kv = bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(sK + off));
-            const float dqv = __uint_as_float(xq[e]);
-            const float inter = m.w[t] * __uint_as_float(xe[e]);
-            const float dkv = __uint_as_float(xi[e]) + inter;
-            if (FULL) {
-                z[e] = qv * dqv - kv * dkv;
-                g_part += kv * inter;
-                *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dq + t * 256 + L * 2) = __float2bfloat16_rn(dqv);
-                *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dk + t * 256 + L * 2) = __float2bfloat16_rn(dkv);
-            } else {
-                const int code = m.code[t];
-                z[e] = code == -1 ? 0.f : qv * dqv - kv * dkv;
-                if (code != -1) g_part += kv * inter;
-                if (code >= 0) {
-                    size_t o_ = ((size_t)code * H + h) * D + L;
-                    dq[o_] = __float2bfloat16_rn(dqv);
-                    dk_[o_] = __float2bfloat16_rn(dkv);
-                } else if (code < -1) {
-                    rk[((size_t)(replay_base + t) * H + h) * D + L] = dkv;     // replayed rows sit in chunk 0
-                }
-            }
+    for (int e = 0; e < 16; e++) {
+        const int t = t0 + e;
+        const float dqv = __uint_as_float(xq[e]);
+        const float qv = __uint_as_float(qk[e] << 16);
+        if (FULL) {
+            z[e] = qv * dqv;
+            *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dq + t * 256 + L * 2) = __float2bfloat16_rn(dqv);
+        } else {
+            const int code = m.code[t];
+            z[e] = code == -1 ? 0.f : qv * dqv;
+            if (code >= 0) dq[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dqv);
         }
     }
-    row_total = warp_transpose_reduce16(z, lane);
-    {
-        uint32_t xi[16], xe[16];
-        tmem_ld16(tm_lane + COL_DV + t0, xi);
-        tmem_ld16(tm_lane + COL_DA + t0, xe);
-        tmem_ld_wait();
+}
+
+template <bool FULL>
+__device__ __forceinline__ void epilogue_dk(const Misc& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
+                                            int h, int replay_base, const uint32_t (&qk)[16], __nv_bfloat16* dk_,
+                                            float* rk, float (&z)[16], float& g_part) {
+    const int t0 = grp * 16;
+    uint32_t xi[16], xe[16];
+    tmem_ld16(tm_lane + COL_DK + t0, xi);
+    tmem_ld16(tm_lane + COL_A + t0, xe);
+    tmem_ld_wait();
 #pragma unroll
-        for (int e = 0; e < 16; e++) {
-            const int t = t0 + e;
-            const float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
-            if (FULL) {
-                *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dv + t * 256 + L * 2) = __float2bfloat16_rn(dvv);
-            } else {
-                const int code = m.code[t];
-                if (code >= 0) dv_[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dvv);
-                else if (code < -1) rv[((size_t)(replay_base + t) * H + h) * D + L] = dvv;
+    for (int e = 0; e < 16; e++) {
+        const int t = t0 + e;
+        const float kv = __uint_as_float(qk[e] & 0xffff0000u);
+        const float inter = m.w[t] * __uint_as_float(xe[e]);
+        const float dkv = __uint_as_float(xi[e]) + inter;
+        if (FULL) {
+            z[e] -= kv * dkv;
+            g_part += kv * inter;
+            *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dk + t * 256 + L * 2) = __float2bfloat16_rn(dkv);
+        } else {
+            const int code = m.code[t];
+            if (code != -1) {
+                z[e] -= kv * dkv;
+                g_part += kv * inter;
             }
+            if (code >= 0) dk_[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dkv);
+            else if (code < -1) rk[((size_t)(replay_base + t) * H + h) * D + L] = dkv;     // replayed rows sit in chunk 0
+        }
+    }
+}
+
+template <bool FULL>
+__device__ __forceinline__ void epilogue_dv(const Misc& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
+                                            int h, int replay_base, __nv_bfloat16* dv_, float* rv) {
+    const int t0 = grp * 16;
+    uint32_t xi[16], xe[16];
+    tmem_ld16(tm_lane + COL_DV + t0, xi);
+    tmem_ld16(tm_lane + COL_DA + t0, xe);
+    tmem_ld_wait();
+#pragma unroll
+    for (int e = 0; e < 16; e++) {
+        const int t = t0 + e;
+        const float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
+        if (FULL) {
+            *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dv + t * 256 + L * 2) = __float2bfloat16_rn(dvv);
+        } else {
+            const int code = m.code[t];
+            if (code >= 0) dv_[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dvv);
+            else if (code < -1) rv[((size_t)(replay_base + t) * H + h) * D + L] = dvv;
         }
     }
 }
@@ -195,10 +213,11 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const size_t state_elems = (size_t)D * D;
 
     if (tid == 0) {
-        mbar_init(&m.bar_vds, 1);
-        mbar_init(&m.bar_qk, 1);
+        mbar_init(&m.bar_tiles, 1);
         mbar_init(&m.bar_a, 1);
         mbar_init(&m.bar_o, 1);
+        mbar_init(&m.bar_o2, 1);
+        mbar_init(&m.bar_o3, 1);
         fence_barrier_init();
     }
     if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
@@ -223,27 +242,29 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     constexpr uint32_t I_MM64 = instr_desc(128, 64, 1, 1);
     constexpr uint32_t I_MM128 = instr_desc(128, 128, 1, 1);
 
-    // v, dO and the start-of-chunk state are free as soon as the chunk's MMAs are done; q and k are still
-    // read by the epilogue, so they travel on a barrier of their own.
-    auto issue_vds = [&](int c, bool tiles) {
+    // loop-invariant operand descriptors (k-step 0); "K" = contraction dimension contiguous, "M" = the other one
+    const uint64_t dQk = desc_kmajor_base(aQ), dKk = desc_kmajor_base(aK), dVk = desc_kmajor_base(aV),
+                   dDOk_hi = desc_kmajor_base(aDO - PANEL),   // rows 64..127 of this operand are the dO tile
+                   dDOsk = desc_kmajor_base(aDOs), dDPk = desc_kmajor_base(aDP), dDSk = desc_kmajor_base(aDS);
+    const uint64_t dQm = desc_mnmajor_base<BT>(aQ), dKm = desc_mnmajor_base<BT>(aK), dDOm = desc_mnmajor_base<BT>(aDO),
+                   dDOsm = desc_mnmajor_base<BT>(aDOs), dPm = desc_mnmajor_base<BT>(aP),
+                   dDPm = desc_mnmajor_base<BT>(aDP), dSm = desc_mnmajor_base<D>(aS), dDSm = desc_mnmajor_base<D>(aDS);
+
+    // All tiles of a chunk travel on one barrier.  They are requested as soon as the previous chunk's MMAs are done
+    // (the epilogue works from registers and tensor memory only), so the loads overlap the epilogue.
+    auto issue_tiles = [&](int c, bool tiles) {
         int row0 = s.own_begin - s.n_replay + c * BT;
         int idx = (s.chunk_base + c) * H + h;
-        mbar_expect_tx(&m.bar_vds, (tiles ? 2 * TILE : 0) + 2 * S_PANEL);
-        tma_load_3d(sS, &map_cs, 0, 0, idx, &m.bar_vds);
-        tma_load_3d(sS + S_PANEL, &map_cs, 64, 0, idx, &m.bar_vds);
+        mbar_expect_tx(&m.bar_tiles, (tiles ? 4 * TILE : 0) + 2 * S_PANEL);
+        tma_load_3d(sS, &map_cs, 0, 0, idx, &m.bar_tiles);
+        tma_load_3d(sS + S_PANEL, &map_cs, 64, 0, idx, &m.bar_tiles);
         if (tiles)
             for (int p = 0; p < 2; p++) {
-                tma_load_3d(sV + p * PANEL, &map_v, p * 64, h, row0, &m.bar_vds);
-                tma_load_3d(sDO + p * PANEL, &map_do, p * 64, h, row0, &m.bar_vds);
+                tma_load_3d(sV + p * PANEL, &map_v, p * 64, h, row0, &m.bar_tiles);
+                tma_load_3d(sDO + p * PANEL, &map_do, p * 64, h, row0, &m.bar_tiles);
+                tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_tiles);
+                tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tiles);
             }
-    };
-    auto issue_qk = [&](int c) {
-        int row0 = s.own_begin - s.n_replay + c * BT;
-        mbar_expect_tx(&m.bar_qk, 2 * TILE);
-        for (int p = 0; p < 2; p++) {
-            tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_qk);
-            tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_qk);
-        }
     };
     auto row_code = [&](int c, int& code, float& gval) {
         code = -1;
@@ -257,21 +278,21 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     };
 
     const bool gather_first = s.n_replay > 0;
-    uint32_t ph_vds = 0, ph_qk = 0, ph_a = 0, ph_o = 0;
+    uint32_t ph_tiles = 0, ph_a = 0, ph_o = 0;
     int next_req = s.req_hi - 1;
-    if (tid == 0) {
-        const bool tiles = !(gather_first && s.n_chunks == 1);
-        issue_vds(s.n_chunks - 1, tiles);
-        if (tiles) issue_qk(s.n_chunks - 1);
-    }
+    if (tid == 0) issue_tiles(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
     int my_code;
     float gval;
     row_code(s.n_chunks - 1, my_code, gval);
 
+#ifdef HARTS_PHASE_CLOCKS
+    long long last_ = clock64();
+#endif
     for (int c = s.n_chunks - 1; c >= 0; c--) {
         const bool gathered = c == 0 && gather_first;
         // all 64 rows are own rows: outputs leave through staged TMA stores
         const bool full = !gathered && (c + 1) * BT <= s.n_virtual;
+        PHASE(0);
         tc_fence_before();
         __syncthreads();                          // (1) the previous chunk's epilogue is over everywhere
         tc_fence_after();
@@ -318,16 +339,23 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             m.w[tid] = ex2((bn - b) * LOG2E);
             if (tid == 0) m.gamma = ex2(bn * LOG2E);
         }
-        mbar_wait(&m.bar_vds, ph_vds, status);
-        ph_vds ^= 1;
-        // ---- dA = dO V^T can start before q and k have landed -----------------------------------------------------
+        PHASE(1);
+        mbar_wait(&m.bar_tiles, ph_tiles, status);
+        ph_tiles ^= 1;
+        PHASE(2);
+        // ---- A = Q K^T on lanes 0..63, dA = dO V^T on lanes 64..127 (rows 0..63 of that operand are unused) ----------
         if (tid == 0) {
             tc_fence_after();
+#pragma unroll
             for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_DA, desc_kmajor<BT>(aDO, ks), desc_kmajor<BT>(aV, ks), I_KK64, ks > 0);
-            tma_store_wait_read();                // the previous chunk's output stores have left their staging tiles
+                mma_ss(tmem + COL_A, dQk + kstep_kmajor<BT>(ks), dKk + kstep_kmajor<BT>(ks), I_KK64, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_DA, dDOk_hi + kstep_kmajor<BT>(ks), dVk + kstep_kmajor<BT>(ks), I_KK64, ks > 0);
+            mma_commit(&m.bar_a);
         }
-        __syncthreads();                          // (3) b2 / eb / w / gamma visible; staging tiles reusable
+        __syncthreads();                          // (3) b2 / eb / w / gamma visible
+        PHASE(3);
         // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma ---------------------
         float g_part = 0.f;                       // this thread's share of <S_{c+1}, dS_{c+1}>
         {
@@ -380,48 +408,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             tmem_st_wait();
             if (boundary) next_req--;
             g_part = gamma * dot;
-            fence_async_smem();
-        }
-        // ---- A = Q K^T once q and k are here ---------------------------------------------------------------------
-        if (!gathered) {
-            mbar_wait(&m.bar_qk, ph_qk, status);
-            ph_qk ^= 1;
-        }
-        if (tid == 0) {
-            for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_A, desc_kmajor<BT>(aQ, ks), desc_kmajor<BT>(aK, ks), I_KK64, ks > 0);
-            mma_commit(&m.bar_a);
-        }
-        // ---- P, dP (lanes 0..63 of the four column groups) | dO~ = e^{b_t} dO (the other eight warps) ------------------
-        mbar_wait(&m.bar_a, ph_a, status);
-        ph_a ^= 1;
-        tc_fence_after();
-        if ((warp & 3) < 2) {
-            const int t = L;
-            const float bt = m.b2[t];
-            const bool live = m.code[t] >= 0;     // replay rows and rows past the end have no dO and no q
-            uint32_t xa[16], xd[16];
-            tmem_ld16(tm_lane + COL_A + grp * 16, xa);
-            tmem_ld16(tm_lane + COL_DA + grp * 16, xd);
-            tmem_ld_wait();
-#pragma unroll
-            for (int v4 = 0; v4 < 2; v4++) {
-                float ya[8], yd[8];
-#pragma unroll
-                for (int e = 0; e < 8; e++) {
-                    int j = grp * 16 + v4 * 8 + e;
-                    float dec = (live && j <= t) ? ex2(bt - m.b2[j]) : 0.f;
-                    ya[e] = dec != 0.f ? __uint_as_float(xa[v4 * 8 + e]) * dec : 0.f;
-                    yd[e] = dec != 0.f ? __uint_as_float(xd[v4 * 8 + e]) * dec : 0.f;
-                }
-                uint32_t off = sw128_chunk(t, grp * 2 + v4);
-                *reinterpret_cast<uint4*>(sP + off) = make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]),
-                                                                 pack_bf16(ya[4], ya[5]), pack_bf16(ya[6], ya[7]));
-                *reinterpret_cast<uint4*>(sDP + off) = make_uint4(pack_bf16(yd[0], yd[1]), pack_bf16(yd[2], yd[3]),
-                                                                  pack_bf16(yd[4], yd[5]), pack_bf16(yd[6], yd[7]));
-            }
-        } else {
-            for (int e = ((warp & 3) - 2) * 32 + lane + 64 * grp; e < BT * 16; e += 64 * NGRP) {
+            // dO~ = e^{b_t} dO (zero on rows without an output): two 16-byte vectors per thread
+            for (int e = tid; e < BT * 16; e += NT) {
                 uint32_t off = e * 16;
                 float sc = m.eb[(off % PANEL) >> 7];
                 uint4 raw = *reinterpret_cast<const uint4*>(sDO + off);
@@ -433,51 +421,119 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 }
                 *reinterpret_cast<uint4*>(sDOs + off) = raw;
             }
+            fence_async_smem();
         }
+        PHASE(4);
+        // ---- P, dP (lanes 0..63 of the four column groups) | dO~ = e^{b_t} dO (the other eight warps) ------------------
+        PHASE(5);
+        mbar_wait(&m.bar_a, ph_a, status);
+        ph_a ^= 1;
+        PHASE(6);
+        tc_fence_after();
+        {
+            // lanes 0..63 hold A (warps with (w&3) < 2), lanes 64..127 hold dA: each thread masks 16 columns of one
+            const bool is_p = (warp & 3) < 2;
+            const int t = L & 63;
+            const float bt = m.b2[t];
+            const bool live = m.code[t] >= 0;     // replay rows and rows past the end have no dO and no q
+            uint32_t xa[16];
+            tmem_ld16(tm_lane + (is_p ? COL_A : COL_DA) + grp * 16, xa);
+            tmem_ld_wait();
+            unsigned char* dst = is_p ? sP : sDP;
+#pragma unroll
+            for (int v4 = 0; v4 < 2; v4++) {
+                float ya[8];
+#pragma unroll
+                for (int e = 0; e < 8; e++) {
+                    int j = grp * 16 + v4 * 8 + e;
+                    float dec = (live && j <= t) ? ex2(bt - m.b2[j]) : 0.f;
+                    ya[e] = dec != 0.f ? __uint_as_float(xa[v4 * 8 + e]) * dec : 0.f;
+                }
+                *reinterpret_cast<uint4*>(dst + sw128_chunk(t, grp * 2 + v4)) =
+                    make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]), pack_bf16(ya[4], ya[5]),
+                               pack_bf16(ya[6], ya[7]));
+            }
+        }
+        // q[t][L], k[t][L] of this thread's 16 rows, for the dg terms of the epilogue
+        uint32_t qk[16];
+        {
+            const uint32_t qk_base = (L >> 6) * PANEL + (L & 7) * 2;
+            const uint32_t cL = (L & 63) >> 3;
+#pragma unroll
+            for (int e = 0; e < 16; e++) {
+                const int t = grp * 16 + e;
+                const uint32_t off = qk_base + t * 128 + ((cL ^ (uint32_t)(t & 7)) << 4);
+                qk[e] = (uint32_t)*reinterpret_cast<const unsigned short*>(sQ + off) |
+                        ((uint32_t)*reinterpret_cast<const unsigned short*>(sK + off) << 16);
+            }
+        }
+        PHASE(7);
+        if (tid == 0) tma_store_wait_read();      // the previous chunk's output stores have left the staging tiles
         fence_async_smem();
         tc_fence_before();
         __syncthreads();                          // (4) all operand tiles and the scaled dS are in place
         tc_fence_after();
+        PHASE(8);
         if (tid == 0) {
             // dq^T = K^T dP^T + S_c dO~^T
+#pragma unroll
             for (int ks = 0; ks < 4; ks++)
-                mma_ss(tmem + COL_DQ, desc_mnmajor<BT>(aK, ks), desc_kmajor<BT>(aDP, ks), I_MK64, ks > 0);
+                mma_ss(tmem + COL_DQ, dKm + kstep_mnmajor(ks), dDPk + kstep_kmajor<BT>(ks), I_MK64, ks > 0);
+#pragma unroll
             for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_DQ, desc_mnmajor<D>(aS, ks), desc_kmajor<BT>(aDOs, ks), I_MK64, true);
-            // dk^T: Q^T dP   |   dS V^T (into the columns A occupied)
-            for (int ks = 0; ks < 4; ks++)
-                mma_ss(tmem + COL_DK, desc_mnmajor<BT>(aQ, ks), desc_mnmajor<BT>(aDP, ks), I_MM64, ks > 0);
-            for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_A, desc_kmajor<D>(aDS, ks), desc_kmajor<BT>(aV, ks), I_KK64, ks > 0);
-            // dv^T: dO^T P   |   dS^T K^T (into the columns dA occupied)
-            for (int ks = 0; ks < 4; ks++)
-                mma_ss(tmem + COL_DV, desc_mnmajor<BT>(aDO, ks), desc_mnmajor<BT>(aP, ks), I_MM64, ks > 0);
-            for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_DA, desc_mnmajor<D>(aDS, ks), desc_kmajor<BT>(aK, ks), I_MK64, ks > 0);
-            // dS += Q^T dO~   (dS was pre-scaled by e^{b_n})
-            for (int ks = 0; ks < 4; ks++)
-                mma_ss(tmem + COL_DS, desc_mnmajor<BT>(aQ, ks), desc_mnmajor<BT>(aDOs, ks), I_MM128, true);
+                mma_ss(tmem + COL_DQ, dSm + kstep_mnmajor(ks), dDOsk + kstep_kmajor<BT>(ks), I_MK64, true);
             mma_commit(&m.bar_o);
+            // dk^T: Q^T dP   |   dS V^T (into the columns A occupied)
+#pragma unroll
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_DK, dQm + kstep_mnmajor(ks), dDPm + kstep_mnmajor(ks), I_MM64, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_A, dDSk + kstep_kmajor<D>(ks), dVk + kstep_kmajor<BT>(ks), I_KK64, ks > 0);
+            mma_commit(&m.bar_o2);
+            // dv^T: dO^T P   |   dS^T K^T (into the columns dA occupied)
+#pragma unroll
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_DV, dDOm + kstep_mnmajor(ks), dPm + kstep_mnmajor(ks), I_MM64, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_DA, dDSm + kstep_mnmajor(ks), dKk + kstep_kmajor<BT>(ks), I_MK64, ks > 0);
+            // dS += Q^T dO~   (dS was pre-scaled by e^{b_n})
+#pragma unroll
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_DS, dQm + kstep_mnmajor(ks), dDOsm + kstep_mnmajor(ks), I_MM128, true);
+            mma_commit(&m.bar_o3);
         }
-        mbar_wait(&m.bar_o, ph_o, status);
-        ph_o ^= 1;
-        tc_fence_after();
-        const bool next_tiles = !(c - 1 == 0 && gather_first);
-        if (tid == 0 && c > 0) issue_vds(c - 1, next_tiles);
+        PHASE(9);
         row_code(c - 1, my_code, gval);           // next chunk's rows and g, in flight during the epilogue
-        // ---- epilogue (lane = feature index, 16 rows per column group) ---------------------------------------------------
-        float row_total;
-        if (full)
-            epilogue<true>(m, smem, tm_lane, grp, L, lane, H, h, s.replay_base, dq, dk_, dv_, rk, rv, g_part, row_total);
-        else
-            epilogue<false>(m, smem, tm_lane, grp, L, lane, H, h, s.replay_base, dq, dk_, dv_, rk, rv, g_part, row_total);
+        const bool next_tiles = !(c - 1 == 0 && gather_first);
+        // ---- epilogue in three parts, each as soon as its accumulators are complete ---------------------------------------
+        float z[16];
+        mbar_wait(&m.bar_o, ph_o, status);
+        tc_fence_after();
+        PHASE(10);
+        if (full) epilogue_dq<true>(m, smem, tm_lane, grp, L, H, h, qk, dq, z);
+        else epilogue_dq<false>(m, smem, tm_lane, grp, L, H, h, qk, dq, z);
+        mbar_wait(&m.bar_o2, ph_o, status);
+        tc_fence_after();
+        if (full) epilogue_dk<true>(m, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
+        else epilogue_dk<false>(m, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
+        const float row_total = warp_transpose_reduce16(z, lane);
+        PHASE(11);
         if (lane < 16) m.red[warp][lane] = row_total;
 #pragma unroll
         for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
         if (lane == 0) m.gred[warp] = g_part;
+        mbar_wait(&m.bar_o3, ph_o, status);
+        ph_o ^= 1;
+        tc_fence_after();
+        if (tid == 0 && c > 0) issue_tiles(c - 1, next_tiles);   // every tile is free: the epilogue does not read them
+        if (full) epilogue_dv<true>(m, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
+        else epilogue_dv<false>(m, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
         if (full) fence_async_smem();
         tc_fence_before();
         __syncthreads();                          // (5) tiles are no longer read; staged outputs and partial sums visible
+        PHASE(12);
         if (tid == 0) {
             if (full) {
                 int row0 = s.own_begin - s.n_replay + c * BT;
@@ -486,31 +542,35 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
                 tma_store_commit();
             }
-            if (c > 0 && next_tiles) issue_qk(c - 1);
         }
         if (tid < BT) {
-            const int g4 = (tid >> 4) * 4;
-            const int e = tid & 15;
-            float r = m.red[g4][e] + m.red[g4 + 1][e] + m.red[g4 + 2][e] + m.red[g4 + 3][e];
-            // inclusive suffix sum over the 64 rows (two warps)
-            float x = r;
+            // dg_t = sum_{tau >= t} r_tau + <S_{c+1}, dS_{c+1}>: suffix scan inside each of the two warps; the first
+            // warp adds the second warp's total, which it sums itself (no second block-wide barrier)
+            auto row_sum = [&](int t) {
+                const int g4 = (t >> 4) * 4, e = t & 15;
+                return m.red[g4][e] + m.red[g4 + 1][e] + m.red[g4 + 2][e] + m.red[g4 + 3][e];
+            };
+            float x = row_sum(tid);
 #pragma unroll
             for (int o_ = 1; o_ < 32; o_ <<= 1) {
                 float y = __shfl_down_sync(0xffffffffu, x, o_);
                 if (lane + o_ < 32) x += y;
             }
-            m.part[tid] = x;
-        }
-        __syncthreads();                          // (6)
-        if (tid < BT) {
+            float upper = 0.f;
+            if (tid < 32) {
+                upper = row_sum(tid + 32);
+#pragma unroll
+                for (int o_ = 16; o_ > 0; o_ >>= 1) upper += __shfl_xor_sync(0xffffffffu, upper, o_);
+            }
             float G = 0.f;
 #pragma unroll
             for (int w_ = 0; w_ < NT / 32; w_++) G += m.gred[w_];
-            float val = m.part[tid] + (tid < 32 ? m.part[32] : 0.f) + G;
+            float val = x + upper + G;
             int code = m.code[tid];
             if (code >= 0) dg[(size_t)code * H + h] = val;
             else if (code < -1) rg[(size_t)(s.replay_base + tid) * H + h] = val;
         }
+        PHASE(13);
     }
     // gradient w.r.t. the initial state: the hand-off into the producing sequence
     tc_fence_before();

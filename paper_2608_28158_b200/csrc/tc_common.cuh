@@ -150,6 +150,17 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t tile, int ks) {
     return smem_desc(tile + ks * 2048, KROWS * 128, 1024);
 }
 
+// The same descriptors split into a loop-invariant base (k-step 0) and a k-step increment of the start-address
+// field, so that the issuing thread only adds a constant per MMA.
+__device__ __forceinline__ uint64_t desc_kmajor_base(uint32_t tile) { return smem_desc(tile, 16, 1024); }
+template <int ROWS>
+__host__ __device__ constexpr uint64_t kstep_kmajor(int ks) {
+    return (uint64_t)(((ks >> 2) * (ROWS * 128) + (ks & 3) * 32) >> 4);
+}
+template <int KROWS>
+__device__ __forceinline__ uint64_t desc_mnmajor_base(uint32_t tile) { return smem_desc(tile, KROWS * 128, 1024); }
+__host__ __device__ constexpr uint64_t kstep_mnmajor(int ks) { return (uint64_t)((ks * 2048) >> 4); }
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
