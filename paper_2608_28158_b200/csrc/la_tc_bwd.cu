@@ -30,15 +30,12 @@ namespace {
 
 using namespace tc;
 
-#ifdef HARTS_PHASE_CLOCKS
-#define PHASE(i) do { if (tid == 0 && blockIdx.x == 0) { long long now_ = clock64(); atomicAdd((unsigned long long*)(status + 8) + (i), (unsigned long long)(now_ - last_)); last_ = now_; } } while (0)
-#else
-#define PHASE(i) do {} while (0)
-#endif
+
 
 constexpr int BT = 64, D = 128;
-constexpr int NT = 512;                       // 16 warps: warp w works on tensor-memory lanes 32(w&3)..+31 and on
-                                              //           column group w>>2 (a quarter of every accumulator)
+constexpr int NC = 512;                       // 16 compute warps: warp w works on tensor-memory lanes 32(w&3)..+31 and
+                                              // on column group w>>2 (a quarter of every accumulator)
+constexpr int NT = NC + 32;                   // plus one warp whose first lane issues every TMA and MMA
 constexpr int TILE = BT * D * 2;              // 16 KB
 constexpr int PANEL = BT * 128;               // 8 KB
 constexpr int S_PANEL = D * 128;              // 16 KB
@@ -53,15 +50,17 @@ struct Smem {
                          misc = stage_dv + TILE;       // stage_*: outputs of a full chunk, [row][feature], for TMA stores
     static constexpr int bytes = misc + 4096;
 };
+struct RowData {             // per-chunk row quantities, double-buffered (the next chunk's are prepared in the tail)
+    float b2[BT];            // running log-decay in log2 units
+    float eb[BT];            // e^{b_t} on rows with an output, 0 elsewhere
+    float w[BT];             // e^{b_n - b_t}
+    int code[BT];            // physical row (>= 0 own), -2 - row (replayed), -1 (past the end)
+    float gamma;             // e^{b_n}
+};
 struct Misc {
-    float part[BT];
-    float b2[BT];
-    float eb[BT];
-    float w[BT];
-    int code[BT];
-    float red[NT / 32][16];   // per-warp partial sums of q.dq - k.dk (warp w covers rows 16(w>>2)..+15)
-    float gred[NT / 32];
-    float gamma;
+    RowData rows[2];
+    float red[NC / 32][16];  // per-warp partial sums of q.dq - k.dk (warp w covers rows 16(w>>2)..+15)
+    float gred[NC / 32];
     uint32_t tmem;
     uint64_t bar_tiles, bar_a, bar_o, bar_o2, bar_o3;
 };
@@ -107,7 +106,7 @@ __device__ __forceinline__ float bf16_bits_to_float(unsigned short b) { return _
 // own rows, so the outputs are staged in shared memory ([row][feature], plain layout) for one TMA store per tensor;
 // otherwise every row is checked and written on its own (own rows to the outputs, replayed rows to the scratch).
 template <bool FULL>
-__device__ __forceinline__ void epilogue_dq(const Misc& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
+__device__ __forceinline__ void epilogue_dq(const RowData& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
                                             int h, const uint32_t (&qk)[16], __nv_bfloat16* dq, float (&z)[16]) {
     const int t0 = grp * 16;
     uint32_t xq[16];
@@ -130,7 +129,7 @@ __device__ __forceinline__ void epilogue_dq(const Misc& m, unsigned char* smem, 
 }
 
 template <bool FULL>
-__device__ __forceinline__ void epilogue_dk(const Misc& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
+__device__ __forceinline__ void epilogue_dk(const RowData& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
                                             int h, int replay_base, const uint32_t (&qk)[16], __nv_bfloat16* dk_,
                                             float* rk, float (&z)[16], float& g_part) {
     const int t0 = grp * 16;
@@ -161,7 +160,7 @@ __device__ __forceinline__ void epilogue_dk(const Misc& m, unsigned char* smem, 
 }
 
 template <bool FULL>
-__device__ __forceinline__ void epilogue_dv(const Misc& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
+__device__ __forceinline__ void epilogue_dv(const RowData& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
                                             int h, int replay_base, __nv_bfloat16* dv_, float* rv) {
     const int t0 = grp * 16;
     uint32_t xi[16], xe[16];
@@ -206,7 +205,9 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int grp = warp >> 2;                    // column group
+    const bool is_compute = warp < NC / 32;
+    const bool is_issuer = tid == NC;              // first lane of the extra warp
+    const int grp = warp >> 2;                    // column group (compute warps)
     const int L = (warp & 3) * 32 + lane;         // tensor-memory lane = feature index (or row t) of this thread
     const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
     const SeqInfo s = seq_info(tb, seq);
@@ -227,7 +228,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const uint32_t tmem = m.tmem;
     const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
-    {   // dS = 0: nothing follows the last chunk
+    if (is_compute) {   // dS = 0: nothing follows the last chunk
         uint32_t zero[32];
 #pragma unroll
         for (int i = 0; i < 32; i++) zero[i] = 0u;
@@ -242,7 +243,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     constexpr uint32_t I_MM64 = instr_desc(128, 64, 1, 1);
     constexpr uint32_t I_MM128 = instr_desc(128, 128, 1, 1);
 
-    // loop-invariant operand descriptors (k-step 0); "K" = contraction dimension contiguous, "M" = the other one
+    // loop-invariant operand descriptors (k-step 0); "k" = contraction dimension contiguous, "m" = the other one
     const uint64_t dQk = desc_kmajor_base(aQ), dKk = desc_kmajor_base(aK), dVk = desc_kmajor_base(aV),
                    dDOk_hi = desc_kmajor_base(aDO - PANEL),   // rows 64..127 of this operand are the dO tile
                    dDOsk = desc_kmajor_base(aDOs), dDPk = desc_kmajor_base(aDP), dDSk = desc_kmajor_base(aDS);
@@ -266,50 +267,67 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tiles);
             }
     };
-    auto row_code = [&](int c, int& code, float& gval) {
-        code = -1;
-        gval = 0.f;
-        int vr = c * BT + tid;
-        if (tid < BT && c >= 0 && vr < s.n_virtual) {
-            int r = vr < s.n_replay ? tb.replay_row[s.replay_base + vr] : s.own_begin + (vr - s.n_replay);
-            code = vr < s.n_replay ? -2 - r : r;
-            gval = g[(size_t)r * H + h];
+    // Row codes and g of chunk c for rows `lane` and `lane + 32` (warp 0 prepares a chunk's row data on its own).
+    auto load_rows = [&](int c, int (&code)[2], float (&gv)[2]) {
+#pragma unroll
+        for (int r = 0; r < 2; r++) {
+            code[r] = -1;
+            gv[r] = 0.f;
+            int vr = c * BT + lane + 32 * r;
+            if (c >= 0 && vr < s.n_virtual) {
+                int row = vr < s.n_replay ? tb.replay_row[s.replay_base + vr] : s.own_begin + (vr - s.n_replay);
+                code[r] = vr < s.n_replay ? -2 - row : row;
+                gv[r] = g[(size_t)row * H + h];
+            }
         }
+    };
+    auto store_rows = [&](RowData& rd, const int (&code)[2], const float (&gv)[2]) {
+        float x0 = gv[0], x1 = gv[1];
+#pragma unroll
+        for (int o_ = 1; o_ < 32; o_ <<= 1) {
+            float y0 = __shfl_up_sync(0xffffffffu, x0, o_), y1 = __shfl_up_sync(0xffffffffu, x1, o_);
+            if (lane >= o_) {
+                x0 += y0;
+                x1 += y1;
+            }
+        }
+        x1 += __shfl_sync(0xffffffffu, x0, 31);
+        const float bn = __shfl_sync(0xffffffffu, x1, 31);
+        const float b[2] = {x0, x1};
+#pragma unroll
+        for (int r = 0; r < 2; r++) {
+            int t = lane + 32 * r;
+            rd.code[t] = code[r];
+            rd.b2[t] = b[r] * LOG2E;
+            rd.eb[t] = code[r] >= 0 ? ex2(b[r] * LOG2E) : 0.f;     // rows without an output carry no dO
+            rd.w[t] = ex2((bn - b[r]) * LOG2E);
+        }
+        if (lane == 0) rd.gamma = ex2(bn * LOG2E);
     };
 
     const bool gather_first = s.n_replay > 0;
     uint32_t ph_tiles = 0, ph_a = 0, ph_o = 0;
     int next_req = s.req_hi - 1;
-    if (tid == 0) issue_tiles(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
-    int my_code;
-    float gval;
-    row_code(s.n_chunks - 1, my_code, gval);
+    if (is_issuer) issue_tiles(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
+    int nx_code[2];
+    float nx_g[2];
+    if (warp == 0) {
+        load_rows(s.n_chunks - 1, nx_code, nx_g);
+        store_rows(m.rows[0], nx_code, nx_g);
+    }
+    int cur = 0;
 
-#ifdef HARTS_PHASE_CLOCKS
-    long long last_ = clock64();
-#endif
-    for (int c = s.n_chunks - 1; c >= 0; c--) {
+    for (int c = s.n_chunks - 1; c >= 0; c--, cur ^= 1) {
         const bool gathered = c == 0 && gather_first;
         // all 64 rows are own rows: outputs leave through staged TMA stores
         const bool full = !gathered && (c + 1) * BT <= s.n_virtual;
-        PHASE(0);
+        const RowData& rd = m.rows[cur];
         tc_fence_before();
-        __syncthreads();                          // (1) the previous chunk's epilogue is over everywhere
+        __syncthreads();                          // (1) row data of this chunk visible; the previous epilogue is over
         tc_fence_after();
-        if (tid < BT) {
-            m.code[tid] = my_code;
-            float x = gval;
-#pragma unroll
-            for (int o_ = 1; o_ < 32; o_ <<= 1) {
-                float y = __shfl_up_sync(0xffffffffu, x, o_);
-                if (lane >= o_) x += y;
-            }
-            m.part[tid] = x;
-        }
         if (gathered) {
-            __syncthreads();
             for (int e = tid; e < BT * 16; e += NT) {
-                int row = e >> 4, ch = e & 15, code = m.code[row];
+                int row = e >> 4, ch = e & 15, code = rd.code[row];
                 uint4 zero = make_uint4(0, 0, 0, 0), kq = zero, vq = zero, qq = zero, dq4 = zero;
                 if (code != -1) {
                     int r = code >= 0 ? code : -2 - code;
@@ -328,23 +346,12 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 *reinterpret_cast<uint4*>(sDO + dst) = dq4;
             }
             fence_async_smem();
+            __syncthreads();
         }
-        __syncthreads();                          // (2)
-        if (tid < BT) {
-            float first_half_total = m.part[31];
-            float b = m.part[tid] + (tid >= 32 ? first_half_total : 0.f);
-            float bn = m.part[63] + first_half_total;
-            m.b2[tid] = b * LOG2E;
-            m.eb[tid] = m.code[tid] >= 0 ? ex2(b * LOG2E) : 0.f;    // rows without an output carry no dO
-            m.w[tid] = ex2((bn - b) * LOG2E);
-            if (tid == 0) m.gamma = ex2(bn * LOG2E);
-        }
-        PHASE(1);
         mbar_wait(&m.bar_tiles, ph_tiles, status);
         ph_tiles ^= 1;
-        PHASE(2);
         // ---- A = Q K^T on lanes 0..63, dA = dO V^T on lanes 64..127 (rows 0..63 of that operand are unused) ----------
-        if (tid == 0) {
+        if (is_issuer) {
             tc_fence_after();
 #pragma unroll
             for (int ks = 0; ks < 8; ks++)
@@ -353,128 +360,122 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             for (int ks = 0; ks < 8; ks++)
                 mma_ss(tmem + COL_DA, dDOk_hi + kstep_kmajor<BT>(ks), dVk + kstep_kmajor<BT>(ks), I_KK64, ks > 0);
             mma_commit(&m.bar_a);
+            tma_store_wait_read();                // the previous chunk's output stores have left the staging tiles
         }
-        __syncthreads();                          // (3) b2 / eb / w / gamma visible
-        PHASE(3);
-        // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma ---------------------
         float g_part = 0.f;                       // this thread's share of <S_{c+1}, dS_{c+1}>
-        {
-            const bool boundary = next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1;
-            const int cons_lo = boundary ? tb.slot_cons_ptr[next_req] : 0;
-            const int cons_hi = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
-            const float gamma = m.gamma;
-            float dot = 0.f;
-            const int blk = grp;
-            uint32_t x[32];
-            tmem_ld32(tm_lane + COL_DS + blk * 32, x);
-            tmem_ld_wait();
-            for (int u = cons_lo; u < cons_hi; u++) {
-                const float4* src = reinterpret_cast<const float4*>(
-                    ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + (size_t)L * D + blk * 32);
+        uint32_t qk[16];                          // q[t][L] | k[t][L] << 16 of this thread's 16 rows (bf16 bits)
+        if (is_compute) {
+            // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma -----------------
+            {
+                const bool boundary = next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1;
+                const int cons_lo = boundary ? tb.slot_cons_ptr[next_req] : 0;
+                const int cons_hi = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
+                const float gamma = rd.gamma;
+                float dot = 0.f;
+                const int blk = grp;
+                uint32_t x[32];
+                tmem_ld32(tm_lane + COL_DS + blk * 32, x);
+                tmem_ld_wait();
+                for (int u = cons_lo; u < cons_hi; u++) {
+                    const float4* src = reinterpret_cast<const float4*>(
+                        ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + (size_t)L * D + blk * 32);
 #pragma unroll
-                for (int i4 = 0; i4 < 8; i4++) {
-                    float4 a = src[i4];
-                    x[i4 * 4 + 0] = __float_as_uint(__uint_as_float(x[i4 * 4 + 0]) + a.x);
-                    x[i4 * 4 + 1] = __float_as_uint(__uint_as_float(x[i4 * 4 + 1]) + a.y);
-                    x[i4 * 4 + 2] = __float_as_uint(__uint_as_float(x[i4 * 4 + 2]) + a.z);
-                    x[i4 * 4 + 3] = __float_as_uint(__uint_as_float(x[i4 * 4 + 3]) + a.w);
+                    for (int i4 = 0; i4 < 8; i4++) {
+                        float4 a = src[i4];
+                        x[i4 * 4 + 0] = __float_as_uint(__uint_as_float(x[i4 * 4 + 0]) + a.x);
+                        x[i4 * 4 + 1] = __float_as_uint(__uint_as_float(x[i4 * 4 + 1]) + a.y);
+                        x[i4 * 4 + 2] = __float_as_uint(__uint_as_float(x[i4 * 4 + 2]) + a.z);
+                        x[i4 * 4 + 3] = __float_as_uint(__uint_as_float(x[i4 * 4 + 3]) + a.w);
+                    }
+                }
+#pragma unroll
+                for (int v4 = 0; v4 < 4; v4++) {
+                    uint4 pk;
+                    pk.x = pack_bf16(__uint_as_float(x[v4 * 8 + 0]), __uint_as_float(x[v4 * 8 + 1]));
+                    pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
+                    pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
+                    pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
+                    int col = blk * 32 + v4 * 8;
+                    *reinterpret_cast<uint4*>(sDS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3)) = pk;
+                }
+                // S_c[i][j'] sits at row j', column i of the state tile (i = L)
+                {
+                    const unsigned char* sbase = sS + (L >> 6) * S_PANEL + (L & 7) * 2;
+                    const uint32_t cL = (L & 63) >> 3;
+#pragma unroll
+                    for (int e = 0; e < 32; e++) {
+                        const int jp = blk * 32 + e;
+                        float sv = bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(
+                            sbase + jp * 128 + ((cL ^ (uint32_t)(e & 7)) << 4)));
+                        dot += sv * __uint_as_float(x[e]);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
+                tmem_st32(tm_lane + COL_DS + blk * 32, x);
+                tmem_st_wait();
+                if (boundary) next_req--;
+                g_part = gamma * dot;
+                // dO~ = e^{b_t} dO (zero on rows without an output): two 16-byte vectors per thread
+                for (int e = tid; e < BT * 16; e += NC) {
+                    uint32_t off = e * 16;
+                    float sc = rd.eb[(off % PANEL) >> 7];
+                    uint4 raw = *reinterpret_cast<const uint4*>(sDO + off);
+                    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+                    for (int e2 = 0; e2 < 4; e2++) {
+                        float2 f = __bfloat1622float2(h2[e2]);
+                        h2[e2] = sc != 0.f ? __floats2bfloat162_rn(f.x * sc, f.y * sc) : __floats2bfloat162_rn(0.f, 0.f);
+                    }
+                    *reinterpret_cast<uint4*>(sDOs + off) = raw;
                 }
             }
-#pragma unroll
-            for (int v4 = 0; v4 < 4; v4++) {
-                uint4 pk;
-                pk.x = pack_bf16(__uint_as_float(x[v4 * 8 + 0]), __uint_as_float(x[v4 * 8 + 1]));
-                pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
-                pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
-                pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
-                int col = blk * 32 + v4 * 8;
-                *reinterpret_cast<uint4*>(sDS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3)) = pk;
-            }
-            // S_c[i][j'] sits at row j', column i of the state tile (i = L)
+            // ---- P = A .* decay (lanes 0..63), dP = dA .* decay (lanes 64..127): 16 columns of one of them per thread ------
+            mbar_wait(&m.bar_a, ph_a, status);
+            tc_fence_after();
             {
-                const unsigned char* sbase = sS + (L >> 6) * S_PANEL + (L & 7) * 2;
+                const bool is_p = (warp & 3) < 2;
+                const int t = L & 63;
+                const float bt = rd.b2[t];
+                const bool live = rd.code[t] >= 0;    // replay rows and rows past the end have no dO and no q
+                uint32_t xa[16];
+                tmem_ld16(tm_lane + (is_p ? COL_A : COL_DA) + grp * 16, xa);
+                tmem_ld_wait();
+                unsigned char* dst = is_p ? sP : sDP;
+#pragma unroll
+                for (int v4 = 0; v4 < 2; v4++) {
+                    float ya[8];
+#pragma unroll
+                    for (int e = 0; e < 8; e++) {
+                        int j = grp * 16 + v4 * 8 + e;
+                        float dec = (live && j <= t) ? ex2(bt - rd.b2[j]) : 0.f;
+                        ya[e] = dec != 0.f ? __uint_as_float(xa[v4 * 8 + e]) * dec : 0.f;
+                    }
+                    *reinterpret_cast<uint4*>(dst + sw128_chunk(t, grp * 2 + v4)) =
+                        make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]), pack_bf16(ya[4], ya[5]),
+                                   pack_bf16(ya[6], ya[7]));
+                }
+            }
+            // q[t][L], k[t][L] of this thread's 16 rows, for the dg terms of the epilogue
+            {
+                const uint32_t qk_base = (L >> 6) * PANEL + (L & 7) * 2;
                 const uint32_t cL = (L & 63) >> 3;
 #pragma unroll
-                for (int e = 0; e < 32; e++) {
-                    const int jp = blk * 32 + e;
-                    float sv = bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(
-                        sbase + jp * 128 + ((cL ^ (uint32_t)(e & 7)) << 4)));
-                    dot += sv * __uint_as_float(x[e]);
+                for (int e = 0; e < 16; e++) {
+                    const int t = grp * 16 + e;
+                    const uint32_t off = qk_base + t * 128 + ((cL ^ (uint32_t)(t & 7)) << 4);
+                    qk[e] = (uint32_t)*reinterpret_cast<const unsigned short*>(sQ + off) |
+                            ((uint32_t)*reinterpret_cast<const unsigned short*>(sK + off) << 16);
                 }
-            }
-#pragma unroll
-            for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
-            tmem_st32(tm_lane + COL_DS + blk * 32, x);
-            tmem_st_wait();
-            if (boundary) next_req--;
-            g_part = gamma * dot;
-            // dO~ = e^{b_t} dO (zero on rows without an output): two 16-byte vectors per thread
-            for (int e = tid; e < BT * 16; e += NT) {
-                uint32_t off = e * 16;
-                float sc = m.eb[(off % PANEL) >> 7];
-                uint4 raw = *reinterpret_cast<const uint4*>(sDO + off);
-                __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
-#pragma unroll
-                for (int e2 = 0; e2 < 4; e2++) {
-                    float2 f = __bfloat1622float2(h2[e2]);
-                    h2[e2] = sc != 0.f ? __floats2bfloat162_rn(f.x * sc, f.y * sc) : __floats2bfloat162_rn(0.f, 0.f);
-                }
-                *reinterpret_cast<uint4*>(sDOs + off) = raw;
             }
             fence_async_smem();
         }
-        PHASE(4);
-        // ---- P, dP (lanes 0..63 of the four column groups) | dO~ = e^{b_t} dO (the other eight warps) ------------------
-        PHASE(5);
-        mbar_wait(&m.bar_a, ph_a, status);
         ph_a ^= 1;
-        PHASE(6);
-        tc_fence_after();
-        {
-            // lanes 0..63 hold A (warps with (w&3) < 2), lanes 64..127 hold dA: each thread masks 16 columns of one
-            const bool is_p = (warp & 3) < 2;
-            const int t = L & 63;
-            const float bt = m.b2[t];
-            const bool live = m.code[t] >= 0;     // replay rows and rows past the end have no dO and no q
-            uint32_t xa[16];
-            tmem_ld16(tm_lane + (is_p ? COL_A : COL_DA) + grp * 16, xa);
-            tmem_ld_wait();
-            unsigned char* dst = is_p ? sP : sDP;
-#pragma unroll
-            for (int v4 = 0; v4 < 2; v4++) {
-                float ya[8];
-#pragma unroll
-                for (int e = 0; e < 8; e++) {
-                    int j = grp * 16 + v4 * 8 + e;
-                    float dec = (live && j <= t) ? ex2(bt - m.b2[j]) : 0.f;
-                    ya[e] = dec != 0.f ? __uint_as_float(xa[v4 * 8 + e]) * dec : 0.f;
-                }
-                *reinterpret_cast<uint4*>(dst + sw128_chunk(t, grp * 2 + v4)) =
-                    make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]), pack_bf16(ya[4], ya[5]),
-                               pack_bf16(ya[6], ya[7]));
-            }
-        }
-        // q[t][L], k[t][L] of this thread's 16 rows, for the dg terms of the epilogue
-        uint32_t qk[16];
-        {
-            const uint32_t qk_base = (L >> 6) * PANEL + (L & 7) * 2;
-            const uint32_t cL = (L & 63) >> 3;
-#pragma unroll
-            for (int e = 0; e < 16; e++) {
-                const int t = grp * 16 + e;
-                const uint32_t off = qk_base + t * 128 + ((cL ^ (uint32_t)(t & 7)) << 4);
-                qk[e] = (uint32_t)*reinterpret_cast<const unsigned short*>(sQ + off) |
-                        ((uint32_t)*reinterpret_cast<const unsigned short*>(sK + off) << 16);
-            }
-        }
-        PHASE(7);
-        if (tid == 0) tma_store_wait_read();      // the previous chunk's output stores have left the staging tiles
-        fence_async_smem();
         tc_fence_before();
         __syncthreads();                          // (4) all operand tiles and the scaled dS are in place
         tc_fence_after();
-        PHASE(8);
-        if (tid == 0) {
+        const bool next_tiles = !(c - 1 == 0 && gather_first);
+        if (is_issuer) {
             // dq^T = K^T dP^T + S_c dO~^T
 #pragma unroll
             for (int ks = 0; ks < 4; ks++)
@@ -503,49 +504,46 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             for (int ks = 0; ks < 4; ks++)
                 mma_ss(tmem + COL_DS, dQm + kstep_mnmajor(ks), dDOsm + kstep_mnmajor(ks), I_MM128, true);
             mma_commit(&m.bar_o3);
+            // every tile is free once these are done: the epilogue works from registers and tensor memory
+            mbar_wait(&m.bar_o3, ph_o, status);
+            if (c > 0) issue_tiles(c - 1, next_tiles);
         }
-        PHASE(9);
-        row_code(c - 1, my_code, gval);           // next chunk's rows and g, in flight during the epilogue
-        const bool next_tiles = !(c - 1 == 0 && gather_first);
-        // ---- epilogue in three parts, each as soon as its accumulators are complete ---------------------------------------
-        float z[16];
-        mbar_wait(&m.bar_o, ph_o, status);
-        tc_fence_after();
-        PHASE(10);
-        if (full) epilogue_dq<true>(m, smem, tm_lane, grp, L, H, h, qk, dq, z);
-        else epilogue_dq<false>(m, smem, tm_lane, grp, L, H, h, qk, dq, z);
-        mbar_wait(&m.bar_o2, ph_o, status);
-        tc_fence_after();
-        if (full) epilogue_dk<true>(m, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
-        else epilogue_dk<false>(m, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
-        const float row_total = warp_transpose_reduce16(z, lane);
-        PHASE(11);
-        if (lane < 16) m.red[warp][lane] = row_total;
+        if (warp == 0) load_rows(c - 1, nx_code, nx_g);   // next chunk's rows and g, in flight during the epilogue
+        if (is_compute) {
+            // ---- epilogue in three parts, each as soon as its accumulators are complete -------------------------------
+            float z[16];
+            mbar_wait(&m.bar_o, ph_o, status);
+            tc_fence_after();
+            if (full) epilogue_dq<true>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
+            else epilogue_dq<false>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
+            mbar_wait(&m.bar_o2, ph_o, status);
+            tc_fence_after();
+            if (full) epilogue_dk<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
+            else epilogue_dk<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
+            const float row_total = warp_transpose_reduce16(z, lane);
+            if (lane < 16) m.red[warp][lane] = row_total;
 #pragma unroll
-        for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
-        if (lane == 0) m.gred[warp] = g_part;
-        mbar_wait(&m.bar_o3, ph_o, status);
+            for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
+            if (lane == 0) m.gred[warp] = g_part;
+            mbar_wait(&m.bar_o3, ph_o, status);
+            tc_fence_after();
+            if (full) epilogue_dv<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
+            else epilogue_dv<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
+            if (full) fence_async_smem();
+        }
         ph_o ^= 1;
-        tc_fence_after();
-        if (tid == 0 && c > 0) issue_tiles(c - 1, next_tiles);   // every tile is free: the epilogue does not read them
-        if (full) epilogue_dv<true>(m, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
-        else epilogue_dv<false>(m, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
-        if (full) fence_async_smem();
         tc_fence_before();
-        __syncthreads();                          // (5) tiles are no longer read; staged outputs and partial sums visible
-        PHASE(12);
-        if (tid == 0) {
-            if (full) {
-                int row0 = s.own_begin - s.n_replay + c * BT;
-                tma_store_3d(&map_dq, smem + Smem::stage_dq, 0, h, row0);
-                tma_store_3d(&map_dk, smem + Smem::stage_dk, 0, h, row0);
-                tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
-                tma_store_commit();
-            }
+        __syncthreads();                          // (5) staged outputs and partial sums visible
+        if (is_issuer && full) {
+            int row0 = s.own_begin - s.n_replay + c * BT;
+            tma_store_3d(&map_dq, smem + Smem::stage_dq, 0, h, row0);
+            tma_store_3d(&map_dk, smem + Smem::stage_dk, 0, h, row0);
+            tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
+            tma_store_commit();
         }
         if (tid < BT) {
             // dg_t = sum_{tau >= t} r_tau + <S_{c+1}, dS_{c+1}>: suffix scan inside each of the two warps; the first
-            // warp adds the second warp's total, which it sums itself (no second block-wide barrier)
+            // warp adds the second warp's total, which it sums itself (no further block-wide barrier)
             auto row_sum = [&](int t) {
                 const int g4 = (t >> 4) * 4, e = t & 15;
                 return m.red[g4][e] + m.red[g4 + 1][e] + m.red[g4 + 2][e] + m.red[g4 + 3][e];
@@ -564,19 +562,19 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             }
             float G = 0.f;
 #pragma unroll
-            for (int w_ = 0; w_ < NT / 32; w_++) G += m.gred[w_];
+            for (int w_ = 0; w_ < NC / 32; w_++) G += m.gred[w_];
             float val = x + upper + G;
-            int code = m.code[tid];
+            int code = rd.code[tid];
             if (code >= 0) dg[(size_t)code * H + h] = val;
             else if (code < -1) rg[(size_t)(s.replay_base + tid) * H + h] = val;
         }
-        PHASE(13);
+        if (warp == 0 && c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);
     }
     // gradient w.r.t. the initial state: the hand-off into the producing sequence
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (s.init_slot >= 0) {
+    if (is_compute && s.init_slot >= 0) {
         float* dst = ds0 + ((size_t)seq * H + h) * state_elems + (size_t)L * D;
         uint32_t x[32];
         tmem_ld32(tm_lane + COL_DS + grp * 32, x);
@@ -587,7 +585,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 make_float4(__uint_as_float(x[i4 * 4]), __uint_as_float(x[i4 * 4 + 1]), __uint_as_float(x[i4 * 4 + 2]),
                             __uint_as_float(x[i4 * 4 + 3]));
     }
-    if (tid == 0) tma_store_wait_all();
+    if (is_issuer) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc<TMEM_COLS>(tmem);
