@@ -62,7 +62,7 @@ struct Misc {
     float red[NC / 32][16];  // per-warp partial sums of q.dq - k.dk (warp w covers rows 16(w>>2)..+15)
     float gred[NC / 32];
     uint32_t tmem;
-    uint64_t bar_tiles, bar_a, bar_o, bar_o2, bar_o3;
+    uint64_t bar_tiles, bar_a, bar_o, bar_o2, bar_o3, bar_qk_read;
 };
 
 struct SeqInfo {
@@ -219,6 +219,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         mbar_init(&m.bar_o, 1);
         mbar_init(&m.bar_o2, 1);
         mbar_init(&m.bar_o3, 1);
+        mbar_init(&m.bar_qk_read, NC / 32);
         fence_barrier_init();
     }
     if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
@@ -317,14 +318,18 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     }
     int cur = 0;
 
+    tc_fence_before();
+    __syncthreads();                              // row data of the first chunk visible
+    tc_fence_after();
+
+    // Two block-wide barriers per chunk: (A) before the MMA batch, (B) at the end of the epilogue.  After (B) the
+    // compute warps go straight on to the next chunk, while the extra warp sends the staged outputs off and
+    // finishes dg for the chunk just done.
     for (int c = s.n_chunks - 1; c >= 0; c--, cur ^= 1) {
         const bool gathered = c == 0 && gather_first;
         // all 64 rows are own rows: outputs leave through staged TMA stores
         const bool full = !gathered && (c + 1) * BT <= s.n_virtual;
         const RowData& rd = m.rows[cur];
-        tc_fence_before();
-        __syncthreads();                          // (1) row data of this chunk visible; the previous epilogue is over
-        tc_fence_after();
         if (gathered) {
             for (int e = tid; e < BT * 16; e += NT) {
                 int row = e >> 4, ch = e & 15, code = rd.code[row];
@@ -436,12 +441,17 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             {
                 const bool is_p = (warp & 3) < 2;
                 const int t = L & 63;
+                unsigned char* dst = is_p ? sP : sDP;
+                if (grp * 16 > ((warp & 1) * 32 + 31)) {
+                    // this warp's 32 rows x 16 columns lie entirely above the diagonal
+                    *reinterpret_cast<uint4*>(dst + sw128_chunk(t, grp * 2)) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(dst + sw128_chunk(t, grp * 2 + 1)) = make_uint4(0, 0, 0, 0);
+                } else {
                 const float bt = rd.b2[t];
                 const bool live = rd.code[t] >= 0;    // replay rows and rows past the end have no dO and no q
                 uint32_t xa[16];
                 tmem_ld16(tm_lane + (is_p ? COL_A : COL_DA) + grp * 16, xa);
                 tmem_ld_wait();
-                unsigned char* dst = is_p ? sP : sDP;
 #pragma unroll
                 for (int v4 = 0; v4 < 2; v4++) {
                     float ya[8];
@@ -455,24 +465,13 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                         make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]), pack_bf16(ya[4], ya[5]),
                                    pack_bf16(ya[6], ya[7]));
                 }
-            }
-            // q[t][L], k[t][L] of this thread's 16 rows, for the dg terms of the epilogue
-            {
-                const uint32_t qk_base = (L >> 6) * PANEL + (L & 7) * 2;
-                const uint32_t cL = (L & 63) >> 3;
-#pragma unroll
-                for (int e = 0; e < 16; e++) {
-                    const int t = grp * 16 + e;
-                    const uint32_t off = qk_base + t * 128 + ((cL ^ (uint32_t)(t & 7)) << 4);
-                    qk[e] = (uint32_t)*reinterpret_cast<const unsigned short*>(sQ + off) |
-                            ((uint32_t)*reinterpret_cast<const unsigned short*>(sK + off) << 16);
                 }
             }
             fence_async_smem();
         }
         ph_a ^= 1;
         tc_fence_before();
-        __syncthreads();                          // (4) all operand tiles and the scaled dS are in place
+        __syncthreads();                          // (A) all operand tiles and the scaled dS are in place
         tc_fence_after();
         const bool next_tiles = !(c - 1 == 0 && gather_first);
         if (is_issuer) {
@@ -506,10 +505,26 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             mma_commit(&m.bar_o3);
             // every tile is free once these are done: the epilogue works from registers and tensor memory
             mbar_wait(&m.bar_o3, ph_o, status);
+            mbar_wait(&m.bar_qk_read, ph_o, status);      // every compute warp has taken its q and k values
             if (c > 0) issue_tiles(c - 1, next_tiles);
         }
         if (warp == 0) load_rows(c - 1, nx_code, nx_g);   // next chunk's rows and g, in flight during the epilogue
         if (is_compute) {
+            // q[t][L], k[t][L] of this thread's 16 rows, for the dg terms (read while the first MMAs run; after this
+            // the epilogue does not touch the tiles, which are reloaded as soon as the MMAs are done)
+            {
+                const uint32_t qk_base = (L >> 6) * PANEL + (L & 7) * 2;
+                const uint32_t cL = (L & 63) >> 3;
+#pragma unroll
+                for (int e = 0; e < 16; e++) {
+                    const int t = grp * 16 + e;
+                    const uint32_t off = qk_base + t * 128 + ((cL ^ (uint32_t)(t & 7)) << 4);
+                    qk[e] = (uint32_t)*reinterpret_cast<const unsigned short*>(sQ + off) |
+                            ((uint32_t)*reinterpret_cast<const unsigned short*>(sK + off) << 16);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&m.bar_qk_read);
+            }
             // ---- epilogue in three parts, each as soon as its accumulators are complete -------------------------------
             float z[16];
             mbar_wait(&m.bar_o, ph_o, status);
@@ -530,45 +545,46 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             if (full) epilogue_dv<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
             else epilogue_dv<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
             if (full) fence_async_smem();
+            if (warp == 0 && c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);
         }
         ph_o ^= 1;
         tc_fence_before();
-        __syncthreads();                          // (5) staged outputs and partial sums visible
-        if (is_issuer && full) {
-            int row0 = s.own_begin - s.n_replay + c * BT;
-            tma_store_3d(&map_dq, smem + Smem::stage_dq, 0, h, row0);
-            tma_store_3d(&map_dk, smem + Smem::stage_dk, 0, h, row0);
-            tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
-            tma_store_commit();
-        }
-        if (tid < BT) {
-            // dg_t = sum_{tau >= t} r_tau + <S_{c+1}, dS_{c+1}>: suffix scan inside each of the two warps; the first
-            // warp adds the second warp's total, which it sums itself (no further block-wide barrier)
+        __syncthreads();                          // (B) staged outputs, partial sums and the next chunk's row data visible
+        tc_fence_after();
+        if (!is_compute) {
+            if (is_issuer && full) {
+                int row0 = s.own_begin - s.n_replay + c * BT;
+                tma_store_3d(&map_dq, smem + Smem::stage_dq, 0, h, row0);
+                tma_store_3d(&map_dk, smem + Smem::stage_dk, 0, h, row0);
+                tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
+                tma_store_commit();
+            }
+            // dg_t = sum_{tau >= t} r_tau + <S_{c+1}, dS_{c+1}>, rows `lane` and `lane + 32` per thread of this warp
             auto row_sum = [&](int t) {
                 const int g4 = (t >> 4) * 4, e = t & 15;
                 return m.red[g4][e] + m.red[g4 + 1][e] + m.red[g4 + 2][e] + m.red[g4 + 3][e];
             };
-            float x = row_sum(tid);
+            float lo = row_sum(lane), hi = row_sum(lane + 32);
 #pragma unroll
             for (int o_ = 1; o_ < 32; o_ <<= 1) {
-                float y = __shfl_down_sync(0xffffffffu, x, o_);
-                if (lane + o_ < 32) x += y;
+                float y0 = __shfl_down_sync(0xffffffffu, lo, o_), y1 = __shfl_down_sync(0xffffffffu, hi, o_);
+                if (lane + o_ < 32) {
+                    lo += y0;
+                    hi += y1;
+                }
             }
-            float upper = 0.f;
-            if (tid < 32) {
-                upper = row_sum(tid + 32);
+            float G = __shfl_sync(0xffffffffu, hi, 0);     // total of rows 32..63
+            float Gs = 0.f;
 #pragma unroll
-                for (int o_ = 16; o_ > 0; o_ >>= 1) upper += __shfl_xor_sync(0xffffffffu, upper, o_);
+            for (int w_ = 0; w_ < NC / 32; w_++) Gs += m.gred[w_];
+            const float val[2] = {lo + G + Gs, hi + Gs};
+#pragma unroll
+            for (int r = 0; r < 2; r++) {
+                int t = lane + 32 * r, code = rd.code[t];
+                if (code >= 0) dg[(size_t)code * H + h] = val[r];
+                else if (code < -1) rg[(size_t)(s.replay_base + t) * H + h] = val[r];
             }
-            float G = 0.f;
-#pragma unroll
-            for (int w_ = 0; w_ < NC / 32; w_++) G += m.gred[w_];
-            float val = x + upper + G;
-            int code = rd.code[tid];
-            if (code >= 0) dg[(size_t)code * H + h] = val;
-            else if (code < -1) rg[(size_t)(s.replay_base + tid) * H + h] = val;
         }
-        if (warp == 0 && c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);
     }
     // gradient w.r.t. the initial state: the hand-off into the producing sequence
     tc_fence_before();

@@ -36,6 +36,9 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* s
         if (mbar_try(bar, parity)) return;
     if (status) atomicExch(status, STATUS_TIMEOUT);
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
