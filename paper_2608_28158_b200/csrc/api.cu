@@ -91,7 +91,7 @@ int32_t harts_la_bwd_seqs(const harts_la_tables_t* tb, int32_t seq_lo, int32_t s
         misaligned(dk_) || misaligned(dv_) || misaligned(dg) || misaligned(chunk_states) || misaligned(scratch))
         return HARTS_EINVAL;
     harts::BwdArgs a{*tb, seq_lo, seq_hi, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, scratch, H, dk, dv, dtype,
-                     flags, dev_status, static_cast<cudaStream_t>(stream), 0};
+                     flags, dev_status, static_cast<cudaStream_t>(stream)};
     if (use_tc(dtype, dk, dv, flags)) return harts::tc_bwd(a);
     return harts::fma_bwd(a);
 }

@@ -38,7 +38,6 @@ struct BwdArgs {
     uint32_t flags;
     int32_t* dev_status;
     cudaStream_t stream;
-    int32_t cs_transposed;   // chunk states stored [dv][dk] (tensor-core forward) instead of [dk][dv]
 };
 
 // Byte offsets inside the backward scratch buffer (each region 256-byte aligned).

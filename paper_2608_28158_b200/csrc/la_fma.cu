@@ -211,7 +211,7 @@ template <typename T, int DK, int DV>
 __global__ void __launch_bounds__(NT) fma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const T* q,
                                                      const T* k, const T* v, const float* g, const T* dO, T* dq,
                                                      T* dk_, T* dv_, float* dg, const T* chunk_states,
-                                                     float* ds0, float* rk, float* rv, float* rg, int cs_transposed) {
+                                                     float* ds0, float* rk, float* rv, float* rg) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* sS = reinterpret_cast<float*>(smem_raw);       // S_c           [DK][DV]
     float* sdS = sS + DK * DV;                            // dS            [DK][DV]
@@ -247,10 +247,7 @@ __global__ void __launch_bounds__(NT) fma_bwd_kernel(harts_la_tables_t tb, int s
         load_chunk<T, DK, DV, true>(tb, s, c, h, H, q, k, v, g, dO, sq, sk, sv, sdo, sb, srow);
         {
             const T* src = chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems;
-            if (cs_transposed)      // states kept as [DV][DK] by the tensor-core forward
-                for (int e = tid; e < DK * DV; e += NT) sS[tix<DV>(e % DK, e / DK)] = to_f(src[e]);
-            else
-                for (int e = tid; e < DK * DV; e += NT) sS[tix<DV>(e / DV, e % DV)] = to_f(src[e]);
+            for (int e = tid; e < DK * DV; e += NT) sS[tix<DV>(e / DV, e % DV)] = to_f(src[e]);
         }
         if (tid < BT) sr[tid] = 0.f;
         // A and dA, decay-masked lower triangles
@@ -469,7 +466,7 @@ int32_t launch_bwd(const BwdArgs& a) {
     kern<<<n, NT, smem, a.stream>>>(a.tb, a.seq_lo, a.H, (const T*)a.q, (const T*)a.k, (const T*)a.v, a.g,
                                     (const T*)a.dO, (T*)a.dq, (T*)a.dk_, (T*)a.dv_, a.dg, (const T*)a.chunk_states,
                                     (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
-                                    (float*)(base + sl.rg), a.cs_transposed);
+                                    (float*)(base + sl.rg));
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 

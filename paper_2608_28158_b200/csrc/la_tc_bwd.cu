@@ -14,7 +14,7 @@
 //     dS  <- e^{b_n} dS + Q^T dO~                            accumulate in tensor memory
 // where dS includes, at an exported boundary, the initial-state gradients of every sequence that
 // started there (read from the scratch area, where those sequences' calls left them).
-// S_c comes from the chunk-state workspace written by the forward ([d_v][d_k] bf16 per chunk-head).
+// S_c comes from the chunk-state workspace written by the forward ([d_k][d_v] bf16 per chunk-head).
 // Gradients of replayed rows go to the scratch area (fp32) and are folded into their ancestor rows by
 // the replay-reduce kernel.  Every wait is bounded.
 #include "kernels.h"
@@ -97,8 +97,6 @@ __device__ __forceinline__ float warp_transpose_reduce16(float (&z)[16], int lan
     }
     return z[0] + __shfl_xor_sync(0xffffffffu, z[0], 16);
 }
-
-__device__ __forceinline__ float bf16_bits_to_float(unsigned short b) { return __uint_as_float((uint32_t)b << 16); }
 
 // Epilogue of one chunk for this thread's feature index L and its 16 rows, in three parts that follow the three
 // commits of the MMA batch (dq, dk, dv).  qk[e] holds q[t][L] (low half) and k[t][L] (high half) as bf16 bits, read
@@ -250,7 +248,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                    dDOsk = desc_kmajor_base(aDOs), dDPk = desc_kmajor_base(aDP), dDSk = desc_kmajor_base(aDS);
     const uint64_t dQm = desc_mnmajor_base<BT>(aQ), dKm = desc_mnmajor_base<BT>(aK), dDOm = desc_mnmajor_base<BT>(aDO),
                    dDOsm = desc_mnmajor_base<BT>(aDOs), dPm = desc_mnmajor_base<BT>(aP),
-                   dDPm = desc_mnmajor_base<BT>(aDP), dSm = desc_mnmajor_base<D>(aS), dDSm = desc_mnmajor_base<D>(aDS);
+                   dDPm = desc_mnmajor_base<BT>(aDP), dDSm = desc_mnmajor_base<D>(aDS);
+    const uint64_t dSk = desc_kmajor_base(aS);
 
     // All tiles of a chunk travel on one barrier.  They are requested as soon as the previous chunk's MMAs are done
     // (the epilogue works from registers and tensor memory only), so the loads overlap the epilogue.
@@ -403,16 +402,16 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                     int col = blk * 32 + v4 * 8;
                     *reinterpret_cast<uint4*>(sDS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3)) = pk;
                 }
-                // S_c[i][j'] sits at row j', column i of the state tile (i = L)
-                {
-                    const unsigned char* sbase = sS + (L >> 6) * S_PANEL + (L & 7) * 2;
-                    const uint32_t cL = (L & 63) >> 3;
+                // <S_c[i][:], dS[i][:]> over this thread's 32 columns: row i = L of the state tile, four 16-byte chunks
 #pragma unroll
-                    for (int e = 0; e < 32; e++) {
-                        const int jp = blk * 32 + e;
-                        float sv = bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(
-                            sbase + jp * 128 + ((cL ^ (uint32_t)(e & 7)) << 4)));
-                        dot += sv * __uint_as_float(x[e]);
+                for (int v4 = 0; v4 < 4; v4++) {
+                    int col = blk * 32 + v4 * 8;
+                    uint4 raw = *reinterpret_cast<const uint4*>(sS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3));
+                    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+                    for (int e2 = 0; e2 < 4; e2++) {
+                        float2 f = __bfloat1622float2(h2[e2]);
+                        dot += f.x * __uint_as_float(x[v4 * 8 + 2 * e2]) + f.y * __uint_as_float(x[v4 * 8 + 2 * e2 + 1]);
                     }
                 }
 #pragma unroll
@@ -481,7 +480,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 mma_ss(tmem + COL_DQ, dKm + kstep_mnmajor(ks), dDPk + kstep_kmajor<BT>(ks), I_MK64, ks > 0);
 #pragma unroll
             for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_DQ, dSm + kstep_mnmajor(ks), dDOsk + kstep_kmajor<BT>(ks), I_MK64, true);
+                mma_ss(tmem + COL_DQ, dSk + kstep_kmajor<D>(ks), dDOsk + kstep_kmajor<BT>(ks), I_KK64, true);
             mma_commit(&m.bar_o);
             // dk^T: Q^T dP   |   dS V^T (into the columns A occupied)
 #pragma unroll

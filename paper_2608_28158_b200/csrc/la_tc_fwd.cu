@@ -1,17 +1,17 @@
 // Tensor-core forward of the packed chunkwise call (Eq. 16) for bf16, d_k = d_v = 128, chunk 64.
 //
 // One CTA per (sequence, head) walks the chunks in order.  The recurrent state lives in tensor
-// memory for the whole walk, TRANSPOSED: lane j' (0..127) holds row j' of S^T, i.e. S[i][j'] for all
-// i in its 128 fp32 columns.  Per chunk (b_t = running sum of g, n = last row, w_j = e^{b_n-b_j}):
+// memory for the whole walk: lane i (0..127) holds row i of S (S[i][j'] for all j' in its 128 fp32
+// columns).  Per chunk (b_t = running sum of g, n = last row, w_j = e^{b_n-b_j}):
 //     A     = Q K^T                      tcgen05, M=128 (rows 64..127 unused) N=64  K=128
 //     P     = A .* e^{b_t-b_j} [j<=t]    registers -> bf16 tile in shared memory
 //     O1^T  = V^T P^T                    tcgen05, M=128 (d_v) N=64 (t) K=64 (j)
-//     O2^T  = S_c^T Q^T                  tcgen05, M=128 N=64 K=128, S_c^T as bf16 tile
+//     O2^T  = S_c^T Q^T                  tcgen05, M=128 N=64 K=128, S_c as bf16 tile [d_k][d_v]
 //     o_t   = O1 + e^{b_t} O2            epilogue, own rows only
-//     S^T   = e^{b_n} S^T + V^T (w .* K) tcgen05 accumulate, M=128 N=128 K=64
+//     S     = e^{b_n} S + (w .* K)^T V   tcgen05 accumulate, M=128 N=128 K=64
 // q/k/v tiles arrive by TMA as 128-byte-swizzled panels; the first chunk of a replay-started
 // sequence is gathered row by row instead (replay rows come from arbitrary ancestor rows).  The
-// start-of-chunk state goes to the chunk-state workspace (bf16, [d_v][d_k] per chunk-head) by TMA
+// start-of-chunk state goes to the chunk-state workspace (bf16, [d_k][d_v] per chunk-head) by TMA
 // store, and to its slot (fp32, [d_k][d_v]) when the plan requests that boundary.
 // Every wait is bounded; a wait that runs out sets the status word and the walk carries on.
 #include "kernels.h"
@@ -104,13 +104,19 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const uint32_t tmem = m.tmem;
     const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
-    // initial state S^T into tensor memory: lane j' = L, column i
+    // initial state into tensor memory: lane i = L holds S[i][:]
     {
-        const float* src = s.init_slot < 0 ? nullptr : slots + ((size_t)s.init_slot * H + h) * state_elems;
+        const float* src = s.init_slot < 0 ? nullptr : slots + ((size_t)s.init_slot * H + h) * state_elems + (size_t)L * D;
         for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
             uint32_t x[32];
 #pragma unroll
-            for (int i = 0; i < 32; i++) x[i] = src ? __float_as_uint(src[(size_t)(blk * 32 + i) * D + L]) : 0u;
+            for (int i4 = 0; i4 < 8; i4++) {
+                float4 a = src ? reinterpret_cast<const float4*>(src + blk * 32)[i4] : make_float4(0.f, 0.f, 0.f, 0.f);
+                x[i4 * 4 + 0] = __float_as_uint(a.x);
+                x[i4 * 4 + 1] = __float_as_uint(a.y);
+                x[i4 * 4 + 2] = __float_as_uint(a.z);
+                x[i4 * 4 + 3] = __float_as_uint(a.w);
+            }
             tmem_st32(tm_lane + COL_S + blk * 32, x);
         }
         tmem_st_wait();
@@ -119,8 +125,8 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV), aP = smem_u32(sP), aS = smem_u32(sS);
     constexpr uint32_t IDESC_A = instr_desc(128, 64, 0, 0);    // Q (K-major) x K (K-major)
     constexpr uint32_t IDESC_O1 = instr_desc(128, 64, 1, 0);   // V^T (MN-major) x P (K-major)
-    constexpr uint32_t IDESC_O2 = instr_desc(128, 64, 0, 0);   // S^T (K-major) x Q (K-major)
-    constexpr uint32_t IDESC_S = instr_desc(128, 128, 1, 1);   // V^T (MN-major) x K~ (MN-major)
+    constexpr uint32_t IDESC_O2 = instr_desc(128, 64, 1, 0);   // S^T from the [d_k][d_v] tile (MN-major) x Q (K-major)
+    constexpr uint32_t IDESC_S = instr_desc(128, 128, 1, 1);   // K~^T (MN-major) x V (MN-major)
 
     auto issue_tma = [&](int c) {
         int row0 = s.own_begin - s.n_replay + c * BT;
@@ -207,7 +213,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         // ---- state pass: S_c^T -> bf16 operand tile (+ slot), S^T <- gamma S^T ----------------------------
         {
             const bool export_slot = next_req < s.req_hi && tb.slot_chunk[next_req] == c;
-            float* slot_dst = export_slot ? slots + ((size_t)next_req * H + h) * state_elems : nullptr;
+            float* slot_dst = export_slot ? slots + ((size_t)next_req * H + h) * state_elems + (size_t)L * D : nullptr;
             const float gamma = m.gamma;
             for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
                 uint32_t x[32];
@@ -215,7 +221,10 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 tmem_ld_wait();
                 if (slot_dst) {
 #pragma unroll
-                    for (int i = 0; i < 32; i++) slot_dst[(size_t)(blk * 32 + i) * D + L] = __uint_as_float(x[i]);
+                    for (int i4 = 0; i4 < 8; i4++)
+                        reinterpret_cast<float4*>(slot_dst + blk * 32)[i4] =
+                            make_float4(__uint_as_float(x[i4 * 4]), __uint_as_float(x[i4 * 4 + 1]),
+                                        __uint_as_float(x[i4 * 4 + 2]), __uint_as_float(x[i4 * 4 + 3]));
                 }
 #pragma unroll
                 for (int v4 = 0; v4 < 4; v4++) {
@@ -224,7 +233,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                     pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
                     pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
                     pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
-                    int col = blk * 32 + v4 * 8;           // first of 8 consecutive i
+                    int col = blk * 32 + v4 * 8;           // first of 8 consecutive j'
                     *reinterpret_cast<uint4*>(sS + (col >> 6) * S_PANEL + sw128_chunk(L, (col & 63) >> 3)) = pk;
                 }
 #pragma unroll
@@ -289,9 +298,9 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             for (int ks = 0; ks < 4; ks++)
                 mma_ss(tmem + COL_O1, desc_mnmajor<BT>(aV, ks), desc_kmajor<BT>(aP, ks), IDESC_O1, ks > 0);
             for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_A, desc_kmajor<D>(aS, ks), desc_kmajor<BT>(aQ, ks), IDESC_O2, ks > 0);
+                mma_ss(tmem + COL_A, desc_mnmajor<D>(aS, ks), desc_kmajor<BT>(aQ, ks), IDESC_O2, ks > 0);
             for (int ks = 0; ks < 4; ks++)
-                mma_ss(tmem + COL_S, desc_mnmajor<BT>(aV, ks), desc_mnmajor<BT>(aK, ks), IDESC_S, true);
+                mma_ss(tmem + COL_S, desc_mnmajor<BT>(aK, ks), desc_mnmajor<BT>(aV, ks), IDESC_S, true);
             mma_commit(&m.bar_o);
         }
         mbar_wait(&m.bar_o, ph_o, status);
