@@ -308,6 +308,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const bool gather_first = s.n_replay > 0;
     uint32_t ph_tiles = 0, ph_a = 0, ph_o = 0;
     int next_req = s.req_hi - 1;
+    // chunk index of the next exported boundary on the way down (kept in a register: no global load per chunk)
+    int next_boundary = next_req >= s.req_lo ? tb.slot_chunk[next_req] : -1;
     if (is_issuer) issue_tiles(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
     int nx_code[2];
     float nx_g[2];
@@ -371,7 +373,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         if (is_compute) {
             // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma -----------------
             {
-                const bool boundary = next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1;
+                const bool boundary = next_boundary == c + 1;
                 const int cons_lo = boundary ? tb.slot_cons_ptr[next_req] : 0;
                 const int cons_hi = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
                 const float gamma = rd.gamma;
@@ -418,7 +420,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
                 tmem_st32(tm_lane + COL_DS + blk * 32, x);
                 tmem_st_wait();
-                if (boundary) next_req--;
+                if (boundary) {
+                    next_req--;
+                    next_boundary = next_req >= s.req_lo ? tb.slot_chunk[next_req] : -1;
+                }
                 g_part = gamma * dot;
                 // dO~ = e^{b_t} dO (zero on rows without an output): two 16-byte vectors per thread
                 for (int e = tid; e < BT * 16; e += NC) {

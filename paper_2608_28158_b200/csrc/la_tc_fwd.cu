@@ -141,6 +141,8 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const bool gather_first = s.n_replay > 0;
     uint32_t ph_tma = 0, ph_a = 0, ph_o = 0;
     int next_req = s.req_lo;
+    // chunk index of the next requested boundary (kept in a register: no global load per chunk)
+    int next_boundary = next_req < s.req_hi ? tb.slot_chunk[next_req] : -1;
     if (!gather_first && tid == 0) issue_tma(0);
 
     for (int c = 0; c < s.n_chunks; c++) {
@@ -212,7 +214,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         __syncthreads();                          // (3) b2 / eb / w / gamma visible
         // ---- state pass: S_c^T -> bf16 operand tile (+ slot), S^T <- gamma S^T ----------------------------
         {
-            const bool export_slot = next_req < s.req_hi && tb.slot_chunk[next_req] == c;
+            const bool export_slot = next_boundary == c;
             float* slot_dst = export_slot ? slots + ((size_t)next_req * H + h) * state_elems + (size_t)L * D : nullptr;
             const float gamma = m.gamma;
             for (int blk = 2 * grp; blk < 2 * grp + 2; blk++) {
@@ -241,7 +243,10 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 tmem_st32(tm_lane + COL_S + blk * 32, x);
             }
             tmem_st_wait();
-            if (export_slot) next_req++;
+            if (export_slot) {
+                next_req++;
+                next_boundary = next_req < s.req_hi ? tb.slot_chunk[next_req] : -1;
+            }
             fence_async_smem();
         }
         // ---- P = A .* decay (warps 0,1)  |  K <- w .* K (warps 2,3) ------------------------------------------
