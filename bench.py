@@ -200,6 +200,54 @@ def trajectory_wise_ms(H, fo, cfg, inp, flags, trees_per_batch=4):
     return total_ms, total_rows
 
 
+def per_config_table(args):
+    """Compact tokens/s, strict roofline fraction and trajectory-wise speedup of every bf16 configuration (cfg0 is
+    fp32 and runs the FMA kernels).  Opt-in (--per-config): printed to stderr, the JSON line is unchanged."""
+    import torch
+    import paper_2608_28158_b200 as H
+    from workloads import CONFIGS, config_forest, make_inputs
+
+    peaks = measured_peaks()
+    rows = []
+    for name in ("cfg0", "cfg1", "cfg2", "cfg3", "cfg4"):
+        cfg = CONFIGS[name]
+        fo = config_forest(name)
+        plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, cfg["chunk"]).upload()
+        canon = make_inputs(plan.C, cfg["H"], cfg["dk"], cfg["dv"], cfg["dtype"], cfg["seed"], device="cuda")
+        rows_t = torch.as_tensor(plan.row_of_token.astype(np.int64), device="cuda")
+        inp = {}
+        for n, x in canon.items():
+            y = torch.empty_like(x)
+            y[rows_t] = x
+            inp[n] = y
+        ws = H.Workspace(plan, cfg["H"], cfg["dk"], cfg["dv"], inp["q"].dtype)
+        out = None
+        for _ in range(3):
+            out = H.run_fwd_bwd(plan, ws, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"], out=out)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(5):
+            H.run_fwd_bwd(plan, ws, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"], out=out)
+        b.record()
+        torch.cuda.synchronize()
+        H.harts_la_check(ws.dev_status)
+        ms = a.elapsed_time(b) / 5
+        del inp, ws, out
+        t_ms, t_rows = trajectory_wise_ms(H, fo, cfg, canon, 0, trees_per_batch=4)
+        elem = canon["q"].element_size()
+        th = plan.C * cfg["H"]
+        bytes_ = th * ((6 * cfg["dk"] + 5 * cfg["dv"]) * elem + 12)
+        rows.append((name, plan.C, t_rows, plan.R, plan.n_rounds, plan.n_seq, ms, plan.C / ms * 1e3,
+                     bytes_ / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms, t_ms / ms))
+        del canon
+        torch.cuda.empty_cache()
+    print("config  compact  traj-wise  replay  rounds  seqs   ms/step  compact tok/s  strict-roof  speedup vs traj-wise",
+          file=sys.stderr)
+    for r in rows:
+        print(f"{r[0]:6s} {r[1]:8d} {r[2]:10d} {r[3]:7d} {r[4]:7d} {r[5]:6d} {r[6]:8.3f} {r[7]:14.0f} {r[8]:11.3f} {r[9]:10.2f}",
+              file=sys.stderr)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -403,6 +451,10 @@ def run_ours(args):
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+    elif args.per_config:
+        del inp, out, ws
+        torch.cuda.empty_cache()
+        per_config_table(args)
 
 
 def main():
@@ -417,6 +469,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-trajwise", action="store_true")
+    ap.add_argument("--per-config", action="store_true", help="also print a table over all configurations to stderr")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
