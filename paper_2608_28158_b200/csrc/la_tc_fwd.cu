@@ -145,18 +145,22 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     int next_boundary = next_req < s.req_hi ? tb.slot_chunk[next_req] : -1;
     if (!gather_first && tid == 0) issue_tma(0);
 
-    for (int c = 0; c < s.n_chunks; c++) {
-        // ---- row codes and g for this chunk (registers first: the previous epilogue still reads m.code) ----
-        float gval = 0.f;
-        int my_code = -1;
-        if (tid < BT) {
-            int vr = c * BT + tid;
-            if (vr < s.n_virtual) {
-                int r = vr < s.n_replay ? tb.replay_row[s.replay_base + vr] : s.own_begin + (vr - s.n_replay);
-                my_code = vr < s.n_replay ? -2 - r : r;
-                gval = g[(size_t)r * H + h];
-            }
+    // row codes and g of a chunk, loaded one chunk ahead (during the previous epilogue)
+    auto row_code = [&](int c, int& code, float& gv) {
+        code = -1;
+        gv = 0.f;
+        int vr = c * BT + tid;
+        if (tid < BT && c < s.n_chunks && vr < s.n_virtual) {
+            int r = vr < s.n_replay ? tb.replay_row[s.replay_base + vr] : s.own_begin + (vr - s.n_replay);
+            code = vr < s.n_replay ? -2 - r : r;
+            gv = g[(size_t)r * H + h];
         }
+    };
+    float gval;
+    int my_code;
+    row_code(0, my_code, gval);
+
+    for (int c = 0; c < s.n_chunks; c++) {
         if (tid == 0) tma_store_wait_read();      // the previous chunk's state store has left sS
         tc_fence_before();
         __syncthreads();                          // (1) epilogue of the previous chunk is over everywhere
@@ -312,6 +316,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
         ph_o ^= 1;
         tc_fence_after();
         if (tid == 0 && c + 1 < s.n_chunks) issue_tma(c + 1);   // tiles are free: every MMA that read them is done
+        row_code(c + 1, my_code, gval);
         // ---- epilogue: o_t = O1 + e^{b_t} O2, lane = output column j', 32 rows per column half ---------------
         const bool full = !(c == 0 && gather_first) && (c + 1) * BT <= s.n_virtual;
         {
