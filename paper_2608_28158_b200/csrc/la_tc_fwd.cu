@@ -326,10 +326,19 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             tmem_ld32(tm_lane + COL_A + t0, x2);
             tmem_ld_wait();
             if (full) {            // all 64 rows are own rows: stage [row][feature] for one TMA store
+                float ebt[32];
+#pragma unroll
+                for (int i4 = 0; i4 < 8; i4++) {
+                    float4 e4 = reinterpret_cast<const float4*>(m.eb + t0)[i4];
+                    ebt[i4 * 4 + 0] = e4.x;
+                    ebt[i4 * 4 + 1] = e4.y;
+                    ebt[i4 * 4 + 2] = e4.z;
+                    ebt[i4 * 4 + 3] = e4.w;
+                }
 #pragma unroll
                 for (int e = 0; e < 32; e++) {
                     int t = t0 + e;
-                    float val = __uint_as_float(x1[e]) + m.eb[t] * __uint_as_float(x2[e]);
+                    float val = __uint_as_float(x1[e]) + ebt[e] * __uint_as_float(x2[e]);
                     *reinterpret_cast<__nv_bfloat16*>(sO + t * 256 + L * 2) = __float2bfloat16_rn(val);
                 }
                 fence_async_smem();
