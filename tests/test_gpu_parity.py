@@ -58,8 +58,10 @@ def test_compact_equals_trajectory_wise_on_gpu(name):
     _, exp_out = run_gpu(exp_fo, exp_inp, backward=False)
     a = exp_out["o"].float().cpu().numpy()
     b = out["o"][src_t.cuda()].float().cpu().numpy()
-    # the chunk grid of a replay-started branch coincides with the trajectory's own grid
-    assert rel_err(a, b) < (1e-6 if cfg["dtype"] == "fp32" else 2e-3)
+    # the chunk grid of a replay-started branch coincides with the trajectory's own grid and the exported boundary
+    # states are exact fp32 copies, so the two runs take the same floating-point path
+    print(name, "compact vs trajectory-wise: max abs diff", float(np.abs(a - b).max()), "rel", rel_err(a, b))
+    assert np.array_equal(a, b)
 
 
 def edge_forests():
@@ -103,6 +105,44 @@ def test_rounds_issued_one_by_one_match_round_zero():
     torch.cuda.synchronize()
     for n, x in (("o", o), ("dq", dq), ("dk", dk), ("dv", dv), ("dg", dg)):
         assert torch.equal(x, ref[n]), n
+
+
+def test_hand_built_tables_drive_one_packed_call():
+    # Eq. 16 without the planner: two sequences in one call, the second starts from a caller-provided state in a slot
+    # and the first exports its boundary after chunk 0 into another slot.
+    import ctypes
+    H_, d, n0, n1 = 2, 128, 150, 70
+    inp = make_inputs(n0 + n1, H_, d, d, "bf16", 23)
+    dev = {n: x.cuda() for n, x in inp.items()}
+    i32 = lambda *v: torch.tensor(v, dtype=torch.int32, device="cuda")  # noqa: E731
+    arrays = dict(seq_own_begin=i32(0, n0, n0 + n1), seq_init_slot=i32(-1, 1), seq_replay_ptr=i32(0, 0, 0),
+                  replay_row=i32(0), seq_req_ptr=i32(0, 1, 1), slot_chunk=i32(1), seq_chunk_ptr=i32(0, 3, 5),
+                  slot_cons_ptr=i32(0, 0), slot_cons_seq=i32(0), rg_row=i32(0), rg_ptr=i32(0), rg_entry=i32(0))
+    tb = H.binding.Tables()
+    tb.chunk, tb.n_rows, tb.n_replay, tb.n_seq, tb.n_slots, tb.n_chunks, tb.n_rg_rows = 64, n0 + n1, 0, 2, 2, 5, 0
+    for n, a in arrays.items():
+        setattr(tb, n, a.data_ptr())
+    S0 = torch.randn(H_, d, d, device="cuda") * 0.1
+    slots = torch.zeros(2, H_, d, d, device="cuda")
+    slots[1] = S0
+    o = torch.empty_like(dev["v"])
+    H.harts_la_fwd_seqs(tb, 0, 2, dev["q"], dev["k"], dev["v"], dev["g"], o, slots, None)
+    torch.cuda.synchronize()
+    # fp64 token recurrence for both sequences
+    q, k, v, g = (inp[n].double().numpy() for n in ("q", "k", "v", "g"))
+    ref = np.zeros((n0 + n1, H_, d))
+    S = np.zeros((H_, d, d))
+    for t in range(n0):
+        if t == 64:
+            exported = S.copy()
+        S = np.exp(g[t])[:, None, None] * S + k[t][:, :, None] * v[t][:, None, :]
+        ref[t] = np.einsum("hi,hij->hj", q[t], S)
+    S = S0.double().cpu().numpy()
+    for t in range(n0, n0 + n1):
+        S = np.exp(g[t])[:, None, None] * S + k[t][:, :, None] * v[t][:, None, :]
+        ref[t] = np.einsum("hi,hij->hj", q[t], S)
+    assert rel_err(o.float().cpu().numpy(), ref) < 5e-3
+    assert rel_err(slots[0].cpu().numpy(), exported) < 5e-3
 
 
 def test_errors_are_reported_without_launching():
