@@ -381,6 +381,19 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 const int blk = grp;
                 uint32_t x[32];
                 tmem_ld32(tm_lane + COL_DS + blk * 32, x);
+                // dO~ = e^{b_t} dO (zero on rows without an output): two 16-byte vectors per thread
+                for (int e = tid; e < BT * 16; e += NC) {
+                    uint32_t off = e * 16;
+                    float sc = rd.eb[(off % PANEL) >> 7];
+                    uint4 raw = *reinterpret_cast<const uint4*>(sDO + off);
+                    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+                    for (int e2 = 0; e2 < 4; e2++) {
+                        float2 f = __bfloat1622float2(h2[e2]);
+                        h2[e2] = sc != 0.f ? __floats2bfloat162_rn(f.x * sc, f.y * sc) : __floats2bfloat162_rn(0.f, 0.f);
+                    }
+                    *reinterpret_cast<uint4*>(sDOs + off) = raw;
+                }
                 tmem_ld_wait();
                 for (int u = cons_lo; u < cons_hi; u++) {
                     const float4* src = reinterpret_cast<const float4*>(
@@ -418,26 +431,12 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 }
 #pragma unroll
                 for (int i = 0; i < 32; i++) x[i] = __float_as_uint(__uint_as_float(x[i]) * gamma);
-                tmem_st32(tm_lane + COL_DS + blk * 32, x);
-                tmem_st_wait();
+                tmem_st32(tm_lane + COL_DS + blk * 32, x);     // awaited at the end of the masking pass
                 if (boundary) {
                     next_req--;
                     next_boundary = next_req >= s.req_lo ? tb.slot_chunk[next_req] : -1;
                 }
                 g_part = gamma * dot;
-                // dO~ = e^{b_t} dO (zero on rows without an output): two 16-byte vectors per thread
-                for (int e = tid; e < BT * 16; e += NC) {
-                    uint32_t off = e * 16;
-                    float sc = rd.eb[(off % PANEL) >> 7];
-                    uint4 raw = *reinterpret_cast<const uint4*>(sDO + off);
-                    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
-#pragma unroll
-                    for (int e2 = 0; e2 < 4; e2++) {
-                        float2 f = __bfloat1622float2(h2[e2]);
-                        h2[e2] = sc != 0.f ? __floats2bfloat162_rn(f.x * sc, f.y * sc) : __floats2bfloat162_rn(0.f, 0.f);
-                    }
-                    *reinterpret_cast<uint4*>(sDOs + off) = raw;
-                }
             }
             // ---- P = A .* decay (lanes 0..63), dP = dA .* decay (lanes 64..127): 16 columns of one of them per thread ------
             mbar_wait(&m.bar_a, ph_a, status);
@@ -471,6 +470,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 }
                 }
             }
+            tmem_st_wait();
             fence_async_smem();
         }
         ph_a ^= 1;
