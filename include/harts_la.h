@@ -85,6 +85,8 @@ typedef struct harts_la_plan_view {
     const int32_t* rg_row;         /* [n_rg_rows] replayed physical rows, ascending */
     const int32_t* rg_ptr;         /* [n_rg_rows+1] CSR into rg_entry */
     const int32_t* rg_entry;       /* [n_replay] indices into replay_row whose gradients land on rg_row */
+    const int32_t* seq_order;      /* [n_seq] per round, its sequences sorted by decreasing chunk count: the order in
+                                      which the kernels pick up work (longest first); a scheduling hint only */
 } harts_la_plan_view_t;
 
 /*
@@ -106,6 +108,7 @@ typedef struct harts_la_tables {
     const int32_t* rg_row;
     const int32_t* rg_ptr;
     const int32_t* rg_entry;
+    const int32_t* seq_order;      /* may be NULL: sequences are then processed in index order */
 } harts_la_tables_t;
 
 const char* harts_la_strerror(int32_t code);

@@ -27,14 +27,14 @@ class _View(C.Structure):
     _counts = ("chunk", "n_rounds", "n_rows", "n_replay", "n_seq", "n_slots", "n_chunks", "n_rg_rows")
     _arrays = ("row_of_token", "round_seq_ptr", "seq_tree", "seq_own_begin", "seq_own_len", "seq_start_pos",
                "seq_init_slot", "seq_replay_ptr", "replay_row", "seq_req_ptr", "slot_chunk", "seq_chunk_ptr",
-               "slot_cons_ptr", "slot_cons_seq", "rg_row", "rg_ptr", "rg_entry")
+               "slot_cons_ptr", "slot_cons_seq", "rg_row", "rg_ptr", "rg_entry", "seq_order")
     _fields_ = [(n, C.c_int32) for n in _counts] + [(n, _I32P) for n in _arrays]
 
 
 class Tables(C.Structure):
     _counts = ("chunk", "n_rows", "n_replay", "n_seq", "n_slots", "n_chunks", "n_rg_rows")
     _arrays = ("seq_own_begin", "seq_init_slot", "seq_replay_ptr", "replay_row", "seq_req_ptr", "slot_chunk",
-               "seq_chunk_ptr", "slot_cons_ptr", "slot_cons_seq", "rg_row", "rg_ptr", "rg_entry")
+               "seq_chunk_ptr", "slot_cons_ptr", "slot_cons_seq", "rg_row", "rg_ptr", "rg_entry", "seq_order")
     _fields_ = [(n, C.c_int32) for n in _counts] + [(n, C.c_void_p) for n in _arrays]
 
 
@@ -105,7 +105,8 @@ class Plan:
                      seq_init_slot=self.n_seq, seq_replay_ptr=self.n_seq + 1, replay_row=self.n_replay,
                      seq_req_ptr=self.n_seq + 1, slot_chunk=self.n_slots, seq_chunk_ptr=self.n_seq + 1,
                      slot_cons_ptr=self.n_slots + 1, slot_cons_seq=None, rg_row=self.n_rg_rows,
-                     rg_ptr=self.n_rg_rows + 1 if self.n_rg_rows else 1, rg_entry=self.n_replay)
+                     rg_ptr=self.n_rg_rows + 1 if self.n_rg_rows else 1, rg_entry=self.n_replay,
+                     seq_order=self.n_seq)
         for n in _View._arrays:
             size = sizes[n]
             if n == "slot_cons_seq":

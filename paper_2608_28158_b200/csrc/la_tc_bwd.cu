@@ -25,6 +25,7 @@ namespace harts {
 int32_t make_row_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H);
 int32_t make_state_map(CUtensorMap* map, const void* base, int64_t n);
 int32_t make_out_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H);
+int sm_count();
 
 namespace {
 
@@ -180,7 +181,7 @@ __device__ __forceinline__ void epilogue_dv(const RowData& m, unsigned char* sme
 }
 
 __global__ void __launch_bounds__(NT, 1)
-tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_constant__ CUtensorMap map_q,
+tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const __grid_constant__ CUtensorMap map_q,
               const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_cs,
               const __grid_constant__ CUtensorMap map_dq, const __grid_constant__ CUtensorMap map_dk,
@@ -207,8 +208,6 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const bool is_issuer = tid == NC;              // first lane of the extra warp
     const int grp = warp >> 2;                    // column group (compute warps)
     const int L = (warp & 3) * 32 + lane;         // tensor-memory lane = feature index (or row t) of this thread
-    const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
-    const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)D * D;
 
     if (tid == 0) {
@@ -227,6 +226,16 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const uint32_t tmem = m.tmem;
     const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
+    // Persistent CTAs: work item = (sequence, head); items are ordered longest sequence first and dealt to the CTAs
+    // in a snake pattern, so that every CTA gets a similar amount of work.
+    uint32_t ph_tiles = 0, ph_a = 0, ph_o = 0;
+    const int G = gridDim.x;
+    for (int tier = 0; tier * G < n_items; tier++) {
+    const int item = (tier & 1) ? tier * G + (G - 1 - (int)blockIdx.x) : tier * G + (int)blockIdx.x;
+    if (item >= n_items) continue;
+    const int seq_pos = seq_lo + item / H, h = item % H;
+    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
+    const SeqInfo s = seq_info(tb, seq);
     if (is_compute) {   // dS = 0: nothing follows the last chunk
         uint32_t zero[32];
 #pragma unroll
@@ -306,7 +315,6 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     };
 
     const bool gather_first = s.n_replay > 0;
-    uint32_t ph_tiles = 0, ph_a = 0, ph_o = 0;
     int next_req = s.req_hi - 1;
     // chunk index of the next exported boundary on the way down (kept in a register: no global load per chunk)
     int next_boundary = next_req >= s.req_lo ? tb.slot_chunk[next_req] : -1;
@@ -605,6 +613,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
                 make_float4(__uint_as_float(x[i4 * 4]), __uint_as_float(x[i4 * 4 + 1]), __uint_as_float(x[i4 * 4 + 2]),
                             __uint_as_float(x[i4 * 4 + 3]));
     }
+    }   // work items
     if (is_issuer) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
@@ -631,8 +640,9 @@ int32_t tc_bwd(const BwdArgs& a) {
     ScratchLayout sl = scratch_layout(a.tb, a.H, a.dk, a.dv);
     char* base = static_cast<char*>(a.scratch);
     int n = (a.seq_hi - a.seq_lo) * a.H;
-    tc_bwd_kernel<<<n, NT, Smem::bytes + 1024, a.stream>>>(
-        a.tb, a.seq_lo, a.H, mq, mk, mv, mdo, mcs, mdq, mdk, mdv, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
+    int grid = n < sm_count() ? n : sm_count();
+    tc_bwd_kernel<<<grid, NT, Smem::bytes + 1024, a.stream>>>(
+        a.tb, a.seq_lo, n, a.H, mq, mk, mv, mdo, mcs, mdq, mdk, mdv, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_,
         (__nv_bfloat16*)a.dv_, a.dg, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
         (float*)(base + sl.rg), a.dev_status);

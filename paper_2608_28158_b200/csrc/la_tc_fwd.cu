@@ -68,7 +68,7 @@ __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq
 }
 
 __global__ void __launch_bounds__(NT, 2)
-tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_constant__ CUtensorMap map_q,
+tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const __grid_constant__ CUtensorMap map_q,
               const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const __grid_constant__ CUtensorMap map_cs, const __grid_constant__ CUtensorMap map_o,
               const __nv_bfloat16* __restrict__ q,
@@ -87,8 +87,6 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int grp = warp >> 2;                    // column half
     const int L = (warp & 3) * 32 + lane;         // tensor-memory lane of this thread
-    const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
-    const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)D * D;
 
     if (tid == 0) {
@@ -104,6 +102,16 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     const uint32_t tmem = m.tmem;
     const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
+    // Persistent CTAs: work item = (sequence, head); items are ordered longest sequence first and dealt to the CTAs
+    // in a snake pattern, so that every CTA gets a similar amount of work.
+    uint32_t ph_tma = 0, ph_a = 0, ph_o = 0;
+    const int G = gridDim.x;
+    for (int tier = 0; tier * G < n_items; tier++) {
+    const int item = (tier & 1) ? tier * G + (G - 1 - (int)blockIdx.x) : tier * G + (int)blockIdx.x;
+    if (item >= n_items) continue;
+    const int seq_pos = seq_lo + item / H, h = item % H;
+    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
+    const SeqInfo s = seq_info(tb, seq);
     // initial state into tensor memory: lane i = L holds S[i][:]
     {
         const float* src = s.init_slot < 0 ? nullptr : slots + ((size_t)s.init_slot * H + h) * state_elems + (size_t)L * D;
@@ -139,7 +147,6 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
     };
 
     const bool gather_first = s.n_replay > 0;
-    uint32_t ph_tma = 0, ph_a = 0, ph_o = 0;
     int next_req = s.req_lo;
     // chunk index of the next requested boundary (kept in a register: no global load per chunk)
     int next_boundary = next_req < s.req_hi ? tb.slot_chunk[next_req] : -1;
@@ -362,6 +369,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int H, const __grid_consta
             }
         }
     }
+    }   // work items
     if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
@@ -423,6 +431,16 @@ int32_t make_out_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H
     return r == CUDA_SUCCESS ? HARTS_OK : HARTS_ECUDA;
 }
 
+int sm_count() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1)
+            v = 148;
+        return v;
+    }();
+    return n;
+}
+
 int32_t tc_supported(int32_t dtype, int32_t dk, int32_t dv) { return dtype == HARTS_BF16 && dk == 128 && dv == 128; }
 
 int32_t tc_fwd(const FwdArgs& a) {
@@ -439,8 +457,9 @@ int32_t tc_fwd(const FwdArgs& a) {
         cudaSuccess)
         return HARTS_ECUDA;
     int n = (a.seq_hi - a.seq_lo) * a.H;
-    tc_fwd_kernel<<<n, NT, Smem::bytes + 1024, a.stream>>>(
-        a.tb, a.seq_lo, a.H, mq, mk, mv, mcs, mo, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
+    int grid = n < 2 * sm_count() ? n : 2 * sm_count();
+    tc_fwd_kernel<<<grid, NT, Smem::bytes + 1024, a.stream>>>(
+        a.tb, a.seq_lo, n, a.H, mq, mk, mv, mcs, mo, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (__nv_bfloat16*)a.o, a.slots, a.chunk_states != nullptr, a.dev_status);
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }

@@ -388,6 +388,14 @@ int32_t build_plan(int32_t n_trees, const int32_t* tree_node_ptr, const int32_t*
         if (R > 0) P.rg_ptr.push_back(R);
         P.n_rg_rows = (int32_t)P.rg_row.size();
     }
+    // work order: inside every round the sequences by decreasing chunk count (longest chains start first)
+    P.seq_order.resize(n_seq);
+    for (int32_t i = 0; i < n_seq; i++) P.seq_order[i] = i;
+    for (int32_t r = 0; r < n_rounds; r++)
+        std::stable_sort(P.seq_order.begin() + P.round_seq_ptr[r], P.seq_order.begin() + P.round_seq_ptr[r + 1],
+                         [&](int32_t a, int32_t b) {
+                             return P.seq_chunk_ptr[a + 1] - P.seq_chunk_ptr[a] > P.seq_chunk_ptr[b + 1] - P.seq_chunk_ptr[b];
+                         });
     P.pack();
     return HARTS_OK;
 }
@@ -396,7 +404,7 @@ int32_t build_plan(int32_t n_trees, const int32_t* tree_node_ptr, const int32_t*
 void Plan::pack() {
     const std::vector<int32_t>* arrays[N_DEVICE_TABLES] = {
         &seq_own_begin, &seq_init_slot, &seq_replay_ptr, &replay_row, &seq_req_ptr, &slot_chunk,
-        &seq_chunk_ptr, &slot_cons_ptr, &slot_cons_seq, &rg_row, &rg_ptr, &rg_entry};
+        &seq_chunk_ptr, &slot_cons_ptr, &slot_cons_seq, &rg_row, &rg_ptr, &rg_entry, &seq_order};
     size_t words = 0;
     for (int i = 0; i < N_DEVICE_TABLES; i++) {
         table_offset[i] = words;
@@ -430,6 +438,7 @@ void Plan::tables(const void* dev_blob, harts_la_tables_t* t) const {
     t->rg_row = base + table_offset[9];
     t->rg_ptr = base + table_offset[10];
     t->rg_entry = base + table_offset[11];
+    t->seq_order = base + table_offset[12];
 }
 
 }  // namespace harts
@@ -493,6 +502,7 @@ int32_t harts_la_plan_view(const harts_la_plan_t* plan, harts_la_plan_view_t* v)
     v->rg_row = p.rg_row.data();
     v->rg_ptr = p.rg_ptr.data();
     v->rg_entry = p.rg_entry.data();
+    v->seq_order = p.seq_order.data();
     return HARTS_OK;
 }
 

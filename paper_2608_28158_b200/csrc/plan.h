@@ -7,14 +7,14 @@
 
 namespace harts {
 
-constexpr int N_DEVICE_TABLES = 12;
+constexpr int N_DEVICE_TABLES = 13;
 
 struct Plan {
     int32_t chunk = 0, n_rounds = 0, n_rows = 0, n_replay = 0, n_seq = 0, n_slots = 0, n_chunks = 0,
             n_rg_rows = 0;
     std::vector<int32_t> row_of_token, round_seq_ptr, seq_tree, seq_own_begin, seq_own_len, seq_start_pos,
         seq_init_slot, seq_replay_ptr, replay_row, seq_req_ptr, slot_chunk, seq_chunk_ptr, slot_cons_ptr,
-        slot_cons_seq, rg_row, rg_ptr, rg_entry;
+        slot_cons_seq, rg_row, rg_ptr, rg_entry, seq_order;
     std::vector<int32_t> blob;                 // device tables back to back, 16-byte aligned starts
     size_t table_offset[N_DEVICE_TABLES] = {}; // in int32 words
     void pack();
