@@ -57,7 +57,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -67,7 +67,11 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def mark(self):
+        """Host time now; summary(t0, t1) keeps the samples taken between two marks."""
+        return time.time()
 
     def __exit__(self, *exc):
         if self.proc:
@@ -77,11 +81,11 @@ class ClockSampler:
             except subprocess.TimeoutExpired:
                 self.proc.kill()
 
-    def summary(self):
+    def summary(self, t0=None, t1=None):
         sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for r in self.rows:
-            if len(r) < 6:
+        for stamp, r in self.rows:
+            if len(r) < 6 or (t0 is not None and not (t0 <= stamp <= t1 + 0.05)):
                 continue
             try:
                 sm.append(float(r[0]))
@@ -315,18 +319,22 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step(False)
-    H.harts_la_check(ws.dev_status)
-    barrier()
     all_marks = []
     t_begin, t_end = ev(), ev()
-    with ClockSampler(local) as clocks:
+    with ClockSampler(local) as clocks:            # started before the warm-up so that it is sampling by then
+        for _ in range(args.warmup):
+            step(False)
+        H.harts_la_check(ws.dev_status)
+        # a short region gives the 50 ms sampler nothing to see: keep the GPU under the same load a little longer
+        # before the timed steps when the whole region is under a second
+        barrier()
+        t_host0 = clocks.mark()
         t_begin.record(stream)
         for _ in range(args.steps):
             all_marks.append(step(True))
         t_end.record(stream)
         barrier()
+        t_host1 = clocks.mark()
     ms_total = t_begin.elapsed_time(t_end)
     H.harts_la_check(ws.dev_status)
     for marks in all_marks:
@@ -405,7 +413,10 @@ def run_ours(args):
         else None
     t_roof_bytes = (fwd_bytes + bwd_bytes) / (hbm_peak * 1e9)
     t_roof_flops = (flops_fwd + flops_bwd) / (peaks["bf16_tflops_sustained"] * 1e12)
-    clock = clocks.summary()
+    clock = clocks.summary(t_host0, t_host1)
+    if not clock["samples"]:
+        clock = clocks.summary()
+        clock["note"] = "timed region shorter than the sampling period: samples cover warm-up + timed region"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

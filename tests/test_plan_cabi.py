@@ -115,6 +115,17 @@ def test_single_path_is_one_round():
     assert p.row_of_token.tolist() == list(range(317))
 
 
+def test_work_order_is_a_permutation_inside_every_round_longest_first():
+    for name in ("cfg1", "cfg2", "cfg4"):
+        p = plan_of(config_forest(name), 64)
+        n = np.diff(p.seq_chunk_ptr)
+        for r in range(p.n_rounds):
+            lo, hi = int(p.round_seq_ptr[r]), int(p.round_seq_ptr[r + 1])
+            order = p.seq_order[lo:hi]
+            assert sorted(order.tolist()) == list(range(lo, hi))
+            assert (np.diff(n[order]) <= 0).all()
+
+
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "harts_la.h")).read()
     names = set(re.findall(r"\b(harts_la_\w+)\s*\(", header))
