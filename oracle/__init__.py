@@ -12,6 +12,10 @@ Pins (see tests/test_oracle_*.py, tests/test_plan_oracle.py):
   * plan_oracle -- Algorithm 1: brute-force minimum call counts on tiny trees, the worked
                    examples of Figs. 1-3, the strict boundary cases, the replay total of
                    Eq. 15, fp64 execution of the plan against la_oracle.
+  * logp_oracle -- Eqs. 17/19/20 (mapped log-probability, its gradient, multiplicity): uniform
+                   and two-word closed forms, torch log_softmax + autograd on the expanded
+                   rows, central finite differences, zero row sums and shift invariance,
+                   hand-counted positions of the five-node tree.
   * Appendix planning cases I-III: parity unpinned (the trees' token counts were only in
                    the figures); only the printed totals are checked for self-consistency.
 """

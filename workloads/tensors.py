@@ -30,3 +30,39 @@ def make_inputs(n_tokens: int, H: int, dk: int, dv: int, dtype: str, seed: int, 
     g = torch.nn.functional.logsigmoid(normal(n_tokens, H) + 3.0).contiguous()
     dO = normal(n_tokens, H, dv).to(dt)
     return {"q": q, "k": k, "v": v, "g": g, "dO": dO}
+
+
+def make_logits(n_rows: int, V: int, dtype: str, seed: int, device="cpu", peak: float = 6.0):
+    """Compact logit rows and token ids for the log-probability step.
+
+    z [n_rows, V]: N(0, 2^2) background with one favoured word per row raised by ``peak`` (a language-model
+    row is peaked, not flat); rounded to the run dtype.  token_id int32 [n_rows]: the vocabulary id of each
+    compact token, uniform over the vocabulary except that with probability 1/2 a token is the favoured
+    word of the row before it (so that target logits cover both the peak and the background).
+    Rows are drawn in slabs so that the fp32 staging buffer stays small."""
+    dt = _DTYPES[dtype]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(7000003 * (seed + 1))
+    fav = torch.randint(0, V, (n_rows,), generator=gen, device=device)
+    uni = torch.randint(0, V, (n_rows,), generator=gen, device=device)
+    coin = torch.rand(n_rows, generator=gen, device=device) < 0.5
+    token_id = uni.clone()
+    token_id[1:] = torch.where(coin[1:], fav[:-1], uni[1:])
+    z = torch.empty(n_rows, V, dtype=dt, device=device)
+    slab = max(1, (64 << 20) // max(V, 1))
+    for lo in range(0, n_rows, slab):
+        hi = min(n_rows, lo + slab)
+        blk = torch.randn(hi - lo, V, generator=gen, device=device, dtype=torch.float32) * 2.0
+        blk[torch.arange(hi - lo, device=device), fav[lo:hi]] += peak
+        z[lo:hi] = blk.to(dt)
+    return {"z": z, "token_id": token_id.to(torch.int32)}
+
+
+def make_logp_grad(n_pos: int, seed: int, device="cpu", keep: float = 0.6):
+    """dL/dlambda for every non-terminal semantic position: an advantage-like N(0,1) value divided by the
+    number of positions, exactly zero where a Bernoulli(keep) action mask drops the position."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(9000011 * (seed + 1))
+    adv = torch.randn(n_pos, generator=gen, device=device, dtype=torch.float32)
+    mask = torch.rand(n_pos, generator=gen, device=device) < keep
+    return torch.where(mask, adv / max(n_pos, 1), torch.zeros_like(adv))
