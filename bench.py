@@ -10,6 +10,9 @@ metric through the host-buffer call (pinned host inputs copied in, results copie
 timed region).  With N > 1 (torchrun) every rank runs its own copy of the workload (weak scaling,
 no collective on the data path); time is the maximum over ranks.
 
+``--workload logp`` runs the second path instead, the compact-to-semantic log-probability (one step = its
+forward + backward over one microbatch of compact logit rows), with the same JSON keys.
+
 ``--impl reference`` times the fp64 CPU oracle (oracle/), as it stands, on the host cores, on a
 bounded sample of the same workload.
 """
@@ -154,6 +157,75 @@ def run_reference(args):
                              "unit": UNIT},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------------
+# Second workload: compact-to-semantic log-probability (Eqs. 17, 19), `--workload logp`
+# --------------------------------------------------------------------------------------------------
+LOGP_METRIC = "mapped log-prob fwd+bwd compact rows/s"
+LOGP_UNIT = "compact rows/s"
+LOGP_V = 157184            # vocabulary of the evaluated model
+LOGP_ROWS = 65536          # compact-row capacity of one microbatch
+
+
+def logp_forest(rank=0):
+    """Whole trees of cfg3, starting at a rank-dependent tree, while they fit the microbatch capacity."""
+    fo = config_forest_cached("cfg3")
+    base = fo.token_base()
+    first = (3 * rank) % fo.n_trees
+    trees, rows = [], 0
+    for t in list(range(first, fo.n_trees)) + list(range(first)):
+        c = int(base[fo.tree_node_ptr[t + 1]] - base[fo.tree_node_ptr[t]])
+        if rows + c > LOGP_ROWS:
+            break
+        trees.append(t)
+        rows += c
+    return fo.subset(trees), trees
+
+
+def config_forest_cached(name):
+    from workloads import config_forest
+    return config_forest(name)
+
+
+def logp_oracle_sample(small=False):
+    """The fp64 oracle of Eqs. 17/19 on one small tree at the full vocabulary."""
+    from oracle import logp_oracle
+    from workloads import config_forest, make_forest, make_logits, make_logp_grad
+    # small: a 256-row tree (root 128, one child at its end, one forking at offset 100) for the many-step arm
+    fo = make_forest([([-1, 0, 0], [0, 128, 100], [128, 64, 64])]) if small else config_forest("cfg0b")
+    name = "three-node tree" if small else "cfg0b tree"
+    data = make_logits(fo.n_tokens, LOGP_V, "bf16", 0)
+    m, y, _ = logp_oracle.positions(fo, data["token_id"].numpy())
+    g = make_logp_grad(len(m), 0, keep=1.0).double().numpy()
+    z = data["z"].double().numpy()
+    t0 = time.perf_counter()
+    logp_oracle.mapped_logp(z, m, y)
+    logp_oracle.mapped_logp_grad(z, m, y, g)
+    dt = time.perf_counter() - t0
+    return {"value": fo.n_tokens / dt, "unit": LOGP_UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{name}: {fo.n_tokens} compact rows, {len(m)} positions, V={LOGP_V}, fwd+bwd, {dt:.1f} s",
+            "seconds": dt}
+
+
+def run_logp_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    vals, secs, last = [], [], None
+    for i in range(args.warmup + args.steps):
+        last = logp_oracle_sample(small=True)
+        if i >= args.warmup:
+            vals.append(last["value"])
+            secs.append(last["seconds"])
+    value = statistics.mean(vals)
+    print(json.dumps({
+        "impl": "reference", "metric": LOGP_METRIC, "value": value, "unit": LOGP_UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(secs) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "logp", "V": LOGP_V},
+        "cpu_baseline": {"kind": last["kind"], "cores": last["cores"], "sample": last["sample"], "value": value,
+                         "unit": LOGP_UNIT},
+        "e2e": {"value": value, "unit": LOGP_UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
 # --------------------------------------------------------------------------------------------------
@@ -468,6 +540,152 @@ def run_ours(args):
         per_config_table(args)
 
 
+def run_logp(args):
+    """One step = forward (row max / sum-exp over V, lambda for every position) + backward (dz for every compact row)."""
+    import torch
+    import torch.distributed as dist
+
+    import paper_2608_28158_b200 as H
+    from workloads import make_logits, make_logp_grad
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    fo, trees = logp_forest(rank)
+    C, V = fo.n_tokens, LOGP_V
+    plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
+    data = make_logits(C, V, "bf16", 50 + rank, device="cuda")
+    t0 = time.perf_counter()
+    m, y, _ = H.harts_logp_positions(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len,
+                                     data["token_id"].cpu().numpy(), plan.row_of_token)
+    ptr, pos = H.harts_logp_csr(C, m)
+    t_host = time.perf_counter() - t0
+    P = len(m)
+    z = data["z"]
+    dev = {"m": torch.as_tensor(m).cuda(), "y": torch.as_tensor(y).cuda(), "ptr": torch.as_tensor(ptr).cuda(),
+           "pos": torch.as_tensor(pos).cuda(), "g": make_logp_grad(P, 50 + rank, device="cuda", keep=1.0)}
+    lse = torch.empty(C, device="cuda")
+    lam = torch.empty(P, device="cuda")
+    dz = torch.empty_like(z)
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+
+    def step(marks=None):
+        a, b, c = ev(), ev(), ev()
+        a.record(stream)
+        H.harts_logp_fwd(z, dev["m"], dev["y"], lse, lam, dev_status=status)
+        b.record(stream)
+        H.harts_logp_bwd(z, dev["y"], dev["ptr"], dev["pos"], lse, dev["g"], dz, dev_status=status)
+        c.record(stream)
+        if marks is not None:
+            marks.append((a, b, c))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    marks = []
+    t_begin, t_end = ev(), ev()
+    with ClockSampler(local) as clocks:
+        for _ in range(args.warmup):
+            step()
+        H.harts_la_check(status)
+        barrier()
+        h0 = clocks.mark()
+        t_begin.record(stream)
+        for _ in range(args.steps):
+            step(marks)
+        t_end.record(stream)
+        barrier()
+        h1 = clocks.mark()
+    H.harts_la_check(status)
+    ms_step = t_begin.elapsed_time(t_end) / args.steps
+    fwd_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in marks)
+    bwd_ms = statistics.mean(b.elapsed_time(c) for _, b, c in marks)
+
+    e2e = None
+    if not args.no_e2e:
+        small = {n: x for n, x in dev.items()}
+        host_in = {"z": torch.empty(z.shape, dtype=z.dtype, pin_memory=True)}
+        host_in.update({n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in small.items()})
+        host_out = {"lam": torch.empty(P, pin_memory=True), "dz": torch.empty(z.shape, dtype=z.dtype, pin_memory=True)}
+        host_in["z"].copy_(z)
+        for n, x in small.items():
+            host_in[n].copy_(x)
+        torch.cuda.synchronize()
+
+        def e2e_step():
+            z.copy_(host_in["z"], non_blocking=True)
+            for n, x in small.items():
+                x.copy_(host_in[n], non_blocking=True)
+            step()
+            host_out["lam"].copy_(lam, non_blocking=True)
+            host_out["dz"].copy_(dz, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b = ev(), ev()
+        n_e2e = max(1, min(args.steps, args.e2e_steps))
+        a.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e2e = {"ms": a.elapsed_time(b) / n_e2e, "steps": n_e2e,
+               "h2d": sum(x.numel() * x.element_size() for x in host_in.values()),
+               "d2h": sum(x.numel() * x.element_size() for x in host_out.values())}
+        del host_in, host_out
+
+    if world > 1:
+        ms_step, e2e_ms = max_over_ranks([ms_step, e2e["ms"] if e2e else 0.0], "cuda")
+        if e2e:
+            e2e["ms"] = e2e_ms
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    row_bytes = V * z.element_size()
+    fwd_bytes = C * row_bytes + P * 12 + C * 4              # z once; m, y read and lambda written; lse written
+    bwd_bytes = 2 * C * row_bytes + P * 12 + C * 12         # z read, dz written; y, g, row_pos; lse, row_pos_ptr
+    achieved = bwd_bytes / (bwd_ms * 1e-3) / 1e9
+    clock = clocks.summary(h0, h1)
+    if not clock["samples"]:
+        clock = clocks.summary()
+    line = {
+        "metric": LOGP_METRIC, "value": C * world / (ms_step * 1e-3), "unit": LOGP_UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "logp", "V": V, "compact_rows": C, "positions": P, "trees": f"cfg3 trees {trees}",
+                   "action_mask": "every position selected (no idle rows)",
+                   "l2": f"inputs larger than L2 ({C * row_bytes / 2**30:.2f} GiB of logits)",
+                   "host_index_ms": t_host * 1e3},
+        "roofline": {"bound": "hbm", "kernel": "dz_kernel (backward)", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                     "algorithmic_bytes_per_launch": bwd_bytes, "peak_source": peaks["source"],
+                     "forward": {"achieved": fwd_bytes / (fwd_ms * 1e-3) / 1e9,
+                                 "frac": fwd_bytes / (fwd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                     "whole_path": {"roof_ms": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                                    "frac_strict": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms_step}},
+        "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms},
+        "gpu_launches": 3 * args.steps,
+        "clocks": clock,
+    }
+    if e2e:
+        line["e2e"] = {"value": C * world / (e2e["ms"] * 1e-3), "unit": LOGP_UNIT, "h2d_bytes_per_step": e2e["h2d"],
+                       "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"], "pinned_host_memory": True}
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = logp_oracle_sample()
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -482,7 +700,9 @@ def main():
     ap.add_argument("--no-trajwise", action="store_true")
     ap.add_argument("--per-config", action="store_true", help="also print a table over all configurations to stderr")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload == "logp":
+        (run_logp_reference if args.impl == "reference" else run_logp)(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

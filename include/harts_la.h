@@ -224,8 +224,8 @@ int32_t harts_la_bwd_static(const harts_la_plan_t* plan, const void* dev_blob, c
                             const void* chunk_states, int32_t H, int32_t dk, int32_t dv, int32_t dtype, uint32_t flags,
                             int32_t* dev_status, void* stream);
 
-/* Synchronises `stream`, reads the device status word and returns HARTS_OK, HARTS_ETIMEOUT or
- * HARTS_ECUDA.  dev_status must be zeroed by the caller before the first launch. */
+/* Synchronises `stream`, reads the device status word and returns HARTS_OK, HARTS_ETIMEOUT,
+ * HARTS_EINVAL (an out-of-range index met by a harts_logp_* kernel, see harts_logp.h) or HARTS_ECUDA.  dev_status must be zeroed by the caller before the first launch. */
 int32_t harts_la_check(const int32_t* dev_status, void* stream);
 
 #ifdef __cplusplus

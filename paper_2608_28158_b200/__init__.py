@@ -10,3 +10,6 @@ from .binding import (  # noqa: F401
     harts_la_bwd_seqs, harts_la_check, harts_la_fwd, harts_la_fwd_seqs, harts_la_plan, harts_la_strerror,
     harts_la_workspace_bytes, lib, run_fwd_bwd, run_fwd_bwd_host, expand_trajectories,
 )
+from .logp import (  # noqa: F401
+    harts_logp_positions, harts_logp_csr, harts_logp_fwd, harts_logp_bwd, harts_logp_fwd_shard, harts_logp_combine,
+)

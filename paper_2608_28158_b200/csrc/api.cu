@@ -146,7 +146,8 @@ int32_t harts_la_check(const int32_t* dev_status, void* stream) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(&host, dev_status, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess) return HARTS_ECUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return HARTS_ECUDA;
-    return host == 0 ? HARTS_OK : HARTS_ETIMEOUT;
+    if (host == 0) return HARTS_OK;
+    return host == HARTS_EINVAL ? HARTS_EINVAL : HARTS_ETIMEOUT;   // EINVAL: an index check of harts_logp_*
 }
 
 }  // extern "C"
