@@ -276,7 +276,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tiles);
             }
     };
-    // Row codes and g of chunk c for rows `lane` and `lane + 32` (warp 0 prepares a chunk's row data on its own).
+    // Row codes and g of chunk c for rows `lane` and `lane + 32` (the extra warp prepares a chunk's row data on its own).
     auto load_rows = [&](int c, int (&code)[2], float (&gv)[2]) {
 #pragma unroll
         for (int r = 0; r < 2; r++) {
@@ -321,7 +321,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     if (is_issuer) issue_tiles(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
     int nx_code[2];
     float nx_g[2];
-    if (warp == 0) {
+    if (!is_compute) {
         load_rows(s.n_chunks - 1, nx_code, nx_g);
         store_rows(m.rows[0], nx_code, nx_g);
     }
@@ -375,6 +375,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 mma_ss(tmem + COL_DA, dDOk_hi + kstep_kmajor<BT>(ks), dVk + kstep_kmajor<BT>(ks), I_KK64, ks > 0);
             mma_commit(&m.bar_a);
             tma_store_wait_read();                // the previous chunk's output stores have left the staging tiles
+        }
+        if (!is_compute) {                        // next chunk's rows and g: requested ahead of the next tile loads
+            __syncwarp();
+            load_rows(c - 1, nx_code, nx_g);
         }
         float g_part = 0.f;                       // this thread's share of <S_{c+1}, dS_{c+1}>
         uint32_t qk[16];                          // q[t][L] | k[t][L] << 16 of this thread's 16 rows (bf16 bits)
@@ -520,7 +524,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             mbar_wait(&m.bar_qk_read, ph_o, status);      // every compute warp has taken its q and k values
             if (c > 0) issue_tiles(c - 1, next_tiles);
         }
-        if (warp == 0) load_rows(c - 1, nx_code, nx_g);   // next chunk's rows and g, in flight during the epilogue
+        if (!is_compute) {                        // the extra warp prepares the next chunk's row data during the epilogue
+            __syncwarp();
+            if (c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);
+        }
         if (is_compute) {
             // q[t][L], k[t][L] of this thread's 16 rows, for the dg terms (read while the first MMAs run; after this
             // the epilogue does not touch the tiles, which are reloaded as soon as the MMAs are done)
@@ -557,7 +564,6 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             if (full) epilogue_dv<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
             else epilogue_dv<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
             if (full) fence_async_smem();
-            if (warp == 0 && c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);
         }
         ph_o ^= 1;
         tc_fence_before();
