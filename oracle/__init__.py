@@ -16,6 +16,9 @@ Pins (see tests/test_oracle_*.py, tests/test_plan_oracle.py):
                    and two-word closed forms, torch log_softmax + autograd on the expanded
                    rows, central finite differences, zero row sums and shift invariance,
                    hand-counted positions of the five-node tree.
+  * conv_oracle -- tree-aware causal convolution (Section 4.2): torch conv1d on every expanded
+                   trajectory, autograd through the expansion, identity/shift filters on the
+                   five-node tree, central differences.
   * Appendix planning cases I-III: parity unpinned (the trees' token counts were only in
                    the figures); only the printed totals are checked for self-consistency.
 """
