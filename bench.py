@@ -11,7 +11,8 @@ timed region).  With N > 1 (torchrun) every rank runs its own copy of the worklo
 no collective on the data path); time is the maximum over ranks.
 
 ``--workload logp`` runs the second path instead, the compact-to-semantic log-probability (one step = its
-forward + backward over one microbatch of compact logit rows), with the same JSON keys.
+forward + backward over one microbatch of compact logit rows), ``--workload conv`` the tree-aware causal
+convolution that precedes the linear-attention core; both print the same JSON keys.
 
 ``--impl reference`` times the fp64 CPU oracle (oracle/), as it stands, on the host cores, on a
 bounded sample of the same workload.
@@ -696,6 +697,183 @@ def run_logp(args):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------------------
+# Third workload: tree-aware causal convolution before the linear-attention core (Section 4.2), `--workload conv`
+# --------------------------------------------------------------------------------------------------
+CONV_METRIC = "tree-aware causal conv fwd+bwd compact tokens/s"
+CONV_W = 4
+
+
+def conv_oracle_sample(small=False):
+    from oracle import conv_oracle
+    from workloads import CONFIGS, config_forest, make_conv_inputs, make_forest
+    D = 256 if small else 4096
+    fo = config_forest("cfg0b") if small else make_forest(CONFIGS["cfg1"]["build"]() * 2)
+    inp = make_conv_inputs(fo.n_tokens, D, CONV_W, "bf16", 0)
+    x, dy, W = (inp[n].double().numpy() for n in ("x", "dy", "W"))
+    t0 = time.perf_counter()
+    conv_oracle.conv_fwd(fo, x, W)
+    conv_oracle.conv_bwd(fo, x, W, dy)
+    dt = time.perf_counter() - t0
+    # compact tokens/s at the benchmark's channel count (the sample has D channels of 4096)
+    return {"value": fo.n_tokens * D / 4096 / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{fo.n_tokens} compact tokens ({'cfg0b tree' if small else '2 x cfg1 tree'}), {D} of 4096 channels, w={CONV_W}, fwd+bwd, {dt:.1f} s",
+            "seconds": dt}
+
+
+def run_conv_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    vals, secs, last = [], [], None
+    for i in range(args.warmup + args.steps):
+        last = conv_oracle_sample(small=True)
+        if i >= args.warmup:
+            vals.append(last["value"])
+            secs.append(last["seconds"])
+    value = statistics.mean(vals)
+    print(json.dumps({
+        "impl": "reference", "metric": CONV_METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(secs) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "conv", "D": 4096, "w": CONV_W},
+        "cpu_baseline": {"kind": last["kind"], "cores": last["cores"], "sample": last["sample"], "value": value,
+                         "unit": UNIT},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def run_conv(args):
+    """One step = forward + backward (dx, dW) of the width-4 depthwise convolution over cfg3's compact tokens,
+    D = 32 heads x 128 = 4096 channels (the q/k/v projections each see one such call)."""
+    import torch
+    import torch.distributed as dist
+
+    import paper_2608_28158_b200 as H
+    from workloads import config_forest, make_conv_inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    fo = config_forest(args.conv_trees)
+    C, D, w = fo.n_tokens, 4096, CONV_W
+    plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
+    t0 = time.perf_counter()
+    prev, nxt, cptr, crow = H.harts_conv_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len,
+                                               plan.row_of_token)
+    t_host = time.perf_counter() - t0
+    inp = make_conv_inputs(C, D, w, "bf16", 70 + rank, device="cuda")
+    idx = {n: torch.as_tensor(np.ascontiguousarray(a)).cuda() for n, a in
+           (("prev", prev), ("next", nxt), ("cptr", cptr), ("crow", crow))}
+    y, dx, dW = torch.empty_like(inp["x"]), torch.empty_like(inp["x"]), torch.empty_like(inp["W"])
+    scratch = torch.empty(H.harts_conv_scratch_bytes(D, w), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+
+    def step(marks=None):
+        a, b, c = ev(), ev(), ev()
+        a.record(stream)
+        H.harts_conv_fwd(inp["x"], inp["W"], idx["prev"], y)
+        b.record(stream)
+        H.harts_conv_bwd(inp["x"], inp["W"], inp["dy"], idx["next"], idx["cptr"], idx["crow"], dx, dW, scratch)
+        c.record(stream)
+        if marks is not None:
+            marks.append((a, b, c))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    marks = []
+    t_begin, t_end = ev(), ev()
+    with ClockSampler(local) as clocks:
+        for _ in range(args.warmup):
+            step()
+        barrier()
+        h0 = clocks.mark()
+        t_begin.record(stream)
+        for _ in range(args.steps):
+            step(marks)
+        t_end.record(stream)
+        barrier()
+        h1 = clocks.mark()
+    ms_step = t_begin.elapsed_time(t_end) / args.steps
+    fwd_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in marks)
+    bwd_ms = statistics.mean(b.elapsed_time(c) for _, b, c in marks)
+    e2e = None
+    if not args.no_e2e:
+        host = {n: torch.empty(inp[n].shape, dtype=inp[n].dtype, pin_memory=True) for n in ("x", "dy", "W")}
+        for n in host:
+            host[n].copy_(inp[n])
+        out_h = {"y": torch.empty(y.shape, dtype=y.dtype, pin_memory=True),
+                 "dx": torch.empty(y.shape, dtype=y.dtype, pin_memory=True), "dW": torch.empty(dW.shape, pin_memory=True)}
+        torch.cuda.synchronize()
+
+        def e2e_step():
+            for n in host:
+                inp[n].copy_(host[n], non_blocking=True)
+            step()
+            out_h["y"].copy_(y, non_blocking=True)
+            out_h["dx"].copy_(dx, non_blocking=True)
+            out_h["dW"].copy_(dW, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b = ev(), ev()
+        n_e2e = max(1, min(args.steps, args.e2e_steps))
+        a.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e2e = {"ms": a.elapsed_time(b) / n_e2e, "steps": n_e2e,
+               "h2d": sum(t.numel() * t.element_size() for t in host.values()),
+               "d2h": sum(t.numel() * t.element_size() for t in out_h.values())}
+        del host, out_h
+    if world > 1:
+        ms_step, e2e_ms = max_over_ranks([ms_step, e2e["ms"] if e2e else 0.0], "cuda")
+        if e2e:
+            e2e["ms"] = e2e_ms
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    unit = C * D * 2
+    fwd_bytes, bwd_bytes = 2 * unit + C * 4, 3 * unit + C * 4
+    achieved = bwd_bytes / (bwd_ms * 1e-3) / 1e9
+    clock = clocks.summary(h0, h1)
+    if not clock["samples"]:
+        clock = clocks.summary()
+    line = {
+        "metric": CONV_METRIC, "value": C * world / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "conv", "trees": args.conv_trees, "compact_tokens": C, "D": D, "w": w,
+                   "l2": f"inputs larger than L2 ({unit / 2**30:.2f} GiB per tensor)", "host_index_ms": t_host * 1e3},
+        "roofline": {"bound": "hbm", "kernel": "conv_bwd_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                     "algorithmic_bytes_per_launch": bwd_bytes, "peak_source": peaks["source"],
+                     "forward": {"achieved": fwd_bytes / (fwd_ms * 1e-3) / 1e9,
+                                 "frac": fwd_bytes / (fwd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                     "whole_path": {"roof_ms": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                                    "frac_strict": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms_step}},
+        "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms},
+        "gpu_launches": 3 * args.steps,
+        "clocks": clock,
+    }
+    if e2e:
+        line["e2e"] = {"value": C * world / (e2e["ms"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
+                       "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"], "pinned_host_memory": True}
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = conv_oracle_sample()
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -709,10 +887,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-trajwise", action="store_true")
     ap.add_argument("--logp-rows", type=int, default=LOGP_ROWS, help="compact-row capacity of the logp workload")
+    ap.add_argument("--conv-trees", default="cfg3", help="forest of the conv workload (cfg2: a small case for captures)")
     ap.add_argument("--per-config", action="store_true", help="also print a table over all configurations to stderr")
     args = ap.parse_args()
     if args.workload == "logp":
         (run_logp_reference if args.impl == "reference" else run_logp)(args)
+    elif args.workload == "conv":
+        (run_conv_reference if args.impl == "reference" else run_conv)(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -66,3 +66,14 @@ def make_logp_grad(n_pos: int, seed: int, device="cpu", keep: float = 0.6):
     adv = torch.randn(n_pos, generator=gen, device=device, dtype=torch.float32)
     mask = torch.rand(n_pos, generator=gen, device=device) < keep
     return torch.where(mask, adv / max(n_pos, 1), torch.zeros_like(adv))
+
+
+def make_conv_inputs(n_rows: int, D: int, w: int, dtype: str, seed: int, device="cpu"):
+    """Inputs of the short causal convolution: x, dy ~ N(0,1) rounded to the run dtype, W ~ N(0,1)/sqrt(w) fp32."""
+    dt = _DTYPES[dtype]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(3000017 * (seed + 1))
+    x = torch.randn(n_rows, D, generator=gen, device=device, dtype=torch.float32).to(dt)
+    dy = torch.randn(n_rows, D, generator=gen, device=device, dtype=torch.float32).to(dt)
+    W = torch.randn(D, w, generator=gen, device=device, dtype=torch.float32) / (w ** 0.5)
+    return {"x": x, "dy": dy, "W": W}
