@@ -19,6 +19,10 @@ Pins (see tests/test_oracle_*.py, tests/test_plan_oracle.py):
   * conv_oracle -- tree-aware causal convolution (Section 4.2): torch conv1d on every expanded
                    trajectory, autograd through the expansion, identity/shift filters on the
                    five-node tree, central differences.
+  * attn_oracle -- full attention on compact tokens (Section 3.4, Eqs. 21-22): torch causal
+                   scaled_dot_product_attention on every expanded trajectory with autograd
+                   through the expansion, the bottom-right mask of a branch view, equal-keys
+                   closed form, central differences.
   * Appendix planning cases I-III: parity unpinned (the trees' token counts were only in
                    the figures); only the printed totals are checked for self-consistency.
 """
