@@ -19,28 +19,33 @@ import numpy as np
 from .conv_oracle import predecessors
 
 
+def _path(pred, t):
+    chain = []
+    a = t
+    while a >= 0:
+        chain.append(a)
+        a = pred[a]
+    return np.asarray(chain[::-1], np.int64)
+
+
 def paths(forest):
     """path[t] = canonical indices of the tokens t attends to, root first, t last."""
     pred = predecessors(forest)
-    out = []
-    for t in range(forest.n_tokens):
-        chain = []
-        a = t
-        while a >= 0:
-            chain.append(a)
-            a = pred[a]
-        out.append(np.asarray(chain[::-1], np.int64))
-    return out
+    return [_path(pred, t) for t in range(forest.n_tokens)]
 
 
-def attn_fwd(forest, q, k, v, scale):
-    """q [C,Hq,d], k,v [C,Hkv,d] canonical order -> (o [C,Hq,d], lse [C,Hq]) in fp64; lse in natural log units."""
+def attn_fwd(forest, q, k, v, scale, tokens=None):
+    """q [C,Hq,d], k,v [C,Hkv,d] canonical order -> (o [C,Hq,d], lse [C,Hq]) in fp64; lse in natural log units.
+    tokens: compute only these queries (the other rows of the result stay zero)."""
     q, k, v = (np.asarray(a, np.float64) for a in (q, k, v))
     C, Hq, d = q.shape
     G = Hq // k.shape[1]
     o = np.zeros((C, Hq, v.shape[2]))
     lse = np.zeros((C, Hq))
-    for t, path in enumerate(paths(forest)):
+    pred = predecessors(forest)
+    for t in (range(C) if tokens is None else tokens):
+        t = int(t)
+        path = _path(pred, t)
         for h in range(Hq):
             s = scale * (k[path, h // G] @ q[t, h])
             m = s.max()
@@ -56,7 +61,9 @@ def attn_bwd(forest, q, k, v, dO, scale):
     C, Hq, d = q.shape
     G = Hq // k.shape[1]
     dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
-    for t, path in enumerate(paths(forest)):
+    pred = predecessors(forest)
+    for t in range(C):
+        path = _path(pred, t)
         for h in range(Hq):
             hk = h // G
             s = scale * (k[path, hk] @ q[t, h])

@@ -14,3 +14,4 @@ from .logp import (  # noqa: F401
     harts_logp_positions, harts_logp_csr, harts_logp_fwd, harts_logp_bwd, harts_logp_fwd_shard, harts_logp_combine,
 )
 from .conv import harts_conv_index, harts_conv_fwd, harts_conv_scratch_bytes, harts_conv_bwd  # noqa: F401
+from .attn import AttnIndex, harts_attn_index, harts_attn_fwd, harts_attn_bwd  # noqa: F401

@@ -1,0 +1,355 @@
+// Forward of full attention on compact tokens (Section 3.4, Eqs. 21-22) for bf16, head dimension 128, on tcgen05.
+//
+// One work item = (piece, tile of 128 query rows, query head).  The CTA walks the key/value rows that tile sees --
+// the piece's ancestor rows (all visible), then the piece's own rows up to the diagonal (Eq. 22) -- in tiles of 64:
+//     S = Q K^T            tcgen05.mma, operands in shared memory (TMA, 128-byte swizzle), S in tensor memory
+//     P = exp2(S - m)      four warps, one query row per thread; P goes back to tensor memory as bf16 over S
+//     O += P V             tcgen05.mma with P as the tensor-memory operand
+// with the running maximum m raised only when a row's maximum grows by more than 2^8 (the values of P stay
+// representable and O is rescaled rarely).  K/V tiles are double-buffered; two CTAs share an SM, so one CTA's
+// softmax overlaps the other's MMAs.  Every wait is bounded.
+#include "kernels.h"
+#include "tc_common.cuh"
+
+#include "../../include/harts_attn.h"
+
+namespace harts {
+
+int32_t make_row_map(CUtensorMap* map, const void* base, int64_t rows, int32_t H);
+int sm_count();
+
+namespace {
+
+using namespace tc;
+
+constexpr int BQ = 128, BK = 64, D = 128;
+constexpr int NS = 128;                 // softmax threads (4 warps), thread = query row = tensor-memory lane
+constexpr int NT = NS + 32;             // plus one warp whose first lane issues TMA and MMA
+constexpr int Q_BYTES = BQ * D * 2;     // 32 KB: two panels [128 rows][64 columns]
+constexpr int KV_BYTES = BK * D * 2;    // 16 KB: two panels [64 rows][64 columns]
+constexpr int COL_S = 0, COL_O = 128, TMEM_COLS = 256;
+constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
+constexpr float RAISE = 8.f;            // the reference maximum follows the row maximum in steps of at least 2^8
+constexpr int NO_DIAG = -(1 << 28);
+
+struct Smem {
+    static constexpr int q = 0, k0 = Q_BYTES, v0 = k0 + 2 * KV_BYTES, misc = v0 + 2 * KV_BYTES;
+    static constexpr int bytes = misc + 256;
+};
+struct Misc {
+    uint64_t bar_q, bar_kv[2], bar_s, bar_p, bar_o;
+    uint32_t tmem;
+};
+
+struct Index {
+    const int32_t *piece_row0, *piece_len, *anc_ptr, *anc_row0, *anc_len, *q_item;
+    int n_q_items;
+};
+
+// The t-th key tile of an item: rows [row, row + n_valid), and the diagonal shift (key column j is visible to
+// query row i iff j + shift <= i; NO_DIAG for ancestor rows).
+struct KvTile {
+    int row, n_valid, shift;
+};
+
+struct TileWalk {       // enumerates the key tiles of one item in order
+    const Index& ix;
+    int run, run_end, off, own_row0, own_end, q0;
+    bool in_own;
+    __device__ TileWalk(const Index& ix_, int piece, int qt) : ix(ix_) {
+        run = ix.anc_ptr[piece];
+        run_end = ix.anc_ptr[piece + 1];
+        off = 0;
+        own_row0 = ix.piece_row0[piece];
+        q0 = qt * BQ;
+        own_end = min(ix.piece_len[piece], q0 + BQ);      // own rows up to the end of the query tile
+        in_own = run == run_end;
+    }
+    __device__ bool next(KvTile& t) {
+        if (!in_own) {
+            const int len = ix.anc_len[run];
+            t.row = ix.anc_row0[run] + off;
+            t.n_valid = min(BK, len - off);
+            t.shift = NO_DIAG;
+            off += BK;
+            if (off >= len) {
+                off = 0;
+                if (++run == run_end) in_own = true;
+            }
+            return true;
+        }
+        if (off >= own_end) return false;
+        t.row = own_row0 + off;
+        t.n_valid = min(BK, own_end - off);
+        t.shift = off - q0;
+        off += BK;
+        return true;
+    }
+};
+
+__global__ void __launch_bounds__(NT, 2)
+attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant__ CUtensorMap map_q,
+                const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                const __grid_constant__ CUtensorMap map_o, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
+                int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    unsigned char* sQ = smem + Smem::q;
+    Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool is_softmax = warp < NS / 32;
+    const bool is_issuer = tid == NS;
+
+    if (tid == 0) {
+        mbar_init(&m.bar_q, 1);
+        mbar_init(&m.bar_kv[0], 1);
+        mbar_init(&m.bar_kv[1], 1);
+        mbar_init(&m.bar_s, 1);
+        mbar_init(&m.bar_p, NS / 32);
+        mbar_init(&m.bar_o, 1);
+        fence_barrier_init();
+    }
+    if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = m.tmem;
+    const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+
+    constexpr uint32_t I_S = instr_desc(BQ, BK, 0, 0);      // S[128 x 64] = Q (K-major) . K (K-major)
+    constexpr uint32_t I_O = instr_desc(BQ, D, 0, 1);       // O[128 x 128] += P (tensor memory) . V (rows = keys)
+    const uint32_t aQ = smem_u32(sQ);
+    const uint64_t dQ = desc_kmajor_base(aQ);
+
+    uint32_t ph_q = 0, ph_kv[2] = {0, 0}, ph_s = 0, ph_p = 0, ph_o = 0;
+    const int n_work = ix.n_q_items * Hq;
+    for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
+        const int item = w / Hq, h = w % Hq, hk = h / G;
+        const int piece = ix.q_item[2 * item], qt = ix.q_item[2 * item + 1];
+        const int q_row0 = ix.piece_row0[piece] + qt * BQ;
+        const int q_valid = min(BQ, ix.piece_len[piece] - qt * BQ);
+
+        if (is_issuer) {
+            // ---- producer + MMA issue ------------------------------------------------------------------------------
+            TileWalk load_walk(ix, piece, qt), walk(ix, piece, qt);
+            KvTile lt, t;
+            auto load_kv = [&](int stage, const KvTile& kt) {
+                unsigned char* sK = smem + Smem::k0 + stage * KV_BYTES;
+                unsigned char* sV = smem + Smem::v0 + stage * KV_BYTES;
+                mbar_expect_tx(&m.bar_kv[stage], 2 * KV_BYTES);
+                for (int p = 0; p < 2; p++) {
+                    tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, kt.row, &m.bar_kv[stage]);
+                    tma_load_3d(sV + p * (KV_BYTES / 2), &map_v, p * 64, hk, kt.row, &m.bar_kv[stage]);
+                }
+            };
+            mbar_expect_tx(&m.bar_q, Q_BYTES);
+            for (int p = 0; p < 2; p++)
+                for (int r = 0; r < 2; r++)
+                    tma_load_3d(sQ + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_q, p * 64, h, q_row0 + r * 64, &m.bar_q);
+            bool more_loads = load_walk.next(lt);
+            if (more_loads) load_kv(0, lt);
+            more_loads = more_loads && load_walk.next(lt);
+            if (more_loads) load_kv(1, lt);
+            mbar_wait(&m.bar_q, ph_q, status);
+            ph_q ^= 1;
+            int n = 0;
+            bool have = walk.next(t);
+            // S of the first tile
+            if (have) {
+                mbar_wait(&m.bar_kv[0], ph_kv[0], status);
+                ph_kv[0] ^= 1;
+                tc_fence_after();
+                const uint64_t dK = desc_kmajor_base(smem_u32(smem + Smem::k0));
+#pragma unroll
+                for (int ks = 0; ks < 8; ks++)
+                    mma_ss(tmem + COL_S, dQ + kstep_kmajor<BQ>(ks), dK + kstep_kmajor<BK>(ks), I_S, ks > 0);
+                mma_commit(&m.bar_s);
+                ph_s ^= 1;                                    // this thread does not wait for S(0)
+            }
+            while (have) {
+                const int stage = n & 1;
+                KvTile t_next;
+                const bool have_next = walk.next(t_next);
+                // O += P V for tile n as soon as the softmax warps have written P
+                mbar_wait(&m.bar_p, ph_p, status);
+                ph_p ^= 1;
+                tc_fence_after();
+                const uint64_t dV = desc_mnmajor_base<BK>(smem_u32(smem + Smem::v0 + stage * KV_BYTES));
+#pragma unroll
+                for (int ks = 0; ks < 4; ks++)
+                    mma_ts(tmem + COL_O, tmem + COL_S + ks * 8, dV + kstep_mnmajor(ks), I_O, n > 0 || ks > 0);
+                if (have_next) {
+                    // S of tile n+1 queues behind it (it overwrites P only after the MMAs above have read it)
+                    const int s2 = stage ^ 1;
+                    mbar_wait(&m.bar_kv[s2], ph_kv[s2], status);
+                    ph_kv[s2] ^= 1;
+                    tc_fence_after();
+                    const uint64_t dK = desc_kmajor_base(smem_u32(smem + Smem::k0 + s2 * KV_BYTES));
+#pragma unroll
+                    for (int ks = 0; ks < 8; ks++)
+                        mma_ss(tmem + COL_S, dQ + kstep_kmajor<BQ>(ks), dK + kstep_kmajor<BK>(ks), I_S, ks > 0);
+                    mma_commit(&m.bar_s);
+                } else {
+                    mma_commit(&m.bar_o);
+                }
+                // stage `stage` is free once the PV MMAs are done: known when S(n+1) completes (in order) or at bar_o
+                if (more_loads) {
+                    more_loads = load_walk.next(lt);
+                    if (more_loads) {
+                        // wait for the MMAs that read this stage: they precede S(n+1), whose completion bar_s reports
+                        mbar_wait(&m.bar_s, ph_s, status);
+                        load_kv(stage, lt);
+                    }
+                }
+                if (have_next) ph_s ^= 1;
+                t = t_next;
+                have = have_next;
+                n++;
+            }
+        }
+
+        float m_ref = -INFINITY, l_sum = 0.f;
+        if (is_softmax) {
+            TileWalk walk(ix, piece, qt);
+            KvTile t;
+            const int i = tid;                                // query row inside the tile
+            int n = 0;
+            while (walk.next(t)) {
+                mbar_wait(&m.bar_s, ph_s, status);
+                ph_s ^= 1;
+                tc_fence_after();
+                const int limit = min(t.n_valid, t.shift == NO_DIAG ? BK : i - t.shift + 1);   // visible: j < limit
+                // pass 1: row maximum
+                float mx = -INFINITY;
+                uint32_t x[32];
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    tmem_ld32(tm_lane + COL_S + c * 32, x);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; e++)
+                        if (c * 32 + e < limit) mx = fmaxf(mx, __uint_as_float(x[e]));
+                }
+                mx *= scale_log2;
+                // raise the reference only by big steps; the whole warp decides together whether O must be rescaled
+                const bool raise = mx > m_ref + RAISE || m_ref == -INFINITY;
+                if (__any_sync(0xffffffffu, raise && n > 0)) {
+                    const float m_new = raise ? mx : m_ref;
+                    const float alpha = m_new == -INFINITY ? 1.f : ex2(m_ref - m_new);   // m_ref = -inf: O and l are still 0
+                    l_sum *= alpha;
+#pragma unroll
+                    for (int c = 0; c < 4; c++) {
+                        tmem_ld32(tm_lane + COL_O + c * 32, x);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; e++) x[e] = __float_as_uint(__uint_as_float(x[e]) * alpha);
+                        tmem_st32(tm_lane + COL_O + c * 32, x);
+                    }
+                    m_ref = m_new;
+                } else if (raise) {
+                    m_ref = mx;                               // first tile: nothing accumulated yet
+                }
+                // pass 2: P = exp2(s - m_ref), written over S as bf16 pairs
+                const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    tmem_ld32(tm_lane + COL_S + c * 32, x);
+                    tmem_ld_wait();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const float p0 = c * 32 + e < limit ? ex2(fmaf(__uint_as_float(x[e]), scale_log2, neg_m)) : 0.f;
+                        const float p1 = c * 32 + e + 1 < limit ? ex2(fmaf(__uint_as_float(x[e + 1]), scale_log2, neg_m)) : 0.f;
+                        pk[e >> 1] = pack_bf16(p0, p1);
+                        // the sum uses the rounded values the MMA will see
+                        l_sum += __uint_as_float(pk[e >> 1] << 16) + __uint_as_float(pk[e >> 1] & 0xffff0000u);
+                    }
+                    tmem_st16(tm_lane + COL_S + c * 16, pk);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&m.bar_p);
+                n++;
+            }
+            // ---- epilogue: O / l -> bf16, lse ----------------------------------------------------------------------
+            mbar_wait(&m.bar_o, ph_o, status);
+            tc_fence_after();
+            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            const bool full = q_valid == BQ;
+            if (i < q_valid) lse[(size_t)(q_row0 + i) * Hq + h] = (m_ref + log2f(l_sum)) * LN2;
+#pragma unroll
+            for (int c = 0; c < 4; c++) {
+                uint32_t x[32];
+                tmem_ld32(tm_lane + COL_O + c * 32, x);
+                tmem_ld_wait();
+#pragma unroll
+                for (int v4 = 0; v4 < 4; v4++) {
+                    uint4 pk;
+                    pk.x = pack_bf16(__uint_as_float(x[v4 * 8 + 0]) * inv, __uint_as_float(x[v4 * 8 + 1]) * inv);
+                    pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]) * inv, __uint_as_float(x[v4 * 8 + 3]) * inv);
+                    pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]) * inv, __uint_as_float(x[v4 * 8 + 5]) * inv);
+                    pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]) * inv, __uint_as_float(x[v4 * 8 + 7]) * inv);
+                    const int col = c * 32 + v4 * 8;
+                    if (full)       // staged over the Q tile in the swizzled panel layout, for TMA stores
+                        *reinterpret_cast<uint4*>(sQ + (col >> 6) * (Q_BYTES / 2) + sw128_chunk(i, (col & 63) >> 3)) = pk;
+                    else if (i < q_valid)
+                        *reinterpret_cast<uint4*>(o + ((size_t)(q_row0 + i) * Hq + h) * D + col) = pk;
+                }
+            }
+            if (full) fence_async_smem();
+        }
+        ph_o ^= 1;
+        tc_fence_before();
+        __syncthreads();                                      // O staged; tensor memory and Q tile free for the next item
+        tc_fence_after();
+        if (is_issuer && q_valid == BQ) {
+            for (int p = 0; p < 2; p++)
+                for (int r = 0; r < 2; r++)
+                    tma_store_3d(&map_o, sQ + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), p * 64, h, q_row0 + r * 64);
+            tma_store_commit();
+            tma_store_wait_read();                            // the Q tile is reloaded right away
+        }
+        __syncthreads();
+    }
+    if (is_issuer) tma_store_wait_all();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc<TMEM_COLS>(tmem);
+}
+
+}  // namespace
+
+int32_t attn_index_ok(const int32_t* host_index) {
+    return host_index && host_index[0] >= 0 && host_index[6] >= HARTS_ATTN_HEADER_WORDS ? HARTS_OK : HARTS_EINVAL;
+}
+
+int32_t attn_fwd_launch(const int32_t* hi, const int32_t* di, const void* q, const void* k, const void* v, void* o,
+                        float* lse, int Hq, int Hkv, float scale, int32_t* status, cudaStream_t st) {
+    const int n_rows = hi[0];
+    if (n_rows == 0 || hi[4] == 0) return HARTS_OK;
+    CUtensorMap mq, mk, mv, mo;
+    int32_t rc;
+    if ((rc = make_row_map(&mq, q, n_rows, Hq)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mk, k, n_rows, Hkv)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mv, v, n_rows, Hkv)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mo, o, n_rows, Hq)) != HARTS_OK) return rc;
+    if (cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+        cudaSuccess)
+        return HARTS_ECUDA;
+    Index ix;
+    ix.piece_row0 = di + hi[8];
+    ix.piece_len = di + hi[9];
+    ix.anc_ptr = di + hi[11];
+    ix.anc_row0 = di + hi[12];
+    ix.anc_len = di + hi[13];
+    ix.q_item = di + hi[16];
+    ix.n_q_items = hi[4];
+    const long long n_work = (long long)ix.n_q_items * Hq;
+    const int grid = (int)(n_work < 2LL * sm_count() ? n_work : 2LL * sm_count());
+    attn_fwd_kernel<<<grid, NT, Smem::bytes + 1024, st>>>(ix, Hq, Hq / Hkv, scale * LOG2E, mq, mk, mv, mo,
+                                                         (__nv_bfloat16*)o, lse, status);
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+}  // namespace harts

@@ -77,3 +77,12 @@ def make_conv_inputs(n_rows: int, D: int, w: int, dtype: str, seed: int, device=
     dy = torch.randn(n_rows, D, generator=gen, device=device, dtype=torch.float32).to(dt)
     W = torch.randn(D, w, generator=gen, device=device, dtype=torch.float32) / (w ** 0.5)
     return {"x": x, "dy": dy, "W": W}
+
+
+def make_attn_inputs(n_rows: int, Hq: int, Hkv: int, d: int, dtype: str, seed: int, device="cpu"):
+    """q, k, v, dO ~ N(0,1) rounded to the run dtype (scores scaled by 1/sqrt(d) have unit variance)."""
+    dt = _DTYPES[dtype]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(5000011 * (seed + 1))
+    mk = lambda h: torch.randn(n_rows, h, d, generator=gen, device=device, dtype=torch.float32).to(dt)  # noqa: E731
+    return {"q": mk(Hq), "k": mk(Hkv), "v": mk(Hkv), "dO": mk(Hq)}
