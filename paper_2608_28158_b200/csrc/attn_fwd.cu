@@ -12,6 +12,7 @@
 #include "tc_common.cuh"
 
 #include "../../include/harts_attn.h"
+#include "attn_common.cuh"
 
 namespace harts {
 
@@ -22,7 +23,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int BQ = 128, BK = 64, D = 128;
+using namespace attn;
 constexpr int NS = 128;                 // softmax threads (4 warps), thread = query row = tensor-memory lane
 constexpr int NT = NS + 32;             // plus one warp whose first lane issues TMA and MMA
 constexpr int Q_BYTES = BQ * D * 2;     // 32 KB: two panels [128 rows][64 columns]
@@ -30,7 +31,6 @@ constexpr int KV_BYTES = BK * D * 2;    // 16 KB: two panels [64 rows][64 column
 constexpr int COL_S = 0, COL_O = 128, TMEM_COLS = 256;
 constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
 constexpr float RAISE = 8.f;            // the reference maximum follows the row maximum in steps of at least 2^8
-constexpr int NO_DIAG = -(1 << 28);
 
 struct Smem {
     static constexpr int q = 0, k0 = Q_BYTES, v0 = k0 + 2 * KV_BYTES, misc = v0 + 2 * KV_BYTES;
@@ -39,52 +39,6 @@ struct Smem {
 struct Misc {
     uint64_t bar_q, bar_kv[2], bar_s, bar_p, bar_o;
     uint32_t tmem;
-};
-
-struct Index {
-    const int32_t *piece_row0, *piece_len, *anc_ptr, *anc_row0, *anc_len, *q_item;
-    int n_q_items;
-};
-
-// The t-th key tile of an item: rows [row, row + n_valid), and the diagonal shift (key column j is visible to
-// query row i iff j + shift <= i; NO_DIAG for ancestor rows).
-struct KvTile {
-    int row, n_valid, shift;
-};
-
-struct TileWalk {       // enumerates the key tiles of one item in order
-    const Index& ix;
-    int run, run_end, off, own_row0, own_end, q0;
-    bool in_own;
-    __device__ TileWalk(const Index& ix_, int piece, int qt) : ix(ix_) {
-        run = ix.anc_ptr[piece];
-        run_end = ix.anc_ptr[piece + 1];
-        off = 0;
-        own_row0 = ix.piece_row0[piece];
-        q0 = qt * BQ;
-        own_end = min(ix.piece_len[piece], q0 + BQ);      // own rows up to the end of the query tile
-        in_own = run == run_end;
-    }
-    __device__ bool next(KvTile& t) {
-        if (!in_own) {
-            const int len = ix.anc_len[run];
-            t.row = ix.anc_row0[run] + off;
-            t.n_valid = min(BK, len - off);
-            t.shift = NO_DIAG;
-            off += BK;
-            if (off >= len) {
-                off = 0;
-                if (++run == run_end) in_own = true;
-            }
-            return true;
-        }
-        if (off >= own_end) return false;
-        t.row = own_row0 + off;
-        t.n_valid = min(BK, own_end - off);
-        t.shift = off - q0;
-        off += BK;
-        return true;
-    }
 };
 
 __global__ void __launch_bounds__(NT, 2)
@@ -337,14 +291,7 @@ int32_t attn_fwd_launch(const int32_t* hi, const int32_t* di, const void* q, con
     if (cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
-    Index ix;
-    ix.piece_row0 = di + hi[8];
-    ix.piece_len = di + hi[9];
-    ix.anc_ptr = di + hi[11];
-    ix.anc_row0 = di + hi[12];
-    ix.anc_len = di + hi[13];
-    ix.q_item = di + hi[16];
-    ix.n_q_items = hi[4];
+    const Index ix = make_index(hi, di);
     const long long n_work = (long long)ix.n_q_items * Hq;
     const int grid = (int)(n_work < 2LL * sm_count() ? n_work : 2LL * sm_count());
     attn_fwd_kernel<<<grid, NT, Smem::bytes + 1024, st>>>(ix, Hq, Hq / Hkv, scale * LOG2E, mq, mk, mv, mo,

@@ -79,3 +79,35 @@ def test_forward_cfg1_sampled_queries():
     assert _rel(got[tok], o_ref[tok]) <= 5e-3
     assert np.abs(lse[rows].double().cpu().numpy()[tok] - lse_ref[tok]).max() <= 2e-3
     assert bool(torch.isfinite(o.float()).all()) and bool(torch.isfinite(lse).all())
+
+
+def _backward(phys, index, o, lse):
+    dq = torch.full_like(phys["q"], float("nan")); dk = torch.full_like(phys["k"], float("nan"))
+    dv = torch.full_like(phys["v"], float("nan"))
+    delta = torch.empty(phys["q"].shape[:2], device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    H.harts_attn_bwd(index, phys["q"], phys["k"], phys["v"], o, lse, phys["dO"], dq, dk, dv, delta, SCALE, dev_status=status)
+    H.harts_la_check(status)
+    return dq, dk, dv
+
+
+def _check_backward(fo, Hq, Hkv, seed, use_plan=True):
+    inp, phys, index, rows = _setup(fo, Hq, Hkv, seed, use_plan)
+    o, lse = _forward(phys, index)
+    dq, dk, dv = _backward(phys, index, o, lse)
+    ref = ao.attn_bwd(fo, *(inp[n].double().numpy() for n in ("q", "k", "v", "dO")), SCALE)
+    errs = [_rel(x[rows].double().cpu().numpy(), r) for x, r in zip((dq, dk, dv), ref)]
+    assert max(errs) <= 1e-2, errs
+    return errs
+
+
+@pytest.mark.parametrize("name,Hq,Hkv", [("cfg0", 1, 1), ("cfg0b", 2, 2), ("cfg0b", 4, 2)])
+def test_backward_small_trees(name, Hq, Hkv):
+    _check_backward(config_forest(name), Hq, Hkv, 4)
+
+
+def test_backward_bushy_random_forest():
+    rnd = random.Random(6)
+    fo = make_forest([random_tree(rnd, 9, 300) for _ in range(3)] + [([-1], [0], [1])])
+    _check_backward(fo, 2, 1, 5, use_plan=False)
+    _check_backward(fo, 2, 2, 5, use_plan=True)
