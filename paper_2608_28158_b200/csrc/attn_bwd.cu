@@ -28,10 +28,10 @@ namespace {
 using namespace tc;
 using namespace attn;
 
-constexpr int NS = 128, NT = NS + 32;
+constexpr int NS = 256, NT = NS + 64;     // 8 element-wise warps: warp w and w + 4 share a lane quarter and split the columns
 constexpr int Q_BYTES = BQ * D * 2;       // 32 KB
 constexpr int KV_BYTES = BK * D * 2;      // 16 KB
-constexpr int STAGES = 3;
+constexpr int STAGES = 4;
 constexpr float LOG2E = 1.4426950408889634f;
 
 __global__ void __launch_bounds__(256) delta_kernel(const __nv_bfloat16* __restrict__ o,
@@ -80,7 +80,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
     unsigned char* sDO = smem + SmemQ::dO;
     MiscQ& m = *reinterpret_cast<MiscQ*>(smem + SmemQ::misc);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const bool is_softmax = warp < NS / 32, is_issuer = tid == NS;
+    const bool is_softmax = warp < NS / 32, is_issuer = tid == NS, is_producer = tid == NS + 32;
     if (tid == 0) {
         mbar_init(&m.bar_q, 1);
         for (int s = 0; s < STAGES; s++) { mbar_init(&m.bar_kv[s], 1); mbar_init(&m.bar_free[s], 1); }
@@ -99,7 +99,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
     const uint64_t dQd = desc_kmajor_base(smem_u32(sQ)), dDOd = desc_kmajor_base(smem_u32(sDO));
     const float scale_log2 = scale * LOG2E;
 
-    uint32_t ph_q = 0, ph_kv[STAGES] = {0, 0, 0}, ph_free[STAGES] = {0, 0, 0}, ph_s[2] = {0, 0}, ph_p[2] = {0, 0}, ph_o = 0;
+    uint32_t ph_q = 0, ph_kv[STAGES] = {}, ph_free[STAGES] = {}, ph_s[2] = {0, 0}, ph_p[2] = {0, 0}, ph_o = 0;
     const int n_work = ix.n_q_items * Hq;
     for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
         const int item = w / Hq, h = w % Hq, hk = h / G;
@@ -107,18 +107,34 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
         const int q_row0 = ix.piece_row0[piece] + qt * BQ;
         const int q_valid = min(BQ, ix.piece_len[piece] - qt * BQ);
 
-        if (is_issuer) {
-            TileWalk load_walk(ix, piece, qt), walk(ix, piece, qt);
-            KvTile lt, t;
-            auto load_kv = [&](int stage, const KvTile& kt) {
+        if (is_producer) {
+            // ---- TMA producer: Q and dO tiles, then the key/value tiles STAGES deep ---------------------------------
+            TileWalk lw(ix, piece, qt);
+            KvTile lt;
+            mbar_expect_tx(&m.bar_q, 2 * Q_BYTES);
+            for (int p = 0; p < 2; p++)
+                for (int r = 0; r < 2; r++) {
+                    tma_load_3d(sQ + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_q, p * 64, h, q_row0 + r * 64, &m.bar_q);
+                    tma_load_3d(sDO + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_do, p * 64, h, q_row0 + r * 64, &m.bar_q);
+                }
+            for (int n = 0; lw.next(lt); n++) {
+                const int stage = n % STAGES;
+                if (n >= STAGES) {
+                    mbar_wait(&m.bar_free[stage], ph_free[stage], status);
+                    ph_free[stage] ^= 1;
+                }
                 unsigned char* sK = smem + SmemQ::k0 + stage * KV_BYTES;
                 unsigned char* sV = smem + SmemQ::v0 + stage * KV_BYTES;
                 mbar_expect_tx(&m.bar_kv[stage], 2 * KV_BYTES);
                 for (int p = 0; p < 2; p++) {
-                    tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, kt.row, &m.bar_kv[stage]);
-                    tma_load_3d(sV + p * (KV_BYTES / 2), &map_v, p * 64, hk, kt.row, &m.bar_kv[stage]);
+                    tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, lt.row, &m.bar_kv[stage]);
+                    tma_load_3d(sV + p * (KV_BYTES / 2), &map_v, p * 64, hk, lt.row, &m.bar_kv[stage]);
                 }
-            };
+            }
+        }
+        if (is_issuer) {
+            // ---- MMA issue: this thread does nothing else, a tcgen05.mma holds it until the pipe has room ---------
+            const int n_tiles = TileWalk(ix, piece, qt).count();
             auto issue_s = [&](int n) {      // S(n) and dP(n) into buffer n & 1
                 const int stage = n % STAGES, b = n & 1;
                 mbar_wait(&m.bar_kv[stage], ph_kv[stage], status);
@@ -134,26 +150,11 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                     mma_ss(tmem + b * 128 + 64, dDOd + kstep_kmajor<BQ>(ks), dV + kstep_kmajor<BK>(ks), I_S, ks > 0);
                 mma_commit(&m.bar_s[b]);
             };
-            mbar_expect_tx(&m.bar_q, 2 * Q_BYTES);
-            for (int p = 0; p < 2; p++)
-                for (int r = 0; r < 2; r++) {
-                    tma_load_3d(sQ + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_q, p * 64, h, q_row0 + r * 64, &m.bar_q);
-                    tma_load_3d(sDO + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_do, p * 64, h, q_row0 + r * 64, &m.bar_q);
-                }
-            bool more_loads = true;
-            for (int s = 0; s < STAGES && more_loads; s++) {
-                more_loads = load_walk.next(lt);
-                if (more_loads) load_kv(s, lt);
-            }
             mbar_wait(&m.bar_q, ph_q, status);
             ph_q ^= 1;
-            const int n_tiles = walk.count();
-            bool have = walk.next(t);
-            if (have) issue_s(0);
-            for (int n = 0; have; n++) {
-                KvTile t_next;
-                const bool have_next = walk.next(t_next);
-                if (have_next) issue_s(n + 1);            // runs under the element-wise pass of tile n
+            issue_s(0);
+            for (int n = 0; n < n_tiles; n++) {
+                if (n + 1 < n_tiles) issue_s(n + 1);            // runs under the element-wise pass of tile n
                 const int stage = n % STAGES, b = n & 1;
                 mbar_wait(&m.bar_p[b], ph_p[b], status);
                 ph_p[b] ^= 1;
@@ -161,38 +162,26 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                 const uint64_t dKm = desc_mnmajor_base<BK>(smem_u32(smem + SmemQ::k0 + stage * KV_BYTES));
 #pragma unroll
                 for (int ks = 0; ks < 4; ks++)
-                    mma_ts(tmem + COL_DQ, tmem + b * 128 + ks * 8, dKm + kstep_mnmajor(ks), I_DQ, n > 0 || ks > 0);
+                    mma_ts(tmem + COL_DQ, tmem + b * 128 + (ks >> 1) * 32 + (ks & 1) * 8, dKm + kstep_mnmajor(ks), I_DQ, n > 0 || ks > 0);
                 if (n + STAGES < n_tiles) mma_commit(&m.bar_free[stage]);     // this stage will be refilled
-                if (!have_next) mma_commit(&m.bar_o);
-                // the stage of tile n-1 is free once dQ(n-1) is done: refill it with tile n+2
-                if (n >= 1 && more_loads) {
-                    more_loads = load_walk.next(lt);
-                    if (more_loads) {
-                        const int sf = (n - 1) % STAGES;
-                        mbar_wait(&m.bar_free[sf], ph_free[sf], status);
-                        ph_free[sf] ^= 1;
-                        load_kv(sf, lt);
-                    }
-                }
-                have = have_next;
+                if (n + 1 == n_tiles) mma_commit(&m.bar_o);
             }
         }
         if (is_softmax) {
             TileWalk walk(ix, piece, qt);
             KvTile t;
-            const int i = tid;
+            const int i = tid & 127, c = tid >> 7;           // query row, and which 32 of a tile's 64 key columns
             const bool row_ok = i < q_valid;
             // rows past the end of the piece: lse = +inf makes every probability 0
             const float lse2 = row_ok ? lse[(size_t)(q_row0 + i) * Hq + h] * LOG2E : INFINITY;
             const float dl = row_ok ? delta[(size_t)(q_row0 + i) * Hq + h] : 0.f;
             for (int n = 0; walk.next(t); n++) {
                 const int b = n & 1;
-                mbar_wait(&m.bar_s[b], ph_s[b], status);
+                mbar_wait_warp(&m.bar_s[b], ph_s[b], status);
                 ph_s[b] ^= 1;
                 tc_fence_after();
                 const int limit = min(t.n_valid, t.shift == NO_DIAG ? BK : i - t.shift + 1);
-#pragma unroll
-                for (int c = 0; c < 2; c++) {
+                {
                     uint32_t xs[32], xp[32], pk[16];
                     tmem_ld32(tm_lane + b * 128 + c * 32, xs);
                     tmem_ld32(tm_lane + b * 128 + 64 + c * 32, xp);
@@ -207,7 +196,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                         }
                         pk[e >> 1] = pack_bf16(ds[0], ds[1]);
                     }
-                    tmem_st16(tm_lane + b * 128 + c * 16, pk);
+                    tmem_st16(tm_lane + b * 128 + c * 32, pk);      // over this warp's own half of S (the other warp may still be reading its half)
                 }
                 tmem_st_wait();
                 tc_fence_before();
@@ -215,13 +204,14 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                 if (lane == 0) mbar_arrive(&m.bar_p[b]);
             }
             // ---- epilogue: dQ -> bf16 ------------------------------------------------------------------------------
-            mbar_wait(&m.bar_o, ph_o, status);
+            mbar_wait_warp(&m.bar_o, ph_o, status);
             tc_fence_after();
             const bool full = q_valid == BQ;
 #pragma unroll
-            for (int c = 0; c < 4; c++) {
+            for (int cc = 0; cc < 2; cc++) {
+                const int c4 = c * 2 + cc;
                 uint32_t x[32];
-                tmem_ld32(tm_lane + COL_DQ + c * 32, x);
+                tmem_ld32(tm_lane + COL_DQ + c4 * 32, x);
                 tmem_ld_wait();
 #pragma unroll
                 for (int v4 = 0; v4 < 4; v4++) {
@@ -230,7 +220,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                     pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
                     pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
                     pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
-                    const int col = c * 32 + v4 * 8;
+                    const int col = c4 * 32 + v4 * 8;
                     if (full)
                         *reinterpret_cast<uint4*>(sQ + (col >> 6) * (Q_BYTES / 2) + sw128_chunk(i, (col & 63) >> 3)) = pk;
                     else if (row_ok)

@@ -35,9 +35,9 @@ struct KvTile {
     int row, n_valid, shift;
 };
 
-struct TileWalk {       // enumerates the key tiles of one item in order
+struct TileWalk {       // enumerates the key tiles of one item in order; run data is read once per run, not per tile
     const Index& ix;
-    int run0, run, run_end, off, own_row0, own_end, q0;
+    int run0, run, run_end, off, own_row0, own_end, q0, cur_row0, cur_len;
     bool in_own;
     __device__ TileWalk(const Index& ix_, int piece, int qt) : ix(ix_) {
         run0 = run = ix.anc_ptr[piece];
@@ -47,6 +47,11 @@ struct TileWalk {       // enumerates the key tiles of one item in order
         q0 = qt * BQ;
         own_end = min(ix.piece_len[piece], q0 + BQ);      // own rows up to the end of the query tile
         in_own = run == run_end;
+        cur_row0 = cur_len = 0;
+        if (!in_own) {
+            cur_row0 = ix.anc_row0[run];
+            cur_len = ix.anc_len[run];
+        }
     }
     __device__ int count() const {          // number of tiles next() will deliver from a fresh walk
         int n = (own_end + BK - 1) / BK;
@@ -55,14 +60,18 @@ struct TileWalk {       // enumerates the key tiles of one item in order
     }
     __device__ bool next(KvTile& t) {
         if (!in_own) {
-            const int len = ix.anc_len[run];
-            t.row = ix.anc_row0[run] + off;
-            t.n_valid = min(BK, len - off);
+            t.row = cur_row0 + off;
+            t.n_valid = min(BK, cur_len - off);
             t.shift = NO_DIAG;
             off += BK;
-            if (off >= len) {
+            if (off >= cur_len) {
                 off = 0;
-                if (++run == run_end) in_own = true;
+                if (++run == run_end) {
+                    in_own = true;
+                } else {
+                    cur_row0 = ix.anc_row0[run];
+                    cur_len = ix.anc_len[run];
+                }
             }
             return true;
         }
@@ -74,7 +83,6 @@ struct TileWalk {       // enumerates the key tiles of one item in order
         return true;
     }
 };
-
 
 // The query tiles (64 rows) that see the key tile `kt` (128 rows) of a piece: for every query head of the group,
 // the rest of the piece from the key tile's first row on (causal inside), then all rows of every descendant piece.

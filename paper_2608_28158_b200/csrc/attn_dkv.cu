@@ -25,11 +25,11 @@ namespace {
 using namespace tc;
 using namespace attn;
 
-constexpr int NS = 128, NT = NS + 32;
+constexpr int NS = 256, NT = NS + 64;     // 8 element-wise warps: warp w and w + 4 share a lane quarter and split the columns
 constexpr int BKV = 128, BQT = 64;
 constexpr int KV_TILE = BKV * D * 2;      // 32 KB: two panels [128 rows][64 columns]
 constexpr int Q_TILE = BQT * D * 2;       // 16 KB: two panels [64 rows][64 columns]
-constexpr int STAGES = 3;
+constexpr int STAGES = 4;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr int COL_DV = 256, COL_DK = 384, TMEM_COLS = 512;   // S^T at 128 b, dP^T at 128 b + 64
 
@@ -57,7 +57,7 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
     float* sVec = reinterpret_cast<float*>(smem + Smem::vec);       // [2 buffers][lse2 | delta][64]
     Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const bool is_softmax = warp < NS / 32, is_issuer = tid == NS;
+    const bool is_softmax = warp < NS / 32, is_issuer = tid == NS, is_producer = tid == NS + 32;
     if (tid == 0) {
         mbar_init(&m.bar_kv, 1);
         for (int s = 0; s < STAGES; s++) { mbar_init(&m.bar_q[s], 1); mbar_init(&m.bar_free[s], 1); }
@@ -76,7 +76,7 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
     const uint64_t dKd = desc_kmajor_base(smem_u32(sK)), dVd = desc_kmajor_base(smem_u32(sV));
     const float scale_log2 = scale * LOG2E;
 
-    uint32_t ph_kv = 0, ph_q[STAGES] = {0, 0, 0}, ph_free[STAGES] = {0, 0, 0}, ph_s[2] = {0, 0}, ph_p[2] = {0, 0}, ph_o = 0;
+    uint32_t ph_kv = 0, ph_q[STAGES] = {}, ph_free[STAGES] = {}, ph_s[2] = {0, 0}, ph_p[2] = {0, 0}, ph_o = 0;
     const int n_work = ix.n_kv_items * Hkv;
     for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
         const int item = w / Hkv, hk = w % Hkv;
@@ -84,18 +84,34 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
         const int kv_row0 = ix.piece_row0[piece] + kt * BKV;
         const int kv_valid = min(BKV, ix.piece_len[piece] - kt * BKV);
 
-        if (is_issuer) {
-            QWalk load_walk(ix, piece, kt, hk, G), walk(ix, piece, kt, hk, G);
-            QTile lt, t;
-            auto load_q = [&](int stage, const QTile& qt) {
+        if (is_producer) {
+            // ---- TMA producer: the K and V tiles, then the query / dO tiles STAGES deep -----------------------------
+            QWalk lw(ix, piece, kt, hk, G);
+            QTile lt;
+            mbar_expect_tx(&m.bar_kv, 2 * KV_TILE);
+            for (int p = 0; p < 2; p++)
+                for (int r = 0; r < 2; r++) {
+                    tma_load_3d(sK + p * (KV_TILE / 2) + r * (KV_TILE / 4), &map_k, p * 64, hk, kv_row0 + r * 64, &m.bar_kv);
+                    tma_load_3d(sV + p * (KV_TILE / 2) + r * (KV_TILE / 4), &map_v, p * 64, hk, kv_row0 + r * 64, &m.bar_kv);
+                }
+            for (int n = 0; lw.next(lt); n++) {
+                const int stage = n % STAGES;
+                if (n >= STAGES) {
+                    mbar_wait(&m.bar_free[stage], ph_free[stage], status);
+                    ph_free[stage] ^= 1;
+                }
                 unsigned char* sQ = smem + Smem::q0 + stage * Q_TILE;
                 unsigned char* sDO = smem + Smem::do0 + stage * Q_TILE;
                 mbar_expect_tx(&m.bar_q[stage], 2 * Q_TILE);
                 for (int p = 0; p < 2; p++) {
-                    tma_load_3d(sQ + p * (Q_TILE / 2), &map_q, p * 64, qt.head, qt.row, &m.bar_q[stage]);
-                    tma_load_3d(sDO + p * (Q_TILE / 2), &map_do, p * 64, qt.head, qt.row, &m.bar_q[stage]);
+                    tma_load_3d(sQ + p * (Q_TILE / 2), &map_q, p * 64, lt.head, lt.row, &m.bar_q[stage]);
+                    tma_load_3d(sDO + p * (Q_TILE / 2), &map_do, p * 64, lt.head, lt.row, &m.bar_q[stage]);
                 }
-            };
+            }
+        }
+        if (is_issuer) {
+            // ---- MMA issue: this thread does nothing else, a tcgen05.mma holds it until the pipe has room ---------
+            const int n_tiles = QWalk(ix, piece, kt, hk, G).count();
             auto issue_s = [&](int n) {      // S^T(n), dP^T(n) into buffer n & 1
                 const int stage = n % STAGES, b = n & 1;
                 mbar_wait(&m.bar_q[stage], ph_q[stage], status);
@@ -111,26 +127,11 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
                     mma_ss(tmem + b * 128 + 64, dVd + kstep_kmajor<BKV>(ks), dDO + kstep_kmajor<BQT>(ks), I_ST, ks > 0);
                 mma_commit(&m.bar_s[b]);
             };
-            mbar_expect_tx(&m.bar_kv, 2 * KV_TILE);
-            for (int p = 0; p < 2; p++)
-                for (int r = 0; r < 2; r++) {
-                    tma_load_3d(sK + p * (KV_TILE / 2) + r * (KV_TILE / 4), &map_k, p * 64, hk, kv_row0 + r * 64, &m.bar_kv);
-                    tma_load_3d(sV + p * (KV_TILE / 2) + r * (KV_TILE / 4), &map_v, p * 64, hk, kv_row0 + r * 64, &m.bar_kv);
-                }
-            bool more_loads = true;
-            for (int s = 0; s < STAGES && more_loads; s++) {
-                more_loads = load_walk.next(lt);
-                if (more_loads) load_q(s, lt);
-            }
             mbar_wait(&m.bar_kv, ph_kv, status);
             ph_kv ^= 1;
-            const int n_tiles = walk.count();
-            bool have = walk.next(t);
-            if (have) issue_s(0);
-            for (int n = 0; have; n++) {
-                QTile t_next;
-                const bool have_next = walk.next(t_next);
-                if (have_next) issue_s(n + 1);
+            issue_s(0);
+            for (int n = 0; n < n_tiles; n++) {
+                if (n + 1 < n_tiles) issue_s(n + 1);
                 const int stage = n % STAGES, b = n & 1;
                 mbar_wait(&m.bar_p[b], ph_p[b], status);
                 ph_p[b] ^= 1;
@@ -139,54 +140,44 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
                 const uint64_t dQm = desc_mnmajor_base<BQT>(smem_u32(smem + Smem::q0 + stage * Q_TILE));
 #pragma unroll
                 for (int ks = 0; ks < 4; ks++)
-                    mma_ts(tmem + COL_DV, tmem + b * 128 + ks * 8, dDOm + kstep_mnmajor(ks), I_ACC, n > 0 || ks > 0);
+                    mma_ts(tmem + COL_DV, tmem + b * 128 + (ks >> 1) * 32 + (ks & 1) * 8, dDOm + kstep_mnmajor(ks), I_ACC, n > 0 || ks > 0);
 #pragma unroll
                 for (int ks = 0; ks < 4; ks++)
-                    mma_ts(tmem + COL_DK, tmem + b * 128 + 64 + ks * 8, dQm + kstep_mnmajor(ks), I_ACC, n > 0 || ks > 0);
+                    mma_ts(tmem + COL_DK, tmem + b * 128 + 64 + (ks >> 1) * 32 + (ks & 1) * 8, dQm + kstep_mnmajor(ks), I_ACC, n > 0 || ks > 0);
                 if (n + STAGES < n_tiles) mma_commit(&m.bar_free[stage]);
-                if (!have_next) mma_commit(&m.bar_o);
-                if (n >= 1 && more_loads) {
-                    more_loads = load_walk.next(lt);
-                    if (more_loads) {
-                        const int sf = (n - 1) % STAGES;
-                        mbar_wait(&m.bar_free[sf], ph_free[sf], status);
-                        ph_free[sf] ^= 1;
-                        load_q(sf, lt);
-                    }
-                }
-                have = have_next;
+                if (n + 1 == n_tiles) mma_commit(&m.bar_o);
             }
         }
         if (is_softmax) {
             QWalk walk(ix, piece, kt, hk, G), ahead(ix, piece, kt, hk, G);
             QTile t, ta;
-            const int i = tid;                                 // key row inside the tile
+            const int i = tid & 127, c = tid >> 7;             // key row inside the tile, and which 32 of the 64 query columns
             const bool row_ok = i < kv_valid;
             // per-column lse (log2 units) and delta of a query tile: thread j < 64 fetches lse, thread 64 + j delta;
             // fetched one tile ahead, handed over through shared memory
-            auto fetch = [&](const QTile& qt) -> float {
-                const int j = i & 63;
-                if (j >= qt.n_valid) return i < 64 ? INFINITY : 0.f;      // columns past the end: probability 0
+            auto fetch = [&](const QTile& qt) -> float {              // threads 0..127 only
+                const int j = tid & 63;
+                if (tid >= 128) return 0.f;
+                if (j >= qt.n_valid) return tid < 64 ? INFINITY : 0.f;    // columns past the end: probability 0
                 const size_t at = (size_t)(qt.row + j) * Hq + qt.head;
-                return i < 64 ? lse[at] * LOG2E : delta[at];
+                return tid < 64 ? lse[at] * LOG2E : delta[at];
             };
             bool more_ahead = ahead.next(ta);
             float pre = more_ahead ? fetch(ta) : 0.f;
-            sVec[(i >> 6) * BQT + (i & 63)] = pre;            // buffer 0
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (tid < 128) sVec[(tid >> 6) * BQT + (tid & 63)] = pre;            // buffer 0
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             for (int n = 0; walk.next(t); n++) {
                 const int b = n & 1;
                 more_ahead = more_ahead && ahead.next(ta);
                 if (more_ahead) pre = fetch(ta);              // in flight during this tile
-                mbar_wait(&m.bar_s[b], ph_s[b], status);
+                mbar_wait_warp(&m.bar_s[b], ph_s[b], status);
                 ph_s[b] ^= 1;
                 tc_fence_after();
                 const float* vl = sVec + b * 2 * BQT;
                 const float* vd = vl + BQT;
                 // visible columns of key row i: jmin <= j < n_valid
                 const int jmin = !row_ok ? BQT : (t.lead < 0 ? 0 : max(0, i - t.lead));
-#pragma unroll
-                for (int c = 0; c < 2; c++) {
+                {
                     uint32_t xs[32], xp[32], pp[16], pd[16];
                     tmem_ld32(tm_lane + b * 128 + c * 32, xs);
                     tmem_ld32(tm_lane + b * 128 + 64 + c * 32, xp);
@@ -208,17 +199,17 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
                         pd[e >> 1] = pack_bf16(ds[0], ds[1]);
                         pd[(e >> 1) + 1] = pack_bf16(ds[2], ds[3]);
                     }
-                    tmem_st16(tm_lane + b * 128 + c * 16, pp);
-                    tmem_st16(tm_lane + b * 128 + 64 + c * 16, pd);
+                    tmem_st16(tm_lane + b * 128 + c * 32, pp);          // over this warp's own half (the other warp may still read its half)
+                    tmem_st16(tm_lane + b * 128 + 64 + c * 32, pd);
                 }
                 tmem_st_wait();
                 tc_fence_before();
-                if (more_ahead) sVec[((b ^ 1) * 2 + (i >> 6)) * BQT + (i & 63)] = pre;
-                asm volatile("bar.sync 1, 128;" ::: "memory");      // next tile's vectors visible; this tile's reads done
+                if (more_ahead && tid < 128) sVec[((b ^ 1) * 2 + (tid >> 6)) * BQT + (tid & 63)] = pre;
+                asm volatile("bar.sync 1, 256;" ::: "memory");      // next tile's vectors visible; this tile's reads done
                 if (lane == 0) mbar_arrive(&m.bar_p[b]);
             }
             // ---- epilogue: dV, dK -> bf16 ---------------------------------------------------------------------------
-            mbar_wait(&m.bar_o, ph_o, status);
+            mbar_wait_warp(&m.bar_o, ph_o, status);
             tc_fence_after();
             const bool full = kv_valid == BKV;
 #pragma unroll
@@ -226,9 +217,10 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
                 unsigned char* stage_buf = which ? sK : sV;              // the K / V tiles are no longer needed
                 __nv_bfloat16* out = which ? dk_ : dv_;
 #pragma unroll
-                for (int c = 0; c < 4; c++) {
+                for (int cc = 0; cc < 2; cc++) {
+                    const int c4 = c * 2 + cc;
                     uint32_t x[32];
-                    tmem_ld32(tm_lane + (which ? COL_DK : COL_DV) + c * 32, x);
+                    tmem_ld32(tm_lane + (which ? COL_DK : COL_DV) + c4 * 32, x);
                     tmem_ld_wait();
 #pragma unroll
                     for (int v4 = 0; v4 < 4; v4++) {
@@ -237,7 +229,7 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
                         pk.y = pack_bf16(__uint_as_float(x[v4 * 8 + 2]), __uint_as_float(x[v4 * 8 + 3]));
                         pk.z = pack_bf16(__uint_as_float(x[v4 * 8 + 4]), __uint_as_float(x[v4 * 8 + 5]));
                         pk.w = pack_bf16(__uint_as_float(x[v4 * 8 + 6]), __uint_as_float(x[v4 * 8 + 7]));
-                        const int col = c * 32 + v4 * 8;
+                        const int col = c4 * 32 + v4 * 8;
                         if (full)
                             *reinterpret_cast<uint4*>(stage_buf + (col >> 6) * (KV_TILE / 2) + sw128_chunk(i, (col & 63) >> 3)) = pk;
                         else if (row_ok)

@@ -25,7 +25,7 @@ using namespace tc;
 
 using namespace attn;
 constexpr int NS = 128;                 // softmax threads (4 warps), thread = query row = tensor-memory lane
-constexpr int NT = NS + 32;             // plus one warp whose first lane issues TMA and MMA
+constexpr int NT = NS + 64;             // plus one warp whose first lane issues the MMAs and one whose first lane issues the TMA loads
 constexpr int Q_BYTES = BQ * D * 2;     // 32 KB: two panels [128 rows][64 columns]
 constexpr int KV_BYTES = BK * D * 2;    // 16 KB: two panels [64 rows][64 columns]
 constexpr int COL_S = 0, COL_O = 128, TMEM_COLS = 256;
@@ -37,7 +37,7 @@ struct Smem {
     static constexpr int bytes = misc + 256;
 };
 struct Misc {
-    uint64_t bar_q, bar_kv[2], bar_s, bar_p, bar_o;
+    uint64_t bar_q, bar_kv[2], bar_free[2], bar_s, bar_p, bar_o;
     uint32_t tmem;
 };
 
@@ -52,12 +52,14 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
     Misc& m = *reinterpret_cast<Misc*>(smem + Smem::misc);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool is_softmax = warp < NS / 32;
-    const bool is_issuer = tid == NS;
+    const bool is_issuer = tid == NS, is_producer = tid == NS + 32;
 
     if (tid == 0) {
         mbar_init(&m.bar_q, 1);
         mbar_init(&m.bar_kv[0], 1);
         mbar_init(&m.bar_kv[1], 1);
+        mbar_init(&m.bar_free[0], 1);
+        mbar_init(&m.bar_free[1], 1);
         mbar_init(&m.bar_s, 1);
         mbar_init(&m.bar_p, NS / 32);
         mbar_init(&m.bar_o, 1);
@@ -75,7 +77,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
     const uint32_t aQ = smem_u32(sQ);
     const uint64_t dQ = desc_kmajor_base(aQ);
 
-    uint32_t ph_q = 0, ph_kv[2] = {0, 0}, ph_s = 0, ph_p = 0, ph_o = 0;
+    uint32_t ph_q = 0, ph_kv[2] = {0, 0}, ph_free[2] = {0, 0}, ph_s = 0, ph_p = 0, ph_o = 0;
     const int n_work = ix.n_q_items * Hq;
     for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
         const int item = w / Hq, h = w % Hq, hk = h / G;
@@ -83,47 +85,47 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
         const int q_row0 = ix.piece_row0[piece] + qt * BQ;
         const int q_valid = min(BQ, ix.piece_len[piece] - qt * BQ);
 
-        if (is_issuer) {
-            // ---- producer + MMA issue ------------------------------------------------------------------------------
-            TileWalk load_walk(ix, piece, qt), walk(ix, piece, qt);
-            KvTile lt, t;
-            auto load_kv = [&](int stage, const KvTile& kt) {
-                unsigned char* sK = smem + Smem::k0 + stage * KV_BYTES;
-                unsigned char* sV = smem + Smem::v0 + stage * KV_BYTES;
-                mbar_expect_tx(&m.bar_kv[stage], 2 * KV_BYTES);
-                for (int p = 0; p < 2; p++) {
-                    tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, kt.row, &m.bar_kv[stage]);
-                    tma_load_3d(sV + p * (KV_BYTES / 2), &map_v, p * 64, hk, kt.row, &m.bar_kv[stage]);
-                }
-            };
+        if (is_producer) {
+            // ---- TMA producer: the Q tile, then the key/value tiles two stages deep ---------------------------------
+            TileWalk lw(ix, piece, qt);
+            KvTile lt;
             mbar_expect_tx(&m.bar_q, Q_BYTES);
             for (int p = 0; p < 2; p++)
                 for (int r = 0; r < 2; r++)
                     tma_load_3d(sQ + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_q, p * 64, h, q_row0 + r * 64, &m.bar_q);
-            bool more_loads = load_walk.next(lt);
-            if (more_loads) load_kv(0, lt);
-            more_loads = more_loads && load_walk.next(lt);
-            if (more_loads) load_kv(1, lt);
-            mbar_wait(&m.bar_q, ph_q, status);
-            ph_q ^= 1;
-            int n = 0;
-            bool have = walk.next(t);
-            // S of the first tile
-            if (have) {
-                mbar_wait(&m.bar_kv[0], ph_kv[0], status);
-                ph_kv[0] ^= 1;
+            for (int n = 0; lw.next(lt); n++) {
+                const int stage = n & 1;
+                if (n >= 2) {                                 // the MMAs that read this stage are done
+                    mbar_wait(&m.bar_free[stage], ph_free[stage], status);
+                    ph_free[stage] ^= 1;
+                }
+                unsigned char* sK = smem + Smem::k0 + stage * KV_BYTES;
+                unsigned char* sV = smem + Smem::v0 + stage * KV_BYTES;
+                mbar_expect_tx(&m.bar_kv[stage], 2 * KV_BYTES);
+                for (int p = 0; p < 2; p++) {
+                    tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, lt.row, &m.bar_kv[stage]);
+                    tma_load_3d(sV + p * (KV_BYTES / 2), &map_v, p * 64, hk, lt.row, &m.bar_kv[stage]);
+                }
+            }
+        }
+        if (is_issuer) {
+            // ---- MMA issue: this thread does nothing else, a tcgen05.mma holds it until the pipe has room ---------
+            const int n_tiles = TileWalk(ix, piece, qt).count();
+            auto issue_s = [&](int stage) {
+                mbar_wait(&m.bar_kv[stage], ph_kv[stage], status);
+                ph_kv[stage] ^= 1;
                 tc_fence_after();
-                const uint64_t dK = desc_kmajor_base(smem_u32(smem + Smem::k0));
+                const uint64_t dK = desc_kmajor_base(smem_u32(smem + Smem::k0 + stage * KV_BYTES));
 #pragma unroll
                 for (int ks = 0; ks < 8; ks++)
                     mma_ss(tmem + COL_S, dQ + kstep_kmajor<BQ>(ks), dK + kstep_kmajor<BK>(ks), I_S, ks > 0);
                 mma_commit(&m.bar_s);
-                ph_s ^= 1;                                    // this thread does not wait for S(0)
-            }
-            while (have) {
+            };
+            mbar_wait(&m.bar_q, ph_q, status);
+            ph_q ^= 1;
+            issue_s(0);
+            for (int n = 0; n < n_tiles; n++) {
                 const int stage = n & 1;
-                KvTile t_next;
-                const bool have_next = walk.next(t_next);
                 // O += P V for tile n as soon as the softmax warps have written P
                 mbar_wait(&m.bar_p, ph_p, status);
                 ph_p ^= 1;
@@ -132,33 +134,10 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
 #pragma unroll
                 for (int ks = 0; ks < 4; ks++)
                     mma_ts(tmem + COL_O, tmem + COL_S + ks * 8, dV + kstep_mnmajor(ks), I_O, n > 0 || ks > 0);
-                if (have_next) {
-                    // S of tile n+1 queues behind it (it overwrites P only after the MMAs above have read it)
-                    const int s2 = stage ^ 1;
-                    mbar_wait(&m.bar_kv[s2], ph_kv[s2], status);
-                    ph_kv[s2] ^= 1;
-                    tc_fence_after();
-                    const uint64_t dK = desc_kmajor_base(smem_u32(smem + Smem::k0 + s2 * KV_BYTES));
-#pragma unroll
-                    for (int ks = 0; ks < 8; ks++)
-                        mma_ss(tmem + COL_S, dQ + kstep_kmajor<BQ>(ks), dK + kstep_kmajor<BK>(ks), I_S, ks > 0);
-                    mma_commit(&m.bar_s);
-                } else {
-                    mma_commit(&m.bar_o);
-                }
-                // stage `stage` is free once the PV MMAs are done: known when S(n+1) completes (in order) or at bar_o
-                if (more_loads) {
-                    more_loads = load_walk.next(lt);
-                    if (more_loads) {
-                        // wait for the MMAs that read this stage: they precede S(n+1), whose completion bar_s reports
-                        mbar_wait(&m.bar_s, ph_s, status);
-                        load_kv(stage, lt);
-                    }
-                }
-                if (have_next) ph_s ^= 1;
-                t = t_next;
-                have = have_next;
-                n++;
+                if (n + 2 < n_tiles) mma_commit(&m.bar_free[stage]);      // the stage will be refilled
+                // S of tile n+1 queues behind it (it overwrites P only after the MMAs above have read it)
+                if (n + 1 < n_tiles) issue_s(stage ^ 1);
+                else mma_commit(&m.bar_o);
             }
         }
 
@@ -169,7 +148,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
             const int i = tid;                                // query row inside the tile
             int n = 0;
             while (walk.next(t)) {
-                mbar_wait(&m.bar_s, ph_s, status);
+                mbar_wait_warp(&m.bar_s, ph_s, status);
                 ph_s ^= 1;
                 tc_fence_after();
                 const int limit = min(t.n_valid, t.shift == NO_DIAG ? BK : i - t.shift + 1);   // visible: j < limit
@@ -227,7 +206,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 n++;
             }
             // ---- epilogue: O / l -> bf16, lse ----------------------------------------------------------------------
-            mbar_wait(&m.bar_o, ph_o, status);
+            mbar_wait_warp(&m.bar_o, ph_o, status);
             tc_fence_after();
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
             const bool full = q_valid == BQ;

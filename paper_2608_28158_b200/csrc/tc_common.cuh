@@ -36,6 +36,11 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* s
         if (mbar_try(bar, parity)) return;
     if (status) atomicExch(status, STATUS_TIMEOUT);
 }
+// The same for a whole (converged) warp: one lane polls, so that 31 lanes do not spend shared-memory cycles on it.
+__device__ __forceinline__ void mbar_wait_warp(uint64_t* bar, uint32_t parity, int* status) {
+    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, status);
+    __syncwarp();
+}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
