@@ -12,7 +12,8 @@ no collective on the data path); time is the maximum over ranks.
 
 ``--workload logp`` runs the second path instead, the compact-to-semantic log-probability (one step = its
 forward + backward over one microbatch of compact logit rows), ``--workload conv`` the tree-aware causal
-convolution that precedes the linear-attention core; both print the same JSON keys.
+convolution that precedes the linear-attention core, ``--workload attn`` full attention on compact tokens; all
+print the same JSON keys.
 
 ``--impl reference`` times the fp64 CPU oracle (oracle/), as it stands, on the host cores, on a
 bounded sample of the same workload.
@@ -874,6 +875,197 @@ def run_conv(args):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------------------
+# Fourth workload: full attention on compact tokens (Section 3.4, Eqs. 21-22), `--workload attn`
+# --------------------------------------------------------------------------------------------------
+ATTN_METRIC = "compact-token attention fwd+bwd compact tokens/s"
+ATTN_H, ATTN_D = 16, 128
+
+
+def attn_oracle_sample(small=False, copies=1):
+    """The fp64 attention oracle on copies of the cfg0b tree, 2 of the 16 heads."""
+    from oracle import attn_oracle
+    from workloads import CONFIGS, make_attn_inputs, make_forest
+    heads = 1 if small else 2
+    fo = make_forest([CONFIGS["cfg0b"]["build"]()[0]] * copies)
+    inp = make_attn_inputs(fo.n_tokens, heads, heads, ATTN_D, "bf16", 0)
+    q, k, v, dO = (inp[n].double().numpy() for n in ("q", "k", "v", "dO"))
+    t0 = time.perf_counter()
+    attn_oracle.attn_fwd(fo, q, k, v, ATTN_D ** -0.5)
+    attn_oracle.attn_bwd(fo, q, k, v, dO, ATTN_D ** -0.5)
+    dt = time.perf_counter() - t0
+    if not small and copies == 1 and dt < 8.0:
+        return attn_oracle_sample(False, copies=int(min(32, max(2, round(12.0 / dt)))))
+    return {"value": fo.n_tokens * heads / ATTN_H / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{copies} x cfg0b tree ({fo.n_tokens} compact tokens), {heads} of {ATTN_H} heads, fwd+bwd, {dt:.1f} s",
+            "seconds": dt}
+
+
+def run_attn_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    vals, secs, last = [], [], None
+    for i in range(args.warmup + args.steps):
+        last = attn_oracle_sample(small=True)
+        if i >= args.warmup:
+            vals.append(last["value"])
+            secs.append(last["seconds"])
+    value = statistics.mean(vals)
+    print(json.dumps({
+        "impl": "reference", "metric": ATTN_METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(secs) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "attn", "Hq": ATTN_H, "Hkv": ATTN_H, "d": ATTN_D},
+        "cpu_baseline": {"kind": last["kind"], "cores": last["cores"], "sample": last["sample"], "value": value,
+                         "unit": UNIT},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def run_attn(args):
+    """One step = forward + backward of multi-head attention (16 heads, d = 128, bf16) over the compact tokens of
+    a forest (default cfg2): every token attends to its ancestors in the tree and to itself."""
+    import torch
+    import torch.distributed as dist
+
+    import paper_2608_28158_b200 as H
+    from workloads import config_forest, make_attn_inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    fo = config_forest(args.attn_trees)
+    C, Hq, Hkv, d = fo.n_tokens, ATTN_H, args.attn_kv_heads, ATTN_D
+    scale = d ** -0.5
+    plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
+    t0 = time.perf_counter()
+    index = H.harts_attn_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, plan.row_of_token)
+    t_host = time.perf_counter() - t0
+    index.upload()
+    anc = np.array([int(index.anc_len[index.anc_ptr[p]:index.anc_ptr[p + 1]].sum()) for p in range(index.n_pieces)],
+                   dtype=np.int64)
+    L = index.piece_len.astype(np.int64)
+    pairs = int((L * anc + L * (L + 1) // 2).sum())             # visible (query, key) pairs per head
+    inp = make_attn_inputs(C, Hq, Hkv, d, "bf16", 90 + rank, device="cuda")
+    o, lse = torch.empty_like(inp["q"]), torch.empty(C, Hq, device="cuda")
+    grads = {"dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]), "dv": torch.empty_like(inp["v"])}
+    delta = torch.empty(C, Hq, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+
+    def step(marks=None):
+        a, b, c = ev(), ev(), ev()
+        a.record(stream)
+        H.harts_attn_fwd(index, inp["q"], inp["k"], inp["v"], o, lse, scale, dev_status=status)
+        b.record(stream)
+        H.harts_attn_bwd(index, inp["q"], inp["k"], inp["v"], o, lse, inp["dO"], grads["dq"], grads["dk"], grads["dv"],
+                         delta, scale, dev_status=status)
+        c.record(stream)
+        if marks is not None:
+            marks.append((a, b, c))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    marks = []
+    t_begin, t_end = ev(), ev()
+    with ClockSampler(local) as clocks:
+        for _ in range(args.warmup):
+            step()
+        H.harts_la_check(status)
+        barrier()
+        h0 = clocks.mark()
+        t_begin.record(stream)
+        for _ in range(args.steps):
+            step(marks)
+        t_end.record(stream)
+        barrier()
+        h1 = clocks.mark()
+    H.harts_la_check(status)
+    ms_step = t_begin.elapsed_time(t_end) / args.steps
+    fwd_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in marks)
+    bwd_ms = statistics.mean(b.elapsed_time(c) for _, b, c in marks)
+    e2e = None
+    if not args.no_e2e:
+        host = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in inp.items()}
+        for n in host:
+            host[n].copy_(inp[n])
+        out_h = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in
+                 list(grads.items()) + [("o", o)]}
+        torch.cuda.synchronize()
+
+        def e2e_step():
+            for n in host:
+                inp[n].copy_(host[n], non_blocking=True)
+            step()
+            out_h["o"].copy_(o, non_blocking=True)
+            for n in grads:
+                out_h[n].copy_(grads[n], non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b = ev(), ev()
+        n_e2e = max(1, min(args.steps, args.e2e_steps))
+        a.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e2e = {"ms": a.elapsed_time(b) / n_e2e, "steps": n_e2e,
+               "h2d": sum(t.numel() * t.element_size() for t in host.values()),
+               "d2h": sum(t.numel() * t.element_size() for t in out_h.values())}
+        del host, out_h
+    if world > 1:
+        ms_step, e2e_ms = max_over_ranks([ms_step, e2e["ms"] if e2e else 0.0], "cuda")
+        if e2e:
+            e2e["ms"] = e2e_ms
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    peak = peaks["bf16_tflops_sustained"]
+    fwd_flops = 4.0 * d * pairs * Hq                     # Q K^T and P V on the visible pairs only
+    bwd_flops = 2.5 * fwd_flops                          # five GEMMs (the kernels execute seven: S and dP twice)
+    achieved = bwd_flops / (bwd_ms * 1e-3) / 1e12
+    clock = clocks.summary(h0, h1)
+    if not clock["samples"]:
+        clock = clocks.summary()
+    line = {
+        "metric": ATTN_METRIC, "value": C * world / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "attn", "trees": args.attn_trees, "compact_tokens": C, "Hq": Hq, "Hkv": Hkv, "d": d,
+                   "pieces": index.n_pieces, "visible_pairs_per_head": pairs,
+                   "mean_context": pairs / C, "l2": "flushed by the step itself: q, k, v, dO, o and the gradients "
+                   f"({9 * C * Hq * d * 2 / 2**30:.2f} GiB) exceed L2", "host_index_ms": t_host * 1e3},
+        "roofline": {"bound": "tensor", "kernel": "backward call (attn_dq_kernel + attn_dkv_kernel)",
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                     "algorithmic_flops_per_launch": bwd_flops, "executed_flops_per_launch": bwd_flops * 7 / 5,
+                     "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
+                     "forward": {"achieved": fwd_flops / (fwd_ms * 1e-3) / 1e12,
+                                 "frac": fwd_flops / (fwd_ms * 1e-3) / 1e12 / peak},
+                     "whole_path": {"roof_ms": (fwd_flops + bwd_flops) / (peak * 1e12) * 1e3,
+                                    "frac_strict": (fwd_flops + bwd_flops) / (peak * 1e12) * 1e3 / ms_step}},
+        "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms},
+        "gpu_launches": 4 * args.steps,
+        "clocks": clock,
+    }
+    if e2e:
+        line["e2e"] = {"value": C * world / (e2e["ms"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
+                       "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"], "pinned_host_memory": True}
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = attn_oracle_sample()
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -888,12 +1080,16 @@ def main():
     ap.add_argument("--no-trajwise", action="store_true")
     ap.add_argument("--logp-rows", type=int, default=LOGP_ROWS, help="compact-row capacity of the logp workload")
     ap.add_argument("--conv-trees", default="cfg3", help="forest of the conv workload (cfg2: a small case for captures)")
+    ap.add_argument("--attn-trees", default="cfg2", help="forest of the attn workload (cfg1: a small case for captures)")
+    ap.add_argument("--attn-kv-heads", type=int, default=ATTN_H, help="kv heads of the attn workload (16 = MHA)")
     ap.add_argument("--per-config", action="store_true", help="also print a table over all configurations to stderr")
     args = ap.parse_args()
     if args.workload == "logp":
         (run_logp_reference if args.impl == "reference" else run_logp)(args)
     elif args.workload == "conv":
         (run_conv_reference if args.impl == "reference" else run_conv)(args)
+    elif args.workload == "attn":
+        (run_attn_reference if args.impl == "reference" else run_attn)(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

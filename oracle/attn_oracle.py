@@ -55,14 +55,16 @@ def attn_fwd(forest, q, k, v, scale, tokens=None):
     return o, lse
 
 
-def attn_bwd(forest, q, k, v, dO, scale):
-    """(dq, dk, dv) of sum_t <dO_t, o_t>."""
+def attn_bwd(forest, q, k, v, dO, scale, tokens=None):
+    """(dq, dk, dv) of sum_t <dO_t, o_t>.  tokens: only these queries (dq rows of the others stay zero; dk, dv then
+    hold the contributions of these queries alone)."""
     q, k, v, dO = (np.asarray(a, np.float64) for a in (q, k, v, dO))
     C, Hq, d = q.shape
     G = Hq // k.shape[1]
     dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
     pred = predecessors(forest)
-    for t in range(C):
+    for t in (range(C) if tokens is None else tokens):
+        t = int(t)
         path = _path(pred, t)
         for h in range(Hq):
             hk = h // G

@@ -111,3 +111,32 @@ def test_backward_bushy_random_forest():
     fo = make_forest([random_tree(rnd, 9, 300) for _ in range(3)] + [([-1], [0], [1])])
     _check_backward(fo, 2, 1, 5, use_plan=False)
     _check_backward(fo, 2, 2, 5, use_plan=True)
+
+
+def test_full_size_sampled_queries_and_invariants():
+    """The benchmark's workload (cfg2, 16 heads): o, lse and dq of sampled queries against the oracle one by one;
+    dv through an identity that holds at any size (every softmax row sums to 1, so sum_s dv_s = sum_t dO_t)."""
+    fo = config_forest("cfg2")
+    Hq = Hkv = 16
+    inp = make_attn_inputs(fo.n_tokens, Hq, Hkv, D, "bf16", 90, device="cuda")
+    rot = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64).row_of_token
+    index = H.harts_attn_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, rot).upload()
+    rows = torch.as_tensor(rot.astype(np.int64)).cuda()
+    phys = {}
+    for n, x in inp.items():
+        t = torch.empty_like(x); t[rows] = x; phys[n] = t
+    o, lse = _forward(phys, index)
+    dq, dk, dv = _backward(phys, index, o, lse)
+    tok = np.unique(np.concatenate([np.linspace(0, fo.n_tokens - 1, 12).astype(np.int64), fo.token_base()[1:4] - 1]))
+    heads = [0, 7, 15]
+    cpu = {n: x[:, heads].double().cpu().numpy() for n, x in inp.items()}
+    o_ref, lse_ref = ao.attn_fwd(fo, cpu["q"], cpu["k"], cpu["v"], SCALE, tokens=tok)
+    dq_ref, _, _ = ao.attn_bwd(fo, cpu["q"], cpu["k"], cpu["v"], cpu["dO"], SCALE, tokens=tok)
+    pick = lambda x: x[rows][:, heads].double().cpu().numpy()[tok]  # noqa: E731
+    assert _rel(pick(o), o_ref[tok]) <= 5e-3
+    assert np.abs(pick(lse) - lse_ref[tok]).max() <= 2e-3
+    assert _rel(pick(dq), dq_ref[tok]) <= 1e-2
+    total_dv = dv.double().sum(dim=0).cpu().numpy()
+    total_dO = inp["dO"].double().sum(dim=0).cpu().numpy()
+    assert _rel(total_dv, total_dO) <= 5e-3
+    assert all(bool(torch.isfinite(x.float()).all()) for x in (o, dq, dk, dv))
