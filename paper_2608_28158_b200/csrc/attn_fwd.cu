@@ -28,8 +28,13 @@ constexpr int NS = 128;                 // softmax threads (4 warps), thread = q
 constexpr int NT = NS + 64;             // plus one warp whose first lane issues the MMAs and one whose first lane issues the TMA loads
 constexpr int Q_BYTES = BQ * D * 2;     // 32 KB: two panels [128 rows][64 columns]
 constexpr int KV_BYTES = BK * D * 2;    // 16 KB: two panels [64 rows][64 columns]
-constexpr int COL_S = 0, COL_O = 128, TMEM_COLS = 256;
+constexpr int COL_S = 0, COL_O = 128, TMEM_COLS = 256;     // S / P of tile n at COL_S + 64 (n & 1)
 constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 constexpr float RAISE = 8.f;            // the reference maximum follows the row maximum in steps of at least 2^8
 
 struct Smem {
@@ -37,7 +42,7 @@ struct Smem {
     static constexpr int bytes = misc + 256;
 };
 struct Misc {
-    uint64_t bar_q, bar_kv[2], bar_free[2], bar_s, bar_p, bar_o;
+    uint64_t bar_q, bar_k[2], bar_v[2], bar_kfree[2], bar_vfree[2], bar_s[2], bar_p, bar_o;
     uint32_t tmem;
 };
 
@@ -56,11 +61,14 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
 
     if (tid == 0) {
         mbar_init(&m.bar_q, 1);
-        mbar_init(&m.bar_kv[0], 1);
-        mbar_init(&m.bar_kv[1], 1);
-        mbar_init(&m.bar_free[0], 1);
-        mbar_init(&m.bar_free[1], 1);
-        mbar_init(&m.bar_s, 1);
+        for (int st = 0; st < 2; st++) {
+            mbar_init(&m.bar_k[st], 1);
+            mbar_init(&m.bar_v[st], 1);
+            mbar_init(&m.bar_kfree[st], 1);
+            mbar_init(&m.bar_vfree[st], 1);
+        }
+        mbar_init(&m.bar_s[0], 1);
+        mbar_init(&m.bar_s[1], 1);
         mbar_init(&m.bar_p, NS / 32);
         mbar_init(&m.bar_o, 1);
         fence_barrier_init();
@@ -77,7 +85,8 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
     const uint32_t aQ = smem_u32(sQ);
     const uint64_t dQ = desc_kmajor_base(aQ);
 
-    uint32_t ph_q = 0, ph_kv[2] = {0, 0}, ph_free[2] = {0, 0}, ph_s = 0, ph_p = 0, ph_o = 0;
+    uint32_t ph_q = 0, ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_kfree[2] = {0, 0}, ph_vfree[2] = {0, 0}, ph_s[2] = {0, 0},
+             ph_p = 0, ph_o = 0;
     const int n_work = ix.n_q_items * Hq;
     for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
         const int item = w / Hq, h = w % Hq, hk = h / G;
@@ -95,49 +104,60 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                     tma_load_3d(sQ + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_q, p * 64, h, q_row0 + r * 64, &m.bar_q);
             for (int n = 0; lw.next(lt); n++) {
                 const int stage = n & 1;
-                if (n >= 2) {                                 // the MMAs that read this stage are done
-                    mbar_wait(&m.bar_free[stage], ph_free[stage], status);
-                    ph_free[stage] ^= 1;
-                }
                 unsigned char* sK = smem + Smem::k0 + stage * KV_BYTES;
                 unsigned char* sV = smem + Smem::v0 + stage * KV_BYTES;
-                mbar_expect_tx(&m.bar_kv[stage], 2 * KV_BYTES);
-                for (int p = 0; p < 2; p++) {
-                    tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, lt.row, &m.bar_kv[stage]);
-                    tma_load_3d(sV + p * (KV_BYTES / 2), &map_v, p * 64, hk, lt.row, &m.bar_kv[stage]);
+                // the K tile of a stage is free as soon as S of its previous tile is done, the V tile only after P V
+                if (n >= 2) {
+                    mbar_wait(&m.bar_kfree[stage], ph_kfree[stage], status);
+                    ph_kfree[stage] ^= 1;
                 }
+                mbar_expect_tx(&m.bar_k[stage], KV_BYTES);
+                for (int p = 0; p < 2; p++)
+                    tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, lt.row, &m.bar_k[stage]);
+                if (n >= 2) {
+                    mbar_wait(&m.bar_vfree[stage], ph_vfree[stage], status);
+                    ph_vfree[stage] ^= 1;
+                }
+                mbar_expect_tx(&m.bar_v[stage], KV_BYTES);
+                for (int p = 0; p < 2; p++)
+                    tma_load_3d(sV + p * (KV_BYTES / 2), &map_v, p * 64, hk, lt.row, &m.bar_v[stage]);
             }
         }
         if (is_issuer) {
             // ---- MMA issue: this thread does nothing else, a tcgen05.mma holds it until the pipe has room ---------
             const int n_tiles = TileWalk(ix, piece, qt).count();
-            auto issue_s = [&](int stage) {
-                mbar_wait(&m.bar_kv[stage], ph_kv[stage], status);
-                ph_kv[stage] ^= 1;
+            auto issue_s = [&](int n) {                     // S(n) into buffer n & 1, from stage n & 1
+                const int stage = n & 1;
+                mbar_wait(&m.bar_k[stage], ph_k[stage], status);
+                ph_k[stage] ^= 1;
                 tc_fence_after();
                 const uint64_t dK = desc_kmajor_base(smem_u32(smem + Smem::k0 + stage * KV_BYTES));
 #pragma unroll
                 for (int ks = 0; ks < 8; ks++)
-                    mma_ss(tmem + COL_S, dQ + kstep_kmajor<BQ>(ks), dK + kstep_kmajor<BK>(ks), I_S, ks > 0);
-                mma_commit(&m.bar_s);
+                    mma_ss(tmem + COL_S + stage * 64, dQ + kstep_kmajor<BQ>(ks), dK + kstep_kmajor<BK>(ks), I_S, ks > 0);
+                mma_commit(&m.bar_s[stage]);
+                if (n + 2 < n_tiles) mma_commit(&m.bar_kfree[stage]);     // the K tile will be refilled
             };
             mbar_wait(&m.bar_q, ph_q, status);
             ph_q ^= 1;
             issue_s(0);
             for (int n = 0; n < n_tiles; n++) {
                 const int stage = n & 1;
+                // S of tile n+1 goes to the other buffer and runs under the softmax of tile n (its K stage was freed
+                // by the P V MMAs of tile n-1, which precede it in the pipe)
+                if (n + 1 < n_tiles) issue_s(n + 1);
                 // O += P V for tile n as soon as the softmax warps have written P
                 mbar_wait(&m.bar_p, ph_p, status);
                 ph_p ^= 1;
+                mbar_wait(&m.bar_v[stage], ph_v[stage], status);
+                ph_v[stage] ^= 1;
                 tc_fence_after();
                 const uint64_t dV = desc_mnmajor_base<BK>(smem_u32(smem + Smem::v0 + stage * KV_BYTES));
 #pragma unroll
                 for (int ks = 0; ks < 4; ks++)
-                    mma_ts(tmem + COL_O, tmem + COL_S + ks * 8, dV + kstep_mnmajor(ks), I_O, n > 0 || ks > 0);
-                if (n + 2 < n_tiles) mma_commit(&m.bar_free[stage]);      // the stage will be refilled
-                // S of tile n+1 queues behind it (it overwrites P only after the MMAs above have read it)
-                if (n + 1 < n_tiles) issue_s(stage ^ 1);
-                else mma_commit(&m.bar_o);
+                    mma_ts(tmem + COL_O, tmem + COL_S + stage * 64 + ks * 8, dV + kstep_mnmajor(ks), I_O, n > 0 || ks > 0);
+                if (n + 2 < n_tiles) mma_commit(&m.bar_vfree[stage]);     // the V tile will be refilled
+                if (n + 1 == n_tiles) mma_commit(&m.bar_o);
             }
         }
 
@@ -148,22 +168,26 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
             const int i = tid;                                // query row inside the tile
             int n = 0;
             while (walk.next(t)) {
-                mbar_wait_warp(&m.bar_s, ph_s, status);
-                ph_s ^= 1;
+                const int b = n & 1;
+                mbar_wait_warp(&m.bar_s[b], ph_s[b], status);
+                ph_s[b] ^= 1;
                 tc_fence_after();
                 const int limit = min(t.n_valid, t.shift == NO_DIAG ? BK : i - t.shift + 1);   // visible: j < limit
-                // pass 1: row maximum
-                float mx = -INFINITY;
-                uint32_t x[32];
+                // the whole row of S in registers; hidden columns become -inf (exp2 gives 0), only in tiles that have some
+                uint32_t x[BK];
+                tmem_ld32(tm_lane + COL_S + b * 64, x);
+                tmem_ld32(tm_lane + COL_S + b * 64 + 32, x + 32);
+                tmem_ld_wait();
+                if (!__all_sync(0xffffffffu, limit >= BK)) {
 #pragma unroll
-                for (int c = 0; c < 2; c++) {
-                    tmem_ld32(tm_lane + COL_S + c * 32, x);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 32; e++)
-                        if (c * 32 + e < limit) mx = fmaxf(mx, __uint_as_float(x[e]));
+                    for (int e = 0; e < BK; e++)
+                        if (e >= limit) x[e] = __float_as_uint(-INFINITY);
                 }
-                mx *= scale_log2;
+                // row maximum (three-input max: 32 instructions for 64 values)
+                float mx = __uint_as_float(x[0]);
+#pragma unroll
+                for (int e = 1; e + 1 < BK; e += 2) mx = max3(mx, __uint_as_float(x[e]), __uint_as_float(x[e + 1]));
+                mx = fmaxf(mx, __uint_as_float(x[BK - 1])) * scale_log2;
                 // raise the reference only by big steps; the whole warp decides together whether O must be rescaled
                 const bool raise = mx > m_ref + RAISE || m_ref == -INFINITY;
                 if (__any_sync(0xffffffffu, raise && n > 0)) {
@@ -172,33 +196,33 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                     l_sum *= alpha;
 #pragma unroll
                     for (int c = 0; c < 4; c++) {
-                        tmem_ld32(tm_lane + COL_O + c * 32, x);
+                        uint32_t y[32];
+                        tmem_ld32(tm_lane + COL_O + c * 32, y);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int e = 0; e < 32; e++) x[e] = __float_as_uint(__uint_as_float(x[e]) * alpha);
-                        tmem_st32(tm_lane + COL_O + c * 32, x);
+                        for (int e = 0; e < 32; e++) y[e] = __float_as_uint(__uint_as_float(y[e]) * alpha);
+                        tmem_st32(tm_lane + COL_O + c * 32, y);
                     }
                     m_ref = m_new;
                 } else if (raise) {
                     m_ref = mx;                               // first tile: nothing accumulated yet
                 }
-                // pass 2: P = exp2(s - m_ref), written over S as bf16 pairs
+                // P = exp2(s - m_ref), written over S as bf16 pairs; four independent partial sums
                 const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
+                float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int c = 0; c < 2; c++) {
-                    tmem_ld32(tm_lane + COL_S + c * 32, x);
-                    tmem_ld_wait();
                     uint32_t pk[16];
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
-                        const float p0 = c * 32 + e < limit ? ex2(fmaf(__uint_as_float(x[e]), scale_log2, neg_m)) : 0.f;
-                        const float p1 = c * 32 + e + 1 < limit ? ex2(fmaf(__uint_as_float(x[e + 1]), scale_log2, neg_m)) : 0.f;
+                        const float p0 = ex2(fmaf(__uint_as_float(x[c * 32 + e]), scale_log2, neg_m));
+                        const float p1 = ex2(fmaf(__uint_as_float(x[c * 32 + e + 1]), scale_log2, neg_m));
                         pk[e >> 1] = pack_bf16(p0, p1);
-                        // the sum uses the rounded values the MMA will see
-                        l_sum += __uint_as_float(pk[e >> 1] << 16) + __uint_as_float(pk[e >> 1] & 0xffff0000u);
+                        part[(e >> 1) & 3] += p0 + p1;
                     }
-                    tmem_st16(tm_lane + COL_S + c * 16, pk);
+                    tmem_st16(tm_lane + COL_S + b * 64 + c * 16, pk);
                 }
+                l_sum += (part[0] + part[1]) + (part[2] + part[3]);
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
