@@ -30,8 +30,6 @@ using namespace attn;
 
 constexpr int NS = 256, NT = NS + 64;     // 8 element-wise warps: warp w and w + 4 share a lane quarter and split the columns
 constexpr int Q_BYTES = BQ * D * 2;       // 32 KB
-constexpr int KV_BYTES = BK * D * 2;      // 16 KB
-constexpr int STAGES = 4;
 constexpr float LOG2E = 1.4426950408889634f;
 
 __global__ void __launch_bounds__(256) delta_kernel(const __nv_bfloat16* __restrict__ o,
@@ -55,18 +53,22 @@ __global__ void __launch_bounds__(256) delta_kernel(const __nv_bfloat16* __restr
 }
 
 // ------------------------------------------------------------------------------------------------------------------
-// dQ
+// dQ: key tiles of 128 rows, so that every MMA has N = 128 (the N = 64 shape is bound by operand reads, not by the
+// tensor pipe).  Tensor memory: S in two buffers (S of tile n+1 runs under the element-wise pass of tile n), dP, dQ.
 // ------------------------------------------------------------------------------------------------------------------
+constexpr int BKW = 128;                       // key rows per tile
+constexpr int KW_BYTES = BKW * D * 2;          // 32 KB: two panels [128 rows][64 columns]
+constexpr int KST = 3;                         // K stages (a K tile is held from S to dQ); V has two (held for dP only)
 struct SmemQ {
-    static constexpr int q = 0, dO = Q_BYTES, k0 = 2 * Q_BYTES, v0 = k0 + STAGES * KV_BYTES,
-                         misc = v0 + STAGES * KV_BYTES;
+    static constexpr int q = 0, dO = Q_BYTES, k0 = 2 * Q_BYTES, v0 = k0 + KST * KW_BYTES, misc = v0 + 2 * KW_BYTES;
     static constexpr int bytes = misc + 256;
 };
 struct MiscQ {
-    uint64_t bar_q, bar_kv[STAGES], bar_s[2], bar_p[2], bar_free[STAGES], bar_o;
+    uint64_t bar_q, bar_k[KST], bar_v[2], bar_kfree[KST], bar_vfree[2], bar_s, bar_dpfree, bar_p, bar_o;
     uint32_t tmem;
 };
-constexpr int COL_DQ = 256, TMEM_Q = 512;     // S at 128 b, dP at 128 b + 64 (b = buffer), dQ at 256
+constexpr int COL_DP = 256, COL_DQ = 384, TMEM_Q = 512;     // S of tile n at 128 (n & 1)
+using WalkW = TileWalkT<BKW>;
 
 __global__ void __launch_bounds__(NT, 1)
 attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUtensorMap map_q,
@@ -83,8 +85,17 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
     const bool is_softmax = warp < NS / 32, is_issuer = tid == NS, is_producer = tid == NS + 32;
     if (tid == 0) {
         mbar_init(&m.bar_q, 1);
-        for (int s = 0; s < STAGES; s++) { mbar_init(&m.bar_kv[s], 1); mbar_init(&m.bar_free[s], 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(&m.bar_s[b], 1); mbar_init(&m.bar_p[b], NS / 32); }
+        for (int st = 0; st < KST; st++) {
+            mbar_init(&m.bar_k[st], 1);
+            mbar_init(&m.bar_kfree[st], 1);
+        }
+        for (int st = 0; st < 2; st++) {
+            mbar_init(&m.bar_v[st], 1);
+            mbar_init(&m.bar_vfree[st], 1);
+        }
+        mbar_init(&m.bar_s, 1);
+        mbar_init(&m.bar_dpfree, NS / 32);
+        mbar_init(&m.bar_p, NS / 32);
         mbar_init(&m.bar_o, 1);
         fence_barrier_init();
     }
@@ -94,12 +105,13 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
     tc_fence_after();
     const uint32_t tmem = m.tmem;
     const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    constexpr uint32_t I_S = instr_desc(BQ, BK, 0, 0);     // [128 x 64] = (Q | dO) (K-major) . (K | V) (K-major)
+    constexpr uint32_t I_S = instr_desc(BQ, BKW, 0, 0);    // [128 x 128] = (Q | dO) (K-major) . (K | V) (K-major)
     constexpr uint32_t I_DQ = instr_desc(BQ, D, 0, 1);     // dQ[128 x 128] += dS (tensor memory) . K (rows = keys)
     const uint64_t dQd = desc_kmajor_base(smem_u32(sQ)), dDOd = desc_kmajor_base(smem_u32(sDO));
     const float scale_log2 = scale * LOG2E;
 
-    uint32_t ph_q = 0, ph_kv[STAGES] = {}, ph_free[STAGES] = {}, ph_s[2] = {0, 0}, ph_p[2] = {0, 0}, ph_o = 0;
+    uint32_t ph_q = 0, ph_k[KST] = {}, ph_v[2] = {0, 0}, ph_kfree[KST] = {}, ph_vfree[2] = {0, 0}, ph_s = 0, ph_p = 0,
+             ph_dpfree = 0, ph_o = 0;
     const int n_work = ix.n_q_items * Hq;
     for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
         const int item = w / Hq, h = w % Hq, hk = h / G;
@@ -108,8 +120,8 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
         const int q_valid = min(BQ, ix.piece_len[piece] - qt * BQ);
 
         if (is_producer) {
-            // ---- TMA producer: Q and dO tiles, then the key/value tiles STAGES deep ---------------------------------
-            TileWalk lw(ix, piece, qt);
+            // ---- TMA producer: Q and dO tiles, then K and V tiles two deep (released separately) --------------------
+            WalkW lw(ix, piece, qt);
             KvTile lt;
             mbar_expect_tx(&m.bar_q, 2 * Q_BYTES);
             for (int p = 0; p < 2; p++)
@@ -118,90 +130,125 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                     tma_load_3d(sDO + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_do, p * 64, h, q_row0 + r * 64, &m.bar_q);
                 }
             for (int n = 0; lw.next(lt); n++) {
-                const int stage = n % STAGES;
-                if (n >= STAGES) {
-                    mbar_wait(&m.bar_free[stage], ph_free[stage], status);
-                    ph_free[stage] ^= 1;
+                const int stage = n & 1, kst = n % KST;
+                unsigned char* sK = smem + SmemQ::k0 + kst * KW_BYTES;
+                unsigned char* sV = smem + SmemQ::v0 + stage * KW_BYTES;
+                if (n >= KST) {
+                    mbar_wait(&m.bar_kfree[kst], ph_kfree[kst], status);         // released after dQ of tile n - KST
+                    ph_kfree[kst] ^= 1;
                 }
-                unsigned char* sK = smem + SmemQ::k0 + stage * KV_BYTES;
-                unsigned char* sV = smem + SmemQ::v0 + stage * KV_BYTES;
-                mbar_expect_tx(&m.bar_kv[stage], 2 * KV_BYTES);
-                for (int p = 0; p < 2; p++) {
-                    tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, lt.row, &m.bar_kv[stage]);
-                    tma_load_3d(sV + p * (KV_BYTES / 2), &map_v, p * 64, hk, lt.row, &m.bar_kv[stage]);
+                mbar_expect_tx(&m.bar_k[kst], KW_BYTES);
+                for (int p = 0; p < 2; p++)
+                    for (int r = 0; r < 2; r++)
+                        tma_load_3d(sK + p * (KW_BYTES / 2) + r * (KW_BYTES / 4), &map_k, p * 64, hk, lt.row + r * 64, &m.bar_k[kst]);
+                if (n >= 2) {
+                    mbar_wait(&m.bar_vfree[stage], ph_vfree[stage], status);     // released after dP of tile n - 2
+                    ph_vfree[stage] ^= 1;
                 }
+                mbar_expect_tx(&m.bar_v[stage], KW_BYTES);
+                for (int p = 0; p < 2; p++)
+                    for (int r = 0; r < 2; r++)
+                        tma_load_3d(sV + p * (KW_BYTES / 2) + r * (KW_BYTES / 4), &map_v, p * 64, hk, lt.row + r * 64, &m.bar_v[stage]);
             }
         }
         if (is_issuer) {
             // ---- MMA issue: this thread does nothing else, a tcgen05.mma holds it until the pipe has room ---------
-            const int n_tiles = TileWalk(ix, piece, qt).count();
-            auto issue_s = [&](int n) {      // S(n) and dP(n) into buffer n & 1
-                const int stage = n % STAGES, b = n & 1;
-                mbar_wait(&m.bar_kv[stage], ph_kv[stage], status);
-                ph_kv[stage] ^= 1;
+            const int n_tiles = WalkW(ix, piece, qt).count();
+            auto issue_s = [&](int n) {      // S(n) into buffer n & 1
+                const int stage = n & 1, kst = n % KST;
+                mbar_wait(&m.bar_k[kst], ph_k[kst], status);
+                ph_k[kst] ^= 1;
                 tc_fence_after();
-                const uint64_t dK = desc_kmajor_base(smem_u32(smem + SmemQ::k0 + stage * KV_BYTES));
-                const uint64_t dV = desc_kmajor_base(smem_u32(smem + SmemQ::v0 + stage * KV_BYTES));
+                const uint64_t dK = desc_kmajor_base(smem_u32(smem + SmemQ::k0 + kst * KW_BYTES));
 #pragma unroll
                 for (int ks = 0; ks < 8; ks++)
-                    mma_ss(tmem + b * 128, dQd + kstep_kmajor<BQ>(ks), dK + kstep_kmajor<BK>(ks), I_S, ks > 0);
+                    mma_ss(tmem + stage * 128, dQd + kstep_kmajor<BQ>(ks), dK + kstep_kmajor<BKW>(ks), I_S, ks > 0);
+            };
+            auto issue_dp = [&](int n) {     // dP(n); its commit also covers S(n), issued before it
+                const int stage = n & 1;
+                mbar_wait(&m.bar_v[stage], ph_v[stage], status);
+                ph_v[stage] ^= 1;
+                tc_fence_after();
+                const uint64_t dV = desc_kmajor_base(smem_u32(smem + SmemQ::v0 + stage * KW_BYTES));
 #pragma unroll
                 for (int ks = 0; ks < 8; ks++)
-                    mma_ss(tmem + b * 128 + 64, dDOd + kstep_kmajor<BQ>(ks), dV + kstep_kmajor<BK>(ks), I_S, ks > 0);
-                mma_commit(&m.bar_s[b]);
+                    mma_ss(tmem + COL_DP, dDOd + kstep_kmajor<BQ>(ks), dV + kstep_kmajor<BKW>(ks), I_S, ks > 0);
+                mma_commit(&m.bar_s);
+                if (n + 2 < n_tiles) mma_commit(&m.bar_vfree[stage]);
             };
             mbar_wait(&m.bar_q, ph_q, status);
             ph_q ^= 1;
             issue_s(0);
+            issue_dp(0);
             for (int n = 0; n < n_tiles; n++) {
-                if (n + 1 < n_tiles) issue_s(n + 1);            // runs under the element-wise pass of tile n
-                const int stage = n % STAGES, b = n & 1;
-                mbar_wait(&m.bar_p[b], ph_p[b], status);
-                ph_p[b] ^= 1;
+                const int stage = n & 1;
+                // S(n+1) and dP(n+1) run under the element-wise pass of tile n: S has a second buffer, and the pass
+                // takes dP(n) into registers first and says so
+                if (n + 1 < n_tiles) {
+                    issue_s(n + 1);
+                    mbar_wait(&m.bar_dpfree, ph_dpfree, status);
+                    ph_dpfree ^= 1;
+                    tc_fence_after();
+                    issue_dp(n + 1);
+                }
+                mbar_wait(&m.bar_p, ph_p, status);              // dS(n) written, S(n) read
+                ph_p ^= 1;
                 tc_fence_after();
-                const uint64_t dKm = desc_mnmajor_base<BK>(smem_u32(smem + SmemQ::k0 + stage * KV_BYTES));
+                const uint64_t dKm = desc_mnmajor_base<BKW>(smem_u32(smem + SmemQ::k0 + (n % KST) * KW_BYTES));
 #pragma unroll
-                for (int ks = 0; ks < 4; ks++)
-                    mma_ts(tmem + COL_DQ, tmem + b * 128 + (ks >> 1) * 32 + (ks & 1) * 8, dKm + kstep_mnmajor(ks), I_DQ, n > 0 || ks > 0);
-                if (n + STAGES < n_tiles) mma_commit(&m.bar_free[stage]);     // this stage will be refilled
+                for (int ks = 0; ks < 8; ks++)
+                    mma_ts(tmem + COL_DQ, tmem + stage * 128 + (ks >> 2) * 64 + (ks & 3) * 8, dKm + kstep_mnmajor(ks), I_DQ,
+                           n > 0 || ks > 0);
+                if (n + KST < n_tiles) mma_commit(&m.bar_kfree[n % KST]);
                 if (n + 1 == n_tiles) mma_commit(&m.bar_o);
             }
         }
         if (is_softmax) {
-            TileWalk walk(ix, piece, qt);
+            WalkW walk(ix, piece, qt);
             KvTile t;
-            const int i = tid & 127, c = tid >> 7;           // query row, and which 32 of a tile's 64 key columns
+            const int i = tid & 127, c = tid >> 7;           // query row, and which 64 of a tile's 128 key columns
             const bool row_ok = i < q_valid;
             // rows past the end of the piece: lse = +inf makes every probability 0
             const float lse2 = row_ok ? lse[(size_t)(q_row0 + i) * Hq + h] * LOG2E : INFINITY;
             const float dl = row_ok ? delta[(size_t)(q_row0 + i) * Hq + h] : 0.f;
             for (int n = 0; walk.next(t); n++) {
                 const int b = n & 1;
-                mbar_wait_warp(&m.bar_s[b], ph_s[b], status);
-                ph_s[b] ^= 1;
+                mbar_wait_warp(&m.bar_s, ph_s, status);
+                ph_s ^= 1;
                 tc_fence_after();
-                const int limit = min(t.n_valid, t.shift == NO_DIAG ? BK : i - t.shift + 1);
-                {
-                    uint32_t xs[32], xp[32], pk[16];
-                    tmem_ld32(tm_lane + b * 128 + c * 32, xs);
-                    tmem_ld32(tm_lane + b * 128 + 64 + c * 32, xp);
+                const int limit = min(t.n_valid, t.shift == NO_DIAG ? BKW : i - t.shift + 1);
+                // dP of this thread's 64 columns into registers, so that the buffer can take dP of the next tile
+                uint32_t xp[64];
+                tmem_ld32(tm_lane + COL_DP + c * 64, xp);
+                tmem_ld32(tm_lane + COL_DP + c * 64 + 32, xp + 32);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                const bool last_tile = walk.in_own && walk.off >= walk.own_end;     // no dP follows the last tile
+                if (lane == 0 && !last_tile) mbar_arrive(&m.bar_dpfree);
+#pragma unroll
+                for (int cc = 0; cc < 2; cc++) {
+                    const int j0 = c * 64 + cc * 32;
+                    uint32_t xs[32], pk[16];
+                    tmem_ld32(tm_lane + b * 128 + j0, xs);
                     tmem_ld_wait();
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
                         float ds[2];
 #pragma unroll
                         for (int u = 0; u < 2; u++) {
-                            const float p = c * 32 + e + u < limit ? ex2(fmaf(__uint_as_float(xs[e + u]), scale_log2, -lse2)) : 0.f;
-                            ds[u] = p * (__uint_as_float(xp[e + u]) - dl) * scale;
+                            const float p = j0 + e + u < limit ? ex2(fmaf(__uint_as_float(xs[e + u]), scale_log2, -lse2)) : 0.f;
+                            ds[u] = p * (__uint_as_float(xp[cc * 32 + e + u]) - dl) * scale;
                         }
                         pk[e >> 1] = pack_bf16(ds[0], ds[1]);
                     }
-                    tmem_st16(tm_lane + b * 128 + c * 32, pk);      // over this warp's own half of S (the other warp may still be reading its half)
+                    // over this thread's own half of S (columns it has already read)
+                    tmem_st16(tm_lane + b * 128 + c * 64 + cc * 16, pk);
                 }
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&m.bar_p[b]);
+                if (lane == 0) mbar_arrive(&m.bar_p);
             }
             // ---- epilogue: dQ -> bf16 ------------------------------------------------------------------------------
             mbar_wait_warp(&m.bar_o, ph_o, status);

@@ -35,11 +35,12 @@ struct KvTile {
     int row, n_valid, shift;
 };
 
-struct TileWalk {       // enumerates the key tiles of one item in order; run data is read once per run, not per tile
+template <int W>
+struct TileWalkT {      // enumerates the key tiles (W rows) of one item in order; run data is read once per run, not per tile
     const Index& ix;
     int run0, run, run_end, off, own_row0, own_end, q0, cur_row0, cur_len;
     bool in_own;
-    __device__ TileWalk(const Index& ix_, int piece, int qt) : ix(ix_) {
+    __device__ TileWalkT(const Index& ix_, int piece, int qt) : ix(ix_) {
         run0 = run = ix.anc_ptr[piece];
         run_end = ix.anc_ptr[piece + 1];
         off = 0;
@@ -54,16 +55,16 @@ struct TileWalk {       // enumerates the key tiles of one item in order; run da
         }
     }
     __device__ int count() const {          // number of tiles next() will deliver from a fresh walk
-        int n = (own_end + BK - 1) / BK;
-        for (int r = run0; r < run_end; r++) n += (ix.anc_len[r] + BK - 1) / BK;
+        int n = (own_end + W - 1) / W;
+        for (int r = run0; r < run_end; r++) n += (ix.anc_len[r] + W - 1) / W;
         return n;
     }
     __device__ bool next(KvTile& t) {
         if (!in_own) {
             t.row = cur_row0 + off;
-            t.n_valid = min(BK, cur_len - off);
+            t.n_valid = min(W, cur_len - off);
             t.shift = NO_DIAG;
-            off += BK;
+            off += W;
             if (off >= cur_len) {
                 off = 0;
                 if (++run == run_end) {
@@ -77,12 +78,13 @@ struct TileWalk {       // enumerates the key tiles of one item in order; run da
         }
         if (off >= own_end) return false;
         t.row = own_row0 + off;
-        t.n_valid = min(BK, own_end - off);
+        t.n_valid = min(W, own_end - off);
         t.shift = off - q0;
-        off += BK;
+        off += W;
         return true;
     }
 };
+using TileWalk = TileWalkT<BK>;
 
 // The query tiles (64 rows) that see the key tile `kt` (128 rows) of a piece: for every query head of the group,
 // the rest of the piece from the key tile's first row on (causal inside), then all rows of every descendant piece.
