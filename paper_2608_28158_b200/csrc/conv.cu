@@ -4,7 +4,9 @@
 // Both passes are HBM-bound streams: a thread owns 8 channels (one 16-byte vector of bf16), keeps its filter taps
 // in registers and walks a strip of consecutive rows with the w-1 neighbouring rows it needs in a register window,
 // so every row of x and dy leaves HBM once; only where the packed order is not the trajectory order (a branch or
-// sequence start, a fork) does it follow the index tables, and those rows come from L2.  Algorithmic bytes per row: forward 2*D*e, backward 3*D*e.  No contraction, no tensor cores.
+// sequence start, a fork) does it follow the index tables, and those rows come from L2.  The rows of the walk are
+// prefetched eight iterations ahead with cp.async into per-thread shared-memory slots, so the bytes in flight do
+// not cost registers (the backward holds 32 taps and 32 dW accumulators per thread).  Algorithmic bytes per row: forward 2*D*e, backward 3*D*e.  No contraction, no tensor cores.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -98,12 +100,21 @@ template <> struct Raw<float> {
     }
 };
 
+// Register-free prefetch: a thread copies the rows it will need a few iterations ahead into its own slots of a
+// shared-memory ring with cp.async (nobody else reads them, so no barrier is needed, only wait_group).
+template <typename T> struct Ring { static constexpr int DEPTH = sizeof(T) == 2 ? 8 : 4; };
+template <typename T>
+__device__ __forceinline__ void ring_fetch(Raw<T>* slot, const T* src) {
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(slot));
+#pragma unroll
+    for (int i = 0; i < static_cast<int>(sizeof(Raw<T>)) / 16; ++i)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16 * i), "l"(reinterpret_cast<const char*>(src) + 16 * i)
+                     : "memory");
+}
+__device__ __forceinline__ void ring_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void ring_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 constexpr int STRIP = 128;   // consecutive rows one thread walks with its sliding window
-constexpr int UNR = 4;       // rows whose loads are in flight together (forward)
-#ifndef CONV_UNR_B
-#define CONV_UNR_B 3
-#endif
-constexpr int UNR_B = CONV_UNR_B;   // the same for the backward, which streams two tensors
 
 // Forward.  A thread walks a strip of consecutive rows upwards and keeps the last w-1 rows in registers: as long
 // as a row's predecessor is the row before it (inside a sequence) the window just shifts and the row costs one
@@ -115,25 +126,31 @@ __global__ void __launch_bounds__(NT, 3) conv_fwd_kernel(const T* __restrict__ x
                                                          int n_rows, int D, int CX) {
     const Lane l = lane_of(CX, D / 8);
     if (!l.active) return;
+    constexpr int DEPTH = Ring<T>::DEPTH;
+    extern __shared__ __align__(16) unsigned char ring_raw[];
+    Raw<T>* ring_x = reinterpret_cast<Raw<T>*>(ring_raw) + threadIdx.x;          // [DEPTH][NT] slots of this thread
     float taps[W_][8];
     load_taps<W_>(W, l.g, taps);
     const size_t col = 8 * (size_t)l.g;
     for (int strip = blockIdx.x * l.RY + l.ry; strip * STRIP < n_rows; strip += gridDim.x * l.RY) {
         const int r0 = strip * STRIP, r1 = min(n_rows, r0 + STRIP);
         Raw<T> h[W_ - 1];                                  // h[i] = x of the (i+1)-th ancestor of the current row
-        for (int rb = r0; rb < r1; rb += UNR) {
-            Raw<T> xs[UNR];
-            int pv[UNR];
 #pragma unroll
-            for (int u = 0; u < UNR; ++u)
-                if (rb + u < r1) {
-                    xs[u].load(x + (size_t)(rb + u) * D + col);
-                    pv[u] = prev[rb + u];
-                }
-#pragma unroll
-            for (int u = 0; u < UNR; ++u) {
-                const int r = rb + u;
-                if (r >= r1) break;
+        for (int k = 0; k < DEPTH; ++k) {                  // prologue of the ring: the first DEPTH rows of the strip
+            if (r0 + k < r1) ring_fetch(ring_x + k * NT, x + (size_t)(r0 + k) * D + col);
+            ring_commit();
+        }
+        int pv_next = prev[r0];
+        for (int k = 0, r = r0; r < r1; ++k, ++r) {
+            {
+                const int slot = k % DEPTH;
+                ring_wait<DEPTH - 1>();                    // row r has landed
+                Raw<T> xs[1] = {ring_x[slot * NT]};
+                if (r + DEPTH < r1) ring_fetch(ring_x + slot * NT, x + (size_t)(r + DEPTH) * D + col);
+                ring_commit();
+                const int pv[1] = {pv_next};
+                if (r + 1 < r1) pv_next = prev[r + 1];
+                constexpr int u = 0;
                 if (pv[u] != r - 1 || r == r0) {           // chain break: rebuild the window from the true ancestors
                     int a = pv[u];
 #pragma unroll
@@ -162,6 +179,7 @@ __global__ void __launch_bounds__(NT, 3) conv_fwd_kernel(const T* __restrict__ x
                 h[0] = xs[u];
             }
         }
+        ring_wait<0>();
     }
 }
 
@@ -178,6 +196,10 @@ __global__ void __launch_bounds__(NT, 2) conv_bwd_kernel(const T* __restrict__ x
                                                          float* __restrict__ partial, int n_rows, int D, int CX) {
     const Lane l = lane_of(CX, D / 8);
     if (!l.active) return;
+    constexpr int DEPTH = Ring<T>::DEPTH;
+    extern __shared__ __align__(16) unsigned char ring_raw[];
+    Raw<T>* ring_x = reinterpret_cast<Raw<T>*>(ring_raw) + threadIdx.x;          // [DEPTH][NT] slots of this thread
+    Raw<T>* ring_g = ring_x + DEPTH * NT;
     float taps[W_][8], dw[W_][8];
     load_taps<W_>(W, l.g, taps);
 #pragma unroll
@@ -189,20 +211,33 @@ __global__ void __launch_bounds__(NT, 2) conv_bwd_kernel(const T* __restrict__ x
         const int r0 = strip * STRIP, r1 = min(n_rows, r0 + STRIP);
         Raw<T> d[W_ - 1];                                  // d[i] = dy of row r + 1 + i (valid while `run` says so)
         int run = 0;                                       // plain-chain links known below the current row
-        for (int rt = r1 - 1; rt >= r0; rt -= UNR_B) {
-            Raw<T> xs[UNR_B], gs[UNR_B];
-            int nx[UNR_B];
+        // prologue of the ring: the first DEPTH rows of the walk (top of the strip downwards)
 #pragma unroll
-            for (int u = 0; u < UNR_B; ++u)
-                if (rt - u >= r0) {
-                    xs[u].load(x + (size_t)(rt - u) * D + col);
-                    gs[u].load(dy + (size_t)(rt - u) * D + col);
-                    nx[u] = next_row[rt - u];
+        for (int k = 0; k < DEPTH; ++k) {
+            const int r = r1 - 1 - k;
+            if (r >= r0) {
+                ring_fetch(ring_x + k * NT, x + (size_t)r * D + col);
+                ring_fetch(ring_g + k * NT, dy + (size_t)r * D + col);
+            }
+            ring_commit();
+        }
+        int nx_next = next_row[r1 - 1];
+        for (int k = 0, r = r1 - 1; r >= r0; ++k, --r) {
+            {
+                const int slot = k % DEPTH;
+                ring_wait<DEPTH - 1>();                    // the oldest group, i.e. row r, has landed
+                const Raw<T> xs_r = ring_x[slot * NT], gs_r = ring_g[slot * NT];
+                const int rn = r - DEPTH;                  // refill the slot with the row DEPTH iterations ahead
+                if (rn >= r0) {
+                    ring_fetch(ring_x + slot * NT, x + (size_t)rn * D + col);
+                    ring_fetch(ring_g + slot * NT, dy + (size_t)rn * D + col);
                 }
-#pragma unroll
-            for (int u = 0; u < UNR_B; ++u) {
-                const int r = rt - u;
-                if (r < r0) break;
+                ring_commit();
+                const int nx_r = nx_next;
+                if (r > r0) nx_next = next_row[r - 1];
+                Raw<T> xs[1] = {xs_r}, gs[1] = {gs_r};
+                const int nx[1] = {nx_r};
+                constexpr int u = 0;
                 float xf[8], g0[8], acc[8], f[8];
                 xs[u].get(xf);
                 gs[u].get(g0);
@@ -259,6 +294,7 @@ __global__ void __launch_bounds__(NT, 2) conv_bwd_kernel(const T* __restrict__ x
                 d[0] = gs[u];
             }
         }
+        ring_wait<0>();
     }
     // partial[slot][channel][tap], slot = (blockIdx.x, ry)
     float* dst = partial + ((size_t)(blockIdx.x * l.RY + l.ry) * D + col) * W_;
@@ -320,18 +356,23 @@ void launch_fwd(const Shape& s, cudaStream_t st, const void* x, const float* W, 
                 int D, int w) {
     const T* xx = static_cast<const T*>(x);
     T* yy = static_cast<T*>(y);
-    if (w == 2) conv_fwd_kernel<T, 2><<<s.grid, NT, 0, st>>>(xx, W, prev, yy, n, D, s.CX);
-    if (w == 3) conv_fwd_kernel<T, 3><<<s.grid, NT, 0, st>>>(xx, W, prev, yy, n, D, s.CX);
-    if (w == 4) conv_fwd_kernel<T, 4><<<s.grid, NT, 0, st>>>(xx, W, prev, yy, n, D, s.CX);
+    constexpr size_t ring_bytes = (size_t)Ring<T>::DEPTH * NT * sizeof(Raw<T>);          // 32 KB
+    if (w == 2) conv_fwd_kernel<T, 2><<<s.grid, NT, ring_bytes, st>>>(xx, W, prev, yy, n, D, s.CX);
+    if (w == 3) conv_fwd_kernel<T, 3><<<s.grid, NT, ring_bytes, st>>>(xx, W, prev, yy, n, D, s.CX);
+    if (w == 4) conv_fwd_kernel<T, 4><<<s.grid, NT, ring_bytes, st>>>(xx, W, prev, yy, n, D, s.CX);
 }
 template <typename T>
 void launch_bwd(const Shape& s, cudaStream_t st, const void* x, const float* W, const void* dy, const int32_t* prev,
                 const int32_t* cp, const int32_t* cr, void* dx, float* partial, int n, int D, int w) {
     const T *xx = static_cast<const T*>(x), *gg = static_cast<const T*>(dy);
     T* dd = static_cast<T*>(dx);
-    if (w == 2) conv_bwd_kernel<T, 2><<<s.grid, NT, 0, st>>>(xx, W, gg, prev, cp, cr, dd, partial, n, D, s.CX);
-    if (w == 3) conv_bwd_kernel<T, 3><<<s.grid, NT, 0, st>>>(xx, W, gg, prev, cp, cr, dd, partial, n, D, s.CX);
-    if (w == 4) conv_bwd_kernel<T, 4><<<s.grid, NT, 0, st>>>(xx, W, gg, prev, cp, cr, dd, partial, n, D, s.CX);
+    constexpr size_t ring_bytes = 2 * (size_t)Ring<T>::DEPTH * NT * sizeof(Raw<T>);      // 64 KB
+    cudaFuncSetAttribute(conv_bwd_kernel<T, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring_bytes);
+    cudaFuncSetAttribute(conv_bwd_kernel<T, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring_bytes);
+    cudaFuncSetAttribute(conv_bwd_kernel<T, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring_bytes);
+    if (w == 2) conv_bwd_kernel<T, 2><<<s.grid, NT, ring_bytes, st>>>(xx, W, gg, prev, cp, cr, dd, partial, n, D, s.CX);
+    if (w == 3) conv_bwd_kernel<T, 3><<<s.grid, NT, ring_bytes, st>>>(xx, W, gg, prev, cp, cr, dd, partial, n, D, s.CX);
+    if (w == 4) conv_bwd_kernel<T, 4><<<s.grid, NT, ring_bytes, st>>>(xx, W, gg, prev, cp, cr, dd, partial, n, D, s.CX);
 }
 
 }  // namespace
