@@ -23,6 +23,10 @@ Pins (see tests/test_oracle_*.py, tests/test_plan_oracle.py):
                    scaled_dot_product_attention on every expanded trajectory with autograd
                    through the expansion, the bottom-right mask of a branch view, equal-keys
                    closed form, central differences.
+  * mb_oracle   -- microbatch planning (Section 3.2): Eq. 5 / Eq. 6 / the range-minimum LCP rule
+                   against the brute-force trie count, hand-counted costs of the five-node tree,
+                   the slot-schedule rule; the search itself has no closed form and is checked
+                   for validity and against brute force over contiguous cuts.
   * Appendix planning cases I-III: parity unpinned (the trees' token counts were only in
                    the figures); only the printed totals are checked for self-consistency.
 """
