@@ -15,3 +15,4 @@ from .logp import (  # noqa: F401
 )
 from .conv import harts_conv_index, harts_conv_fwd, harts_conv_scratch_bytes, harts_conv_bwd  # noqa: F401
 from .attn import AttnIndex, harts_attn_index, harts_attn_fwd, harts_attn_bwd  # noqa: F401
+from .mb import MbPlan, harts_mb_plan  # noqa: F401

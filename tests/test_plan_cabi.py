@@ -131,7 +131,9 @@ def test_library_exports_every_declared_symbol():
     header += open(os.path.join(ROOT, "include", "harts_logp.h")).read()
     header += open(os.path.join(ROOT, "include", "harts_conv.h")).read()
     header += open(os.path.join(ROOT, "include", "harts_attn.h")).read()
-    names = set(re.findall(r"\b(harts_(?:la|logp|conv|attn)_\w+)\s*\(", header))
+    header += open(os.path.join(ROOT, "include", "harts_mb.h")).read()
+    names = set(re.findall(r"\b(harts_(?:la|logp|conv|attn|mb)_\w+)\s*\(", header))
+    assert {"harts_mb_plan", "harts_mb_plan_free", "harts_mb_plan_view", "harts_mb_extract"} <= names
     assert {"harts_attn_index", "harts_attn_fwd", "harts_attn_bwd"} <= names
     assert {"harts_conv_index", "harts_conv_fwd", "harts_conv_bwd", "harts_conv_scratch_bytes"} <= names
     assert {"harts_la_plan", "harts_la_fwd", "harts_la_bwd", "harts_logp_fwd", "harts_logp_bwd",
