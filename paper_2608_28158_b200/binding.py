@@ -242,6 +242,50 @@ def run_fwd_bwd_host(plan: Plan, ws: Workspace, host_in: dict, dev_in: dict, dev
     return host_out
 
 
+class HostPipeline:
+    """End-to-end steps on HOST buffers with the copies of neighbouring steps overlapped: three streams (inputs
+    in, kernels, results out) and two sets of device tensors, so that while step i computes, the inputs of step
+    i+1 arrive and the results of step i-1 leave.  Every step still copies all of its inputs from the (pinned)
+    host buffers and all of its results back; the kernels of successive steps share one workspace and run in order."""
+
+    def __init__(self, plan: Plan, ws: Workspace, like_in: dict, like_out: dict):
+        self.plan, self.ws = plan, ws
+        self.sets = [({n: torch.empty_like(x) for n, x in like_in.items()},
+                      {n: torch.empty_like(x) for n, x in like_out.items()}) for _ in range(2)]
+        self.s_in, self.s_run, self.s_out = (torch.cuda.Stream() for _ in range(3))
+        self.ev_in = [torch.cuda.Event() for _ in range(2)]
+        self.ev_run = [torch.cuda.Event() for _ in range(2)]
+        self.ev_out = [torch.cuda.Event() for _ in range(2)]
+        self.n = 0
+
+    def step(self, host_in: dict, host_out: dict):
+        i = self.n % 2
+        dev_in, dev_out = self.sets[i]
+        with torch.cuda.stream(self.s_in):
+            if self.n >= 2:
+                self.s_in.wait_event(self.ev_run[i])          # the kernels of step n-2 have read this input set
+            for n in ("q", "k", "v", "g", "dO"):
+                dev_in[n].copy_(host_in[n], non_blocking=True)
+            self.ev_in[i].record(self.s_in)
+        with torch.cuda.stream(self.s_run):
+            self.s_run.wait_event(self.ev_in[i])
+            if self.n >= 2:
+                self.s_run.wait_event(self.ev_out[i])         # the results of step n-2 have left this output set
+            run_fwd_bwd(self.plan, self.ws, dev_in["q"], dev_in["k"], dev_in["v"], dev_in["g"], dev_in["dO"], out=dev_out,
+                        stream=self.s_run)
+            self.ev_run[i].record(self.s_run)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_run[i])
+            for n in ("o", "dq", "dk", "dv", "dg"):
+                host_out[n].copy_(dev_out[n], non_blocking=True)
+            self.ev_out[i].record(self.s_out)
+        self.n += 1
+
+    def finish(self):
+        for s in (self.s_in, self.s_run, self.s_out):
+            s.synchronize()
+
+
 def expand_trajectories(tree_node_ptr, node_parent, node_fork_off, node_len):
     """Trajectory-wise view of a forest (the conventional baseline of Section 5): every root-to-leaf
     path becomes its own single-node tree.  Returns (forest arrays of the expanded problem,
