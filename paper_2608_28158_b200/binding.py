@@ -92,7 +92,8 @@ def _stream(stream):
 
 
 class Plan:
-    """Host plan (owned by the library) plus, after ``upload``, its device index blob."""
+    """Host plan (owned by the library) plus, after ``upload``, its device index blob.  The index arrays are
+    read-only views of the library's memory; copy them if they must outlive the plan."""
 
     def __init__(self, handle):
         self._h = handle
@@ -111,7 +112,9 @@ class Plan:
             size = sizes[n]
             if n == "slot_cons_seq":
                 size = int(self.slot_cons_ptr[-1])
-            arr = np.ctypeslib.as_array(getattr(v, n), shape=(size,)).copy() if size else np.zeros(0, np.int32)
+            # views into the library-owned plan (no copy): valid as long as this object lives
+            arr = np.ctypeslib.as_array(getattr(v, n), shape=(size,)) if size else np.zeros(0, np.int32)
+            arr.flags.writeable = False
             setattr(self, n, arr)
         self.C, self.R = self.n_rows, self.n_replay
         self.blob = None

@@ -371,18 +371,31 @@ int32_t build_plan(int32_t n_trees, const int32_t* tree_node_ptr, const int32_t*
     // replay-gradient CSR: for every replayed physical row the replay entries that read it
     {
         const int32_t R = P.n_replay;
-        std::vector<int32_t> ent(R);
-        for (int32_t e = 0; e < R; e++) ent[e] = e;
-        std::stable_sort(ent.begin(), ent.end(),
-                         [&](int32_t a, int32_t b) { return P.replay_row[a] < P.replay_row[b]; });
         P.rg_row.clear();
         P.rg_ptr.assign(1, 0);
-        P.rg_entry.assign(ent.begin(), ent.end());
-        for (int32_t e = 0; e < R; e++) {
-            int32_t r = P.replay_row[ent[e]];
-            if (P.rg_row.empty() || P.rg_row.back() != r) {
-                if (!P.rg_row.empty()) P.rg_ptr.push_back(e);
-                P.rg_row.push_back(r);
+        P.rg_entry.resize(R);
+        if ((int64_t)R * 16 > C) {
+            // many replay entries: counting sort by the row they read (stable: one row's entries stay in entry order)
+            std::vector<int32_t> first(C + 1, 0);
+            for (int32_t e = 0; e < R; e++) first[P.replay_row[e] + 1]++;
+            for (int32_t r = 0; r < C; r++) {
+                if (first[r + 1]) {
+                    if (!P.rg_row.empty()) P.rg_ptr.push_back(first[r]);
+                    P.rg_row.push_back(r);
+                }
+                first[r + 1] += first[r];
+            }
+            for (int32_t e = 0; e < R; e++) P.rg_entry[first[P.replay_row[e]]++] = e;
+        } else {
+            for (int32_t e = 0; e < R; e++) P.rg_entry[e] = e;
+            std::stable_sort(P.rg_entry.begin(), P.rg_entry.end(),
+                             [&](int32_t a, int32_t b) { return P.replay_row[a] < P.replay_row[b]; });
+            for (int32_t e = 0; e < R; e++) {
+                int32_t r = P.replay_row[P.rg_entry[e]];
+                if (P.rg_row.empty() || P.rg_row.back() != r) {
+                    if (!P.rg_row.empty()) P.rg_ptr.push_back(e);
+                    P.rg_row.push_back(r);
+                }
             }
         }
         if (R > 0) P.rg_ptr.push_back(R);
