@@ -42,7 +42,7 @@ struct Smem {
     static constexpr int bytes = misc + 256;
 };
 struct Misc {
-    uint64_t bar_q, bar_k[2], bar_v[2], bar_kfree[2], bar_vfree[2], bar_s[2], bar_p, bar_o;
+    uint64_t bar_q, bar_k[2], bar_v[2], bar_kfree[2], bar_vfree[2], bar_s[2], bar_p, bar_pv, bar_o;
     uint32_t tmem;
 };
 
@@ -70,6 +70,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
         mbar_init(&m.bar_s[0], 1);
         mbar_init(&m.bar_s[1], 1);
         mbar_init(&m.bar_p, NS / 32);
+        mbar_init(&m.bar_pv, 1);
         mbar_init(&m.bar_o, 1);
         fence_barrier_init();
     }
@@ -85,6 +86,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
     const uint32_t aQ = smem_u32(sQ);
     const uint64_t dQ = desc_kmajor_base(aQ);
 
+    uint32_t tiles_done = 0;                     // key tiles this CTA has processed (the phase index of bar_pv)
     uint32_t ph_q = 0, ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_kfree[2] = {0, 0}, ph_vfree[2] = {0, 0}, ph_s[2] = {0, 0},
              ph_p = 0, ph_o = 0;
     const int n_work = ix.n_q_items * Hq;
@@ -156,6 +158,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
 #pragma unroll
                 for (int ks = 0; ks < 4; ks++)
                     mma_ts(tmem + COL_O, tmem + COL_S + stage * 64 + ks * 8, dV + kstep_mnmajor(ks), I_O, n > 0 || ks > 0);
+                mma_commit(&m.bar_pv);                                    // one phase per tile, in order
                 if (n + 2 < n_tiles) mma_commit(&m.bar_vfree[stage]);     // the V tile will be refilled
                 if (n + 1 == n_tiles) mma_commit(&m.bar_o);
             }
@@ -191,6 +194,12 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 // raise the reference only by big steps; the whole warp decides together whether O must be rescaled
                 const bool raise = mx > m_ref + RAISE || m_ref == -INFINITY;
                 if (__any_sync(0xffffffffu, raise && n > 0)) {
+                    // O is about to be read and rewritten: the P V MMAs of the previous tile must be done.  S of this tile
+                    // was issued before them (it has its own buffer), so its completion does not say so; bar_pv does.  Its
+                    // phase index is the running tile count; this warp is never more than one phase behind (P V of this tile
+                    // cannot be issued before this warp arrives on bar_p), so the parity alone identifies the phase.
+                    mbar_wait_warp(&m.bar_pv, (tiles_done - 1) & 1, status);
+                    tc_fence_after();
                     const float m_new = raise ? mx : m_ref;
                     const float alpha = m_new == -INFINITY ? 1.f : ex2(m_ref - m_new);   // m_ref = -inf: O and l are still 0
                     l_sum *= alpha;
@@ -228,6 +237,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&m.bar_p);
                 n++;
+                tiles_done++;
             }
             // ---- epilogue: O / l -> bf16, lse ----------------------------------------------------------------------
             mbar_wait_warp(&m.bar_o, ph_o, status);

@@ -163,3 +163,27 @@ def test_many_short_pieces():
     _, dk_ref, dv_ref = ao.attn_bwd(fo, cpu["q"], cpu["k"], cpu["v"], cpu["dO"], SCALE)
     assert _rel(dk[rows].double().cpu().numpy(), dk_ref) <= 1e-2
     assert _rel(dv[rows].double().cpu().numpy(), dv_ref) <= 1e-2
+
+
+@pytest.mark.parametrize("seed", [2052, 3017])
+def test_forward_rescale_waits_for_the_previous_tile(seed):
+    """Two random forests on which an early version rescaled O (a row whose maximum jumps by more than 2^8 late in
+    the walk) while the previous tile's P.V MMAs were still accumulating into it: one wrong row in thousands."""
+    rnd = random.Random(seed)
+    max_len = rnd.choice([5, 70, 200, 700])
+    fo = make_forest([random_tree(rnd, rnd.randint(1, 10), max_len) for _ in range(rnd.randint(1, 4))])
+    rnd.choice([1, 2, 3])
+    Hkv = rnd.choice([1, 2]); Hq = Hkv * rnd.choice([1, 2])
+    inp = make_attn_inputs(fo.n_tokens, Hq, Hkv, D, "bf16", seed % 1000)
+    use_plan = rnd.random() < 0.7
+    rot = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64).row_of_token if use_plan else None
+    index = H.harts_attn_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, rot).upload()
+    rows = torch.arange(fo.n_tokens) if rot is None else torch.as_tensor(np.asarray(rot).astype(np.int64))
+    phys = {}
+    for n, x in inp.items():
+        t = torch.empty_like(x); t[rows] = x; phys[n] = t.cuda()
+    o, lse = _forward(phys, index)
+    o_ref, lse_ref = ao.attn_fwd(fo, inp["q"].double().numpy(), inp["k"].double().numpy(), inp["v"].double().numpy(), SCALE)
+    got = o[rows.cuda()].double().cpu().numpy()
+    assert np.abs(got - o_ref).max() <= 0.05                   # no single row off (the relative norm alone would hide one)
+    assert _rel(got, o_ref) <= 5e-3
