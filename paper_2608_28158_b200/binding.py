@@ -91,11 +91,32 @@ def _stream(stream):
     return C.c_void_p(stream.cuda_stream)
 
 
-class Plan:
-    """Host plan (owned by the library) plus, after ``upload``, its device index blob.  The index arrays are
-    read-only views of the library's memory; copy them if they must outlive the plan."""
+class _PlanHandle:
+    """Owns the library's plan object; freed when the last user (the Plan or one of its array views) is gone."""
 
     def __init__(self, handle):
+        self.h = handle
+
+    def __del__(self):
+        h, self.h = getattr(self, "h", None), None
+        if h:
+            lib.harts_la_plan_free(h)
+
+
+class _PlanArray(np.ndarray):
+    """Read-only view of a plan table in the library's memory; keeps the plan alive."""
+    _owner = None
+
+    def __array_finalize__(self, obj):
+        self._owner = getattr(obj, "_owner", None)
+
+
+class Plan:
+    """Host plan (owned by the library) plus, after ``upload``, its device index blob.  The index arrays are
+    read-only views of the library's memory (no copies); each keeps the plan alive."""
+
+    def __init__(self, handle):
+        self._handle = _PlanHandle(handle)
         self._h = handle
         v = _View()
         _check(lib.harts_la_plan_view(handle, C.byref(v)), "harts_la_plan_view")
@@ -112,18 +133,16 @@ class Plan:
             size = sizes[n]
             if n == "slot_cons_seq":
                 size = int(self.slot_cons_ptr[-1])
-            # views into the library-owned plan (no copy): valid as long as this object lives
-            arr = np.ctypeslib.as_array(getattr(v, n), shape=(size,)) if size else np.zeros(0, np.int32)
-            arr.flags.writeable = False
+            if size:
+                arr = np.ctypeslib.as_array(getattr(v, n), shape=(size,)).view(_PlanArray)
+                arr._owner = self._handle
+                arr.flags.writeable = False
+            else:
+                arr = np.zeros(0, np.int32)
             setattr(self, n, arr)
         self.C, self.R = self.n_rows, self.n_replay
         self.blob = None
         self.tables = None
-
-    def __del__(self):
-        h, self._h = getattr(self, "_h", None), None
-        if h:
-            lib.harts_la_plan_free(h)
 
     def upload(self, device="cuda", stream=None):
         n = C.c_size_t(0)
