@@ -539,7 +539,9 @@ def run_ours(args):
                                     "frac_strict_nominal": max((fwd_bytes + bwd_bytes) / 8e12,
                                                                (flops_fwd + flops_bwd) / 2.25e15) * 1e3 / ms_step}},
         "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms, "fold": fold_ms},
-        "gpu_launches": (2 * K + (1 if plan.n_rg_rows else 0)) * args.steps,
+        # per step: K forward calls, K backward calls each preceded by the hand-off reduction when the plan has
+        # exported boundaries, and the replay-gradient fold
+        "gpu_launches": (2 * K + (K if plan.n_slots else 0) + (1 if plan.n_rg_rows else 0)) * args.steps,
         "clocks": clock,
     }
     if e2e:

@@ -72,6 +72,7 @@ int32_t fma_bwd(const BwdArgs& a);
 int32_t tc_supported(int32_t dtype, int32_t dk, int32_t dv);
 int32_t tc_fwd(const FwdArgs& a);
 int32_t tc_bwd(const BwdArgs& a);
+int32_t handoff_reduce(const BwdArgs& a);
 int32_t replay_reduce(const harts_la_tables_t& tb, void* dk_, void* dv_, float* dg, const void* scratch, int32_t H,
                       int32_t dk, int32_t dv, int32_t dtype, cudaStream_t stream);
 

@@ -238,8 +238,9 @@ __global__ void __launch_bounds__(NT) fma_bwd_kernel(harts_la_tables_t tb, int s
     for (int c = s.n_chunks - 1; c >= 0; c--) {
         // gradient arriving at boundary c+1 from the sequences that started there
         if (next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1) {
-            for (int u = tb.slot_cons_ptr[next_req]; u < tb.slot_cons_ptr[next_req + 1]; u++) {
-                const float* src = ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems;
+            // all consumers' gradients were summed into the first consumer's buffer by handoff_reduce
+            if (tb.slot_cons_ptr[next_req] < tb.slot_cons_ptr[next_req + 1]) {
+                const float* src = ds0 + ((size_t)tb.slot_cons_seq[tb.slot_cons_ptr[next_req]] * H + h) * state_elems;
                 for (int e = tid; e < DK * DV; e += NT) sdS[tix<DV>(e / DV, e % DV)] += src[e];
             }
             next_req--;
@@ -486,8 +487,52 @@ int32_t fma_fwd(const FwdArgs& a) {
     return HARTS_EUNSUPPORTED;
 }
 
+// Sums the initial-state gradients of all sequences that started from one exported boundary (Section 3.4: several
+// consumers of one boundary tensor are summed) into the first consumer's buffer, for the boundaries that the
+// sequences [seq_lo, seq_hi) exported: a bandwidth-bound pass, in consumer order (deterministic), so that the
+// backward kernels add one tensor per boundary instead of walking the consumer list under their own latency.
+__global__ void __launch_bounds__(256) handoff_reduce_kernel(const harts_la_tables_t tb, int seq_lo, int seq_hi, int H,
+                                                             int elems, float* __restrict__ ds0) {
+    const int slot = blockIdx.x;
+    if (slot < tb.seq_req_ptr[seq_lo] || slot >= tb.seq_req_ptr[seq_hi]) return;
+    const int c0 = tb.slot_cons_ptr[slot], c1 = tb.slot_cons_ptr[slot + 1];
+    if (c1 - c0 < 2) return;
+    const int h = blockIdx.y;
+    float4* dst = reinterpret_cast<float4*>(ds0 + ((size_t)tb.slot_cons_seq[c0] * H + h) * elems);
+    for (int e = blockIdx.z * 256 + threadIdx.x; e < elems / 4; e += gridDim.z * 256) {
+        float4 acc = dst[e];
+        int u = c0 + 1;
+        for (; u + 3 < c1; u += 4) {              // four independent loads in flight
+            float4 v[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++)
+                v[i] = reinterpret_cast<const float4*>(ds0 + ((size_t)tb.slot_cons_seq[u + i] * H + h) * elems)[e];
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w;
+            }
+        }
+        for (; u < c1; u++) {
+            const float4 v = reinterpret_cast<const float4*>(ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * elems)[e];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        dst[e] = acc;
+    }
+}
+
+int32_t handoff_reduce(const BwdArgs& a) {
+    if (a.tb.n_slots == 0 || a.seq_hi == a.seq_lo) return HARTS_OK;
+    ScratchLayout sl = scratch_layout(a.tb, a.H, a.dk, a.dv);
+    float* ds0 = reinterpret_cast<float*>(static_cast<char*>(a.scratch) + sl.ds0);
+    const int elems = a.dk * a.dv;
+    dim3 grid(a.tb.n_slots, a.H, (elems / 4 + 1023) / 1024);
+    handoff_reduce_kernel<<<grid, 256, 0, a.stream>>>(a.tb, a.seq_lo, a.seq_hi, a.H, elems, ds0);
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
 int32_t fma_bwd(const BwdArgs& a) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
+    if (int32_t rc = handoff_reduce(a); rc != HARTS_OK) return rc;
     if (a.dtype == HARTS_FP32 && a.dk == 64 && a.dv == 64) return launch_bwd<float, 64, 64>(a);
     if (a.dtype == HARTS_BF16 && a.dk == 64 && a.dv == 64) return launch_bwd<__nv_bfloat16, 64, 64>(a);
     if (a.dtype == HARTS_BF16 && a.dk == 128 && a.dv == 128) return launch_bwd<__nv_bfloat16, 128, 128>(a);

@@ -386,8 +386,9 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma -----------------
             {
                 const bool boundary = next_boundary == c + 1;
+                // all consumers' gradients were summed into the first consumer's buffer by handoff_reduce
                 const int cons_lo = boundary ? tb.slot_cons_ptr[next_req] : 0;
-                const int cons_hi = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
+                const int cons_hi = boundary ? min(tb.slot_cons_ptr[next_req + 1], cons_lo + 1) : 0;
                 const float gamma = rd.gamma;
                 float dot = 0.f;
                 const int blk = grp;
@@ -630,6 +631,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
 
 int32_t tc_bwd(const BwdArgs& a) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
+    if (int32_t rc0 = handoff_reduce(a); rc0 != HARTS_OK) return rc0;
     CUtensorMap mq, mk, mv, mdo, mcs, mdq, mdk, mdv;
     int32_t rc;
     if ((rc = make_row_map(&mq, a.q, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
