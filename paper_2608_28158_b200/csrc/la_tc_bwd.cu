@@ -101,9 +101,10 @@ __device__ __forceinline__ float warp_transpose_reduce16(float (&z)[16], int lan
 
 // Epilogue of one chunk for this thread's feature index L and its 16 rows, in three parts that follow the three
 // commits of the MMA batch (dq, dk, dv).  qk[e] holds q[t][L] (low half) and k[t][L] (high half) as bf16 bits, read
-// from the tiles before the batch so that the tiles can be reloaded while the epilogue runs.  FULL: all 64 rows are
-// own rows, so the outputs are staged in shared memory ([row][feature], plain layout) for one TMA store per tensor;
-// otherwise every row is checked and written on its own (own rows to the outputs, replayed rows to the scratch).
+// from the tiles before the batch so that the tiles can be reloaded while the epilogue runs.  The outputs are staged
+// in shared memory ([row][feature], plain layout).  FULL: all 64 rows are own rows and leave by one TMA store per
+// tensor; otherwise the compute warps copy the valid rows out after the epilogue (own rows to the outputs, replayed
+// rows, staged in fp32, to the scratch).
 template <bool FULL>
 __device__ __forceinline__ void epilogue_dq(const RowData& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
                                             int h, const uint32_t (&qk)[16], __nv_bfloat16* dq, float (&z)[16]) {
@@ -116,14 +117,8 @@ __device__ __forceinline__ void epilogue_dq(const RowData& m, unsigned char* sme
         const int t = t0 + e;
         const float dqv = __uint_as_float(xq[e]);
         const float qv = __uint_as_float(qk[e] << 16);
-        if (FULL) {
-            z[e] = qv * dqv;
-            *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dq + t * 256 + L * 2) = __float2bfloat16_rn(dqv);
-        } else {
-            const int code = m.code[t];
-            z[e] = code == -1 ? 0.f : qv * dqv;
-            if (code >= 0) dq[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dqv);
-        }
+        z[e] = (FULL || m.code[t] != -1) ? qv * dqv : 0.f;
+        *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dq + t * 256 + L * 2) = __float2bfloat16_rn(dqv);
     }
 }
 
@@ -142,19 +137,13 @@ __device__ __forceinline__ void epilogue_dk(const RowData& m, unsigned char* sme
         const float kv = __uint_as_float(qk[e] & 0xffff0000u);
         const float inter = m.w[t] * __uint_as_float(xe[e]);
         const float dkv = __uint_as_float(xi[e]) + inter;
-        if (FULL) {
+        if (FULL || m.code[t] != -1) {
             z[e] -= kv * dkv;
             g_part += kv * inter;
-            *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dk + t * 256 + L * 2) = __float2bfloat16_rn(dkv);
-        } else {
-            const int code = m.code[t];
-            if (code != -1) {
-                z[e] -= kv * dkv;
-                g_part += kv * inter;
-            }
-            if (code >= 0) dk_[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dkv);
-            else if (code < -1) rk[((size_t)(replay_base + t) * H + h) * D + L] = dkv;     // replayed rows sit in chunk 0
         }
+        *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dk + t * 256 + L * 2) = __float2bfloat16_rn(dkv);
+        // replayed rows (chunk 0 only) keep fp32: staged over the S tile, which nothing reads after the dq MMAs
+        if (!FULL && m.code[t] < -1) *reinterpret_cast<float*>(smem + Smem::s + t * 512 + L * 4) = dkv;
     }
 }
 
@@ -170,13 +159,9 @@ __device__ __forceinline__ void epilogue_dv(const RowData& m, unsigned char* sme
     for (int e = 0; e < 16; e++) {
         const int t = t0 + e;
         const float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
-        if (FULL) {
-            *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dv + t * 256 + L * 2) = __float2bfloat16_rn(dvv);
-        } else {
-            const int code = m.code[t];
-            if (code >= 0) dv_[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(dvv);
-            else if (code < -1) rv[((size_t)(replay_base + t) * H + h) * D + L] = dvv;
-        }
+        *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dv + t * 256 + L * 2) = __float2bfloat16_rn(dvv);
+        // replayed rows: fp32 over the q/k tiles (every MMA is done by now, and chunk 0 loads no further tiles)
+        if (!FULL && m.code[t] < -1) *reinterpret_cast<float*>(smem + Smem::q + t * 512 + L * 4) = dvv;
     }
 }
 
@@ -570,6 +555,26 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         tc_fence_before();
         __syncthreads();                          // (B) staged outputs, partial sums and the next chunk's row data visible
         tc_fence_after();
+        if (is_compute && !full) {
+            // partial chunk: the staged rows leave with 16-byte stores, own rows to the outputs (bf16), replayed rows
+            // to the scratch (fp32); rows past the end go nowhere
+            for (int e = tid; e < BT * 16 * 3; e += NC) {
+                const int which = e / (BT * 16), t = (e / 16) % BT, j = e % 16, code = rd.code[t];
+                if (code < 0) continue;
+                __nv_bfloat16* out = which == 0 ? dq : (which == 1 ? dk_ : dv_);
+                const int stage = which == 0 ? Smem::stage_dq : (which == 1 ? Smem::stage_dk : Smem::stage_dv);
+                *reinterpret_cast<uint4*>(out + ((size_t)code * H + h) * D + j * 8) =
+                    *reinterpret_cast<const uint4*>(smem + stage + t * 256 + j * 16);
+            }
+            if (gathered)
+                for (int e = tid; e < BT * 32 * 2; e += NC) {
+                    const int which = e / (BT * 32), t = (e / 32) % BT, j = e % 32;
+                    if (rd.code[t] >= -1) continue;
+                    float* out = which == 0 ? rk : rv;
+                    *reinterpret_cast<float4*>(out + ((size_t)(s.replay_base + t) * H + h) * D + j * 4) =
+                        *reinterpret_cast<const float4*>(smem + (which == 0 ? Smem::s : Smem::q) + t * 512 + j * 16);
+                }
+        }
         if (!is_compute) {
             if (is_issuer && full) {
                 int row0 = s.own_begin - s.n_replay + c * BT;
