@@ -64,7 +64,7 @@ struct SmemQ {
     static constexpr int bytes = misc + 256;
 };
 struct MiscQ {
-    uint64_t bar_q, bar_k[KST], bar_v[2], bar_kfree[KST], bar_vfree[2], bar_s, bar_dpfree, bar_p, bar_o;
+    uint64_t bar_q, bar_k[KST], bar_v[2], bar_kfree[KST], bar_vfree[2], bar_s, bar_dpfree, bar_p[2], bar_o;
     uint32_t tmem;
 };
 constexpr int COL_DP = 256, COL_DQ = 384, TMEM_Q = 512;     // S of tile n at 128 (n & 1)
@@ -95,7 +95,8 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
         }
         mbar_init(&m.bar_s, 1);
         mbar_init(&m.bar_dpfree, NS / 32);
-        mbar_init(&m.bar_p, NS / 32);
+        mbar_init(&m.bar_p[0], NS / 32);
+        mbar_init(&m.bar_p[1], NS / 32);
         mbar_init(&m.bar_o, 1);
         fence_barrier_init();
     }
@@ -110,7 +111,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
     const uint64_t dQd = desc_kmajor_base(smem_u32(sQ)), dDOd = desc_kmajor_base(smem_u32(sDO));
     const float scale_log2 = scale * LOG2E;
 
-    uint32_t ph_q = 0, ph_k[KST] = {}, ph_v[2] = {0, 0}, ph_kfree[KST] = {}, ph_vfree[2] = {0, 0}, ph_s = 0, ph_p = 0,
+    uint32_t ph_q = 0, ph_k[KST] = {}, ph_v[2] = {0, 0}, ph_kfree[KST] = {}, ph_vfree[2] = {0, 0}, ph_s = 0, ph_p[2] = {0, 0},
              ph_dpfree = 0, ph_o = 0;
     const int n_work = ix.n_q_items * Hq;
     for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
@@ -191,8 +192,10 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                     tc_fence_after();
                     issue_dp(n + 1);
                 }
-                mbar_wait(&m.bar_p, ph_p, status);              // dS(n) written, S(n) read
-                ph_p ^= 1;
+                // dS(n) written, S(n) read.  One barrier per S buffer: a warp that is done with tile n may already work
+                // on tile n+1 (its S and dP are complete) and arrive for it, and that arrival must not count for tile n.
+                mbar_wait(&m.bar_p[stage], ph_p[stage], status);
+                ph_p[stage] ^= 1;
                 tc_fence_after();
                 const uint64_t dKm = desc_mnmajor_base<BKW>(smem_u32(smem + SmemQ::k0 + (n % KST) * KW_BYTES));
 #pragma unroll
@@ -248,7 +251,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&m.bar_p);
+                if (lane == 0) mbar_arrive(&m.bar_p[b]);
             }
             // ---- epilogue: dQ -> bf16 ------------------------------------------------------------------------------
             mbar_wait_warp(&m.bar_o, ph_o, status);

@@ -42,7 +42,7 @@ struct Smem {
     static constexpr int bytes = misc + 256;
 };
 struct Misc {
-    uint64_t bar_q, bar_k[2], bar_v[2], bar_kfree[2], bar_vfree[2], bar_s[2], bar_p, bar_pv, bar_o;
+    uint64_t bar_q, bar_k[2], bar_v[2], bar_kfree[2], bar_vfree[2], bar_s[2], bar_p[2], bar_pv, bar_o;
     uint32_t tmem;
 };
 
@@ -69,7 +69,8 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
         }
         mbar_init(&m.bar_s[0], 1);
         mbar_init(&m.bar_s[1], 1);
-        mbar_init(&m.bar_p, NS / 32);
+        mbar_init(&m.bar_p[0], NS / 32);
+        mbar_init(&m.bar_p[1], NS / 32);
         mbar_init(&m.bar_pv, 1);
         mbar_init(&m.bar_o, 1);
         fence_barrier_init();
@@ -88,7 +89,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
 
     uint32_t tiles_done = 0;                     // key tiles this CTA has processed (the phase index of bar_pv)
     uint32_t ph_q = 0, ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_kfree[2] = {0, 0}, ph_vfree[2] = {0, 0}, ph_s[2] = {0, 0},
-             ph_p = 0, ph_o = 0;
+             ph_p[2] = {0, 0}, ph_o = 0;
     const int n_work = ix.n_q_items * Hq;
     for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
         const int item = w / Hq, h = w % Hq, hk = h / G;
@@ -148,9 +149,11 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 // S of tile n+1 goes to the other buffer and runs under the softmax of tile n (its K stage was freed
                 // by the P V MMAs of tile n-1, which precede it in the pipe)
                 if (n + 1 < n_tiles) issue_s(n + 1);
-                // O += P V for tile n as soon as the softmax warps have written P
-                mbar_wait(&m.bar_p, ph_p, status);
-                ph_p ^= 1;
+                // O += P V for tile n as soon as the softmax warps have written P.  One barrier per S buffer: a warp that
+                // is done with tile n may already work on tile n+1 (its S is complete) and arrive for it, and that
+                // arrival must not count for tile n.
+                mbar_wait(&m.bar_p[stage], ph_p[stage], status);
+                ph_p[stage] ^= 1;
                 mbar_wait(&m.bar_v[stage], ph_v[stage], status);
                 ph_v[stage] ^= 1;
                 tc_fence_after();
@@ -235,7 +238,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&m.bar_p);
+                if (lane == 0) mbar_arrive(&m.bar_p[b]);
                 n++;
                 tiles_done++;
             }
