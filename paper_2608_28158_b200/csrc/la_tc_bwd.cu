@@ -57,6 +57,7 @@ struct RowData {             // per-chunk row quantities, double-buffered (the n
     float w[BT];             // e^{b_n - b_t}
     int code[BT];            // physical row (>= 0 own), -2 - row (replayed), -1 (past the end)
     float gamma;             // e^{b_n}
+    float pad[3];            // keeps the second buffer 16-byte aligned (vector loads of b2)
 };
 struct Misc {
     RowData rows[2];
@@ -449,18 +450,24 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                     *reinterpret_cast<uint4*>(dst + sw128_chunk(t, grp * 2 + 1)) = make_uint4(0, 0, 0, 0);
                 } else {
                 const float bt = rd.b2[t];
-                const bool live = rd.code[t] >= 0;    // replay rows and rows past the end have no dO and no q
+                // replay rows and rows past the end have no dO and no q: nothing is visible to them (limit = -1)
+                const int limit = rd.code[t] >= 0 ? t : -1;
                 uint32_t xa[16];
                 tmem_ld16(tm_lane + (is_p ? COL_A : COL_DA) + grp * 16, xa);
+                // the 16 column decays with four 16-byte loads; no load or branch under the per-element condition
+                float bj[16];
+#pragma unroll
+                for (int v = 0; v < 4; v++)
+                    *reinterpret_cast<float4*>(bj + 4 * v) = *reinterpret_cast<const float4*>(rd.b2 + grp * 16 + 4 * v);
                 tmem_ld_wait();
 #pragma unroll
                 for (int v4 = 0; v4 < 2; v4++) {
                     float ya[8];
 #pragma unroll
                     for (int e = 0; e < 8; e++) {
-                        int j = grp * 16 + v4 * 8 + e;
-                        float dec = (live && j <= t) ? ex2(bt - rd.b2[j]) : 0.f;
-                        ya[e] = dec != 0.f ? __uint_as_float(xa[v4 * 8 + e]) * dec : 0.f;
+                        const int j = grp * 16 + v4 * 8 + e;
+                        const float y = __uint_as_float(xa[v4 * 8 + e]) * ex2(bt - bj[v4 * 8 + e]);
+                        ya[e] = j <= limit ? y : 0.f;      // a select: above the diagonal the product may be inf or NaN
                     }
                     *reinterpret_cast<uint4*>(dst + sw128_chunk(t, grp * 2 + v4)) =
                         make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]), pack_bf16(ya[4], ya[5]),

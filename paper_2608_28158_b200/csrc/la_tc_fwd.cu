@@ -274,11 +274,16 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 tmem_ld_wait();
 #pragma unroll
                 for (int v4 = 0; v4 < 4; v4++) {
+                    // the eight column decays with two 16-byte loads; no load or branch under the per-element condition
+                    float bj[8];
+                    *reinterpret_cast<float4*>(bj) = *reinterpret_cast<const float4*>(m.b2 + half * 32 + v4 * 8);
+                    *reinterpret_cast<float4*>(bj + 4) = *reinterpret_cast<const float4*>(m.b2 + half * 32 + v4 * 8 + 4);
                     float y[8];
 #pragma unroll
                     for (int e = 0; e < 8; e++) {
-                        int j = half * 32 + v4 * 8 + e;
-                        y[e] = j <= t ? __uint_as_float(x[v4 * 8 + e]) * ex2(bt - m.b2[j]) : 0.f;
+                        const int j = half * 32 + v4 * 8 + e;
+                        const float p = __uint_as_float(x[v4 * 8 + e]) * ex2(bt - bj[e]);
+                        y[e] = j <= t ? p : 0.f;           // a select: above the diagonal the product may be inf or NaN
                     }
                     uint4 pk = make_uint4(pack_bf16(y[0], y[1]), pack_bf16(y[2], y[3]), pack_bf16(y[4], y[5]),
                                           pack_bf16(y[6], y[7]));
