@@ -216,3 +216,30 @@ def test_repeated_runs_are_bit_identical_with_a_wide_query_group():
     o_ref, lse_ref = ao.attn_fwd(fo, cpu["q"], cpu["k"], cpu["v"], SCALE, tokens=tok)
     got = o0[rows][:, [0, Hq - 1]].double().cpu().numpy()[tok]
     assert np.abs(got - o_ref[tok]).max() <= 0.06
+
+
+def test_degenerate_forests_have_closed_forms():
+    """One token: o = v, lse = scale q.k, dq = dk = 0, dv = dO.  A chain of one-token nodes (every token its own
+    piece, each the child of the previous one) is plain causal attention over the chain."""
+    fo = make_forest([([-1], [0], [1])])
+    inp, phys, index, rows = _setup(fo, 2, 1, 11)
+    o, lse = _forward(phys, index)
+    dq, dk, dv = _backward(phys, index, o, lse)
+    assert torch.equal(o, phys["v"].expand(-1, 2, -1))
+    want = (phys["q"].float() * phys["k"].float()).sum(-1) * SCALE
+    assert float((lse - want).abs().max()) <= 1e-5
+    assert float(dq.float().abs().max()) == 0.0 and float(dk.float().abs().max()) <= 1e-6
+    assert _rel(dv.double().cpu().numpy(), phys["dO"].double().sum(dim=1, keepdim=True).cpu().numpy()) <= 4e-3
+
+    n = 70                                                  # more than one 64-row tile of one-token pieces
+    fo = make_forest([([-1] + list(range(n - 1)), [0] + [1] * (n - 1), [1] * n)])
+    inp, phys, index, rows = _setup(fo, 2, 2, 12)
+    o, lse = _forward(phys, index)
+    dq, dk, dv = _backward(phys, index, o, lse)
+    q, k, v, dO = (inp[x].float().cuda().transpose(0, 1).requires_grad_(x != "dO") for x in ("q", "k", "v", "dO"))
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, scale=SCALE)
+    ref.backward(dO)
+    pick = lambda x: x[rows].float().transpose(0, 1)     # noqa: E731
+    assert _rel(pick(o).cpu().numpy(), ref.detach().cpu().numpy()) <= 5e-3
+    for got, want_ in ((dq, q.grad), (dk, k.grad), (dv, v.grad)):
+        assert _rel(pick(got).cpu().numpy(), want_.cpu().numpy()) <= 1e-2
