@@ -36,7 +36,8 @@ using namespace tc;
 constexpr int BT = 64, D = 128;
 constexpr int NC = 512;                       // 16 compute warps: warp w works on tensor-memory lanes 32(w&3)..+31 and
                                               // on column group w>>2 (a quarter of every accumulator)
-constexpr int NT = NC + 32;                   // plus one warp whose first lane issues every TMA and MMA
+constexpr int NT = NC + 64;                   // plus one warp whose first lane issues every TMA and MMA, and one
+                                              // that prepares row data and finishes dg (off the issuing thread's path)
 constexpr int TILE = BT * D * 2;              // 16 KB
 constexpr int PANEL = BT * 128;               // 8 KB
 constexpr int S_PANEL = D * 128;              // 16 KB
@@ -191,7 +192,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool is_compute = warp < NC / 32;
-    const bool is_issuer = tid == NC;              // first lane of the extra warp
+    const bool is_issuer = tid == NC;              // first lane of the issuing warp
+    const bool is_aux = warp == NC / 32 + 1;       // row data of the next chunk, dg of the finished one
     const int grp = warp >> 2;                    // column group (compute warps)
     const int L = (warp & 3) * 32 + lane;         // tensor-memory lane = feature index (or row t) of this thread
     const size_t state_elems = (size_t)D * D;
@@ -262,7 +264,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tiles);
             }
     };
-    // Row codes and g of chunk c for rows `lane` and `lane + 32` (the extra warp prepares a chunk's row data on its own).
+    // Row codes and g of chunk c for rows `lane` and `lane + 32` (the auxiliary warp prepares a chunk's row data on its own).
     auto load_rows = [&](int c, int (&code)[2], float (&gv)[2]) {
 #pragma unroll
         for (int r = 0; r < 2; r++) {
@@ -307,7 +309,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     if (is_issuer) issue_tiles(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
     int nx_code[2];
     float nx_g[2];
-    if (!is_compute) {
+    if (is_aux) {
         load_rows(s.n_chunks - 1, nx_code, nx_g);
         store_rows(m.rows[0], nx_code, nx_g);
     }
@@ -318,8 +320,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     tc_fence_after();
 
     // Two block-wide barriers per chunk: (A) before the MMA batch, (B) at the end of the epilogue.  After (B) the
-    // compute warps go straight on to the next chunk, while the extra warp sends the staged outputs off and
-    // finishes dg for the chunk just done.
+    // compute warps go straight on to the next chunk, while the issuing thread sends the staged outputs off and the
+    // auxiliary warp finishes dg for the chunk just done.
     for (int c = s.n_chunks - 1; c >= 0; c--, cur ^= 1) {
         const bool gathered = c == 0 && gather_first;
         // all 64 rows are own rows: outputs leave through staged TMA stores
@@ -362,10 +364,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             mma_commit(&m.bar_a);
             tma_store_wait_read();                // the previous chunk's output stores have left the staging tiles
         }
-        if (!is_compute) {                        // next chunk's rows and g: requested ahead of the next tile loads
-            __syncwarp();
-            load_rows(c - 1, nx_code, nx_g);
-        }
+        if (is_aux) load_rows(c - 1, nx_code, nx_g);      // next chunk's rows and g, in flight during this chunk
         float g_part = 0.f;                       // this thread's share of <S_{c+1}, dS_{c+1}>
         uint32_t qk[16];                          // q[t][L] | k[t][L] << 16 of this thread's 16 rows (bf16 bits)
         if (is_compute) {
@@ -517,10 +516,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             mbar_wait(&m.bar_qk_read, ph_o, status);      // every compute warp has taken its q and k values
             if (c > 0) issue_tiles(c - 1, next_tiles);
         }
-        if (!is_compute) {                        // the extra warp prepares the next chunk's row data during the epilogue
-            __syncwarp();
-            if (c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);
-        }
+        if (is_aux && c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);   // visible to the others at barrier (B)
         if (is_compute) {
             // q[t][L], k[t][L] of this thread's 16 rows, for the dg terms (read while the first MMAs run; after this
             // the epilogue does not touch the tiles, which are reloaded as soon as the MMAs are done)
@@ -582,14 +578,14 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                         *reinterpret_cast<const float4*>(smem + (which == 0 ? Smem::s : Smem::q) + t * 512 + j * 16);
                 }
         }
-        if (!is_compute) {
-            if (is_issuer && full) {
-                int row0 = s.own_begin - s.n_replay + c * BT;
-                tma_store_3d(&map_dq, smem + Smem::stage_dq, 0, h, row0);
-                tma_store_3d(&map_dk, smem + Smem::stage_dk, 0, h, row0);
-                tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
-                tma_store_commit();
-            }
+        if (is_issuer && full) {
+            int row0 = s.own_begin - s.n_replay + c * BT;
+            tma_store_3d(&map_dq, smem + Smem::stage_dq, 0, h, row0);
+            tma_store_3d(&map_dk, smem + Smem::stage_dk, 0, h, row0);
+            tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
+            tma_store_commit();
+        }
+        if (is_aux) {
             // dg_t = sum_{tau >= t} r_tau + <S_{c+1}, dS_{c+1}>, rows `lane` and `lane + 32` per thread of this warp
             auto row_sum = [&](int t) {
                 const int g4 = (t >> 4) * 4, e = t & 15;
