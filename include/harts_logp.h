@@ -54,6 +54,19 @@ int32_t harts_logp_positions(int32_t n_trees, const int32_t* tree_node_ptr, cons
                              int64_t* n_pos, int64_t* n_traj);
 
 /*
+ * Multiplicity of every compact token (Section 3.5, Eq. 20: q_c = |{s : m(s) = c}|, terminal positions included):
+ * the number of root-to-leaf trajectories that contain the token.  A loss or auxiliary statistic that the
+ * trajectory-wise run would average over semantic positions is reproduced on compact rows by weighting row c with q_c.
+ *   forest arrays, row_of_token: host, as for harts_logp_positions()
+ *   n_rows: rows of the compact tensors (>= number of compact tokens);  mult [n_rows] host out (rows that hold no
+ *   token get 0)
+ * Errors: HARTS_EINVAL for a malformed forest, n_rows too small or a row_of_token entry outside [0, n_rows).
+ */
+int32_t harts_logp_multiplicity(int32_t n_trees, const int32_t* tree_node_ptr, const int32_t* node_parent,
+                                const int32_t* node_fork_off, const int32_t* node_len, const int32_t* row_of_token,
+                                int64_t n_rows, int32_t* mult);
+
+/*
  * Positions grouped by the row they reuse (the index set of the sum in Eq. 19), stable in position order.
  *   m [n_pos] host;  row_pos_ptr [n_rows+1] host out;  row_pos [n_pos] host out (position ids)
  * Errors: HARTS_EINVAL if some m[s] is outside [0, n_rows).

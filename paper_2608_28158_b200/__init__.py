@@ -11,7 +11,7 @@ from .binding import (  # noqa: F401
     harts_la_workspace_bytes, lib, run_fwd_bwd, run_fwd_bwd_host, HostPipeline, expand_trajectories,
 )
 from .logp import (  # noqa: F401
-    harts_logp_positions, harts_logp_csr, harts_logp_fwd, harts_logp_bwd, harts_logp_fwd_shard, harts_logp_combine,
+    harts_logp_positions, harts_logp_csr, harts_logp_multiplicity, harts_logp_fwd, harts_logp_bwd, harts_logp_fwd_shard, harts_logp_combine,
 )
 from .conv import harts_conv_index, harts_conv_fwd, harts_conv_scratch_bytes, harts_conv_bwd  # noqa: F401
 from .attn import AttnIndex, harts_attn_index, harts_attn_fwd, harts_attn_bwd  # noqa: F401

@@ -2,6 +2,7 @@
 // non-terminal semantic positions with their compact row m(s) and target y_s, and the grouping of
 // positions by row that the backward sums over.
 #include <cstdint>
+#include <utility>
 #include <vector>
 
 #include "../../include/harts_logp.h"
@@ -107,5 +108,54 @@ extern "C" int32_t harts_logp_csr(int32_t n_rows, int64_t n_pos, const int32_t* 
     for (int32_t c = 0; c < n_rows; ++c) row_pos_ptr[c + 1] += row_pos_ptr[c];
     std::vector<int32_t> fill(row_pos_ptr, row_pos_ptr + n_rows);
     for (int64_t s = 0; s < n_pos; ++s) row_pos[fill[m[s]]++] = static_cast<int32_t>(s);
+    return HARTS_OK;
+}
+
+extern "C" int32_t harts_logp_multiplicity(int32_t n_trees, const int32_t* tree_node_ptr, const int32_t* node_parent,
+                                           const int32_t* node_fork_off, const int32_t* node_len,
+                                           const int32_t* row_of_token, int64_t n_rows, int32_t* mult) {
+    if (!node_parent || !node_fork_off || !node_len || !mult) return HARTS_EINVAL;
+    int64_t C = 0;
+    if (!forest_ok(n_trees, tree_node_ptr, node_parent, node_fork_off, node_len, &C)) return HARTS_EINVAL;
+    if (n_rows < C) return HARTS_EINVAL;
+    if (row_of_token)
+        for (int64_t c = 0; c < C; ++c)
+            if (row_of_token[c] < 0 || row_of_token[c] >= n_rows) return HARTS_EINVAL;
+    const int32_t n_nodes = n_trees ? tree_node_ptr[n_trees] : 0;
+    for (int64_t r = 0; r < n_rows; ++r) mult[r] = 0;
+    std::vector<int64_t> base(n_nodes + 1, 0);
+    for (int32_t i = 0; i < n_nodes; ++i) base[i + 1] = base[i] + node_len[i];
+    // through[i]: trajectories that contain node i's first token.  Children come after their parent, so one reverse
+    // sweep sees every child before its parent.  add[o] of a node: trajectories that leave it right after its token
+    // o - 1 (children forking at offset o; at o = len also the node's own end if no child continues it).
+    std::vector<int64_t> through(n_nodes, 0);
+    std::vector<std::vector<std::pair<int32_t, int64_t>>> forks(n_nodes);   // (fork offset, trajectories) per parent
+    for (int32_t t = n_trees - 1; t >= 0; --t) {
+        const int32_t lo = tree_node_ptr[t], hi = tree_node_ptr[t + 1];
+        for (int32_t i = hi - 1; i >= lo; --i) {
+            auto& f = forks[i];
+            bool continued = false;
+            int64_t total = 0;
+            for (auto& e : f) {
+                continued = continued || e.first == node_len[i];
+                total += e.second;
+            }
+            if (!continued) total += 1;                   // the node's end is a trajectory end
+            through[i] = total;
+            if (total >= INT32_MAX) return HARTS_EINVAL;
+            // tokens o = len-1 .. 0: a token at offset o is on every trajectory that leaves at an offset > o
+            std::vector<int64_t> leave(node_len[i] + 1, 0);
+            for (auto& e : f) leave[e.first] += e.second;
+            if (!continued) leave[node_len[i]] += 1;
+            int64_t run = 0;
+            for (int32_t o = node_len[i] - 1; o >= 0; --o) {
+                run += leave[o + 1];
+                const int64_t canon = base[i] + o;
+                mult[row_of_token ? row_of_token[canon] : canon] = static_cast<int32_t>(run);
+            }
+            if (i > lo) forks[lo + node_parent[i]].emplace_back(node_fork_off[i], total);
+            std::vector<std::pair<int32_t, int64_t>>().swap(f);
+        }
+    }
     return HARTS_OK;
 }

@@ -14,12 +14,13 @@ _vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
 lib.harts_logp_positions.argtypes = [_i32, _I32P, _I32P, _I32P, _I32P, _I32P, _I32P, _i64, _I32P, _I32P, _I64P, _I64P,
                                      _I64P]
 lib.harts_logp_csr.argtypes = [_i32, _i64, _I32P, _I32P, _I32P]
+lib.harts_logp_multiplicity.argtypes = [_i32, _I32P, _I32P, _I32P, _I32P, _I32P, _i64, _I32P]
 lib.harts_logp_fwd.argtypes = [_vp, _i32, _i32, _i32, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.harts_logp_bwd.argtypes = [_vp, _i32, _i32, _i32, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _vp,
                                _vp]
 lib.harts_logp_fwd_shard.argtypes = [_vp, _i32, _i32, _i32, _i64, _i32, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.harts_logp_combine.argtypes = [_i32, _i32, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
-for _n in ("harts_logp_positions", "harts_logp_csr", "harts_logp_fwd", "harts_logp_bwd", "harts_logp_fwd_shard",
+for _n in ("harts_logp_positions", "harts_logp_csr", "harts_logp_multiplicity", "harts_logp_fwd", "harts_logp_bwd", "harts_logp_fwd_shard",
            "harts_logp_combine"):
     getattr(lib, _n).restype = _i32
 
@@ -47,6 +48,17 @@ def harts_logp_positions(tree_node_ptr, node_parent, node_fork_off, node_len, to
                                     n_pos.value, _ip(m), _ip(y), tp.ctypes.data_as(_I64P), C.byref(n_pos),
                                     C.byref(n_traj)), "harts_logp_positions")
     return m[:n_pos.value], y[:n_pos.value], tp
+
+
+def harts_logp_multiplicity(tree_node_ptr, node_parent, node_fork_off, node_len, row_of_token=None, n_rows=None):
+    """int32 [n_rows] on the host: the number of trajectories that contain each compact token (Eq. 20)."""
+    ptr, par, off, ln = map(_i32arr, (tree_node_ptr, node_parent, node_fork_off, node_len))
+    rot = None if row_of_token is None else _i32arr(row_of_token)
+    n_rows = int(ln.sum()) if n_rows is None else int(n_rows)
+    mult = np.empty(max(n_rows, 1), np.int32)
+    _check(lib.harts_logp_multiplicity(len(ptr) - 1, _ip(ptr), _ip(par), _ip(off), _ip(ln), _ip(rot), n_rows, _ip(mult)),
+           "harts_logp_multiplicity")
+    return mult[:n_rows]
 
 
 def harts_logp_csr(n_rows, m):

@@ -45,6 +45,28 @@ def test_csr_groups_positions_by_row_in_order():
         assert pos[ptr[c]:ptr[c + 1]].tolist() == np.nonzero(m == c)[0].tolist()
 
 
+def test_multiplicity_counts_the_trajectories_through_every_token():
+    """Eq. 20 against the oracle (expansion of every trajectory) and two closed forms: a root token lies on every
+    trajectory of its tree, and the multiplicities sum to the trajectory-wise token count."""
+    rnd = random.Random(12)
+    forests = [config_forest(n) for n in ("cfg0", "cfg0b", "cfg1")]
+    forests += [make_forest([random_tree(rnd, rnd.randint(1, 12), 30) for _ in range(rnd.randint(1, 3))]) for _ in range(200)]
+    for fo in forests:
+        arrs = (fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len)
+        want = lo.multiplicity(fo.n_tokens, fo)
+        got = H.harts_logp_multiplicity(*arrs)
+        assert np.array_equal(got, want)
+        m0, _, tp0 = lo.positions(fo, np.zeros(fo.n_tokens, np.int32))
+        assert int(got.sum()) == len(m0) + len(tp0) - 1      # non-terminal positions + one terminal per trajectory
+        plan = H.harts_la_plan(*arrs, 8)
+        phys = H.harts_logp_multiplicity(*arrs, row_of_token=plan.row_of_token, n_rows=fo.n_tokens + 3)
+        assert np.array_equal(phys[plan.row_of_token], want) and int(phys.sum()) == int(want.sum())
+    # five-node tree of cfg0: the root's 256 tokens are on all three trajectories
+    fo = config_forest("cfg0")
+    got = H.harts_logp_multiplicity(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len)
+    assert set(got[:100].tolist()) == {3}
+
+
 def test_errors():
     with pytest.raises(H.HartsError):
         H.harts_logp_csr(5, np.array([0, 5], np.int32))
@@ -52,3 +74,6 @@ def test_errors():
         H.harts_logp_positions([0, 2], [-1, 0], [0, 9], [4, 4], np.zeros(8, np.int32))   # fork beyond the parent
     ptr, pos = H.harts_logp_csr(3, np.zeros(0, np.int32))
     assert ptr.tolist() == [0, 0, 0, 0] and len(pos) == 0
+    fo = config_forest("cfg0")
+    with pytest.raises(H.HartsError):                       # fewer rows than compact tokens
+        H.harts_logp_multiplicity(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, n_rows=10)
