@@ -102,7 +102,7 @@ __device__ __forceinline__ float warp_transpose_reduce16(float (&z)[16], int lan
 }
 
 // Epilogue of one chunk for this thread's feature index L and its 16 rows, in three parts that follow the three
-// commits of the MMA batch (dq, dk, dv).  qk[e] holds q[t][L] (low half) and k[t][L] (high half) as bf16 bits, read
+// commits of the MMA batch (dk, dv, dq: the longest part first, so that little is left after the last MMA).  qk[e] holds q[t][L] (low half) and k[t][L] (high half) as bf16 bits, read
 // from the tiles before the batch so that the tiles can be reloaded while the epilogue runs.  The outputs are staged
 // in shared memory ([row][feature], plain layout).  FULL: all 64 rows are own rows and leave by one TMA store per
 // tensor; otherwise the compute warps copy the valid rows out after the epilogue (own rows to the outputs, replayed
@@ -119,8 +119,10 @@ __device__ __forceinline__ void epilogue_dq(const RowData& m, unsigned char* sme
         const int t = t0 + e;
         const float dqv = __uint_as_float(xq[e]);
         const float qv = __uint_as_float(qk[e] << 16);
-        z[e] = (FULL || m.code[t] != -1) ? qv * dqv : 0.f;
-        *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dq + t * 256 + L * 2) = __float2bfloat16_rn(dqv);
+        z[e] += (FULL || m.code[t] != -1) ? qv * dqv : 0.f;
+        // replayed rows have no dq; their row of this staging tile holds one half of their fp32 dk (epilogue_dk)
+        if (FULL || m.code[t] >= -1)
+            *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dq + t * 256 + L * 2) = __float2bfloat16_rn(dqv);
     }
 }
 
@@ -139,13 +141,15 @@ __device__ __forceinline__ void epilogue_dk(const RowData& m, unsigned char* sme
         const float kv = __uint_as_float(qk[e] & 0xffff0000u);
         const float inter = m.w[t] * __uint_as_float(xe[e]);
         const float dkv = __uint_as_float(xi[e]) + inter;
-        if (FULL || m.code[t] != -1) {
-            z[e] -= kv * dkv;
-            g_part += kv * inter;
-        }
-        *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dk + t * 256 + L * 2) = __float2bfloat16_rn(dkv);
-        // replayed rows (chunk 0 only) keep fp32: staged over the S tile, which nothing reads after the dq MMAs
-        if (!FULL && m.code[t] < -1) *reinterpret_cast<float*>(smem + Smem::s + t * 512 + L * 4) = dkv;
+        const bool row_ok = FULL || m.code[t] != -1;
+        z[e] = row_ok ? -kv * dkv : 0.f;
+        g_part += row_ok ? kv * inter : 0.f;
+        // replayed rows (chunk 0 only) keep fp32: features 0..63 in the row's 256 bytes of the dk staging tile,
+        // 64..127 in its row of the dq staging tile (replayed rows have no dq); every operand tile is still being read
+        if (!FULL && m.code[t] < -1)
+            *reinterpret_cast<float*>(smem + (L < 64 ? Smem::stage_dk : Smem::stage_dq) + t * 256 + (L & 63) * 4) = dkv;
+        else
+            *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dk + t * 256 + L * 2) = __float2bfloat16_rn(dkv);
     }
 }
 
@@ -162,8 +166,8 @@ __device__ __forceinline__ void epilogue_dv(const RowData& m, unsigned char* sme
         const int t = t0 + e;
         const float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
         *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dv + t * 256 + L * 2) = __float2bfloat16_rn(dvv);
-        // replayed rows: fp32 over the q/k tiles (every MMA is done by now, and chunk 0 loads no further tiles)
-        if (!FULL && m.code[t] < -1) *reinterpret_cast<float*>(smem + Smem::q + t * 512 + L * 4) = dvv;
+        // replayed rows: fp32 over the bf16 copy of dS, which no MMA reads once the dk and dv groups are done
+        if (!FULL && m.code[t] < -1) *reinterpret_cast<float*>(smem + Smem::ds + t * 512 + L * 4) = dvv;
     }
 }
 
@@ -483,14 +487,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         tc_fence_after();
         const bool next_tiles = !(c - 1 == 0 && gather_first);
         if (is_issuer) {
-            // dq^T = K^T dP^T + S_c dO~^T
-#pragma unroll
-            for (int ks = 0; ks < 4; ks++)
-                mma_ss(tmem + COL_DQ, dKm + kstep_mnmajor(ks), dDPk + kstep_kmajor<BT>(ks), I_MK64, ks > 0);
-#pragma unroll
-            for (int ks = 0; ks < 8; ks++)
-                mma_ss(tmem + COL_DQ, dSk + kstep_kmajor<D>(ks), dDOsk + kstep_kmajor<BT>(ks), I_KK64, true);
-            mma_commit(&m.bar_o);
+            // Order of the three groups: the one with the longest epilogue first, the shortest last, so that little is
+            // left to do once the last MMA is done.
             // dk^T: Q^T dP   |   dS V^T (into the columns A occupied)
 #pragma unroll
             for (int ks = 0; ks < 4; ks++)
@@ -498,7 +496,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
 #pragma unroll
             for (int ks = 0; ks < 8; ks++)
                 mma_ss(tmem + COL_A, dDSk + kstep_kmajor<D>(ks), dVk + kstep_kmajor<BT>(ks), I_KK64, ks > 0);
-            mma_commit(&m.bar_o2);
+            mma_commit(&m.bar_o);
             // dv^T: dO^T P   |   dS^T K^T (into the columns dA occupied)
 #pragma unroll
             for (int ks = 0; ks < 4; ks++)
@@ -506,6 +504,14 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
 #pragma unroll
             for (int ks = 0; ks < 8; ks++)
                 mma_ss(tmem + COL_DA, dDSm + kstep_mnmajor(ks), dKk + kstep_kmajor<BT>(ks), I_MK64, ks > 0);
+            mma_commit(&m.bar_o2);
+            // dq^T = K^T dP^T + S_c dO~^T
+#pragma unroll
+            for (int ks = 0; ks < 4; ks++)
+                mma_ss(tmem + COL_DQ, dKm + kstep_mnmajor(ks), dDPk + kstep_kmajor<BT>(ks), I_MK64, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < 8; ks++)
+                mma_ss(tmem + COL_DQ, dSk + kstep_kmajor<D>(ks), dDOsk + kstep_kmajor<BT>(ks), I_KK64, true);
             // dS += Q^T dO~   (dS was pre-scaled by e^{b_n})
 #pragma unroll
             for (int ks = 0; ks < 4; ks++)
@@ -537,21 +543,21 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             float z[16];
             mbar_wait(&m.bar_o, ph_o, status);
             tc_fence_after();
-            if (full) epilogue_dq<true>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
-            else epilogue_dq<false>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
-            mbar_wait(&m.bar_o2, ph_o, status);
-            tc_fence_after();
             if (full) epilogue_dk<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
             else epilogue_dk<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
-            const float row_total = warp_transpose_reduce16(z, lane);
-            if (lane < 16) m.red[warp][lane] = row_total;
 #pragma unroll
             for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
             if (lane == 0) m.gred[warp] = g_part;
-            mbar_wait(&m.bar_o3, ph_o, status);
+            mbar_wait(&m.bar_o2, ph_o, status);
             tc_fence_after();
             if (full) epilogue_dv<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
             else epilogue_dv<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
+            mbar_wait(&m.bar_o3, ph_o, status);
+            tc_fence_after();
+            if (full) epilogue_dq<true>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
+            else epilogue_dq<false>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
+            const float row_total = warp_transpose_reduce16(z, lane);
+            if (lane < 16) m.red[warp][lane] = row_total;
             if (full) fence_async_smem();
         }
         ph_o ^= 1;
@@ -574,8 +580,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                     const int which = e / (BT * 32), t = (e / 32) % BT, j = e % 32;
                     if (rd.code[t] >= -1) continue;
                     float* out = which == 0 ? rk : rv;
+                    const int src = which == 1 ? Smem::ds + t * 512 + j * 16
+                                               : (j < 16 ? Smem::stage_dk : Smem::stage_dq) + t * 256 + (j & 15) * 16;
                     *reinterpret_cast<float4*>(out + ((size_t)(s.replay_base + t) * H + h) * D + j * 4) =
-                        *reinterpret_cast<const float4*>(smem + (which == 0 ? Smem::s : Smem::q) + t * 512 + j * 16);
+                        *reinterpret_cast<const float4*>(smem + src);
                 }
         }
         if (is_issuer && full) {
