@@ -509,7 +509,7 @@ def run_ours(args):
     achieved = bwd_bytes / (bwd_ms * 1e-3) / 1e9
     # DRAM bytes per token-head of the backward kernel from the ncu capture on cfg2 (profiles/
     # tc_bwd_kernel_cfg2_ncu_full.md), scaled to this workload's token-heads; traffic grows in proportion to them
-    BWD_DRAM_BYTES_PER_TOKEN_HEAD = 2369.0
+    BWD_DRAM_BYTES_PER_TOKEN_HEAD = 2356.0
     bwd_traffic_per_launch = (BWD_DRAM_BYTES_PER_TOKEN_HEAD * th / K) if (dk == 128 and not args.fma and elem == 2) \
         else None
     t_roof_bytes = (fwd_bytes + bwd_bytes) / (hbm_peak * 1e9)
