@@ -194,3 +194,31 @@ def test_repeated_runs_are_bit_identical():
             else:
                 for n in out:
                     assert torch.equal(out[n], first[n]), (k, n)
+
+
+def test_a_whole_step_can_be_captured_in_a_cuda_graph():
+    """The calls only enqueue work on the caller's stream (no allocation, no synchronisation), so all rounds of a
+    forward+backward step can be captured once and replayed; the replay gives the same bits as the eager step."""
+    cfg, fo, inp = config_case("cfg1")
+    plan = plan_of(fo).upload()
+    phys = to_physical(plan, inp)
+    ws = H.Workspace(plan, cfg["H"], cfg["dk"], cfg["dv"], phys["q"].dtype, 0)
+    out = H.run_fwd_bwd(plan, ws, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"])
+    ref = {n: x.clone() for n, x in out.items()}
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        H.run_fwd_bwd(plan, ws, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"], out=out, stream=s)   # warm-up
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=s):
+            H.run_fwd_bwd(plan, ws, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"], out=out, stream=s)
+    torch.cuda.synchronize()
+    for x in out.values():
+        x.zero_()
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    H.harts_la_check(ws.dev_status)
+    for n in out:
+        assert torch.equal(out[n], ref[n]), n
