@@ -143,8 +143,10 @@ def run_reference(args):
     if rank != 0:
         return
     times, secs, last = [], [], None
+    # every step is a bounded sample; its size shrinks with the step count so that the whole run stays within minutes
+    hint = min(8.0, 150.0 / max(1, args.warmup + args.steps))
     for i in range(args.warmup + args.steps):
-        last = oracle_sample(args.workload, seconds_hint=8.0)
+        last = oracle_sample(args.workload, seconds_hint=hint)
         if i >= args.warmup:
             times.append(last["value"])
             secs.append(last["seconds"])
@@ -1090,7 +1092,7 @@ def run_attn(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
