@@ -20,7 +20,8 @@
  *   - "host" / "device" in a comment says where the pointer must point.
  *   - Kernels are enqueued on the caller's stream (a cudaStream_t passed as void*) and the calls
  *     return without synchronising.  Device-detected errors (a bounded wait that ran out) are
- *     written to a caller-owned device status word and read back by harts_la_check().
+ *     written to a caller-owned device status word and read back by harts_la_check().  After a time-out the
+ *     outputs of that call are undefined; zero the status word before reusing it.
  *   - There is no CPU fallback: an unsupported (dtype, dk, dv, chunk) gives HARTS_EUNSUPPORTED.
  *   - Tensor layout: row-major [rows, H, d] with physical compact rows outermost (plan order,
  *     see row_of_token), heads next, the feature dimension contiguous.  Base pointers must be
@@ -227,6 +228,18 @@ int32_t harts_la_bwd_static(const harts_la_plan_t* plan, const void* dev_blob, c
 /* Synchronises `stream`, reads the device status word and returns HARTS_OK, HARTS_ETIMEOUT,
  * HARTS_EINVAL (an out-of-range index met by a harts_logp_* kernel, see harts_logp.h) or HARTS_ECUDA.  dev_status must be zeroed by the caller before the first launch. */
 int32_t harts_la_check(const int32_t* dev_status, void* stream);
+
+/*
+ * Self-test of the failure path of the device-side waits (every wait on an mbarrier in the kernels of this library is
+ * bounded: about half a second of wall time, after which the CTA records HARTS_ETIMEOUT in the status word, stops
+ * waiting anywhere else, leaves its loops, lets its copies and MMAs in flight finish, frees its tensor memory and
+ * returns).  This call launches one small CTA that waits, with a limit of one millisecond, on a barrier nothing arrives
+ * at.  Afterwards harts_la_check(dev_status) gives HARTS_ETIMEOUT and the context stays usable.
+ *   dev_status  DEVICE int32 status word (zeroed by the caller)
+ *   dev_report  DEVICE int32[5] or NULL: {first wait succeeded (0 expected), second wait succeeded (0), microseconds
+ *               in the first wait (about 1000), microseconds in the second (about 0: the latch was set), CTA saw the latch (1)}
+ */
+int32_t harts_la_selftest_timeout(int32_t* dev_status, int32_t* dev_report, void* stream);
 
 #ifdef __cplusplus
 }

@@ -39,9 +39,7 @@ class Tables(C.Structure):
 
 
 def _load():
-    path = _build.LIB
-    if not os.path.exists(path):
-        path = _build.build()
+    path = _build.build()      # recompiles only what is older than its sources
     lib = C.CDLL(path)
     vp, i32, u32, sz = C.c_void_p, C.c_int32, C.c_uint32, C.c_size_t
     lib.harts_la_strerror.argtypes = [i32]
@@ -62,6 +60,8 @@ def _load():
     lib.harts_la_check.argtypes = [vp, vp]
     lib.harts_la_bwd_static.argtypes = [vp, vp] + [vp] * 10 + [i32] * 4 + [u32, vp, vp]
     lib.harts_la_bwd_static.restype = i32
+    lib.harts_la_selftest_timeout.argtypes = [vp, vp, vp]
+    lib.harts_la_selftest_timeout.restype = i32
     for name in ("harts_la_plan", "harts_la_plan_view", "harts_la_plan_device_bytes", "harts_la_plan_upload",
                  "harts_la_plan_tables", "harts_la_workspace_bytes", "harts_la_fwd_seqs", "harts_la_bwd_seqs",
                  "harts_la_bwd_finish", "harts_la_fwd", "harts_la_bwd", "harts_la_check"):
@@ -218,6 +218,10 @@ def harts_la_bwd_static(plan, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, fl
     _check(lib.harts_la_bwd_static(plan._h, _ptr(plan.blob), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(dO), _ptr(dq),
                                    _ptr(dk_), _ptr(dv_), _ptr(dg), _ptr(chunk_states), H, dk, dv, dt, flags,
                                    _ptr(dev_status), _stream(stream)), "harts_la_bwd_static")
+
+
+def harts_la_selftest_timeout(dev_status, dev_report=None, stream=None):
+    _check(lib.harts_la_selftest_timeout(_ptr(dev_status), _ptr(dev_report), _stream(stream)), "harts_la_selftest_timeout")
 
 
 def harts_la_check(dev_status, stream=None):

@@ -1,34 +1,53 @@
-"""Builds the C-ABI shared library (libharts_la.so) in-tree with nvcc for sm_100a."""
+"""Builds the C-ABI shared library (libharts_la.so) in-tree with nvcc for sm_100a.
+
+Every source is compiled to an object of its own (in parallel, only when it or a header is newer than the
+object) and the objects are linked into the library."""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libharts_la.so")
 
 EXTRA = os.environ.get("HARTS_NVCC_EXTRA", "").split()
 NVCC_FLAGS = EXTRA + ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-shared"]
+                      "-Xcompiler", "-fPIC"]
 
 
 def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cc")) + glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _newest_input():
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(HERE, "..", "include", "*.h"))
-    return max(os.path.getmtime(p) for p in deps)
+def headers():
+    return (glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) +
+            glob.glob(os.path.join(HERE, "..", "include", "*.h")))
+
+
+def _mtime(path):
+    return os.path.getmtime(path) if os.path.exists(path) else -1.0
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_input():
-        return LIB
+    """Returns the library's path; recompiles what is older than its source or than any header."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + sources()
-    subprocess.check_call(cmd)
+    os.makedirs(OBJ, exist_ok=True)
+    hdr_time = max(_mtime(p) for p in headers())
+    jobs, objs = [], []
+    for src in sources():
+        obj = os.path.join(OBJ, os.path.basename(src) + ".o")
+        objs.append(obj)
+        if force or _mtime(obj) < max(_mtime(src), hdr_time):
+            jobs.append([nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", obj, src])
+    if jobs:
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 4)) as pool:
+            list(pool.map(subprocess.check_call, jobs))
+    if jobs or _mtime(LIB) < max(_mtime(o) for o in objs):
+        subprocess.check_call([nvcc, "-shared", "-o", LIB] + objs)
     return LIB
 
 

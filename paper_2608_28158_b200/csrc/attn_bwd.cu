@@ -64,7 +64,8 @@ struct SmemQ {
     static constexpr int bytes = misc + 256;
 };
 struct MiscQ {
-    uint64_t bar_q, bar_k[KST], bar_v[2], bar_kfree[KST], bar_vfree[2], bar_s, bar_dpfree, bar_p[2], bar_o;
+    uint64_t bar_q, bar_k[KST], bar_v[2], bar_kfree[KST], bar_vfree[2], bar_s, bar_dpfree, bar_p[2], bar_o, bar_exit;
+    int dead;        // latch: a wait of this CTA ran out, the CTA is abandoning its work
     uint32_t tmem;
 };
 constexpr int COL_DP = 256, COL_DQ = 384, TMEM_Q = 512;     // S of tile n at 128 (n & 1)
@@ -98,6 +99,8 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
         mbar_init(&m.bar_p[0], NS / 32);
         mbar_init(&m.bar_p[1], NS / 32);
         mbar_init(&m.bar_o, 1);
+        mbar_init(&m.bar_exit, 1);
+        m.dead = 0;
         fence_barrier_init();
     }
     if (warp == 0) tmem_alloc<TMEM_Q>(&m.tmem);
@@ -131,11 +134,12 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                     tma_load_3d(sDO + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_do, p * 64, h, q_row0 + r * 64, &m.bar_q);
                 }
             for (int n = 0; lw.next(lt); n++) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 const int stage = n & 1, kst = n % KST;
                 unsigned char* sK = smem + SmemQ::k0 + kst * KW_BYTES;
                 unsigned char* sV = smem + SmemQ::v0 + stage * KW_BYTES;
                 if (n >= KST) {
-                    mbar_wait(&m.bar_kfree[kst], ph_kfree[kst], status);         // released after dQ of tile n - KST
+                    mbar_wait(&m.bar_kfree[kst], ph_kfree[kst], status, &m.dead);         // released after dQ of tile n - KST
                     ph_kfree[kst] ^= 1;
                 }
                 mbar_expect_tx(&m.bar_k[kst], KW_BYTES);
@@ -143,7 +147,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                     for (int r = 0; r < 2; r++)
                         tma_load_3d(sK + p * (KW_BYTES / 2) + r * (KW_BYTES / 4), &map_k, p * 64, hk, lt.row + r * 64, &m.bar_k[kst]);
                 if (n >= 2) {
-                    mbar_wait(&m.bar_vfree[stage], ph_vfree[stage], status);     // released after dP of tile n - 2
+                    mbar_wait(&m.bar_vfree[stage], ph_vfree[stage], status, &m.dead);     // released after dP of tile n - 2
                     ph_vfree[stage] ^= 1;
                 }
                 mbar_expect_tx(&m.bar_v[stage], KW_BYTES);
@@ -157,7 +161,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
             const int n_tiles = WalkW(ix, piece, qt).count();
             auto issue_s = [&](int n) {      // S(n) into buffer n & 1
                 const int stage = n & 1, kst = n % KST;
-                mbar_wait(&m.bar_k[kst], ph_k[kst], status);
+                mbar_wait(&m.bar_k[kst], ph_k[kst], status, &m.dead);
                 ph_k[kst] ^= 1;
                 tc_fence_after();
                 const uint64_t dK = desc_kmajor_base(smem_u32(smem + SmemQ::k0 + kst * KW_BYTES));
@@ -167,7 +171,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
             };
             auto issue_dp = [&](int n) {     // dP(n); its commit also covers S(n), issued before it
                 const int stage = n & 1;
-                mbar_wait(&m.bar_v[stage], ph_v[stage], status);
+                mbar_wait(&m.bar_v[stage], ph_v[stage], status, &m.dead);
                 ph_v[stage] ^= 1;
                 tc_fence_after();
                 const uint64_t dV = desc_kmajor_base(smem_u32(smem + SmemQ::v0 + stage * KW_BYTES));
@@ -177,24 +181,25 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                 mma_commit(&m.bar_s);
                 if (n + 2 < n_tiles) mma_commit(&m.bar_vfree[stage]);
             };
-            mbar_wait(&m.bar_q, ph_q, status);
+            mbar_wait(&m.bar_q, ph_q, status, &m.dead);
             ph_q ^= 1;
             issue_s(0);
             issue_dp(0);
             for (int n = 0; n < n_tiles; n++) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 const int stage = n & 1;
                 // S(n+1) and dP(n+1) run under the element-wise pass of tile n: S has a second buffer, and the pass
                 // takes dP(n) into registers first and says so
                 if (n + 1 < n_tiles) {
                     issue_s(n + 1);
-                    mbar_wait(&m.bar_dpfree, ph_dpfree, status);
+                    mbar_wait(&m.bar_dpfree, ph_dpfree, status, &m.dead);
                     ph_dpfree ^= 1;
                     tc_fence_after();
                     issue_dp(n + 1);
                 }
                 // dS(n) written, S(n) read.  One barrier per S buffer: a warp that is done with tile n may already work
                 // on tile n+1 (its S and dP are complete) and arrive for it, and that arrival must not count for tile n.
-                mbar_wait(&m.bar_p[stage], ph_p[stage], status);
+                mbar_wait(&m.bar_p[stage], ph_p[stage], status, &m.dead);
                 ph_p[stage] ^= 1;
                 tc_fence_after();
                 const uint64_t dKm = desc_mnmajor_base<BKW>(smem_u32(smem + SmemQ::k0 + (n % KST) * KW_BYTES));
@@ -215,8 +220,9 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
             const float lse2 = row_ok ? lse[(size_t)(q_row0 + i) * Hq + h] * LOG2E : INFINITY;
             const float dl = row_ok ? delta[(size_t)(q_row0 + i) * Hq + h] : 0.f;
             for (int n = 0; walk.next(t); n++) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 const int b = n & 1;
-                mbar_wait_warp(&m.bar_s, ph_s, status);
+                mbar_wait_warp(&m.bar_s, ph_s, status, &m.dead);
                 ph_s ^= 1;
                 tc_fence_after();
                 const int limit = min(t.n_valid, t.shift == NO_DIAG ? BKW : i - t.shift + 1);
@@ -254,7 +260,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
                 if (lane == 0) mbar_arrive(&m.bar_p[b]);
             }
             // ---- epilogue: dQ -> bf16 ------------------------------------------------------------------------------
-            mbar_wait_warp(&m.bar_o, ph_o, status);
+            mbar_wait_warp(&m.bar_o, ph_o, status, &m.dead);
             tc_fence_after();
             const bool full = q_valid == BQ;
 #pragma unroll
@@ -281,7 +287,7 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
         }
         ph_o ^= 1;
         tc_fence_before();
-        __syncthreads();
+        if (__syncthreads_or(m.dead)) break;
         tc_fence_after();
         if (is_issuer && q_valid == BQ) {
             for (int p = 0; p < 2; p++)
@@ -291,6 +297,13 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
             tma_store_wait_read();
         }
         __syncthreads();
+    }
+    if (__syncthreads_or(m.dead)) {               // abandoned: let the loads and MMAs in flight finish (bounded)
+        if (is_issuer) {
+            mma_commit(&m.bar_exit);
+            mbar_wait_drain(&m.bar_exit, 0);
+        }
+        drain_delay();
     }
     if (is_issuer) tma_store_wait_all();
     tc_fence_before();

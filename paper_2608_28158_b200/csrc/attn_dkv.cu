@@ -39,7 +39,8 @@ struct Smem {
     static constexpr int bytes = misc + 256;
 };
 struct Misc {
-    uint64_t bar_kv, bar_q[STAGES], bar_s[2], bar_p[2], bar_free[STAGES], bar_o;
+    uint64_t bar_kv, bar_q[STAGES], bar_s[2], bar_p[2], bar_free[STAGES], bar_o, bar_exit;
+    int dead;        // latch: a wait of this CTA ran out, the CTA is abandoning its work
     uint32_t tmem;
 };
 
@@ -63,6 +64,8 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
         for (int s = 0; s < STAGES; s++) { mbar_init(&m.bar_q[s], 1); mbar_init(&m.bar_free[s], 1); }
         for (int b = 0; b < 2; b++) { mbar_init(&m.bar_s[b], 1); mbar_init(&m.bar_p[b], NS / 32); }
         mbar_init(&m.bar_o, 1);
+        mbar_init(&m.bar_exit, 1);
+        m.dead = 0;
         fence_barrier_init();
     }
     if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
@@ -95,9 +98,10 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
                     tma_load_3d(sV + p * (KV_TILE / 2) + r * (KV_TILE / 4), &map_v, p * 64, hk, kv_row0 + r * 64, &m.bar_kv);
                 }
             for (int n = 0; lw.next(lt); n++) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 const int stage = n % STAGES;
                 if (n >= STAGES) {
-                    mbar_wait(&m.bar_free[stage], ph_free[stage], status);
+                    mbar_wait(&m.bar_free[stage], ph_free[stage], status, &m.dead);
                     ph_free[stage] ^= 1;
                 }
                 unsigned char* sQ = smem + Smem::q0 + stage * Q_TILE;
@@ -114,7 +118,7 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
             const int n_tiles = QWalk(ix, piece, kt, hk, G).count();
             auto issue_s = [&](int n) {      // S^T(n), dP^T(n) into buffer n & 1
                 const int stage = n % STAGES, b = n & 1;
-                mbar_wait(&m.bar_q[stage], ph_q[stage], status);
+                mbar_wait(&m.bar_q[stage], ph_q[stage], status, &m.dead);
                 ph_q[stage] ^= 1;
                 tc_fence_after();
                 const uint64_t dQ = desc_kmajor_base(smem_u32(smem + Smem::q0 + stage * Q_TILE));
@@ -127,13 +131,14 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
                     mma_ss(tmem + b * 128 + 64, dVd + kstep_kmajor<BKV>(ks), dDO + kstep_kmajor<BQT>(ks), I_ST, ks > 0);
                 mma_commit(&m.bar_s[b]);
             };
-            mbar_wait(&m.bar_kv, ph_kv, status);
+            mbar_wait(&m.bar_kv, ph_kv, status, &m.dead);
             ph_kv ^= 1;
             issue_s(0);
             for (int n = 0; n < n_tiles; n++) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 if (n + 1 < n_tiles) issue_s(n + 1);
                 const int stage = n % STAGES, b = n & 1;
-                mbar_wait(&m.bar_p[b], ph_p[b], status);
+                mbar_wait(&m.bar_p[b], ph_p[b], status, &m.dead);
                 ph_p[b] ^= 1;
                 tc_fence_after();
                 const uint64_t dDOm = desc_mnmajor_base<BQT>(smem_u32(smem + Smem::do0 + stage * Q_TILE));
@@ -167,10 +172,11 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
             if (tid < 128) sVec[(tid >> 6) * BQT + (tid & 63)] = pre;            // buffer 0
             asm volatile("bar.sync 1, 256;" ::: "memory");
             for (int n = 0; walk.next(t); n++) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 const int b = n & 1;
                 more_ahead = more_ahead && ahead.next(ta);
                 if (more_ahead) pre = fetch(ta);              // in flight during this tile
-                mbar_wait_warp(&m.bar_s[b], ph_s[b], status);
+                mbar_wait_warp(&m.bar_s[b], ph_s[b], status, &m.dead);
                 ph_s[b] ^= 1;
                 tc_fence_after();
                 const float* vl = sVec + b * 2 * BQT;
@@ -209,7 +215,7 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
                 if (lane == 0) mbar_arrive(&m.bar_p[b]);
             }
             // ---- epilogue: dV, dK -> bf16 ---------------------------------------------------------------------------
-            mbar_wait_warp(&m.bar_o, ph_o, status);
+            mbar_wait_warp(&m.bar_o, ph_o, status, &m.dead);
             tc_fence_after();
             const bool full = kv_valid == BKV;
 #pragma unroll
@@ -241,7 +247,7 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
         }
         ph_o ^= 1;
         tc_fence_before();
-        __syncthreads();
+        if (__syncthreads_or(m.dead)) break;
         tc_fence_after();
         if (is_issuer && kv_valid == BKV) {
             for (int p = 0; p < 2; p++)
@@ -253,6 +259,13 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
             tma_store_wait_read();
         }
         __syncthreads();
+    }
+    if (__syncthreads_or(m.dead)) {               // abandoned: let the loads and MMAs in flight finish (bounded)
+        if (is_issuer) {
+            mma_commit(&m.bar_exit);
+            mbar_wait_drain(&m.bar_exit, 0);
+        }
+        drain_delay();
     }
     if (is_issuer) tma_store_wait_all();
     tc_fence_before();

@@ -42,7 +42,8 @@ struct Smem {
     static constexpr int bytes = misc + 256;
 };
 struct Misc {
-    uint64_t bar_q, bar_k[2], bar_v[2], bar_kfree[2], bar_vfree[2], bar_s[2], bar_p[2], bar_pv, bar_o;
+    uint64_t bar_q, bar_k[2], bar_v[2], bar_kfree[2], bar_vfree[2], bar_s[2], bar_p[2], bar_pv, bar_o, bar_exit;
+    int dead;        // latch: a wait of this CTA ran out, the CTA is abandoning its work
     uint32_t tmem;
 };
 
@@ -73,6 +74,8 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
         mbar_init(&m.bar_p[1], NS / 32);
         mbar_init(&m.bar_pv, 1);
         mbar_init(&m.bar_o, 1);
+        mbar_init(&m.bar_exit, 1);
+        m.dead = 0;
         fence_barrier_init();
     }
     if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
@@ -106,19 +109,20 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 for (int r = 0; r < 2; r++)
                     tma_load_3d(sQ + p * (Q_BYTES / 2) + r * (Q_BYTES / 4), &map_q, p * 64, h, q_row0 + r * 64, &m.bar_q);
             for (int n = 0; lw.next(lt); n++) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 const int stage = n & 1;
                 unsigned char* sK = smem + Smem::k0 + stage * KV_BYTES;
                 unsigned char* sV = smem + Smem::v0 + stage * KV_BYTES;
                 // the K tile of a stage is free as soon as S of its previous tile is done, the V tile only after P V
                 if (n >= 2) {
-                    mbar_wait(&m.bar_kfree[stage], ph_kfree[stage], status);
+                    mbar_wait(&m.bar_kfree[stage], ph_kfree[stage], status, &m.dead);
                     ph_kfree[stage] ^= 1;
                 }
                 mbar_expect_tx(&m.bar_k[stage], KV_BYTES);
                 for (int p = 0; p < 2; p++)
                     tma_load_3d(sK + p * (KV_BYTES / 2), &map_k, p * 64, hk, lt.row, &m.bar_k[stage]);
                 if (n >= 2) {
-                    mbar_wait(&m.bar_vfree[stage], ph_vfree[stage], status);
+                    mbar_wait(&m.bar_vfree[stage], ph_vfree[stage], status, &m.dead);
                     ph_vfree[stage] ^= 1;
                 }
                 mbar_expect_tx(&m.bar_v[stage], KV_BYTES);
@@ -131,7 +135,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
             const int n_tiles = TileWalk(ix, piece, qt).count();
             auto issue_s = [&](int n) {                     // S(n) into buffer n & 1, from stage n & 1
                 const int stage = n & 1;
-                mbar_wait(&m.bar_k[stage], ph_k[stage], status);
+                mbar_wait(&m.bar_k[stage], ph_k[stage], status, &m.dead);
                 ph_k[stage] ^= 1;
                 tc_fence_after();
                 const uint64_t dK = desc_kmajor_base(smem_u32(smem + Smem::k0 + stage * KV_BYTES));
@@ -141,10 +145,11 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 mma_commit(&m.bar_s[stage]);
                 if (n + 2 < n_tiles) mma_commit(&m.bar_kfree[stage]);     // the K tile will be refilled
             };
-            mbar_wait(&m.bar_q, ph_q, status);
+            mbar_wait(&m.bar_q, ph_q, status, &m.dead);
             ph_q ^= 1;
             issue_s(0);
             for (int n = 0; n < n_tiles; n++) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 const int stage = n & 1;
                 // S of tile n+1 goes to the other buffer and runs under the softmax of tile n (its K stage was freed
                 // by the P V MMAs of tile n-1, which precede it in the pipe)
@@ -152,9 +157,9 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 // O += P V for tile n as soon as the softmax warps have written P.  One barrier per S buffer: a warp that
                 // is done with tile n may already work on tile n+1 (its S is complete) and arrive for it, and that
                 // arrival must not count for tile n.
-                mbar_wait(&m.bar_p[stage], ph_p[stage], status);
+                mbar_wait(&m.bar_p[stage], ph_p[stage], status, &m.dead);
                 ph_p[stage] ^= 1;
-                mbar_wait(&m.bar_v[stage], ph_v[stage], status);
+                mbar_wait(&m.bar_v[stage], ph_v[stage], status, &m.dead);
                 ph_v[stage] ^= 1;
                 tc_fence_after();
                 const uint64_t dV = desc_mnmajor_base<BK>(smem_u32(smem + Smem::v0 + stage * KV_BYTES));
@@ -174,8 +179,9 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
             const int i = tid;                                // query row inside the tile
             int n = 0;
             while (walk.next(t)) {
+                if (*(volatile int*)&m.dead) break;       // a wait ran out: abandon the item
                 const int b = n & 1;
-                mbar_wait_warp(&m.bar_s[b], ph_s[b], status);
+                mbar_wait_warp(&m.bar_s[b], ph_s[b], status, &m.dead);
                 ph_s[b] ^= 1;
                 tc_fence_after();
                 const int limit = min(t.n_valid, t.shift == NO_DIAG ? BK : i - t.shift + 1);   // visible: j < limit
@@ -201,7 +207,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                     // was issued before them (it has its own buffer), so its completion does not say so; bar_pv does.  Its
                     // phase index is the running tile count; this warp is never more than one phase behind (P V of this tile
                     // cannot be issued before this warp arrives on bar_p), so the parity alone identifies the phase.
-                    mbar_wait_warp(&m.bar_pv, (tiles_done - 1) & 1, status);
+                    mbar_wait_warp(&m.bar_pv, (tiles_done - 1) & 1, status, &m.dead);
                     tc_fence_after();
                     const float m_new = raise ? mx : m_ref;
                     const float alpha = m_new == -INFINITY ? 1.f : ex2(m_ref - m_new);   // m_ref = -inf: O and l are still 0
@@ -243,7 +249,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
                 tiles_done++;
             }
             // ---- epilogue: O / l -> bf16, lse ----------------------------------------------------------------------
-            mbar_wait_warp(&m.bar_o, ph_o, status);
+            mbar_wait_warp(&m.bar_o, ph_o, status, &m.dead);
             tc_fence_after();
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
             const bool full = q_valid == BQ;
@@ -271,7 +277,7 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
         }
         ph_o ^= 1;
         tc_fence_before();
-        __syncthreads();                                      // O staged; tensor memory and Q tile free for the next item
+        if (__syncthreads_or(m.dead)) break;                                      // O staged; tensor memory and Q tile free for the next item
         tc_fence_after();
         if (is_issuer && q_valid == BQ) {
             for (int p = 0; p < 2; p++)
@@ -281,6 +287,13 @@ attn_fwd_kernel(Index ix, int Hq, int G, float scale_log2, const __grid_constant
             tma_store_wait_read();                            // the Q tile is reloaded right away
         }
         __syncthreads();
+    }
+    if (__syncthreads_or(m.dead)) {               // abandoned: let the loads and MMAs in flight finish (bounded)
+        if (is_issuer) {
+            mma_commit(&m.bar_exit);
+            mbar_wait_drain(&m.bar_exit, 0);
+        }
+        drain_delay();
     }
     if (is_issuer) tma_store_wait_all();
     tc_fence_before();

@@ -324,7 +324,11 @@ __global__ void __launch_bounds__(NT) fma_bwd_kernel(harts_la_tables_t tb, int s
                     rk[((size_t)(s.replay_base + c * BT + t) * H + h) * DK + i] = dkv;   // replay rows sit in chunk 0
                 }
             }
-            atomicAdd(&sr[t], rsum);
+            // the 16 threads of a row are one half of a warp: fixed-order butterfly, one writer (no atomics)
+            const unsigned half_mask = 0xffffu << (tid & 16);
+#pragma unroll
+            for (int o_ = 8; o_ > 0; o_ >>= 1) rsum += __shfl_xor_sync(half_mask, rsum, o_);
+            if (tx == 0) sr[t] = rsum;
         }
         // dv
         for (int r = 0; r < 4; r++) {

@@ -16,7 +16,8 @@
 // started there (read from the scratch area, where those sequences' calls left them).
 // S_c comes from the chunk-state workspace written by the forward ([d_k][d_v] bf16 per chunk-head).
 // Gradients of replayed rows go to the scratch area (fp32) and are folded into their ancestor rows by
-// the replay-reduce kernel.  Every wait is bounded.
+// the replay-reduce kernel.  Every wait is bounded; one that runs out sets the status word and a CTA-wide latch, and the
+// CTA leaves its loops at the end of the chunk, drains what it has in flight, releases tensor memory and returns.
 #include "kernels.h"
 #include "tc_common.cuh"
 
@@ -65,7 +66,8 @@ struct Misc {
     float red[NC / 32][16];  // per-warp partial sums of q.dq - k.dk (warp w covers rows 16(w>>2)..+15)
     float gred[NC / 32];
     uint32_t tmem;
-    uint64_t bar_tiles, bar_a, bar_o, bar_o2, bar_o3, bar_qk_read;
+    uint64_t bar_tiles, bar_a, bar_o, bar_o2, bar_o3, bar_qk_read, bar_exit;
+    int dead;                // latch: a wait of this CTA ran out, the walk is being abandoned
 };
 
 struct SeqInfo {
@@ -209,6 +211,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         mbar_init(&m.bar_o2, 1);
         mbar_init(&m.bar_o3, 1);
         mbar_init(&m.bar_qk_read, NC / 32);
+        mbar_init(&m.bar_exit, 1);
+        m.dead = 0;
         fence_barrier_init();
     }
     if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
@@ -221,6 +225,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     // Persistent CTAs: work item = (sequence, head); items are ordered longest sequence first and dealt to the CTAs
     // in a snake pattern, so that every CTA gets a similar amount of work.
     uint32_t ph_tiles = 0, ph_a = 0, ph_o = 0;
+    bool tiles_pending = false, gave_up = false;   // tiles_pending is kept by the issuing thread only
     const int G = gridDim.x;
     for (int tier = 0; tier * G < n_items; tier++) {
     const int item = (tier & 1) ? tier * G + (G - 1 - (int)blockIdx.x) : tier * G + (int)blockIdx.x;
@@ -257,6 +262,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     auto issue_tiles = [&](int c, bool tiles) {
         int row0 = s.own_begin - s.n_replay + c * BT;
         int idx = (s.chunk_base + c) * H + h;
+        tiles_pending = true;
         mbar_expect_tx(&m.bar_tiles, (tiles ? 4 * TILE : 0) + 2 * S_PANEL);
         tma_load_3d(sS, &map_cs, 0, 0, idx, &m.bar_tiles);
         tma_load_3d(sS + S_PANEL, &map_cs, 64, 0, idx, &m.bar_tiles);
@@ -354,8 +360,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             fence_async_smem();
             __syncthreads();
         }
-        mbar_wait(&m.bar_tiles, ph_tiles, status);
-        ph_tiles ^= 1;
+        if (mbar_wait(&m.bar_tiles, ph_tiles, status, &m.dead)) {
+            tiles_pending = false;
+            ph_tiles ^= 1;
+        }
         // ---- A = Q K^T on lanes 0..63, dA = dO V^T on lanes 64..127 (rows 0..63 of that operand are unused) ----------
         if (is_issuer) {
             tc_fence_after();
@@ -441,7 +449,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 g_part = gamma * dot;
             }
             // ---- P = A .* decay (lanes 0..63), dP = dA .* decay (lanes 64..127): 16 columns of one of them per thread ------
-            mbar_wait(&m.bar_a, ph_a, status);
+            mbar_wait(&m.bar_a, ph_a, status, &m.dead);
             tc_fence_after();
             {
                 const bool is_p = (warp & 3) < 2;
@@ -518,8 +526,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 mma_ss(tmem + COL_DS, dQm + kstep_mnmajor(ks), dDOsm + kstep_mnmajor(ks), I_MM128, true);
             mma_commit(&m.bar_o3);
             // every tile is free once these are done: the epilogue works from registers and tensor memory
-            mbar_wait(&m.bar_o3, ph_o, status);
-            mbar_wait(&m.bar_qk_read, ph_o, status);      // every compute warp has taken its q and k values
+            mbar_wait(&m.bar_o3, ph_o, status, &m.dead);
+            mbar_wait(&m.bar_qk_read, ph_o, status, &m.dead);      // every compute warp has taken its q and k values
             if (c > 0) issue_tiles(c - 1, next_tiles);
         }
         if (is_aux && c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);   // visible to the others at barrier (B)
@@ -541,18 +549,18 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             }
             // ---- epilogue in three parts, each as soon as its accumulators are complete -------------------------------
             float z[16];
-            mbar_wait(&m.bar_o, ph_o, status);
+            mbar_wait(&m.bar_o, ph_o, status, &m.dead);
             tc_fence_after();
             if (full) epilogue_dk<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
             else epilogue_dk<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
 #pragma unroll
             for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
             if (lane == 0) m.gred[warp] = g_part;
-            mbar_wait(&m.bar_o2, ph_o, status);
+            mbar_wait(&m.bar_o2, ph_o, status, &m.dead);
             tc_fence_after();
             if (full) epilogue_dv<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
             else epilogue_dv<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
-            mbar_wait(&m.bar_o3, ph_o, status);
+            mbar_wait(&m.bar_o3, ph_o, status, &m.dead);
             tc_fence_after();
             if (full) epilogue_dq<true>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
             else epilogue_dq<false>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
@@ -562,8 +570,9 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         }
         ph_o ^= 1;
         tc_fence_before();
-        __syncthreads();                          // (B) staged outputs, partial sums and the next chunk's row data visible
+        gave_up = __syncthreads_or(m.dead) != 0;  // (B) staged outputs, partial sums and the next chunk's row data visible
         tc_fence_after();
+        if (gave_up) break;
         if (is_compute && !full) {
             // partial chunk: the staged rows leave with 16-byte stores, own rows to the outputs (bf16), replayed rows
             // to the scratch (fp32); rows past the end go nowhere
@@ -621,6 +630,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             }
         }
     }
+    if (gave_up) break;
     // gradient w.r.t. the initial state: the hand-off into the producing sequence
     tc_fence_before();
     __syncthreads();
@@ -637,6 +647,11 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                             __uint_as_float(x[i4 * 4 + 3]));
     }
     }   // work items
+    if (__syncthreads_or(m.dead) && is_issuer) {  // abandoned: let copies and MMAs in flight finish (bounded)
+        if (tiles_pending) mbar_wait_drain(&m.bar_tiles, ph_tiles);
+        mma_commit(&m.bar_exit);
+        mbar_wait_drain(&m.bar_exit, 0);
+    }
     if (is_issuer) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();

@@ -13,7 +13,8 @@
 // sequence is gathered row by row instead (replay rows come from arbitrary ancestor rows).  The
 // start-of-chunk state goes to the chunk-state workspace (bf16, [d_k][d_v] per chunk-head) by TMA
 // store, and to its slot (fp32, [d_k][d_v]) when the plan requests that boundary.
-// Every wait is bounded; a wait that runs out sets the status word and the walk carries on.
+// Every wait is bounded; a wait that runs out sets the status word and a CTA-wide latch: the CTA leaves its loops at
+// the next chunk boundary, waits (bounded) for what it still has in flight, releases tensor memory and returns.
 #include "kernels.h"
 #include "tc_common.cuh"
 
@@ -46,7 +47,8 @@ struct Misc {
     int code[BT];        // physical row (>= 0 own), -2 - row (replay), -1 (past the end)
     float gamma;
     uint32_t tmem;
-    uint64_t bar_tma, bar_a, bar_o;
+    uint64_t bar_tma, bar_a, bar_o, bar_exit;
+    int dead;            // latch: a wait of this CTA ran out, the walk is being abandoned
 };
 
 struct SeqInfo {
@@ -93,6 +95,8 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         mbar_init(&m.bar_tma, 1);
         mbar_init(&m.bar_a, 1);
         mbar_init(&m.bar_o, 1);
+        mbar_init(&m.bar_exit, 1);
+        m.dead = 0;
         fence_barrier_init();
     }
     if (warp == 0) tmem_alloc<TMEM_COLS>(&m.tmem);
@@ -105,6 +109,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     // Persistent CTAs: work item = (sequence, head); items are ordered longest sequence first and dealt to the CTAs
     // in a snake pattern, so that every CTA gets a similar amount of work.
     uint32_t ph_tma = 0, ph_a = 0, ph_o = 0;
+    bool tma_pending = false, gave_up = false;     // tma_pending is kept by thread 0 only
     const int G = gridDim.x;
     for (int tier = 0; tier * G < n_items; tier++) {
     const int item = (tier & 1) ? tier * G + (G - 1 - (int)blockIdx.x) : tier * G + (int)blockIdx.x;
@@ -138,6 +143,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
 
     auto issue_tma = [&](int c) {
         int row0 = s.own_begin - s.n_replay + c * BT;
+        tma_pending = true;
         mbar_expect_tx(&m.bar_tma, 3 * TILE);
         for (int p = 0; p < 2; p++) {
             tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_tma);
@@ -170,8 +176,9 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     for (int c = 0; c < s.n_chunks; c++) {
         if (tid == 0) tma_store_wait_read();      // the previous chunk's state store has left sS
         tc_fence_before();
-        __syncthreads();                          // (1) epilogue of the previous chunk is over everywhere
+        gave_up = __syncthreads_or(m.dead) != 0;  // (1) epilogue of the previous chunk is over everywhere
         tc_fence_after();
+        if (gave_up) break;
         if (tid < BT) {
             m.code[tid] = my_code;
             float x = gval;                       // inclusive scan inside each of the two warps
@@ -212,8 +219,10 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             if (tid == 0) m.gamma = ex2(bn * LOG2E);
         }
         if (!(c == 0 && gather_first)) {
-            mbar_wait(&m.bar_tma, ph_tma, status);
-            ph_tma ^= 1;
+            if (mbar_wait(&m.bar_tma, ph_tma, status, &m.dead)) {
+                ph_tma ^= 1;
+                tma_pending = false;
+            }
         }
         // ---- A = Q K^T ----------------------------------------------------------------------------------
         if (tid == 0) {
@@ -261,7 +270,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             fence_async_smem();
         }
         // ---- P = A .* decay (warps 0,1)  |  K <- w .* K (warps 2,3) ------------------------------------------
-        mbar_wait(&m.bar_a, ph_a, status);
+        mbar_wait(&m.bar_a, ph_a, status, &m.dead);
         ph_a ^= 1;
         tc_fence_after();
         if ((warp & 3) < 2) {
@@ -324,7 +333,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 mma_ss(tmem + COL_S, desc_mnmajor<BT>(aK, ks), desc_mnmajor<BT>(aV, ks), IDESC_S, true);
             mma_commit(&m.bar_o);
         }
-        mbar_wait(&m.bar_o, ph_o, status);
+        mbar_wait(&m.bar_o, ph_o, status, &m.dead);
         ph_o ^= 1;
         tc_fence_after();
         if (tid == 0 && c + 1 < s.n_chunks) issue_tma(c + 1);   // tiles are free: every MMA that read them is done
@@ -374,7 +383,13 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             }
         }
     }
+    if (gave_up) break;
     }   // work items
+    if (__syncthreads_or(m.dead) && tid == 0) {   // abandoned: let copies and MMAs in flight finish (bounded)
+        if (tma_pending) mbar_wait_drain(&m.bar_tma, ph_tma);
+        mma_commit(&m.bar_exit);
+        mbar_wait_drain(&m.bar_exit, 0);
+    }
     if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();

@@ -10,10 +10,10 @@
 namespace harts {
 namespace tc {
 
-// A wait that ran out reports this code in the status word and lets the kernel run to its end
-// (results are garbage, nothing hangs, tensor memory is released).
+// A wait that ran out reports this code in the status word and latches a flag shared by the CTA: every later
+// wait of that CTA returns at once, its loops end, tensor memory is released (results are garbage, nothing hangs).
 constexpr int STATUS_TIMEOUT = 1;
-constexpr int WAIT_LIMIT = 1 << 22;
+constexpr unsigned long long WAIT_LIMIT_NS = 500ull * 1000 * 1000;   // wall time per wait; a healthy wait takes microseconds
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -31,15 +31,49 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
-    for (int i = 0; i < WAIT_LIMIT; i++)
-        if (mbar_try(bar, parity)) return;
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  `dead` points to the CTA's latch in shared memory (0 at kernel start).  Returns false when the wait
+// gave up: because this one ran out of time (the latch and the status word are then set), or because the latch was
+// already set by an earlier one.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, volatile int* dead,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
+    if (mbar_try(bar, parity)) return true;
+    if (*dead) return false;
+    const unsigned long long t0 = global_ns();
+    for (int round = 0; round < (1 << 24); round++) {            // the poll count is bounded too, should the timer stall
+#pragma unroll 1
+        for (int i = 0; i < 32; i++)
+            if (mbar_try(bar, parity)) return true;
+        if (*dead) return false;
+        if (global_ns() - t0 > limit_ns) break;
+    }
+    *dead = 1;
     if (status) atomicExch(status, STATUS_TIMEOUT);
+    return false;
 }
 // The same for a whole (converged) warp: one lane polls, so that 31 lanes do not spend shared-memory cycles on it.
-__device__ __forceinline__ void mbar_wait_warp(uint64_t* bar, uint32_t parity, int* status) {
-    if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, status);
-    __syncwarp();
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, int* status, volatile int* dead) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, status, dead);
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+// Last wait of a CTA that is giving up: waits (bounded, whatever the latch says) for a copy or MMA group still in
+// flight, so that nothing lands in shared or tensor memory after the CTA has gone.
+__device__ __forceinline__ void mbar_wait_drain(uint64_t* bar, uint32_t parity) {
+    const unsigned long long t0 = global_ns();
+    for (int round = 0; round < (1 << 20); round++) {
+        if (mbar_try(bar, parity)) return;
+        if (global_ns() - t0 > 20ull * 1000 * 1000) return;
+    }
+}
+// Fixed pause (about 0.2 ms, bounded) of a CTA that is giving up and cannot name the barriers of its loads in flight.
+__device__ __forceinline__ void drain_delay() {
+    const unsigned long long t0 = global_ns();
+    for (int i = 0; i < (1 << 20) && global_ns() - t0 < 200000ull; i++) {}
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
