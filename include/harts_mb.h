@@ -80,6 +80,21 @@ int32_t harts_mb_extract(const harts_mb_plan_t* plan, int32_t mb, int32_t cap_tr
                          int32_t* tree_node_ptr, int32_t* node_parent, int32_t* node_fork_off, int32_t* node_len,
                          int32_t* node_src, int32_t* n_trees, int32_t* n_nodes);
 
+/*
+ * The placement pass of the trie-aware greedy (Section 3.2 "Scale-independent trie-aware greedy", Eq. 10) on the
+ * trajectories of `plan`, step by step, as a record that can be checked against the definition of the compact-work
+ * increase: step i placed trajectory step_traj[i] (index in the plan's lexicographic order) into microbatch
+ * step_mb[i] (numbered in creation order; step_created[i] = 1 when it was opened for this trajectory) and claimed
+ * the work increase step_delta[i].
+ *   order  0 ascending lexicographic, 1 descending, 2 descending length, 3 descending unique-suffix score
+ *   policy 0 best-fit (largest work after insertion), 1 max-shared (largest |x| - delta); ties: earliest microbatch
+ *   cap    capacity of the four HOST output arrays; pass NULL arrays to get *n_steps (= number of trajectories) only
+ * The capacity T is the plan's.  Errors: HARTS_EINVAL.
+ */
+int32_t harts_mb_greedy_trace(const harts_mb_plan_t* plan, int32_t order, int32_t policy, int32_t cap,
+                              int32_t* step_traj, int32_t* step_mb, int32_t* step_created, int64_t* step_delta,
+                              int32_t* n_steps);
+
 #ifdef __cplusplus
 }
 #endif

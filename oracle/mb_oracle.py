@@ -117,3 +117,67 @@ def check_plan(trajs, mb_of_traj, replica, slot, D, T):
     slot_crit = sum(max(works[m] for m in range(K) if slot[m] == j) for j in range(K // D))
     load = [sum(works[m] for m in range(K) if replica[m] == d) for d in range(D)]
     return (sum(works), slot_crit, max(load)), works
+
+
+def delta_c(members, x):
+    """The compact-work increase that Eq. 10 gives in closed form, here from its definition: unique token nodes of the
+    microbatch's trie with the candidate trajectory minus without it."""
+    return trie_cost(list(members) + [x]) - trie_cost(list(members))
+
+
+def delta_c_eq10(members_sorted, x):
+    """Eq. 10 itself: members in lexicographic order, p / q the neighbours of x at its insertion position; a missing
+    neighbour's terms are left out."""
+    import bisect
+    pos = bisect.bisect_left(members_sorted, x)
+    p = members_sorted[pos - 1] if pos > 0 else None
+    q = members_sorted[pos] if pos < len(members_sorted) else None
+    d = len(x)
+    if p is not None:
+        d -= lcp(p, x)
+    if q is not None:
+        d -= lcp(x, q)
+    if p is not None and q is not None:
+        d += lcp(p, q)
+    return d
+
+
+def greedy_orders(trajs_sorted):
+    """The four processing orders of the greedy as index lists into the lexicographically sorted trajectories:
+    ascending, descending, descending length, descending unique-suffix score u(x) = |x| - max(LCP(p_x, x), LCP(x, q_x))
+    with p_x, q_x the global neighbours (ties keep lexicographic order)."""
+    n = len(trajs_sorted)
+    asc = list(range(n))
+    u = []
+    for i, x in enumerate(trajs_sorted):
+        left = lcp(trajs_sorted[i - 1], x) if i > 0 else 0
+        right = lcp(x, trajs_sorted[i + 1]) if i + 1 < n else 0
+        u.append(len(x) - max(left, right))
+    return [asc, asc[::-1], sorted(asc, key=lambda i: -len(trajs_sorted[i])), sorted(asc, key=lambda i: -u[i])]
+
+
+def greedy_place(trajs_sorted, order, T, best_fit):
+    """Placement pass of the trie-aware greedy with the work increase taken from the trie count (delta_c): each
+    trajectory goes to the capacity-feasible microbatch with the largest work after insertion (best-fit) or the
+    largest shared amount |x| - delta (max-shared), the earliest on ties, else a new microbatch.
+    Returns the steps [(trajectory index, microbatch, created, delta)]."""
+    bins = []
+    steps = []
+    for i in order:
+        x = trajs_sorted[i]
+        best, best_key, best_d = None, -1, 0
+        for b, members in enumerate(bins):
+            work = trie_cost(members)
+            d = delta_c(members, x)
+            if work + d > T:
+                continue
+            key = work + d if best_fit else len(x) - d
+            if key > best_key:
+                best, best_key, best_d = b, key, d
+        created = best is None
+        if created:
+            bins.append([])
+            best, best_d = len(bins) - 1, len(x)
+        bins[best].append(x)
+        steps.append((i, best, int(created), best_d))
+    return steps

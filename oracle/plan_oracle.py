@@ -413,3 +413,87 @@ def simulate_plan_autograd(plan, q, k, v, g, dO):
     o = torch.stack(outs)
     (o * dO).sum().backward()
     return tuple(x.detach().numpy() for x in (o, q.grad, k.grad, v.grad, g.grad))
+
+
+def simulate_plan_bwd_tables(plan, q, k, v, g, dO):
+    """Reverse pass over a plan that routes every gradient through the plan's OWN backward tables (no autograd):
+    the chunk-start states a backward would re-read are stored and addressed with `seq_chunk_ptr`; at a requested
+    boundary the initial-state gradients of the consuming sequences are collected through `slot_cons_ptr` /
+    `slot_cons_seq` (Section 3.4, "Differentiable boundary states": several consumers of one boundary are summed);
+    gradients of replayed rows are kept per replay entry and folded into their producer rows through `rg_row` /
+    `rg_ptr` / `rg_entry` (Section 4.2: the gather's backward accumulates into the unique producer row).  Inside a
+    chunk it is the plain reverse token recurrence, so a wrong table shows up against the trajectory-wise oracle.
+    Inputs on PHYSICAL rows, fp64 numpy.  Returns dq, dk, dv, dg on physical rows."""
+    C, H, dk_ = q.shape
+    dv_ = v.shape[2]
+    B = plan.chunk
+    n_chunks = int(plan.seq_chunk_ptr[-1])
+    chunk_state = [None] * n_chunks
+    slots = [None] * plan.n_slots
+    seq_rows = []
+    for r in range(plan.n_rounds):
+        produced = {}
+        for i in range(plan.round_seq_ptr[r], plan.round_seq_ptr[r + 1]):
+            s0 = plan.seq_init_slot[i]
+            S = np.zeros((H, dk_, dv_)) if s0 < 0 else slots[s0].copy()
+            rep = list(plan.replay_row[plan.seq_replay_ptr[i]:plan.seq_replay_ptr[i + 1]])
+            rows = rep + list(range(plan.seq_own_begin[i], plan.seq_own_begin[i] + plan.seq_own_len[i]))
+            req = {int(plan.slot_chunk[s]): s for s in range(plan.seq_req_ptr[i], plan.seq_req_ptr[i + 1])}
+            assert plan.seq_chunk_ptr[i + 1] - plan.seq_chunk_ptr[i] == (len(rows) + B - 1) // B
+            for j, row in enumerate(rows):
+                if j % B == 0:
+                    chunk_state[plan.seq_chunk_ptr[i] + j // B] = S.copy()
+                    if (j // B) in req:
+                        produced[req[j // B]] = S.copy()
+                S = np.exp(g[row])[:, None, None] * S + k[row][:, :, None] * v[row][:, None, :]
+        for s, val in produced.items():
+            slots[s] = val
+    assert all(x is not None for x in chunk_state)
+
+    dq, dk, dv, dg = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v), np.zeros_like(g)
+    ds0 = [None] * plan.n_seq                           # gradient w.r.t. each sequence's initial state
+    rk = np.zeros((len(plan.replay_row), H, dk_))       # gradients of replayed rows, per replay entry
+    rv = np.zeros((len(plan.replay_row), H, dv_))
+    rgr = np.zeros((len(plan.replay_row), H))
+    for r in reversed(range(plan.n_rounds)):
+        for i in range(plan.round_seq_ptr[r], plan.round_seq_ptr[r + 1]):
+            n_rep = int(plan.seq_replay_ptr[i + 1] - plan.seq_replay_ptr[i])
+            rows = list(plan.replay_row[plan.seq_replay_ptr[i]:plan.seq_replay_ptr[i + 1]]) + \
+                list(range(plan.seq_own_begin[i], plan.seq_own_begin[i] + plan.seq_own_len[i]))
+            req = {int(plan.slot_chunk[s]): s for s in range(plan.seq_req_ptr[i], plan.seq_req_ptr[i + 1])}
+            carry = np.zeros((H, dk_, dv_))             # dL/dS after the current token, already decayed to it
+            for c in reversed(range((len(rows) + B - 1) // B)):
+                lo_, hi_ = c * B, min((c + 1) * B, len(rows))
+                # recompute the states inside the chunk from its stored start state
+                S_prev = [chunk_state[plan.seq_chunk_ptr[i] + c]]
+                for j in range(lo_, hi_):
+                    row = rows[j]
+                    S_prev.append(np.exp(g[row])[:, None, None] * S_prev[-1] + k[row][:, :, None] * v[row][:, None, :])
+                for j in reversed(range(lo_, hi_)):
+                    row = rows[j]
+                    S_t, S_tm1 = S_prev[j - lo_ + 1], S_prev[j - lo_]
+                    dS = carry
+                    if j >= n_rep:
+                        dS = dS + q[row][:, :, None] * dO[row][:, None, :]
+                        dq[row] = np.einsum("hij,hj->hi", S_t, dO[row])
+                    gk = np.einsum("hij,hj->hi", dS, v[row])
+                    gv = np.einsum("hij,hi->hj", dS, k[row])
+                    gg = np.exp(g[row]) * np.einsum("hij,hij->h", S_tm1, dS)
+                    if j >= n_rep:
+                        dk[row], dv[row], dg[row] = gk, gv, gg
+                    else:
+                        e = plan.seq_replay_ptr[i] + j
+                        rk[e], rv[e], rgr[e] = gk, gv, gg
+                    carry = np.exp(g[row])[:, None, None] * dS
+                if c in req:                            # boundary c was exported: add every consumer's gradient
+                    s = req[c]
+                    for u in plan.slot_cons_seq[plan.slot_cons_ptr[s]:plan.slot_cons_ptr[s + 1]]:
+                        assert ds0[u] is not None       # consumers run in a later round: already done
+                        carry = carry + ds0[u]
+            ds0[i] = carry
+    for n, row in enumerate(plan.rg_row):
+        for e in plan.rg_entry[plan.rg_ptr[n]:plan.rg_ptr[n + 1]]:
+            dk[row] += rk[e]
+            dv[row] += rv[e]
+            dg[row] += rgr[e]
+    return dq, dk, dv, dg

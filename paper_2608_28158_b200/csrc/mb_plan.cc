@@ -241,26 +241,56 @@ void bin_erase(const Costs& c, Bin& b, int x) {
     b.work -= insert_delta(c, b, x);
 }
 
-bool greedy_plan(const Costs& c, i64 T, int D, const std::vector<int>& order, bool best_fit, Grouping* out) {
-    std::vector<Bin> bins;
+// One placement step as the greedy saw it: trajectory x went to microbatch dest (a new one when created == 1) with
+// work increase delta (Eq. 10).
+struct GreedyStep {
+    int x, dest, created;
+    i64 delta;
+};
+// The placement pass of the greedy: every trajectory, in the given order, goes to the capacity-feasible microbatch
+// with the largest work after insertion (best-fit) or the largest shared amount |x| - delta (max-shared); ties go to
+// the earliest microbatch; a new microbatch is opened when none fits.
+void greedy_place(const Costs& c, i64 T, const std::vector<int>& order, bool best_fit, std::vector<Bin>& bins,
+                  std::vector<GreedyStep>* trace) {
     for (int x : order) {
         int best = -1;
-        i64 best_key = -1;
+        i64 best_key = -1, best_delta = 0;
         for (size_t k = 0; k < bins.size(); ++k) {
             const i64 d = insert_delta(c, bins[k], x);
             if (bins[k].work + d > T) continue;
             const i64 key = best_fit ? bins[k].work + d : c.len[x] - d;     // work after insertion | shared amount
             if (key > best_key) {
                 best_key = key;
+                best_delta = d;
                 best = static_cast<int>(k);
             }
         }
-        if (best < 0) {
+        const bool created = best < 0;
+        if (created) {
             bins.emplace_back();
             best = static_cast<int>(bins.size()) - 1;
+            best_delta = c.len[x];
         }
         bin_insert(c, bins[best], x);
+        if (trace) trace->push_back({x, best, created ? 1 : 0, best_delta});
     }
+}
+// The four processing orders: ascending and descending lexicographic, descending length, descending unique-suffix
+// score u(x) = |x| - max(LCP with the global predecessor, LCP with the global successor); stable.
+std::vector<std::vector<int>> greedy_orders(const Costs& c) {
+    const int N = static_cast<int>(c.len.size());
+    std::vector<std::vector<int>> orders(4, std::vector<int>(N));
+    for (int i = 0; i < N; ++i) orders[0][i] = i, orders[1][i] = N - 1 - i, orders[2][i] = i, orders[3][i] = i;
+    std::stable_sort(orders[2].begin(), orders[2].end(), [&](int a, int b) { return c.len[a] > c.len[b]; });
+    std::vector<int> uniq(N);
+    for (int i = 0; i < N; ++i) uniq[i] = c.len[i] - std::max(c.L[i], i + 1 < N ? c.L[i + 1] : 0);
+    std::stable_sort(orders[3].begin(), orders[3].end(), [&](int a, int b) { return uniq[a] > uniq[b]; });
+    return orders;
+}
+
+bool greedy_plan(const Costs& c, i64 T, int D, const std::vector<int>& order, bool best_fit, Grouping* out) {
+    std::vector<Bin> bins;
+    greedy_place(c, T, order, best_fit, bins, nullptr);
     // eliminate small microbatches: re-place all members of the lightest one (max-shared destination), all or nothing
     while (bins.size() > 1) {
         size_t lightest = 0;
@@ -590,16 +620,11 @@ int32_t build(harts_mb_plan_t& p, int32_t n_trees, int32_t D, i64 T) {
     const size_t n_base_end = cands.size();
 
     // greedy: four processing orders x two placement policies, one candidate (fewest microbatches, then least work)
-    std::vector<std::vector<int>> orders(4, std::vector<int>(N));
-    for (int i = 0; i < N; ++i) orders[0][i] = i, orders[1][i] = N - 1 - i, orders[2][i] = i, orders[3][i] = i;
-    std::stable_sort(orders[2].begin(), orders[2].end(), [&](int a, int b) { return c.len[a] > c.len[b]; });
-    std::vector<int> uniq(N);
-    for (int i = 0; i < N; ++i) uniq[i] = c.len[i] - std::max(c.L[i], i + 1 < N ? c.L[i + 1] : 0);
-    std::stable_sort(orders[3].begin(), orders[3].end(), [&](int a, int b) { return uniq[a] > uniq[b]; });
+    const std::vector<std::vector<int>> orders = greedy_orders(c);
     bool have_greedy = false;
     Grouping greedy;
     i64 greedy_work = 0;
-    for (auto& order : orders)
+    for (const auto& order : orders)
         for (int policy = 0; policy < 2; ++policy) {
             Grouping g;
             if (!greedy_plan(c, T, D, order, policy == 0, &g)) continue;
@@ -725,6 +750,34 @@ extern "C" int32_t harts_mb_plan(int32_t n_trees, const int32_t* tree_node_ptr, 
     v.mb_replica = p->mb_replica.data();
     v.mb_slot = p->mb_slot.data();
     *out = p;
+    return HARTS_OK;
+}
+
+extern "C" int32_t harts_mb_greedy_trace(const harts_mb_plan_t* plan, int32_t order, int32_t policy, int32_t cap,
+                                         int32_t* step_traj, int32_t* step_mb, int32_t* step_created,
+                                         int64_t* step_delta, int32_t* n_steps) {
+    if (!plan || order < 0 || order > 3 || policy < 0 || policy > 1 || !n_steps) return HARTS_EINVAL;
+    try {
+        const int N = static_cast<int>(plan->traj_len.size());
+        Costs c;
+        c.len.assign(plan->traj_len.begin(), plan->traj_len.end());
+        c.L.assign(plan->traj_lcp.begin(), plan->traj_lcp.end());
+        c.build();
+        std::vector<Bin> bins;
+        std::vector<GreedyStep> trace;
+        greedy_place(c, plan->view.T, greedy_orders(c)[order], policy == 0, bins, &trace);
+        *n_steps = N;
+        if (!step_traj && !step_mb && !step_created && !step_delta) return HARTS_OK;
+        if (cap < N || !step_traj || !step_mb || !step_created || !step_delta) return HARTS_EINVAL;
+        for (int i = 0; i < N; ++i) {
+            step_traj[i] = trace[i].x;
+            step_mb[i] = trace[i].dest;
+            step_created[i] = trace[i].created;
+            step_delta[i] = trace[i].delta;
+        }
+    } catch (const std::bad_alloc&) {
+        return HARTS_ENOMEM;
+    }
     return HARTS_OK;
 }
 

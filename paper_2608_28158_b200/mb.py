@@ -25,7 +25,8 @@ lib.harts_mb_plan_free.argtypes = [_vp]
 lib.harts_mb_plan_free.restype = None
 lib.harts_mb_plan_view.argtypes = [_vp, C.POINTER(_MbView)]
 lib.harts_mb_extract.argtypes = [_vp, _i32, _i32, _i32, _I32P, _I32P, _I32P, _I32P, _I32P, _I32P, _I32P]
-for _n in ("harts_mb_plan", "harts_mb_plan_view", "harts_mb_extract"):
+lib.harts_mb_greedy_trace.argtypes = [_vp, _i32, _i32, _i32, _I32P, _I32P, _I32P, _I64P, _I32P]
+for _n in ("harts_mb_plan", "harts_mb_plan_view", "harts_mb_extract", "harts_mb_greedy_trace"):
     getattr(lib, _n).restype = _i32
 
 
@@ -50,6 +51,17 @@ class MbPlan:
         h, self._h = getattr(self, "_h", None), None
         if h:
             lib.harts_mb_plan_free(h)
+
+    def greedy_trace(self, order, policy):
+        """(trajectory, microbatch, created, delta) of every step of the greedy's placement pass."""
+        n = self.n_traj
+        x, mb, created = (np.empty(n, np.int32) for _ in range(3))
+        delta = np.empty(n, np.int64)
+        cnt = _i32(0)
+        ip = lambda a: a.ctypes.data_as(_I32P)  # noqa: E731
+        _check(lib.harts_mb_greedy_trace(self._h, order, policy, n, ip(x), ip(mb), ip(created),
+                                         delta.ctypes.data_as(_I64P), C.byref(cnt)), "harts_mb_greedy_trace")
+        return x, mb, created, delta
 
     def extract(self, mb):
         """(tree_node_ptr, node_parent, node_fork_off, node_len, node_src) of one microbatch's compact forest."""

@@ -155,3 +155,31 @@ def test_errors():
         _plan(fo, 4, 10 ** 6)                                    # fewer trajectories than replicas
     with pytest.raises(H.HartsError):
         H.harts_mb_plan([0, 2], [-1, 0], [0, 9], [4, 4], 1, 100)
+
+
+def test_greedy_increments_and_destinations_follow_eq10():
+    """Every step of the planner's greedy placement pass -- the processing order, the work increase it claims
+    (Eq. 10 through the LCP index), the destination under best-fit / max-shared, the moment a new microbatch is
+    opened -- against the oracle's pass, which takes the increase from the trie count with and without the
+    candidate.  A greedy that ignored sharing, used the wrong neighbours or broke ties differently fails here."""
+    rnd = random.Random(12)
+    shared_steps = 0
+    for trial in range(40):
+        fo = make_forest([random_tree(rnd, 9, 12) for _ in range(rnd.randint(1, 4))])
+        all_t = mo.trajectory_tokens(fo)
+        longest = max(len(t) for t in all_t)
+        T = rnd.randint(longest, max(longest, fo.n_tokens // 2 + longest))
+        try:
+            plan = _plan(fo, 1, T)
+        except H.HartsError:
+            continue
+        trajs = _lex_trajs(fo, plan)
+        orders = mo.greedy_orders(trajs)
+        for order in range(4):
+            for policy in range(2):
+                x, mb, created, delta = plan.greedy_trace(order, policy)
+                want = mo.greedy_place(trajs, orders[order], T, best_fit=(policy == 0))
+                got = list(zip(x.tolist(), mb.tolist(), created.tolist(), delta.tolist()))
+                assert got == want, (trial, order, policy)
+                shared_steps += sum(1 for (i, _, c, d) in want if not c and d < len(trajs[i]))
+    assert shared_steps > 200                                    # sharing did decide many placements

@@ -52,3 +52,31 @@ def test_slot_schedule_rule():
     # heaviest first: 9, 7 | 5, 1; second slot: 5 goes to the replica that has 7, 1 to the one that has 9
     assert slot == [1, 0, 0, 1] and replica[1] != replica[2] and replica[0] == replica[2] and replica[3] == replica[1]
     assert tail == (9 + 5, 12)
+
+
+def test_eq10_closed_form_equals_the_trie_count_difference():
+    """Pins both sides of Eq. 10: the brute-force definition (trie with x minus trie without x) and the printed
+    closed form agree for insertion in the middle, at either end, and into an empty microbatch."""
+    import random
+    from test_plan_oracle import random_tree
+    from workloads import make_forest
+    rng = random.Random(5)
+    seen_middle = seen_end = 0
+    for _ in range(40):
+        fo = make_forest([random_tree(rng, rng.randint(2, 10), 12) for _ in range(rng.randint(1, 2))])
+        trajs = sorted(mo.trajectory_tokens(fo))
+        for _ in range(6):
+            k = rng.randint(0, len(trajs) - 1)
+            members = sorted(rng.sample(trajs, k))
+            rest = [t for t in trajs if t not in members]
+            x = rng.choice(rest)
+            assert mo.delta_c(members, x) == mo.delta_c_eq10(members, x)
+            if members:
+                if members[0] < x < members[-1]:
+                    seen_middle += 1
+                else:
+                    seen_end += 1
+    assert seen_middle > 10 and seen_end > 10
+    # hand-counted: members {ab, abc... } on explicit token tuples
+    a, b, c = (1, 2, 3, 4), (1, 2, 5), (1, 2, 3, 9, 9)
+    assert mo.delta_c([a, b], c) == 2 and mo.delta_c([], c) == 5 and mo.delta_c([b], a) == 2

@@ -196,3 +196,60 @@ def test_appendix_totals_are_self_consistent():
         assert sum(per_call) == int(R)
         assert [sum(m) for m in members] == per_call
         assert all(0 <= x < 64 for m in members for x in m)
+
+
+def _phys_inputs(fo, plan, H, dk, dv, seed):
+    inp = {n: x.double().numpy() for n, x in make_inputs(fo.n_tokens, H, dk, dv, "fp32", seed).items()}
+    phys = {n: np.empty_like(x) for n, x in inp.items()}
+    for n in inp:
+        phys[n][plan.row_of_token] = inp[n]
+    return inp, phys
+
+
+def test_backward_tables_route_gradients_to_the_oracle():
+    """Pins the plan's backward tables (slot consumers, replayed-row gradient CSR, chunk-state addressing): a plain
+    reverse token recurrence that takes every hand-off and replay gradient THROUGH those tables must reproduce the
+    trajectory-wise oracle."""
+    rng = random.Random(11)
+    cases = [config_forest("cfg0"), config_forest("cfg0b")]
+    cases += [make_forest([random_tree(rng, rng.randint(2, 9), 40) for _ in range(rng.randint(1, 3))]) for _ in range(14)]
+    seen_shared_slot = seen_multi_replay = 0
+    for n, fo in enumerate(cases):
+        B = 64 if n < 2 else rng.choice([4, 8])
+        plan = po.plan_forest(fo, B)
+        inp, phys = _phys_inputs(fo, plan, 2, 3, 2, 100 + n)
+        ref = lo.forest_eval(fo, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"])
+        got = po.simulate_plan_bwd_tables(plan, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"])
+        for mine, name in zip(got, ("dq", "dk", "dv", "dg")):
+            np.testing.assert_allclose(mine[plan.row_of_token], ref[name], rtol=1e-9, atol=1e-11, err_msg=f"{n} {name}")
+        seen_shared_slot += int((np.diff(plan.slot_cons_ptr) > 1).any())
+        seen_multi_replay += int((np.diff(plan.rg_ptr) > 1).any())
+    assert seen_shared_slot >= 3 and seen_multi_replay >= 3     # the cases do exercise summed consumers
+
+
+@pytest.mark.parametrize("table", ["slot_cons_seq", "slot_cons_ptr", "rg_entry", "rg_row", "seq_chunk_ptr"])
+def test_a_wrong_backward_table_is_caught(table):
+    """The pin above has teeth: corrupting any one backward table changes the gradients (or trips a check)."""
+    fo = config_forest("cfg0b")
+    plan = po.plan_forest(fo, 64)
+    inp, phys = _phys_inputs(fo, plan, 1, 3, 2, 5)
+    ref = lo.forest_eval(fo, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"])
+    bad = getattr(plan, table).copy()
+    if table == "slot_cons_seq":
+        assert len(bad) >= 2
+        bad[0] = bad[1]                       # one consumer counted twice, another dropped
+    elif table == "slot_cons_ptr":
+        bad[-1] -= 1                          # last consumer dropped
+    elif table == "rg_entry":
+        bad[0] = bad[-1]                      # a replay entry folded into the wrong row
+    elif table == "rg_row":
+        bad[0] += 1
+    else:
+        bad[1:] += 1                          # chunk states read from the neighbouring chunk
+    setattr(plan, table, bad)
+    try:
+        got = po.simulate_plan_bwd_tables(plan, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"])
+    except (AssertionError, IndexError, TypeError):
+        return
+    worst = max(np.abs(m[plan.row_of_token] - ref[n]).max() for m, n in zip(got, ("dq", "dk", "dv", "dg")))
+    assert worst > 1e-6
