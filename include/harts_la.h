@@ -109,7 +109,11 @@ typedef struct harts_la_tables {
     const int32_t* rg_row;
     const int32_t* rg_ptr;
     const int32_t* rg_entry;
-    const int32_t* seq_order;      /* may be NULL: sequences are then processed in index order */
+    const int32_t* seq_order;      /* may be NULL: sequences are then processed in index order.  When set, a call's
+                                      range [seq_lo, seq_hi) must be one over which seq_order is a permutation of
+                                      itself (the planner's table is one per whole round): the tensor-core kernels
+                                      take sequence seq_order[seq_lo + i] as their i-th work item, so a sub-range of
+                                      a round needs seq_order = NULL */
 } harts_la_tables_t;
 
 const char* harts_la_strerror(int32_t code);
@@ -213,7 +217,10 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
  *     holds until the process ends.  A problem whose scratch need (harts_la_workspace_bytes) is larger is rejected
  *     with HARTS_ESCRATCH before anything is launched.
  *   - The first call on a device looks up the array's device address (one runtime query, result kept per device);
- *     make that first call with the device current and before any stream capture begins.
+ *     make that first call with the device current and before any stream capture begins.  With CUDA's lazy module
+ *     loading that query is also the moment the driver sets the array up on the device, so make the first call while
+ *     the device still has HARTS_STATIC_SCRATCH_BYTES to spare: HARTS_ECUDA from a first call can mean exactly that
+ *     the device had no room left for it.  Later calls touch no allocator at all.
  *   - All calls on a device share the one array, and it keeps whatever the last call left in it.  The backward
  *     writes every scratch entry before it reads it, so nothing needs clearing; but two calls that overlap on the
  *     GPU (different streams, or another host thread) race on the array and corrupt each other's gradients.

@@ -84,3 +84,40 @@ def branch_view_mask(h, l):
     i = np.arange(l)[:, None]
     j = np.arange(h + l)[None, :]
     return j <= h + i
+
+
+def descendants(forest, s):
+    """Canonical indices of every token whose path contains token s (s itself included), ascending."""
+    pred = predecessors(forest)
+    inside = np.zeros(forest.n_tokens, bool)
+    inside[s] = True
+    for t in range(s + 1, forest.n_tokens):       # canonical order puts a token after its predecessor
+        p = pred[t]
+        if p >= 0 and inside[p]:
+            inside[t] = True
+    return np.nonzero(inside)[0]
+
+
+def attn_bwd_key_row(forest, q, k, v, dO, scale, s):
+    """dk[s], dv[s] ([Hkv, d] each) written out from the definition for ONE key row: the sum, over every query t
+    that sees s (its descendants on every branch, and s itself) and every query head of the group, of
+        dv_s += p_t(s) dO_t,      dk_s += scale * p_t(s) (dO_t . v_s - sum_r p_t(r) dO_t . v_r) q_t
+    with p_t the softmax of t's scores over its own path.  Same arithmetic as attn_bwd restricted to one row, so that
+    a shared ancestor of thousands of queries can be checked at full problem size."""
+    q, k, v, dO = (np.asarray(a, np.float64) for a in (q, k, v, dO))
+    Hq, Hkv = q.shape[1], k.shape[1]
+    G = Hq // Hkv
+    dk_s, dv_s = np.zeros((Hkv, k.shape[2])), np.zeros((Hkv, v.shape[2]))
+    pred = predecessors(forest)
+    for t in descendants(forest, s):
+        path = _path(pred, int(t))
+        at = int(np.nonzero(path == s)[0][0])
+        for h in range(Hq):
+            hk = h // G
+            sc = scale * (k[path, hk] @ q[t, h])
+            p = np.exp(sc - sc.max())
+            p /= p.sum()
+            dp = v[path, hk] @ dO[t, h]
+            dv_s[hk] += p[at] * dO[t, h]
+            dk_s[hk] += scale * p[at] * (dp[at] - np.dot(p, dp)) * q[t, h]
+    return dk_s, dv_s

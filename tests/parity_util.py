@@ -18,6 +18,19 @@ def rel_err(x, ref):
     return float(np.linalg.norm(x - ref) / max(np.linalg.norm(ref), 1e-3 * np.sqrt(ref.size)))
 
 
+def row_err(x, ref):
+    """Largest per-row error: a row is the feature vector of one (token, head) -- for dg, its one number -- and its
+    error is measured against max(norm of the reference row, RMS norm of a row of the tensor), so that a row that is
+    nearly zero is held to the tensor's typical size.  One wrong row among half a million moves the Frobenius error
+    of the tensor by nothing; it moves this."""
+    x = np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    width = x.shape[-1] if x.ndim == 3 else 1
+    x, ref = x.reshape(-1, width), ref.reshape(-1, width)
+    floor = max(np.sqrt((ref ** 2).mean() * width), 1e-3 * np.sqrt(width))
+    return float((np.linalg.norm(x - ref, axis=1) / np.maximum(np.linalg.norm(ref, axis=1), floor)).max())
+
+
 def plan_of(fo, chunk=64):
     return H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, chunk)
 
@@ -57,10 +70,17 @@ def oracle_subset(fo, inp_canon, tree_ids, heads, backward=True):
     return tok, res
 
 
-def compare(out_canon, tok, heads, ref, names=("o", "dq", "dk", "dv", "dg")):
+def compare(out_canon, tok, heads, ref, names=("o", "dq", "dk", "dv", "dg"), rows=False):
+    """Relative Frobenius error per tensor; with rows=True also the largest per-row error (keys "<name>.row")."""
     ti = torch.as_tensor(tok, device="cuda")
     hi = torch.as_tensor(heads, device="cuda")
-    return {n: rel_err(out_canon[n][ti][:, hi].float().cpu().numpy(), ref[n]) for n in names}
+    errs = {}
+    for n in names:
+        got = out_canon[n][ti][:, hi].float().cpu().numpy()
+        errs[n] = rel_err(got, ref[n])
+        if rows:
+            errs[n + ".row"] = row_err(got, ref[n])
+    return errs
 
 
 def config_case(name, device="cpu"):

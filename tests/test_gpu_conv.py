@@ -55,6 +55,43 @@ def test_parity_on_trees(name, D, w, dtype):
     assert ey <= TOL[dtype] and ex <= TOL[dtype] and ew <= 1e-4, (ey, ex, ew)
 
 
+def test_bench_size_all_rows_of_sampled_channels():
+    """The benchmark's workload (cfg3's 588,899 compact rows x 4096 channels, bf16, w = 4, plan row order).  The
+    convolution is depthwise, so a channel can be checked on its own: for eight channels spread over the width, every
+    row of y and dx (all strip heads and tails, every fork row) and the channels' dW against the oracle."""
+    fo = config_forest("cfg3")
+    C, Dm, w = fo.n_tokens, 4096, 4
+    inp = make_conv_inputs(C, Dm, w, "bf16", 7, device="cuda")
+    rot = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64).row_of_token
+    prev, nxt, cptr, crow = H.harts_conv_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, rot)
+    rows = torch.as_tensor(rot.astype(np.int64)).cuda()
+    x = torch.empty_like(inp["x"]); x[rows] = inp["x"]
+    dy = torch.empty_like(inp["dy"]); dy[rows] = inp["dy"]
+    W = inp["W"]
+    dev = lambda a: torch.as_tensor(np.ascontiguousarray(a)).cuda()  # noqa: E731
+    y = torch.full_like(x, float("nan")); dx = torch.full_like(x, float("nan")); dW = torch.full_like(W, float("nan"))
+    scratch = torch.empty(H.harts_conv_scratch_bytes(Dm, w), dtype=torch.uint8, device="cuda")
+    H.harts_conv_fwd(x, W, dev(prev), y)
+    H.harts_conv_bwd(x, W, dy, dev(nxt), dev(cptr), dev(crow), dx, dW, scratch)
+    torch.cuda.synchronize()
+    ch = [0, 1, 7, 8, 1023, 2048, 4094, 4095]
+    cht = torch.as_tensor(ch).cuda()
+    x64, dy64 = (inp[n][:, cht].double().cpu().numpy() for n in ("x", "dy"))
+    W64 = W[cht].double().cpu().numpy()
+    y_ref = co.conv_fwd(fo, x64, W64)
+    dx_ref, dW_ref = co.conv_bwd(fo, x64, W64, dy64)
+    got_y = y[rows][:, cht].double().cpu().numpy()
+    got_dx = dx[rows][:, cht].double().cpu().numpy()
+    assert _rel(got_y, y_ref) <= TOL["bf16"] and _rel(got_dx, dx_ref) <= TOL["bf16"]
+    # row by row as well: one wrong row must not hide in the norm over 589 k rows (bf16 rounding: 2^-9 per element)
+    for got, ref in ((got_y, y_ref), (got_dx, dx_ref)):
+        row_err = np.linalg.norm(got - ref, axis=1)
+        floor = np.sqrt((ref ** 2).mean() * ref.shape[1])
+        assert (row_err / np.maximum(np.linalg.norm(ref, axis=1), floor)).max() <= 2 * TOL["bf16"]
+    assert _rel(dW[cht].double().cpu().numpy(), dW_ref) <= 1e-4
+    assert bool(torch.isfinite(y.float()).all()) and bool(torch.isfinite(dx.float()).all())
+
+
 def test_parity_without_a_row_map_and_on_bushy_trees():
     # every token forks: roots of 3 tokens with children at every offset, grandchildren too
     par = [-1, 0, 0, 0, 1, 1, 2, 4]

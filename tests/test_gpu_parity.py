@@ -16,9 +16,16 @@ TOL = {"fp32": dict(o=1e-4, dq=1e-4, dk=1e-4, dv=1e-4, dg=1e-4),
        "bf16": dict(o=5e-3, dq=1e-2, dk=1e-2, dv=1e-2, dg=1e-2)}
 
 
+# Besides the Frobenius tolerance per tensor, every single (token, head) row is held to ROW_MULT times that tolerance (observed worst rows: 0.9x for o, 0.5x for dq, dk, dv, 1.5x for dg)
+# (relative to the larger of its own norm and the tensor's RMS row norm): the Frobenius error is an RMS over rows, the
+# worst of 10^5..10^6 rows of independent bf16 roundings lies a few standard deviations above it.
+ROW_MULT = 2.0
+
+
 def check(errs, dtype):
     for n, e in errs.items():
-        assert e <= TOL[dtype][n], (n, e, errs)
+        base = n.split(".")[0]
+        assert e <= TOL[dtype][base] * (ROW_MULT if n.endswith(".row") else 1.0), (n, e, errs)
 
 
 @pytest.mark.parametrize("name", ["cfg0", "cfg0b", "cfg1"])
@@ -27,19 +34,19 @@ def test_small_configs_full_parity(name):
     plan, out = run_gpu(fo, inp)
     tok, ref = oracle_subset(fo, inp, list(range(fo.n_trees)), list(range(cfg["H"])))
     assert ref["copy_gap"] < 1e-9
-    errs = compare(out, tok, list(range(cfg["H"])), ref)
+    errs = compare(out, tok, list(range(cfg["H"])), ref, rows=True)
     print(name, errs)
     check(errs, cfg["dtype"])
 
 
-@pytest.mark.parametrize("name,trees", [("cfg2", [0, 5]), ("cfg3", [3]), ("cfg4", [0, 63])])
+@pytest.mark.parametrize("name,trees", [("cfg2", [0, 5]), ("cfg3", [3, 17, 31]), ("cfg4", [0, 63])])
 def test_large_configs_sampled_parity(name, trees):
     # full-size launch on the GPU; the oracle evaluates whole trees for three heads
     cfg, fo, inp = config_case(name, device="cuda")
     plan, out = run_gpu(fo, inp)
     heads = [0, cfg["H"] // 2, cfg["H"] - 1]
     tok, ref = oracle_subset(fo, inp, trees, heads)
-    errs = compare(out, tok, heads, ref)
+    errs = compare(out, tok, heads, ref, rows=True)
     print(name, "C", plan.C, "R", plan.R, "rounds", plan.n_rounds, "seqs", plan.n_seq, errs)
     check(errs, cfg["dtype"])
     for x in out.values():
@@ -82,9 +89,44 @@ def test_edge_cases(case, dtype, d):
     inp = make_inputs(fo.n_tokens, 2, d, d, dtype, 17)
     plan, out = run_gpu(fo, inp)
     tok, ref = oracle_subset(fo, inp, list(range(fo.n_trees)), [0, 1])
-    errs = compare(out, tok, [0, 1], ref)
+    errs = compare(out, tok, [0, 1], ref, rows=True)
     print(case, dtype, errs)
     check(errs, dtype)
+
+
+def random_forest_cases(n_cases=36, seed=2024):
+    """Seeded forests of the kinds that random testing needs to meet: forks nested inside one chunk, replay spans that
+    cross several ancestor segments, several consumers of one exported state, chains of short branches, long roots."""
+    import random
+    from test_plan_oracle import random_tree
+    rnd = random.Random(seed)
+    cases = []
+    for i in range(n_cases):
+        max_len = rnd.choice([5, 40, 70, 200, 700])
+        trees = [random_tree(rnd, rnd.randint(1, 12), max_len) for _ in range(rnd.randint(1, 4))]
+        cases.append((make_forest(trees), rnd.choice([1, 2, 3, 4]), 500 + i))
+    return cases
+
+
+def test_random_forests_through_the_tensor_core_kernels():
+    """36 seeded random forests (1-4 heads, bf16, d = 128: the tcgen05 kernels) against the oracle, per tensor and
+    per row; also checks that the set covers the structures it is meant to cover."""
+    nested = multi_seg_replay = shared_slot = multi_round = 0
+    for fo, heads, seed in random_forest_cases():
+        inp = make_inputs(fo.n_tokens, heads, 128, 128, "bf16", seed)
+        plan, out = run_gpu(fo, inp)
+        tok, ref = oracle_subset(fo, inp, list(range(fo.n_trees)), list(range(heads)))
+        errs = compare(out, tok, list(range(heads)), ref, rows=True)
+        check(errs, "bf16")
+        rp = np.diff(plan.seq_replay_ptr)
+        for i in np.nonzero(rp > 0)[0]:
+            r = plan.replay_row[plan.seq_replay_ptr[i]:plan.seq_replay_ptr[i + 1]]
+            multi_seg_replay += int((np.diff(r) != 1).any())          # replayed rows from more than one row range
+        nested += int((np.diff(plan.rg_ptr) > 1).any())               # a row replayed by several sequences
+        shared_slot += int((np.diff(plan.slot_cons_ptr) > 1).any())
+        multi_round += int(plan.n_rounds >= 3)
+    print("coverage:", nested, multi_seg_replay, shared_slot, multi_round)
+    assert nested >= 5 and multi_seg_replay >= 5 and shared_slot >= 5 and multi_round >= 2
 
 
 def test_rounds_issued_one_by_one_match_round_zero():

@@ -97,3 +97,21 @@ def test_central_differences():
         assert abs((f(q, kp, v) - f(q, km, v)) / (2 * h) - dk[idx]) < 1e-7
         vp, vm = v.copy(), v.copy(); vp[idx] += h; vm[idx] -= h
         assert abs((f(q, k, vp) - f(q, k, vm)) / (2 * h) - dv[idx]) < 1e-7
+
+
+def test_key_row_gradients_equal_the_full_backward_rows():
+    """attn_bwd_key_row (one key row from the definition, used for full-size checks) against attn_bwd, which is
+    pinned above by autograd: a root row with many descendants, a fork row, a leaf row; MHA and GQA."""
+    import random
+    from test_plan_oracle import random_tree
+    from workloads import make_attn_inputs, make_forest
+    rnd = random.Random(21)
+    fo = make_forest([random_tree(rnd, 7, 9) for _ in range(2)])
+    for Hq, Hkv in ((2, 2), (4, 2)):
+        inp = {n: x.double().numpy() for n, x in make_attn_inputs(fo.n_tokens, Hq, Hkv, 8, "fp32", 3).items()}
+        _, dk, dv = ao.attn_bwd(fo, inp["q"], inp["k"], inp["v"], inp["dO"], 0.3)
+        for s in (0, 1, fo.n_tokens // 2, fo.n_tokens - 1):
+            dk_s, dv_s = ao.attn_bwd_key_row(fo, inp["q"], inp["k"], inp["v"], inp["dO"], 0.3, s)
+            np.testing.assert_allclose(dk_s, dk[s], rtol=1e-10, atol=1e-13)
+            np.testing.assert_allclose(dv_s, dv[s], rtol=1e-10, atol=1e-13)
+    assert len(ao.descendants(fo, 0)) > 5
