@@ -17,6 +17,11 @@ print the same JSON keys.
 
 ``--impl reference`` times the fp64 CPU oracle (oracle/), as it stands, on the host cores, on a
 bounded sample of the same workload.
+
+Timing: W warm-up steps, then blocks of exactly K steps each, every block bracketed by a barrier and a device
+synchronisation and timed with CUDA events on the launching stream; when K steps take less than about two seconds,
+several blocks are run back to back and the MEDIAN block gives ``ms_per_step`` (the per-block times and clock medians
+are kept under ``timing``).  With ``--gpus N`` and no torchrun environment the script starts its N ranks itself.
 """
 from __future__ import annotations
 
@@ -105,6 +110,159 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------------------
+# Scaffold shared by every workload: ranks, timed blocks, end-to-end steps, JSON line
+# --------------------------------------------------------------------------------------------------
+class Ranks:
+    """This process' place in the job (torchrun's environment, or a single rank) and the job-wide barrier."""
+
+    def __init__(self):
+        import torch
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        torch.cuda.set_device(self.local)
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+
+    def barrier(self):
+        import torch
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def close(self):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+def max_over_ranks(values, device):
+    """Element-wise maximum of a few per-rank timings over all ranks (identity when not distributed)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def plan_blocks(steps, est_ms_per_step, target_ms=2000.0, most=9):
+    """How many blocks of `steps` steps to time: one when a block already lasts `target_ms`, else enough blocks to
+    fill it (an odd number, so that the median is a measured block), at most `most`."""
+    block = max(steps * est_ms_per_step, 1e-3)
+    if block >= target_ms:
+        return 1
+    n = min(most, int(-(-target_ms // block)))
+    return n if n % 2 == 1 else min(most, n + 1)
+
+
+def time_blocks(work, args, ranks):
+    """Warm-up, then the timed blocks.  Returns ms_per_step (median block, each block the max over ranks), the
+    per-launch event pairs of every timed step, and the clocks sampled during the blocks."""
+    import torch
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+    marks, block_ms, block_host = [], [], []
+    with ClockSampler(ranks.local) as clocks:      # started before the warm-up so that it is sampling by then
+        a, b = ev(), ev()
+        a.record(stream)
+        for _ in range(args.warmup):
+            work.step(None)
+        b.record(stream)
+        ranks.barrier()
+        work.check()
+        est = max_over_ranks([a.elapsed_time(b) / max(1, args.warmup)], "cuda")[0]
+        n_blocks = args.blocks if args.blocks > 0 else plan_blocks(args.steps, est)
+        for _ in range(n_blocks):
+            ranks.barrier()
+            h0 = clocks.mark()
+            a, b = ev(), ev()
+            a.record(stream)
+            for _ in range(args.steps):
+                work.step(marks)
+            b.record(stream)
+            ranks.barrier()
+            block_host.append((h0, clocks.mark()))
+            block_ms.append(a.elapsed_time(b))
+    work.check()
+    block_ms = max_over_ranks(block_ms, "cuda")
+    clock = clocks.summary(block_host[0][0], block_host[-1][1])
+    if not clock["samples"]:
+        clock = clocks.summary()
+        clock["note"] = "timed region shorter than the sampling period: samples cover warm-up + timed region"
+    per_block = [clocks.summary(h0, h1)["sm_mhz"] for h0, h1 in block_host]
+    kernel_ms = {}
+    for name, a, b in marks:
+        kernel_ms.setdefault(name, []).append(a.elapsed_time(b))
+    n_steps = n_blocks * args.steps
+    return {"ms_per_step": statistics.median(block_ms) / args.steps,
+            "kernel_ms": {n: sum(v) / n_steps for n, v in kernel_ms.items()},
+            "clocks": clock,
+            "timing": {"blocks": n_blocks, "steps_per_block": args.steps,
+                       "block_ms_per_step": [x / args.steps for x in block_ms], "block_sm_mhz": per_block,
+                       "ms_per_step": "median block"}}
+
+
+def host_copies(tensors):
+    """Pinned host twins of a dict of device tensors, filled with their contents."""
+    import torch
+    host = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in tensors.items()}
+    for n, x in tensors.items():
+        host[n].copy_(x)
+    torch.cuda.synchronize()
+    return host
+
+
+def time_e2e(work, dev_in, dev_out, n_steps, ranks):
+    """End-to-end steps on one stream: every step copies all inputs from pinned host memory, runs the path and copies
+    all results back, inside the timed region."""
+    import torch
+    stream = torch.cuda.current_stream()
+    host_in, host_out = host_copies(dev_in), host_copies(dev_out)
+
+    def e2e_step():
+        for n, x in dev_in.items():
+            x.copy_(host_in[n], non_blocking=True)
+        work.step(None)
+        for n, x in dev_out.items():
+            host_out[n].copy_(x, non_blocking=True)
+
+    e2e_step()
+    ranks.barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(n_steps):
+        e2e_step()
+    b.record(stream)
+    ranks.barrier()
+    nbytes = lambda d: sum(t.numel() * t.element_size() for t in d.values())  # noqa: E731
+    return {"ms": a.elapsed_time(b) / n_steps, "steps": n_steps, "h2d": nbytes(host_in), "d2h": nbytes(host_out)}
+
+
+# ---- measured DRAM traffic of the dominant kernels -----------------------------------------------------------------
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic.json")
+
+
+def measured_traffic(kernel):
+    """DRAM bytes per unit of `kernel` from the last profiler capture, or None when there is none or when a source
+    file of the kernel has changed since (the record carries the sources' hash; see paper_2608_28158_b200/traffic.py)."""
+    from paper_2608_28158_b200 import traffic
+    rec = traffic.load(TRAFFIC_FILE).get(kernel)
+    if not rec or rec.get("source_sha256") != traffic.source_hash(rec.get("sources", [])):
+        return None
+    return rec
+
+
+def hbm_roofline(kernel, bytes_per_launch, ms, peaks, traffic_per_launch, **extra):
+    achieved = bytes_per_launch / (ms * 1e-3) / 1e9
+    out = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+           "frac": achieved / peaks["hbm_gbs"], "traffic": traffic_per_launch,
+           "algorithmic_bytes_per_launch": bytes_per_launch, "peak_source": peaks["source"]}
+    out.update(extra)
+    return out
+# --------------------------------------------------------------------------------------------------
 def oracle_sample(name, seconds_hint=15.0):
     """The fp64 oracle on a bounded sample of the workload: whole trees, a few heads."""
     import torch
@@ -136,121 +294,6 @@ def oracle_sample(name, seconds_hint=15.0):
             "sample": f"{name}: trees {trees[0]}..{trees[-1]} ({sub.n_tokens} compact / {res['S']} trajectory-wise "
                       f"tokens), {len(heads)} of {cfg['H']} heads, fwd+bwd, {dt:.1f} s",
             "semantic_token_heads_per_s": res["S"] * len(heads) / dt, "seconds": dt}
-
-
-def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
-    times, secs, last = [], [], None
-    # every step is a bounded sample; its size shrinks with the step count so that the whole run stays within minutes
-    hint = min(8.0, 150.0 / max(1, args.warmup + args.steps))
-    for i in range(args.warmup + args.steps):
-        last = oracle_sample(args.workload, seconds_hint=hint)
-        if i >= args.warmup:
-            times.append(last["value"])
-            secs.append(last["seconds"])
-    value = statistics.mean(times)
-    from workloads import CONFIGS
-    cfg = CONFIGS[args.workload]
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(secs) * 1e3,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "H": cfg["H"], "dk": cfg["dk"], "dv": cfg["dv"], "chunk": 64},
-            "cpu_baseline": {"kind": last["kind"], "cores": last["cores"], "sample": last["sample"], "value": value,
-                             "unit": UNIT},
-            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
-    print(json.dumps(line))
-
-
-# --------------------------------------------------------------------------------------------------
-# Second workload: compact-to-semantic log-probability (Eqs. 17, 19), `--workload logp`
-# --------------------------------------------------------------------------------------------------
-LOGP_METRIC = "mapped log-prob fwd+bwd compact rows/s"
-LOGP_UNIT = "compact rows/s"
-LOGP_V = 157184            # vocabulary of the evaluated model
-LOGP_ROWS = 65536          # compact-row capacity of one microbatch
-
-
-def logp_forest(rank=0, capacity=LOGP_ROWS):
-    """Whole trees of cfg3, starting at a rank-dependent tree, while they fit the microbatch capacity.  A capacity
-    below the first tree's size (a small case for a profiler capture) gives copies of the cfg0b tree instead."""
-    from workloads import CONFIGS, make_forest
-    fo = config_forest_cached("cfg3")
-    base = fo.token_base()
-    first = (3 * rank) % fo.n_trees
-    trees, rows = [], 0
-    for t in list(range(first, fo.n_trees)) + list(range(first)):
-        c = int(base[fo.tree_node_ptr[t + 1]] - base[fo.tree_node_ptr[t]])
-        if rows + c > capacity:
-            break
-        trees.append(t)
-        rows += c
-    if not trees:
-        tree = CONFIGS["cfg0b"]["build"]()[0]
-        n = max(1, capacity // sum(tree[2]))
-        return make_forest([tree] * n), f"{n} x cfg0b"
-    return fo.subset(trees), f"cfg3 trees {trees}"
-
-
-def config_forest_cached(name):
-    from workloads import config_forest
-    return config_forest(name)
-
-
-def logp_oracle_sample(small=False, copies=1):
-    """The fp64 oracle of Eqs. 17/19 on small trees at the full vocabulary.  The full leg first times one cfg0b
-    tree, then sizes a forest of such trees to about 12 s of work and reports that run."""
-    from oracle import logp_oracle
-    from workloads import CONFIGS, make_forest, make_logits, make_logp_grad
-    # small: a 256-row tree (root 128, one child at its end, one forking at offset 100) for the many-step arm
-    tree = ([-1, 0, 0], [0, 128, 100], [128, 64, 64]) if small else CONFIGS["cfg0b"]["build"]()[0]
-    fo = make_forest([tree] * copies)
-    name = "three-node tree" if small else f"{copies} x cfg0b tree"
-    data = make_logits(fo.n_tokens, LOGP_V, "bf16", 0)
-    m, y, _ = logp_oracle.positions(fo, data["token_id"].numpy())
-    g = make_logp_grad(len(m), 0, keep=1.0).double().numpy()
-    z = data["z"].double().numpy()
-    t0 = time.perf_counter()
-    logp_oracle.mapped_logp(z, m, y)
-    logp_oracle.mapped_logp_grad(z, m, y, g)
-    dt = time.perf_counter() - t0
-    if not small and copies == 1 and dt < 8.0:
-        return logp_oracle_sample(False, copies=int(min(8, max(2, round(12.0 / dt)))))
-    return {"value": fo.n_tokens / dt, "unit": LOGP_UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"{name}: {fo.n_tokens} compact rows, {len(m)} positions, V={LOGP_V}, fwd+bwd, {dt:.1f} s",
-            "seconds": dt}
-
-
-def run_logp_reference(args):
-    if int(os.environ.get("RANK", "0")) != 0:
-        return
-    vals, secs, last = [], [], None
-    for i in range(args.warmup + args.steps):
-        last = logp_oracle_sample(small=True)
-        if i >= args.warmup:
-            vals.append(last["value"])
-            secs.append(last["seconds"])
-    value = statistics.mean(vals)
-    print(json.dumps({
-        "impl": "reference", "metric": LOGP_METRIC, "value": value, "unit": LOGP_UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(secs) * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "logp", "V": LOGP_V},
-        "cpu_baseline": {"kind": last["kind"], "cores": last["cores"], "sample": last["sample"], "value": value,
-                         "unit": LOGP_UNIT},
-        "e2e": {"value": value, "unit": LOGP_UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
-
-
-# --------------------------------------------------------------------------------------------------
-def max_over_ranks(values, device):
-    """Element-wise maximum of a few per-rank timings over all ranks (identity when not distributed)."""
-    import torch
-    import torch.distributed as dist
-    t = torch.tensor(list(values), dtype=torch.float64, device=device)
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return [float(x) for x in t]
 
 
 def trajectory_wise_ms(H, fo, cfg, inp, flags, trees_per_batch=4):
@@ -338,389 +381,290 @@ def per_config_table(args):
               file=sys.stderr)
 
 
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
+class LaWorkload:
+    """The hot path: one step = every forward round, every backward round and the replay-gradient fold of a
+    configuration (default cfg3)."""
+    metric, unit = METRIC, UNIT
 
-    import paper_2608_28158_b200 as H
-    from workloads import CONFIGS, config_forest, make_inputs
+    def __init__(self, args, ranks):
+        import torch
+        import paper_2608_28158_b200 as H
+        from workloads import CONFIGS, config_forest, make_inputs
+        self.H, self.args, self.ranks = H, args, ranks
+        self.cfg = cfg = CONFIGS[args.workload]
+        self.fo = fo = config_forest(args.workload)
+        t_plans = []
+        for _ in range(3):                                 # host planning time: median of three calls
+            t0 = time.perf_counter()
+            plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, cfg["chunk"])
+            t_plans.append(time.perf_counter() - t0)
+        self.t_plan = statistics.median(t_plans)
+        self.plan = plan.upload()
+        Hh, dk, dv = cfg["H"], cfg["dk"], cfg["dv"]
+        # every rank draws its own tensors (independent batches of the same shape)
+        self.inp = inp = make_inputs(plan.C, Hh, dk, dv, cfg["dtype"], cfg["seed"] + 100 * ranks.rank, device="cuda")
+        self.flags = H.HARTS_FLAG_FMA_KERNELS if args.fma else 0
+        self.ws = H.Workspace(plan, Hh, dk, dv, inp["q"].dtype, self.flags)
+        self.out = {"o": torch.empty_like(inp["v"]), "dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]),
+                    "dv": torch.empty_like(inp["v"]), "dg": torch.empty_like(inp["g"])}
+        self.units = plan.C
+        self.stream = torch.cuda.current_stream()
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    def step(self, marks):
+        import torch
+        H, plan, inp, out, ws, stream = self.H, self.plan, self.inp, self.out, self.ws, self.stream
+        ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+        K = plan.n_rounds
 
-    cfg = CONFIGS[args.workload]
-    fo = config_forest(args.workload)
-    t_plans = []
-    for _ in range(3):                                 # host planning time: median of three calls
-        t0 = time.perf_counter()
-        plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, cfg["chunk"])
-        t_plans.append(time.perf_counter() - t0)
-    t_plan = statistics.median(t_plans)
-    plan.upload()
-    Hh, dk, dv = cfg["H"], cfg["dk"], cfg["dv"]
-    # every rank draws its own tensors (independent batches of the same shape)
-    inp = make_inputs(plan.C, Hh, dk, dv, cfg["dtype"], cfg["seed"] + 100 * rank, device="cuda")
-    flags = H.HARTS_FLAG_FMA_KERNELS if args.fma else 0
-    ws = H.Workspace(plan, Hh, dk, dv, inp["q"].dtype, flags)
-    out = {"o": torch.empty_like(inp["v"]), "dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]),
-           "dv": torch.empty_like(inp["v"]), "dg": torch.empty_like(inp["g"])}
-    elem = inp["q"].element_size()
-    in_bytes = sum(x.numel() * x.element_size() for x in inp.values())
-    out_bytes = sum(x.numel() * x.element_size() for x in out.values())
-    stream = torch.cuda.current_stream()
-    K = plan.n_rounds
+        def timed(name, call):
+            if marks is None:
+                call()
+                return
+            a, b = ev(), ev()
+            a.record(stream)
+            call()
+            b.record(stream)
+            marks.append((name, a, b))
 
-    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
-    launch_times = {"fwd": [], "bwd": [], "fold": []}
-
-    def step(record):
-        marks = []
         for r in range(1, K + 1):
-            a, b = ev(), ev()
-            a.record(stream)
-            H.harts_la_fwd(plan, r, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], ws.slots, ws.chunk_states,
-                           flags, ws.dev_status)
-            b.record(stream)
-            marks.append(("fwd", a, b))
+            timed("fwd", lambda: H.harts_la_fwd(plan, r, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], ws.slots,
+                                               ws.chunk_states, self.flags, ws.dev_status))
         for r in range(K, 0, -1):
-            a, b = ev(), ev()
-            a.record(stream)
-            H.harts_la_bwd_seqs(plan.tables, int(plan.round_seq_ptr[r - 1]), int(plan.round_seq_ptr[r]), inp["q"],
-                                inp["k"], inp["v"], inp["g"], inp["dO"], out["dq"], out["dk"], out["dv"], out["dg"],
-                                ws.chunk_states, ws.scratch, flags, ws.dev_status)
-            b.record(stream)
-            marks.append(("bwd", a, b))
-        a, b = ev(), ev()
-        a.record(stream)
-        H.harts_la_bwd_finish(plan.tables, out["dk"], out["dv"], out["dg"], ws.scratch)
-        b.record(stream)
-        marks.append(("fold", a, b))
-        if record:
-            return marks
-        return None
+            timed("bwd", lambda: H.harts_la_bwd_seqs(plan.tables, int(plan.round_seq_ptr[r - 1]),
+                                                    int(plan.round_seq_ptr[r]), inp["q"], inp["k"], inp["v"], inp["g"],
+                                                    inp["dO"], out["dq"], out["dk"], out["dv"], out["dg"],
+                                                    ws.chunk_states, ws.scratch, self.flags, ws.dev_status))
+        timed("fold", lambda: H.harts_la_bwd_finish(plan.tables, out["dk"], out["dv"], out["dg"], ws.scratch))
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    def check(self):
+        self.H.harts_la_check(self.ws.dev_status)
 
-    all_marks = []
-    t_begin, t_end = ev(), ev()
-    with ClockSampler(local) as clocks:            # started before the warm-up so that it is sampling by then
-        for _ in range(args.warmup):
-            step(False)
-        H.harts_la_check(ws.dev_status)
-        # a short region gives the 50 ms sampler nothing to see: keep the GPU under the same load a little longer
-        # before the timed steps when the whole region is under a second
-        barrier()
-        t_host0 = clocks.mark()
-        t_begin.record(stream)
-        for _ in range(args.steps):
-            all_marks.append(step(True))
-        t_end.record(stream)
-        barrier()
-        t_host1 = clocks.mark()
-    ms_total = t_begin.elapsed_time(t_end)
-    H.harts_la_check(ws.dev_status)
-    for marks in all_marks:
-        for kind, a, b in marks:
-            launch_times[kind].append(a.elapsed_time(b))
-
-    # ---- end to end through host buffers -----------------------------------------------------------
-    e2e = None
-    if not args.no_e2e:
-        pinned = True
-        try:
-            host_in = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in inp.items()}
-            host_out = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in out.items()}
-        except RuntimeError:
-            pinned = False
-            host_in = {n: torch.empty(x.shape, dtype=x.dtype) for n, x in inp.items()}
-            host_out = {n: torch.empty(x.shape, dtype=x.dtype) for n, x in out.items()}
-        for n in inp:
-            host_in[n].copy_(inp[n])
-        torch.cuda.synchronize()
-        e2e_steps = max(1, min(args.steps, args.e2e_steps))
-        H.run_fwd_bwd_host(plan, ws, host_in, inp, out, host_out)       # warm-up; also the unpipelined reference
-        barrier()
+    def e2e(self, n_steps):
+        """Through host buffers, pipelined: the copies of neighbouring steps overlap the kernels (three streams, two
+        device buffer sets); every step still moves all of its inputs in and all of its results out."""
+        import torch
+        H, plan, ws, inp, out, ranks = self.H, self.plan, self.ws, self.inp, self.out, self.ranks
+        host_in, host_out = host_copies(inp), host_copies(out)
+        stream = torch.cuda.current_stream()
+        ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+        H.run_fwd_bwd_host(plan, ws, host_in, inp, out, host_out)       # warm-up; then the unpipelined reference
+        ranks.barrier()
         a, b = ev(), ev()
         a.record(stream)
         H.run_fwd_bwd_host(plan, ws, host_in, inp, out, host_out)
         b.record(stream)
-        barrier()
+        ranks.barrier()
         serial_ms = a.elapsed_time(b)
-        # pipelined: the copies of neighbouring steps overlap (three streams, two device buffer sets); every step
-        # still moves all of its inputs in and all of its results out
         pipe = H.HostPipeline(plan, ws, inp, out)
         pipe.step(host_in, host_out)                                    # warm-up of the streams
         pipe.finish()
-        barrier()
-        t0 = time.perf_counter()
+        ranks.barrier()
         a, b = ev(), ev()
         a.record(pipe.s_in)
-        for _ in range(e2e_steps):
+        for _ in range(n_steps):
             pipe.step(host_in, host_out)
         b.record(pipe.s_out)
         pipe.finish()
-        barrier()
-        e2e_ms = a.elapsed_time(b) / e2e_steps
-        e2e = {"ms_per_step": e2e_ms, "steps": e2e_steps, "pinned": pinned, "serial_ms_per_step": serial_ms,
-               "wall_ms_per_step": (time.perf_counter() - t0) * 1e3 / e2e_steps}
-        del pipe
-        del host_in, host_out
+        ranks.barrier()
+        nbytes = lambda d: sum(t.numel() * t.element_size() for t in d.values())  # noqa: E731
+        return {"ms": a.elapsed_time(b) / n_steps, "steps": n_steps, "h2d": nbytes(host_in), "d2h": nbytes(host_out),
+                "extra": {"overlap": "copies of neighbouring steps overlap the kernels (3 streams, 2 device buffer sets)",
+                          "unpipelined_value": plan.C * ranks.world / (serial_ms * 1e-3)}}
 
-    # ---- the same kernels, trajectory-wise (Section 5 baseline) ---------------------------------------------
-    traj = None
-    if world == 1 and not args.no_trajwise:
-        # inputs are in physical order here; the expansion wants canonical order
-        rows = torch.as_tensor(plan.row_of_token.astype(np.int64), device="cuda")
-        canon = {n: x[rows] for n, x in inp.items()}
-        t_ms, t_rows = trajectory_wise_ms(H, fo, cfg, canon, flags)
-        traj = {"ms": t_ms, "rows": t_rows}
-        del canon
+    def describe(self, ms_step, kernel_ms, peaks):
+        plan, cfg, args = self.plan, self.cfg, self.args
+        Hh, dk, dv = cfg["H"], cfg["dk"], cfg["dv"]
+        elem = self.inp["q"].element_size()
+        K = plan.n_rounds
+        th = plan.C * Hh                                  # token-heads per rank and step
+        # algorithmic (compulsory) bytes per token-head: fwd reads q,k,v,g and writes o; bwd reads q,k,v,dO,g and
+        # writes dq,dk,dv,dg
+        fwd_bytes = th * ((2 * dk + 2 * dv) * elem + 4)
+        bwd_bytes = th * ((4 * dk + 3 * dv) * elem + 8)
+        flops_fwd = th * (2 * 64 * dk + 2 * 64 * dv + 4 * dk * dv)
+        flops_bwd = th * (5 * 2 * 64 * (dk + dv) // 2 + 4 * 2 * dk * dv)
+        in_bytes = sum(x.numel() * x.element_size() for x in self.inp.values())
+        tc = dk == 128 and not args.fma and elem == 2
+        rec = measured_traffic("tc_bwd_kernel") if tc else None
+        traffic = rec["dram_bytes_per_unit"] * th / K if rec else None
+        t_bytes = (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9)
+        t_flops = (flops_fwd + flops_bwd) / (peaks["bf16_tflops_sustained"] * 1e12)
+        # method traffic on top of the compulsory bytes: replayed rows (k, v, g read in both passes, gradient
+        # contributions written and folded), state hand-offs (initial state read + its gradient written, slot written
+        # + consumers' gradients read), chunk states (written by the forward, read by the backward, 2 B per element)
+        n_side = int((plan.seq_init_slot >= 0).sum())
+        method_bytes = (fwd_bytes + bwd_bytes + plan.R * Hh * (6 * dk * elem + 12)
+                        + (n_side + plan.n_slots) * Hh * dk * dv * 4 * 2 + plan.n_chunks * Hh * dk * dv * 2 * 2)
+        roof = hbm_roofline(
+            "backward packed call (all rounds)", bwd_bytes / K, kernel_ms["bwd"] / K, peaks, traffic,
+            traffic_note=(f"bytes per launch (mean over the rounds): {rec['dram_bytes_per_unit']:.0f} B per token-head "
+                          f"from the ncu capture on {rec['workload']} at commit {rec['commit']}, scaled by token-heads"
+                          if rec else "no capture of the current kernel sources on record"),
+            forward={"achieved": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9,
+                     "frac": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            whole_path={"roof_ms": max(t_bytes, t_flops) * 1e3, "frac_strict": max(t_bytes, t_flops) * 1e3 / ms_step,
+                        "frac_strict_nominal": max((fwd_bytes + bwd_bytes) / 8e12,
+                                                   (flops_fwd + flops_bwd) / 2.25e15) * 1e3 / ms_step,
+                        "frac_method": max(method_bytes / (peaks["hbm_gbs"] * 1e9), t_flops) * 1e3 / ms_step})
+        return {
+            "dtype": cfg["dtype"] if cfg["dtype"] != "fp32" else "f32",
+            "config": {"workload": args.workload, "H": Hh, "dk": dk, "dv": dv, "chunk": cfg["chunk"],
+                       "compact_tokens": plan.C, "replay_rows": plan.R, "rounds": plan.n_rounds,
+                       "sequences": plan.n_seq, "slots": plan.n_slots, "chunks": plan.n_chunks,
+                       "l2": f"inputs larger than L2 ({in_bytes / 2**30:.2f} GiB read per step)"
+                             if in_bytes > 2 * L2_BYTES else "inputs smaller than L2: no flush (small workload)",
+                       "kernels": "fma" if args.fma or cfg["dtype"] == "fp32" else "default",
+                       "plan_ms": self.t_plan * 1e3},
+            "roofline": roof,
+            # per step: K forward calls, K backward calls each preceded by the hand-off reduction when the plan has
+            # exported boundaries, and the replay-gradient fold
+            "gpu_launches_per_step": 2 * K + (K if plan.n_slots else 0) + (1 if plan.n_rg_rows else 0)}
 
-    # ---- reduce over ranks ------------------------------------------------------------------------
-    ms_step = ms_total / args.steps
-    if world > 1:
-        ms_step, e2e_ms_max = max_over_ranks([ms_step, e2e["ms_per_step"] if e2e else 0.0], "cuda")
-        if e2e:
-            e2e["ms_per_step"] = e2e_ms_max
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+    def extras(self, ms_step):
+        """The same kernels, trajectory-wise (the conventional baseline of Section 5); one GPU only."""
+        import torch
+        if self.ranks.world > 1 or self.args.no_trajwise:
+            return {}
+        rows = torch.as_tensor(self.plan.row_of_token.astype(np.int64), device="cuda")
+        canon = {n: x[rows] for n, x in self.inp.items()}      # the expansion wants canonical order
+        t_ms, t_rows = trajectory_wise_ms(self.H, self.fo, self.cfg, canon, self.flags)
+        return {"trajectory_wise": {
+            "ms": t_ms, "rows": t_rows, "rows_ratio": t_rows / self.plan.C, "speedup": t_ms / ms_step,
+            "speedup_with_plan": t_ms / (ms_step + self.t_plan * 1e3),
+            "paper_context": "4.81-4.87x F/B/Grad on a whole hybrid MoE model, 8x H20-3e (Table 4)"}}
 
-    peaks = measured_peaks()
-    tokens = plan.C * world
-    value = tokens / (ms_step * 1e-3)
-    th = plan.C * Hh                                  # token-heads per rank and step
-    # algorithmic (compulsory) bytes per token-head: fwd reads q,k,v,g and writes o; bwd reads q,k,v,dO,g
-    # and writes dq,dk,dv,dg
-    fwd_bytes = th * ((2 * dk + 2 * dv) * elem + 4)
-    bwd_bytes = th * ((4 * dk + 3 * dv) * elem + 8)
-    flops_fwd = th * (2 * 64 * dk + 2 * 64 * dv + 4 * dk * dv)
-    flops_bwd = th * (5 * 2 * 64 * (dk + dv) // 2 + 4 * 2 * dk * dv)
-    bwd_ms = sum(launch_times["bwd"]) / args.steps
-    fwd_ms = sum(launch_times["fwd"]) / args.steps
-    fold_ms = sum(launch_times["fold"]) / args.steps
-    hbm_peak = peaks["hbm_gbs"]
-    achieved = bwd_bytes / (bwd_ms * 1e-3) / 1e9
-    # DRAM bytes per token-head of the backward kernel from the ncu capture on cfg2 (profiles/
-    # tc_bwd_kernel_cfg2_ncu_full.md), scaled to this workload's token-heads; traffic grows in proportion to them
-    BWD_DRAM_BYTES_PER_TOKEN_HEAD = 2356.0
-    bwd_traffic_per_launch = (BWD_DRAM_BYTES_PER_TOKEN_HEAD * th / K) if (dk == 128 and not args.fma and elem == 2) \
-        else None
-    t_roof_bytes = (fwd_bytes + bwd_bytes) / (hbm_peak * 1e9)
-    t_roof_flops = (flops_fwd + flops_bwd) / (peaks["bf16_tflops_sustained"] * 1e12)
-    clock = clocks.summary(t_host0, t_host1)
-    if not clock["samples"]:
-        clock = clocks.summary()
-        clock["note"] = "timed region shorter than the sampling period: samples cover warm-up + timed region"
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": cfg["dtype"] if cfg["dtype"] != "fp32" else "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "H": Hh, "dk": dk, "dv": dv, "chunk": cfg["chunk"],
-                   "compact_tokens": plan.C, "replay_rows": plan.R, "rounds": plan.n_rounds,
-                   "sequences": plan.n_seq, "slots": plan.n_slots, "chunks": plan.n_chunks,
-                   "l2": f"inputs larger than L2 ({in_bytes / 2**30:.2f} GiB read per step)"
-                         if in_bytes > 2 * L2_BYTES else "inputs smaller than L2: no flush (small workload)",
-                   "kernels": "fma" if args.fma or cfg["dtype"] == "fp32" else "default",
-                   "plan_ms": t_plan * 1e3},
-        "roofline": {"bound": "hbm", "kernel": "backward packed call (all rounds)", "achieved": achieved,
-                     "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak, "traffic": bwd_traffic_per_launch,
-                     "traffic_note": "bytes per launch (mean over the rounds), scaled from the ncu capture on cfg2",
-                     "algorithmic_bytes_per_launch": bwd_bytes / K,
-                     "peak_source": peaks["source"],
-                     "whole_path": {"roof_ms": max(t_roof_bytes, t_roof_flops) * 1e3,
-                                    "frac_strict": max(t_roof_bytes, t_roof_flops) * 1e3 / ms_step,
-                                    "frac_strict_nominal": max((fwd_bytes + bwd_bytes) / 8e12,
-                                                               (flops_fwd + flops_bwd) / 2.25e15) * 1e3 / ms_step}},
-        "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms, "fold": fold_ms},
-        # per step: K forward calls, K backward calls each preceded by the hand-off reduction when the plan has
-        # exported boundaries, and the replay-gradient fold
-        "gpu_launches": (2 * K + (K if plan.n_slots else 0) + (1 if plan.n_rg_rows else 0)) * args.steps,
-        "clocks": clock,
-    }
-    if e2e:
-        line["e2e"] = {"value": tokens / (e2e["ms_per_step"] * 1e-3), "unit": UNIT,
-                       "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out_bytes, "steps": e2e["steps"],
-                       "pinned_host_memory": e2e["pinned"],
-                       "overlap": "copies of neighbouring steps overlap the kernels (3 streams, 2 device buffer sets)",
-                       "unpipelined_value": tokens / (e2e["serial_ms_per_step"] * 1e-3)}
-    # method traffic on top of the compulsory bytes: replayed rows (k, v, g read in both passes, gradient
-    # contributions written and folded), state hand-offs (initial state read + its gradient written, slot written +
-    # consumers' gradients read), chunk states (written by the forward, read by the backward, 2 B per element)
-    n_side = int((plan.seq_init_slot >= 0).sum())
-    method_bytes = (fwd_bytes + bwd_bytes + plan.R * Hh * (6 * dk * elem + 12)
-                    + (n_side + plan.n_slots) * Hh * dk * dv * 4 * 2 + plan.n_chunks * Hh * dk * dv * 2 * 2)
-    line["roofline"]["whole_path"]["frac_method"] = max(method_bytes / (hbm_peak * 1e9), t_roof_flops) * 1e3 / ms_step
-    if traj:
-        line["trajectory_wise"] = {"ms": traj["ms"], "rows": traj["rows"], "rows_ratio": traj["rows"] / plan.C,
-                                   "speedup": traj["ms"] / ms_step,
-                                   "speedup_with_plan": traj["ms"] / (ms_step + t_plan * 1e3),
-                                   "paper_context": "4.81-4.87x F/B/Grad on a whole hybrid MoE model, 8x H20-3e (Table 4)"}
-    if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = oracle_sample(args.workload)
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
-    elif args.per_config:
-        del inp, out, ws
-        torch.cuda.empty_cache()
-        per_config_table(args)
+    def cpu_baseline(self):
+        return oracle_sample(self.args.workload)
+
+    def reference_sample(self, hint):
+        return oracle_sample(self.args.workload, seconds_hint=hint)
+# --------------------------------------------------------------------------------------------------
+# Second workload: compact-to-semantic log-probability (Eqs. 17, 19), `--workload logp`
+# --------------------------------------------------------------------------------------------------
+LOGP_METRIC = "mapped log-prob fwd+bwd compact rows/s"
+LOGP_UNIT = "compact rows/s"
+LOGP_V = 157184            # vocabulary of the evaluated model
+LOGP_ROWS = 65536          # compact-row capacity of one microbatch
 
 
-def run_logp(args):
-    """One step = forward (row max / sum-exp over V, lambda for every position) + backward (dz for every compact row)."""
-    import torch
-    import torch.distributed as dist
+def logp_forest(rank=0, capacity=LOGP_ROWS):
+    """Whole trees of cfg3, starting at a rank-dependent tree, while they fit the microbatch capacity.  A capacity
+    below the first tree's size (a small case for a profiler capture) gives copies of the cfg0b tree instead."""
+    from workloads import CONFIGS, make_forest
+    fo = config_forest_cached("cfg3")
+    base = fo.token_base()
+    first = (3 * rank) % fo.n_trees
+    trees, rows = [], 0
+    for t in list(range(first, fo.n_trees)) + list(range(first)):
+        c = int(base[fo.tree_node_ptr[t + 1]] - base[fo.tree_node_ptr[t]])
+        if rows + c > capacity:
+            break
+        trees.append(t)
+        rows += c
+    if not trees:
+        tree = CONFIGS["cfg0b"]["build"]()[0]
+        n = max(1, capacity // sum(tree[2]))
+        return make_forest([tree] * n), f"{n} x cfg0b"
+    return fo.subset(trees), f"cfg3 trees {trees}"
 
-    import paper_2608_28158_b200 as H
-    from workloads import make_logits, make_logp_grad
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    fo, trees = logp_forest(rank, args.logp_rows)
-    C, V = fo.n_tokens, LOGP_V
-    plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
-    data = make_logits(C, V, "bf16", 50 + rank, device="cuda")
+def config_forest_cached(name):
+    from workloads import config_forest
+    return config_forest(name)
+
+
+def logp_oracle_sample(small=False, copies=1):
+    """The fp64 oracle of Eqs. 17/19 on small trees at the full vocabulary.  The full leg first times one cfg0b
+    tree, then sizes a forest of such trees to about 12 s of work and reports that run."""
+    from oracle import logp_oracle
+    from workloads import CONFIGS, make_forest, make_logits, make_logp_grad
+    # small: a 256-row tree (root 128, one child at its end, one forking at offset 100) for the many-step arm
+    tree = ([-1, 0, 0], [0, 128, 100], [128, 64, 64]) if small else CONFIGS["cfg0b"]["build"]()[0]
+    fo = make_forest([tree] * copies)
+    name = "three-node tree" if small else f"{copies} x cfg0b tree"
+    data = make_logits(fo.n_tokens, LOGP_V, "bf16", 0)
+    m, y, _ = logp_oracle.positions(fo, data["token_id"].numpy())
+    g = make_logp_grad(len(m), 0, keep=1.0).double().numpy()
+    z = data["z"].double().numpy()
     t0 = time.perf_counter()
-    m, y, _ = H.harts_logp_positions(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len,
-                                     data["token_id"].cpu().numpy(), plan.row_of_token)
-    ptr, pos = H.harts_logp_csr(C, m)
-    t_host = time.perf_counter() - t0
-    P = len(m)
-    z = data["z"]
-    dev = {"m": torch.as_tensor(m).cuda(), "y": torch.as_tensor(y).cuda(), "ptr": torch.as_tensor(ptr).cuda(),
-           "pos": torch.as_tensor(pos).cuda(), "g": make_logp_grad(P, 50 + rank, device="cuda", keep=1.0)}
-    lse = torch.empty(C, device="cuda")
-    lam = torch.empty(P, device="cuda")
-    dz = torch.empty_like(z)
-    status = torch.zeros(2, dtype=torch.int32, device="cuda")
-    stream = torch.cuda.current_stream()
-    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+    logp_oracle.mapped_logp(z, m, y)
+    logp_oracle.mapped_logp_grad(z, m, y, g)
+    dt = time.perf_counter() - t0
+    if not small and copies == 1 and dt < 8.0:
+        return logp_oracle_sample(False, copies=int(min(8, max(2, round(12.0 / dt)))))
+    return {"value": fo.n_tokens / dt, "unit": LOGP_UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{name}: {fo.n_tokens} compact rows, {len(m)} positions, V={LOGP_V}, fwd+bwd, {dt:.1f} s",
+            "seconds": dt}
 
-    def step(marks=None):
-        a, b, c = ev(), ev(), ev()
-        a.record(stream)
-        H.harts_logp_fwd(z, dev["m"], dev["y"], lse, lam, dev_status=status)
-        b.record(stream)
-        H.harts_logp_bwd(z, dev["y"], dev["ptr"], dev["pos"], lse, dev["g"], dz, dev_status=status)
-        c.record(stream)
+
+class LogpWorkload:
+    """One step = forward (row max / sum-exp over V, lambda for every position) + backward (dz for every compact row)."""
+    metric, unit = LOGP_METRIC, LOGP_UNIT
+
+    def __init__(self, args, ranks):
+        import torch
+        import paper_2608_28158_b200 as H
+        from workloads import make_logits, make_logp_grad
+        self.H, self.args, self.ranks = H, args, ranks
+        fo, self.trees = logp_forest(ranks.rank, args.logp_rows)
+        self.C, self.V = C, V = fo.n_tokens, LOGP_V
+        plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
+        data = make_logits(C, V, "bf16", 50 + ranks.rank, device="cuda")
+        t0 = time.perf_counter()
+        m, y, _ = H.harts_logp_positions(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len,
+                                         data["token_id"].cpu().numpy(), plan.row_of_token)
+        ptr, pos = H.harts_logp_csr(C, m)
+        self.t_host = time.perf_counter() - t0
+        self.P = P = len(m)
+        self.z = data["z"]
+        self.dev = {"m": torch.as_tensor(m).cuda(), "y": torch.as_tensor(y).cuda(), "ptr": torch.as_tensor(ptr).cuda(),
+                    "pos": torch.as_tensor(pos).cuda(), "g": make_logp_grad(P, 50 + ranks.rank, device="cuda", keep=1.0)}
+        self.lse, self.lam, self.dz = torch.empty(C, device="cuda"), torch.empty(P, device="cuda"), torch.empty_like(self.z)
+        self.status = torch.zeros(2, dtype=torch.int32, device="cuda")
+        self.units = C
+        self.stream = torch.cuda.current_stream()
+
+    def step(self, marks):
+        import torch
+        H, dev = self.H, self.dev
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        a.record(self.stream)
+        H.harts_logp_fwd(self.z, dev["m"], dev["y"], self.lse, self.lam, dev_status=self.status)
+        b.record(self.stream)
+        H.harts_logp_bwd(self.z, dev["y"], dev["ptr"], dev["pos"], self.lse, dev["g"], self.dz, dev_status=self.status)
+        c.record(self.stream)
         if marks is not None:
-            marks.append((a, b, c))
+            marks += [("fwd", a, b), ("bwd", b, c)]
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    def check(self):
+        self.H.harts_la_check(self.status)
 
-    marks = []
-    t_begin, t_end = ev(), ev()
-    with ClockSampler(local) as clocks:
-        for _ in range(args.warmup):
-            step()
-        H.harts_la_check(status)
-        barrier()
-        h0 = clocks.mark()
-        t_begin.record(stream)
-        for _ in range(args.steps):
-            step(marks)
-        t_end.record(stream)
-        barrier()
-        h1 = clocks.mark()
-    H.harts_la_check(status)
-    ms_step = t_begin.elapsed_time(t_end) / args.steps
-    fwd_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in marks)
-    bwd_ms = statistics.mean(b.elapsed_time(c) for _, b, c in marks)
+    def e2e(self, n_steps):
+        dev_in = dict(self.dev, z=self.z)
+        return time_e2e(self, dev_in, {"lam": self.lam, "dz": self.dz}, n_steps, self.ranks)
 
-    e2e = None
-    if not args.no_e2e:
-        small = {n: x for n, x in dev.items()}
-        host_in = {"z": torch.empty(z.shape, dtype=z.dtype, pin_memory=True)}
-        host_in.update({n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in small.items()})
-        host_out = {"lam": torch.empty(P, pin_memory=True), "dz": torch.empty(z.shape, dtype=z.dtype, pin_memory=True)}
-        host_in["z"].copy_(z)
-        for n, x in small.items():
-            host_in[n].copy_(x)
-        torch.cuda.synchronize()
+    def describe(self, ms_step, kernel_ms, peaks):
+        C, V, P = self.C, self.V, self.P
+        row_bytes = V * self.z.element_size()
+        fwd_bytes = C * row_bytes + P * 12 + C * 4              # z once; m, y read and lambda written; lse written
+        bwd_bytes = 2 * C * row_bytes + P * 12 + C * 12         # z read, dz written; y, g, row_pos; lse, row_pos_ptr
+        roof_ms = (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3
+        return {"dtype": "bf16",
+                "config": {"workload": "logp", "V": V, "compact_rows": C, "positions": P, "trees": self.trees,
+                           "action_mask": "every position selected (no idle rows)",
+                           "l2": f"inputs larger than L2 ({C * row_bytes / 2**30:.2f} GiB of logits)",
+                           "host_index_ms": self.t_host * 1e3},
+                "roofline": hbm_roofline("dz_kernel (backward)", bwd_bytes, kernel_ms["bwd"], peaks, None,
+                                         forward={"achieved": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9,
+                                                  "frac": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                                         whole_path={"roof_ms": roof_ms, "frac_strict": roof_ms / ms_step}),
+                "gpu_launches_per_step": 3}
 
-        def e2e_step():
-            z.copy_(host_in["z"], non_blocking=True)
-            for n, x in small.items():
-                x.copy_(host_in[n], non_blocking=True)
-            step()
-            host_out["lam"].copy_(lam, non_blocking=True)
-            host_out["dz"].copy_(dz, non_blocking=True)
+    def extras(self, ms_step):
+        return {}
 
-        e2e_step()
-        barrier()
-        a, b = ev(), ev()
-        n_e2e = max(1, min(args.steps, args.e2e_steps))
-        a.record(stream)
-        for _ in range(n_e2e):
-            e2e_step()
-        b.record(stream)
-        barrier()
-        e2e = {"ms": a.elapsed_time(b) / n_e2e, "steps": n_e2e,
-               "h2d": sum(x.numel() * x.element_size() for x in host_in.values()),
-               "d2h": sum(x.numel() * x.element_size() for x in host_out.values())}
-        del host_in, host_out
-
-    if world > 1:
-        ms_step, e2e_ms = max_over_ranks([ms_step, e2e["ms"] if e2e else 0.0], "cuda")
-        if e2e:
-            e2e["ms"] = e2e_ms
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-    peaks = measured_peaks()
-    row_bytes = V * z.element_size()
-    fwd_bytes = C * row_bytes + P * 12 + C * 4              # z once; m, y read and lambda written; lse written
-    bwd_bytes = 2 * C * row_bytes + P * 12 + C * 12         # z read, dz written; y, g, row_pos; lse, row_pos_ptr
-    achieved = bwd_bytes / (bwd_ms * 1e-3) / 1e9
-    clock = clocks.summary(h0, h1)
-    if not clock["samples"]:
-        clock = clocks.summary()
-    line = {
-        "metric": LOGP_METRIC, "value": C * world / (ms_step * 1e-3), "unit": LOGP_UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "logp", "V": V, "compact_rows": C, "positions": P, "trees": trees,
-                   "action_mask": "every position selected (no idle rows)",
-                   "l2": f"inputs larger than L2 ({C * row_bytes / 2**30:.2f} GiB of logits)",
-                   "host_index_ms": t_host * 1e3},
-        "roofline": {"bound": "hbm", "kernel": "dz_kernel (backward)", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
-                     "algorithmic_bytes_per_launch": bwd_bytes, "peak_source": peaks["source"],
-                     "forward": {"achieved": fwd_bytes / (fwd_ms * 1e-3) / 1e9,
-                                 "frac": fwd_bytes / (fwd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
-                     "whole_path": {"roof_ms": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3,
-                                    "frac_strict": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms_step}},
-        "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms},
-        "gpu_launches": 3 * args.steps,
-        "clocks": clock,
-    }
-    if e2e:
-        line["e2e"] = {"value": C * world / (e2e["ms"] * 1e-3), "unit": LOGP_UNIT, "h2d_bytes_per_step": e2e["h2d"],
-                       "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"], "pinned_host_memory": True}
-    if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = logp_oracle_sample()
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
-
-
+    def cpu_baseline(self):
+        return logp_oracle_sample()
 # --------------------------------------------------------------------------------------------------
 # Third workload: tree-aware causal convolution before the linear-attention core (Section 4.2), `--workload conv`
 # --------------------------------------------------------------------------------------------------
@@ -745,159 +689,72 @@ def conv_oracle_sample(small=False):
             "seconds": dt}
 
 
-def run_conv_reference(args):
-    if int(os.environ.get("RANK", "0")) != 0:
-        return
-    vals, secs, last = [], [], None
-    for i in range(args.warmup + args.steps):
-        last = conv_oracle_sample(small=True)
-        if i >= args.warmup:
-            vals.append(last["value"])
-            secs.append(last["seconds"])
-    value = statistics.mean(vals)
-    print(json.dumps({
-        "impl": "reference", "metric": CONV_METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(secs) * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "conv", "D": 4096, "w": CONV_W},
-        "cpu_baseline": {"kind": last["kind"], "cores": last["cores"], "sample": last["sample"], "value": value,
-                         "unit": UNIT},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
-
-
-def run_conv(args):
+class ConvWorkload:
     """One step = forward + backward (dx, dW) of the width-4 depthwise convolution over cfg3's compact tokens,
     D = 32 heads x 128 = 4096 channels (the q/k/v projections each see one such call)."""
-    import torch
-    import torch.distributed as dist
+    metric, unit = CONV_METRIC, UNIT
 
-    import paper_2608_28158_b200 as H
-    from workloads import config_forest, make_conv_inputs
+    def __init__(self, args, ranks):
+        import torch
+        import paper_2608_28158_b200 as H
+        from workloads import config_forest, make_conv_inputs
+        self.H, self.args, self.ranks = H, args, ranks
+        fo = config_forest(args.conv_trees)
+        self.C, self.D, self.w = C, D, w = fo.n_tokens, 4096, CONV_W
+        plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
+        t0 = time.perf_counter()
+        prev, nxt, cptr, crow = H.harts_conv_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len,
+                                                   plan.row_of_token)
+        self.t_host = time.perf_counter() - t0
+        self.inp = make_conv_inputs(C, D, w, "bf16", 70 + ranks.rank, device="cuda")
+        self.idx = {n: torch.as_tensor(np.ascontiguousarray(a)).cuda() for n, a in
+                    (("prev", prev), ("next", nxt), ("cptr", cptr), ("crow", crow))}
+        self.y, self.dx = torch.empty_like(self.inp["x"]), torch.empty_like(self.inp["x"])
+        self.dW = torch.empty_like(self.inp["W"])
+        self.scratch = torch.empty(H.harts_conv_scratch_bytes(D, w), dtype=torch.uint8, device="cuda")
+        self.units = C
+        self.stream = torch.cuda.current_stream()
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    fo = config_forest(args.conv_trees)
-    C, D, w = fo.n_tokens, 4096, CONV_W
-    plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
-    t0 = time.perf_counter()
-    prev, nxt, cptr, crow = H.harts_conv_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len,
-                                               plan.row_of_token)
-    t_host = time.perf_counter() - t0
-    inp = make_conv_inputs(C, D, w, "bf16", 70 + rank, device="cuda")
-    idx = {n: torch.as_tensor(np.ascontiguousarray(a)).cuda() for n, a in
-           (("prev", prev), ("next", nxt), ("cptr", cptr), ("crow", crow))}
-    y, dx, dW = torch.empty_like(inp["x"]), torch.empty_like(inp["x"]), torch.empty_like(inp["W"])
-    scratch = torch.empty(H.harts_conv_scratch_bytes(D, w), dtype=torch.uint8, device="cuda")
-    stream = torch.cuda.current_stream()
-    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
-
-    def step(marks=None):
-        a, b, c = ev(), ev(), ev()
-        a.record(stream)
-        H.harts_conv_fwd(inp["x"], inp["W"], idx["prev"], y)
-        b.record(stream)
-        H.harts_conv_bwd(inp["x"], inp["W"], inp["dy"], idx["next"], idx["cptr"], idx["crow"], dx, dW, scratch)
-        c.record(stream)
+    def step(self, marks):
+        import torch
+        H, inp, idx = self.H, self.inp, self.idx
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        a.record(self.stream)
+        H.harts_conv_fwd(inp["x"], inp["W"], idx["prev"], self.y)
+        b.record(self.stream)
+        H.harts_conv_bwd(inp["x"], inp["W"], inp["dy"], idx["next"], idx["cptr"], idx["crow"], self.dx, self.dW,
+                         self.scratch)
+        c.record(self.stream)
         if marks is not None:
-            marks.append((a, b, c))
+            marks += [("fwd", a, b), ("bwd", b, c)]
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    def check(self):
+        pass
 
-    marks = []
-    t_begin, t_end = ev(), ev()
-    with ClockSampler(local) as clocks:
-        for _ in range(args.warmup):
-            step()
-        barrier()
-        h0 = clocks.mark()
-        t_begin.record(stream)
-        for _ in range(args.steps):
-            step(marks)
-        t_end.record(stream)
-        barrier()
-        h1 = clocks.mark()
-    ms_step = t_begin.elapsed_time(t_end) / args.steps
-    fwd_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in marks)
-    bwd_ms = statistics.mean(b.elapsed_time(c) for _, b, c in marks)
-    e2e = None
-    if not args.no_e2e:
-        host = {n: torch.empty(inp[n].shape, dtype=inp[n].dtype, pin_memory=True) for n in ("x", "dy", "W")}
-        for n in host:
-            host[n].copy_(inp[n])
-        out_h = {"y": torch.empty(y.shape, dtype=y.dtype, pin_memory=True),
-                 "dx": torch.empty(y.shape, dtype=y.dtype, pin_memory=True), "dW": torch.empty(dW.shape, pin_memory=True)}
-        torch.cuda.synchronize()
+    def e2e(self, n_steps):
+        dev_in = {n: self.inp[n] for n in ("x", "dy", "W")}
+        return time_e2e(self, dev_in, {"y": self.y, "dx": self.dx, "dW": self.dW}, n_steps, self.ranks)
 
-        def e2e_step():
-            for n in host:
-                inp[n].copy_(host[n], non_blocking=True)
-            step()
-            out_h["y"].copy_(y, non_blocking=True)
-            out_h["dx"].copy_(dx, non_blocking=True)
-            out_h["dW"].copy_(dW, non_blocking=True)
+    def describe(self, ms_step, kernel_ms, peaks):
+        C, D = self.C, self.D
+        unit = C * D * 2
+        fwd_bytes, bwd_bytes = 2 * unit + C * 4, 3 * unit + C * 4
+        roof_ms = (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3
+        return {"dtype": "bf16",
+                "config": {"workload": "conv", "trees": self.args.conv_trees, "compact_tokens": C, "D": D, "w": self.w,
+                           "l2": f"inputs larger than L2 ({unit / 2**30:.2f} GiB per tensor)",
+                           "host_index_ms": self.t_host * 1e3},
+                "roofline": hbm_roofline("conv_bwd_kernel", bwd_bytes, kernel_ms["bwd"], peaks, None,
+                                         forward={"achieved": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9,
+                                                  "frac": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                                         whole_path={"roof_ms": roof_ms, "frac_strict": roof_ms / ms_step}),
+                "gpu_launches_per_step": 3}
 
-        e2e_step()
-        barrier()
-        a, b = ev(), ev()
-        n_e2e = max(1, min(args.steps, args.e2e_steps))
-        a.record(stream)
-        for _ in range(n_e2e):
-            e2e_step()
-        b.record(stream)
-        barrier()
-        e2e = {"ms": a.elapsed_time(b) / n_e2e, "steps": n_e2e,
-               "h2d": sum(t.numel() * t.element_size() for t in host.values()),
-               "d2h": sum(t.numel() * t.element_size() for t in out_h.values())}
-        del host, out_h
-    if world > 1:
-        ms_step, e2e_ms = max_over_ranks([ms_step, e2e["ms"] if e2e else 0.0], "cuda")
-        if e2e:
-            e2e["ms"] = e2e_ms
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-    peaks = measured_peaks()
-    unit = C * D * 2
-    fwd_bytes, bwd_bytes = 2 * unit + C * 4, 3 * unit + C * 4
-    achieved = bwd_bytes / (bwd_ms * 1e-3) / 1e9
-    clock = clocks.summary(h0, h1)
-    if not clock["samples"]:
-        clock = clocks.summary()
-    line = {
-        "metric": CONV_METRIC, "value": C * world / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "conv", "trees": args.conv_trees, "compact_tokens": C, "D": D, "w": w,
-                   "l2": f"inputs larger than L2 ({unit / 2**30:.2f} GiB per tensor)", "host_index_ms": t_host * 1e3},
-        "roofline": {"bound": "hbm", "kernel": "conv_bwd_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
-                     "algorithmic_bytes_per_launch": bwd_bytes, "peak_source": peaks["source"],
-                     "forward": {"achieved": fwd_bytes / (fwd_ms * 1e-3) / 1e9,
-                                 "frac": fwd_bytes / (fwd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
-                     "whole_path": {"roof_ms": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3,
-                                    "frac_strict": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms_step}},
-        "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms},
-        "gpu_launches": 3 * args.steps,
-        "clocks": clock,
-    }
-    if e2e:
-        line["e2e"] = {"value": C * world / (e2e["ms"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
-                       "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"], "pinned_host_memory": True}
-    if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = conv_oracle_sample()
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    def extras(self, ms_step):
+        return {}
 
-
+    def cpu_baseline(self):
+        return conv_oracle_sample()
 # --------------------------------------------------------------------------------------------------
 # Fourth workload: full attention on compact tokens (Section 3.4, Eqs. 21-22), `--workload attn`
 # --------------------------------------------------------------------------------------------------
@@ -924,196 +781,251 @@ def attn_oracle_sample(small=False, copies=1):
             "seconds": dt}
 
 
-def run_attn_reference(args):
+class AttnWorkload:
+    """One step = forward + backward of multi-head attention (16 heads, d = 128, bf16) over the compact tokens of
+    a forest (default cfg2): every token attends to its ancestors in the tree and to itself."""
+    metric, unit = ATTN_METRIC, UNIT
+
+    def __init__(self, args, ranks):
+        import torch
+        import paper_2608_28158_b200 as H
+        from workloads import config_forest, make_attn_inputs
+        self.H, self.args, self.ranks = H, args, ranks
+        fo = config_forest(args.attn_trees)
+        self.C, self.Hq, self.Hkv, self.d = C, Hq, Hkv, d = fo.n_tokens, ATTN_H, args.attn_kv_heads, ATTN_D
+        self.scale = d ** -0.5
+        plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
+        t0 = time.perf_counter()
+        self.index = index = H.harts_attn_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len,
+                                                plan.row_of_token)
+        self.t_host = time.perf_counter() - t0
+        index.upload()
+        anc = np.array([int(index.anc_len[index.anc_ptr[p]:index.anc_ptr[p + 1]].sum()) for p in range(index.n_pieces)],
+                       dtype=np.int64)
+        L = index.piece_len.astype(np.int64)
+        self.pairs = int((L * anc + L * (L + 1) // 2).sum())             # visible (query, key) pairs per head
+        self.inp = inp = make_attn_inputs(C, Hq, Hkv, d, "bf16", 90 + ranks.rank, device="cuda")
+        self.o, self.lse = torch.empty_like(inp["q"]), torch.empty(C, Hq, device="cuda")
+        self.grads = {"dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]), "dv": torch.empty_like(inp["v"])}
+        self.delta = torch.empty(C, Hq, device="cuda")
+        self.status = torch.zeros(4, dtype=torch.int32, device="cuda")
+        self.units = C
+        self.stream = torch.cuda.current_stream()
+
+    def step(self, marks):
+        import torch
+        H, inp, g = self.H, self.inp, self.grads
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        a.record(self.stream)
+        H.harts_attn_fwd(self.index, inp["q"], inp["k"], inp["v"], self.o, self.lse, self.scale, dev_status=self.status)
+        b.record(self.stream)
+        H.harts_attn_bwd(self.index, inp["q"], inp["k"], inp["v"], self.o, self.lse, inp["dO"], g["dq"], g["dk"], g["dv"],
+                         self.delta, self.scale, dev_status=self.status)
+        c.record(self.stream)
+        if marks is not None:
+            marks += [("fwd", a, b), ("bwd", b, c)]
+
+    def check(self):
+        self.H.harts_la_check(self.status)
+
+    def e2e(self, n_steps):
+        return time_e2e(self, dict(self.inp), dict(self.grads, o=self.o), n_steps, self.ranks)
+
+    def describe(self, ms_step, kernel_ms, peaks):
+        C, Hq, d, pairs = self.C, self.Hq, self.d, self.pairs
+        peak = peaks["bf16_tflops_sustained"]
+        fwd_flops = 4.0 * d * pairs * Hq                     # Q K^T and P V on the visible pairs only
+        bwd_flops = 2.5 * fwd_flops                          # five GEMMs (the kernels execute seven: S and dP twice)
+        achieved = bwd_flops / (kernel_ms["bwd"] * 1e-3) / 1e12
+        roof_ms = (fwd_flops + bwd_flops) / (peak * 1e12) * 1e3
+        return {"dtype": "bf16",
+                "config": {"workload": "attn", "trees": self.args.attn_trees, "compact_tokens": C, "Hq": Hq,
+                           "Hkv": self.Hkv, "d": d, "pieces": self.index.n_pieces, "visible_pairs_per_head": pairs,
+                           "mean_context": pairs / C,
+                           "l2": "flushed by the step itself: q, k, v, dO, o and the gradients "
+                                 f"({9 * C * Hq * d * 2 / 2**30:.2f} GiB) exceed L2",
+                           "host_index_ms": self.t_host * 1e3},
+                "roofline": {"bound": "tensor", "kernel": "backward call (attn_dq_kernel + attn_dkv_kernel)",
+                             "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                             "traffic": None, "algorithmic_flops_per_launch": bwd_flops,
+                             "executed_flops_per_launch": bwd_flops * 7 / 5,
+                             "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
+                             "forward": {"achieved": fwd_flops / (kernel_ms["fwd"] * 1e-3) / 1e12,
+                                         "frac": fwd_flops / (kernel_ms["fwd"] * 1e-3) / 1e12 / peak},
+                             "whole_path": {"roof_ms": roof_ms, "frac_strict": roof_ms / ms_step}},
+                "gpu_launches_per_step": 4}
+
+    def extras(self, ms_step):
+        return {}
+
+    def cpu_baseline(self):
+        return attn_oracle_sample()
+# --------------------------------------------------------------------------------------------------
+# Driver: one workload -> one JSON line
+# --------------------------------------------------------------------------------------------------
+WORKLOADS = {"logp": LogpWorkload, "conv": ConvWorkload, "attn": AttnWorkload}    # anything else: a cfg name
+
+
+def workload_class(name):
+    return WORKLOADS.get(name, LaWorkload)
+
+
+def measure(args, ranks, short=False):
+    """Builds the workload, times it and returns its JSON line as a dict (None on ranks other than 0)."""
+    import torch
+    work = workload_class(args.workload)(args, ranks)
+    t = time_blocks(work, args, ranks)
+    e2e = None
+    if not args.no_e2e and not short:
+        e2e = work.e2e(max(1, min(args.steps, args.e2e_steps)))
+        if ranks.world > 1:
+            e2e["ms"] = max_over_ranks([e2e["ms"]], "cuda")[0]
+    ms_step = t["ms_per_step"]
+    line = None
+    if ranks.rank == 0:
+        peaks = measured_peaks()
+        d = work.describe(ms_step, t["kernel_ms"], peaks)
+        units = work.units * ranks.world
+        line = {"metric": work.metric, "value": units / (ms_step * 1e-3), "unit": work.unit, "n_gpus": ranks.world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": d["dtype"], "data": "synthetic",
+                "config": d["config"], "roofline": d["roofline"], "kernel_ms": t["kernel_ms"],
+                "gpu_launches": d["gpu_launches_per_step"] * args.steps * t["timing"]["blocks"],
+                "clocks": t["clocks"], "timing": t["timing"]}
+        if e2e:
+            line["e2e"] = {"value": units / (e2e["ms"] * 1e-3), "unit": work.unit, "h2d_bytes_per_step": e2e["h2d"],
+                           "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"], "pinned_host_memory": True}
+            line["e2e"].update(e2e.get("extra", {}))
+        if not short:
+            line.update(work.extras(ms_step))
+    del work
+    torch.cuda.empty_cache()
+    return line
+
+
+def other_paths(args, ranks):
+    """Short runs of the three other built paths (log-probability, convolution, attention) for the record: value,
+    kernel times, roofline fraction and clocks of each, without their end-to-end and CPU legs."""
+    import copy
+    out = {}
+    for name in ("logp", "conv", "attn"):
+        a = copy.copy(args)
+        a.workload, a.steps, a.warmup, a.blocks = name, min(args.steps, 5), 3, 1
+        try:
+            line = measure(a, ranks, short=True)
+        except Exception as e:                       # a failure here must not lose the main line
+            out[name] = {"error": f"{type(e).__name__}: {e}"}
+            continue
+        out[name] = {"metric": line["metric"], "value": line["value"], "unit": line["unit"], "steps": a.steps,
+                     "ms_per_step": line["ms_per_step"], "kernel_ms": line["kernel_ms"],
+                     "roofline": {k: line["roofline"][k] for k in ("bound", "kernel", "achieved", "peak", "unit", "frac")},
+                     "roofline_forward_frac": line["roofline"]["forward"]["frac"],
+                     "roofline_whole_path_frac": line["roofline"]["whole_path"]["frac_strict"],
+                     "clocks": line["clocks"], "workload": line["config"]}
+    return out
+
+
+def run_ours(args):
+    ranks = Ranks()
+    line = measure(args, ranks)
+    if ranks.rank == 0:
+        la = workload_class(args.workload) is LaWorkload
+        if la and ranks.world == 1 and not args.no_other_paths:
+            line["other_paths"] = other_paths(args, ranks)
+        if ranks.world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = REFERENCE_SAMPLES[args.workload if not la else "la"](args, False)
+        print(json.dumps(line))
+    ranks.close()
+    if ranks.world == 1 and args.per_config:
+        per_config_table(args)
+
+
+# ---- reference arm: the oracle, as it stands, on the host cores ------------------------------------------------------
+def _la_sample(args, many_steps):
+    # every step is a bounded sample; its size shrinks with the step count so that the whole run stays within minutes
+    hint = min(8.0, 150.0 / max(1, args.warmup + args.steps)) if many_steps else 15.0
+    return oracle_sample(args.workload, seconds_hint=hint)
+
+
+REFERENCE_SAMPLES = {"la": _la_sample,
+                     "logp": lambda args, many: logp_oracle_sample(small=many),
+                     "conv": lambda args, many: conv_oracle_sample(small=many),
+                     "attn": lambda args, many: attn_oracle_sample(small=many)}
+
+
+def reference_config(args):
+    if args.workload == "logp":
+        return LOGP_METRIC, LOGP_UNIT, {"workload": "logp", "V": LOGP_V}
+    if args.workload == "conv":
+        return CONV_METRIC, UNIT, {"workload": "conv", "D": 4096, "w": CONV_W}
+    if args.workload == "attn":
+        return ATTN_METRIC, UNIT, {"workload": "attn", "Hq": ATTN_H, "Hkv": ATTN_H, "d": ATTN_D}
+    from workloads import CONFIGS
+    cfg = CONFIGS[args.workload]
+    return METRIC, UNIT, {"workload": args.workload, "H": cfg["H"], "dk": cfg["dk"], "dv": cfg["dv"], "chunk": 64}
+
+
+def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
+    sample = REFERENCE_SAMPLES[args.workload if args.workload in WORKLOADS else "la"]
     vals, secs, last = [], [], None
     for i in range(args.warmup + args.steps):
-        last = attn_oracle_sample(small=True)
+        last = sample(args, True)
         if i >= args.warmup:
             vals.append(last["value"])
             secs.append(last["seconds"])
     value = statistics.mean(vals)
+    metric, unit, config = reference_config(args)
     print(json.dumps({
-        "impl": "reference", "metric": ATTN_METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(secs) * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "attn", "Hq": ATTN_H, "Hkv": ATTN_H, "d": ATTN_D},
+        "config": config,
         "cpu_baseline": {"kind": last["kind"], "cores": last["cores"], "sample": last["sample"], "value": value,
-                         "unit": UNIT},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+                         "unit": unit},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
-def run_attn(args):
-    """One step = forward + backward of multi-head attention (16 heads, d = 128, bf16) over the compact tokens of
-    a forest (default cfg2): every token attends to its ancestors in the tree and to itself."""
-    import torch
-    import torch.distributed as dist
-
-    import paper_2608_28158_b200 as H
-    from workloads import config_forest, make_attn_inputs
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    fo = config_forest(args.attn_trees)
-    C, Hq, Hkv, d = fo.n_tokens, ATTN_H, args.attn_kv_heads, ATTN_D
-    scale = d ** -0.5
-    plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64)
-    t0 = time.perf_counter()
-    index = H.harts_attn_index(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, plan.row_of_token)
-    t_host = time.perf_counter() - t0
-    index.upload()
-    anc = np.array([int(index.anc_len[index.anc_ptr[p]:index.anc_ptr[p + 1]].sum()) for p in range(index.n_pieces)],
-                   dtype=np.int64)
-    L = index.piece_len.astype(np.int64)
-    pairs = int((L * anc + L * (L + 1) // 2).sum())             # visible (query, key) pairs per head
-    inp = make_attn_inputs(C, Hq, Hkv, d, "bf16", 90 + rank, device="cuda")
-    o, lse = torch.empty_like(inp["q"]), torch.empty(C, Hq, device="cuda")
-    grads = {"dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]), "dv": torch.empty_like(inp["v"])}
-    delta = torch.empty(C, Hq, device="cuda")
-    status = torch.zeros(4, dtype=torch.int32, device="cuda")
-    stream = torch.cuda.current_stream()
-    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
-
-    def step(marks=None):
-        a, b, c = ev(), ev(), ev()
-        a.record(stream)
-        H.harts_attn_fwd(index, inp["q"], inp["k"], inp["v"], o, lse, scale, dev_status=status)
-        b.record(stream)
-        H.harts_attn_bwd(index, inp["q"], inp["k"], inp["v"], o, lse, inp["dO"], grads["dq"], grads["dk"], grads["dv"],
-                         delta, scale, dev_status=status)
-        c.record(stream)
-        if marks is not None:
-            marks.append((a, b, c))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    marks = []
-    t_begin, t_end = ev(), ev()
-    with ClockSampler(local) as clocks:
-        for _ in range(args.warmup):
-            step()
-        H.harts_la_check(status)
-        barrier()
-        h0 = clocks.mark()
-        t_begin.record(stream)
-        for _ in range(args.steps):
-            step(marks)
-        t_end.record(stream)
-        barrier()
-        h1 = clocks.mark()
-    H.harts_la_check(status)
-    ms_step = t_begin.elapsed_time(t_end) / args.steps
-    fwd_ms = statistics.mean(a.elapsed_time(b) for a, b, _ in marks)
-    bwd_ms = statistics.mean(b.elapsed_time(c) for _, b, c in marks)
-    e2e = None
-    if not args.no_e2e:
-        host = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in inp.items()}
-        for n in host:
-            host[n].copy_(inp[n])
-        out_h = {n: torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for n, x in
-                 list(grads.items()) + [("o", o)]}
-        torch.cuda.synchronize()
-
-        def e2e_step():
-            for n in host:
-                inp[n].copy_(host[n], non_blocking=True)
-            step()
-            out_h["o"].copy_(o, non_blocking=True)
-            for n in grads:
-                out_h[n].copy_(grads[n], non_blocking=True)
-
-        e2e_step()
-        barrier()
-        a, b = ev(), ev()
-        n_e2e = max(1, min(args.steps, args.e2e_steps))
-        a.record(stream)
-        for _ in range(n_e2e):
-            e2e_step()
-        b.record(stream)
-        barrier()
-        e2e = {"ms": a.elapsed_time(b) / n_e2e, "steps": n_e2e,
-               "h2d": sum(t.numel() * t.element_size() for t in host.values()),
-               "d2h": sum(t.numel() * t.element_size() for t in out_h.values())}
-        del host, out_h
-    if world > 1:
-        ms_step, e2e_ms = max_over_ranks([ms_step, e2e["ms"] if e2e else 0.0], "cuda")
-        if e2e:
-            e2e["ms"] = e2e_ms
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-    peaks = measured_peaks()
-    peak = peaks["bf16_tflops_sustained"]
-    fwd_flops = 4.0 * d * pairs * Hq                     # Q K^T and P V on the visible pairs only
-    bwd_flops = 2.5 * fwd_flops                          # five GEMMs (the kernels execute seven: S and dP twice)
-    achieved = bwd_flops / (bwd_ms * 1e-3) / 1e12
-    clock = clocks.summary(h0, h1)
-    if not clock["samples"]:
-        clock = clocks.summary()
-    line = {
-        "metric": ATTN_METRIC, "value": C * world / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "attn", "trees": args.attn_trees, "compact_tokens": C, "Hq": Hq, "Hkv": Hkv, "d": d,
-                   "pieces": index.n_pieces, "visible_pairs_per_head": pairs,
-                   "mean_context": pairs / C, "l2": "flushed by the step itself: q, k, v, dO, o and the gradients "
-                   f"({9 * C * Hq * d * 2 / 2**30:.2f} GiB) exceed L2", "host_index_ms": t_host * 1e3},
-        "roofline": {"bound": "tensor", "kernel": "backward call (attn_dq_kernel + attn_dkv_kernel)",
-                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
-                     "algorithmic_flops_per_launch": bwd_flops, "executed_flops_per_launch": bwd_flops * 7 / 5,
-                     "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
-                     "forward": {"achieved": fwd_flops / (fwd_ms * 1e-3) / 1e12,
-                                 "frac": fwd_flops / (fwd_ms * 1e-3) / 1e12 / peak},
-                     "whole_path": {"roof_ms": (fwd_flops + bwd_flops) / (peak * 1e12) * 1e3,
-                                    "frac_strict": (fwd_flops + bwd_flops) / (peak * 1e12) * 1e3 / ms_step}},
-        "kernel_ms": {"fwd": fwd_ms, "bwd": bwd_ms},
-        "gpu_launches": 4 * args.steps,
-        "clocks": clock,
-    }
-    if e2e:
-        line["e2e"] = {"value": C * world / (e2e["ms"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
-                       "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"], "pinned_host_memory": True}
-    if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = attn_oracle_sample()
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+# ---- N ranks on one node ----------------------------------------------------------------------------------------------
+def spawn_command(argv, gpus, port):
+    """The torchrun command that starts `gpus` ranks of this script with the same arguments."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.join(ROOT, "bench.py")] + list(argv)
 
 
-def main():
+def free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--blocks", type=int, default=0, help="timed blocks of --steps steps (0: enough for ~2 s)")
     ap.add_argument("--fma", action="store_true", help="force the fp32-FMA kernels")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-trajwise", action="store_true")
+    ap.add_argument("--no-other-paths", action="store_true", help="skip the short runs of the logp / conv / attn paths")
     ap.add_argument("--logp-rows", type=int, default=LOGP_ROWS, help="compact-row capacity of the logp workload")
     ap.add_argument("--conv-trees", default="cfg3", help="forest of the conv workload (cfg2: a small case for captures)")
     ap.add_argument("--attn-trees", default="cfg2", help="forest of the attn workload (cfg1: a small case for captures)")
     ap.add_argument("--attn-kv-heads", type=int, default=ATTN_H, help="kv heads of the attn workload (16 = MHA)")
     ap.add_argument("--per-config", action="store_true", help="also print a table over all configurations to stderr")
-    args = ap.parse_args()
-    if args.workload == "logp":
-        (run_logp_reference if args.impl == "reference" else run_logp)(args)
-    elif args.workload == "conv":
-        (run_conv_reference if args.impl == "reference" else run_conv)(args)
-    elif args.workload == "attn":
-        (run_attn_reference if args.impl == "reference" else run_attn)(args)
-    elif args.impl == "reference":
+    args = ap.parse_args(argv)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly: become the launcher of one process per GPU (replicas, no collective on the data path)
+        sys.exit(subprocess.call(spawn_command(argv, args.gpus, free_port())))
+    if args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -39,3 +39,27 @@ def test_reference_arm_runs_on_rank_zero_only():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg0",
                         "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_plain_start_with_several_gpus_becomes_a_launcher():
+    """`python bench.py --gpus N` without torchrun's environment starts N ranks of itself (one process per GPU)."""
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.spawn_command(["--gpus", "4", "--steps", "2"], 4, 29999)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-4:] == ["--gpus", "4", "--steps", "2"]
+    assert cmd[cmd.index("--master-port") + 2].endswith("bench.py")
+    # under torchrun (WORLD_SIZE set) the script must NOT spawn again: the reference arm on rank 1 simply returns
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                        "--workload", "cfg0", "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True,
+                       timeout=300)
+    assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_block_count_fills_about_two_seconds():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.plan_blocks(20, 18.0) == 7          # 0.36 s blocks: 6 needed, made odd
+    assert bench.plan_blocks(20, 200.0) == 1         # a 4 s block is enough
+    assert bench.plan_blocks(20, 0.9) == 9           # capped
