@@ -51,6 +51,13 @@ extern "C" {
 
 /* flags */
 #define HARTS_FLAG_FMA_KERNELS 1u /* use the fp32-FMA (non tensor-core) kernels also for bf16 inputs */
+/* Debug check for hand-built tables (harts_la_fwd_seqs / harts_la_bwd_seqs): before the kernels of the call a small
+ * validation kernel checks every index they would follow (CSR pointers monotone and in range, rows < n_rows, slots <
+ * n_slots, replay shorter than a chunk, chunk counts consistent, consumer and replay-gradient tables in range).  On a
+ * bad entry the status word becomes HARTS_EINVAL (dev_status[1] = which table, 1-based in the order of
+ * harts_la_tables_t; dev_status[2] = position), the kernels of this and of later calls with the flag return without
+ * reading or writing anything, and harts_la_check() reports HARTS_EINVAL.  Needs dev_status (at least 4 int32). */
+#define HARTS_FLAG_CHECK_TABLES 2u
 
 typedef struct harts_la_plan harts_la_plan_t; /* opaque, host memory, library-owned */
 
@@ -231,6 +238,21 @@ int32_t harts_la_bwd_static(const harts_la_plan_t* plan, const void* dev_blob, c
                             const void* v, const float* g, const void* dO, void* dq, void* dk_, void* dv_, float* dg,
                             const void* chunk_states, int32_t H, int32_t dk, int32_t dv, int32_t dtype, uint32_t flags,
                             int32_t* dev_status, void* stream);
+
+/*
+ * Trajectory-wise view of a forest (host; the conventional execution the paper compares with in Section 5): every
+ * root-to-leaf trajectory as a sequence of its own, with the semantic map m of Eq. 3 -- for every position of every
+ * trajectory the canonical index (tree, node, offset order of the input) of the compact token it shares.  A
+ * trajectory ends in every node that no child continues from its last token; trajectories are listed by tree, then
+ * by the index of that node.  Running harts_la_plan on single-node trees of the returned lengths, with inputs
+ * gathered through src_token, is the trajectory-wise run of the same kernels.
+ *   traj_len  [cap_traj]   host, out: tokens of every trajectory
+ *   src_token [cap_tokens] host, out: canonical compact token of every expanded position, trajectories back to back
+ * Pass both arrays NULL to get *n_traj and *n_tokens only.  Errors: HARTS_EINVAL (malformed forest, capacity).
+ */
+int32_t harts_la_expand(int32_t n_trees, const int32_t* tree_node_ptr, const int32_t* node_parent,
+                        const int32_t* node_fork_off, const int32_t* node_len, int64_t cap_traj, int64_t cap_tokens,
+                        int32_t* traj_len, int64_t* src_token, int64_t* n_traj, int64_t* n_tokens);
 
 /* Synchronises `stream`, reads the device status word and returns HARTS_OK, HARTS_ETIMEOUT,
  * HARTS_EINVAL (an out-of-range index met by a harts_logp_* kernel, see harts_logp.h) or HARTS_ECUDA.  dev_status must be zeroed by the caller before the first launch. */

@@ -12,6 +12,7 @@ from . import build as _build
 HARTS_OK = 0
 HARTS_FP32, HARTS_BF16 = 0, 1
 HARTS_FLAG_FMA_KERNELS = 1
+HARTS_FLAG_CHECK_TABLES = 2
 _DTYPE_CODE = {torch.float32: HARTS_FP32, torch.bfloat16: HARTS_BF16}
 
 _I32P = C.POINTER(C.c_int32)
@@ -62,6 +63,9 @@ def _load():
     lib.harts_la_bwd_static.restype = i32
     lib.harts_la_selftest_timeout.argtypes = [vp, vp, vp]
     lib.harts_la_selftest_timeout.restype = i32
+    lib.harts_la_expand.argtypes = [i32, _I32P, _I32P, _I32P, _I32P, C.c_int64, C.c_int64, _I32P, C.POINTER(C.c_int64),
+                                    C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    lib.harts_la_expand.restype = i32
     for name in ("harts_la_plan", "harts_la_plan_view", "harts_la_plan_device_bytes", "harts_la_plan_upload",
                  "harts_la_plan_tables", "harts_la_workspace_bytes", "harts_la_fwd_seqs", "harts_la_bwd_seqs",
                  "harts_la_bwd_finish", "harts_la_fwd", "harts_la_bwd", "harts_la_check"):
@@ -312,37 +316,25 @@ class HostPipeline:
             s.synchronize()
 
 
+def harts_la_expand(tree_node_ptr, node_parent, node_fork_off, node_len):
+    """Trajectory-wise view of a forest (the conventional baseline of Section 5): returns (length of every
+    root-to-leaf trajectory, canonical compact token index of every expanded position)."""
+    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in (tree_node_ptr, node_parent, node_fork_off, node_len)]
+    ptrs = [a.ctypes.data_as(_I32P) for a in arrs]
+    n_traj, n_tok = C.c_int64(0), C.c_int64(0)
+    _check(lib.harts_la_expand(len(arrs[0]) - 1, *ptrs, 0, 0, None, None, C.byref(n_traj), C.byref(n_tok)),
+           "harts_la_expand")
+    lens = np.empty(n_traj.value, np.int32)
+    src = np.empty(n_tok.value, np.int64)
+    _check(lib.harts_la_expand(len(arrs[0]) - 1, *ptrs, n_traj.value, n_tok.value, lens.ctypes.data_as(_I32P),
+                               src.ctypes.data_as(C.POINTER(C.c_int64)), C.byref(n_traj), C.byref(n_tok)),
+           "harts_la_expand")
+    return lens, src
+
+
 def expand_trajectories(tree_node_ptr, node_parent, node_fork_off, node_len):
-    """Trajectory-wise view of a forest (the conventional baseline of Section 5): every root-to-leaf
-    path becomes its own single-node tree.  Returns (forest arrays of the expanded problem,
-    canonical compact token index of every expanded token)."""
-    tree_node_ptr, node_parent, node_fork_off, node_len = (np.asarray(a) for a in
-                                                            (tree_node_ptr, node_parent, node_fork_off, node_len))
-    base = np.zeros(len(node_len) + 1, dtype=np.int64)
-    np.cumsum(node_len, out=base[1:])
-    lens, src = [], []
-    for t in range(len(tree_node_ptr) - 1):
-        lo, hi = int(tree_node_ptr[t]), int(tree_node_ptr[t + 1])
-        has_tail_child = np.zeros(hi - lo, dtype=bool)
-        for i in range(lo + 1, hi):
-            p = lo + int(node_parent[i])
-            if node_fork_off[i] == node_len[p]:
-                has_tail_child[p - lo] = True
-        for leaf in range(lo, hi):
-            if has_tail_child[leaf - lo]:
-                continue
-            parts, node, upto = [], leaf, int(node_len[leaf])
-            while True:
-                parts.append(np.arange(base[node], base[node] + upto, dtype=np.int64))
-                if node_parent[node] < 0:
-                    break
-                upto = int(node_fork_off[node])
-                node = lo + int(node_parent[node])
-            parts.reverse()
-            rows = np.concatenate(parts)
-            src.append(rows)
-            lens.append(len(rows))
+    """The expanded problem as forest arrays (every trajectory a single-node tree) plus the source-token map."""
+    lens, src = harts_la_expand(tree_node_ptr, node_parent, node_fork_off, node_len)
     n = len(lens)
-    forest = (np.arange(n + 1, dtype=np.int32), np.full(n, -1, np.int32), np.zeros(n, np.int32),
-              np.asarray(lens, np.int32))
-    return forest, np.concatenate(src)
+    forest = (np.arange(n + 1, dtype=np.int32), np.full(n, -1, np.int32), np.zeros(n, np.int32), lens)
+    return forest, src

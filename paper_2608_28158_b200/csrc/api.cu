@@ -76,6 +76,8 @@ int32_t harts_la_fwd_seqs(const harts_la_tables_t* tb, int32_t seq_lo, int32_t s
         return HARTS_EINVAL;
     harts::FwdArgs a{*tb, seq_lo, seq_hi, q, k, v, g, o, slots, chunk_states, H, dk, dv, dtype, flags, dev_status,
                      static_cast<cudaStream_t>(stream)};
+    if (flags & HARTS_FLAG_CHECK_TABLES)
+        if ((rc = harts::check_tables(*tb, seq_lo, seq_hi, dev_status, a.stream)) != HARTS_OK) return rc;
     if (use_tc(dtype, dk, dv, flags)) return harts::tc_fwd(a);
     return harts::fma_fwd(a);
 }
@@ -92,6 +94,8 @@ int32_t harts_la_bwd_seqs(const harts_la_tables_t* tb, int32_t seq_lo, int32_t s
         return HARTS_EINVAL;
     harts::BwdArgs a{*tb, seq_lo, seq_hi, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, scratch, H, dk, dv, dtype,
                      flags, dev_status, static_cast<cudaStream_t>(stream)};
+    if (flags & HARTS_FLAG_CHECK_TABLES)
+        if ((rc = harts::check_tables(*tb, seq_lo, seq_hi, dev_status, a.stream)) != HARTS_OK) return rc;
     if (use_tc(dtype, dk, dv, flags)) return harts::tc_bwd(a);
     return harts::fma_bwd(a);
 }

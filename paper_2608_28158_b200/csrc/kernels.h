@@ -66,6 +66,22 @@ inline ScratchLayout scratch_layout(const harts_la_tables_t& tb, int32_t H, int3
     return s;
 }
 
+// With HARTS_FLAG_CHECK_TABLES the kernels of a call run only while the status word is still zero: check_tables (a
+// validation kernel ahead of them on the stream) records a bad index there, and nothing is dereferenced after it.
+inline const int32_t* status_gate(uint32_t flags, const int32_t* dev_status) {
+    return (flags & HARTS_FLAG_CHECK_TABLES) ? dev_status : nullptr;
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ bool gate_closed(const int32_t* gate) {     // called by every thread of the CTA
+    if (!gate) return false;
+    __shared__ int closed;
+    if (threadIdx.x == 0) closed = *reinterpret_cast<const volatile int32_t*>(gate);
+    __syncthreads();
+    return closed != 0;
+}
+#endif
+int32_t check_tables(const harts_la_tables_t& tb, int32_t seq_lo, int32_t seq_hi, int32_t* dev_status, cudaStream_t stream);
+
 int32_t fma_supported(int32_t dtype, int32_t dk, int32_t dv);
 int32_t fma_fwd(const FwdArgs& a);
 int32_t fma_bwd(const BwdArgs& a);

@@ -102,7 +102,8 @@ __device__ void load_chunk(const harts_la_tables_t& tb, const SeqInfo& s, int c,
 template <typename T, int DK, int DV>
 __global__ void __launch_bounds__(NT) fma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const T* q,
                                                      const T* k, const T* v, const float* g, T* o, float* slots,
-                                                     T* chunk_states) {
+                                                     T* chunk_states, const int32_t* gate) {
+    if (gate_closed(gate)) return;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* sS = reinterpret_cast<float*>(smem_raw);       // [DK][DV]
     float* sA = sS + DK * DV;                             // [BT][BT+1]
@@ -211,7 +212,8 @@ template <typename T, int DK, int DV>
 __global__ void __launch_bounds__(NT) fma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const T* q,
                                                      const T* k, const T* v, const float* g, const T* dO, T* dq,
                                                      T* dk_, T* dv_, float* dg, const T* chunk_states,
-                                                     float* ds0, float* rk, float* rv, float* rg) {
+                                                     float* ds0, float* rk, float* rv, float* rg, const int32_t* gate) {
+    if (gate_closed(gate)) return;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* sS = reinterpret_cast<float*>(smem_raw);       // S_c           [DK][DV]
     float* sdS = sS + DK * DV;                            // dS            [DK][DV]
@@ -454,7 +456,7 @@ int32_t launch_fwd(const FwdArgs& a) {
         return HARTS_ECUDA;
     int n = (a.seq_hi - a.seq_lo) * a.H;
     kern<<<n, NT, smem, a.stream>>>(a.tb, a.seq_lo, a.H, (const T*)a.q, (const T*)a.k, (const T*)a.v, a.g, (T*)a.o,
-                                    a.slots, (T*)a.chunk_states);
+                                    a.slots, (T*)a.chunk_states, status_gate(a.flags, a.dev_status));
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
@@ -471,7 +473,7 @@ int32_t launch_bwd(const BwdArgs& a) {
     kern<<<n, NT, smem, a.stream>>>(a.tb, a.seq_lo, a.H, (const T*)a.q, (const T*)a.k, (const T*)a.v, a.g,
                                     (const T*)a.dO, (T*)a.dq, (T*)a.dk_, (T*)a.dv_, a.dg, (const T*)a.chunk_states,
                                     (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
-                                    (float*)(base + sl.rg));
+                                    (float*)(base + sl.rg), status_gate(a.flags, a.dev_status));
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
@@ -496,7 +498,8 @@ int32_t fma_fwd(const FwdArgs& a) {
 // sequences [seq_lo, seq_hi) exported: a bandwidth-bound pass, in consumer order (deterministic), so that the
 // backward kernels add one tensor per boundary instead of walking the consumer list under their own latency.
 __global__ void __launch_bounds__(256) handoff_reduce_kernel(const harts_la_tables_t tb, int seq_lo, int seq_hi, int H,
-                                                             int elems, float* __restrict__ ds0) {
+                                                             int elems, float* __restrict__ ds0, const int32_t* gate) {
+    if (gate_closed(gate)) return;
     const int slot = blockIdx.x;
     if (slot < tb.seq_req_ptr[seq_lo] || slot >= tb.seq_req_ptr[seq_hi]) return;
     const int c0 = tb.slot_cons_ptr[slot], c1 = tb.slot_cons_ptr[slot + 1];
@@ -530,7 +533,8 @@ int32_t handoff_reduce(const BwdArgs& a) {
     float* ds0 = reinterpret_cast<float*>(static_cast<char*>(a.scratch) + sl.ds0);
     const int elems = a.dk * a.dv;
     dim3 grid(a.tb.n_slots, a.H, (elems / 4 + 1023) / 1024);
-    handoff_reduce_kernel<<<grid, 256, 0, a.stream>>>(a.tb, a.seq_lo, a.seq_hi, a.H, elems, ds0);
+    handoff_reduce_kernel<<<grid, 256, 0, a.stream>>>(a.tb, a.seq_lo, a.seq_hi, a.H, elems, ds0,
+                                                      status_gate(a.flags, a.dev_status));
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 

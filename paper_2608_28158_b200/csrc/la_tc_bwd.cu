@@ -182,7 +182,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
               const __nv_bfloat16* __restrict__ dO, __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk_,
               __nv_bfloat16* __restrict__ dv_, float* __restrict__ dg, float* __restrict__ ds0, float* __restrict__ rk,
-              float* __restrict__ rv, float* __restrict__ rg, int* status) {
+              float* __restrict__ rv, float* __restrict__ rg, int* status, const int32_t* gate) {
+    if (gate_closed(gate)) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     unsigned char* sQ = smem + Smem::q;
@@ -684,7 +685,7 @@ int32_t tc_bwd(const BwdArgs& a) {
         a.tb, a.seq_lo, n, a.H, mq, mk, mv, mdo, mcs, mdq, mdk, mdv, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_,
         (__nv_bfloat16*)a.dv_, a.dg, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
-        (float*)(base + sl.rg), a.dev_status);
+        (float*)(base + sl.rg), a.dev_status, status_gate(a.flags, a.dev_status));
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 

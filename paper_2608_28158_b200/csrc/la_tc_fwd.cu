@@ -75,7 +75,9 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
               const __grid_constant__ CUtensorMap map_cs, const __grid_constant__ CUtensorMap map_o,
               const __nv_bfloat16* __restrict__ q,
               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
-              __nv_bfloat16* __restrict__ o, float* __restrict__ slots, int store_states, int* status) {
+              __nv_bfloat16* __restrict__ o, float* __restrict__ slots, int store_states, int* status,
+              const int32_t* gate) {
+    if (gate_closed(gate)) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     unsigned char* sQ = smem + Smem::q;
@@ -480,7 +482,8 @@ int32_t tc_fwd(const FwdArgs& a) {
     int grid = n < 2 * sm_count() ? n : 2 * sm_count();
     tc_fwd_kernel<<<grid, NT, Smem::bytes + 1024, a.stream>>>(
         a.tb, a.seq_lo, n, a.H, mq, mk, mv, mcs, mo, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
-        (const __nv_bfloat16*)a.v, a.g, (__nv_bfloat16*)a.o, a.slots, a.chunk_states != nullptr, a.dev_status);
+        (const __nv_bfloat16*)a.v, a.g, (__nv_bfloat16*)a.o, a.slots, a.chunk_states != nullptr, a.dev_status,
+        status_gate(a.flags, a.dev_status));
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 

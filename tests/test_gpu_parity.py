@@ -187,6 +187,55 @@ def test_hand_built_tables_drive_one_packed_call():
     assert rel_err(slots[0].cpu().numpy(), exported) < 5e-3
 
 
+def test_bad_hand_built_tables_are_caught_on_the_device_and_nothing_is_dereferenced():
+    """HARTS_FLAG_CHECK_TABLES: a replay row far outside the tensors, an initial-state slot that does not exist, a
+    boundary request past the sequence's end.  The validation kernel records HARTS_EINVAL, the kernels of the call do
+    not run (the outputs keep their fill value), nothing faults; the same tables without the mistake pass the check
+    and give the bits of an unchecked run."""
+    H_, d, n0, n1 = 2, 128, 150, 70
+    inp = make_inputs(n0 + n1, H_, d, d, "bf16", 23)
+    dev = {n: x.cuda() for n, x in inp.items()}
+    i32 = lambda *v: torch.tensor(v, dtype=torch.int32, device="cuda")  # noqa: E731
+
+    def tables(replay_row=5, init_slot=0, slot_chunk=1):
+        # sequence 0: 150 rows from the zero state, exports the state after its first chunk into slot 0;
+        # sequence 1: replays row `replay_row`, then its 70 own rows, from slot `init_slot`
+        arrays = dict(seq_own_begin=i32(0, n0, n0 + n1), seq_init_slot=i32(-1, init_slot), seq_replay_ptr=i32(0, 0, 1),
+                      replay_row=i32(replay_row), seq_req_ptr=i32(0, 1, 1), slot_chunk=i32(slot_chunk),
+                      seq_chunk_ptr=i32(0, 3, 5), slot_cons_ptr=i32(0, 1), slot_cons_seq=i32(1), rg_row=i32(5),
+                      rg_ptr=i32(0, 1), rg_entry=i32(0))
+        tb = H.binding.Tables()
+        tb.chunk, tb.n_rows, tb.n_replay, tb.n_seq, tb.n_slots, tb.n_chunks, tb.n_rg_rows = 64, n0 + n1, 1, 2, 1, 5, 1
+        for n, a in arrays.items():
+            setattr(tb, n, a.data_ptr())
+        return tb, arrays
+
+    def forward(tb, flags):
+        status = torch.zeros(4, dtype=torch.int32, device="cuda")
+        slots = torch.zeros(1, H_, d, d, device="cuda")
+        o = torch.full_like(dev["v"], 7.0)
+        H.harts_la_fwd_seqs(tb, 0, 1, dev["q"], dev["k"], dev["v"], dev["g"], o, slots, None, flags, status)
+        H.harts_la_fwd_seqs(tb, 1, 2, dev["q"], dev["k"], dev["v"], dev["g"], o, slots, None, flags, status)
+        return o, status
+
+    good, keep = tables()
+    o_ref, st = forward(good, 0)
+    H.harts_la_check(st)
+    o_chk, st = forward(good, H.HARTS_FLAG_CHECK_TABLES)
+    H.harts_la_check(st)
+    assert torch.equal(o_ref, o_chk)
+    for kwargs, table in ((dict(replay_row=10 ** 9), 4), (dict(init_slot=3), 2), (dict(slot_chunk=3), 6)):
+        bad, keep = tables(**kwargs)
+        o, st = forward(bad, H.HARTS_FLAG_CHECK_TABLES)
+        with pytest.raises(H.HartsError) as e:
+            H.harts_la_check(st)
+        assert e.value.code == -1 and int(st[1]) == table, (kwargs, st.tolist())
+        # the call that held the bad entry, and every later call on this status word, left the outputs alone
+        lo_ = 0 if table == 6 else n0
+        assert bool((o[lo_:] == 7.0).all())
+    torch.cuda.synchronize()
+
+
 def test_errors_are_reported_without_launching():
     cfg, fo, inp = config_case("cfg0")
     plan = plan_of(fo).upload()

@@ -140,3 +140,20 @@ def test_library_exports_every_declared_symbol():
             "harts_logp_positions", "harts_logp_csr", "harts_logp_fwd_shard", "harts_logp_combine"} <= names
     for n in names:
         assert hasattr(H.lib, n), n
+
+
+def test_expand_matches_the_oracles_semantic_map():
+    """harts_la_expand (the trajectory-wise view behind the C ABI) against the oracle's own enumeration of the
+    root-to-leaf trajectories and of the map m of Eq. 3: same trajectories, same order, same source tokens."""
+    import random
+    from oracle import la_oracle as lo
+    from test_plan_oracle import random_tree
+    rnd = random.Random(31)
+    cases = [config_forest("cfg0"), config_forest("cfg0b"), config_forest("cfg1")]
+    cases += [make_forest([random_tree(rnd, rnd.randint(1, 12), 30) for _ in range(rnd.randint(1, 4))]) for _ in range(200)]
+    for fo in cases:
+        lens, src = H.harts_la_expand(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len)
+        ptr, rows = lo.trajectories(fo)
+        assert np.array_equal(np.diff(ptr), lens) and np.array_equal(rows, src)
+    with pytest.raises(H.HartsError):
+        H.harts_la_expand([0, 2], [-1, 0], [0, 9], [3, 2])          # fork offset beyond the parent
