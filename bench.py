@@ -403,7 +403,7 @@ class LaWorkload:
         Hh, dk, dv = cfg["H"], cfg["dk"], cfg["dv"]
         # every rank draws its own tensors (independent batches of the same shape)
         self.inp = inp = make_inputs(plan.C, Hh, dk, dv, cfg["dtype"], cfg["seed"] + 100 * ranks.rank, device="cuda")
-        self.flags = H.HARTS_FLAG_FMA_KERNELS if args.fma else 0
+        self.flags = (H.HARTS_FLAG_FMA_KERNELS if args.fma else 0)
         self.ws = H.Workspace(plan, Hh, dk, dv, inp["q"].dtype, self.flags)
         self.out = {"o": torch.empty_like(inp["v"]), "dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]),
                     "dv": torch.empty_like(inp["v"]), "dg": torch.empty_like(inp["g"])}

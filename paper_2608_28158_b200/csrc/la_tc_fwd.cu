@@ -361,7 +361,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
 #pragma unroll
                 for (int e = 0; e < 32; e++) {
                     int t = t0 + e;
-                    float val = __uint_as_float(x1[e]) + ebt[e] * __uint_as_float(x2[e]);
+                    float val = __fmaf_rn(ebt[e], __uint_as_float(x2[e]), __uint_as_float(x1[e]));
                     *reinterpret_cast<__nv_bfloat16*>(sO + t * 256 + L * 2) = __float2bfloat16_rn(val);
                 }
                 fence_async_smem();
@@ -370,7 +370,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 for (int e = 0; e < 32; e++) {
                     int t = t0 + e, code = m.code[t];
                     if (code >= 0) {
-                        float val = __uint_as_float(x1[e]) + m.eb[t] * __uint_as_float(x2[e]);
+                        float val = __fmaf_rn(m.eb[t], __uint_as_float(x2[e]), __uint_as_float(x1[e]));
                         o[((size_t)code * H + h) * D + L] = __float2bfloat16_rn(val);
                     }
                 }
