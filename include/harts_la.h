@@ -212,6 +212,32 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
                      int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream);
 
 /*
+ * The same path for the recurrence with a PER-CHANNEL decay, the first term of Eq. 1 (Section 2.2, the Diag(gamma)
+ * decay on the key dimension of the state; Section 4.1 names a backend of this family as the one evaluated):
+ *
+ *     S_t = Diag(exp(g_t)) S_{t-1} + k_t^T v_t,     o_t = q_t S_t,       g_t in R^{dk}, g_t <= 0
+ *
+ * (the scalar gate above is its special case with all channels equal; the delta-rule part of Eq. 1, U - W S, is not
+ * defined by the paper and is not provided).  Plan, uploaded tables, slots, replay rows, chunk states and the
+ * hand-off of initial-state gradients are exactly those of harts_la_fwd / harts_la_bwd; only
+ *   gk  [n_rows, H, dk] fp32 DEVICE: the per-channel log-decay (never modified), and
+ *   dgk [n_rows, H, dk] fp32 DEVICE: its gradient (own rows overwritten; replayed rows folded in by the round-1 call)
+ * replace g and dg, and the backward scratch is larger (harts_la_gk_workspace_bytes: the replay-row gradient of g is
+ * a vector).  Rounds as for harts_la_fwd / harts_la_bwd (0 = all).  Served: fp32 with dk = dv = 64, bf16 with
+ * dk = dv = 64 or 128, chunk 64; fp32 arithmetic on the CUDA cores (every decay factor is evaluated as
+ * exp(b_t[i] - b_j[i]) with j <= t, so no gate value can overflow).  Errors as for harts_la_fwd / harts_la_bwd.
+ */
+int32_t harts_la_gk_workspace_bytes(const harts_la_tables_t* tables, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                                    size_t* chunk_state_bytes, size_t* scratch_bytes);
+int32_t harts_la_gk_fwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t round, const void* q, const void* k,
+                        const void* v, const float* gk, void* o, float* slots, void* chunk_states, int32_t H, int32_t dk,
+                        int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream);
+int32_t harts_la_gk_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t round, const void* q, const void* k,
+                        const void* v, const float* gk, const void* dO, void* dq, void* dk_, void* dv_, float* dgk,
+                        const void* chunk_states, void* scratch, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                        uint32_t flags, int32_t* dev_status, void* stream);
+
+/*
  * (No counterpart in the paper: an addition for a kind of caller, not part of the method.)
  * Backward of ALL rounds followed by the replay-gradient fold, like harts_la_bwd(plan, blob, 0, ...), but with the
  * scratch area inside the library instead of in a caller-owned buffer.  It is meant for callers that have no way to

@@ -66,6 +66,11 @@ def _load():
     lib.harts_la_expand.argtypes = [i32, _I32P, _I32P, _I32P, _I32P, C.c_int64, C.c_int64, _I32P, C.POINTER(C.c_int64),
                                     C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
     lib.harts_la_expand.restype = i32
+    lib.harts_la_gk_workspace_bytes.argtypes = [C.POINTER(Tables), i32, i32, i32, i32, C.POINTER(sz), C.POINTER(sz)]
+    lib.harts_la_gk_fwd.argtypes = [vp, vp, i32] + [vp] * 7 + [i32] * 4 + [u32, vp, vp]
+    lib.harts_la_gk_bwd.argtypes = [vp, vp, i32] + [vp] * 11 + [i32] * 4 + [u32, vp, vp]
+    for name in ("harts_la_gk_workspace_bytes", "harts_la_gk_fwd", "harts_la_gk_bwd"):
+        getattr(lib, name).restype = i32
     for name in ("harts_la_plan", "harts_la_plan_view", "harts_la_plan_device_bytes", "harts_la_plan_upload",
                  "harts_la_plan_tables", "harts_la_workspace_bytes", "harts_la_fwd_seqs", "harts_la_bwd_seqs",
                  "harts_la_bwd_finish", "harts_la_fwd", "harts_la_bwd", "harts_la_check"):
@@ -222,6 +227,28 @@ def harts_la_bwd_static(plan, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, fl
     _check(lib.harts_la_bwd_static(plan._h, _ptr(plan.blob), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(dO), _ptr(dq),
                                    _ptr(dk_), _ptr(dv_), _ptr(dg), _ptr(chunk_states), H, dk, dv, dt, flags,
                                    _ptr(dev_status), _stream(stream)), "harts_la_bwd_static")
+
+
+def harts_la_gk_workspace_bytes(tables, H, dk, dv, dtype):
+    a, b = C.c_size_t(0), C.c_size_t(0)
+    _check(lib.harts_la_gk_workspace_bytes(C.byref(tables), H, dk, dv, dtype, C.byref(a), C.byref(b)),
+           "harts_la_gk_workspace_bytes")
+    return int(a.value), int(b.value)
+
+
+def harts_la_gk_fwd(plan, round, q, k, v, gk, o, slots, chunk_states, flags=0, dev_status=None, stream=None):
+    H, dk, dv, dt = _dims(q, v)
+    _check(lib.harts_la_gk_fwd(plan._h, _ptr(plan.blob), round, _ptr(q), _ptr(k), _ptr(v), _ptr(gk), _ptr(o),
+                               _ptr(slots), _ptr(chunk_states), H, dk, dv, dt, flags, _ptr(dev_status),
+                               _stream(stream)), "harts_la_gk_fwd")
+
+
+def harts_la_gk_bwd(plan, round, q, k, v, gk, dO, dq, dk_, dv_, dgk, chunk_states, scratch, flags=0, dev_status=None,
+                    stream=None):
+    H, dk, dv, dt = _dims(q, v)
+    _check(lib.harts_la_gk_bwd(plan._h, _ptr(plan.blob), round, _ptr(q), _ptr(k), _ptr(v), _ptr(gk), _ptr(dO),
+                               _ptr(dq), _ptr(dk_), _ptr(dv_), _ptr(dgk), _ptr(chunk_states), _ptr(scratch), H, dk, dv,
+                               dt, flags, _ptr(dev_status), _stream(stream)), "harts_la_gk_bwd")
 
 
 def harts_la_selftest_timeout(dev_status, dev_report=None, stream=None):

@@ -144,6 +144,73 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
     return HARTS_OK;
 }
 
+// ---- per-channel decay (the Diag(gamma) term of Eq. 1) -------------------------------------------------------------------
+int32_t harts_la_gk_workspace_bytes(const harts_la_tables_t* tb, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                                    size_t* chunk_state_bytes, size_t* scratch_bytes) {
+    if (!tb || H < 1 || dk < 1 || dv < 1) return HARTS_EINVAL;
+    if (dtype != HARTS_FP32 && dtype != HARTS_BF16) return HARTS_EUNSUPPORTED;
+    const size_t elem = dtype == HARTS_FP32 ? 4 : 2;
+    if (chunk_state_bytes) {
+        const size_t b = (size_t)tb->n_chunks * H * dk * dv * elem;
+        *chunk_state_bytes = b < 256 ? 256 : b;
+    }
+    if (scratch_bytes) *scratch_bytes = harts::gk_scratch_layout(*tb, H, dk, dv).total;
+    return HARTS_OK;
+}
+
+int32_t harts_la_gk_fwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t round, const void* q, const void* k,
+                        const void* v, const float* gk, void* o, float* slots, void* chunk_states, int32_t H, int32_t dk,
+                        int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream) {
+    const harts::Plan* p = harts_la_plan_internal(plan);
+    if (!p || round < 0 || round > p->n_rounds) return HARTS_EINVAL;
+    harts_la_tables_t tb;
+    int32_t rc = harts_la_plan_tables(plan, dev_blob, &tb);
+    if (rc != HARTS_OK) return rc;
+    if (H < 1 || tb.chunk != 64 || !harts::gk_supported(dtype, dk, dv)) return H < 1 ? HARTS_EINVAL : HARTS_EUNSUPPORTED;
+    if (!q || !k || !v || !gk || !o || (tb.n_slots > 0 && !slots)) return HARTS_EINVAL;
+    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(gk) || misaligned(o) || misaligned(slots) ||
+        misaligned(chunk_states))
+        return HARTS_EINVAL;
+    if ((flags & HARTS_FLAG_CHECK_TABLES) && !dev_status) return HARTS_EINVAL;
+    const int32_t r0 = round == 0 ? 1 : round, r1 = round == 0 ? p->n_rounds : round;
+    for (int32_t r = r0; r <= r1; r++) {
+        harts::FwdArgs a{tb, p->round_seq_ptr[r - 1], p->round_seq_ptr[r], q, k, v, gk, o, slots, chunk_states, H, dk, dv,
+                         dtype, flags, dev_status, static_cast<cudaStream_t>(stream)};
+        if (flags & HARTS_FLAG_CHECK_TABLES)
+            if ((rc = harts::check_tables(tb, a.seq_lo, a.seq_hi, dev_status, a.stream)) != HARTS_OK) return rc;
+        if ((rc = harts::gk_fwd(a)) != HARTS_OK) return rc;
+    }
+    return HARTS_OK;
+}
+
+int32_t harts_la_gk_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t round, const void* q, const void* k,
+                        const void* v, const float* gk, const void* dO, void* dq, void* dk_, void* dv_, float* dgk,
+                        const void* chunk_states, void* scratch, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
+                        uint32_t flags, int32_t* dev_status, void* stream) {
+    const harts::Plan* p = harts_la_plan_internal(plan);
+    if (!p || round < 0 || round > p->n_rounds) return HARTS_EINVAL;
+    harts_la_tables_t tb;
+    int32_t rc = harts_la_plan_tables(plan, dev_blob, &tb);
+    if (rc != HARTS_OK) return rc;
+    if (H < 1 || tb.chunk != 64 || !harts::gk_supported(dtype, dk, dv)) return H < 1 ? HARTS_EINVAL : HARTS_EUNSUPPORTED;
+    if (!q || !k || !v || !gk || !dO || !dq || !dk_ || !dv_ || !dgk || !chunk_states || !scratch) return HARTS_EINVAL;
+    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(gk) || misaligned(dO) || misaligned(dq) ||
+        misaligned(dk_) || misaligned(dv_) || misaligned(dgk) || misaligned(chunk_states) || misaligned(scratch))
+        return HARTS_EINVAL;
+    if ((flags & HARTS_FLAG_CHECK_TABLES) && !dev_status) return HARTS_EINVAL;
+    const int32_t r1 = round == 0 ? p->n_rounds : round, r0 = round == 0 ? 1 : round;
+    for (int32_t r = r1; r >= r0; r--) {
+        harts::BwdArgs a{tb, p->round_seq_ptr[r - 1], p->round_seq_ptr[r], q, k, v, gk, dO, dq, dk_, dv_, dgk,
+                         chunk_states, scratch, H, dk, dv, dtype, flags, dev_status, static_cast<cudaStream_t>(stream)};
+        if (flags & HARTS_FLAG_CHECK_TABLES)
+            if ((rc = harts::check_tables(tb, a.seq_lo, a.seq_hi, dev_status, a.stream)) != HARTS_OK) return rc;
+        if ((rc = harts::gk_bwd(a)) != HARTS_OK) return rc;
+    }
+    if (r0 == 1)
+        return harts::gk_replay_reduce(tb, dk_, dv_, dgk, scratch, H, dk, dv, dtype, static_cast<cudaStream_t>(stream));
+    return HARTS_OK;
+}
+
 int32_t harts_la_check(const int32_t* dev_status, void* stream) {
     if (!dev_status) return HARTS_EINVAL;
     int32_t host = 0;

@@ -82,6 +82,31 @@ __device__ __forceinline__ bool gate_closed(const int32_t* gate) {     // called
 #endif
 int32_t check_tables(const harts_la_tables_t& tb, int32_t seq_lo, int32_t seq_hi, int32_t* dev_status, cudaStream_t stream);
 
+// The same for the per-channel-decay calls: the replay-row gradient of g is a vector over the key channels.
+struct GkScratchLayout {
+    size_t ds0, rk, rv, rg, total;     // rg: [n_replay, H, dk] fp32
+};
+inline GkScratchLayout gk_scratch_layout(const harts_la_tables_t& tb, int32_t H, int32_t dk, int32_t dv) {
+    GkScratchLayout s;
+    size_t off = 0;
+    s.ds0 = off;
+    off = align_up(off + (size_t)tb.n_seq * H * dk * dv * sizeof(float), 256);
+    s.rk = off;
+    off = align_up(off + (size_t)tb.n_replay * H * dk * sizeof(float), 256);
+    s.rv = off;
+    off = align_up(off + (size_t)tb.n_replay * H * dv * sizeof(float), 256);
+    s.rg = off;
+    off = align_up(off + (size_t)tb.n_replay * H * dk * sizeof(float), 256);
+    s.total = off < 256 ? 256 : off;
+    return s;
+}
+
+int32_t gk_supported(int32_t dtype, int32_t dk, int32_t dv);
+int32_t gk_fwd(const FwdArgs& a);      // FwdArgs::g / BwdArgs::g, ::dg point to [rows, H, dk] arrays here
+int32_t gk_bwd(const BwdArgs& a);
+int32_t gk_replay_reduce(const harts_la_tables_t& tb, void* dk_, void* dv_, float* dgk, const void* scratch, int32_t H,
+                         int32_t dk, int32_t dv, int32_t dtype, cudaStream_t stream);
+
 int32_t fma_supported(int32_t dtype, int32_t dk, int32_t dv);
 int32_t fma_fwd(const FwdArgs& a);
 int32_t fma_bwd(const BwdArgs& a);
