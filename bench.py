@@ -861,9 +861,113 @@ class AttnWorkload:
     def cpu_baseline(self):
         return attn_oracle_sample()
 # --------------------------------------------------------------------------------------------------
+# Fifth workload: the per-channel-decay recurrence (Diag(gamma) term of Eq. 1), `--workload gk`
+# --------------------------------------------------------------------------------------------------
+GK_METRIC = "tree-packed per-channel-decay linear-attn fwd+bwd compact tokens/s"
+GK_CONFIG = "cfg2"
+
+
+def gk_oracle_sample(small=False):
+    """The fp64 per-channel oracle on whole trees of the workload's forest, one head."""
+    from oracle import gk_oracle
+    from workloads import CONFIGS, config_forest, make_gk, make_inputs
+    cfg = CONFIGS[GK_CONFIG]
+    fo = config_forest("cfg0b") if small else config_forest(GK_CONFIG).subset([0])
+    d = cfg["dk"]
+    inp = make_inputs(fo.n_tokens, 1, d, d, "bf16", 0)
+    gk = make_gk(fo.n_tokens, 1, d, 0)
+    t0 = time.perf_counter()
+    res = gk_oracle.forest_eval(fo, inp["q"], inp["k"], inp["v"], gk, inp["dO"])
+    dt = time.perf_counter() - t0
+    return {"value": fo.n_tokens / cfg["H"] / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"{'cfg0b tree' if small else GK_CONFIG + ' tree 0'}: {fo.n_tokens} compact / {res['S']} "
+                      f"trajectory-wise tokens, 1 of {cfg['H']} heads, fwd+bwd, {dt:.1f} s", "seconds": dt}
+
+
+class GkWorkload:
+    """One step = every forward round and every backward round (with the replay-gradient fold) of the per-channel-
+    decay calls on cfg2's forest (16 heads, d = 128, bf16)."""
+    metric, unit = GK_METRIC, UNIT
+
+    def __init__(self, args, ranks):
+        import torch
+        import paper_2608_28158_b200 as H
+        from workloads import CONFIGS, config_forest, make_gk, make_inputs
+        self.H, self.args, self.ranks = H, args, ranks
+        self.cfg = cfg = CONFIGS[GK_CONFIG]
+        fo = config_forest(GK_CONFIG)
+        self.plan = plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64).upload()
+        Hh, d = cfg["H"], cfg["dk"]
+        self.inp = inp = make_inputs(plan.C, Hh, d, d, "bf16", 60 + ranks.rank, device="cuda")
+        inp["g"] = make_gk(plan.C, Hh, d, 60 + ranks.rank, device="cuda")
+        cs, sc = H.harts_la_gk_workspace_bytes(plan.tables, Hh, d, d, H.HARTS_BF16)
+        self.slots = torch.empty(max(plan.n_slots, 1) * Hh * d * d, device="cuda")
+        self.cs = torch.empty(cs, dtype=torch.uint8, device="cuda")
+        self.scratch = torch.empty(sc, dtype=torch.uint8, device="cuda")
+        self.status = torch.zeros(4, dtype=torch.int32, device="cuda")
+        self.out = {"o": torch.empty_like(inp["v"]), "dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]),
+                    "dv": torch.empty_like(inp["v"]), "dg": torch.empty_like(inp["g"])}
+        self.units = plan.C
+        self.stream = torch.cuda.current_stream()
+
+    def step(self, marks):
+        import torch
+        H, plan, inp, out = self.H, self.plan, self.inp, self.out
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        a.record(self.stream)
+        H.harts_la_gk_fwd(plan, 0, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], self.slots, self.cs,
+                          dev_status=self.status)
+        b.record(self.stream)
+        H.harts_la_gk_bwd(plan, 0, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"], out["dq"], out["dk"], out["dv"],
+                          out["dg"], self.cs, self.scratch, dev_status=self.status)
+        c.record(self.stream)
+        if marks is not None:
+            marks += [("fwd", a, b), ("bwd", b, c)]
+
+    def check(self):
+        self.H.harts_la_check(self.status)
+
+    def e2e(self, n_steps):
+        return time_e2e(self, dict(self.inp), dict(self.out), n_steps, self.ranks)
+
+    def describe(self, ms_step, kernel_ms, peaks):
+        plan, cfg = self.plan, self.cfg
+        Hh, d = cfg["H"], cfg["dk"]
+        th = plan.C * Hh
+        # the contractions of the chunk form (as for the scalar gate) plus one exponential, one multiply and one add per
+        # (t, j <= t, channel) for the per-channel decay, in both passes
+        flops_fwd = th * (2 * 64 * d + 2 * 64 * d + 4 * d * d) + th * 33 * d * 3
+        flops_bwd = th * (5 * 2 * 64 * d + 4 * 2 * d * d) + th * 33 * d * 3
+        # fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x max SM clock
+        peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        K = plan.n_rounds
+        achieved = flops_bwd / (kernel_ms["bwd"] * 1e-3) / 1e12
+        return {"dtype": "f32",
+                "config": {"workload": "gk", "trees": GK_CONFIG, "H": Hh, "dk": d, "dv": d, "chunk": 64,
+                           "compact_tokens": plan.C, "rounds": K, "sequences": plan.n_seq,
+                           "inputs": "bf16 q, k, v, dO; fp32 per-channel log-decay; fp32 arithmetic on the CUDA cores",
+                           "l2": "inputs larger than L2"},
+                "roofline": {"bound": "alu", "kernel": "gk_bwd_kernel (all rounds)", "achieved": achieved, "peak": peak,
+                             "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                             "algorithmic_flops_per_launch": flops_bwd / K,
+                             "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                             "forward": {"achieved": flops_fwd / (kernel_ms["fwd"] * 1e-3) / 1e12,
+                                         "frac": flops_fwd / (kernel_ms["fwd"] * 1e-3) / 1e12 / peak},
+                             "whole_path": {"roof_ms": (flops_fwd + flops_bwd) / (peak * 1e12) * 1e3,
+                                            "frac_strict": (flops_fwd + flops_bwd) / (peak * 1e12) * 1e3 / ms_step}},
+                "gpu_launches_per_step": 2 * K + (K if plan.n_slots else 0) + (1 if plan.n_rg_rows else 0)}
+
+    def extras(self, ms_step):
+        return {}
+
+    def cpu_baseline(self):
+        return gk_oracle_sample()
+
+
+# --------------------------------------------------------------------------------------------------
 # Driver: one workload -> one JSON line
 # --------------------------------------------------------------------------------------------------
-WORKLOADS = {"logp": LogpWorkload, "conv": ConvWorkload, "attn": AttnWorkload}    # anything else: a cfg name
+WORKLOADS = {"logp": LogpWorkload, "conv": ConvWorkload, "attn": AttnWorkload, "gk": GkWorkload}    # anything else: a cfg name
 
 
 def workload_class(name):
@@ -908,7 +1012,7 @@ def other_paths(args, ranks):
     kernel times, roofline fraction and clocks of each, without their end-to-end and CPU legs."""
     import copy
     out = {}
-    for name in ("logp", "conv", "attn"):
+    for name in ("logp", "conv", "attn", "gk"):
         a = copy.copy(args)
         a.workload, a.steps, a.warmup, a.blocks = name, min(args.steps, 5), 3, 1
         try:
@@ -950,7 +1054,8 @@ def _la_sample(args, many_steps):
 REFERENCE_SAMPLES = {"la": _la_sample,
                      "logp": lambda args, many: logp_oracle_sample(small=many),
                      "conv": lambda args, many: conv_oracle_sample(small=many),
-                     "attn": lambda args, many: attn_oracle_sample(small=many)}
+                     "attn": lambda args, many: attn_oracle_sample(small=many),
+                     "gk": lambda args, many: gk_oracle_sample(small=many)}
 
 
 def reference_config(args):
@@ -960,6 +1065,8 @@ def reference_config(args):
         return CONV_METRIC, UNIT, {"workload": "conv", "D": 4096, "w": CONV_W}
     if args.workload == "attn":
         return ATTN_METRIC, UNIT, {"workload": "attn", "Hq": ATTN_H, "Hkv": ATTN_H, "d": ATTN_D}
+    if args.workload == "gk":
+        return GK_METRIC, UNIT, {"workload": "gk", "trees": GK_CONFIG, "H": 16, "dk": 128, "dv": 128, "chunk": 64}
     from workloads import CONFIGS
     cfg = CONFIGS[args.workload]
     return METRIC, UNIT, {"workload": args.workload, "H": cfg["H"], "dk": cfg["dk"], "dv": cfg["dv"], "chunk": 64}

@@ -41,11 +41,13 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // already set by an earlier one.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, volatile int* dead,
                                           unsigned long long limit_ns = WAIT_LIMIT_NS) {
-    // a healthy wait ends within these polls; the timer (slow to read) is consulted only after them
-#pragma unroll 1
-    for (int i = 0; i < 4096; i++)
-        if (mbar_try(bar, parity)) return true;
     if (*dead) return false;
+    // a healthy wait ends within these polls; the timer is consulted only after them
+#pragma unroll 1
+    for (int i = 0; i < 2048; i++) {
+        if (mbar_try(bar, parity)) return true;
+        if ((i & 255) == 255 && *dead) return false;
+    }
     const unsigned long long t0 = global_ns();
     for (int round = 0; round < (1 << 24); round++) {            // the poll count is bounded too, should the timer stall
 #pragma unroll 1
