@@ -13,8 +13,8 @@
 //   dv_j    = sum_{t>=j} A_tj dO_t + (k_j .* e^{b_n-b_j}) dS
 //   dg_t[i] = sum_{tau>=t} (q_tau[i] dq_tau[i] - k_tau[i] dk_tau[i]) + <S_{c+1}[i,:], dS[i,:]>
 //   dS     <- Diag(e^{b_n}) dS + sum_t (q_t .* e^{b_t})^T dO_t
-// In the backward one thread owns one key channel i for the decay-dependent sums, so that every e^{b_t[i]-b_j[i]} is
-// evaluated once and serves dq and dk alike.
+// In the backward a pair of threads owns one key channel i for the decay-dependent sums, so that every
+// e^{b_t[i]-b_j[i]} is evaluated once and serves dq and dk alike.
 #include "kernels.h"
 
 namespace harts {
@@ -53,6 +53,70 @@ __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq
     return s;
 }
 
+// One [BT][D] tile of a [rows, H, D] tensor into shared memory: every thread fetches its 16-byte pieces first (all in
+// flight together), then scatters them element by element into the rotated layout.  need_own: only rows with an
+// output are taken (q, dO); otherwise every valid row (k, v).  Rows that are not taken become zero.
+template <typename T, int D, bool ROTATED, typename Dst>
+__device__ __forceinline__ void load_tile(const T* src, int H, int h, const int* srow, bool need_own, Dst* dst) {
+    constexpr int VE = 16 / sizeof(T);                    // elements per piece
+    constexpr int PER_ROW = D / VE;
+    constexpr int N = BT * PER_ROW / NT;                  // pieces per thread
+    static_assert(BT * PER_ROW % NT == 0, "tile does not divide over the threads");
+    uint4 buf[N];
+#pragma unroll
+    for (int u = 0; u < N; u++) {
+        const int p = threadIdx.x + u * NT, t = p / PER_ROW, part = p % PER_ROW, code = srow[t];
+        const bool take = need_own ? code >= 0 : code != -1;
+        const int r = code >= 0 ? code : -2 - code;
+        buf[u] = take ? *reinterpret_cast<const uint4*>(src + ((size_t)r * H + h) * D + part * VE) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < N; u++) {
+        const int p = threadIdx.x + u * NT, t = p / PER_ROW, part = p % PER_ROW;
+        const T* el = reinterpret_cast<const T*>(&buf[u]);
+#pragma unroll
+        for (int x = 0; x < VE; x++) {
+            const int i = part * VE + x;
+            dst[ROTATED ? tix<D>(t, i) : t * D + i] = static_cast<Dst>(el[x]);
+        }
+    }
+}
+
+// A [DK][DV] state from global memory (plain layout) into the rotated shared-memory layout, or back.
+template <typename Src, typename Dst, int DK, int DV, bool ADD>
+__device__ __forceinline__ void load_state(const Src* src, Dst* dst) {
+    constexpr int VE = 16 / sizeof(Src);
+    constexpr int N = DK * DV / VE / NT;
+    uint4 buf[N];
+#pragma unroll
+    for (int u = 0; u < N; u++) buf[u] = reinterpret_cast<const uint4*>(src)[threadIdx.x + u * NT];
+#pragma unroll
+    for (int u = 0; u < N; u++) {
+        const int e0 = (threadIdx.x + u * NT) * VE;
+        const Src* el = reinterpret_cast<const Src*>(&buf[u]);
+#pragma unroll
+        for (int x = 0; x < VE; x++) {
+            const int e = e0 + x, idx = tix<DV>(e / DV, e % DV);
+            if (ADD) dst[idx] += static_cast<Dst>(el[x]);
+            else dst[idx] = static_cast<Dst>(el[x]);
+        }
+    }
+}
+template <typename Dst, int DK, int DV>
+__device__ __forceinline__ void store_state(const float* sS, Dst* dst) {
+    constexpr int VE = 16 / sizeof(Dst);
+    for (int p = threadIdx.x; p < DK * DV / VE; p += NT) {
+        uint4 out;
+        Dst* el = reinterpret_cast<Dst*>(&out);
+#pragma unroll
+        for (int x = 0; x < VE; x++) {
+            const int e = p * VE + x;
+            el[x] = from_f<Dst>(sS[tix<DV>(e / DV, e % DV)]);
+        }
+        reinterpret_cast<uint4*>(dst)[p] = out;
+    }
+}
+
 // Loads one chunk: row codes (physical row >= 0 own, -2 - row replayed, -1 past the end), k/v of all valid rows, q and
 // dO of own rows (zero elsewhere), and the per-channel running sum of g (rows past the end add nothing).
 template <typename T, int DK, int DV, bool BWD>
@@ -67,21 +131,11 @@ __device__ void load_chunk(const harts_la_tables_t& tb, const SeqInfo& s, int c,
         srow[tid] = code;
     }
     __syncthreads();
-    for (int e = tid; e < BT * DK; e += NT) {
-        const int t = e / DK, i = e % DK, code = srow[t];
-        const int r = code >= 0 ? code : -2 - code;
-        const size_t off = ((size_t)r * H + h) * DK + i;
-        sk[tix<DK>(t, i)] = code == -1 ? from_f<T>(0.f) : k[off];
-        sq[tix<DK>(t, i)] = code >= 0 ? q[off] : from_f<T>(0.f);
-        sb[t * DK + i] = code == -1 ? 0.f : gk[off];
-    }
-    for (int e = tid; e < BT * DV; e += NT) {
-        const int t = e / DV, j = e % DV, code = srow[t];
-        const int r = code >= 0 ? code : -2 - code;
-        const size_t off = ((size_t)r * H + h) * DV + j;
-        sv[tix<DV>(t, j)] = code == -1 ? from_f<T>(0.f) : v[off];
-        if (BWD) sdo[tix<DV>(t, j)] = code >= 0 ? dO[off] : from_f<T>(0.f);
-    }
+    load_tile<T, DK, true>(k, H, h, srow, false, sk);
+    load_tile<T, DK, true>(q, H, h, srow, true, sq);
+    load_tile<float, DK, false>(gk, H, h, srow, false, sb);
+    load_tile<T, DV, true>(v, H, h, srow, false, sv);
+    if (BWD) load_tile<T, DV, true>(dO, H, h, srow, true, sdo);
     __syncthreads();
     if (tid < DK) {
         float acc = 0.f;
@@ -149,8 +203,10 @@ __global__ void __launch_bounds__(NT) gk_fwd_kernel(harts_la_tables_t tb, int se
     const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)DK * DV;
 
-    for (int e = tid; e < DK * DV; e += NT)
-        sS[tix<DV>(e / DV, e % DV)] = s.init_slot < 0 ? 0.f : slots[((size_t)s.init_slot * H + h) * state_elems + e];
+    if (s.init_slot < 0)
+        for (int e = tid; e < DK * DV; e += NT) sS[e] = 0.f;
+    else
+        load_state<float, float, DK, DV, false>(slots + ((size_t)s.init_slot * H + h) * state_elems, sS);
     __syncthreads();
 
     int next_req = s.req_lo;
@@ -158,12 +214,10 @@ __global__ void __launch_bounds__(NT) gk_fwd_kernel(harts_la_tables_t tb, int se
         load_chunk<T, DK, DV, false>(tb, s, c, h, H, q, k, v, gk, nullptr, sq, sk, sv, nullptr, sb, srow);
         // start-of-chunk state: kept for the backward; exported when the plan requests this boundary
         if (chunk_states) {
-            T* dst = chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems;
-            for (int e = tid; e < DK * DV; e += NT) dst[e] = from_f<T>(sS[tix<DV>(e / DV, e % DV)]);
+            store_state<T, DK, DV>(sS, chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems);
         }
         if (next_req < s.req_hi && tb.slot_chunk[next_req] == c) {
-            float* dst = slots + ((size_t)next_req * H + h) * state_elems;
-            for (int e = tid; e < DK * DV; e += NT) dst[e] = sS[tix<DV>(e / DV, e % DV)];
+            store_state<float, DK, DV>(sS, slots + ((size_t)next_req * H + h) * state_elems);
             next_req++;
         }
         intra_scores<T, DK, DV, false>(sq, sk, sv, nullptr, sb, sA, nullptr);
@@ -276,34 +330,37 @@ __global__ void __launch_bounds__(NT) gk_bwd_kernel(harts_la_tables_t tb, int se
         // buffer by handoff_reduce)
         if (next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1) {
             if (tb.slot_cons_ptr[next_req] < tb.slot_cons_ptr[next_req + 1]) {
-                const float* src = ds0 + ((size_t)tb.slot_cons_seq[tb.slot_cons_ptr[next_req]] * H + h) * state_elems;
-                for (int e = tid; e < DK * DV; e += NT) sdS[tix<DV>(e / DV, e % DV)] += src[e];
+                load_state<float, float, DK, DV, true>(
+                    ds0 + ((size_t)tb.slot_cons_seq[tb.slot_cons_ptr[next_req]] * H + h) * state_elems, sdS);
             }
             next_req--;
         }
         load_chunk<T, DK, DV, true>(tb, s, c, h, H, q, k, v, gk, dO, sq, sk, sv, sdo, sb, srow);
         {
-            const T* src = chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems;
-            for (int e = tid; e < DK * DV; e += NT) sS[tix<DV>(e / DV, e % DV)] = src[e];
+            load_state<T, T, DK, DV, false>(chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems, sS);
         }
         intra_scores<T, DK, DV, true>(sq, sk, sv, sdo, sb, sA, sdA);
         __syncthreads();
-        // ---- one thread per key channel i: dq, dk, dg of the chunk, rows in reverse ---------------------------------
-        if (tid < DK) {
-            const int i = tid;
+        // ---- two threads per key channel i (lanes 2i, 2i+1): dq, dk, dg of the chunk, rows in reverse.  Thread hh of the
+        //      pair takes the state columns jj = hh (mod 2) of the two row-dots and the rows j = hh (mod 2) of the
+        //      decay-dependent sums, so that it alone accumulates dk_j for its rows; partial sums meet by shuffles.
+        if (tid < 2 * DK) {
+            const int i = tid >> 1, hh = tid & 1;
+            const unsigned pair_mask = 0x3u << ((tid & 31) & ~1);
             const float bn = sb[(BT - 1) * DK + i];
-            float dk_acc[BT];
+            float dk_acc[BT / 2];                          // rows j = 2 * jh + hh
 #pragma unroll
-            for (int j = 0; j < BT; j++) dk_acc[j] = 0.f;
+            for (int jh = 0; jh < BT / 2; jh++) dk_acc[jh] = 0.f;
             float rowdot = 0.f;                            // <S_c[i,:], dS[i,:]>
-            for (int jj = 0; jj < DV; jj++) rowdot += to_f(sS[tix<DV>(i, jj)]) * sdS[tix<DV>(i, jj)];
+            for (int jj = hh; jj < DV; jj += 2) rowdot += to_f(sS[tix<DV>(i, jj)]) * sdS[tix<DV>(i, jj)];
+            rowdot += __shfl_xor_sync(pair_mask, rowdot, 1);
             float suffix = 0.f, g_inter = 0.f;
 #pragma unroll
             for (int t = BT - 1; t >= 0; t--) {
                 const int code = srow[t];
-                if (code == -1) continue;                  // past the end: nothing there
+                if (code == -1) continue;                  // past the end: nothing there (the same for the whole CTA)
                 float iq = 0.f, ik = 0.f;                  // (dO_t S_c^T)[i], (v_t dS^T)[i]
-                for (int jj = 0; jj < DV; jj++) {
+                for (int jj = hh; jj < DV; jj += 2) {
                     iq += to_f(sdo[tix<DV>(t, jj)]) * to_f(sS[tix<DV>(i, jj)]);
                     ik += to_f(sv[tix<DV>(t, jj)]) * sdS[tix<DV>(i, jj)];
                 }
@@ -311,34 +368,45 @@ __global__ void __launch_bounds__(NT) gk_bwd_kernel(harts_la_tables_t tb, int se
                 const float qt = to_f(sq[tix<DK>(t, i)]), kt = to_f(sk[tix<DK>(t, i)]);
                 float dq_acc = 0.f;
 #pragma unroll
-                for (int j = 0; j <= t; j++) {
-                    const float x = sdA[t * BT + j] * __expf(bt - sb[j * DK + i]);   // one exponential for dq and dk
-                    dq_acc += x * to_f(sk[tix<DK>(j, i)]);
-                    dk_acc[j] += x * qt;
+                for (int jh = 0; 2 * jh <= t; jh++) {
+                    const int j = 2 * jh + hh;
+                    if (j <= t) {
+                        const float x = sdA[t * BT + j] * __expf(bt - sb[j * DK + i]);   // one exponential for dq and dk
+                        dq_acc += x * to_f(sk[tix<DK>(j, i)]);
+                        dk_acc[jh] += x * qt;
+                    }
                 }
+                iq += __shfl_xor_sync(pair_mask, iq, 1);
+                ik += __shfl_xor_sync(pair_mask, ik, 1);
+                dq_acc += __shfl_xor_sync(pair_mask, dq_acc, 1);
+                // row t has received all its contributions (rows >= t are done); its owner is thread t mod 2 of the pair
+                const float dk_intra = __shfl_sync(pair_mask, dk_acc[t >> 1], ((tid & 31) & ~1) + (t & 1));
                 const float ew = __expf(bn - bt);
                 const float dqv = dq_acc + __expf(bt) * iq;
-                const float dkv = dk_acc[t] + ew * ik;     // row t has received all its contributions (rows >= t are done)
+                const float dkv = dk_intra + ew * ik;
                 g_inter += kt * ew * ik;
                 suffix += qt * dqv - kt * dkv;
-                if (code >= 0) {
-                    const size_t off = ((size_t)code * H + h) * DK + i;
-                    dq[off] = from_f<T>(dqv);
-                    dk_[off] = from_f<T>(dkv);
-                    dgk[off] = suffix;
-                } else {                                   // replayed rows sit in chunk 0: virtual row = t
-                    const size_t off = ((size_t)(s.replay_base + t) * H + h) * DK + i;
-                    rk[off] = dkv;
-                    rg[off] = suffix;
+                if (hh == 0) {
+                    if (code >= 0) {
+                        const size_t off = ((size_t)code * H + h) * DK + i;
+                        dq[off] = from_f<T>(dqv);
+                        dk_[off] = from_f<T>(dkv);
+                        dgk[off] = suffix;
+                    } else {                               // replayed rows sit in chunk 0: virtual row = t
+                        const size_t off = ((size_t)(s.replay_base + t) * H + h) * DK + i;
+                        rk[off] = dkv;
+                        rg[off] = suffix;
+                    }
                 }
             }
             // every row of the chunk also gets <S_{c+1}[i,:], dS[i,:]> = e^{b_n[i]} <S_c[i,:], dS[i,:]> + sum_j k_j[i] dk_j(inter)[i]
             const float G = __expf(bn) * rowdot + g_inter;
-            for (int t = 0; t < BT; t++) {
-                const int code = srow[t];
-                if (code >= 0) dgk[((size_t)code * H + h) * DK + i] += G;
-                else if (code < -1) rg[((size_t)(s.replay_base + t) * H + h) * DK + i] += G;
-            }
+            if (hh == 0)
+                for (int t = 0; t < BT; t++) {
+                    const int code = srow[t];
+                    if (code >= 0) dgk[((size_t)code * H + h) * DK + i] += G;
+                    else if (code < -1) rg[((size_t)(s.replay_base + t) * H + h) * DK + i] += G;
+                }
         }
         __syncthreads();
         scale_qk<T, DK>(sq, sk, sb);
@@ -399,8 +467,7 @@ __global__ void __launch_bounds__(NT) gk_bwd_kernel(harts_la_tables_t tb, int se
         __syncthreads();
     }
     if (s.init_slot >= 0) {
-        float* dst = ds0 + ((size_t)seq * H + h) * state_elems;
-        for (int e = tid; e < DK * DV; e += NT) dst[e] = sdS[tix<DV>(e / DV, e % DV)];
+        store_state<float, DK, DV>(sdS, ds0 + ((size_t)seq * H + h) * state_elems);
     }
 }
 
