@@ -212,6 +212,22 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
                      int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream);
 
 /*
+ * One whole step on HOST buffers (the end-to-end form of Eq. 16's round loop): copies q, k, v, g, dO (physical row
+ * order, layouts as above) from host memory into the caller's device tensors, runs every forward round and every
+ * backward round with the replay-gradient fold, and copies o, dq, dk, dv, dg back -- all enqueued on `stream`, in
+ * that order, without synchronising (the host results are complete once the stream has drained; use pinned host
+ * memory for the copies to be asynchronous).  host_*: HOST pointers; dev_*, slots, chunk_states, scratch: caller-owned
+ * DEVICE buffers of the sizes harts_la_fwd / harts_la_bwd expect (the library allocates nothing).
+ * Errors: HARTS_EINVAL (a missing buffer), HARTS_ECUDA (a copy could not be enqueued), those of harts_la_fwd / _bwd.
+ */
+int32_t harts_la_step_host(const harts_la_plan_t* plan, const void* dev_blob, const void* host_q, const void* host_k,
+                           const void* host_v, const float* host_g, const void* host_dO, void* host_o, void* host_dq,
+                           void* host_dk, void* host_dv, float* host_dg, void* dev_q, void* dev_k, void* dev_v,
+                           float* dev_g, void* dev_dO, void* dev_o, void* dev_dq, void* dev_dk, void* dev_dv,
+                           float* dev_dg, float* slots, void* chunk_states, void* scratch, int32_t H, int32_t dk,
+                           int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream);
+
+/*
  * The same path for the recurrence with a PER-CHANNEL decay, the first term of Eq. 1 (Section 2.2, the Diag(gamma)
  * decay on the key dimension of the state; Section 4.1 names a backend of this family as the one evaluated):
  *

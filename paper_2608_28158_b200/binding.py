@@ -66,6 +66,8 @@ def _load():
     lib.harts_la_expand.argtypes = [i32, _I32P, _I32P, _I32P, _I32P, C.c_int64, C.c_int64, _I32P, C.POINTER(C.c_int64),
                                     C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
     lib.harts_la_expand.restype = i32
+    lib.harts_la_step_host.argtypes = [vp, vp] + [vp] * 23 + [i32] * 4 + [u32, vp, vp]
+    lib.harts_la_step_host.restype = i32
     lib.harts_la_gk_workspace_bytes.argtypes = [C.POINTER(Tables), i32, i32, i32, i32, C.POINTER(sz), C.POINTER(sz)]
     lib.harts_la_gk_fwd.argtypes = [vp, vp, i32] + [vp] * 7 + [i32] * 4 + [u32, vp, vp]
     lib.harts_la_gk_bwd.argtypes = [vp, vp, i32] + [vp] * 11 + [i32] * 4 + [u32, vp, vp]
@@ -287,14 +289,21 @@ def run_fwd_bwd(plan: Plan, ws: Workspace, q, k, v, g, dO, out=None, backward=Tr
     return out
 
 
+def harts_la_step_host(plan, ws, host_in: dict, dev_in: dict, dev_out: dict, host_out: dict, stream=None):
+    """One step on HOST buffers through the library: inputs copied in, all rounds forward and backward, results copied
+    out, everything enqueued on one stream (no synchronisation here)."""
+    H, dk, dv, dt = _dims(dev_in["q"], dev_in["v"])
+    args = [_ptr(host_in[n]) for n in ("q", "k", "v", "g", "dO")] + [_ptr(host_out[n]) for n in ("o", "dq", "dk", "dv", "dg")]
+    args += [_ptr(dev_in[n]) for n in ("q", "k", "v", "g", "dO")] + [_ptr(dev_out[n]) for n in ("o", "dq", "dk", "dv", "dg")]
+    _check(lib.harts_la_step_host(plan._h, _ptr(plan.blob), *args, _ptr(ws.slots), _ptr(ws.chunk_states),
+                                  _ptr(ws.scratch), H, dk, dv, dt, ws.flags, _ptr(ws.dev_status), _stream(stream)),
+           "harts_la_step_host")
+
+
 def run_fwd_bwd_host(plan: Plan, ws: Workspace, host_in: dict, dev_in: dict, dev_out: dict, host_out: dict):
-    """End-to-end step on HOST buffers: pinned host inputs -> device, all rounds forward and backward,
-    outputs -> pinned host buffers.  Buffers are preallocated by the caller; returns after a sync."""
-    for n in ("q", "k", "v", "g", "dO"):
-        dev_in[n].copy_(host_in[n], non_blocking=True)
-    run_fwd_bwd(plan, ws, dev_in["q"], dev_in["k"], dev_in["v"], dev_in["g"], dev_in["dO"], out=dev_out)
-    for n in ("o", "dq", "dk", "dv", "dg"):
-        host_out[n].copy_(dev_out[n], non_blocking=True)
+    """End-to-end step on HOST buffers (harts_la_step_host), then a synchronisation.  Buffers are preallocated by the
+    caller."""
+    harts_la_step_host(plan, ws, host_in, dev_in, dev_out, host_out)
     torch.cuda.current_stream().synchronize()
     return host_out
 

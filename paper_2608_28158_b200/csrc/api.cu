@@ -144,6 +144,39 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
     return HARTS_OK;
 }
 
+int32_t harts_la_step_host(const harts_la_plan_t* plan, const void* dev_blob, const void* host_q, const void* host_k,
+                           const void* host_v, const float* host_g, const void* host_dO, void* host_o, void* host_dq,
+                           void* host_dk, void* host_dv, float* host_dg, void* dev_q, void* dev_k, void* dev_v,
+                           float* dev_g, void* dev_dO, void* dev_o, void* dev_dq, void* dev_dk, void* dev_dv,
+                           float* dev_dg, float* slots, void* chunk_states, void* scratch, int32_t H, int32_t dk,
+                           int32_t dv, int32_t dtype, uint32_t flags, int32_t* dev_status, void* stream) {
+    const harts::Plan* p = harts_la_plan_internal(plan);
+    if (!p || H < 1 || dk < 1 || dv < 1) return HARTS_EINVAL;
+    if (dtype != HARTS_FP32 && dtype != HARTS_BF16) return HARTS_EUNSUPPORTED;
+    if (!host_q || !host_k || !host_v || !host_g || !host_dO || !host_o || !host_dq || !host_dk || !host_dv || !host_dg)
+        return HARTS_EINVAL;
+    const size_t elem = dtype == HARTS_FP32 ? 4 : 2, rows = (size_t)p->n_rows * H;
+    const size_t nk = rows * dk * elem, nv = rows * dv * elem, ng = rows * sizeof(float);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const struct { void* dst; const void* src; size_t n; } in[5] = {
+        {dev_q, host_q, nk}, {dev_k, host_k, nk}, {dev_v, host_v, nv}, {dev_g, host_g, ng}, {dev_dO, host_dO, nv}};
+    for (const auto& c : in) {
+        if (!c.dst) return HARTS_EINVAL;
+        if (cudaMemcpyAsync(c.dst, c.src, c.n, cudaMemcpyHostToDevice, s) != cudaSuccess) return HARTS_ECUDA;
+    }
+    int32_t rc = harts_la_fwd(plan, dev_blob, 0, dev_q, dev_k, dev_v, dev_g, dev_o, slots, chunk_states, H, dk, dv, dtype,
+                              flags, dev_status, stream);
+    if (rc != HARTS_OK) return rc;
+    rc = harts_la_bwd(plan, dev_blob, 0, dev_q, dev_k, dev_v, dev_g, dev_dO, dev_dq, dev_dk, dev_dv, dev_dg, chunk_states,
+                      scratch, H, dk, dv, dtype, flags, dev_status, stream);
+    if (rc != HARTS_OK) return rc;
+    const struct { void* dst; const void* src; size_t n; } out[5] = {
+        {host_o, dev_o, nv}, {host_dq, dev_dq, nk}, {host_dk, dev_dk, nk}, {host_dv, dev_dv, nv}, {host_dg, dev_dg, ng}};
+    for (const auto& c : out)
+        if (cudaMemcpyAsync(c.dst, c.src, c.n, cudaMemcpyDeviceToHost, s) != cudaSuccess) return HARTS_ECUDA;
+    return HARTS_OK;
+}
+
 // ---- per-channel decay (the Diag(gamma) term of Eq. 1) -------------------------------------------------------------------
 int32_t harts_la_gk_workspace_bytes(const harts_la_tables_t* tb, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
                                     size_t* chunk_state_bytes, size_t* scratch_bytes) {

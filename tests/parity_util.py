@@ -46,14 +46,41 @@ def to_physical(plan, canon: dict, device="cuda"):
     return out
 
 
+GUARD = 4096      # elements of guard band on either side of every output tensor
+
+
+def guarded_like(x):
+    """A tensor like x that sits between two guard bands filled with a bit pattern no kernel produces; check() fails if
+    anything was written outside the tensor (canary rows around every output)."""
+    n = x.numel()
+    flat = torch.empty(n + 2 * GUARD, dtype=x.dtype, device=x.device)
+    pattern = torch.full((1,), -12345.0, dtype=x.dtype, device=x.device)
+    flat[:GUARD] = pattern
+    flat[GUARD + n:] = pattern
+    view = flat[GUARD:GUARD + n].view(x.shape)
+    view.fill_(float("nan"))
+
+    def check():
+        assert bool((flat[:GUARD] == pattern).all()) and bool((flat[GUARD + n:] == pattern).all()), "write outside an output"
+    return view, check
+
+
 def run_gpu(fo, inp_canon, flags=0, backward=True, chunk=64):
-    """Returns (plan, outputs in CANONICAL order as device tensors)."""
+    """Returns (plan, outputs in CANONICAL order as device tensors).  Every output sits between guard bands that must
+    come back untouched, and starts as NaN so that a row nobody wrote shows up."""
     plan = plan_of(fo, chunk).upload()
     phys = to_physical(plan, inp_canon)
     H_, dk, dv = phys["q"].shape[1], phys["q"].shape[2], phys["v"].shape[2]
     ws = H.Workspace(plan, H_, dk, dv, phys["q"].dtype, flags)
-    out = H.run_fwd_bwd(plan, ws, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"], backward=backward)
+    like = {"o": phys["v"], "dq": phys["q"], "dk": phys["k"], "dv": phys["v"], "dg": phys["g"]}
+    out, checks = {}, []
+    for n in (("o", "dq", "dk", "dv", "dg") if backward else ("o",)):
+        out[n], chk = guarded_like(like[n])
+        checks.append(chk)
+    H.run_fwd_bwd(plan, ws, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"], out=out, backward=backward)
     H.harts_la_check(ws.dev_status)
+    for chk in checks:
+        chk()
     rows = torch.as_tensor(plan.row_of_token.astype(np.int64), device="cuda")
     return plan, {n: x[rows] for n, x in out.items()}
 
