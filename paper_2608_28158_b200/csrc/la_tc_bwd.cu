@@ -16,7 +16,8 @@
 // started there (read from the scratch area, where those sequences' calls left them).
 // S_c comes from the chunk-state workspace written by the forward ([d_k][d_v] bf16 per chunk-head).
 // Gradients of replayed rows go to the scratch area (fp32) and are folded into their ancestor rows by
-// the replay-reduce kernel.  Every wait is bounded; one that runs out sets the status word and a CTA-wide latch, and the
+// the replay-reduce kernel.  Full chunks (all 64 rows own rows, nearly all of them) take the matrix-fragment epilogue
+// (tcgen05.ld 16x256b, ldmatrix / stmatrix transposing, swizzled staging panels, TMA stores).  Every wait is bounded; one that runs out sets the status word and a CTA-wide latch, and the
 // CTA leaves its loops at the end of the chunk, drains what it has in flight, releases tensor memory and returns.
 #include "kernels.h"
 #include "tc_common.cuh"
@@ -103,13 +104,12 @@ __device__ __forceinline__ float warp_transpose_reduce16(float (&z)[16], int lan
     return z[0] + __shfl_xor_sync(0xffffffffu, z[0], 16);
 }
 
-// Epilogue of one chunk for this thread's feature index L and its 16 rows, in three parts that follow the three
-// commits of the MMA batch (dk, dv, dq: the longest part first, so that little is left after the last MMA).  qk[e] holds q[t][L] (low half) and k[t][L] (high half) as bf16 bits, read
-// from the tiles before the batch so that the tiles can be reloaded while the epilogue runs.  The outputs are staged
-// in shared memory ([row][feature], plain layout).  FULL: all 64 rows are own rows and leave by one TMA store per
-// tensor; otherwise the compute warps copy the valid rows out after the epilogue (own rows to the outputs, replayed
-// rows, staged in fp32, to the scratch).
-template <bool FULL>
+// ---- partial chunks (a ragged tail, or chunk 0 of a sequence that replays ancestor rows) ------------------------------
+// Epilogue for this thread's feature index L and its 16 rows, in three parts that follow the three commits of the MMA
+// batch (dk, dv, dq: the longest part first, so that little is left after the last MMA).  qk[e] holds q[t][L] (low
+// half) and k[t][L] (high half) as bf16 bits, read from the tiles before the batch so that the tiles can be reloaded
+// while the epilogue runs.  The outputs are staged in shared memory ([row][feature], plain layout); the compute warps
+// copy the valid rows out after the epilogue (own rows to the outputs, replayed rows, staged in fp32, to the scratch).
 __device__ __forceinline__ void epilogue_dq(const RowData& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
                                             int h, const uint32_t (&qk)[16], __nv_bfloat16* dq, float (&z)[16]) {
     const int t0 = grp * 16;
@@ -121,14 +121,13 @@ __device__ __forceinline__ void epilogue_dq(const RowData& m, unsigned char* sme
         const int t = t0 + e;
         const float dqv = __uint_as_float(xq[e]);
         const float qv = __uint_as_float(qk[e] << 16);
-        z[e] += (FULL || m.code[t] != -1) ? qv * dqv : 0.f;
+        z[e] += (m.code[t] != -1) ? qv * dqv : 0.f;
         // replayed rows have no dq; their row of this staging tile holds one half of their fp32 dk (epilogue_dk)
-        if (FULL || m.code[t] >= -1)
+        if (m.code[t] >= -1)
             *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dq + t * 256 + L * 2) = __float2bfloat16_rn(dqv);
     }
 }
 
-template <bool FULL>
 __device__ __forceinline__ void epilogue_dk(const RowData& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
                                             int h, int replay_base, const uint32_t (&qk)[16], __nv_bfloat16* dk_,
                                             float* rk, float (&z)[16], float& g_part) {
@@ -143,19 +142,18 @@ __device__ __forceinline__ void epilogue_dk(const RowData& m, unsigned char* sme
         const float kv = __uint_as_float(qk[e] & 0xffff0000u);
         const float inter = m.w[t] * __uint_as_float(xe[e]);
         const float dkv = __uint_as_float(xi[e]) + inter;
-        const bool row_ok = FULL || m.code[t] != -1;
+        const bool row_ok = m.code[t] != -1;
         z[e] = row_ok ? -kv * dkv : 0.f;
         g_part += row_ok ? kv * inter : 0.f;
         // replayed rows (chunk 0 only) keep fp32: features 0..63 in the row's 256 bytes of the dk staging tile,
         // 64..127 in its row of the dq staging tile (replayed rows have no dq); every operand tile is still being read
-        if (!FULL && m.code[t] < -1)
+        if (m.code[t] < -1)
             *reinterpret_cast<float*>(smem + (L < 64 ? Smem::stage_dk : Smem::stage_dq) + t * 256 + (L & 63) * 4) = dkv;
         else
             *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dk + t * 256 + L * 2) = __float2bfloat16_rn(dkv);
     }
 }
 
-template <bool FULL>
 __device__ __forceinline__ void epilogue_dv(const RowData& m, unsigned char* smem, uint32_t tm_lane, int grp, int L, int H,
                                             int h, int replay_base, __nv_bfloat16* dv_, float* rv) {
     const int t0 = grp * 16;
@@ -169,7 +167,38 @@ __device__ __forceinline__ void epilogue_dv(const RowData& m, unsigned char* sme
         const float dvv = __uint_as_float(xi[e]) + m.w[t] * __uint_as_float(xe[e]);
         *reinterpret_cast<__nv_bfloat16*>(smem + Smem::stage_dv + t * 256 + L * 2) = __float2bfloat16_rn(dvv);
         // replayed rows: fp32 over the bf16 copy of dS, which no MMA reads once the dk and dv groups are done
-        if (!FULL && m.code[t] < -1) *reinterpret_cast<float*>(smem + Smem::ds + t * 512 + L * 4) = dvv;
+        if (m.code[t] < -1) *reinterpret_cast<float*>(smem + Smem::ds + t * 512 + L * 4) = dvv;
+    }
+}
+
+// ---- full chunks: the epilogue in matrix-fragment layout -------------------------------------------------------------
+// All 64 rows of the chunk are own rows.  A warp covers 32 features (its tensor-memory lane quarter) x 16 rows t (its
+// column group); tcgen05.ld hands every thread 16 values as fragments of 8x8 matrices: features f = m + 8 fa
+// (m = lane >> 2, fa = 0..3), rows t = t0 + 8 ta + 2 c + {0, 1} (c = lane & 3, ta = 0, 1).  q and k arrive in the same
+// layout by ldmatrix (transposing), the outputs leave by stmatrix (transposing) into 128-byte-swizzled [row][64
+// features] panels that TMA stores pick up: no 2-byte shared-memory accesses and no transposed reads.
+struct Frag {
+    uint32_t q[2][4], k[2][4];      // [ta][fa], two bf16 per register: rows t, t + 1
+};
+// value index -> (fa, ta, low/high row of the pair) for register r of load l (l = 0: lanes +0, l = 1: lanes +16)
+__device__ __forceinline__ float frag_elem(const uint32_t (&f)[2][4], int l, int r) {
+    const uint32_t pair = f[r >> 2][2 * l + ((r >> 1) & 1)];
+    return __uint_as_float((r & 1) ? (pair & 0xffff0000u) : (pair << 16));
+}
+__device__ __forceinline__ uint32_t frag_addr(uint32_t tile, int lane, int Lq, int t0, int ta) {
+    const int f = Lq + 8 * (lane >> 3), t = t0 + 8 * ta + (lane & 7);
+    return tile + (f >> 6) * PANEL + sw128_chunk(t, (f & 63) >> 3);
+}
+__device__ __forceinline__ void frag_store(uint32_t stage, int lane, int Lq, int t0, const float (&val)[2][8]) {
+#pragma unroll
+    for (int ta = 0; ta < 2; ta++) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int fa = 0; fa < 4; fa++) {
+            const int l = fa >> 1, r = 4 * ta + 2 * (fa & 1);
+            pk[fa] = pack_bf16(val[l][r], val[l][r + 1]);
+        }
+        stmatrix_x4_trans(frag_addr(stage, lane, Lq, t0, ta), pk);
     }
 }
 
@@ -533,6 +562,92 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         }
         if (is_aux && c > 0) store_rows(m.rows[cur ^ 1], nx_code, nx_g);   // visible to the others at barrier (B)
         if (is_compute) {
+            if (full) {
+                const int c4 = lane & 3, Lq = (warp & 3) * 32, t0 = grp * 16;
+                Frag fr;
+#pragma unroll
+                for (int ta = 0; ta < 2; ta++) {
+                    ldmatrix_x4_trans(frag_addr(aQ, lane, Lq, t0, ta), fr.q[ta]);
+                    ldmatrix_x4_trans(frag_addr(aK, lane, Lq, t0, ta), fr.k[ta]);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&m.bar_qk_read);
+                // e^{b_n - b_t} of this thread's four rows: t0 + 2c, +1, t0 + 8 + 2c, +1
+                const float2 wlo = *reinterpret_cast<const float2*>(rd.w + t0 + 2 * c4);
+                const float2 whi = *reinterpret_cast<const float2*>(rd.w + t0 + 8 + 2 * c4);
+                const float wv[4] = {wlo.x, wlo.y, whi.x, whi.y};
+                float zf[4] = {0.f, 0.f, 0.f, 0.f};              // q.dq - k.dk over this thread's features, per row
+                float val[2][8];
+                uint32_t xi[2][8], xe[2][8];
+                // ---- dk -----------------------------------------------------------------------------------------------
+                mbar_wait(&m.bar_o, ph_o, status, &m.dead);
+                tc_fence_after();
+#pragma unroll
+                for (int l = 0; l < 2; l++) {
+                    tmem_ld_frag16(tm_lane + ((uint32_t)(16 * l) << 16) + COL_DK + t0, xi[l]);
+                    tmem_ld_frag16(tm_lane + ((uint32_t)(16 * l) << 16) + COL_A + t0, xe[l]);
+                }
+                tmem_ld_wait();
+#pragma unroll
+                for (int l = 0; l < 2; l++)
+#pragma unroll
+                    for (int r = 0; r < 8; r++) {
+                        const int ti = 2 * (r >> 2) + (r & 1);
+                        const float kv = frag_elem(fr.k, l, r);
+                        const float inter = wv[ti] * __uint_as_float(xe[l][r]);
+                        const float dkv = __uint_as_float(xi[l][r]) + inter;
+                        zf[ti] -= kv * dkv;
+                        g_part += kv * inter;
+                        val[l][r] = dkv;
+                    }
+                frag_store(smem_u32(smem + Smem::stage_dk), lane, Lq, t0, val);
+#pragma unroll
+                for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
+                if (lane == 0) m.gred[warp] = g_part;
+                // ---- dv -----------------------------------------------------------------------------------------------
+                mbar_wait(&m.bar_o2, ph_o, status, &m.dead);
+                tc_fence_after();
+#pragma unroll
+                for (int l = 0; l < 2; l++) {
+                    tmem_ld_frag16(tm_lane + ((uint32_t)(16 * l) << 16) + COL_DV + t0, xi[l]);
+                    tmem_ld_frag16(tm_lane + ((uint32_t)(16 * l) << 16) + COL_DA + t0, xe[l]);
+                }
+                tmem_ld_wait();
+#pragma unroll
+                for (int l = 0; l < 2; l++)
+#pragma unroll
+                    for (int r = 0; r < 8; r++)
+                        val[l][r] = __uint_as_float(xi[l][r]) + wv[2 * (r >> 2) + (r & 1)] * __uint_as_float(xe[l][r]);
+                frag_store(smem_u32(smem + Smem::stage_dv), lane, Lq, t0, val);
+                // ---- dq -----------------------------------------------------------------------------------------------
+                mbar_wait(&m.bar_o3, ph_o, status, &m.dead);
+                tc_fence_after();
+#pragma unroll
+                for (int l = 0; l < 2; l++) tmem_ld_frag16(tm_lane + ((uint32_t)(16 * l) << 16) + COL_DQ + t0, xi[l]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int l = 0; l < 2; l++)
+#pragma unroll
+                    for (int r = 0; r < 8; r++) {
+                        const float dqv = __uint_as_float(xi[l][r]);
+                        zf[2 * (r >> 2) + (r & 1)] += frag_elem(fr.q, l, r) * dqv;
+                        val[l][r] = dqv;
+                    }
+                frag_store(smem_u32(smem + Smem::stage_dq), lane, Lq, t0, val);
+                // rows are shared by the eight threads with the same c: sum over them, then one writer per row
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    zf[i] += __shfl_xor_sync(0xffffffffu, zf[i], 4);
+                    zf[i] += __shfl_xor_sync(0xffffffffu, zf[i], 8);
+                    zf[i] += __shfl_xor_sync(0xffffffffu, zf[i], 16);
+                }
+                if (lane < 4) {
+                    m.red[warp][2 * c4] = zf[0];
+                    m.red[warp][2 * c4 + 1] = zf[1];
+                    m.red[warp][8 + 2 * c4] = zf[2];
+                    m.red[warp][8 + 2 * c4 + 1] = zf[3];
+                }
+            } else {
             // q[t][L], k[t][L] of this thread's 16 rows, for the dg terms (read while the first MMAs run; after this
             // the epilogue does not touch the tiles, which are reloaded as soon as the MMAs are done)
             {
@@ -552,21 +667,19 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             float z[16];
             mbar_wait(&m.bar_o, ph_o, status, &m.dead);
             tc_fence_after();
-            if (full) epilogue_dk<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
-            else epilogue_dk<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
+            epilogue_dk(rd, smem, tm_lane, grp, L, H, h, s.replay_base, qk, dk_, rk, z, g_part);
 #pragma unroll
             for (int o_ = 16; o_ > 0; o_ >>= 1) g_part += __shfl_xor_sync(0xffffffffu, g_part, o_);
             if (lane == 0) m.gred[warp] = g_part;
             mbar_wait(&m.bar_o2, ph_o, status, &m.dead);
             tc_fence_after();
-            if (full) epilogue_dv<true>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
-            else epilogue_dv<false>(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
+            epilogue_dv(rd, smem, tm_lane, grp, L, H, h, s.replay_base, dv_, rv);
             mbar_wait(&m.bar_o3, ph_o, status, &m.dead);
             tc_fence_after();
-            if (full) epilogue_dq<true>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
-            else epilogue_dq<false>(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
+            epilogue_dq(rd, smem, tm_lane, grp, L, H, h, qk, dq, z);
             const float row_total = warp_transpose_reduce16(z, lane);
             if (lane < 16) m.red[warp][lane] = row_total;
+            }
             if (full) fence_async_smem();
         }
         ph_o ^= 1;
@@ -598,9 +711,11 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         }
         if (is_issuer && full) {
             int row0 = s.own_begin - s.n_replay + c * BT;
-            tma_store_3d(&map_dq, smem + Smem::stage_dq, 0, h, row0);
-            tma_store_3d(&map_dk, smem + Smem::stage_dk, 0, h, row0);
-            tma_store_3d(&map_dv, smem + Smem::stage_dv, 0, h, row0);
+            for (int p = 0; p < 2; p++) {         // the staging tiles of a full chunk are swizzled [row][64] panels
+                tma_store_3d(&map_dq, smem + Smem::stage_dq + p * PANEL, p * 64, h, row0);
+                tma_store_3d(&map_dk, smem + Smem::stage_dk + p * PANEL, p * 64, h, row0);
+                tma_store_3d(&map_dv, smem + Smem::stage_dv + p * PANEL, p * 64, h, row0);
+            }
             tma_store_commit();
         }
         if (is_aux) {
@@ -671,9 +786,9 @@ int32_t tc_bwd(const BwdArgs& a) {
     if ((rc = make_row_map(&mv, a.v, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mdo, a.dO, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_state_map(&mcs, a.chunk_states, (int64_t)a.tb.n_chunks * a.H)) != HARTS_OK) return rc;
-    if ((rc = make_out_map(&mdq, a.dq, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
-    if ((rc = make_out_map(&mdk, a.dk_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
-    if ((rc = make_out_map(&mdv, a.dv_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mdq, a.dq, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mdk, a.dk_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mdv, a.dv_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if (cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
