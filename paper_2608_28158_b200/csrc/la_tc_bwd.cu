@@ -67,7 +67,7 @@ struct Misc {
     float red[NC / 32][16];  // per-warp partial sums of q.dq - k.dk (warp w covers rows 16(w>>2)..+15)
     float gred[NC / 32];
     uint32_t tmem;
-    uint64_t bar_tiles, bar_a, bar_o, bar_o2, bar_o3, bar_qk_read, bar_exit;
+    uint64_t bar_tiles, bar_tiles2, bar_a, bar_o, bar_o2, bar_o3, bar_qk_read, bar_exit;
     int dead;                // latch: a wait of this CTA ran out, the walk is being abandoned
 };
 
@@ -236,6 +236,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
 
     if (tid == 0) {
         mbar_init(&m.bar_tiles, 1);
+        mbar_init(&m.bar_tiles2, 1);
         mbar_init(&m.bar_a, 1);
         mbar_init(&m.bar_o, 1);
         mbar_init(&m.bar_o2, 1);
@@ -287,21 +288,25 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                    dDPm = desc_mnmajor_base<BT>(aDP), dDSm = desc_mnmajor_base<D>(aDS);
     const uint64_t dSk = desc_kmajor_base(aS);
 
-    // All tiles of a chunk travel on one barrier.  They are requested as soon as the previous chunk's MMAs are done
-    // (the epilogue works from registers and tensor memory only), so the loads overlap the epilogue.
+    // The tiles of a chunk travel on two barriers, in the order in which the chunk needs them: the chunk state and
+    // dO first (the dS pass starts on them), then q, k, v (the A / dA MMAs, which run under that pass).  They are
+    // requested as soon as the previous chunk's MMAs are done (the epilogue works from registers and tensor memory
+    // only), so the loads overlap the epilogue, and the second half of them the dS pass.
     auto issue_tiles = [&](int c, bool tiles) {
         int row0 = s.own_begin - s.n_replay + c * BT;
         int idx = (s.chunk_base + c) * H + h;
         tiles_pending = true;
-        mbar_expect_tx(&m.bar_tiles, (tiles ? 4 * TILE : 0) + 2 * S_PANEL);
+        mbar_expect_tx(&m.bar_tiles, (tiles ? TILE : 0) + 2 * S_PANEL);
+        if (tiles)
+            for (int p = 0; p < 2; p++) tma_load_3d(sDO + p * PANEL, &map_do, p * 64, h, row0, &m.bar_tiles);
         tma_load_3d(sS, &map_cs, 0, 0, idx, &m.bar_tiles);
         tma_load_3d(sS + S_PANEL, &map_cs, 64, 0, idx, &m.bar_tiles);
+        mbar_expect_tx(&m.bar_tiles2, tiles ? 3 * TILE : 0);
         if (tiles)
             for (int p = 0; p < 2; p++) {
-                tma_load_3d(sV + p * PANEL, &map_v, p * 64, h, row0, &m.bar_tiles);
-                tma_load_3d(sDO + p * PANEL, &map_do, p * 64, h, row0, &m.bar_tiles);
-                tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_tiles);
-                tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tiles);
+                tma_load_3d(sV + p * PANEL, &map_v, p * 64, h, row0, &m.bar_tiles2);
+                tma_load_3d(sQ + p * PANEL, &map_q, p * 64, h, row0, &m.bar_tiles2);
+                tma_load_3d(sK + p * PANEL, &map_k, p * 64, h, row0, &m.bar_tiles2);
             }
     };
     // Row codes and g of chunk c for rows `lane` and `lane + 32` (the auxiliary warp prepares a chunk's row data on its own).
@@ -390,12 +395,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             fence_async_smem();
             __syncthreads();
         }
-        if (mbar_wait(&m.bar_tiles, ph_tiles, status, &m.dead)) {
-            tiles_pending = false;
-            ph_tiles ^= 1;
-        }
+        const bool got_tiles = mbar_wait(&m.bar_tiles, ph_tiles, status, &m.dead);
         // ---- A = Q K^T on lanes 0..63, dA = dO V^T on lanes 64..127 (rows 0..63 of that operand are unused) ----------
         if (is_issuer) {
+            if (mbar_wait(&m.bar_tiles2, ph_tiles, status, &m.dead) && got_tiles) tiles_pending = false;
             tc_fence_after();
 #pragma unroll
             for (int ks = 0; ks < 8; ks++)
@@ -406,6 +409,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             mma_commit(&m.bar_a);
             tma_store_wait_read();                // the previous chunk's output stores have left the staging tiles
         }
+        if (got_tiles) ph_tiles ^= 1;
         if (is_aux) load_rows(c - 1, nx_code, nx_g);      // next chunk's rows and g, in flight during this chunk
         float g_part = 0.f;                       // this thread's share of <S_{c+1}, dS_{c+1}>
         uint32_t qk[16];                          // q[t][L] | k[t][L] << 16 of this thread's 16 rows (bf16 bits)
@@ -764,7 +768,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     }
     }   // work items
     if (__syncthreads_or(m.dead) && is_issuer) {  // abandoned: let copies and MMAs in flight finish (bounded)
-        if (tiles_pending) mbar_wait_drain(&m.bar_tiles, ph_tiles);
+        if (tiles_pending) {
+            mbar_wait_drain(&m.bar_tiles, ph_tiles);
+            mbar_wait_drain(&m.bar_tiles2, ph_tiles);
+        }
         mma_commit(&m.bar_exit);
         mbar_wait_drain(&m.bar_exit, 0);
     }
