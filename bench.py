@@ -426,6 +426,16 @@ class LaWorkload:
             b.record(stream)
             marks.append((name, a, b))
 
+        if self.one_launch():
+            # round 0 = all rounds; on a problem this small the library runs them in one cooperative launch per pass, and
+            # the backward call includes the replay-gradient fold
+            timed("fwd", lambda: H.harts_la_fwd(plan, 0, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], ws.slots,
+                                               ws.chunk_states, self.flags, ws.dev_status))
+            timed("bwd", lambda: H.harts_la_bwd(plan, 0, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"], out["dq"],
+                                               out["dk"], out["dv"], out["dg"], ws.chunk_states, ws.scratch, self.flags,
+                                               ws.dev_status))
+            return
+        # one call per round (what round 0 does on a problem of this size), so that every round's launch is timed alone
         for r in range(1, K + 1):
             timed("fwd", lambda: H.harts_la_fwd(plan, r, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], ws.slots,
                                                ws.chunk_states, self.flags, ws.dev_status))
@@ -435,6 +445,14 @@ class LaWorkload:
                                                     inp["dO"], out["dq"], out["dk"], out["dv"], out["dg"],
                                                     ws.chunk_states, ws.scratch, self.flags, ws.dev_status))
         timed("fold", lambda: H.harts_la_bwd_finish(plan.tables, out["dk"], out["dv"], out["dg"], ws.scratch))
+
+    def one_launch(self):
+        """True when the library's all-rounds call runs as one cooperative launch per pass: bf16 d = 128 kernels, more
+        than one round, and a CTA for every (sequence, head) (two per SM in the forward)."""
+        import torch
+        sms = torch.cuda.get_device_properties(0).multi_processor_count
+        tc = self.cfg["dk"] == 128 and not self.args.fma and self.inp["q"].element_size() == 2
+        return tc and self.plan.n_rounds > 1 and self.plan.n_seq * self.cfg["H"] <= 2 * sms
 
     def check(self):
         self.H.harts_la_check(self.ws.dev_status)
@@ -516,9 +534,19 @@ class LaWorkload:
                        "kernels": "fma" if args.fma or cfg["dtype"] == "fp32" else "default",
                        "plan_ms": self.t_plan * 1e3},
             "roofline": roof,
-            # per step: K forward calls, K backward calls each preceded by the hand-off reduction when the plan has
-            # exported boundaries, and the replay-gradient fold
-            "gpu_launches_per_step": 2 * K + (K if plan.n_slots else 0) + (1 if plan.n_rg_rows else 0)}
+            "gpu_launches_per_step": self.launches_per_step()}
+
+    def launches_per_step(self):
+        """Kernels per step: one launch per round and pass (each backward round preceded by the hand-off reduction when
+        the plan exports boundaries) plus the replay-gradient fold -- or, when every (sequence, head) fits a CTA of its
+        own, one cooperative launch for all forward rounds (up to 2 CTAs per SM) and one for all backward rounds."""
+        import torch
+        plan, K, items = self.plan, self.plan.n_rounds, self.plan.n_seq * self.cfg["H"]
+        sms = torch.cuda.get_device_properties(0).multi_processor_count
+        tc = self.cfg["dk"] == 128 and not self.args.fma and self.inp["q"].element_size() == 2
+        fwd = 1 if tc and K > 1 and items <= 2 * sms else K
+        bwd = 1 if tc and K > 1 and items <= sms else K + (K if plan.n_slots else 0)
+        return fwd + bwd + (1 if plan.n_rg_rows else 0)
 
     def extras(self, ms_step):
         """The same kernels, trajectory-wise (the conventional baseline of Section 5); one GPU only."""

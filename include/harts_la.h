@@ -58,6 +58,12 @@ extern "C" {
  * harts_la_tables_t; dev_status[2] = position), the kernels of this and of later calls with the flag return without
  * reading or writing anything, and harts_la_check() reports HARTS_EINVAL.  Needs dev_status (at least 4 int32). */
 #define HARTS_FLAG_CHECK_TABLES 2u
+/* harts_la_fwd / harts_la_bwd with round 0 run ALL rounds in one cooperative launch when the problem is small enough
+ * for every (sequence, head) to have a CTA of its own (bf16, dk = dv = 128): a sequence then waits for the flag of the
+ * boundary state it starts from (backward: for the initial-state gradients of the sequences that started at a
+ * boundary) instead of for the end of the previous round's kernel, so the rounds overlap as far as the tree allows.
+ * Same arithmetic, same bits.  With this flag every round gets its own launch, as with explicit round numbers. */
+#define HARTS_FLAG_ROUND_LAUNCHES 16u
 
 typedef struct harts_la_plan harts_la_plan_t; /* opaque, host memory, library-owned */
 
@@ -152,7 +158,8 @@ int32_t harts_la_plan_tables(const harts_la_plan_t* plan, const void* dev_blob, 
  * Workspace sizes (Section 3.4 "Full-layer activation recomputation": the forward keeps only
  * chunk-boundary states, the backward recomputes everything inside a chunk from them).
  *   chunk_state_bytes: [n_chunks, H, dk, dv] start-of-chunk states in the run dtype, written by the
- *                      forward, read by the backward.
+ *                      forward, read by the backward, followed by (n_slots + n_seq) * H int32 flags that the
+ *                      one-launch forms of round 0 use (the library clears them itself).
  *   scratch_bytes:     backward scratch: per-sequence initial-state gradients [n_seq, H, dk, dv] fp32
  *                      and replay-row gradients [n_replay, H, dk + dv + 1] fp32.
  */

@@ -6,7 +6,7 @@ host planner; PyTorch only owns device memory and streams.  There is no CPU fall
 library cannot be loaded the import of :mod:`paper_2608_28158_b200.binding` fails.
 """
 from .binding import (  # noqa: F401
-    HARTS_BF16, HARTS_FP32, HARTS_FLAG_FMA_KERNELS, HARTS_FLAG_CHECK_TABLES, HartsError, Plan, Workspace, harts_la_bwd, harts_la_bwd_finish, harts_la_bwd_static, harts_la_selftest_timeout,
+    HARTS_BF16, HARTS_FP32, HARTS_FLAG_FMA_KERNELS, HARTS_FLAG_CHECK_TABLES, HARTS_FLAG_ROUND_LAUNCHES, HartsError, Plan, Workspace, harts_la_bwd, harts_la_bwd_finish, harts_la_bwd_static, harts_la_selftest_timeout,
     harts_la_bwd_seqs, harts_la_check, harts_la_fwd, harts_la_fwd_seqs, harts_la_plan, harts_la_strerror,
     harts_la_workspace_bytes, lib, run_fwd_bwd, run_fwd_bwd_host, harts_la_step_host, HostPipeline, expand_trajectories, harts_la_expand, harts_la_gk_workspace_bytes, harts_la_gk_fwd, harts_la_gk_bwd,
 )

@@ -13,6 +13,7 @@ HARTS_OK = 0
 HARTS_FP32, HARTS_BF16 = 0, 1
 HARTS_FLAG_FMA_KERNELS = 1
 HARTS_FLAG_CHECK_TABLES = 2
+HARTS_FLAG_ROUND_LAUNCHES = 16
 _DTYPE_CODE = {torch.float32: HARTS_FP32, torch.bfloat16: HARTS_BF16}
 
 _I32P = C.POINTER(C.c_int32)

@@ -57,10 +57,8 @@ int32_t harts_la_workspace_bytes(const harts_la_tables_t* tb, int32_t H, int32_t
     if (!tb || H < 1 || dk < 1 || dv < 1) return HARTS_EINVAL;
     if (dtype != HARTS_FP32 && dtype != HARTS_BF16) return HARTS_EUNSUPPORTED;
     size_t elem = dtype == HARTS_FP32 ? 4 : 2;
-    if (chunk_state_bytes) {
-        size_t b = (size_t)tb->n_chunks * H * dk * dv * elem;
-        *chunk_state_bytes = b < 256 ? 256 : b;
-    }
+    if (chunk_state_bytes)      // the states, then the flags of the one-launch forms
+        *chunk_state_bytes = harts::chunk_state_payload(*tb, H, dk, dv, elem) + harts::fused_flag_bytes(*tb, H);
     if (scratch_bytes) *scratch_bytes = harts::scratch_layout(*tb, H, dk, dv).total;
     return HARTS_OK;
 }
@@ -117,6 +115,26 @@ int32_t harts_la_fwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
     int32_t rc = harts_la_plan_tables(plan, dev_blob, &tb);
     if (rc != HARTS_OK) return rc;
     int32_t r0 = round == 0 ? 1 : round, r1 = round == 0 ? p->n_rounds : round;
+    if (round == 0 && p->n_rounds > 1 && chunk_states && !(flags & HARTS_FLAG_ROUND_LAUNCHES) &&
+        use_tc(dtype, dk, dv, flags)) {
+        // every round in one launch: a sequence waits for the flag of the state it starts from instead of for the
+        // end of the previous round's kernel
+        rc = check_common(&tb, 0, tb.n_seq, H, dk, dv, dtype);
+        if (rc != HARTS_OK) return rc;
+        if (!q || !k || !v || !g || !o || (tb.n_slots > 0 && !slots)) return HARTS_EINVAL;
+        if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(g) || misaligned(o) || misaligned(slots) ||
+            misaligned(chunk_states))
+            return HARTS_EINVAL;
+        harts::FwdArgs a{tb, 0, tb.n_seq, q, k, v, g, o, slots, chunk_states, H, dk, dv, dtype, flags, dev_status,
+                         static_cast<cudaStream_t>(stream)};
+        if (flags & HARTS_FLAG_CHECK_TABLES) {
+            if (!dev_status) return HARTS_EINVAL;
+            if ((rc = harts::check_tables(tb, 0, tb.n_seq, dev_status, a.stream)) != HARTS_OK) return rc;
+        }
+        int* fl = reinterpret_cast<int*>(static_cast<char*>(chunk_states) + harts::chunk_state_payload(tb, H, dk, dv, 2));
+        rc = harts::tc_fwd_fused(a, fl);
+        if (rc != HARTS_EUNSUPPORTED) return rc;         // else: not all CTAs can be resident, launch round by round
+    }
     for (int32_t r = r0; r <= r1; r++) {
         rc = harts_la_fwd_seqs(&tb, p->round_seq_ptr[r - 1], p->round_seq_ptr[r], q, k, v, g, o, slots, chunk_states,
                                H, dk, dv, dtype, flags, dev_status, stream);
@@ -135,7 +153,28 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
     int32_t rc = harts_la_plan_tables(plan, dev_blob, &tb);
     if (rc != HARTS_OK) return rc;
     int32_t r1 = round == 0 ? p->n_rounds : round, r0 = round == 0 ? 1 : round;
-    for (int32_t r = r1; r >= r0; r--) {
+    bool done = false;
+    if (round == 0 && p->n_rounds > 1 && !(flags & HARTS_FLAG_ROUND_LAUNCHES) && use_tc(dtype, dk, dv, flags)) {
+        rc = check_common(&tb, 0, tb.n_seq, H, dk, dv, dtype);
+        if (rc != HARTS_OK) return rc;
+        if (!q || !k || !v || !g || !dO || !dq || !dk_ || !dv_ || !dg || !chunk_states || !scratch) return HARTS_EINVAL;
+        if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(g) || misaligned(dO) || misaligned(dq) ||
+            misaligned(dk_) || misaligned(dv_) || misaligned(dg) || misaligned(chunk_states) || misaligned(scratch))
+            return HARTS_EINVAL;
+        harts::BwdArgs a{tb, 0, tb.n_seq, q, k, v, g, dO, dq, dk_, dv_, dg, chunk_states, scratch, H, dk, dv, dtype, flags,
+                         dev_status, static_cast<cudaStream_t>(stream)};
+        if (flags & HARTS_FLAG_CHECK_TABLES) {
+            if (!dev_status) return HARTS_EINVAL;
+            if ((rc = harts::check_tables(tb, 0, tb.n_seq, dev_status, a.stream)) != HARTS_OK) return rc;
+        }
+        // the flags sit behind the chunk states; the backward's come after the forward's (n_slots * H)
+        int* fl = reinterpret_cast<int*>(const_cast<char*>(static_cast<const char*>(chunk_states)) +
+                                         harts::chunk_state_payload(tb, H, dk, dv, 2)) + (size_t)tb.n_slots * H;
+        rc = harts::tc_bwd_fused(a, fl);
+        if (rc == HARTS_OK) done = true;
+        else if (rc != HARTS_EUNSUPPORTED) return rc;
+    }
+    for (int32_t r = r1; r >= r0 && !done; r--) {
         rc = harts_la_bwd_seqs(&tb, p->round_seq_ptr[r - 1], p->round_seq_ptr[r], q, k, v, g, dO, dq, dk_, dv_, dg,
                                chunk_states, scratch, H, dk, dv, dtype, flags, dev_status, stream);
         if (rc != HARTS_OK) return rc;

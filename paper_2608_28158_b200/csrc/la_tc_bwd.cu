@@ -211,7 +211,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
               const __nv_bfloat16* __restrict__ dO, __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk_,
               __nv_bfloat16* __restrict__ dv_, float* __restrict__ dg, float* __restrict__ ds0, float* __restrict__ rk,
-              float* __restrict__ rv, float* __restrict__ rg, int* status, const int32_t* gate) {
+              float* __restrict__ rv, float* __restrict__ rg, int* status, const int32_t* gate, int* ds0_flags) {
     if (gate_closed(gate)) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -256,6 +256,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     // Persistent CTAs: work item = (sequence, head); items are ordered longest sequence first and dealt to the CTAs
     // in a snake pattern, so that every CTA gets a similar amount of work.
     uint32_t ph_tiles = 0, ph_a = 0, ph_o = 0;
+    int done_flag = -1;                            // all rounds in one launch: one item per CTA, its flag is set at the end
     bool tiles_pending = false, gave_up = false;   // tiles_pending is kept by the issuing thread only
     const int G = gridDim.x;
     for (int tier = 0; tier * G < n_items; tier++) {
@@ -351,6 +352,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     int next_req = s.req_hi - 1;
     // chunk index of the next exported boundary on the way down (kept in a register: no global load per chunk)
     int next_boundary = next_req >= s.req_lo ? tb.slot_chunk[next_req] : -1;
+    int aux_req = next_req, aux_boundary = next_boundary;    // the auxiliary warp's own walk over the boundaries
     if (is_issuer) issue_tiles(s.n_chunks - 1, !(gather_first && s.n_chunks == 1));
     int nx_code[2];
     float nx_g[2];
@@ -410,16 +412,32 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             tma_store_wait_read();                // the previous chunk's output stores have left the staging tiles
         }
         if (got_tiles) ph_tiles ^= 1;
-        if (is_aux) load_rows(c - 1, nx_code, nx_g);      // next chunk's rows and g, in flight during this chunk
+        if (is_aux) {
+            load_rows(c - 1, nx_code, nx_g);              // next chunk's rows and g, in flight during this chunk
+            if (aux_boundary == c + 1) {                  // the boundary this chunk's dS pass is crossing
+                aux_req--;
+                aux_boundary = aux_req >= s.req_lo ? tb.slot_chunk[aux_req] : -1;
+            }
+            if (ds0_flags && aux_boundary == c) {
+                // all rounds in one launch: the next chunk crosses an exported boundary; the sequences that started
+                // there may still be running elsewhere.  Waited for here, a chunk ahead and off the compute warps' path;
+                // barrier (B) hands the result on.
+                for (int u = tb.slot_cons_ptr[aux_req] + lane; u < tb.slot_cons_ptr[aux_req + 1]; u += 32)
+                    flag_wait(ds0_flags + (size_t)tb.slot_cons_seq[u] * H + h, status, &m.dead);
+                __syncwarp();
+            }
+        }
         float g_part = 0.f;                       // this thread's share of <S_{c+1}, dS_{c+1}>
         uint32_t qk[16];                          // q[t][L] | k[t][L] << 16 of this thread's 16 rows (bf16 bits)
         if (is_compute) {
             // ---- dS pass: add hand-off gradients, bf16 operand copy, <S_c, dS>, pre-scale by gamma -----------------
             {
                 const bool boundary = next_boundary == c + 1;
-                // all consumers' gradients were summed into the first consumer's buffer by handoff_reduce
+                // one launch per round: all consumers' gradients were summed into the first consumer's buffer by
+                // handoff_reduce; all rounds in one launch (ds0_flags): they are summed here, in the same order
                 const int cons_lo = boundary ? tb.slot_cons_ptr[next_req] : 0;
-                const int cons_hi = boundary ? min(tb.slot_cons_ptr[next_req + 1], cons_lo + 1) : 0;
+                const int cons_all = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
+                const int cons_hi = ds0_flags ? cons_all : min(cons_all, cons_lo + 1);
                 const float gamma = rd.gamma;
                 float dot = 0.f;
                 const int blk = grp;
@@ -439,12 +457,17 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                     *reinterpret_cast<uint4*>(sDOs + off) = raw;
                 }
                 tmem_ld_wait();
-                for (int u = cons_lo; u < cons_hi; u++) {
-                    const float4* src = reinterpret_cast<const float4*>(
-                        ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + (size_t)L * D + blk * 32);
+                if (cons_lo < cons_hi) {
+                    const size_t in_state = (size_t)L * D + blk * 32;
 #pragma unroll
                     for (int i4 = 0; i4 < 8; i4++) {
-                        float4 a = src[i4];
+                        float4 a = __ldcg(reinterpret_cast<const float4*>(
+                                              ds0 + ((size_t)tb.slot_cons_seq[cons_lo] * H + h) * state_elems + in_state) + i4);
+                        for (int u = cons_lo + 1; u < cons_hi; u++) {
+                            const float4 b4 = __ldcg(reinterpret_cast<const float4*>(
+                                ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + in_state) + i4);
+                            a.x += b4.x; a.y += b4.y; a.z += b4.z; a.w += b4.w;
+                        }
                         x[i4 * 4 + 0] = __float_as_uint(__uint_as_float(x[i4 * 4 + 0]) + a.x);
                         x[i4 * 4 + 1] = __float_as_uint(__uint_as_float(x[i4 * 4 + 1]) + a.y);
                         x[i4 * 4 + 2] = __float_as_uint(__uint_as_float(x[i4 * 4 + 2]) + a.z);
@@ -765,9 +788,13 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             reinterpret_cast<float4*>(dst + grp * 32)[i4] =
                 make_float4(__uint_as_float(x[i4 * 4]), __uint_as_float(x[i4 * 4 + 1]), __uint_as_float(x[i4 * 4 + 2]),
                             __uint_as_float(x[i4 * 4 + 3]));
+        if (ds0_flags) __threadfence();           // this thread's part, before the flag that follows the barrier below
     }
+    if (s.init_slot >= 0) done_flag = seq * H + h;
     }   // work items
-    if (__syncthreads_or(m.dead) && is_issuer) {  // abandoned: let copies and MMAs in flight finish (bounded)
+    const bool abandoned = __syncthreads_or(m.dead) != 0;
+    if (ds0_flags && done_flag >= 0 && !abandoned && tid == 0) flag_set(ds0_flags + done_flag);
+    if (abandoned && is_issuer) {                  // let copies and MMAs in flight finish (bounded)
         if (tiles_pending) {
             mbar_wait_drain(&m.bar_tiles, ph_tiles);
             mbar_wait_drain(&m.bar_tiles2, ph_tiles);
@@ -807,8 +834,54 @@ int32_t tc_bwd(const BwdArgs& a) {
         a.tb, a.seq_lo, n, a.H, mq, mk, mv, mdo, mcs, mdq, mdk, mdv, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_,
         (__nv_bfloat16*)a.dv_, a.dg, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
-        (float*)(base + sl.rg), a.dev_status, status_gate(a.flags, a.dev_status));
+        (float*)(base + sl.rg), a.dev_status, status_gate(a.flags, a.dev_status), nullptr);
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+
+// All rounds of a plan in ONE cooperative launch, one CTA per (sequence, head) -- offered only while the whole
+// problem is resident at once.  A sequence's CTA publishes a flag once its initial-state gradient is in the scratch
+// area; a sequence that exported a boundary waits (its auxiliary warp does, one chunk ahead) for the flags of all
+// the sequences that started there and sums their gradients itself, in the order handoff_reduce uses.  `flags`:
+// caller-owned DEVICE array of n_seq * H int32, zeroed here on the stream.
+int32_t tc_bwd_fused(const BwdArgs& a, int* flags) {
+    const int n = (a.seq_hi - a.seq_lo) * a.H;
+    if (n == 0) return HARTS_OK;
+    if (n > sm_count()) return HARTS_EUNSUPPORTED;
+    CUtensorMap mq, mk, mv, mdo, mcs, mdq, mdk, mdv;
+    int32_t rc;
+    if ((rc = make_row_map(&mq, a.q, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mk, a.k, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mv, a.v, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mdo, a.dO, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_state_map(&mcs, a.chunk_states, (int64_t)a.tb.n_chunks * a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mdq, a.dq, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mdk, a.dk_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mdv, a.dv_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if (cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+        cudaSuccess)
+        return HARTS_ECUDA;
+    if (cudaMemsetAsync(flags, 0, (size_t)a.tb.n_seq * a.H * sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
+    ScratchLayout sl = scratch_layout(a.tb, a.H, a.dk, a.dv);
+    char* base = static_cast<char*>(a.scratch);
+    harts_la_tables_t tb = a.tb;
+    int seq_lo = a.seq_lo, n_items = n, H = a.H;
+    const __nv_bfloat16 *q = (const __nv_bfloat16*)a.q, *k = (const __nv_bfloat16*)a.k, *v = (const __nv_bfloat16*)a.v,
+                        *dO = (const __nv_bfloat16*)a.dO;
+    const float* g = a.g;
+    __nv_bfloat16 *dq = (__nv_bfloat16*)a.dq, *dk_ = (__nv_bfloat16*)a.dk_, *dv_ = (__nv_bfloat16*)a.dv_;
+    float *dg = a.dg, *ds0 = (float*)(base + sl.ds0), *rk = (float*)(base + sl.rk), *rv = (float*)(base + sl.rv),
+          *rg = (float*)(base + sl.rg);
+    int* status = a.dev_status;
+    const int32_t* gate = status_gate(a.flags, a.dev_status);
+    void* args[] = {&tb, &seq_lo, &n_items, &H, &mq, &mk, &mv, &mdo, &mcs, &mdq, &mdk, &mdv, &q, &k, &v, &g, &dO, &dq, &dk_,
+                    &dv_, &dg, &ds0, &rk, &rv, &rg, &status, &gate, &flags};
+    if (cudaLaunchCooperativeKernel((const void*)tc_bwd_kernel, dim3(n), dim3(NT), args, Smem::bytes + 1024, a.stream) !=
+        cudaSuccess) {
+        (void)cudaGetLastError();
+        return HARTS_EUNSUPPORTED;
+    }
+    return HARTS_OK;
 }
 
 }  // namespace harts

@@ -76,7 +76,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
               const __nv_bfloat16* __restrict__ q,
               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
               __nv_bfloat16* __restrict__ o, float* __restrict__ slots, int store_states, int* status,
-              const int32_t* gate) {
+              const int32_t* gate, int* slot_flags) {
     if (gate_closed(gate)) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -119,6 +119,11 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     const int seq_pos = seq_lo + item / H, h = item % H;
     const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
     const SeqInfo s = seq_info(tb, seq);
+    if (slot_flags && s.init_slot >= 0) {
+        // all rounds in one launch: the producer of this sequence's initial state may still be running elsewhere
+        if (tid == 0) flag_wait(slot_flags + (size_t)s.init_slot * H + h, status, &m.dead);
+        __syncthreads();
+    }
     // initial state into tensor memory: lane i = L holds S[i][:]
     {
         const float* src = s.init_slot < 0 ? nullptr : slots + ((size_t)s.init_slot * H + h) * state_elems + (size_t)L * D;
@@ -126,7 +131,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             uint32_t x[32];
 #pragma unroll
             for (int i4 = 0; i4 < 8; i4++) {
-                float4 a = src ? reinterpret_cast<const float4*>(src + blk * 32)[i4] : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 a = src ? __ldcg(reinterpret_cast<const float4*>(src + blk * 32) + i4) : make_float4(0.f, 0.f, 0.f, 0.f);
                 x[i4 * 4 + 0] = __float_as_uint(a.x);
                 x[i4 * 4 + 1] = __float_as_uint(a.y);
                 x[i4 * 4 + 2] = __float_as_uint(a.z);
@@ -176,6 +181,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     row_code(0, my_code, gval);
 
     for (int c = 0; c < s.n_chunks; c++) {
+        int exported = -1;                        // slot written during this chunk's state pass
         if (tid == 0) tma_store_wait_read();      // the previous chunk's state store has left sS
         tc_fence_before();
         gave_up = __syncthreads_or(m.dead) != 0;  // (1) epilogue of the previous chunk is over everywhere
@@ -266,6 +272,8 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             }
             tmem_st_wait();
             if (export_slot) {
+                if (slot_flags) __threadfence();           // this thread's part of the slot, before the flag below
+                exported = next_req;
                 next_req++;
                 next_boundary = next_req < s.req_hi ? tb.slot_chunk[next_req] : -1;
             }
@@ -321,6 +329,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         tc_fence_after();
         // ---- O1^T, O2^T, state update --------------------------------------------------------------------
         if (tid == 0) {
+            if (slot_flags && exported >= 0) flag_set(slot_flags + (size_t)exported * H + h);   // every part was fenced
             if (store_states) {
                 int idx = (s.chunk_base + c) * H + h;
                 tma_store_3d(&map_cs, sS, 0, 0, idx);
@@ -483,8 +492,59 @@ int32_t tc_fwd(const FwdArgs& a) {
     tc_fwd_kernel<<<grid, NT, Smem::bytes + 1024, a.stream>>>(
         a.tb, a.seq_lo, n, a.H, mq, mk, mv, mcs, mo, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (__nv_bfloat16*)a.o, a.slots, a.chunk_states != nullptr, a.dev_status,
-        status_gate(a.flags, a.dev_status));
+        status_gate(a.flags, a.dev_status), nullptr);
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+
+// All rounds of a plan in ONE launch: sequences [seq_lo, seq_hi) span several rounds (they are numbered round by
+// round, and every CTA takes its work items in that order), and a sequence that starts from an exported state waits
+// for the flag its producer sets after writing the slot.  A consumer's producer always sits in an earlier round, so the
+// earliest unfinished round can always run: no deadlock as long as all CTAs are resident, which the cooperative launch
+// guarantees (it fails otherwise, and the caller falls back to one launch per round).  `flags` is a caller-owned DEVICE
+// array of n_slots * H int32, zeroed here on the stream.
+int32_t tc_fwd_fused(const FwdArgs& a, int* flags) {
+    if (a.seq_hi == a.seq_lo) return HARTS_OK;
+    CUtensorMap mq, mk, mv, mcs, mo;
+    int32_t rc;
+    if ((rc = make_row_map(&mq, a.q, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mk, a.k, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if ((rc = make_row_map(&mv, a.v, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    const void* cs = a.chunk_states ? a.chunk_states : a.q;
+    if ((rc = make_state_map(&mcs, cs, a.chunk_states ? (int64_t)a.tb.n_chunks * a.H : 1)) != HARTS_OK) return rc;
+    if ((rc = make_out_map(&mo, a.o, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
+    if (cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+        cudaSuccess)
+        return HARTS_ECUDA;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tc_fwd_kernel, NT, Smem::bytes + 1024) != cudaSuccess ||
+        per_sm < 1)
+        return HARTS_EUNSUPPORTED;
+    if (per_sm > 2) per_sm = 2;
+    // It pays only while every work item has a CTA of its own: with queues of items per CTA, a CTA that waits for a
+    // producer cannot take other work, and one launch per round is faster (cfg3 forward: 6.2 ms against 8.9).
+    if ((int64_t)(a.seq_hi - a.seq_lo) * a.H > (int64_t)per_sm * sm_count()) return HARTS_EUNSUPPORTED;
+    if (a.tb.n_slots > 0 &&
+        cudaMemsetAsync(flags, 0, (size_t)a.tb.n_slots * a.H * sizeof(int), a.stream) != cudaSuccess)
+        return HARTS_ECUDA;
+    int n = (a.seq_hi - a.seq_lo) * a.H;
+    int grid = n < per_sm * sm_count() ? n : per_sm * sm_count();
+    harts_la_tables_t tb = a.tb;
+    int seq_lo = a.seq_lo, H = a.H, store = a.chunk_states != nullptr;
+    const __nv_bfloat16 *q = (const __nv_bfloat16*)a.q, *k = (const __nv_bfloat16*)a.k, *v = (const __nv_bfloat16*)a.v;
+    const float* g = a.g;
+    __nv_bfloat16* o = (__nv_bfloat16*)a.o;
+    float* slots = a.slots;
+    int* status = a.dev_status;
+    const int32_t* gate = status_gate(a.flags, a.dev_status);
+    void* args[] = {&tb, &seq_lo, &n, &H, &mq, &mk, &mv, &mcs, &mo, &q, &k, &v, &g, &o, &slots, &store, &status, &gate,
+                    &flags};
+    if (cudaLaunchCooperativeKernel((const void*)tc_fwd_kernel, dim3(grid), dim3(NT), args, Smem::bytes + 1024,
+                                    a.stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return HARTS_EUNSUPPORTED;                 // the caller launches round by round instead
+    }
+    return HARTS_OK;
 }
 
 }  // namespace harts

@@ -93,6 +93,32 @@ __device__ __forceinline__ void mbar_expect_tx_only(uint64_t* bar, uint32_t byte
     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 
+// ---- flags between CTAs of one (cooperative) launch -----------------------------------------------------------------------
+// A CTA that has produced something another CTA of the same launch consumes publishes a flag in global memory; the
+// consumer polls it.  Every writer of the data fences before the CTA-wide barrier that precedes flag_set; the consumer
+// reads the data only after flag_wait returned true and a CTA-wide barrier.  The wait is bounded like the others (a
+// longer limit: the producer may be a long sequence) and honours the CTA's latch.
+constexpr unsigned long long FLAG_WAIT_LIMIT_NS = 4000ull * 1000 * 1000;
+__device__ __forceinline__ void flag_set(int* flag) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(1) : "memory");
+}
+__device__ __forceinline__ bool flag_wait(const int* flag, int* status, volatile int* dead) {
+    const unsigned long long t0 = global_ns();
+    for (int round = 0; round < (1 << 26); round++) {
+        int v;
+#pragma unroll 1
+        for (int i = 0; i < 16; i++) {
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+            if (v != 0) return true;
+        }
+        if (*dead) return false;
+        if (global_ns() - t0 > FLAG_WAIT_LIMIT_NS) break;
+    }
+    *dead = 1;
+    if (status) atomicExch(status, STATUS_TIMEOUT);
+    return false;
+}
+
 // ---- fences ---------------------------------------------------------------------------------------
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }

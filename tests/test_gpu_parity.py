@@ -129,6 +129,40 @@ def test_random_forests_through_the_tensor_core_kernels():
     assert nested >= 5 and multi_seg_replay >= 5 and shared_slot >= 5 and multi_round >= 2
 
 
+def test_all_rounds_in_one_launch_give_the_bits_of_one_launch_per_round():
+    """Small problems (every (sequence, head) gets a CTA of its own) run all rounds in one cooperative launch, the
+    sequences waiting for each other through flags instead of kernel boundaries.  Outputs, gradients, exported states
+    and chunk states must equal, bit for bit, those of one launch per round -- on forests with several consumers per
+    boundary, replayed first chunks and three rounds."""
+    import random
+    from test_plan_oracle import random_tree
+    rnd = random.Random(3)
+    cases = [(config_case("cfg1")[1], 1, 5)]
+    cases += [(make_forest([random_tree(rnd, rnd.randint(3, 14), rnd.choice([40, 200, 700])) for _ in range(rnd.randint(1, 3))]),
+               rnd.choice([1, 2]), 60 + i) for i in range(14)]
+    one_launch = shared = 0
+    for fo, heads, seed in cases:
+        inp = make_inputs(fo.n_tokens, heads, 128, 128, "bf16", seed)
+        plan = plan_of(fo).upload()
+        phys = to_physical(plan, inp)
+        got = {}
+        for name, flags in (("rounds", H.HARTS_FLAG_ROUND_LAUNCHES), ("one", 0)):
+            ws = H.Workspace(plan, heads, 128, 128, phys["q"].dtype, flags)
+            ws.slots.fill_(float("nan"))
+            ws.chunk_states.zero_()
+            out = H.run_fwd_bwd(plan, ws, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"])
+            H.harts_la_check(ws.dev_status)
+            n_state = plan.n_chunks * heads * 128 * 128 * 2
+            got[name] = dict(out, slots=ws.slots[:plan.n_slots * heads * 128 * 128].clone(),
+                             states=ws.chunk_states[:n_state].clone())
+        for n in got["one"]:
+            assert torch.equal(got["one"][n], got["rounds"][n]), (n, fo.n_tokens, heads)
+        if plan.n_rounds > 1 and plan.n_seq * heads <= 148:
+            one_launch += 1
+            shared += int((np.diff(plan.slot_cons_ptr) > 1).any())
+    assert one_launch >= 8 and shared >= 3, (one_launch, shared)
+
+
 def test_rounds_issued_one_by_one_match_round_zero():
     cfg, fo, inp = config_case("cfg0b")
     plan = plan_of(fo).upload()
