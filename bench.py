@@ -426,7 +426,7 @@ class LaWorkload:
             b.record(stream)
             marks.append((name, a, b))
 
-        if self.one_launch():
+        if self.one_launch()[0]:
             # round 0 = all rounds; on a problem this small the library runs them in one cooperative launch per pass, and
             # the backward call includes the replay-gradient fold
             timed("fwd", lambda: H.harts_la_fwd(plan, 0, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], ws.slots,
@@ -447,12 +447,15 @@ class LaWorkload:
         timed("fold", lambda: H.harts_la_bwd_finish(plan.tables, out["dk"], out["dv"], out["dg"], ws.scratch))
 
     def one_launch(self):
-        """True when the library's all-rounds call runs as one cooperative launch per pass: bf16 d = 128 kernels, more
-        than one round, and a CTA for every (sequence, head) (two per SM in the forward)."""
+        """(forward, backward): True where the library's all-rounds call runs as one cooperative launch -- bf16 d = 128
+        kernels, more than one round, and at most 8 (sequence, head) items per resident CTA (two CTAs per SM in the
+        forward, one in the backward)."""
         import torch
         sms = torch.cuda.get_device_properties(0).multi_processor_count
         tc = self.cfg["dk"] == 128 and not self.args.fma and self.inp["q"].element_size() == 2
-        return tc and self.plan.n_rounds > 1 and self.plan.n_seq * self.cfg["H"] <= 2 * sms
+        ok = tc and 1 < self.plan.n_rounds <= 32
+        items = self.plan.n_seq * self.cfg["H"]
+        return ok and items <= 16 * sms, ok and items <= 8 * sms
 
     def check(self):
         self.H.harts_la_check(self.ws.dev_status)
@@ -538,14 +541,12 @@ class LaWorkload:
 
     def launches_per_step(self):
         """Kernels per step: one launch per round and pass (each backward round preceded by the hand-off reduction when
-        the plan exports boundaries) plus the replay-gradient fold -- or, when every (sequence, head) fits a CTA of its
-        own, one cooperative launch for all forward rounds (up to 2 CTAs per SM) and one for all backward rounds."""
-        import torch
-        plan, K, items = self.plan, self.plan.n_rounds, self.plan.n_seq * self.cfg["H"]
-        sms = torch.cuda.get_device_properties(0).multi_processor_count
-        tc = self.cfg["dk"] == 128 and not self.args.fma and self.inp["q"].element_size() == 2
-        fwd = 1 if tc and K > 1 and items <= 2 * sms else K
-        bwd = 1 if tc and K > 1 and items <= sms else K + (K if plan.n_slots else 0)
+        the plan exports boundaries) plus the replay-gradient fold -- or, on problems with few items per CTA, one
+        cooperative launch for all forward rounds and one for all backward rounds."""
+        plan, K = self.plan, self.plan.n_rounds
+        one_fwd, one_bwd = self.one_launch()
+        fwd = 1 if one_fwd else K
+        bwd = 1 if one_bwd else K + (K if plan.n_slots else 0)
         return fwd + bwd + (1 if plan.n_rg_rows else 0)
 
     def extras(self, ms_step):

@@ -115,7 +115,8 @@ int32_t harts_la_fwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
     int32_t rc = harts_la_plan_tables(plan, dev_blob, &tb);
     if (rc != HARTS_OK) return rc;
     int32_t r0 = round == 0 ? 1 : round, r1 = round == 0 ? p->n_rounds : round;
-    if (round == 0 && p->n_rounds > 1 && chunk_states && !(flags & HARTS_FLAG_ROUND_LAUNCHES) &&
+    if (round == 0 && p->n_rounds > 1 && p->n_rounds <= harts::MAX_FUSED_ROUNDS && chunk_states &&
+        !(flags & HARTS_FLAG_ROUND_LAUNCHES) &&
         use_tc(dtype, dk, dv, flags)) {
         // every round in one launch: a sequence waits for the flag of the state it starts from instead of for the
         // end of the previous round's kernel
@@ -132,7 +133,7 @@ int32_t harts_la_fwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
             if ((rc = harts::check_tables(tb, 0, tb.n_seq, dev_status, a.stream)) != HARTS_OK) return rc;
         }
         int* fl = reinterpret_cast<int*>(static_cast<char*>(chunk_states) + harts::chunk_state_payload(tb, H, dk, dv, 2));
-        rc = harts::tc_fwd_fused(a, fl);
+        rc = harts::tc_fwd_fused(a, fl, fl + harts::fused_flag_count(tb, H));
         if (rc != HARTS_EUNSUPPORTED) return rc;         // else: not all CTAs can be resident, launch round by round
     }
     for (int32_t r = r0; r <= r1; r++) {
@@ -154,7 +155,8 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
     if (rc != HARTS_OK) return rc;
     int32_t r1 = round == 0 ? p->n_rounds : round, r0 = round == 0 ? 1 : round;
     bool done = false;
-    if (round == 0 && p->n_rounds > 1 && !(flags & HARTS_FLAG_ROUND_LAUNCHES) && use_tc(dtype, dk, dv, flags)) {
+    if (round == 0 && p->n_rounds > 1 && p->n_rounds <= harts::MAX_FUSED_ROUNDS && !(flags & HARTS_FLAG_ROUND_LAUNCHES) &&
+        use_tc(dtype, dk, dv, flags)) {
         rc = check_common(&tb, 0, tb.n_seq, H, dk, dv, dtype);
         if (rc != HARTS_OK) return rc;
         if (!q || !k || !v || !g || !dO || !dq || !dk_ || !dv_ || !dg || !chunk_states || !scratch) return HARTS_EINVAL;
@@ -167,10 +169,14 @@ int32_t harts_la_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32_t 
             if (!dev_status) return HARTS_EINVAL;
             if ((rc = harts::check_tables(tb, 0, tb.n_seq, dev_status, a.stream)) != HARTS_OK) return rc;
         }
-        // the flags sit behind the chunk states; the backward's come after the forward's (n_slots * H)
+        // the flags sit behind the chunk states; the backward's come after the forward's (n_slots * H), the two
+        // ticket counters after both
         int* fl = reinterpret_cast<int*>(const_cast<char*>(static_cast<const char*>(chunk_states)) +
-                                         harts::chunk_state_payload(tb, H, dk, dv, 2)) + (size_t)tb.n_slots * H;
-        rc = harts::tc_bwd_fused(a, fl);
+                                         harts::chunk_state_payload(tb, H, dk, dv, 2));
+        harts::RoundOrder ro;
+        ro.n = p->n_rounds;
+        for (int32_t r = 0; r <= p->n_rounds; r++) ro.ptr[r] = p->round_seq_ptr[r];
+        rc = harts::tc_bwd_fused(a, fl + (size_t)tb.n_slots * H, fl + harts::fused_flag_count(tb, H) + 1, ro);
         if (rc == HARTS_OK) done = true;
         else if (rc != HARTS_EUNSUPPORTED) return rc;
     }

@@ -112,18 +112,27 @@ int32_t fma_fwd(const FwdArgs& a);
 int32_t fma_bwd(const BwdArgs& a);
 int32_t tc_supported(int32_t dtype, int32_t dk, int32_t dv);
 int32_t tc_fwd(const FwdArgs& a);
-int32_t tc_fwd_fused(const FwdArgs& a, int* flags);     // all rounds in one cooperative launch
+int32_t tc_fwd_fused(const FwdArgs& a, int* flags, int* ticket);     // all rounds in one cooperative launch
 
 // Flags for the one-launch forms, kept behind the chunk states in the chunk-state workspace: one int32 per
 // (slot, head) for the forward, one per (sequence, head) for the backward.
 inline size_t chunk_state_payload(const harts_la_tables_t& tb, int32_t H, int32_t dk, int32_t dv, size_t elem) {
     return align_up((size_t)tb.n_chunks * H * dk * dv * elem, 256);
 }
+// flags of the one-launch forms: n_slots * H (forward), n_seq * H (backward), then one ticket counter each
+inline size_t fused_flag_count(const harts_la_tables_t& tb, int32_t H) { return ((size_t)tb.n_slots + tb.n_seq) * H; }
 inline size_t fused_flag_bytes(const harts_la_tables_t& tb, int32_t H) {
-    return align_up(((size_t)tb.n_slots + tb.n_seq) * H * sizeof(int32_t), 256);
+    return align_up((fused_flag_count(tb, H) + 2) * sizeof(int32_t), 256);
 }
+// the plan's round table by value (kernel argument): sequences of round r (0-based) = [ptr[r], ptr[r + 1])
+constexpr int MAX_FUSED_ROUNDS = 32;
+constexpr int ONE_LAUNCH_ITEMS_PER_CTA = 8;    // the one-launch forms are offered up to this many items per resident CTA
+struct RoundOrder {
+    int n;
+    int ptr[MAX_FUSED_ROUNDS + 1];
+};
 int32_t tc_bwd(const BwdArgs& a);
-int32_t tc_bwd_fused(const BwdArgs& a, int* flags);     // all rounds in one cooperative launch
+int32_t tc_bwd_fused(const BwdArgs& a, int* flags, int* ticket, const RoundOrder& rounds);   // all rounds in one launch
 int32_t handoff_reduce(const BwdArgs& a);
 int32_t replay_reduce(const harts_la_tables_t& tb, void* dk_, void* dv_, float* dg, const void* scratch, int32_t H,
                       int32_t dk, int32_t dv, int32_t dtype, cudaStream_t stream);

@@ -69,6 +69,7 @@ struct Misc {
     uint32_t tmem;
     uint64_t bar_tiles, bar_tiles2, bar_a, bar_o, bar_o2, bar_o3, bar_qk_read, bar_exit;
     int dead;                // latch: a wait of this CTA ran out, the walk is being abandoned
+    int item;                // all rounds in one launch: the work item thread 0 drew
 };
 
 struct SeqInfo {
@@ -211,7 +212,8 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
               const __nv_bfloat16* __restrict__ dO, __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk_,
               __nv_bfloat16* __restrict__ dv_, float* __restrict__ dg, float* __restrict__ ds0, float* __restrict__ rk,
-              float* __restrict__ rv, float* __restrict__ rg, int* status, const int32_t* gate, int* ds0_flags) {
+              float* __restrict__ rv, float* __restrict__ rg, int* status, const int32_t* gate, int* ds0_flags,
+              int* ticket, const RoundOrder rounds) {
     if (gate_closed(gate)) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -256,13 +258,32 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     // Persistent CTAs: work item = (sequence, head); items are ordered longest sequence first and dealt to the CTAs
     // in a snake pattern, so that every CTA gets a similar amount of work.
     uint32_t ph_tiles = 0, ph_a = 0, ph_o = 0;
-    int done_flag = -1;                            // all rounds in one launch: one item per CTA, its flag is set at the end
     bool tiles_pending = false, gave_up = false;   // tiles_pending is kept by the issuing thread only
     const int G = gridDim.x;
-    for (int tier = 0; tier * G < n_items; tier++) {
-    const int item = (tier & 1) ? tier * G + (G - 1 - (int)blockIdx.x) : tier * G + (int)blockIdx.x;
-    if (item >= n_items) continue;
-    const int seq_pos = seq_lo + item / H, h = item % H;
+    for (int tier = 0;; tier++) {
+    int item, seq_pos;
+    if (ticket) {
+        // all rounds in one launch: whichever CTA is free draws the next item; the order is last round first, and
+        // inside a round the plan's order (longest sequence first)
+        if (tid == 0) m.item = atomicAdd(ticket, 1);
+        __syncthreads();
+        item = m.item;
+        __syncthreads();
+        if (item >= n_items) break;
+        int j = item / H;
+        seq_pos = -1;
+        for (int r = rounds.n - 1; r >= 0 && seq_pos < 0; r--) {
+            const int cnt = rounds.ptr[r + 1] - rounds.ptr[r];
+            if (j < cnt) seq_pos = rounds.ptr[r] + j;
+            else j -= cnt;
+        }
+    } else {
+        if (tier * G >= n_items) break;
+        item = (tier & 1) ? tier * G + (G - 1 - (int)blockIdx.x) : tier * G + (int)blockIdx.x;
+        if (item >= n_items) continue;
+        seq_pos = seq_lo + item / H;
+    }
+    const int h = item % H;
     const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
     const SeqInfo s = seq_info(tb, seq);
     if (is_compute) {   // dS = 0: nothing follows the last chunk
@@ -790,10 +811,11 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                             __uint_as_float(x[i4 * 4 + 3]));
         if (ds0_flags) __threadfence();           // this thread's part, before the flag that follows the barrier below
     }
-    if (s.init_slot >= 0) done_flag = seq * H + h;
+    if (ds0_flags && s.init_slot >= 0) {           // publish: the gradient of this sequence's initial state is in place
+        if (!__syncthreads_or(m.dead) && tid == 0) flag_set(ds0_flags + (size_t)seq * H + h);
+    }
     }   // work items
     const bool abandoned = __syncthreads_or(m.dead) != 0;
-    if (ds0_flags && done_flag >= 0 && !abandoned && tid == 0) flag_set(ds0_flags + done_flag);
     if (abandoned && is_issuer) {                  // let copies and MMAs in flight finish (bounded)
         if (tiles_pending) {
             mbar_wait_drain(&m.bar_tiles, ph_tiles);
@@ -834,20 +856,26 @@ int32_t tc_bwd(const BwdArgs& a) {
         a.tb, a.seq_lo, n, a.H, mq, mk, mv, mdo, mcs, mdq, mdk, mdv, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_,
         (__nv_bfloat16*)a.dv_, a.dg, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
-        (float*)(base + sl.rg), a.dev_status, status_gate(a.flags, a.dev_status), nullptr);
+        (float*)(base + sl.rg), a.dev_status, status_gate(a.flags, a.dev_status), nullptr, nullptr, RoundOrder{});
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
 
-// All rounds of a plan in ONE cooperative launch, one CTA per (sequence, head) -- offered only while the whole
-// problem is resident at once.  A sequence's CTA publishes a flag once its initial-state gradient is in the scratch
-// area; a sequence that exported a boundary waits (its auxiliary warp does, one chunk ahead) for the flags of all
-// the sequences that started there and sums their gradients itself, in the order handoff_reduce uses.  `flags`:
-// caller-owned DEVICE array of n_seq * H int32, zeroed here on the stream.
-int32_t tc_bwd_fused(const BwdArgs& a, int* flags) {
+// All rounds of a plan in ONE cooperative launch: the persistent CTAs draw the (sequence, head) items from a ticket
+// counter, last round first.  A sequence publishes a flag once its initial-state gradient is in the scratch area; a
+// sequence that exported a boundary waits (its auxiliary warp does, one chunk ahead) for the flags of all the
+// sequences that started there and sums their gradients itself, in the order handoff_reduce uses.  Those sequences
+// sit in later rounds, hold smaller tickets and are running or done: no deadlock while all CTAs are resident, which
+// the cooperative launch guarantees.  `flags`: caller-owned DEVICE array of n_seq * H int32, `ticket`: one int32; both
+// zeroed here on the stream.  rounds: the plan's round table (sequences of round r = [ptr[r], ptr[r+1])).
+int32_t tc_bwd_fused(const BwdArgs& a, int* flags, int* ticket, const RoundOrder& rounds) {
     const int n = (a.seq_hi - a.seq_lo) * a.H;
     if (n == 0) return HARTS_OK;
-    if (n > sm_count()) return HARTS_EUNSUPPORTED;
+    if (rounds.n < 1 || rounds.ptr[0] != a.seq_lo || rounds.ptr[rounds.n] != a.seq_hi) return HARTS_EINVAL;
+    // offered while a CTA gets few items, where the idle tail of every round is what one launch saves (cfg2, 7.5 items
+    // per CTA: 1.92 -> 1.79 ms); with many items per CTA it gains nothing (cfg3: 12.8 ms either way) or loses (cfg4,
+    // 1,800 short items per CTA whose hand-off sums then run inside the kernel: 43 -> 64 ms)
+    if (n > ONE_LAUNCH_ITEMS_PER_CTA * sm_count()) return HARTS_EUNSUPPORTED;
     CUtensorMap mq, mk, mv, mdo, mcs, mdq, mdk, mdv;
     int32_t rc;
     if ((rc = make_row_map(&mq, a.q, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
@@ -862,10 +890,13 @@ int32_t tc_bwd_fused(const BwdArgs& a, int* flags) {
         cudaSuccess)
         return HARTS_ECUDA;
     if (cudaMemsetAsync(flags, 0, (size_t)a.tb.n_seq * a.H * sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
+    if (cudaMemsetAsync(ticket, 0, sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
     ScratchLayout sl = scratch_layout(a.tb, a.H, a.dk, a.dv);
     char* base = static_cast<char*>(a.scratch);
     harts_la_tables_t tb = a.tb;
     int seq_lo = a.seq_lo, n_items = n, H = a.H;
+    const int grid = n < sm_count() ? n : sm_count();
+    RoundOrder ro = rounds;
     const __nv_bfloat16 *q = (const __nv_bfloat16*)a.q, *k = (const __nv_bfloat16*)a.k, *v = (const __nv_bfloat16*)a.v,
                         *dO = (const __nv_bfloat16*)a.dO;
     const float* g = a.g;
@@ -875,8 +906,8 @@ int32_t tc_bwd_fused(const BwdArgs& a, int* flags) {
     int* status = a.dev_status;
     const int32_t* gate = status_gate(a.flags, a.dev_status);
     void* args[] = {&tb, &seq_lo, &n_items, &H, &mq, &mk, &mv, &mdo, &mcs, &mdq, &mdk, &mdv, &q, &k, &v, &g, &dO, &dq, &dk_,
-                    &dv_, &dg, &ds0, &rk, &rv, &rg, &status, &gate, &flags};
-    if (cudaLaunchCooperativeKernel((const void*)tc_bwd_kernel, dim3(n), dim3(NT), args, Smem::bytes + 1024, a.stream) !=
+                    &dv_, &dg, &ds0, &rk, &rv, &rg, &status, &gate, &flags, &ticket, &ro};
+    if (cudaLaunchCooperativeKernel((const void*)tc_bwd_kernel, dim3(grid), dim3(NT), args, Smem::bytes + 1024, a.stream) !=
         cudaSuccess) {
         (void)cudaGetLastError();
         return HARTS_EUNSUPPORTED;

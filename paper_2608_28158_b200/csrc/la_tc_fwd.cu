@@ -39,6 +39,9 @@ struct Smem {
                          misc = stage + TILE;
     static constexpr int bytes = misc + 2048;
 };
+struct SeqInfo {
+    int own_begin, n_replay, n_virtual, n_chunks, replay_base, init_slot, req_lo, req_hi, chunk_base;
+};
 struct Misc {
     float part[BT];      // per-warp partial running sums of g
     float b2[BT];        // running log-decay, in log2 units
@@ -49,11 +52,11 @@ struct Misc {
     uint32_t tmem;
     uint64_t bar_tma, bar_a, bar_o, bar_exit;
     int dead;            // latch: a wait of this CTA ran out, the walk is being abandoned
+    int item;            // all rounds in one launch: the work item thread 0 drew
+    int head;
+    SeqInfo seq;
 };
 
-struct SeqInfo {
-    int own_begin, n_replay, n_virtual, n_chunks, replay_base, init_slot, req_lo, req_hi, chunk_base;
-};
 __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq) {
     SeqInfo s;
     s.own_begin = tb.seq_own_begin[seq];
@@ -69,6 +72,12 @@ __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq
     return s;
 }
 
+// out of line: the wait loop's registers (timer values, counters) must not weigh on the kernel's allocation
+__device__ __noinline__ void wait_for_slot(const int* flag, int* status, int* dead) { flag_wait(flag, status, dead); }
+
+// ONE_LAUNCH: all rounds in one cooperative launch (work items drawn from `ticket`, sequences wait on `slot_flags`);
+// otherwise one round per launch, items dealt statically, and neither pointer is looked at.
+template <bool ONE_LAUNCH>
 __global__ void __launch_bounds__(NT, 2)
 tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const __grid_constant__ CUtensorMap map_q,
               const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -76,7 +85,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
               const __nv_bfloat16* __restrict__ q,
               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ g,
               __nv_bfloat16* __restrict__ o, float* __restrict__ slots, int store_states, int* status,
-              const int32_t* gate, int* slot_flags) {
+              const int32_t* gate, int* slot_flags, int* ticket) {
     if (gate_closed(gate)) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -113,15 +122,36 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     uint32_t ph_tma = 0, ph_a = 0, ph_o = 0;
     bool tma_pending = false, gave_up = false;     // tma_pending is kept by thread 0 only
     const int G = gridDim.x;
-    for (int tier = 0; tier * G < n_items; tier++) {
-    const int item = (tier & 1) ? tier * G + (G - 1 - (int)blockIdx.x) : tier * G + (int)blockIdx.x;
-    if (item >= n_items) continue;
-    const int seq_pos = seq_lo + item / H, h = item % H;
-    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
-    const SeqInfo s = seq_info(tb, seq);
-    if (slot_flags && s.init_slot >= 0) {
+    for (int tier = 0;; tier++) {
+    int item;
+    if constexpr (ONE_LAUNCH) {      // items are drawn in order (round by round) by whichever CTA is free
+        if (tid == 0) m.item = atomicAdd(ticket, 1);
+        __syncthreads();
+        item = m.item;
+        __syncthreads();
+        if (item >= n_items) break;
+    } else {
+        if (tier * G >= n_items) break;
+        item = (tier & 1) ? tier * G + (G - 1 - (int)blockIdx.x) : tier * G + (int)blockIdx.x;
+        if (item >= n_items) continue;
+    }
+    SeqInfo s_own;
+    if constexpr (ONE_LAUNCH) {
+        if (tid == 0) {
+            const int sp = seq_lo + item / H;
+            m.seq = seq_info(tb, tb.seq_order ? tb.seq_order[sp] : sp);
+            m.head = item % H;
+        }
+        __syncthreads();
+    } else {
+        const int sp = seq_lo + item / H;
+        s_own = seq_info(tb, tb.seq_order ? tb.seq_order[sp] : sp);
+    }
+    const SeqInfo& s = ONE_LAUNCH ? const_cast<const SeqInfo&>(m.seq) : s_own;
+    const int h = ONE_LAUNCH ? *(volatile int*)&m.head : item % H;
+    if (ONE_LAUNCH && s.init_slot >= 0) {
         // all rounds in one launch: the producer of this sequence's initial state may still be running elsewhere
-        if (tid == 0) flag_wait(slot_flags + (size_t)s.init_slot * H + h, status, &m.dead);
+        if (tid == 0) wait_for_slot(slot_flags + (size_t)s.init_slot * H + h, status, &m.dead);
         __syncthreads();
     }
     // initial state into tensor memory: lane i = L holds S[i][:]
@@ -181,7 +211,6 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     row_code(0, my_code, gval);
 
     for (int c = 0; c < s.n_chunks; c++) {
-        int exported = -1;                        // slot written during this chunk's state pass
         if (tid == 0) tma_store_wait_read();      // the previous chunk's state store has left sS
         tc_fence_before();
         gave_up = __syncthreads_or(m.dead) != 0;  // (1) epilogue of the previous chunk is over everywhere
@@ -272,8 +301,7 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             }
             tmem_st_wait();
             if (export_slot) {
-                if (slot_flags) __threadfence();           // this thread's part of the slot, before the flag below
-                exported = next_req;
+                if (ONE_LAUNCH) __threadfence();           // this thread's part of the slot, before the flag below
                 next_req++;
                 next_boundary = next_req < s.req_hi ? tb.slot_chunk[next_req] : -1;
             }
@@ -329,7 +357,9 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         tc_fence_after();
         // ---- O1^T, O2^T, state update --------------------------------------------------------------------
         if (tid == 0) {
-            if (slot_flags && exported >= 0) flag_set(slot_flags + (size_t)exported * H + h);   // every part was fenced
+            // the slot written during this chunk's state pass (every thread fenced its part before barrier (4))
+            if (ONE_LAUNCH && next_req > s.req_lo && tb.slot_chunk[next_req - 1] == c)
+                flag_set(slot_flags + (size_t)(next_req - 1) * H + h);
             if (store_states) {
                 int idx = (s.chunk_base + c) * H + h;
                 tma_store_3d(&map_cs, sS, 0, 0, idx);
@@ -484,26 +514,28 @@ int32_t tc_fwd(const FwdArgs& a) {
     const void* cs = a.chunk_states ? a.chunk_states : a.q;   // a valid address for the (unused) map
     if ((rc = make_state_map(&mcs, cs, a.chunk_states ? (int64_t)a.tb.n_chunks * a.H : 1)) != HARTS_OK) return rc;
     if ((rc = make_out_map(&mo, a.o, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
-    if (cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+    if (cudaFuncSetAttribute(tc_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
     int n = (a.seq_hi - a.seq_lo) * a.H;
     int grid = n < 2 * sm_count() ? n : 2 * sm_count();
-    tc_fwd_kernel<<<grid, NT, Smem::bytes + 1024, a.stream>>>(
+    tc_fwd_kernel<false><<<grid, NT, Smem::bytes + 1024, a.stream>>>(
         a.tb, a.seq_lo, n, a.H, mq, mk, mv, mcs, mo, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (__nv_bfloat16*)a.o, a.slots, a.chunk_states != nullptr, a.dev_status,
-        status_gate(a.flags, a.dev_status), nullptr);
+        status_gate(a.flags, a.dev_status), nullptr, nullptr);
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
 
 // All rounds of a plan in ONE launch: sequences [seq_lo, seq_hi) span several rounds (they are numbered round by
-// round, and every CTA takes its work items in that order), and a sequence that starts from an exported state waits
-// for the flag its producer sets after writing the slot.  A consumer's producer always sits in an earlier round, so the
-// earliest unfinished round can always run: no deadlock as long as all CTAs are resident, which the cooperative launch
-// guarantees (it fails otherwise, and the caller falls back to one launch per round).  `flags` is a caller-owned DEVICE
-// array of n_slots * H int32, zeroed here on the stream.
-int32_t tc_fwd_fused(const FwdArgs& a, int* flags) {
+// round), the persistent CTAs draw the work items in that order from a ticket counter, and a sequence that starts from
+// an exported state waits for the flag its producer sets after writing the slot (which it does when it passes the
+// boundary, not at its end).  A waiting item's producer sits in an earlier round, so it holds a smaller ticket and is
+// running or done: no deadlock as long as all CTAs are resident, which the cooperative launch guarantees (it fails
+// otherwise, and the caller falls back to one launch per round).  Which CTA computes an item does not change its
+// arithmetic: the results equal those of one launch per round bit for bit.  `flags`: caller-owned DEVICE array of
+// n_slots * H int32, `ticket`: one int32; both zeroed here on the stream.
+int32_t tc_fwd_fused(const FwdArgs& a, int* flags, int* ticket) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
     CUtensorMap mq, mk, mv, mcs, mo;
     int32_t rc;
@@ -513,20 +545,24 @@ int32_t tc_fwd_fused(const FwdArgs& a, int* flags) {
     const void* cs = a.chunk_states ? a.chunk_states : a.q;
     if ((rc = make_state_map(&mcs, cs, a.chunk_states ? (int64_t)a.tb.n_chunks * a.H : 1)) != HARTS_OK) return rc;
     if ((rc = make_out_map(&mo, a.o, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
-    if (cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+    if (cudaFuncSetAttribute(tc_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tc_fwd_kernel, NT, Smem::bytes + 1024) != cudaSuccess ||
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tc_fwd_kernel<true>, NT, Smem::bytes + 1024) != cudaSuccess ||
         per_sm < 1)
         return HARTS_EUNSUPPORTED;
     if (per_sm > 2) per_sm = 2;
-    // It pays only while every work item has a CTA of its own: with queues of items per CTA, a CTA that waits for a
-    // producer cannot take other work, and one launch per round is faster (cfg3 forward: 6.2 ms against 8.9).
-    if ((int64_t)(a.seq_hi - a.seq_lo) * a.H > (int64_t)per_sm * sm_count()) return HARTS_EUNSUPPORTED;
+    // Offered while a CTA gets few items (at most ONE_LAUNCH_ITEMS_PER_CTA on average): there the idle tail of every
+    // round, about one item long, is what one launch saves (cfg2, 3.7 items per CTA: forward 1.25 -> 1.20 ms; cfg1, one
+    // item per CTA: 0.97 -> 0.62 ms forward + backward).  With many items per CTA one launch per round is faster
+    // (cfg3, 28 items per CTA: 6.2 ms against 8.7, with no time spent waiting on flags).
+    if ((int64_t)(a.seq_hi - a.seq_lo) * a.H > (int64_t)ONE_LAUNCH_ITEMS_PER_CTA * per_sm * sm_count())
+        return HARTS_EUNSUPPORTED;
     if (a.tb.n_slots > 0 &&
         cudaMemsetAsync(flags, 0, (size_t)a.tb.n_slots * a.H * sizeof(int), a.stream) != cudaSuccess)
         return HARTS_ECUDA;
+    if (cudaMemsetAsync(ticket, 0, sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
     int n = (a.seq_hi - a.seq_lo) * a.H;
     int grid = n < per_sm * sm_count() ? n : per_sm * sm_count();
     harts_la_tables_t tb = a.tb;
@@ -538,8 +574,8 @@ int32_t tc_fwd_fused(const FwdArgs& a, int* flags) {
     int* status = a.dev_status;
     const int32_t* gate = status_gate(a.flags, a.dev_status);
     void* args[] = {&tb, &seq_lo, &n, &H, &mq, &mk, &mv, &mcs, &mo, &q, &k, &v, &g, &o, &slots, &store, &status, &gate,
-                    &flags};
-    if (cudaLaunchCooperativeKernel((const void*)tc_fwd_kernel, dim3(grid), dim3(NT), args, Smem::bytes + 1024,
+                    &flags, &ticket};
+    if (cudaLaunchCooperativeKernel((const void*)tc_fwd_kernel<true>, dim3(grid), dim3(NT), args, Smem::bytes + 1024,
                                     a.stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return HARTS_EUNSUPPORTED;                 // the caller launches round by round instead
