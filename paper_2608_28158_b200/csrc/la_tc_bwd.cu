@@ -62,6 +62,9 @@ struct RowData {             // per-chunk row quantities, double-buffered (the n
     float gamma;             // e^{b_n}
     float pad[3];            // keeps the second buffer 16-byte aligned (vector loads of b2)
 };
+struct SeqInfo {
+    int own_begin, n_replay, n_virtual, n_chunks, replay_base, init_slot, req_lo, req_hi, chunk_base;
+};
 struct Misc {
     RowData rows[2];
     float red[NC / 32][16];  // per-warp partial sums of q.dq - k.dk (warp w covers rows 16(w>>2)..+15)
@@ -70,11 +73,10 @@ struct Misc {
     uint64_t bar_tiles, bar_tiles2, bar_a, bar_o, bar_o2, bar_o3, bar_qk_read, bar_exit;
     int dead;                // latch: a wait of this CTA ran out, the walk is being abandoned
     int item;                // all rounds in one launch: the work item thread 0 drew
+    int head;
+    SeqInfo seq;
 };
 
-struct SeqInfo {
-    int own_begin, n_replay, n_virtual, n_chunks, replay_base, init_slot, req_lo, req_hi, chunk_base;
-};
 __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq) {
     SeqInfo s;
     s.own_begin = tb.seq_own_begin[seq];
@@ -283,9 +285,17 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
         if (item >= n_items) continue;
         seq_pos = seq_lo + item / H;
     }
-    const int h = item % H;
     const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
-    const SeqInfo s = seq_info(tb, seq);
+    // the item's record lives in shared memory and is read where it is needed: held in registers over the whole walk it
+    // would push the kernel over its register budget
+    __syncthreads();                               // the previous item's last readers of the record are through
+    if (tid == 0) {
+        m.seq = seq_info(tb, seq);
+        m.head = item % H;
+    }
+    __syncthreads();
+    const SeqInfo& s = m.seq;
+    const int h = *(volatile int*)&m.head;
     if (is_compute) {   // dS = 0: nothing follows the last chunk
         uint32_t zero[32];
 #pragma unroll
