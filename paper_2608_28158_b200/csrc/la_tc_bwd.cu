@@ -205,6 +205,9 @@ __device__ __forceinline__ void frag_store(uint32_t stage, int lane, int Lq, int
     }
 }
 
+// ONE_LAUNCH: all rounds in one cooperative launch (work items drawn from `ticket`, hand-off gradients published
+// and awaited through `ds0_flags`); otherwise one round per launch and neither pointer is looked at.
+template <bool ONE_LAUNCH>
 __global__ void __launch_bounds__(NT, 1)
 tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const __grid_constant__ CUtensorMap map_q,
               const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -264,7 +267,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
     const int G = gridDim.x;
     for (int tier = 0;; tier++) {
     int item, seq_pos;
-    if (ticket) {
+    if constexpr (ONE_LAUNCH) {
         // all rounds in one launch: whichever CTA is free draws the next item; the order is last round first, and
         // inside a round the plan's order (longest sequence first)
         if (tid == 0) m.item = atomicAdd(ticket, 1);
@@ -449,7 +452,7 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 aux_req--;
                 aux_boundary = aux_req >= s.req_lo ? tb.slot_chunk[aux_req] : -1;
             }
-            if (ds0_flags && aux_boundary == c) {
+            if (ONE_LAUNCH && aux_boundary == c) {
                 // all rounds in one launch: the next chunk crosses an exported boundary; the sequences that started
                 // there may still be running elsewhere.  Waited for here, a chunk ahead and off the compute warps' path;
                 // barrier (B) hands the result on.
@@ -465,10 +468,10 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             {
                 const bool boundary = next_boundary == c + 1;
                 // one launch per round: all consumers' gradients were summed into the first consumer's buffer by
-                // handoff_reduce; all rounds in one launch (ds0_flags): they are summed here, in the same order
+                // handoff_reduce; all rounds in one launch: they are summed here, in the same order
                 const int cons_lo = boundary ? tb.slot_cons_ptr[next_req] : 0;
                 const int cons_all = boundary ? tb.slot_cons_ptr[next_req + 1] : 0;
-                const int cons_hi = ds0_flags ? cons_all : min(cons_all, cons_lo + 1);
+                const int cons_hi = ONE_LAUNCH ? cons_all : min(cons_all, cons_lo + 1);
                 const float gamma = rd.gamma;
                 float dot = 0.f;
                 const int blk = grp;
@@ -490,14 +493,20 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
                 tmem_ld_wait();
                 if (cons_lo < cons_hi) {
                     const size_t in_state = (size_t)L * D + blk * 32;
+                    const float4* first = reinterpret_cast<const float4*>(
+                        ds0 + ((size_t)tb.slot_cons_seq[cons_lo] * H + h) * state_elems + in_state);
 #pragma unroll
                     for (int i4 = 0; i4 < 8; i4++) {
-                        float4 a = __ldcg(reinterpret_cast<const float4*>(
-                                              ds0 + ((size_t)tb.slot_cons_seq[cons_lo] * H + h) * state_elems + in_state) + i4);
-                        for (int u = cons_lo + 1; u < cons_hi; u++) {
-                            const float4 b4 = __ldcg(reinterpret_cast<const float4*>(
-                                ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + in_state) + i4);
-                            a.x += b4.x; a.y += b4.y; a.z += b4.z; a.w += b4.w;
+                        float4 a;
+                        if constexpr (ONE_LAUNCH) {       // written during this launch by other CTAs: read past L1
+                            a = __ldcg(first + i4);
+                            for (int u = cons_lo + 1; u < cons_hi; u++) {
+                                const float4 b4 = __ldcg(reinterpret_cast<const float4*>(
+                                    ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems + in_state) + i4);
+                                a.x += b4.x; a.y += b4.y; a.z += b4.z; a.w += b4.w;
+                            }
+                        } else {
+                            a = first[i4];
                         }
                         x[i4 * 4 + 0] = __float_as_uint(__uint_as_float(x[i4 * 4 + 0]) + a.x);
                         x[i4 * 4 + 1] = __float_as_uint(__uint_as_float(x[i4 * 4 + 1]) + a.y);
@@ -819,9 +828,9 @@ tc_bwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             reinterpret_cast<float4*>(dst + grp * 32)[i4] =
                 make_float4(__uint_as_float(x[i4 * 4]), __uint_as_float(x[i4 * 4 + 1]), __uint_as_float(x[i4 * 4 + 2]),
                             __uint_as_float(x[i4 * 4 + 3]));
-        if (ds0_flags) __threadfence();           // this thread's part, before the flag that follows the barrier below
+        if (ONE_LAUNCH) __threadfence();           // this thread's part, before the flag that follows the barrier below
     }
-    if (ds0_flags && s.init_slot >= 0) {           // publish: the gradient of this sequence's initial state is in place
+    if (ONE_LAUNCH && s.init_slot >= 0) {           // publish: the gradient of this sequence's initial state is in place
         if (!__syncthreads_or(m.dead) && tid == 0) flag_set(ds0_flags + (size_t)seq * H + h);
     }
     }   // work items
@@ -855,14 +864,14 @@ int32_t tc_bwd(const BwdArgs& a) {
     if ((rc = make_row_map(&mdq, a.dq, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mdk, a.dk_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mdv, a.dv_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
-    if (cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+    if (cudaFuncSetAttribute(tc_bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
     ScratchLayout sl = scratch_layout(a.tb, a.H, a.dk, a.dv);
     char* base = static_cast<char*>(a.scratch);
     int n = (a.seq_hi - a.seq_lo) * a.H;
     int grid = n < sm_count() ? n : sm_count();
-    tc_bwd_kernel<<<grid, NT, Smem::bytes + 1024, a.stream>>>(
+    tc_bwd_kernel<false><<<grid, NT, Smem::bytes + 1024, a.stream>>>(
         a.tb, a.seq_lo, n, a.H, mq, mk, mv, mdo, mcs, mdq, mdk, mdv, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
         (const __nv_bfloat16*)a.v, a.g, (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_,
         (__nv_bfloat16*)a.dv_, a.dg, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
@@ -896,7 +905,7 @@ int32_t tc_bwd_fused(const BwdArgs& a, int* flags, int* ticket, const RoundOrder
     if ((rc = make_row_map(&mdq, a.dq, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mdk, a.dk_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
     if ((rc = make_row_map(&mdv, a.dv_, a.tb.n_rows, a.H)) != HARTS_OK) return rc;
-    if (cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
+    if (cudaFuncSetAttribute(tc_bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
     if (cudaMemsetAsync(flags, 0, (size_t)a.tb.n_seq * a.H * sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
@@ -917,7 +926,7 @@ int32_t tc_bwd_fused(const BwdArgs& a, int* flags, int* ticket, const RoundOrder
     const int32_t* gate = status_gate(a.flags, a.dev_status);
     void* args[] = {&tb, &seq_lo, &n_items, &H, &mq, &mk, &mv, &mdo, &mcs, &mdq, &mdk, &mdv, &q, &k, &v, &g, &dO, &dq, &dk_,
                     &dv_, &dg, &ds0, &rk, &rv, &rg, &status, &gate, &flags, &ticket, &ro};
-    if (cudaLaunchCooperativeKernel((const void*)tc_bwd_kernel, dim3(grid), dim3(NT), args, Smem::bytes + 1024, a.stream) !=
+    if (cudaLaunchCooperativeKernel((const void*)tc_bwd_kernel<true>, dim3(grid), dim3(NT), args, Smem::bytes + 1024, a.stream) !=
         cudaSuccess) {
         (void)cudaGetLastError();
         return HARTS_EUNSUPPORTED;

@@ -161,7 +161,11 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             uint32_t x[32];
 #pragma unroll
             for (int i4 = 0; i4 < 8; i4++) {
-                float4 a = src ? __ldcg(reinterpret_cast<const float4*>(src + blk * 32) + i4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                // one launch: the slot was written during this launch by another CTA (read past L1); one launch per
+                // round: siblings that start from the same slot on this SM find it in L1
+                float4 a = !src ? make_float4(0.f, 0.f, 0.f, 0.f)
+                           : ONE_LAUNCH ? __ldcg(reinterpret_cast<const float4*>(src + blk * 32) + i4)
+                                        : reinterpret_cast<const float4*>(src + blk * 32)[i4];
                 x[i4 * 4 + 0] = __float_as_uint(a.x);
                 x[i4 * 4 + 1] = __float_as_uint(a.y);
                 x[i4 * 4 + 2] = __float_as_uint(a.z);
