@@ -104,6 +104,10 @@ inline GkScratchLayout gk_scratch_layout(const harts_la_tables_t& tb, int32_t H,
 int32_t gk_supported(int32_t dtype, int32_t dk, int32_t dv);
 int32_t gk_fwd(const FwdArgs& a);      // FwdArgs::g / BwdArgs::g, ::dg point to [rows, H, dk] arrays here
 int32_t gk_bwd(const BwdArgs& a);
+// bf16, d_k = d_v = 128: the dense products on the tensor cores (la_gk_mma.cu); taken unless HARTS_FLAG_FMA_KERNELS
+int32_t gk_mma_supported(int32_t dtype, int32_t dk, int32_t dv);
+int32_t gk_mma_fwd(const FwdArgs& a);
+int32_t gk_mma_bwd(const BwdArgs& a);
 int32_t gk_replay_reduce(const harts_la_tables_t& tb, void* dk_, void* dv_, float* dgk, const void* scratch, int32_t H,
                          int32_t dk, int32_t dv, int32_t dtype, cudaStream_t stream);
 

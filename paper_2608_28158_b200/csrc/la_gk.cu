@@ -532,6 +532,7 @@ int32_t gk_supported(int32_t dtype, int32_t dk, int32_t dv) {
 
 int32_t gk_fwd(const FwdArgs& a) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
+    if (gk_mma_supported(a.dtype, a.dk, a.dv) && !(a.flags & HARTS_FLAG_FMA_KERNELS)) return gk_mma_fwd(a);
     if (a.dtype == HARTS_FP32 && a.dk == 64 && a.dv == 64) return launch_gk_fwd<float, 64, 64>(a);
     if (a.dtype == HARTS_BF16 && a.dk == 64 && a.dv == 64) return launch_gk_fwd<__nv_bfloat16, 64, 64>(a);
     if (a.dtype == HARTS_BF16 && a.dk == 128 && a.dv == 128) return launch_gk_fwd<__nv_bfloat16, 128, 128>(a);
