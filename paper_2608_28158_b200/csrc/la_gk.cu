@@ -542,6 +542,7 @@ int32_t gk_fwd(const FwdArgs& a) {
 int32_t gk_bwd(const BwdArgs& a) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
     if (int32_t rc = handoff_reduce(a); rc != HARTS_OK) return rc;     // ds0 sits at the same place in both layouts
+    if (gk_mma_supported(a.dtype, a.dk, a.dv) && !(a.flags & HARTS_FLAG_FMA_KERNELS)) return gk_mma_bwd(a);
     if (a.dtype == HARTS_FP32 && a.dk == 64 && a.dv == 64) return launch_gk_bwd<float, 64, 64>(a);
     if (a.dtype == HARTS_BF16 && a.dk == 64 && a.dv == 64) return launch_gk_bwd<__nv_bfloat16, 64, 64>(a);
     if (a.dtype == HARTS_BF16 && a.dk == 128 && a.dv == 128) return launch_gk_bwd<__nv_bfloat16, 128, 128>(a);

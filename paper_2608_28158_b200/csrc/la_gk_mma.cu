@@ -451,6 +451,390 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
     }
 }
 
+
+// ---- backward ---------------------------------------------------------------------------------------------------------
+// With dS the gradient of the state at the END of the chunk on entry, dA_tj = dO_t . v_j, ew_j = e^{b_n-b_j}:
+//   dq_t[i] = e^{b_t[i]} (dO_t S_c^T)[i] + sum_{j<=t} dA_tj k_j[i] e^{b_t[i]-b_j[i]}
+//   dk_j[i] = ew_j[i] (v_j dS^T)[i]      + sum_{t>=j} dA_tj q_t[i] e^{b_t[i]-b_j[i]}
+//   dv_j    = sum_{t>=j} A_tj dO_t + (k_j .* ew_j) dS
+//   dg_t[i] = sum_{tau>=t} (q_tau[i] dq_tau[i] - k_tau[i] dk_tau[i]) + e^{b_n[i]} <S_c[i,:], dS[i,:]> + sum_j k_j[i] ew_j[i] (v_j dS^T)[i]
+//   dS     <- Diag(e^{b_n}) dS + (q .* e^{b})^T dO
+// The pair sums are split like the scores of the forward: pairs in different 16-row blocks through the anchored
+// operands (for dk the factor e^{a_I-b_j} of block I multiplies the product of dA's block with q^ afterwards, so one
+// set of anchors serves both), pairs inside a block on the CUDA cores, one thread per (channel, half of the rows).
+struct SharedB {
+    static constexpr int q = 0, k = 16384, v = 32768, dO = 49152;    // bf16 [64][128]
+    static constexpr int b = 65536;                                     // fp32 [64][128]
+    static constexpr int sc = 98304;                                    // bf16 [128][128] S_c; later fp32 [64][128] dq
+    static constexpr int dsb = 131072;                                  // bf16 [128][128] dS as an MMA operand
+    static constexpr int qa = 163840;                                   // bf16 [64][128] anchored q  } later fp32
+    static constexpr int ka = qa + 16384;                               // bf16 [96][128] anchored k  } [64][128] dk
+    static constexpr int p = ka + 96 * 256;                             // bf16 [64][64] scores
+    static constexpr int dab = p + 8192;                                // bf16 [64][64] dA
+    static constexpr int dad = dab + 8192;                              // fp32 [64][16] dA, diagonal blocks
+    static constexpr int tmp = dad + 4096;                              // fp32 [128]
+    static constexpr int rowdot = tmp + 512;                            // fp32 [128]
+    static constexpr int gi = rowdot + 512;                             // fp32 [4][128]
+    static constexpr int row = gi + 2048;                               // int [64]
+    static constexpr int bytes = row + 256;
+};
+static_assert(SharedB::bytes <= 232448, "backward tiles do not fit in shared memory");
+
+// plain row-major [128][128] bf16 in global memory -> swizzled tile
+__device__ __forceinline__ void global_to_tile128(const __nv_bfloat16* src, unsigned char* tile) {
+    uint4 buf[8];
+#pragma unroll
+    for (int u = 0; u < 8; u++) buf[u] = reinterpret_cast<const uint4*>(src)[threadIdx.x + u * NT];
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+        const int p = threadIdx.x + u * NT;
+        *reinterpret_cast<uint4*>(tile + sw256(p >> 4, p & 15)) = buf[u];
+    }
+}
+
+__device__ __forceinline__ float2 ld_bf2(const unsigned char* tile, int r, int col) {      // [r][col], [r][col+1]; col even
+    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(tile + sw256(r, col >> 3) + (col & 7) * 2));
+}
+
+
+__global__ void __launch_bounds__(NT, 1)
+gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* __restrict__ q,
+                  const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ gk,
+                  const __nv_bfloat16* __restrict__ dO, __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk_,
+                  __nv_bfloat16* __restrict__ dv_, float* __restrict__ dgk, const __nv_bfloat16* __restrict__ chunk_states,
+                  float* __restrict__ ds0, float* __restrict__ rk, float* __restrict__ rv, float* __restrict__ rg,
+                  const int32_t* gate) {
+    if (gate_closed(gate)) return;
+    extern __shared__ __align__(1024) unsigned char sm[];
+    unsigned char *sQ = sm + SharedB::q, *sK = sm + SharedB::k, *sV = sm + SharedB::v, *sDO = sm + SharedB::dO,
+                  *sSc = sm + SharedB::sc, *sdSb = sm + SharedB::dsb, *sQa = sm + SharedB::qa, *sKa = sm + SharedB::ka,
+                  *sP = sm + SharedB::p, *sdAb = sm + SharedB::dab;
+    float* sB = reinterpret_cast<float*>(sm + SharedB::b);
+    float* sDQ = reinterpret_cast<float*>(sm + SharedB::sc);       // after S_c is dead
+    float* sDK = reinterpret_cast<float*>(sm + SharedB::qa);       // after the anchored operands are dead
+    float* sdAd = reinterpret_cast<float*>(sm + SharedB::dad);
+    float* sTmp = reinterpret_cast<float*>(sm + SharedB::tmp);
+    float* sRowdot = reinterpret_cast<float*>(sm + SharedB::rowdot);
+    float* sGi = reinterpret_cast<float*>(sm + SharedB::gi);
+    int* srow = reinterpret_cast<int*>(sm + SharedB::row);
+    const uint32_t aQ = s_u32(sQ), aK = s_u32(sK), aV = s_u32(sV), aDO = s_u32(sDO), aSc = s_u32(sSc), adSb = s_u32(sdSb),
+                   aQa = s_u32(sQa), aKa = s_u32(sKa), aP = s_u32(sP), adAb = s_u32(sdAb);
+
+    const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+    const int mb = warp & 3, nh = warp >> 2;          // this warp's 16-row block and 64-column half in [64][128] products
+    const SeqInfo s = seq_info(tb, seq);
+    const size_t state_elems = (size_t)D * D;
+
+    float ds[16][4];                                  // dS rows 16*warp + g (+8), all 128 columns
+#pragma unroll
+    for (int n = 0; n < 16; n++) ds[n][0] = ds[n][1] = ds[n][2] = ds[n][3] = 0.f;
+
+    int next_req = s.req_hi - 1;                      // slots of this sequence are ordered by chunk index
+    for (int c = s.n_chunks - 1; c >= 0; c--) {
+        __syncthreads();                              // the previous chunk's readers of every tile are through
+        // gradient arriving at boundary c+1 from the sequences that started there (summed into the first consumer's
+        // buffer by handoff_reduce)
+        if (next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1) {
+            if (tb.slot_cons_ptr[next_req] < tb.slot_cons_ptr[next_req + 1]) {
+                const float* src = ds0 + ((size_t)tb.slot_cons_seq[tb.slot_cons_ptr[next_req]] * H + h) * state_elems;
+#pragma unroll
+                for (int n = 0; n < 16; n++) {
+                    const float2 lo = *reinterpret_cast<const float2*>(src + (size_t)(warp * 16 + g) * D + n * 8 + tq * 2);
+                    const float2 hi = *reinterpret_cast<const float2*>(src + (size_t)(warp * 16 + g + 8) * D + n * 8 + tq * 2);
+                    ds[n][0] += lo.x; ds[n][1] += lo.y; ds[n][2] += hi.x; ds[n][3] += hi.y;
+                }
+            }
+            next_req--;
+        }
+        load_codes(tb, s, c, srow);
+        __syncthreads();
+        load_tile_bf16(k, H, h, srow, false, sK);
+        load_tile_bf16(q, H, h, srow, true, sQ);
+        load_tile_bf16(v, H, h, srow, false, sV);
+        load_tile_bf16(dO, H, h, srow, true, sDO);
+        load_g(gk, H, h, srow, sB);
+        global_to_tile128(chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems, sSc);
+        state_to_operand(ds, sdSb, warp, lane);
+        __syncthreads();
+        cumsum_rows(sB, sTmp);
+        const int r_lo = 16 * mb + g, r_hi = r_lo + 8;            // this thread's rows in the [64][128] products
+        // ---- dA = dO V^T, iq = dO S_c^T, ik = V dS^T, <S_c, dS> per channel -------------------------------------------
+        float iq[8][4], ik[8][4];
+        {
+            float da[4][4];
+#pragma unroll
+            for (int n = 0; n < 8; n++) {
+                iq[n][0] = iq[n][1] = iq[n][2] = iq[n][3] = 0.f;
+                ik[n][0] = ik[n][1] = ik[n][2] = ik[n][3] = 0.f;
+            }
+#pragma unroll
+            for (int n = 0; n < 4; n++) da[n][0] = da[n][1] = da[n][2] = da[n][3] = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < 8; ks++) {
+                uint32_t a[4], b[4];
+                frag_a<256>(a, aDO, 16 * mb, ks * 16, lane);
+#pragma unroll
+                for (int n2 = 0; n2 < 2; n2++) {
+                    frag_b_nk<256>(b, aV, ks * 16, 32 * nh + 16 * n2, lane);
+                    mma16816(da[2 * n2], a, b[0], b[1]);
+                    mma16816(da[2 * n2 + 1], a, b[2], b[3]);
+                }
+#pragma unroll
+                for (int n2 = 0; n2 < 4; n2++) {
+                    frag_b_nk<256>(b, aSc, ks * 16, 64 * nh + 16 * n2, lane);
+                    mma16816(iq[2 * n2], a, b[0], b[1]);
+                    mma16816(iq[2 * n2 + 1], a, b[2], b[3]);
+                }
+                frag_a<256>(a, aV, 16 * mb, ks * 16, lane);
+#pragma unroll
+                for (int n2 = 0; n2 < 4; n2++) {
+                    frag_b_nk<256>(b, adSb, ks * 16, 64 * nh + 16 * n2, lane);
+                    mma16816(ik[2 * n2], a, b[0], b[1]);
+                    mma16816(ik[2 * n2 + 1], a, b[2], b[3]);
+                }
+            }
+            // dA: bf16 copy for the block products, fp32 copy of the diagonal 16-blocks for the pair sums
+#pragma unroll
+            for (int n = 0; n < 4; n++) {
+                const int col = 32 * nh + 8 * n + 2 * tq;
+                *reinterpret_cast<uint32_t*>(sdAb + sw128(r_lo, col >> 3) + (col & 7) * 2) = pack2(da[n][0], da[n][1]);
+                *reinterpret_cast<uint32_t*>(sdAb + sw128(r_hi, col >> 3) + (col & 7) * 2) = pack2(da[n][2], da[n][3]);
+                if ((col >> 4) == mb) {
+                    *reinterpret_cast<float2*>(sdAd + r_lo * 16 + (col & 15)) = make_float2(da[n][0], da[n][1]);
+                    *reinterpret_cast<float2*>(sdAd + r_hi * 16 + (col & 15)) = make_float2(da[n][2], da[n][3]);
+                }
+            }
+        }
+        {   // <S_c[i,:], dS[i,:]> for the warp's 16 state rows i
+            float d_lo = 0.f, d_hi = 0.f;
+#pragma unroll
+            for (int n = 0; n < 16; n++) {
+                const float2 s_lo = ld_bf2(sSc, warp * 16 + g, n * 8 + tq * 2), s_hi = ld_bf2(sSc, warp * 16 + g + 8, n * 8 + tq * 2);
+                d_lo += s_lo.x * ds[n][0] + s_lo.y * ds[n][1];
+                d_hi += s_hi.x * ds[n][2] + s_hi.y * ds[n][3];
+            }
+            d_lo += __shfl_xor_sync(0xffffffffu, d_lo, 1); d_lo += __shfl_xor_sync(0xffffffffu, d_lo, 2);
+            d_hi += __shfl_xor_sync(0xffffffffu, d_hi, 1); d_hi += __shfl_xor_sync(0xffffffffu, d_hi, 2);
+            if (tq == 0) { sRowdot[warp * 16 + g] = d_lo; sRowdot[warp * 16 + g + 8] = d_hi; }
+        }
+        // inter-chunk parts at the fragment positions: iq <- e^{b_t} iq, ik <- ew ik, and sum_j k_j ew_j ik_j per channel
+#pragma unroll
+        for (int n = 0; n < 8; n++) {
+            const int col = 64 * nh + 8 * n + 2 * tq;
+            const float2 b_lo = *reinterpret_cast<const float2*>(sB + r_lo * D + col);
+            const float2 b_hi = *reinterpret_cast<const float2*>(sB + r_hi * D + col);
+            const float2 b_n = *reinterpret_cast<const float2*>(sB + (BT - 1) * D + col);
+            const float2 k_lo = ld_bf2(sK, r_lo, col), k_hi = ld_bf2(sK, r_hi, col);
+            iq[n][0] *= __expf(b_lo.x); iq[n][1] *= __expf(b_lo.y); iq[n][2] *= __expf(b_hi.x); iq[n][3] *= __expf(b_hi.y);
+            ik[n][0] *= __expf(b_n.x - b_lo.x); ik[n][1] *= __expf(b_n.y - b_lo.y);
+            ik[n][2] *= __expf(b_n.x - b_hi.x); ik[n][3] *= __expf(b_n.y - b_hi.y);
+            float g0 = k_lo.x * ik[n][0] + k_hi.x * ik[n][2], g1 = k_lo.y * ik[n][1] + k_hi.y * ik[n][3];
+#pragma unroll
+            for (int o = 4; o <= 16; o <<= 1) {
+                g0 += __shfl_xor_sync(0xffffffffu, g0, o);
+                g1 += __shfl_xor_sync(0xffffffffu, g1, o);
+            }
+            if (g == 0) *reinterpret_cast<float2*>(sGi + mb * D + col) = make_float2(g0, g1);
+        }
+        // ---- scores and the anchored operands ------------------------------------------------------------------------
+        anchored_operands(sQ, sK, sB, sQa, sKa);
+        scores_diagonal(sQ, sK, sB, sP, warp, lane);
+        __syncthreads();                              // S_c is dead from here on; dA, anchored operands, diagonal scores visible
+        scores_off_diagonal(aQa, aKa, sP, warp, lane);
+        // ---- pairs in different blocks -------------------------------------------------------------------------------
+        if (mb >= 1) {   // dq: rows of block mb against the keys of the blocks before it, anchored at block mb
+            float acc[8][4];
+#pragma unroll
+            for (int n = 0; n < 8; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            for (int ks = 0; ks < mb; ks++) {
+                uint32_t a[4], b[4];
+                frag_a<128>(a, adAb, 16 * mb, 16 * ks, lane);
+#pragma unroll
+                for (int n2 = 0; n2 < 4; n2++) {
+                    frag_b_kn<256>(b, aKa, ka_row0(mb) + 16 * ks, 64 * nh + 16 * n2, lane);
+                    mma16816(acc[2 * n2], a, b[0], b[1]);
+                    mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
+                }
+            }
+#pragma unroll
+            for (int n = 0; n < 8; n++) {
+                const int col = 64 * nh + 8 * n + 2 * tq;
+                const float2 b_lo = *reinterpret_cast<const float2*>(sB + r_lo * D + col);
+                const float2 b_hi = *reinterpret_cast<const float2*>(sB + r_hi * D + col);
+                const float2 an = *reinterpret_cast<const float2*>(sB + 16 * mb * D + col);
+                iq[n][0] += __expf(b_lo.x - an.x) * acc[n][0]; iq[n][1] += __expf(b_lo.y - an.y) * acc[n][1];
+                iq[n][2] += __expf(b_hi.x - an.x) * acc[n][2]; iq[n][3] += __expf(b_hi.y - an.y) * acc[n][3];
+            }
+        }
+        for (int I = mb + 1; I < 4; I++) {   // dk: keys of block mb against the queries of block I, anchored at block I
+            float acc[8][4];
+#pragma unroll
+            for (int n = 0; n < 8; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            uint32_t a[4], b[4];
+            frag_a_t<128>(a, adAb, 16 * mb, 16 * I, lane);
+#pragma unroll
+            for (int n2 = 0; n2 < 4; n2++) {
+                frag_b_kn<256>(b, aQa, 16 * I, 64 * nh + 16 * n2, lane);
+                mma16816(acc[2 * n2], a, b[0], b[1]);
+                mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
+            }
+#pragma unroll
+            for (int n = 0; n < 8; n++) {
+                const int col = 64 * nh + 8 * n + 2 * tq;
+                const float2 b_lo = *reinterpret_cast<const float2*>(sB + r_lo * D + col);
+                const float2 b_hi = *reinterpret_cast<const float2*>(sB + r_hi * D + col);
+                const float2 an = *reinterpret_cast<const float2*>(sB + 16 * I * D + col);
+                ik[n][0] += __expf(an.x - b_lo.x) * acc[n][0]; ik[n][1] += __expf(an.y - b_lo.y) * acc[n][1];
+                ik[n][2] += __expf(an.x - b_hi.x) * acc[n][2]; ik[n][3] += __expf(an.y - b_hi.y) * acc[n][3];
+            }
+        }
+        __syncthreads();                              // the anchored operands are dead
+#pragma unroll
+        for (int n = 0; n < 8; n++) {
+            const int col = 64 * nh + 8 * n + 2 * tq;
+            *reinterpret_cast<float2*>(sDQ + r_lo * D + col) = make_float2(iq[n][0], iq[n][1]);
+            *reinterpret_cast<float2*>(sDQ + r_hi * D + col) = make_float2(iq[n][2], iq[n][3]);
+            *reinterpret_cast<float2*>(sDK + r_lo * D + col) = make_float2(ik[n][0], ik[n][1]);
+            *reinterpret_cast<float2*>(sDK + r_hi * D + col) = make_float2(ik[n][2], ik[n][3]);
+        }
+        __syncthreads();
+
+        // ---- pairs inside a 16-block and dg: thread = (channel i, half hh of the rows) --------------------------------
+        {
+            const int i = tid & (D - 1), hh = tid >> 7;
+            float total = 0.f;                            // sum of q dq - k dk over this thread's rows
+            for (int blk = 2 * hh + 1; blk >= 2 * hh; blk--) {
+                const int t0 = 16 * blk;
+                float dk_acc[16];
+#pragma unroll
+                for (int u = 0; u < 16; u++) dk_acc[u] = 0.f;
+                float kf[16], bj[16];
+#pragma unroll
+                for (int u = 0; u < 16; u++) {
+                    kf[u] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sK + sw256(t0 + u, i >> 3) + (i & 7) * 2));
+                    bj[u] = sB[(t0 + u) * D + i];
+                }
+#pragma unroll
+                for (int tt = 15; tt >= 0; tt--) {
+                    const int t = t0 + tt;
+                    const float qt = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sQ + sw256(t, i >> 3) + (i & 7) * 2));
+                    float dq_acc = 0.f;
+#pragma unroll
+                    for (int u = 0; u <= tt; u++) {
+                        const float x = sdAd[t * 16 + u] * __expf(bj[tt] - bj[u]);     // one exponential for dq and dk
+                        dq_acc += x * kf[u];
+                        dk_acc[u] += x * qt;
+                    }
+                    const float dqv = sDQ[t * D + i] + dq_acc;
+                    const float dkv = sDK[t * D + i] + dk_acc[tt];
+                    sDQ[t * D + i] = dqv;
+                    sDK[t * D + i] = dkv;
+                    total += qt * dqv - kf[tt] * dkv;
+                }
+            }
+            if (hh == 1) sTmp[i] = total;
+            __syncthreads();
+            // dg_t = suffix over the rows + <S_{c+1}[i,:], dS[i,:]> = e^{b_n} <S_c, dS> + sum_j k_j ew_j ik_j
+            const float G = __expf(sB[(BT - 1) * D + i]) * sRowdot[i] + sGi[i] + sGi[D + i] + sGi[2 * D + i] + sGi[3 * D + i];
+            float suffix = G + (hh == 0 ? sTmp[i] : 0.f);
+            for (int t = 32 * hh + 31; t >= 32 * hh; t--) {
+                const int code = srow[t];
+                if (code == -1) continue;
+                const float qt = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sQ + sw256(t, i >> 3) + (i & 7) * 2));
+                const float kt = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sK + sw256(t, i >> 3) + (i & 7) * 2));
+                suffix += qt * sDQ[t * D + i] - kt * sDK[t * D + i];
+                if (code >= 0) dgk[((size_t)code * H + h) * D + i] = suffix;
+                else rg[((size_t)(s.replay_base + t) * H + h) * D + i] = suffix;     // replayed rows sit in chunk 0
+            }
+        }
+        __syncthreads();
+        // ---- dq, dk out: own rows as bf16, replayed rows' dk in fp32 to the scratch -------------------------------------
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            const int p = tid + u * NT, t = p >> 4, c16 = p & 15, code = srow[t];
+            if (code == -1) continue;
+            const float4 q0 = *reinterpret_cast<const float4*>(sDQ + t * D + c16 * 8), q1 = *reinterpret_cast<const float4*>(sDQ + t * D + c16 * 8 + 4);
+            const float4 k0 = *reinterpret_cast<const float4*>(sDK + t * D + c16 * 8), k1 = *reinterpret_cast<const float4*>(sDK + t * D + c16 * 8 + 4);
+            if (code >= 0) {
+                const size_t off = ((size_t)code * H + h) * D + c16 * 8;
+                *reinterpret_cast<uint4*>(dq + off) = make_uint4(pack2(q0.x, q0.y), pack2(q0.z, q0.w), pack2(q1.x, q1.y), pack2(q1.z, q1.w));
+                *reinterpret_cast<uint4*>(dk_ + off) = make_uint4(pack2(k0.x, k0.y), pack2(k0.z, k0.w), pack2(k1.x, k1.y), pack2(k1.z, k1.w));
+            } else {
+                float* dst = rk + ((size_t)(s.replay_base + t) * H + h) * D + c16 * 8;
+                *reinterpret_cast<float4*>(dst) = k0;
+                *reinterpret_cast<float4*>(dst + 4) = k1;
+            }
+        }
+        scale_qk(sQ, sK, sB, sQ, sK);                 // q~, k~ over the raw tiles, which nobody reads any more
+        __syncthreads();
+        // ---- dv_j = sum_{t>=j} A_tj dO_t + k~_j dS : warp -> rows 16*mb, columns 64*nh ------------------------------------
+        {
+            float acc[8][4];
+#pragma unroll
+            for (int n = 0; n < 8; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            for (int ks = mb; ks < 4; ks++) {             // A_tj = 0 for t < j
+                uint32_t a[4], b[4];
+                frag_a_t<128>(a, aP, 16 * mb, 16 * ks, lane);
+#pragma unroll
+                for (int n2 = 0; n2 < 4; n2++) {
+                    frag_b_kn<256>(b, aDO, 16 * ks, 64 * nh + 16 * n2, lane);
+                    mma16816(acc[2 * n2], a, b[0], b[1]);
+                    mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
+                }
+            }
+#pragma unroll
+            for (int ks = 0; ks < 8; ks++) {
+                uint32_t a[4], b[4];
+                frag_a<256>(a, aK, 16 * mb, 16 * ks, lane);
+#pragma unroll
+                for (int n2 = 0; n2 < 4; n2++) {
+                    frag_b_kn<256>(b, adSb, 16 * ks, 64 * nh + 16 * n2, lane);
+                    mma16816(acc[2 * n2], a, b[0], b[1]);
+                    mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
+                }
+            }
+            const int c_lo = srow[r_lo], c_hi = srow[r_hi];
+#pragma unroll
+            for (int n = 0; n < 8; n++) {
+                const int col = 64 * nh + 8 * n + 2 * tq;
+                if (c_lo >= 0) *reinterpret_cast<uint32_t*>(dv_ + ((size_t)c_lo * H + h) * D + col) = pack2(acc[n][0], acc[n][1]);
+                else if (c_lo < -1) *reinterpret_cast<float2*>(rv + ((size_t)(s.replay_base + r_lo) * H + h) * D + col) = make_float2(acc[n][0], acc[n][1]);
+                if (c_hi >= 0) *reinterpret_cast<uint32_t*>(dv_ + ((size_t)c_hi * H + h) * D + col) = pack2(acc[n][2], acc[n][3]);
+                else if (c_hi < -1) *reinterpret_cast<float2*>(rv + ((size_t)(s.replay_base + r_hi) * H + h) * D + col) = make_float2(acc[n][2], acc[n][3]);
+            }
+        }
+        // ---- dS <- Diag(e^{b_n}) dS + q~^T dO : warp -> state rows 16*warp .. ---------------------------------------------
+        {
+            const float g_lo = __expf(sB[(BT - 1) * D + warp * 16 + g]), g_hi = __expf(sB[(BT - 1) * D + warp * 16 + g + 8]);
+#pragma unroll
+            for (int n = 0; n < 16; n++) {
+                ds[n][0] *= g_lo; ds[n][1] *= g_lo; ds[n][2] *= g_hi; ds[n][3] *= g_hi;
+            }
+#pragma unroll
+            for (int ks = 0; ks < 4; ks++) {
+                uint32_t a[4];
+                frag_a_t<256>(a, aQ, warp * 16, ks * 16, lane);
+#pragma unroll
+                for (int n2 = 0; n2 < 8; n2++) {
+                    uint32_t b[4];
+                    frag_b_kn<256>(b, aDO, ks * 16, n2 * 16, lane);
+                    mma16816(ds[2 * n2], a, b[0], b[1]);
+                    mma16816(ds[2 * n2 + 1], a, b[2], b[3]);
+                }
+            }
+        }
+    }
+    if (s.init_slot >= 0) {
+        float* dst = ds0 + ((size_t)seq * H + h) * state_elems;
+#pragma unroll
+        for (int n = 0; n < 16; n++) {
+            *reinterpret_cast<float2*>(dst + (size_t)(warp * 16 + g) * D + n * 8 + tq * 2) = make_float2(ds[n][0], ds[n][1]);
+            *reinterpret_cast<float2*>(dst + (size_t)(warp * 16 + g + 8) * D + n * 8 + tq * 2) = make_float2(ds[n][2], ds[n][3]);
+        }
+    }
+}
+
 }  // namespace
 
 int32_t gk_mma_supported(int32_t dtype, int32_t dk, int32_t dv) { return dtype == HARTS_BF16 && dk == D && dv == D; }
@@ -464,6 +848,22 @@ int32_t gk_mma_fwd(const FwdArgs& a) {
     gk_mma_fwd_kernel<<<n, NT, Shared::fwd_bytes, a.stream>>>(
         a.tb, a.seq_lo, a.H, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v, a.g,
         (__nv_bfloat16*)a.o, a.slots, (__nv_bfloat16*)a.chunk_states, status_gate(a.flags, a.dev_status));
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+
+int32_t gk_mma_bwd(const BwdArgs& a) {
+    if (a.seq_hi == a.seq_lo) return HARTS_OK;
+    if (cudaFuncSetAttribute(gk_mma_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SharedB::bytes) != cudaSuccess)
+        return HARTS_ECUDA;
+    const int n = (a.seq_hi - a.seq_lo) * a.H;
+    const GkScratchLayout sl = gk_scratch_layout(a.tb, a.H, a.dk, a.dv);
+    char* base = static_cast<char*>(a.scratch);
+    gk_mma_bwd_kernel<<<n, NT, SharedB::bytes, a.stream>>>(
+        a.tb, a.seq_lo, a.H, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v, a.g,
+        (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_, (__nv_bfloat16*)a.dv_, a.dg,
+        (const __nv_bfloat16*)a.chunk_states, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
+        (float*)(base + sl.rg), status_gate(a.flags, a.dev_status));
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
