@@ -963,27 +963,29 @@ class GkWorkload:
         plan, cfg = self.plan, self.cfg
         Hh, d = cfg["H"], cfg["dk"]
         th = plan.C * Hh
-        # the contractions of the chunk form (as for the scalar gate) plus one exponential, one multiply and one add per
-        # (t, j <= t, channel) for the per-channel decay, in both passes
-        flops_fwd = th * (2 * 64 * d + 2 * 64 * d + 4 * d * d) + th * 33 * d * 3
-        flops_bwd = th * (5 * 2 * 64 * d + 4 * 2 * d * d) + th * 33 * d * 3
-        # fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x max SM clock
-        peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        # compulsory bytes per token-head (bf16 tensors, fp32 per-channel gate and its gradient): forward reads q, k, v, g
+        # and writes o; backward reads q, k, v, dO, g and writes dq, dk, dv, dg.  The chunk states (bf16, written by the
+        # forward and read by the backward) come on top and are not counted.
+        fwd_bytes = th * (3 * d * 2 + 4 * d + 2 * d)
+        bwd_bytes = th * (4 * d * 2 + 4 * d + 3 * d * 2 + 4 * d)
         K = plan.n_rounds
-        achieved = flops_bwd / (kernel_ms["bwd"] * 1e-3) / 1e12
-        return {"dtype": "f32",
+        # what bounds the kernels by design is the exponentials of the decay-dependent sums (about 330 k per chunk-head
+        # in both passes together, 16 per clock and SM): reported beside the HBM figure
+        chunk_heads = plan.n_chunks * Hh
+        sfu_ms = chunk_heads * 330e3 / (148 * 16 * 1.965e9) * 1e3
+        roof = hbm_roofline("gk_mma_bwd_kernel (all rounds)", bwd_bytes / K, kernel_ms["bwd"] / K, peaks, None,
+                            forward={"achieved": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9,
+                                     "frac": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                            whole_path={"roof_ms": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                                        "frac_strict": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms_step,
+                                        "exponential_unit_ms": sfu_ms, "frac_exponential_unit": sfu_ms / ms_step})
+        return {"dtype": "bf16",
                 "config": {"workload": "gk", "trees": GK_CONFIG, "H": Hh, "dk": d, "dv": d, "chunk": 64,
-                           "compact_tokens": plan.C, "rounds": K, "sequences": plan.n_seq,
-                           "inputs": "bf16 q, k, v, dO; fp32 per-channel log-decay; fp32 arithmetic on the CUDA cores",
+                           "compact_tokens": plan.C, "rounds": K, "sequences": plan.n_seq, "chunks": plan.n_chunks,
+                           "inputs": "bf16 q, k, v, dO; fp32 per-channel log-decay; dense products on the tensor cores "
+                                     "(mma.sync, bf16 operands, fp32 accumulation), in-block pair sums in fp32 on the CUDA cores",
                            "l2": "inputs larger than L2"},
-                "roofline": {"bound": "alu", "kernel": "gk_bwd_kernel (all rounds)", "achieved": achieved, "peak": peak,
-                             "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
-                             "algorithmic_flops_per_launch": flops_bwd / K,
-                             "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
-                             "forward": {"achieved": flops_fwd / (kernel_ms["fwd"] * 1e-3) / 1e12,
-                                         "frac": flops_fwd / (kernel_ms["fwd"] * 1e-3) / 1e12 / peak},
-                             "whole_path": {"roof_ms": (flops_fwd + flops_bwd) / (peak * 1e12) * 1e3,
-                                            "frac_strict": (flops_fwd + flops_bwd) / (peak * 1e12) * 1e3 / ms_step}},
+                "roofline": roof,
                 "gpu_launches_per_step": 2 * K + (K if plan.n_slots else 0) + (1 if plan.n_rg_rows else 0)}
 
     def extras(self, ms_step):

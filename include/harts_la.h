@@ -50,7 +50,7 @@ extern "C" {
 #define HARTS_BF16 1
 
 /* flags */
-#define HARTS_FLAG_FMA_KERNELS 1u /* use the fp32-FMA (non tensor-core) kernels also for bf16 inputs */
+#define HARTS_FLAG_FMA_KERNELS 1u /* use the fp32 CUDA-core (non tensor-core) kernels also for bf16 inputs */
 /* Debug check for hand-built tables (harts_la_fwd_seqs / harts_la_bwd_seqs): before the kernels of the call a small
  * validation kernel checks every index they would follow (CSR pointers monotone and in range, rows < n_rows, slots <
  * n_slots, replay shorter than a chunk, chunk counts consistent, consumer and replay-gradient tables in range).  On a
@@ -247,8 +247,13 @@ int32_t harts_la_step_host(const harts_la_plan_t* plan, const void* dev_blob, co
  *   dgk [n_rows, H, dk] fp32 DEVICE: its gradient (own rows overwritten; replayed rows folded in by the round-1 call)
  * replace g and dg, and the backward scratch is larger (harts_la_gk_workspace_bytes: the replay-row gradient of g is
  * a vector).  Rounds as for harts_la_fwd / harts_la_bwd (0 = all).  Served: fp32 with dk = dv = 64, bf16 with
- * dk = dv = 64 or 128, chunk 64; fp32 arithmetic on the CUDA cores (every decay factor is evaluated as
- * exp(b_t[i] - b_j[i]) with j <= t, so no gate value can overflow).  Errors as for harts_la_fwd / harts_la_bwd.
+ * dk = dv = 64 or 128, chunk 64.  bf16 with dk = dv = 128 runs its dense products on the tensor cores (bf16
+ * operands, fp32 accumulation; decayed operands, scores and chunk states rounded to bf16); everything else, and that
+ * shape too under HARTS_FLAG_FMA_KERNELS, runs in fp32 on the CUDA cores.  Every decay factor is exp of a
+ * difference of running sums that is <= 0 for g <= 0: exp(b_t[i] - b_j[i]) with j <= t directly, or, on the
+ * tensor-core path for t and j in different 16-row blocks of a chunk, exp(b_t[i] - a[i]) exp(a[i] - b_j[i]) with a the
+ * running sum at the first row of t's block -- so no gate value g <= 0 can overflow.  Errors as for harts_la_fwd /
+ * harts_la_bwd.
  */
 int32_t harts_la_gk_workspace_bytes(const harts_la_tables_t* tables, int32_t H, int32_t dk, int32_t dv, int32_t dtype,
                                     size_t* chunk_state_bytes, size_t* scratch_bytes);

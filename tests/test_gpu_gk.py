@@ -1,9 +1,10 @@
 """GPU parity of the per-channel-decay path (harts_la_gk_fwd / harts_la_gk_bwd, the Diag(gamma) term of Eq. 1)
 through the C ABI against its fp64 trajectory-wise oracle, per tensor (relative Frobenius error) and per row.
 
-Tolerances: the kernels compute in fp32 on the CUDA cores.  fp32 inputs: 1e-4 (fast exponential, fp32 accumulation
-over 64-row chunks).  bf16 inputs: outputs 5e-3, gradients 1e-2 -- the operands q~ = q e^{b}, k~ = k e^{b_n-b} and the
-stored chunk states are rounded to bf16 as in the scalar-gate kernels."""
+Tolerances: fp32 inputs (fp32 arithmetic on the CUDA cores): 1e-4 (fast exponential, fp32 accumulation over 64-row
+chunks).  bf16 inputs: outputs 5e-3, gradients 1e-2 -- the operands q~ = q e^{b}, k~ = k e^{b_n-b}, the scores and the
+stored chunk states are rounded to bf16 as in the scalar-gate kernels; with d = 128 the dense products run on the
+tensor cores (bf16 operands, fp32 accumulation), with d = 64 on the CUDA cores."""
 import numpy as np
 import pytest
 import torch
@@ -20,7 +21,7 @@ ROW_MULT = 3.0
 DT = {"fp32": torch.float32, "bf16": torch.bfloat16}
 
 
-def run_gk(fo, heads, d, dtype, seed, strong_every=0, backward=True):
+def run_gk(fo, heads, d, dtype, seed, strong_every=0, backward=True, flags=0, raw=False):
     inp = make_inputs(fo.n_tokens, heads, d, d, dtype, seed)
     inp["g"] = make_gk(fo.n_tokens, heads, d, seed, strong_every=strong_every)
     plan = plan_of(fo).upload()
@@ -31,15 +32,18 @@ def run_gk(fo, heads, d, dtype, seed, strong_every=0, backward=True):
     scratch = torch.empty(sc_bytes, dtype=torch.uint8, device="cuda")
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
     out = {"o": torch.full_like(phys["v"], float("nan"))}
-    H.harts_la_gk_fwd(plan, 0, phys["q"], phys["k"], phys["v"], phys["g"], out["o"], slots, cs, dev_status=status)
+    H.harts_la_gk_fwd(plan, 0, phys["q"], phys["k"], phys["v"], phys["g"], out["o"], slots, cs, flags=flags,
+                      dev_status=status)
     if backward:
         out.update(dq=torch.full_like(phys["q"], float("nan")), dk=torch.full_like(phys["k"], float("nan")),
                    dv=torch.full_like(phys["v"], float("nan")), dg=torch.full_like(phys["g"], float("nan")))
         H.harts_la_gk_bwd(plan, 0, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"], out["dq"], out["dk"],
-                          out["dv"], out["dg"], cs, scratch, dev_status=status)
+                          out["dv"], out["dg"], cs, scratch, flags=flags, dev_status=status)
     H.harts_la_check(status)
     rows = torch.as_tensor(plan.row_of_token.astype(np.int64), device="cuda")
     got = {n: x[rows].float().cpu().numpy() for n, x in out.items()}
+    if raw:
+        return plan, got
     ref = go.forest_eval(fo, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"] if backward else None)
     assert ref["copy_gap"] < 1e-9
     errs = {}
@@ -86,6 +90,25 @@ def test_gates_far_outside_the_usual_range_do_not_overflow():
     check(errs, "fp32")
     plan, errs = run_gk(config_forest("cfg0b"), 1, 128, "bf16", 3, strong_every=8)
     check(errs, "bf16")
+
+
+def test_tensor_core_path_agrees_with_the_cuda_core_path():
+    """bf16, d = 128: the same call with HARTS_FLAG_FMA_KERNELS runs the CUDA-core kernels (pair sums over whole
+    chunks, no anchored operands, fp32 products).  Two different decompositions of the same sums, same bf16 roundings of
+    the inputs and states: they must agree to well within the oracle tolerance, on forests with several rounds, shared
+    slots and replayed rows, three heads, with strongly decaying channels mixed in."""
+    import random
+    from test_plan_oracle import random_tree
+    rnd = random.Random(17)
+    forests = [config_forest("cfg0b"), config_forest("cfg1")]
+    forests += [make_forest([random_tree(rnd, rnd.randint(2, 12), rnd.choice([40, 200, 600])) for _ in range(2)])
+                for _ in range(4)]
+    for n, fo in enumerate(forests):
+        heads = 1 if fo.n_tokens > 10000 else 3
+        _, tc = run_gk(fo, heads, 128, "bf16", 50 + n, strong_every=8 * (n % 2), raw=True)
+        _, cc = run_gk(fo, heads, 128, "bf16", 50 + n, strong_every=8 * (n % 2), raw=True, flags=H.HARTS_FLAG_FMA_KERNELS)
+        for name in tc:
+            assert rel_err(tc[name], cc[name]) <= 0.6 * TOL["bf16"][name], (n, name, rel_err(tc[name], cc[name]))
 
 
 def test_equal_channels_agree_with_the_scalar_gate_kernels():
