@@ -6,9 +6,11 @@
 // in fp32: the decay-dependent pair sums
 //     A_tj      = sum_i q_t[i] k_j[i] e^{b_t[i]-b_j[i]}                          (j <= t)
 //     dq_t[i]  += sum_{j<=t} dA_tj k_j[i] e^{b_t[i]-b_j[i]},   dk_j[i] += sum_{t>=j} dA_tj q_t[i] e^{b_t[i]-b_j[i]}
-// whose exponents are differences of running sums inside the chunk and never positive (no factorisation of
-// e^{b_t} e^{-b_j}: no overflow for any gate).  The operands that carry a decay (q~ = q e^{b_t}, k~ = k e^{b_n-b_j},
-// the scores A, the states) are rounded to bf16 as in the scalar-gate tensor-core kernels.
+// for t and j in the same 16-row block of the chunk; pairs in different blocks become dense products too, through
+// operands anchored at the first row of t's block (see scores_*).  Every exponent is a difference of running sums that
+// is <= 0 for log-decays g <= 0: no gate value can overflow.  The operands that carry a decay (q~ = q e^{b_t},
+// k~ = k e^{b_n-b_j}, the anchored operands, the scores A, the states) are rounded to bf16 as in the scalar-gate
+// tensor-core kernels.
 //
 // Shared-memory tiles of bf16 are row-major with the 16-byte pieces of a row XOR-ed by (row & 7), so that ldmatrix
 // (plain and transposed) is free of bank conflicts.
@@ -19,7 +21,9 @@ namespace {
 
 constexpr int BT = 64;      // chunk rows
 constexpr int D = 128;      // d_k = d_v
-constexpr int NT = 256;     // threads: 8 warps
+constexpr int NT = 512;     // threads: 16 warps
+constexpr int NW = NT / 32;
+constexpr float LOG2E = 1.4426950408889634f;
 
 // ---- shared-memory addressing ---------------------------------------------------------------------------------------
 // [rows][128] bf16 (256-byte rows) and [rows][64] bf16 (128-byte rows); c16 = index of the 16-byte piece in the row
@@ -43,6 +47,13 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// 2^x by the special-function unit; the running log-decays are kept in log2 units so that no multiply precedes it
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 // Fragment loaders.  `tile` is the shared-memory address of a swizzled tile, PITCH its row pitch in bytes.
@@ -106,52 +117,55 @@ __device__ __forceinline__ void load_codes(const harts_la_tables_t& tb, const Se
 // with an output are taken (q, dO); otherwise every valid row (k, v).  Rows that are not taken become zero.
 __device__ __forceinline__ void load_tile_bf16(const __nv_bfloat16* src, int H, int h, const int* srow, bool need_own,
                                                unsigned char* dst) {
-    uint4 buf[4];
+    constexpr int N = BT * 16 / NT;
+    uint4 buf[N];
 #pragma unroll
-    for (int u = 0; u < 4; u++) {
+    for (int u = 0; u < N; u++) {
         const int p = threadIdx.x + u * NT, t = p >> 4, c16 = p & 15, code = srow[t];
         const bool take = need_own ? code >= 0 : code != -1;
         const int r = code >= 0 ? code : -2 - code;
         buf[u] = take ? *reinterpret_cast<const uint4*>(src + ((size_t)r * H + h) * D + c16 * 8) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
-    for (int u = 0; u < 4; u++) {
+    for (int u = 0; u < N; u++) {
         const int p = threadIdx.x + u * NT, t = p >> 4, c16 = p & 15;
         *reinterpret_cast<uint4*>(dst + sw256(t, c16)) = buf[u];
     }
 }
 
-// g of the chunk's valid rows (fp32 [rows, H, 128]) into sB [BT][128], zero elsewhere
+// g of the chunk's valid rows (fp32 [rows, H, 128]) into sB [BT][128] in log2 units (g * log2 e), zero elsewhere
 __device__ __forceinline__ void load_g(const float* gk, int H, int h, const int* srow, float* sB) {
-    float4 buf[8];
+    constexpr int N = BT * 32 / NT;
+    float4 buf[N];
 #pragma unroll
-    for (int u = 0; u < 8; u++) {
+    for (int u = 0; u < N; u++) {
         const int p = threadIdx.x + u * NT, t = p >> 5, c4 = p & 31, code = srow[t];
         const int r = code >= 0 ? code : -2 - code;
         buf[u] = code != -1 ? *reinterpret_cast<const float4*>(gk + ((size_t)r * H + h) * D + c4 * 4)
                             : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
-    for (int u = 0; u < 8; u++) {
+    for (int u = 0; u < N; u++) {
         const int p = threadIdx.x + u * NT;
-        reinterpret_cast<float4*>(sB)[p] = buf[u];
+        reinterpret_cast<float4*>(sB)[p] = make_float4(buf[u].x * LOG2E, buf[u].y * LOG2E, buf[u].z * LOG2E, buf[u].w * LOG2E);
     }
 }
 
-// running sum over the rows, per channel: two threads per channel (rows 0..31 and 32..63), joined through sTmp[128]
+// running sum over the rows, per channel: four threads per channel (16 rows each, scanned in registers), joined through
+// sTmp[4][128]
 __device__ __forceinline__ void cumsum_rows(float* sB, float* sTmp) {
-    const int tid = threadIdx.x, i = tid & (D - 1), half = tid >> 7;
-    float acc = 0.f;
-    for (int t = half * 32; t < half * 32 + 32; t++) {
-        acc += sB[t * D + i];
-        sB[t * D + i] = acc;
-    }
-    if (half == 0) sTmp[i] = acc;
+    const int tid = threadIdx.x, i = tid & (D - 1), part = tid >> 7;
+    float x[16];
+#pragma unroll
+    for (int u = 0; u < 16; u++) x[u] = sB[(part * 16 + u) * D + i];
+#pragma unroll
+    for (int u = 1; u < 16; u++) x[u] += x[u - 1];
+    sTmp[part * D + i] = x[15];
     __syncthreads();
-    if (half == 1) {
-        const float base = sTmp[i];
-        for (int t = 32; t < BT; t++) sB[t * D + i] += base;
-    }
+    float base = 0.f;
+    for (int pp = 0; pp < part; pp++) base += sTmp[pp * D + i];
+#pragma unroll
+    for (int u = 0; u < 16; u++) sB[(part * 16 + u) * D + i] = x[u] + base;
     __syncthreads();
 }
 
@@ -203,8 +217,8 @@ __device__ __forceinline__ void anchored_operands(const unsigned char* sQ, const
             const float2 ba = *reinterpret_cast<const float2*>(sB + anchor_row * D + i);
             const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
             // q^: e^{b_t - a_I};  k^(I): e^{a_I - b_j}
-            const float e0 = is_q ? __expf(bs.x - ba.x) : __expf(ba.x - bs.x);
-            const float e1 = is_q ? __expf(bs.y - ba.y) : __expf(ba.y - bs.y);
+            const float e0 = is_q ? ex2(bs.x - ba.x) : ex2(ba.x - bs.x);
+            const float e1 = is_q ? ex2(bs.y - ba.y) : ex2(ba.y - bs.y);
             w[e] = pack2(f.x * e0, f.y * e1);
         }
         // the local row index of a k^(I) sub-tile is dst_row - its row offset; the offsets are multiples of 8, so the
@@ -213,10 +227,10 @@ __device__ __forceinline__ void anchored_operands(const unsigned char* sQ, const
     }
 }
 
-// blocks left of the diagonal: warp -> row block I = warp & 3, every second 16-column tile
+// blocks left of the diagonal: warp -> row block I = warp & 3, 16-column tile J = warp >> 2
 __device__ __forceinline__ void scores_off_diagonal(uint32_t aQa, uint32_t aKa, unsigned char* sP, int warp, int lane) {
     const int I = warp & 3, g = lane >> 2, tq = lane & 3;
-    for (int J = warp >> 2; J < I; J += 2) {
+    for (int J = warp >> 2; J < I; J += NW / 4) {
         float acc[2][4];
 #pragma unroll
         for (int x = 0; x < 2; x++) acc[x][0] = acc[x][1] = acc[x][2] = acc[x][3] = 0.f;
@@ -257,10 +271,10 @@ __device__ __forceinline__ void scores_diagonal(const unsigned char* sQ, const u
                 const float4 bj = *reinterpret_cast<const float4*>(sB + j * D + lane * 4);
                 const float2 k01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kraw.x));
                 const float2 k23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kraw.y));
-                acc = q01.x * k01.x * __expf(bt.x - bj.x);
-                acc += q01.y * k01.y * __expf(bt.y - bj.y);
-                acc += q23.x * k23.x * __expf(bt.z - bj.z);
-                acc += q23.y * k23.y * __expf(bt.w - bj.w);
+                acc = q01.x * k01.x * ex2(bt.x - bj.x);
+                acc += q01.y * k01.y * ex2(bt.y - bj.y);
+                acc += q23.x * k23.x * ex2(bt.z - bj.z);
+                acc += q23.y * k23.y * ex2(bt.w - bj.w);
             }
             z[u] = acc;
         }
@@ -277,7 +291,7 @@ __device__ __forceinline__ void scores_diagonal(const unsigned char* sQ, const u
 __device__ __forceinline__ void scale_qk(const unsigned char* sQ, const unsigned char* sK, const float* sB,
                                          unsigned char* dQ, unsigned char* dK) {
 #pragma unroll
-    for (int u = 0; u < 4; u++) {
+    for (int u = 0; u < BT * 16 / NT; u++) {
         const int p = threadIdx.x + u * NT, t = p >> 4, c16 = p & 15;
         const uint32_t off = sw256(t, c16);
         uint4 qv = *reinterpret_cast<const uint4*>(sQ + off), kv = *reinterpret_cast<const uint4*>(sK + off);
@@ -290,35 +304,77 @@ __device__ __forceinline__ void scale_qk(const unsigned char* sQ, const unsigned
             const float2 bn = *reinterpret_cast<const float2*>(sB + (BT - 1) * D + i);
             const float2 qf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&qw[e]));
             const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kw[e]));
-            qw[e] = pack2(qf.x * __expf(bt.x), qf.y * __expf(bt.y));
-            kw[e] = pack2(kf.x * __expf(bn.x - bt.x), kf.y * __expf(bn.y - bt.y));
+            qw[e] = pack2(qf.x * ex2(bt.x), qf.y * ex2(bt.y));
+            kw[e] = pack2(kf.x * ex2(bn.x - bt.x), kf.y * ex2(bn.y - bt.y));
         }
         *reinterpret_cast<uint4*>(dQ + off) = qv;
         *reinterpret_cast<uint4*>(dK + off) = kv;
     }
 }
 
-// The state fragments of a warp: rows 16*warp + g and + g + 8 (g = lane / 4), columns 8*n + 2*(lane % 4) + {0, 1} of
-// n-tile n: st[n][0..1] = row g, st[n][2..3] = row g + 8.
+// The state fragments of a warp: rows 16 * (warp & 7) + g and + g + 8 (g = lane / 4), columns
+// 64 * (warp >> 3) + 8 * n + 2 * (lane % 4) + {0, 1} of n-tile n: st[n][0..1] = row g, st[n][2..3] = row g + 8.
 struct Shared {
     static constexpr int q = 0, k = 16384, v = 32768;          // bf16 [64][128]
     static constexpr int p = 49152;                             // bf16 [64][64]
     static constexpr int sb = 57344;                            // bf16 [128][128]: the state as an MMA operand
-    static constexpr int b = 90112;                             // fp32 [64][128]: running log-decay
-    static constexpr int tmp = 122880;                          // fp32 [128]
-    static constexpr int row = tmp + 512;                       // int  [64]
-    static constexpr int qa = 124928;                           // bf16 [64][128]: q anchored at its 16-row block
+    static constexpr int b = 90112;                             // fp32 [64][128]: running log-decay (log2 units)
+    static constexpr int qa = 122880;                           // bf16 [64][128]: q anchored at its 16-row block
     static constexpr int ka = qa + 16384;                       // bf16 [96][128]: k anchored at blocks 1, 2, 3
-    static constexpr int fwd_bytes = ka + 96 * 256;
+    static constexpr int tmp = ka + 96 * 256;                   // fp32 [4][128]
+    static constexpr int row = tmp + 2048;                      // int  [64]
+    static constexpr int fwd_bytes = row + 256;
 };
 
 // state fragments -> bf16 operand tile (swizzled [128][128])
-__device__ __forceinline__ void state_to_operand(const float (&st)[16][4], unsigned char* sSb, int warp, int lane) {
-    const int g = lane >> 2, tq = lane & 3, r0 = warp * 16 + g;
+__device__ __forceinline__ void state_to_operand(const float (&st)[8][4], unsigned char* sSb, int warp, int lane) {
+    const int g = lane >> 2, tq = lane & 3, r0 = (warp & 7) * 16 + g, c0 = (warp >> 3) * 8;
 #pragma unroll
-    for (int n = 0; n < 16; n++) {
-        *reinterpret_cast<uint32_t*>(sSb + sw256(r0, n) + tq * 4) = pack2(st[n][0], st[n][1]);
-        *reinterpret_cast<uint32_t*>(sSb + sw256(r0 + 8, n) + tq * 4) = pack2(st[n][2], st[n][3]);
+    for (int n = 0; n < 8; n++) {
+        *reinterpret_cast<uint32_t*>(sSb + sw256(r0, c0 + n) + tq * 4) = pack2(st[n][0], st[n][1]);
+        *reinterpret_cast<uint32_t*>(sSb + sw256(r0 + 8, c0 + n) + tq * 4) = pack2(st[n][2], st[n][3]);
+    }
+}
+// state fragments <-> fp32 [128][128] in global memory (slots, initial-state gradients)
+template <bool ADD>
+__device__ __forceinline__ void state_from_global(float (&st)[8][4], const float* src, int warp, int lane) {
+    const int g = lane >> 2, tq = lane & 3, r0 = (warp & 7) * 16 + g, c0 = (warp >> 3) * 64 + tq * 2;
+#pragma unroll
+    for (int n = 0; n < 8; n++) {
+        const float2 lo = *reinterpret_cast<const float2*>(src + (size_t)r0 * D + c0 + n * 8);
+        const float2 hi = *reinterpret_cast<const float2*>(src + (size_t)(r0 + 8) * D + c0 + n * 8);
+        if (ADD) { st[n][0] += lo.x; st[n][1] += lo.y; st[n][2] += hi.x; st[n][3] += hi.y; }
+        else { st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y; }
+    }
+}
+__device__ __forceinline__ void state_to_global(const float (&st)[8][4], float* dst, int warp, int lane) {
+    const int g = lane >> 2, tq = lane & 3, r0 = (warp & 7) * 16 + g, c0 = (warp >> 3) * 64 + tq * 2;
+#pragma unroll
+    for (int n = 0; n < 8; n++) {
+        *reinterpret_cast<float2*>(dst + (size_t)r0 * D + c0 + n * 8) = make_float2(st[n][0], st[n][1]);
+        *reinterpret_cast<float2*>(dst + (size_t)(r0 + 8) * D + c0 + n * 8) = make_float2(st[n][2], st[n][3]);
+    }
+}
+// st <- Diag(2^{b_n}) st + X^T Y over the chunk's 64 rows: X stored [row][128] (its transpose is the A operand), Y
+// stored [row][128]
+__device__ __forceinline__ void state_update(float (&st)[8][4], const float* sB, uint32_t aX, uint32_t aY, int warp, int lane) {
+    const int g = lane >> 2, r0 = (warp & 7) * 16, c0 = (warp >> 3) * 64;
+    const float g_lo = ex2(sB[(BT - 1) * D + r0 + g]), g_hi = ex2(sB[(BT - 1) * D + r0 + g + 8]);
+#pragma unroll
+    for (int n = 0; n < 8; n++) {
+        st[n][0] *= g_lo; st[n][1] *= g_lo; st[n][2] *= g_hi; st[n][3] *= g_hi;
+    }
+#pragma unroll
+    for (int ks = 0; ks < 4; ks++) {
+        uint32_t a[4];
+        frag_a_t<256>(a, aX, r0, ks * 16, lane);
+#pragma unroll
+        for (int n2 = 0; n2 < 4; n2++) {
+            uint32_t b[4];
+            frag_b_kn<256>(b, aY, ks * 16, c0 + n2 * 16, lane);
+            mma16816(st[2 * n2], a, b[0], b[1]);
+            mma16816(st[2 * n2 + 1], a, b[2], b[3]);
+        }
     }
 }
 // swizzled bf16 [rows][128] tile -> plain row-major global memory ([rows][128] contiguous), 16 bytes per thread and step
@@ -336,30 +392,24 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
     if (gate_closed(gate)) return;
     extern __shared__ __align__(1024) unsigned char sm[];
     unsigned char *sQ = sm + Shared::q, *sK = sm + Shared::k, *sV = sm + Shared::v, *sP = sm + Shared::p,
-                  *sSb = sm + Shared::sb;
+                  *sSb = sm + Shared::sb, *sQa = sm + Shared::qa, *sKa = sm + Shared::ka;
     float* sB = reinterpret_cast<float*>(sm + Shared::b);
     float* sTmp = reinterpret_cast<float*>(sm + Shared::tmp);
     int* srow = reinterpret_cast<int*>(sm + Shared::row);
-    unsigned char *sQa = sm + Shared::qa, *sKa = sm + Shared::ka;
     const uint32_t aQ = s_u32(sQ), aK = s_u32(sK), aV = s_u32(sV), aP = s_u32(sP), aSb = s_u32(sSb);
 
     const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+    const int mb = warp & 3, nq = warp >> 2;          // this warp's 16-row block and 32-column quarter of [64][128] products
     const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)D * D;
 
-    float st[16][4];                       // S rows 16*warp + g (+8), all 128 columns
+    float st[8][4];
     if (s.init_slot < 0) {
 #pragma unroll
-        for (int n = 0; n < 16; n++) st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
+        for (int n = 0; n < 8; n++) st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
     } else {
-        const float* src = slots + ((size_t)s.init_slot * H + h) * state_elems;
-#pragma unroll
-        for (int n = 0; n < 16; n++) {
-            const float2 lo = *reinterpret_cast<const float2*>(src + (size_t)(warp * 16 + g) * D + n * 8 + tq * 2);
-            const float2 hi = *reinterpret_cast<const float2*>(src + (size_t)(warp * 16 + g + 8) * D + n * 8 + tq * 2);
-            st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
-        }
+        state_from_global<false>(st, slots + ((size_t)s.init_slot * H + h) * state_elems, warp, lane);
     }
 
     int next_req = s.req_lo;
@@ -374,12 +424,7 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         // start-of-chunk state: operand copy, kept for the backward, exported when the plan requests this boundary
         state_to_operand(st, sSb, warp, lane);
         if (next_req < s.req_hi && tb.slot_chunk[next_req] == c) {
-            float* dst = slots + ((size_t)next_req * H + h) * state_elems;
-#pragma unroll
-            for (int n = 0; n < 16; n++) {
-                *reinterpret_cast<float2*>(dst + (size_t)(warp * 16 + g) * D + n * 8 + tq * 2) = make_float2(st[n][0], st[n][1]);
-                *reinterpret_cast<float2*>(dst + (size_t)(warp * 16 + g + 8) * D + n * 8 + tq * 2) = make_float2(st[n][2], st[n][3]);
-            }
+            state_to_global(st, slots + ((size_t)next_req * H + h) * state_elems, warp, lane);
             next_req++;
         }
         __syncthreads();
@@ -391,17 +436,17 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         scores_off_diagonal(s_u32(sQa), s_u32(sKa), sP, warp, lane);
         scale_qk(sQ, sK, sB, sQ, sK);
         __syncthreads();
-        // ---- o = P V + q~ S_c : warp -> rows 16*(warp & 3), columns 64*(warp >> 2) ---------------------------------
+        // ---- o = P V + q~ S_c : warp -> rows 16 * mb, columns 32 * nq ----------------------------------------------
         {
-            const int m0 = (warp & 3) * 16, n_base = (warp >> 2) * 64;
-            float acc[8][4];
+            const int m0 = mb * 16, n_base = nq * 32;
+            float acc[4][4];
 #pragma unroll
-            for (int n = 0; n < 8; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-            for (int ks = 0; ks <= (warp & 3); ks++) {      // P is zero right of the diagonal block
+            for (int n = 0; n < 4; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            for (int ks = 0; ks <= mb; ks++) {              // P is zero right of the diagonal block
                 uint32_t a[4];
                 frag_a<128>(a, aP, m0, ks * 16, lane);
 #pragma unroll
-                for (int n2 = 0; n2 < 4; n2++) {
+                for (int n2 = 0; n2 < 2; n2++) {
                     uint32_t b[4];
                     frag_b_kn<256>(b, aV, ks * 16, n_base + n2 * 16, lane);
                     mma16816(acc[2 * n2], a, b[0], b[1]);
@@ -413,7 +458,7 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
                 uint32_t a[4];
                 frag_a<256>(a, aQ, m0, ks * 16, lane);
 #pragma unroll
-                for (int n2 = 0; n2 < 4; n2++) {
+                for (int n2 = 0; n2 < 2; n2++) {
                     uint32_t b[4];
                     frag_b_kn<256>(b, aSb, ks * 16, n_base + n2 * 16, lane);
                     mma16816(acc[2 * n2], a, b[0], b[1]);
@@ -422,35 +467,16 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
             }
             const int c_lo = srow[m0 + g], c_hi = srow[m0 + g + 8];
 #pragma unroll
-            for (int n = 0; n < 8; n++) {
+            for (int n = 0; n < 4; n++) {
                 const int col = n_base + n * 8 + tq * 2;
                 if (c_lo >= 0) *reinterpret_cast<uint32_t*>(o + ((size_t)c_lo * H + h) * D + col) = pack2(acc[n][0], acc[n][1]);
                 if (c_hi >= 0) *reinterpret_cast<uint32_t*>(o + ((size_t)c_hi * H + h) * D + col) = pack2(acc[n][2], acc[n][3]);
             }
         }
-        // ---- S <- Diag(e^{b_n}) S + k~^T V : warp -> state rows 16*warp .. ------------------------------------------
-        {
-            const float g_lo = __expf(sB[(BT - 1) * D + warp * 16 + g]), g_hi = __expf(sB[(BT - 1) * D + warp * 16 + g + 8]);
-#pragma unroll
-            for (int n = 0; n < 16; n++) {
-                st[n][0] *= g_lo; st[n][1] *= g_lo; st[n][2] *= g_hi; st[n][3] *= g_hi;
-            }
-#pragma unroll
-            for (int ks = 0; ks < 4; ks++) {
-                uint32_t a[4];
-                frag_a_t<256>(a, aK, warp * 16, ks * 16, lane);
-#pragma unroll
-                for (int n2 = 0; n2 < 8; n2++) {
-                    uint32_t b[4];
-                    frag_b_kn<256>(b, aV, ks * 16, n2 * 16, lane);
-                    mma16816(st[2 * n2], a, b[0], b[1]);
-                    mma16816(st[2 * n2 + 1], a, b[2], b[3]);
-                }
-            }
-        }
+        // ---- S <- Diag(e^{b_n}) S + k~^T V ---------------------------------------------------------------------------
+        state_update(st, sB, aK, aV, warp, lane);
     }
 }
-
 
 // ---- backward ---------------------------------------------------------------------------------------------------------
 // With dS the gradient of the state at the END of the chunk on entry, dA_tj = dO_t . v_j, ew_j = e^{b_n-b_j}:
@@ -472,9 +498,9 @@ struct SharedB {
     static constexpr int p = ka + 96 * 256;                             // bf16 [64][64] scores
     static constexpr int dab = p + 8192;                                // bf16 [64][64] dA
     static constexpr int dad = dab + 8192;                              // fp32 [64][16] dA, diagonal blocks
-    static constexpr int tmp = dad + 4096;                              // fp32 [128]
-    static constexpr int rowdot = tmp + 512;                            // fp32 [128]
-    static constexpr int gi = rowdot + 512;                             // fp32 [4][128]
+    static constexpr int tmp = dad + 4096;                              // fp32 [4][128]
+    static constexpr int rowdot = tmp + 2048;                           // fp32 [2][128]
+    static constexpr int gi = rowdot + 1024;                            // fp32 [4][128]
     static constexpr int row = gi + 2048;                               // int [64]
     static constexpr int bytes = row + 256;
 };
@@ -482,11 +508,11 @@ static_assert(SharedB::bytes <= 232448, "backward tiles do not fit in shared mem
 
 // plain row-major [128][128] bf16 in global memory -> swizzled tile
 __device__ __forceinline__ void global_to_tile128(const __nv_bfloat16* src, unsigned char* tile) {
-    uint4 buf[8];
+    uint4 buf[D * 16 / NT];
 #pragma unroll
-    for (int u = 0; u < 8; u++) buf[u] = reinterpret_cast<const uint4*>(src)[threadIdx.x + u * NT];
+    for (int u = 0; u < D * 16 / NT; u++) buf[u] = reinterpret_cast<const uint4*>(src)[threadIdx.x + u * NT];
 #pragma unroll
-    for (int u = 0; u < 8; u++) {
+    for (int u = 0; u < D * 16 / NT; u++) {
         const int p = threadIdx.x + u * NT;
         *reinterpret_cast<uint4*>(tile + sw256(p >> 4, p & 15)) = buf[u];
     }
@@ -522,13 +548,13 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
 
     const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
-    const int mb = warp & 3, nh = warp >> 2;          // this warp's 16-row block and 64-column half in [64][128] products
+    const int mb = warp & 3, nq = warp >> 2;          // this warp's 16-row block and 32-column quarter of [64][128] products
     const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)D * D;
 
-    float ds[16][4];                                  // dS rows 16*warp + g (+8), all 128 columns
+    float ds[8][4];                                   // dS, laid out over the warps like the forward's state
 #pragma unroll
-    for (int n = 0; n < 16; n++) ds[n][0] = ds[n][1] = ds[n][2] = ds[n][3] = 0.f;
+    for (int n = 0; n < 8; n++) ds[n][0] = ds[n][1] = ds[n][2] = ds[n][3] = 0.f;
 
     int next_req = s.req_hi - 1;                      // slots of this sequence are ordered by chunk index
     for (int c = s.n_chunks - 1; c >= 0; c--) {
@@ -537,13 +563,8 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         // buffer by handoff_reduce)
         if (next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1) {
             if (tb.slot_cons_ptr[next_req] < tb.slot_cons_ptr[next_req + 1]) {
-                const float* src = ds0 + ((size_t)tb.slot_cons_seq[tb.slot_cons_ptr[next_req]] * H + h) * state_elems;
-#pragma unroll
-                for (int n = 0; n < 16; n++) {
-                    const float2 lo = *reinterpret_cast<const float2*>(src + (size_t)(warp * 16 + g) * D + n * 8 + tq * 2);
-                    const float2 hi = *reinterpret_cast<const float2*>(src + (size_t)(warp * 16 + g + 8) * D + n * 8 + tq * 2);
-                    ds[n][0] += lo.x; ds[n][1] += lo.y; ds[n][2] += hi.x; ds[n][3] += hi.y;
-                }
+                state_from_global<true>(ds, ds0 + ((size_t)tb.slot_cons_seq[tb.slot_cons_ptr[next_req]] * H + h) * state_elems,
+                                        warp, lane);
             }
             next_req--;
         }
@@ -560,75 +581,73 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         cumsum_rows(sB, sTmp);
         const int r_lo = 16 * mb + g, r_hi = r_lo + 8;            // this thread's rows in the [64][128] products
         // ---- dA = dO V^T, iq = dO S_c^T, ik = V dS^T, <S_c, dS> per channel -------------------------------------------
-        float iq[8][4], ik[8][4];
+        float iq[4][4], ik[4][4];
         {
-            float da[4][4];
+            float da[2][4];
 #pragma unroll
-            for (int n = 0; n < 8; n++) {
+            for (int n = 0; n < 4; n++) {
                 iq[n][0] = iq[n][1] = iq[n][2] = iq[n][3] = 0.f;
                 ik[n][0] = ik[n][1] = ik[n][2] = ik[n][3] = 0.f;
             }
 #pragma unroll
-            for (int n = 0; n < 4; n++) da[n][0] = da[n][1] = da[n][2] = da[n][3] = 0.f;
+            for (int n = 0; n < 2; n++) da[n][0] = da[n][1] = da[n][2] = da[n][3] = 0.f;
 #pragma unroll
             for (int ks = 0; ks < 8; ks++) {
                 uint32_t a[4], b[4];
                 frag_a<256>(a, aDO, 16 * mb, ks * 16, lane);
+                frag_b_nk<256>(b, aV, ks * 16, 16 * nq, lane);          // dA: columns (keys) 16 * nq ..
+                mma16816(da[0], a, b[0], b[1]);
+                mma16816(da[1], a, b[2], b[3]);
 #pragma unroll
                 for (int n2 = 0; n2 < 2; n2++) {
-                    frag_b_nk<256>(b, aV, ks * 16, 32 * nh + 16 * n2, lane);
-                    mma16816(da[2 * n2], a, b[0], b[1]);
-                    mma16816(da[2 * n2 + 1], a, b[2], b[3]);
-                }
-#pragma unroll
-                for (int n2 = 0; n2 < 4; n2++) {
-                    frag_b_nk<256>(b, aSc, ks * 16, 64 * nh + 16 * n2, lane);
+                    frag_b_nk<256>(b, aSc, ks * 16, 32 * nq + 16 * n2, lane);
                     mma16816(iq[2 * n2], a, b[0], b[1]);
                     mma16816(iq[2 * n2 + 1], a, b[2], b[3]);
                 }
                 frag_a<256>(a, aV, 16 * mb, ks * 16, lane);
 #pragma unroll
-                for (int n2 = 0; n2 < 4; n2++) {
-                    frag_b_nk<256>(b, adSb, ks * 16, 64 * nh + 16 * n2, lane);
+                for (int n2 = 0; n2 < 2; n2++) {
+                    frag_b_nk<256>(b, adSb, ks * 16, 32 * nq + 16 * n2, lane);
                     mma16816(ik[2 * n2], a, b[0], b[1]);
                     mma16816(ik[2 * n2 + 1], a, b[2], b[3]);
                 }
             }
             // dA: bf16 copy for the block products, fp32 copy of the diagonal 16-blocks for the pair sums
 #pragma unroll
-            for (int n = 0; n < 4; n++) {
-                const int col = 32 * nh + 8 * n + 2 * tq;
+            for (int n = 0; n < 2; n++) {
+                const int col = 16 * nq + 8 * n + 2 * tq;
                 *reinterpret_cast<uint32_t*>(sdAb + sw128(r_lo, col >> 3) + (col & 7) * 2) = pack2(da[n][0], da[n][1]);
                 *reinterpret_cast<uint32_t*>(sdAb + sw128(r_hi, col >> 3) + (col & 7) * 2) = pack2(da[n][2], da[n][3]);
-                if ((col >> 4) == mb) {
+                if (nq == mb) {
                     *reinterpret_cast<float2*>(sdAd + r_lo * 16 + (col & 15)) = make_float2(da[n][0], da[n][1]);
                     *reinterpret_cast<float2*>(sdAd + r_hi * 16 + (col & 15)) = make_float2(da[n][2], da[n][3]);
                 }
             }
         }
-        {   // <S_c[i,:], dS[i,:]> for the warp's 16 state rows i
+        {   // <S_c[i,:], dS[i,:]> over this warp's 64 columns of its 16 state rows i (the two column halves meet later)
+            const int i0 = (warp & 7) * 16 + g, c0 = (warp >> 3) * 64 + tq * 2;
             float d_lo = 0.f, d_hi = 0.f;
 #pragma unroll
-            for (int n = 0; n < 16; n++) {
-                const float2 s_lo = ld_bf2(sSc, warp * 16 + g, n * 8 + tq * 2), s_hi = ld_bf2(sSc, warp * 16 + g + 8, n * 8 + tq * 2);
+            for (int n = 0; n < 8; n++) {
+                const float2 s_lo = ld_bf2(sSc, i0, c0 + n * 8), s_hi = ld_bf2(sSc, i0 + 8, c0 + n * 8);
                 d_lo += s_lo.x * ds[n][0] + s_lo.y * ds[n][1];
                 d_hi += s_hi.x * ds[n][2] + s_hi.y * ds[n][3];
             }
             d_lo += __shfl_xor_sync(0xffffffffu, d_lo, 1); d_lo += __shfl_xor_sync(0xffffffffu, d_lo, 2);
             d_hi += __shfl_xor_sync(0xffffffffu, d_hi, 1); d_hi += __shfl_xor_sync(0xffffffffu, d_hi, 2);
-            if (tq == 0) { sRowdot[warp * 16 + g] = d_lo; sRowdot[warp * 16 + g + 8] = d_hi; }
+            if (tq == 0) { sRowdot[(warp >> 3) * D + i0] = d_lo; sRowdot[(warp >> 3) * D + i0 + 8] = d_hi; }
         }
         // inter-chunk parts at the fragment positions: iq <- e^{b_t} iq, ik <- ew ik, and sum_j k_j ew_j ik_j per channel
 #pragma unroll
-        for (int n = 0; n < 8; n++) {
-            const int col = 64 * nh + 8 * n + 2 * tq;
+        for (int n = 0; n < 4; n++) {
+            const int col = 32 * nq + 8 * n + 2 * tq;
             const float2 b_lo = *reinterpret_cast<const float2*>(sB + r_lo * D + col);
             const float2 b_hi = *reinterpret_cast<const float2*>(sB + r_hi * D + col);
             const float2 b_n = *reinterpret_cast<const float2*>(sB + (BT - 1) * D + col);
             const float2 k_lo = ld_bf2(sK, r_lo, col), k_hi = ld_bf2(sK, r_hi, col);
-            iq[n][0] *= __expf(b_lo.x); iq[n][1] *= __expf(b_lo.y); iq[n][2] *= __expf(b_hi.x); iq[n][3] *= __expf(b_hi.y);
-            ik[n][0] *= __expf(b_n.x - b_lo.x); ik[n][1] *= __expf(b_n.y - b_lo.y);
-            ik[n][2] *= __expf(b_n.x - b_hi.x); ik[n][3] *= __expf(b_n.y - b_hi.y);
+            iq[n][0] *= ex2(b_lo.x); iq[n][1] *= ex2(b_lo.y); iq[n][2] *= ex2(b_hi.x); iq[n][3] *= ex2(b_hi.y);
+            ik[n][0] *= ex2(b_n.x - b_lo.x); ik[n][1] *= ex2(b_n.y - b_lo.y);
+            ik[n][2] *= ex2(b_n.x - b_hi.x); ik[n][3] *= ex2(b_n.y - b_hi.y);
             float g0 = k_lo.x * ik[n][0] + k_hi.x * ik[n][2], g1 = k_lo.y * ik[n][1] + k_hi.y * ik[n][3];
 #pragma unroll
             for (int o = 4; o <= 16; o <<= 1) {
@@ -644,55 +663,55 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         scores_off_diagonal(aQa, aKa, sP, warp, lane);
         // ---- pairs in different blocks -------------------------------------------------------------------------------
         if (mb >= 1) {   // dq: rows of block mb against the keys of the blocks before it, anchored at block mb
-            float acc[8][4];
+            float acc[4][4];
 #pragma unroll
-            for (int n = 0; n < 8; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            for (int n = 0; n < 4; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
             for (int ks = 0; ks < mb; ks++) {
                 uint32_t a[4], b[4];
                 frag_a<128>(a, adAb, 16 * mb, 16 * ks, lane);
 #pragma unroll
-                for (int n2 = 0; n2 < 4; n2++) {
-                    frag_b_kn<256>(b, aKa, ka_row0(mb) + 16 * ks, 64 * nh + 16 * n2, lane);
+                for (int n2 = 0; n2 < 2; n2++) {
+                    frag_b_kn<256>(b, aKa, ka_row0(mb) + 16 * ks, 32 * nq + 16 * n2, lane);
                     mma16816(acc[2 * n2], a, b[0], b[1]);
                     mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
                 }
             }
 #pragma unroll
-            for (int n = 0; n < 8; n++) {
-                const int col = 64 * nh + 8 * n + 2 * tq;
+            for (int n = 0; n < 4; n++) {
+                const int col = 32 * nq + 8 * n + 2 * tq;
                 const float2 b_lo = *reinterpret_cast<const float2*>(sB + r_lo * D + col);
                 const float2 b_hi = *reinterpret_cast<const float2*>(sB + r_hi * D + col);
                 const float2 an = *reinterpret_cast<const float2*>(sB + 16 * mb * D + col);
-                iq[n][0] += __expf(b_lo.x - an.x) * acc[n][0]; iq[n][1] += __expf(b_lo.y - an.y) * acc[n][1];
-                iq[n][2] += __expf(b_hi.x - an.x) * acc[n][2]; iq[n][3] += __expf(b_hi.y - an.y) * acc[n][3];
+                iq[n][0] += ex2(b_lo.x - an.x) * acc[n][0]; iq[n][1] += ex2(b_lo.y - an.y) * acc[n][1];
+                iq[n][2] += ex2(b_hi.x - an.x) * acc[n][2]; iq[n][3] += ex2(b_hi.y - an.y) * acc[n][3];
             }
         }
         for (int I = mb + 1; I < 4; I++) {   // dk: keys of block mb against the queries of block I, anchored at block I
-            float acc[8][4];
+            float acc[4][4];
 #pragma unroll
-            for (int n = 0; n < 8; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            for (int n = 0; n < 4; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
             uint32_t a[4], b[4];
             frag_a_t<128>(a, adAb, 16 * mb, 16 * I, lane);
 #pragma unroll
-            for (int n2 = 0; n2 < 4; n2++) {
-                frag_b_kn<256>(b, aQa, 16 * I, 64 * nh + 16 * n2, lane);
+            for (int n2 = 0; n2 < 2; n2++) {
+                frag_b_kn<256>(b, aQa, 16 * I, 32 * nq + 16 * n2, lane);
                 mma16816(acc[2 * n2], a, b[0], b[1]);
                 mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
             }
 #pragma unroll
-            for (int n = 0; n < 8; n++) {
-                const int col = 64 * nh + 8 * n + 2 * tq;
+            for (int n = 0; n < 4; n++) {
+                const int col = 32 * nq + 8 * n + 2 * tq;
                 const float2 b_lo = *reinterpret_cast<const float2*>(sB + r_lo * D + col);
                 const float2 b_hi = *reinterpret_cast<const float2*>(sB + r_hi * D + col);
                 const float2 an = *reinterpret_cast<const float2*>(sB + 16 * I * D + col);
-                ik[n][0] += __expf(an.x - b_lo.x) * acc[n][0]; ik[n][1] += __expf(an.y - b_lo.y) * acc[n][1];
-                ik[n][2] += __expf(an.x - b_hi.x) * acc[n][2]; ik[n][3] += __expf(an.y - b_hi.y) * acc[n][3];
+                ik[n][0] += ex2(an.x - b_lo.x) * acc[n][0]; ik[n][1] += ex2(an.y - b_lo.y) * acc[n][1];
+                ik[n][2] += ex2(an.x - b_hi.x) * acc[n][2]; ik[n][3] += ex2(an.y - b_hi.y) * acc[n][3];
             }
         }
         __syncthreads();                              // the anchored operands are dead
 #pragma unroll
-        for (int n = 0; n < 8; n++) {
-            const int col = 64 * nh + 8 * n + 2 * tq;
+        for (int n = 0; n < 4; n++) {
+            const int col = 32 * nq + 8 * n + 2 * tq;
             *reinterpret_cast<float2*>(sDQ + r_lo * D + col) = make_float2(iq[n][0], iq[n][1]);
             *reinterpret_cast<float2*>(sDQ + r_hi * D + col) = make_float2(iq[n][2], iq[n][3]);
             *reinterpret_cast<float2*>(sDK + r_lo * D + col) = make_float2(ik[n][0], ik[n][1]);
@@ -700,18 +719,15 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         }
         __syncthreads();
 
-        // ---- pairs inside a 16-block and dg: thread = (channel i, half hh of the rows) --------------------------------
+        // ---- pairs inside a 16-block and dg: thread = (channel i, 16-row block blk) --------------------------------------
         {
-            const int i = tid & (D - 1), hh = tid >> 7;
+            const int i = tid & (D - 1), blk = tid >> 7, t0 = 16 * blk;
             float total = 0.f;                            // sum of q dq - k dk over this thread's rows
-            for (int blk = 2 * hh + 1; blk >= 2 * hh; blk--) {
-                const int t0 = 16 * blk;
-                float dk_acc[16];
-#pragma unroll
-                for (int u = 0; u < 16; u++) dk_acc[u] = 0.f;
-                float kf[16], bj[16];
+            {
+                float dk_acc[16], kf[16], bj[16];
 #pragma unroll
                 for (int u = 0; u < 16; u++) {
+                    dk_acc[u] = 0.f;
                     kf[u] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sK + sw256(t0 + u, i >> 3) + (i & 7) * 2));
                     bj[u] = sB[(t0 + u) * D + i];
                 }
@@ -722,7 +738,7 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
                     float dq_acc = 0.f;
 #pragma unroll
                     for (int u = 0; u <= tt; u++) {
-                        const float x = sdAd[t * 16 + u] * __expf(bj[tt] - bj[u]);     // one exponential for dq and dk
+                        const float x = sdAd[t * 16 + u] * ex2(bj[tt] - bj[u]);        // one exponential for dq and dk
                         dq_acc += x * kf[u];
                         dk_acc[u] += x * qt;
                     }
@@ -733,12 +749,13 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
                     total += qt * dqv - kf[tt] * dkv;
                 }
             }
-            if (hh == 1) sTmp[i] = total;
+            sTmp[blk * D + i] = total;
             __syncthreads();
             // dg_t = suffix over the rows + <S_{c+1}[i,:], dS[i,:]> = e^{b_n} <S_c, dS> + sum_j k_j ew_j ik_j
-            const float G = __expf(sB[(BT - 1) * D + i]) * sRowdot[i] + sGi[i] + sGi[D + i] + sGi[2 * D + i] + sGi[3 * D + i];
-            float suffix = G + (hh == 0 ? sTmp[i] : 0.f);
-            for (int t = 32 * hh + 31; t >= 32 * hh; t--) {
+            float suffix = ex2(sB[(BT - 1) * D + i]) * (sRowdot[i] + sRowdot[D + i]) + sGi[i] + sGi[D + i] + sGi[2 * D + i] +
+                           sGi[3 * D + i];
+            for (int b2 = 3; b2 > blk; b2--) suffix += sTmp[b2 * D + i];
+            for (int t = t0 + 15; t >= t0; t--) {
                 const int code = srow[t];
                 if (code == -1) continue;
                 const float qt = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sQ + sw256(t, i >> 3) + (i & 7) * 2));
@@ -751,7 +768,7 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         __syncthreads();
         // ---- dq, dk out: own rows as bf16, replayed rows' dk in fp32 to the scratch -------------------------------------
 #pragma unroll
-        for (int u = 0; u < 4; u++) {
+        for (int u = 0; u < BT * 16 / NT; u++) {
             const int p = tid + u * NT, t = p >> 4, c16 = p & 15, code = srow[t];
             if (code == -1) continue;
             const float4 q0 = *reinterpret_cast<const float4*>(sDQ + t * D + c16 * 8), q1 = *reinterpret_cast<const float4*>(sDQ + t * D + c16 * 8 + 4);
@@ -768,17 +785,17 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         }
         scale_qk(sQ, sK, sB, sQ, sK);                 // q~, k~ over the raw tiles, which nobody reads any more
         __syncthreads();
-        // ---- dv_j = sum_{t>=j} A_tj dO_t + k~_j dS : warp -> rows 16*mb, columns 64*nh ------------------------------------
+        // ---- dv_j = sum_{t>=j} A_tj dO_t + k~_j dS : warp -> rows 16 * mb, columns 32 * nq -------------------------------
         {
-            float acc[8][4];
+            float acc[4][4];
 #pragma unroll
-            for (int n = 0; n < 8; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            for (int n = 0; n < 4; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
             for (int ks = mb; ks < 4; ks++) {             // A_tj = 0 for t < j
                 uint32_t a[4], b[4];
                 frag_a_t<128>(a, aP, 16 * mb, 16 * ks, lane);
 #pragma unroll
-                for (int n2 = 0; n2 < 4; n2++) {
-                    frag_b_kn<256>(b, aDO, 16 * ks, 64 * nh + 16 * n2, lane);
+                for (int n2 = 0; n2 < 2; n2++) {
+                    frag_b_kn<256>(b, aDO, 16 * ks, 32 * nq + 16 * n2, lane);
                     mma16816(acc[2 * n2], a, b[0], b[1]);
                     mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
                 }
@@ -788,51 +805,26 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
                 uint32_t a[4], b[4];
                 frag_a<256>(a, aK, 16 * mb, 16 * ks, lane);
 #pragma unroll
-                for (int n2 = 0; n2 < 4; n2++) {
-                    frag_b_kn<256>(b, adSb, 16 * ks, 64 * nh + 16 * n2, lane);
+                for (int n2 = 0; n2 < 2; n2++) {
+                    frag_b_kn<256>(b, adSb, 16 * ks, 32 * nq + 16 * n2, lane);
                     mma16816(acc[2 * n2], a, b[0], b[1]);
                     mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
                 }
             }
             const int c_lo = srow[r_lo], c_hi = srow[r_hi];
 #pragma unroll
-            for (int n = 0; n < 8; n++) {
-                const int col = 64 * nh + 8 * n + 2 * tq;
+            for (int n = 0; n < 4; n++) {
+                const int col = 32 * nq + 8 * n + 2 * tq;
                 if (c_lo >= 0) *reinterpret_cast<uint32_t*>(dv_ + ((size_t)c_lo * H + h) * D + col) = pack2(acc[n][0], acc[n][1]);
                 else if (c_lo < -1) *reinterpret_cast<float2*>(rv + ((size_t)(s.replay_base + r_lo) * H + h) * D + col) = make_float2(acc[n][0], acc[n][1]);
                 if (c_hi >= 0) *reinterpret_cast<uint32_t*>(dv_ + ((size_t)c_hi * H + h) * D + col) = pack2(acc[n][2], acc[n][3]);
                 else if (c_hi < -1) *reinterpret_cast<float2*>(rv + ((size_t)(s.replay_base + r_hi) * H + h) * D + col) = make_float2(acc[n][2], acc[n][3]);
             }
         }
-        // ---- dS <- Diag(e^{b_n}) dS + q~^T dO : warp -> state rows 16*warp .. ---------------------------------------------
-        {
-            const float g_lo = __expf(sB[(BT - 1) * D + warp * 16 + g]), g_hi = __expf(sB[(BT - 1) * D + warp * 16 + g + 8]);
-#pragma unroll
-            for (int n = 0; n < 16; n++) {
-                ds[n][0] *= g_lo; ds[n][1] *= g_lo; ds[n][2] *= g_hi; ds[n][3] *= g_hi;
-            }
-#pragma unroll
-            for (int ks = 0; ks < 4; ks++) {
-                uint32_t a[4];
-                frag_a_t<256>(a, aQ, warp * 16, ks * 16, lane);
-#pragma unroll
-                for (int n2 = 0; n2 < 8; n2++) {
-                    uint32_t b[4];
-                    frag_b_kn<256>(b, aDO, ks * 16, n2 * 16, lane);
-                    mma16816(ds[2 * n2], a, b[0], b[1]);
-                    mma16816(ds[2 * n2 + 1], a, b[2], b[3]);
-                }
-            }
-        }
+        // ---- dS <- Diag(e^{b_n}) dS + q~^T dO ---------------------------------------------------------------------------
+        state_update(ds, sB, aQ, aDO, warp, lane);
     }
-    if (s.init_slot >= 0) {
-        float* dst = ds0 + ((size_t)seq * H + h) * state_elems;
-#pragma unroll
-        for (int n = 0; n < 16; n++) {
-            *reinterpret_cast<float2*>(dst + (size_t)(warp * 16 + g) * D + n * 8 + tq * 2) = make_float2(ds[n][0], ds[n][1]);
-            *reinterpret_cast<float2*>(dst + (size_t)(warp * 16 + g + 8) * D + n * 8 + tq * 2) = make_float2(ds[n][2], ds[n][3]);
-        }
-    }
+    if (s.init_slot >= 0) state_to_global(ds, ds0 + ((size_t)seq * H + h) * state_elems, warp, lane);
 }
 
 }  // namespace
