@@ -398,7 +398,10 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
     int* srow = reinterpret_cast<int*>(sm + Shared::row);
     const uint32_t aQ = s_u32(sQ), aK = s_u32(sK), aV = s_u32(sV), aP = s_u32(sP), aSb = s_u32(sSb);
 
-    const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
+    // blocks are handed to the SMs in index order: with the plan's order (longest sequence of the round first) the long
+    // walks start first and the short ones fill the tail
+    const int seq_pos = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
+    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
     const int mb = warp & 3, nq = warp >> 2;          // this warp's 16-row block and 32-column quarter of [64][128] products
     const SeqInfo s = seq_info(tb, seq);
@@ -546,7 +549,10 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
     const uint32_t aQ = s_u32(sQ), aK = s_u32(sK), aV = s_u32(sV), aDO = s_u32(sDO), aSc = s_u32(sSc), adSb = s_u32(sdSb),
                    aQa = s_u32(sQa), aKa = s_u32(sKa), aP = s_u32(sP), adAb = s_u32(sdAb);
 
-    const int seq = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
+    // blocks are handed to the SMs in index order: with the plan's order (longest sequence of the round first) the long
+    // walks start first and the short ones fill the tail
+    const int seq_pos = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
+    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
     const int mb = warp & 3, nq = warp >> 2;          // this warp's 16-row block and 32-column quarter of [64][128] products
     const SeqInfo s = seq_info(tb, seq);
