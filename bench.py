@@ -403,7 +403,7 @@ class LaWorkload:
         Hh, dk, dv = cfg["H"], cfg["dk"], cfg["dv"]
         # every rank draws its own tensors (independent batches of the same shape)
         self.inp = inp = make_inputs(plan.C, Hh, dk, dv, cfg["dtype"], cfg["seed"] + 100 * ranks.rank, device="cuda")
-        self.flags = (H.HARTS_FLAG_FMA_KERNELS if args.fma else 0)
+        self.flags = (H.HARTS_FLAG_FMA_KERNELS if args.fma else 0) | (H.HARTS_FLAG_ROUND_LAUNCHES if args.round_launches else 0)
         self.ws = H.Workspace(plan, Hh, dk, dv, inp["q"].dtype, self.flags)
         self.out = {"o": torch.empty_like(inp["v"]), "dq": torch.empty_like(inp["q"]), "dk": torch.empty_like(inp["k"]),
                     "dv": torch.empty_like(inp["v"]), "dg": torch.empty_like(inp["g"])}
@@ -453,7 +453,7 @@ class LaWorkload:
         import torch
         sms = torch.cuda.get_device_properties(0).multi_processor_count
         tc = self.cfg["dk"] == 128 and not self.args.fma and self.inp["q"].element_size() == 2
-        ok = tc and 1 < self.plan.n_rounds <= 32
+        ok = tc and 1 < self.plan.n_rounds <= 32 and not self.args.round_launches
         items = self.plan.n_seq * self.cfg["H"]
         return ok and items <= 16 * sms, ok and items <= 8 * sms
 
@@ -1149,6 +1149,8 @@ def main(argv=None):
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--blocks", type=int, default=0, help="timed blocks of --steps steps (0: enough for ~2 s)")
     ap.add_argument("--fma", action="store_true", help="force the fp32-FMA kernels")
+    ap.add_argument("--round-launches", action="store_true",
+                    help="one launch per round also on small problems (HARTS_FLAG_ROUND_LAUNCHES)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
