@@ -251,30 +251,44 @@ __device__ __forceinline__ void scores_off_diagonal(uint32_t aQa, uint32_t aKa, 
     }
 }
 
-// diagonal blocks: one warp per row t, every lane takes 4 channels of all (at most 16) pairs of the row, the warp sums
-// them with a transposed reduction; lanes 0..15 then hold A[t][16 I + lane] (zero right of the diagonal)
-__device__ __forceinline__ void scores_diagonal(const unsigned char* sQ, const unsigned char* sK, const float* sB,
+// one-step decay factors 2^{b_t - b_{t-1}} of the rows 1..63 of a chunk (fp32 [BT][128]; row 0 is not used: the factors
+// serve pairs inside a 16-row block only)
+__device__ __forceinline__ void step_factors(const float* sB, float* sR) {
+    for (int p = threadIdx.x; p < BT * 32; p += NT) {
+        const int t = p >> 5, c4 = p & 31;
+        if (t == 0) continue;
+        const float4 hi = *reinterpret_cast<const float4*>(sB + t * D + c4 * 4);
+        const float4 lo = *reinterpret_cast<const float4*>(sB + (t - 1) * D + c4 * 4);
+        *reinterpret_cast<float4*>(sR + t * D + c4 * 4) = make_float4(ex2(hi.x - lo.x), ex2(hi.y - lo.y), ex2(hi.z - lo.z), ex2(hi.w - lo.w));
+    }
+}
+
+// diagonal blocks: one warp per row t, every lane takes 4 channels of all (at most 16) pairs of the row, walking j from t
+// down with the decay as a running product of the one-step factors (x_{t,j-1} = x_{t,j} r_j: every factor <= 1, no
+// exponential per pair); the warp sums the lanes with a transposed reduction, lanes 0..15 then hold A[t][16 I + lane]
+// (zero right of the diagonal)
+__device__ __forceinline__ void scores_diagonal(const unsigned char* sQ, const unsigned char* sK, const float* sR,
                                                 unsigned char* sP, int warp, int lane) {
-    for (int t = warp; t < BT; t += NT / 32) {
+    for (int t = warp; t < BT; t += NW) {
         const int j_lo = t & ~15;
         const uint2 qraw = *reinterpret_cast<const uint2*>(sQ + sw256(t, lane >> 1) + (lane & 1) * 8);
-        const float4 bt = *reinterpret_cast<const float4*>(sB + t * D + lane * 4);
         const float2 q01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&qraw.x));
         const float2 q23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&qraw.y));
+        float4 qx = make_float4(q01.x, q01.y, q23.x, q23.y);          // q_t .* x_{t,j}, j walking down from t
         float z[16];
 #pragma unroll
-        for (int u = 0; u < 16; u++) {
+        for (int u = 15; u >= 0; u--) {
             const int j = j_lo + u;
             float acc = 0.f;
             if (j <= t) {
                 const uint2 kraw = *reinterpret_cast<const uint2*>(sK + sw256(j, lane >> 1) + (lane & 1) * 8);
-                const float4 bj = *reinterpret_cast<const float4*>(sB + j * D + lane * 4);
                 const float2 k01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kraw.x));
                 const float2 k23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kraw.y));
-                acc = q01.x * k01.x * ex2(bt.x - bj.x);
-                acc += q01.y * k01.y * ex2(bt.y - bj.y);
-                acc += q23.x * k23.x * ex2(bt.z - bj.z);
-                acc += q23.y * k23.y * ex2(bt.w - bj.w);
+                acc = qx.x * k01.x + qx.y * k01.y + qx.z * k23.x + qx.w * k23.y;
+                if (u > 0) {
+                    const float4 r = *reinterpret_cast<const float4*>(sR + j * D + lane * 4);
+                    qx.x *= r.x; qx.y *= r.y; qx.z *= r.z; qx.w *= r.w;
+                }
             }
             z[u] = acc;
         }
@@ -321,7 +335,8 @@ struct Shared {
     static constexpr int b = 90112;                             // fp32 [64][128]: running log-decay (log2 units)
     static constexpr int qa = 122880;                           // bf16 [64][128]: q anchored at its 16-row block
     static constexpr int ka = qa + 16384;                       // bf16 [96][128]: k anchored at blocks 1, 2, 3
-    static constexpr int tmp = ka + 96 * 256;                   // fp32 [4][128]
+    static constexpr int r = ka + 96 * 256;                     // fp32 [64][128]: one-step decay factors
+    static constexpr int tmp = r + 32768;                       // fp32 [4][128]
     static constexpr int row = tmp + 2048;                      // int  [64]
     static constexpr int fwd_bytes = row + 256;
 };
@@ -394,6 +409,7 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
     unsigned char *sQ = sm + Shared::q, *sK = sm + Shared::k, *sV = sm + Shared::v, *sP = sm + Shared::p,
                   *sSb = sm + Shared::sb, *sQa = sm + Shared::qa, *sKa = sm + Shared::ka;
     float* sB = reinterpret_cast<float*>(sm + Shared::b);
+    float* sR = reinterpret_cast<float*>(sm + Shared::r);
     float* sTmp = reinterpret_cast<float*>(sm + Shared::tmp);
     int* srow = reinterpret_cast<int*>(sm + Shared::row);
     const uint32_t aQ = s_u32(sQ), aK = s_u32(sK), aV = s_u32(sV), aP = s_u32(sP), aSb = s_u32(sSb);
@@ -433,10 +449,12 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         __syncthreads();
         if (chunk_states) tile_to_global<D>(sSb, chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems);
         cumsum_rows(sB, sTmp);
+        step_factors(sB, sR);
         anchored_operands(sQ, sK, sB, sQa, sKa);
-        scores_diagonal(sQ, sK, sB, sP, warp, lane);
         __syncthreads();
+        scores_diagonal(sQ, sK, sR, sP, warp, lane);
         scores_off_diagonal(s_u32(sQa), s_u32(sKa), sP, warp, lane);
+        __syncthreads();
         scale_qk(sQ, sK, sB, sQ, sK);
         __syncthreads();
         // ---- o = P V + q~ S_c : warp -> rows 16 * mb, columns 32 * nq ----------------------------------------------
@@ -539,7 +557,8 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
                   *sSc = sm + SharedB::sc, *sdSb = sm + SharedB::dsb, *sQa = sm + SharedB::qa, *sKa = sm + SharedB::ka,
                   *sP = sm + SharedB::p, *sdAb = sm + SharedB::dab;
     float* sB = reinterpret_cast<float*>(sm + SharedB::b);
-    float* sDQ = reinterpret_cast<float*>(sm + SharedB::sc);       // after S_c is dead
+    float* sR = reinterpret_cast<float*>(sm + SharedB::sc);        // one-step decay factors, after S_c is dead
+    float* sDQ = reinterpret_cast<float*>(sm + SharedB::sc);       // after the step factors are dead
     float* sDK = reinterpret_cast<float*>(sm + SharedB::qa);       // after the anchored operands are dead
     float* sdAd = reinterpret_cast<float*>(sm + SharedB::dad);
     float* sTmp = reinterpret_cast<float*>(sm + SharedB::tmp);
@@ -664,8 +683,8 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         }
         // ---- scores and the anchored operands ------------------------------------------------------------------------
         anchored_operands(sQ, sK, sB, sQa, sKa);
-        scores_diagonal(sQ, sK, sB, sP, warp, lane);
-        __syncthreads();                              // S_c is dead from here on; dA, anchored operands, diagonal scores visible
+        __syncthreads();                              // S_c is dead from here on; dA and the anchored operands are visible
+        step_factors(sB, sR);                         // over the dead S_c tile
         scores_off_diagonal(aQa, aKa, sP, warp, lane);
         // ---- pairs in different blocks -------------------------------------------------------------------------------
         if (mb >= 1) {   // dq: rows of block mb against the keys of the blocks before it, anchored at block mb
@@ -714,14 +733,20 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
                 ik[n][2] += ex2(an.x - b_hi.x) * acc[n][2]; ik[n][3] += ex2(an.y - b_hi.y) * acc[n][3];
             }
         }
-        __syncthreads();                              // the anchored operands are dead
+        __syncthreads();                              // the anchored operands are dead, the step factors visible
+        scores_diagonal(sQ, sK, sR, sP, warp, lane);
+#pragma unroll
+        for (int n = 0; n < 4; n++) {
+            const int col = 32 * nq + 8 * n + 2 * tq;
+            *reinterpret_cast<float2*>(sDK + r_lo * D + col) = make_float2(ik[n][0], ik[n][1]);
+            *reinterpret_cast<float2*>(sDK + r_hi * D + col) = make_float2(ik[n][2], ik[n][3]);
+        }
+        __syncthreads();                              // the step factors are dead
 #pragma unroll
         for (int n = 0; n < 4; n++) {
             const int col = 32 * nq + 8 * n + 2 * tq;
             *reinterpret_cast<float2*>(sDQ + r_lo * D + col) = make_float2(iq[n][0], iq[n][1]);
             *reinterpret_cast<float2*>(sDQ + r_hi * D + col) = make_float2(iq[n][2], iq[n][3]);
-            *reinterpret_cast<float2*>(sDK + r_lo * D + col) = make_float2(ik[n][0], ik[n][1]);
-            *reinterpret_cast<float2*>(sDK + r_hi * D + col) = make_float2(ik[n][2], ik[n][3]);
         }
         __syncthreads();
 
@@ -730,30 +755,43 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
             const int i = tid & (D - 1), blk = tid >> 7, t0 = 16 * blk;
             float total = 0.f;                            // sum of q dq - k dk over this thread's rows
             {
-                float dk_acc[16], kf[16], bj[16];
+                // rows ascending; xr[u] = 2^{b_t - b_u} as a running product of the one-step factors (one exponential per
+                // row instead of one per pair; every factor <= 1), the same factor for dq and dk
+                float dk_acc[16], kf[16], xr[16];
 #pragma unroll
                 for (int u = 0; u < 16; u++) {
                     dk_acc[u] = 0.f;
                     kf[u] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sK + sw256(t0 + u, i >> 3) + (i & 7) * 2));
-                    bj[u] = sB[(t0 + u) * D + i];
                 }
+                float b_prev = 0.f;
 #pragma unroll
-                for (int tt = 15; tt >= 0; tt--) {
+                for (int tt = 0; tt < 16; tt++) {
                     const int t = t0 + tt;
                     const float qt = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sQ + sw256(t, i >> 3) + (i & 7) * 2));
+                    const float bt = sB[t * D + i];
+                    const float r = ex2(bt - b_prev);
+                    b_prev = bt;
+                    xr[tt] = 1.f;
                     float dq_acc = 0.f;
 #pragma unroll
                     for (int u = 0; u <= tt; u++) {
-                        const float x = sdAd[t * 16 + u] * ex2(bj[tt] - bj[u]);        // one exponential for dq and dk
+                        if (u < tt) xr[u] *= r;
+                        const float x = sdAd[t * 16 + u] * xr[u];
                         dq_acc += x * kf[u];
                         dk_acc[u] += x * qt;
                     }
-                    const float dqv = sDQ[t * D + i] + dq_acc;
-                    const float dkv = sDK[t * D + i] + dk_acc[tt];
-                    sDQ[t * D + i] = dqv;
-                    sDK[t * D + i] = dkv;
-                    total += qt * dqv - kf[tt] * dkv;
+                    sDQ[t * D + i] += dq_acc;
                 }
+#pragma unroll
+                for (int tt = 0; tt < 16; tt++) sDK[(t0 + tt) * D + i] += dk_acc[tt];
+            }
+            // sum of q dq - k dk over this thread's rows
+#pragma unroll 4
+            for (int tt = 0; tt < 16; tt++) {
+                const int t = t0 + tt;
+                const float qt = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sQ + sw256(t, i >> 3) + (i & 7) * 2));
+                const float kt = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sK + sw256(t, i >> 3) + (i & 7) * 2));
+                total += qt * sDQ[t * D + i] - kt * sDK[t * D + i];
             }
             sTmp[blk * D + i] = total;
             __syncthreads();
