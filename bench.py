@@ -427,7 +427,7 @@ class LaWorkload:
             marks.append((name, a, b))
 
         if self.one_launch()[0]:
-            # round 0 = all rounds; on a problem this small the library runs them in one cooperative launch per pass, and
+            # round 0 = all rounds; on a problem this small the library runs them in one launch per pass, and
             # the backward call includes the replay-gradient fold
             timed("fwd", lambda: H.harts_la_fwd(plan, 0, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], ws.slots,
                                                ws.chunk_states, self.flags, ws.dev_status))
@@ -447,7 +447,7 @@ class LaWorkload:
         timed("fold", lambda: H.harts_la_bwd_finish(plan.tables, out["dk"], out["dv"], out["dg"], ws.scratch))
 
     def one_launch(self):
-        """(forward, backward): True where the library's all-rounds call runs as one cooperative launch -- bf16 d = 128
+        """(forward, backward): True where the library's all-rounds call runs as one launch per pass -- bf16 d = 128
         kernels, more than one round, and at most 8 (sequence, head) items per resident CTA (two CTAs per SM in the
         forward, one in the backward)."""
         import torch
@@ -542,7 +542,7 @@ class LaWorkload:
     def launches_per_step(self):
         """Kernels per step: one launch per round and pass (each backward round preceded by the hand-off reduction when
         the plan exports boundaries) plus the replay-gradient fold -- or, on problems with few items per CTA, one
-        cooperative launch for all forward rounds and one for all backward rounds."""
+        launch for all forward rounds and one for all backward rounds."""
         plan, K = self.plan, self.plan.n_rounds
         one_fwd, one_bwd = self.one_launch()
         fwd = 1 if one_fwd else K

@@ -58,11 +58,12 @@ extern "C" {
  * harts_la_tables_t; dev_status[2] = position), the kernels of this and of later calls with the flag return without
  * reading or writing anything, and harts_la_check() reports HARTS_EINVAL.  Needs dev_status (at least 4 int32). */
 #define HARTS_FLAG_CHECK_TABLES 2u
-/* harts_la_fwd / harts_la_bwd with round 0 run ALL rounds in one cooperative launch when the problem is small enough
- * for every (sequence, head) to have a CTA of its own (bf16, dk = dv = 128): a sequence then waits for the flag of the
- * boundary state it starts from (backward: for the initial-state gradients of the sequences that started at a
- * boundary) instead of for the end of the previous round's kernel, so the rounds overlap as far as the tree allows.
- * Same arithmetic, same bits.  With this flag every round gets its own launch, as with explicit round numbers. */
+/* harts_la_fwd / harts_la_bwd with round 0 run ALL rounds in one launch per pass when the problem has few (sequence,
+ * head) work items per persistent CTA (bf16, dk = dv = 128, at most 32 rounds): the CTAs draw the items from a ticket
+ * counter in round order, and a sequence waits for the flag of the boundary state it starts from (backward: for the
+ * initial-state gradients of the sequences that started at a boundary) instead of for the end of the previous round's
+ * kernel, so the rounds overlap as far as the tree allows.  Same arithmetic, same bits.  With this flag every round
+ * gets its own launch, as with explicit round numbers. */
 #define HARTS_FLAG_ROUND_LAUNCHES 16u
 
 typedef struct harts_la_plan harts_la_plan_t; /* opaque, host memory, library-owned */

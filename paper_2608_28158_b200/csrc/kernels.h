@@ -116,7 +116,7 @@ int32_t fma_fwd(const FwdArgs& a);
 int32_t fma_bwd(const BwdArgs& a);
 int32_t tc_supported(int32_t dtype, int32_t dk, int32_t dv);
 int32_t tc_fwd(const FwdArgs& a);
-int32_t tc_fwd_fused(const FwdArgs& a, int* flags, int* ticket);     // all rounds in one cooperative launch
+int32_t tc_fwd_fused(const FwdArgs& a, int* flags, int* ticket);     // all rounds in one launch
 
 // Flags for the one-launch forms, kept behind the chunk states in the chunk-state workspace: one int32 per
 // (slot, head) for the forward, one per (sequence, head) for the backward.

@@ -205,7 +205,7 @@ __device__ __forceinline__ void frag_store(uint32_t stage, int lane, int Lq, int
     }
 }
 
-// ONE_LAUNCH: all rounds in one cooperative launch (work items drawn from `ticket`, hand-off gradients published
+// ONE_LAUNCH: all rounds in one launch (work items drawn from `ticket`, hand-off gradients published
 // and awaited through `ds0_flags`); otherwise one round per launch and neither pointer is looked at.
 template <bool ONE_LAUNCH>
 __global__ void __launch_bounds__(NT, 1)
@@ -880,20 +880,21 @@ int32_t tc_bwd(const BwdArgs& a) {
 }
 
 
-// All rounds of a plan in ONE cooperative launch: the persistent CTAs draw the (sequence, head) items from a ticket
-// counter, last round first.  A sequence publishes a flag once its initial-state gradient is in the scratch area; a
-// sequence that exported a boundary waits (its auxiliary warp does, one chunk ahead) for the flags of all the
-// sequences that started there and sums their gradients itself, in the order handoff_reduce uses.  Those sequences
-// sit in later rounds, hold smaller tickets and are running or done: no deadlock while all CTAs are resident, which
-// the cooperative launch guarantees.  `flags`: caller-owned DEVICE array of n_seq * H int32, `ticket`: one int32; both
-// zeroed here on the stream.  rounds: the plan's round table (sequences of round r = [ptr[r], ptr[r+1])).
+// All rounds of a plan in ONE launch: the persistent CTAs draw the (sequence, head) items from a ticket counter, last
+// round first.  A sequence publishes a flag once its initial-state gradient is in the scratch area; a sequence that
+// exported a boundary waits (its auxiliary warp does, one chunk ahead) for the flags of all the sequences that started
+// there and sums their gradients itself, in the order handoff_reduce uses.  Those sequences sit in later rounds and
+// hold smaller tickets, and a ticket is only ever held by a running CTA: they are running or done whether or not the
+// whole grid is resident, so an ordinary launch cannot deadlock.  `flags`: caller-owned DEVICE array of n_seq * H
+// int32, `ticket`: one int32; both zeroed here on the stream.  rounds: the plan's round table (sequences of round r =
+// [ptr[r], ptr[r+1])).
 int32_t tc_bwd_fused(const BwdArgs& a, int* flags, int* ticket, const RoundOrder& rounds) {
     const int n = (a.seq_hi - a.seq_lo) * a.H;
     if (n == 0) return HARTS_OK;
     if (rounds.n < 1 || rounds.ptr[0] != a.seq_lo || rounds.ptr[rounds.n] != a.seq_hi) return HARTS_EINVAL;
-    // offered while a CTA gets few items, where the idle tail of every round is what one launch saves (cfg2, 7.5 items
-    // per CTA: 1.92 -> 1.79 ms); with many items per CTA it gains nothing (cfg3: 12.8 ms either way) or loses (cfg4,
-    // 1,800 short items per CTA whose hand-off sums then run inside the kernel: 43 -> 64 ms)
+    // offered while a CTA gets few items, where the idle tail of every round is what one launch saves (cfg1: 0.55 ->
+    // 0.35 ms; cfg2, 7.5 items per CTA: 1.85 -> 1.72 ms); with many items per CTA it loses (cfg3: 12.05 -> 12.45 ms;
+    // cfg4, 1,800 short items per CTA whose hand-off sums then run inside the walk: 42 -> 62 ms)
     if (n > ONE_LAUNCH_ITEMS_PER_CTA * sm_count()) return HARTS_EUNSUPPORTED;
     CUtensorMap mq, mk, mv, mdo, mcs, mdq, mdk, mdv;
     int32_t rc;
@@ -912,26 +913,13 @@ int32_t tc_bwd_fused(const BwdArgs& a, int* flags, int* ticket, const RoundOrder
     if (cudaMemsetAsync(ticket, 0, sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
     ScratchLayout sl = scratch_layout(a.tb, a.H, a.dk, a.dv);
     char* base = static_cast<char*>(a.scratch);
-    harts_la_tables_t tb = a.tb;
-    int seq_lo = a.seq_lo, n_items = n, H = a.H;
     const int grid = n < sm_count() ? n : sm_count();
-    RoundOrder ro = rounds;
-    const __nv_bfloat16 *q = (const __nv_bfloat16*)a.q, *k = (const __nv_bfloat16*)a.k, *v = (const __nv_bfloat16*)a.v,
-                        *dO = (const __nv_bfloat16*)a.dO;
-    const float* g = a.g;
-    __nv_bfloat16 *dq = (__nv_bfloat16*)a.dq, *dk_ = (__nv_bfloat16*)a.dk_, *dv_ = (__nv_bfloat16*)a.dv_;
-    float *dg = a.dg, *ds0 = (float*)(base + sl.ds0), *rk = (float*)(base + sl.rk), *rv = (float*)(base + sl.rv),
-          *rg = (float*)(base + sl.rg);
-    int* status = a.dev_status;
-    const int32_t* gate = status_gate(a.flags, a.dev_status);
-    void* args[] = {&tb, &seq_lo, &n_items, &H, &mq, &mk, &mv, &mdo, &mcs, &mdq, &mdk, &mdv, &q, &k, &v, &g, &dO, &dq, &dk_,
-                    &dv_, &dg, &ds0, &rk, &rv, &rg, &status, &gate, &flags, &ticket, &ro};
-    if (cudaLaunchCooperativeKernel((const void*)tc_bwd_kernel<true>, dim3(grid), dim3(NT), args, Smem::bytes + 1024, a.stream) !=
-        cudaSuccess) {
-        (void)cudaGetLastError();
-        return HARTS_EUNSUPPORTED;
-    }
-    return HARTS_OK;
+    tc_bwd_kernel<true><<<grid, NT, Smem::bytes + 1024, a.stream>>>(
+        a.tb, a.seq_lo, n, a.H, mq, mk, mv, mdo, mcs, mdq, mdk, mdv, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
+        (const __nv_bfloat16*)a.v, a.g, (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_,
+        (__nv_bfloat16*)a.dv_, a.dg, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
+        (float*)(base + sl.rg), a.dev_status, status_gate(a.flags, a.dev_status), flags, ticket, rounds);
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
 }  // namespace harts

@@ -75,7 +75,7 @@ __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq
 // out of line: the wait loop's registers (timer values, counters) must not weigh on the kernel's allocation
 __device__ __noinline__ void wait_for_slot(const int* flag, int* status, int* dead) { flag_wait(flag, status, dead); }
 
-// ONE_LAUNCH: all rounds in one cooperative launch (work items drawn from `ticket`, sequences wait on `slot_flags`);
+// ONE_LAUNCH: all rounds in one launch (work items drawn from `ticket`, sequences wait on `slot_flags`);
 // otherwise one round per launch, items dealt statically, and neither pointer is looked at.
 template <bool ONE_LAUNCH>
 __global__ void __launch_bounds__(NT, 2)
@@ -534,11 +534,12 @@ int32_t tc_fwd(const FwdArgs& a) {
 // All rounds of a plan in ONE launch: sequences [seq_lo, seq_hi) span several rounds (they are numbered round by
 // round), the persistent CTAs draw the work items in that order from a ticket counter, and a sequence that starts from
 // an exported state waits for the flag its producer sets after writing the slot (which it does when it passes the
-// boundary, not at its end).  A waiting item's producer sits in an earlier round, so it holds a smaller ticket and is
-// running or done: no deadlock as long as all CTAs are resident, which the cooperative launch guarantees (it fails
-// otherwise, and the caller falls back to one launch per round).  Which CTA computes an item does not change its
-// arithmetic: the results equal those of one launch per round bit for bit.  `flags`: caller-owned DEVICE array of
-// n_slots * H int32, `ticket`: one int32; both zeroed here on the stream.
+// boundary, not at its end).  A waiting item's producer sits in an earlier round, so it holds a smaller ticket -- and a
+// ticket is only ever held by a CTA that is running: the producer is running or done whether or not every CTA of the
+// grid is resident, so an ordinary launch cannot deadlock (a CTA that is not yet resident holds no ticket and nobody
+// waits for it).  Which CTA computes an item does not change its arithmetic: the results equal those of one launch
+// per round bit for bit.  `flags`: caller-owned DEVICE array of n_slots * H int32, `ticket`: one int32; both zeroed
+// here on the stream.
 int32_t tc_fwd_fused(const FwdArgs& a, int* flags, int* ticket) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
     CUtensorMap mq, mk, mv, mcs, mo;
@@ -552,39 +553,22 @@ int32_t tc_fwd_fused(const FwdArgs& a, int* flags, int* ticket) {
     if (cudaFuncSetAttribute(tc_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes + 1024) !=
         cudaSuccess)
         return HARTS_ECUDA;
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tc_fwd_kernel<true>, NT, Smem::bytes + 1024) != cudaSuccess ||
-        per_sm < 1)
-        return HARTS_EUNSUPPORTED;
-    if (per_sm > 2) per_sm = 2;
     // Offered while a CTA gets few items (at most ONE_LAUNCH_ITEMS_PER_CTA on average): there the idle tail of every
-    // round, about one item long, is what one launch saves (cfg2, 3.7 items per CTA: forward 1.25 -> 1.20 ms; cfg1, one
-    // item per CTA: 0.97 -> 0.62 ms forward + backward).  With many items per CTA one launch per round is faster
-    // (cfg3, 28 items per CTA: 6.2 ms against 8.7, with no time spent waiting on flags).
-    if ((int64_t)(a.seq_hi - a.seq_lo) * a.H > (int64_t)ONE_LAUNCH_ITEMS_PER_CTA * per_sm * sm_count())
-        return HARTS_EUNSUPPORTED;
+    // round, about one item long, is what one launch saves (cfg1, one item per CTA: forward 0.38 -> 0.26 ms; cfg2, 3.7
+    // items per CTA: 1.24 -> 1.03 ms).  With many items per CTA nothing is left to gain (cfg3, 28 items per CTA: 5.98
+    // against 6.03 ms) and the per-item flag traffic costs (cfg4, 900 short items per CTA: 16.7 against 18.0 ms).
+    if ((int64_t)(a.seq_hi - a.seq_lo) * a.H > (int64_t)ONE_LAUNCH_ITEMS_PER_CTA * 2 * sm_count()) return HARTS_EUNSUPPORTED;
     if (a.tb.n_slots > 0 &&
         cudaMemsetAsync(flags, 0, (size_t)a.tb.n_slots * a.H * sizeof(int), a.stream) != cudaSuccess)
         return HARTS_ECUDA;
     if (cudaMemsetAsync(ticket, 0, sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
     int n = (a.seq_hi - a.seq_lo) * a.H;
-    int grid = n < per_sm * sm_count() ? n : per_sm * sm_count();
-    harts_la_tables_t tb = a.tb;
-    int seq_lo = a.seq_lo, H = a.H, store = a.chunk_states != nullptr;
-    const __nv_bfloat16 *q = (const __nv_bfloat16*)a.q, *k = (const __nv_bfloat16*)a.k, *v = (const __nv_bfloat16*)a.v;
-    const float* g = a.g;
-    __nv_bfloat16* o = (__nv_bfloat16*)a.o;
-    float* slots = a.slots;
-    int* status = a.dev_status;
-    const int32_t* gate = status_gate(a.flags, a.dev_status);
-    void* args[] = {&tb, &seq_lo, &n, &H, &mq, &mk, &mv, &mcs, &mo, &q, &k, &v, &g, &o, &slots, &store, &status, &gate,
-                    &flags, &ticket};
-    if (cudaLaunchCooperativeKernel((const void*)tc_fwd_kernel<true>, dim3(grid), dim3(NT), args, Smem::bytes + 1024,
-                                    a.stream) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return HARTS_EUNSUPPORTED;                 // the caller launches round by round instead
-    }
-    return HARTS_OK;
+    int grid = n < 2 * sm_count() ? n : 2 * sm_count();
+    tc_fwd_kernel<true><<<grid, NT, Smem::bytes + 1024, a.stream>>>(
+        a.tb, a.seq_lo, n, a.H, mq, mk, mv, mcs, mo, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k,
+        (const __nv_bfloat16*)a.v, a.g, (__nv_bfloat16*)a.o, a.slots, a.chunk_states != nullptr, a.dev_status,
+        status_gate(a.flags, a.dev_status), flags, ticket);
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
 }  // namespace harts

@@ -93,7 +93,7 @@ __device__ __forceinline__ void mbar_expect_tx_only(uint64_t* bar, uint32_t byte
     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 
-// ---- flags between CTAs of one (cooperative) launch -----------------------------------------------------------------------
+// ---- flags between CTAs of one launch --------------------------------------------------------------------------------------
 // A CTA that has produced something another CTA of the same launch consumes publishes a flag in global memory; the
 // consumer polls it.  Every writer of the data fences before the CTA-wide barrier that precedes flag_set; the consumer
 // reads the data only after flag_wait returned true and a CTA-wide barrier.  The wait is bounded like the others (a

@@ -130,7 +130,7 @@ def test_random_forests_through_the_tensor_core_kernels():
 
 
 def test_all_rounds_in_one_launch_give_the_bits_of_one_launch_per_round():
-    """Problems with few (sequence, head) items per CTA run all rounds in one cooperative launch: the CTAs draw the
+    """Problems with few (sequence, head) items per CTA run all rounds in one launch: the CTAs draw the
     items from a ticket counter and the sequences wait for each other through flags instead of kernel boundaries.  Outputs, gradients, exported states
     and chunk states must equal, bit for bit, those of one launch per round -- on forests with several consumers per
     boundary, replayed first chunks and three rounds."""
