@@ -971,6 +971,8 @@ class GkWorkload:
         K = plan.n_rounds
         # what bounds the kernels by design is the exponentials of the decay-dependent sums (about 330 k per chunk-head
         # in both passes together, 16 per clock and SM): reported beside the HBM figure
+        import torch
+        one_launch = 1 < K <= 32 and plan.n_seq * Hh <= 8 * torch.cuda.get_device_properties(0).multi_processor_count
         chunk_heads = plan.n_chunks * Hh
         sfu_ms = chunk_heads * 330e3 / (148 * 16 * 1.965e9) * 1e3
         roof = hbm_roofline("gk_mma_bwd_kernel (all rounds)", bwd_bytes / K, kernel_ms["bwd"] / K, peaks, None,
@@ -986,7 +988,9 @@ class GkWorkload:
                                      "(mma.sync, bf16 operands, fp32 accumulation), in-block pair sums in fp32 on the CUDA cores",
                            "l2": "inputs larger than L2"},
                 "roofline": roof,
-                "gpu_launches_per_step": 2 * K + (K if plan.n_slots else 0) + (1 if plan.n_rg_rows else 0)}
+                # all rounds in one launch per pass on a problem with at most 8 items per SM (the library's rule), else one
+                # launch per round and pass with the hand-off reduction before every backward round; plus the fold
+                "gpu_launches_per_step": (2 if one_launch else 2 * K + (K if plan.n_slots else 0)) + (1 if plan.n_rg_rows else 0)}
 
     def extras(self, ms_step):
         return {}

@@ -228,10 +228,8 @@ int32_t harts_la_gk_workspace_bytes(const harts_la_tables_t* tb, int32_t H, int3
     if (!tb || H < 1 || dk < 1 || dv < 1) return HARTS_EINVAL;
     if (dtype != HARTS_FP32 && dtype != HARTS_BF16) return HARTS_EUNSUPPORTED;
     const size_t elem = dtype == HARTS_FP32 ? 4 : 2;
-    if (chunk_state_bytes) {
-        const size_t b = (size_t)tb->n_chunks * H * dk * dv * elem;
-        *chunk_state_bytes = b < 256 ? 256 : b;
-    }
+    if (chunk_state_bytes)      // the states, then the flags of the one-launch forms
+        *chunk_state_bytes = harts::chunk_state_payload(*tb, H, dk, dv, elem) + harts::fused_flag_bytes(*tb, H);
     if (scratch_bytes) *scratch_bytes = harts::gk_scratch_layout(*tb, H, dk, dv).total;
     return HARTS_OK;
 }
@@ -251,6 +249,18 @@ int32_t harts_la_gk_fwd(const harts_la_plan_t* plan, const void* dev_blob, int32
         return HARTS_EINVAL;
     if ((flags & HARTS_FLAG_CHECK_TABLES) && !dev_status) return HARTS_EINVAL;
     const int32_t r0 = round == 0 ? 1 : round, r1 = round == 0 ? p->n_rounds : round;
+    const bool one_launch = round == 0 && p->n_rounds > 1 && p->n_rounds <= harts::MAX_FUSED_ROUNDS && chunk_states &&
+                            !(flags & (HARTS_FLAG_ROUND_LAUNCHES | HARTS_FLAG_FMA_KERNELS)) &&
+                            harts::gk_mma_supported(dtype, dk, dv);
+    if (one_launch) {           // flags and tickets sit behind the chunk states, as for the scalar-gate calls
+        harts::FwdArgs a{tb, 0, tb.n_seq, q, k, v, gk, o, slots, chunk_states, H, dk, dv, dtype, flags, dev_status,
+                         static_cast<cudaStream_t>(stream)};
+        if (flags & HARTS_FLAG_CHECK_TABLES)
+            if ((rc = harts::check_tables(tb, 0, tb.n_seq, dev_status, a.stream)) != HARTS_OK) return rc;
+        int* fl = reinterpret_cast<int*>(static_cast<char*>(chunk_states) + harts::chunk_state_payload(tb, H, dk, dv, 2));
+        rc = harts::gk_mma_fwd_all(a, fl, fl + harts::fused_flag_count(tb, H));
+        if (rc != HARTS_EUNSUPPORTED) return rc;
+    }
     for (int32_t r = r0; r <= r1; r++) {
         harts::FwdArgs a{tb, p->round_seq_ptr[r - 1], p->round_seq_ptr[r], q, k, v, gk, o, slots, chunk_states, H, dk, dv,
                          dtype, flags, dev_status, static_cast<cudaStream_t>(stream)};
@@ -277,7 +287,23 @@ int32_t harts_la_gk_bwd(const harts_la_plan_t* plan, const void* dev_blob, int32
         return HARTS_EINVAL;
     if ((flags & HARTS_FLAG_CHECK_TABLES) && !dev_status) return HARTS_EINVAL;
     const int32_t r1 = round == 0 ? p->n_rounds : round, r0 = round == 0 ? 1 : round;
-    for (int32_t r = r1; r >= r0; r--) {
+    bool done = false;
+    if (round == 0 && p->n_rounds > 1 && p->n_rounds <= harts::MAX_FUSED_ROUNDS &&
+        !(flags & (HARTS_FLAG_ROUND_LAUNCHES | HARTS_FLAG_FMA_KERNELS)) && harts::gk_mma_supported(dtype, dk, dv)) {
+        harts::BwdArgs a{tb, 0, tb.n_seq, q, k, v, gk, dO, dq, dk_, dv_, dgk, chunk_states, scratch, H, dk, dv, dtype, flags,
+                         dev_status, static_cast<cudaStream_t>(stream)};
+        if (flags & HARTS_FLAG_CHECK_TABLES)
+            if ((rc = harts::check_tables(tb, 0, tb.n_seq, dev_status, a.stream)) != HARTS_OK) return rc;
+        int* fl = reinterpret_cast<int*>(const_cast<char*>(static_cast<const char*>(chunk_states)) +
+                                         harts::chunk_state_payload(tb, H, dk, dv, 2));
+        harts::RoundOrder ro;
+        ro.n = p->n_rounds;
+        for (int32_t r = 0; r <= p->n_rounds; r++) ro.ptr[r] = p->round_seq_ptr[r];
+        rc = harts::gk_mma_bwd_all(a, fl + (size_t)tb.n_slots * H, fl + harts::fused_flag_count(tb, H) + 1, ro);
+        if (rc == HARTS_OK) done = true;
+        else if (rc != HARTS_EUNSUPPORTED) return rc;
+    }
+    for (int32_t r = r1; r >= r0 && !done; r--) {
         harts::BwdArgs a{tb, p->round_seq_ptr[r - 1], p->round_seq_ptr[r], q, k, v, gk, dO, dq, dk_, dv_, dgk,
                          chunk_states, scratch, H, dk, dv, dtype, flags, dev_status, static_cast<cudaStream_t>(stream)};
         if (flags & HARTS_FLAG_CHECK_TABLES)

@@ -135,6 +135,8 @@ struct RoundOrder {
     int n;
     int ptr[MAX_FUSED_ROUNDS + 1];
 };
+int32_t gk_mma_fwd_all(const FwdArgs& a, int* flags, int* ticket);     // all rounds in one launch (la_gk_mma.cu)
+int32_t gk_mma_bwd_all(const BwdArgs& a, int* flags, int* ticket, const RoundOrder& rounds);
 int32_t tc_bwd(const BwdArgs& a);
 int32_t tc_bwd_fused(const BwdArgs& a, int* flags, int* ticket, const RoundOrder& rounds);   // all rounds in one launch
 int32_t handoff_reduce(const BwdArgs& a);

@@ -15,8 +15,12 @@
 // Shared-memory tiles of bf16 are row-major with the 16-byte pieces of a row XOR-ed by (row & 7), so that ldmatrix
 // (plain and transposed) is free of bank conflicts.
 #include "kernels.h"
+#include "tc_common.cuh"
 
 namespace harts {
+
+int sm_count();
+
 namespace {
 
 constexpr int BT = 64;      // chunk rows
@@ -351,13 +355,16 @@ __device__ __forceinline__ void state_to_operand(const float (&st)[8][4], unsign
     }
 }
 // state fragments <-> fp32 [128][128] in global memory (slots, initial-state gradients)
-template <bool ADD>
+// PAST_L1: the data was written during this launch by another CTA
+template <bool ADD, bool PAST_L1>
 __device__ __forceinline__ void state_from_global(float (&st)[8][4], const float* src, int warp, int lane) {
     const int g = lane >> 2, tq = lane & 3, r0 = (warp & 7) * 16 + g, c0 = (warp >> 3) * 64 + tq * 2;
 #pragma unroll
     for (int n = 0; n < 8; n++) {
-        const float2 lo = *reinterpret_cast<const float2*>(src + (size_t)r0 * D + c0 + n * 8);
-        const float2 hi = *reinterpret_cast<const float2*>(src + (size_t)(r0 + 8) * D + c0 + n * 8);
+        const float2* p_lo = reinterpret_cast<const float2*>(src + (size_t)r0 * D + c0 + n * 8);
+        const float2* p_hi = reinterpret_cast<const float2*>(src + (size_t)(r0 + 8) * D + c0 + n * 8);
+        const float2 lo = PAST_L1 ? __ldcg(p_lo) : *p_lo;
+        const float2 hi = PAST_L1 ? __ldcg(p_hi) : *p_hi;
         if (ADD) { st[n][0] += lo.x; st[n][1] += lo.y; st[n][2] += hi.x; st[n][3] += hi.y; }
         else { st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y; }
     }
@@ -399,12 +406,18 @@ __device__ __forceinline__ void tile_to_global(const unsigned char* tile, __nv_b
         reinterpret_cast<uint4*>(dst)[p] = *reinterpret_cast<const uint4*>(tile + sw256(p >> 4, p & 15));
 }
 
+// ONE_LAUNCH: the grid covers the sequences of ALL rounds (numbered round by round).  Every CTA draws its work item
+// from `ticket`, so an item is only ever held by a running CTA; a sequence that starts from an exported state waits for
+// the flag its producer (an earlier round, a smaller ticket, hence running or done) sets after writing the slot.
+// Otherwise: one launch per round, item = block index, no flags.
+template <bool ONE_LAUNCH>
 __global__ void __launch_bounds__(NT, 1)
 gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* __restrict__ q,
                   const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ gk,
                   __nv_bfloat16* __restrict__ o, float* __restrict__ slots, __nv_bfloat16* __restrict__ chunk_states,
-                  const int32_t* gate) {
+                  const int32_t* gate, int* status, int* slot_flags, int* ticket) {
     if (gate_closed(gate)) return;
+    __shared__ int s_item, s_dead;
     extern __shared__ __align__(1024) unsigned char sm[];
     unsigned char *sQ = sm + Shared::q, *sK = sm + Shared::k, *sV = sm + Shared::v, *sP = sm + Shared::p,
                   *sSb = sm + Shared::sb, *sQa = sm + Shared::qa, *sKa = sm + Shared::ka;
@@ -416,9 +429,18 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
 
     // blocks are handed to the SMs in index order: with the plan's order (longest sequence of the round first) the long
     // walks start first and the short ones fill the tail
-    const int seq_pos = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
-    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+    int item = blockIdx.x;
+    if constexpr (ONE_LAUNCH) {
+        if (tid == 0) {
+            s_item = atomicAdd(ticket, 1);
+            s_dead = 0;
+        }
+        __syncthreads();
+        item = s_item;
+    }
+    const int seq_pos = seq_lo + item / H, h = item % H;
+    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
     const int mb = warp & 3, nq = warp >> 2;          // this warp's 16-row block and 32-column quarter of [64][128] products
     const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)D * D;
@@ -428,7 +450,11 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
 #pragma unroll
         for (int n = 0; n < 8; n++) st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
     } else {
-        state_from_global<false>(st, slots + ((size_t)s.init_slot * H + h) * state_elems, warp, lane);
+        if constexpr (ONE_LAUNCH) {
+            if (tid == 0) tc::flag_wait(slot_flags + (size_t)s.init_slot * H + h, status, &s_dead);
+            if (__syncthreads_or(s_dead)) return;      // the wait ran out (status word set): give the walk up
+        }
+        state_from_global<false, ONE_LAUNCH>(st, slots + ((size_t)s.init_slot * H + h) * state_elems, warp, lane);
     }
 
     int next_req = s.req_lo;
@@ -442,11 +468,14 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         load_g(gk, H, h, srow, sB);
         // start-of-chunk state: operand copy, kept for the backward, exported when the plan requests this boundary
         state_to_operand(st, sSb, warp, lane);
-        if (next_req < s.req_hi && tb.slot_chunk[next_req] == c) {
+        const bool exported = next_req < s.req_hi && tb.slot_chunk[next_req] == c;
+        if (exported) {
             state_to_global(st, slots + ((size_t)next_req * H + h) * state_elems, warp, lane);
+            if (ONE_LAUNCH) __threadfence();               // this thread's part of the slot, before the flag below
             next_req++;
         }
         __syncthreads();
+        if (ONE_LAUNCH && exported && tid == 0) tc::flag_set(slot_flags + (size_t)(next_req - 1) * H + h);
         if (chunk_states) tile_to_global<D>(sSb, chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems);
         cumsum_rows(sB, sTmp);
         step_factors(sB, sR);
@@ -544,14 +573,20 @@ __device__ __forceinline__ float2 ld_bf2(const unsigned char* tile, int r, int c
 }
 
 
+// ONE_LAUNCH: the grid covers the sequences of all rounds; every CTA draws its item from `ticket` (last round first,
+// inside a round the plan's order).  A sequence publishes a flag once its initial-state gradient is in the scratch area;
+// a sequence that exported a boundary waits for the flags of all sequences that started there (later rounds, smaller
+// tickets, hence running or done) and sums their gradients itself in the order handoff_reduce uses.
+template <bool ONE_LAUNCH>
 __global__ void __launch_bounds__(NT, 1)
 gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* __restrict__ q,
                   const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, const float* __restrict__ gk,
                   const __nv_bfloat16* __restrict__ dO, __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk_,
                   __nv_bfloat16* __restrict__ dv_, float* __restrict__ dgk, const __nv_bfloat16* __restrict__ chunk_states,
                   float* __restrict__ ds0, float* __restrict__ rk, float* __restrict__ rv, float* __restrict__ rg,
-                  const int32_t* gate) {
+                  const int32_t* gate, int* status, int* ds0_flags, int* ticket, const RoundOrder rounds) {
     if (gate_closed(gate)) return;
+    __shared__ int s_item, s_dead;
     extern __shared__ __align__(1024) unsigned char sm[];
     unsigned char *sQ = sm + SharedB::q, *sK = sm + SharedB::k, *sV = sm + SharedB::v, *sDO = sm + SharedB::dO,
                   *sSc = sm + SharedB::sc, *sdSb = sm + SharedB::dsb, *sQa = sm + SharedB::qa, *sKa = sm + SharedB::ka,
@@ -570,9 +605,24 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
 
     // blocks are handed to the SMs in index order: with the plan's order (longest sequence of the round first) the long
     // walks start first and the short ones fill the tail
-    const int seq_pos = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
-    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+    int seq_pos = seq_lo + blockIdx.x / H, h = blockIdx.x % H;
+    if constexpr (ONE_LAUNCH) {
+        if (tid == 0) {
+            s_item = atomicAdd(ticket, 1);
+            s_dead = 0;
+        }
+        __syncthreads();
+        int j = s_item / H;
+        h = s_item % H;
+        seq_pos = -1;
+        for (int r = rounds.n - 1; r >= 0 && seq_pos < 0; r--) {      // last round first
+            const int cnt = rounds.ptr[r + 1] - rounds.ptr[r];
+            if (j < cnt) seq_pos = rounds.ptr[r] + j;
+            else j -= cnt;
+        }
+    }
+    const int seq = tb.seq_order ? tb.seq_order[seq_pos] : seq_pos;
     const int mb = warp & 3, nq = warp >> 2;          // this warp's 16-row block and 32-column quarter of [64][128] products
     const SeqInfo s = seq_info(tb, seq);
     const size_t state_elems = (size_t)D * D;
@@ -584,12 +634,28 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
     int next_req = s.req_hi - 1;                      // slots of this sequence are ordered by chunk index
     for (int c = s.n_chunks - 1; c >= 0; c--) {
         __syncthreads();                              // the previous chunk's readers of every tile are through
-        // gradient arriving at boundary c+1 from the sequences that started there (summed into the first consumer's
-        // buffer by handoff_reduce)
+        // gradient arriving at boundary c+1 from the sequences that started there: one launch per round -- summed into
+        // the first consumer's buffer by handoff_reduce; all rounds in one launch -- awaited and summed here, same order
         if (next_req >= s.req_lo && tb.slot_chunk[next_req] == c + 1) {
-            if (tb.slot_cons_ptr[next_req] < tb.slot_cons_ptr[next_req + 1]) {
-                state_from_global<true>(ds, ds0 + ((size_t)tb.slot_cons_seq[tb.slot_cons_ptr[next_req]] * H + h) * state_elems,
-                                        warp, lane);
+            const int cons_lo = tb.slot_cons_ptr[next_req], cons_hi = tb.slot_cons_ptr[next_req + 1];
+            if constexpr (ONE_LAUNCH) {
+                for (int u = cons_lo + tid; u < cons_hi; u += NT)
+                    tc::flag_wait(ds0_flags + (size_t)tb.slot_cons_seq[u] * H + h, status, &s_dead);
+                if (__syncthreads_or(s_dead)) return;      // a wait ran out (status word set): give the walk up
+            }
+            if (cons_lo < cons_hi) {
+                if constexpr (ONE_LAUNCH) {
+                    float a[8][4];
+                    state_from_global<false, true>(a, ds0 + ((size_t)tb.slot_cons_seq[cons_lo] * H + h) * state_elems, warp, lane);
+                    for (int u = cons_lo + 1; u < cons_hi; u++)
+                        state_from_global<true, true>(a, ds0 + ((size_t)tb.slot_cons_seq[u] * H + h) * state_elems, warp, lane);
+#pragma unroll
+                    for (int n = 0; n < 8; n++) {
+                        ds[n][0] += a[n][0]; ds[n][1] += a[n][1]; ds[n][2] += a[n][2]; ds[n][3] += a[n][3];
+                    }
+                } else {
+                    state_from_global<true, false>(ds, ds0 + ((size_t)tb.slot_cons_seq[cons_lo] * H + h) * state_elems, warp, lane);
+                }
             }
             next_req--;
         }
@@ -868,7 +934,14 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         // ---- dS <- Diag(e^{b_n}) dS + q~^T dO ---------------------------------------------------------------------------
         state_update(ds, sB, aQ, aDO, warp, lane);
     }
-    if (s.init_slot >= 0) state_to_global(ds, ds0 + ((size_t)seq * H + h) * state_elems, warp, lane);
+    if (s.init_slot >= 0) {
+        state_to_global(ds, ds0 + ((size_t)seq * H + h) * state_elems, warp, lane);
+        if constexpr (ONE_LAUNCH) {
+            __threadfence();                           // this thread's part, before the flag that follows the barrier
+            __syncthreads();
+            if (tid == 0) tc::flag_set(ds0_flags + (size_t)seq * H + h);
+        }
+    }
 }
 
 }  // namespace
@@ -877,29 +950,71 @@ int32_t gk_mma_supported(int32_t dtype, int32_t dk, int32_t dv) { return dtype =
 
 int32_t gk_mma_fwd(const FwdArgs& a) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
-    if (cudaFuncSetAttribute(gk_mma_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Shared::fwd_bytes) !=
+    if (cudaFuncSetAttribute(gk_mma_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Shared::fwd_bytes) !=
         cudaSuccess)
         return HARTS_ECUDA;
     const int n = (a.seq_hi - a.seq_lo) * a.H;
-    gk_mma_fwd_kernel<<<n, NT, Shared::fwd_bytes, a.stream>>>(
+    gk_mma_fwd_kernel<false><<<n, NT, Shared::fwd_bytes, a.stream>>>(
         a.tb, a.seq_lo, a.H, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v, a.g,
-        (__nv_bfloat16*)a.o, a.slots, (__nv_bfloat16*)a.chunk_states, status_gate(a.flags, a.dev_status));
+        (__nv_bfloat16*)a.o, a.slots, (__nv_bfloat16*)a.chunk_states, status_gate(a.flags, a.dev_status), a.dev_status,
+        nullptr, nullptr);
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
-
 int32_t gk_mma_bwd(const BwdArgs& a) {
     if (a.seq_hi == a.seq_lo) return HARTS_OK;
-    if (cudaFuncSetAttribute(gk_mma_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SharedB::bytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(gk_mma_bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SharedB::bytes) !=
+        cudaSuccess)
         return HARTS_ECUDA;
     const int n = (a.seq_hi - a.seq_lo) * a.H;
     const GkScratchLayout sl = gk_scratch_layout(a.tb, a.H, a.dk, a.dv);
     char* base = static_cast<char*>(a.scratch);
-    gk_mma_bwd_kernel<<<n, NT, SharedB::bytes, a.stream>>>(
+    gk_mma_bwd_kernel<false><<<n, NT, SharedB::bytes, a.stream>>>(
         a.tb, a.seq_lo, a.H, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v, a.g,
         (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_, (__nv_bfloat16*)a.dv_, a.dg,
         (const __nv_bfloat16*)a.chunk_states, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
-        (float*)(base + sl.rg), status_gate(a.flags, a.dev_status));
+        (float*)(base + sl.rg), status_gate(a.flags, a.dev_status), a.dev_status, nullptr, nullptr, RoundOrder{});
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+// All rounds in one launch per pass (sequences [seq_lo, seq_hi) = the whole plan).  flags: n_slots * H (forward) or
+// n_seq * H (backward) int32 on the device, ticket: one int32; both zeroed here on the stream.  Offered while the
+// problem has few items per SM, like the scalar-gate forms; HARTS_EUNSUPPORTED otherwise.
+int32_t gk_mma_fwd_all(const FwdArgs& a, int* flags, int* ticket) {
+    const int64_t n = (int64_t)(a.seq_hi - a.seq_lo) * a.H;
+    if (n == 0) return HARTS_OK;
+    if (n > (int64_t)ONE_LAUNCH_ITEMS_PER_CTA * sm_count()) return HARTS_EUNSUPPORTED;
+    if (cudaFuncSetAttribute(gk_mma_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Shared::fwd_bytes) !=
+        cudaSuccess)
+        return HARTS_ECUDA;
+    if (a.tb.n_slots > 0 &&
+        cudaMemsetAsync(flags, 0, (size_t)a.tb.n_slots * a.H * sizeof(int), a.stream) != cudaSuccess)
+        return HARTS_ECUDA;
+    if (cudaMemsetAsync(ticket, 0, sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
+    gk_mma_fwd_kernel<true><<<(int)n, NT, Shared::fwd_bytes, a.stream>>>(
+        a.tb, a.seq_lo, a.H, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v, a.g,
+        (__nv_bfloat16*)a.o, a.slots, (__nv_bfloat16*)a.chunk_states, status_gate(a.flags, a.dev_status), a.dev_status,
+        flags, ticket);
+    return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
+}
+
+int32_t gk_mma_bwd_all(const BwdArgs& a, int* flags, int* ticket, const RoundOrder& rounds) {
+    const int64_t n = (int64_t)(a.seq_hi - a.seq_lo) * a.H;
+    if (n == 0) return HARTS_OK;
+    if (rounds.n < 1 || rounds.ptr[0] != a.seq_lo || rounds.ptr[rounds.n] != a.seq_hi) return HARTS_EINVAL;
+    if (n > (int64_t)ONE_LAUNCH_ITEMS_PER_CTA * sm_count()) return HARTS_EUNSUPPORTED;
+    if (cudaFuncSetAttribute(gk_mma_bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SharedB::bytes) !=
+        cudaSuccess)
+        return HARTS_ECUDA;
+    if (cudaMemsetAsync(flags, 0, (size_t)a.tb.n_seq * a.H * sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
+    if (cudaMemsetAsync(ticket, 0, sizeof(int), a.stream) != cudaSuccess) return HARTS_ECUDA;
+    const GkScratchLayout sl = gk_scratch_layout(a.tb, a.H, a.dk, a.dv);
+    char* base = static_cast<char*>(a.scratch);
+    gk_mma_bwd_kernel<true><<<(int)n, NT, SharedB::bytes, a.stream>>>(
+        a.tb, a.seq_lo, a.H, (const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v, a.g,
+        (const __nv_bfloat16*)a.dO, (__nv_bfloat16*)a.dq, (__nv_bfloat16*)a.dk_, (__nv_bfloat16*)a.dv_, a.dg,
+        (const __nv_bfloat16*)a.chunk_states, (float*)(base + sl.ds0), (float*)(base + sl.rk), (float*)(base + sl.rv),
+        (float*)(base + sl.rg), status_gate(a.flags, a.dev_status), a.dev_status, flags, ticket, rounds);
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 

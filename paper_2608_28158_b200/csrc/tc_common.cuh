@@ -97,7 +97,8 @@ __device__ __forceinline__ void mbar_expect_tx_only(uint64_t* bar, uint32_t byte
 // A CTA that has produced something another CTA of the same launch consumes publishes a flag in global memory; the
 // consumer polls it.  Every writer of the data fences before the CTA-wide barrier that precedes flag_set; the consumer
 // reads the data only after flag_wait returned true and a CTA-wide barrier.  The wait is bounded like the others (a
-// longer limit: the producer may be a long sequence) and honours the CTA's latch.
+// longer limit: the producer may be a long sequence), honours the CTA's latch, and ends as soon as the launch's status
+// word shows that some CTA has given up, so that one time-out does not become a chain of them.
 constexpr unsigned long long FLAG_WAIT_LIMIT_NS = 4000ull * 1000 * 1000;
 __device__ __forceinline__ void flag_set(int* flag) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(1) : "memory");
@@ -112,6 +113,11 @@ __device__ __forceinline__ bool flag_wait(const int* flag, int* status, volatile
             if (v != 0) return true;
         }
         if (*dead) return false;
+        // another CTA of the launch has already given up (its wait ran out): what this one waits for may never come
+        if (status && *reinterpret_cast<volatile int*>(status) != 0) {
+            *dead = 1;
+            return false;
+        }
         if (global_ns() - t0 > FLAG_WAIT_LIMIT_NS) break;
     }
     *dead = 1;

@@ -111,6 +111,26 @@ def test_tensor_core_path_agrees_with_the_cuda_core_path():
             assert rel_err(tc[name], cc[name]) <= 0.6 * TOL["bf16"][name], (n, name, rel_err(tc[name], cc[name]))
 
 
+def test_all_rounds_in_one_launch_give_the_bits_of_one_launch_per_round():
+    """bf16, d = 128, several rounds: round 0 runs all rounds in one launch per pass (tickets and flags between the
+    CTAs); with HARTS_FLAG_ROUND_LAUNCHES every round is a launch of its own.  Same arithmetic, same bits -- on forests
+    with shared slots, replayed rows and three rounds, two heads."""
+    import random
+    from test_plan_oracle import random_tree
+    rnd = random.Random(23)
+    forests = [config_forest("cfg0b"), config_forest("cfg1")]
+    forests += [make_forest([random_tree(rnd, rnd.randint(3, 14), rnd.choice([40, 200, 700])) for _ in range(rnd.randint(1, 3))])
+                for _ in range(8)]
+    multi = 0
+    for n, fo in enumerate(forests):
+        plan, one = run_gk(fo, 2, 128, "bf16", 70 + n, raw=True)
+        _, per = run_gk(fo, 2, 128, "bf16", 70 + n, raw=True, flags=H.HARTS_FLAG_ROUND_LAUNCHES)
+        for name in one:
+            assert np.array_equal(one[name], per[name]), (n, name)
+        multi += int(plan.n_rounds > 1)
+    assert multi >= 6
+
+
 def test_equal_channels_agree_with_the_scalar_gate_kernels():
     """With every channel's gate equal, the per-channel kernels and the scalar-gate fp32 kernels compute the same
     function (different code): outputs within fp32 accumulation error of each other."""
