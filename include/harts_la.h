@@ -247,7 +247,8 @@ int32_t harts_la_step_host(const harts_la_plan_t* plan, const void* dev_blob, co
  *   gk  [n_rows, H, dk] fp32 DEVICE: the per-channel log-decay (never modified), and
  *   dgk [n_rows, H, dk] fp32 DEVICE: its gradient (own rows overwritten; replayed rows folded in by the round-1 call)
  * replace g and dg, and the backward scratch is larger (harts_la_gk_workspace_bytes: the replay-row gradient of g is
- * a vector).  Rounds as for harts_la_fwd / harts_la_bwd (0 = all).  Served: fp32 with dk = dv = 64, bf16 with
+ * a vector; its chunk-state figure includes the flags of the one-launch forms).  Rounds as for harts_la_fwd /
+ * harts_la_bwd (0 = all; on the tensor-core path in one launch per pass under the same conditions).  Served: fp32 with dk = dv = 64, bf16 with
  * dk = dv = 64 or 128, chunk 64.  bf16 with dk = dv = 128 runs its dense products on the tensor cores (bf16
  * operands, fp32 accumulation; decayed operands, scores and chunk states rounded to bf16); everything else, and that
  * shape too under HARTS_FLAG_FMA_KERNELS, runs in fp32 on the CUDA cores.  Every decay factor is exp of a
@@ -320,8 +321,12 @@ int32_t harts_la_check(const int32_t* dev_status, void* stream);
  * returns).  This call launches one small CTA that waits, with a limit of one millisecond, on a barrier nothing arrives
  * at.  Afterwards harts_la_check(dev_status) gives HARTS_ETIMEOUT and the context stays usable.
  *   dev_status  DEVICE int32 status word (zeroed by the caller)
- *   dev_report  DEVICE int32[5] or NULL: {first wait succeeded (0 expected), second wait succeeded (0), microseconds
- *               in the first wait (about 1000), microseconds in the second (about 0: the latch was set), CTA saw the latch (1)}
+ *   dev_report  DEVICE int32[8] or NULL: {first wait succeeded (0 expected), second wait succeeded (0), microseconds
+ *               in the first wait (about 1000), microseconds in the second (about 0: the latch was set), CTA saw the
+ *               latch (1), then for the flag wait of the one-launch forms (a flag nobody sets; first with a limit of
+ *               one millisecond, then with the status word already set): bits {1: first succeeded, 2: second
+ *               succeeded, 4: first latched, 8: second latched} (12 expected), microseconds in the first (about 1000),
+ *               microseconds in the second (about 0: a set status word ends a flag wait)}
  */
 int32_t harts_la_selftest_timeout(int32_t* dev_status, int32_t* dev_report, void* stream);
 

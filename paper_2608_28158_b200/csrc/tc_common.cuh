@@ -103,7 +103,8 @@ constexpr unsigned long long FLAG_WAIT_LIMIT_NS = 4000ull * 1000 * 1000;
 __device__ __forceinline__ void flag_set(int* flag) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(1) : "memory");
 }
-__device__ __forceinline__ bool flag_wait(const int* flag, int* status, volatile int* dead) {
+__device__ __forceinline__ bool flag_wait(const int* flag, int* status, volatile int* dead,
+                                          unsigned long long limit_ns = FLAG_WAIT_LIMIT_NS) {
     const unsigned long long t0 = global_ns();
     for (int round = 0; round < (1 << 26); round++) {
         int v;
@@ -118,7 +119,7 @@ __device__ __forceinline__ bool flag_wait(const int* flag, int* status, volatile
             *dead = 1;
             return false;
         }
-        if (global_ns() - t0 > FLAG_WAIT_LIMIT_NS) break;
+        if (global_ns() - t0 > limit_ns) break;
     }
     *dead = 1;
     if (status) atomicExch(status, STATUS_TIMEOUT);
