@@ -938,6 +938,7 @@ class GkWorkload:
                     "dv": torch.empty_like(inp["v"]), "dg": torch.empty_like(inp["g"])}
         self.units = plan.C
         self.stream = torch.cuda.current_stream()
+        self.flags = H.HARTS_FLAG_ROUND_LAUNCHES if getattr(args, "round_launches", False) else 0
 
     def step(self, marks):
         import torch
@@ -945,10 +946,10 @@ class GkWorkload:
         a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         a.record(self.stream)
         H.harts_la_gk_fwd(plan, 0, inp["q"], inp["k"], inp["v"], inp["g"], out["o"], self.slots, self.cs,
-                          dev_status=self.status)
+                          flags=self.flags, dev_status=self.status)
         b.record(self.stream)
         H.harts_la_gk_bwd(plan, 0, inp["q"], inp["k"], inp["v"], inp["g"], inp["dO"], out["dq"], out["dk"], out["dv"],
-                          out["dg"], self.cs, self.scratch, dev_status=self.status)
+                          out["dg"], self.cs, self.scratch, flags=self.flags, dev_status=self.status)
         c.record(self.stream)
         if marks is not None:
             marks += [("fwd", a, b), ("bwd", b, c)]
@@ -972,7 +973,8 @@ class GkWorkload:
         # what bounds the kernels by design is the exponentials of the decay-dependent sums (about 330 k per chunk-head
         # in both passes together, 16 per clock and SM): reported beside the HBM figure
         import torch
-        one_launch = 1 < K <= 32 and plan.n_seq * Hh <= 8 * torch.cuda.get_device_properties(0).multi_processor_count
+        one_launch = (not self.flags and 1 < K <= 32 and
+                      plan.n_seq * Hh <= 8 * torch.cuda.get_device_properties(0).multi_processor_count)
         chunk_heads = plan.n_chunks * Hh
         sfu_ms = chunk_heads * 330e3 / (148 * 16 * 1.965e9) * 1e3
         roof = hbm_roofline("gk_mma_bwd_kernel (all rounds)", bwd_bytes / K, kernel_ms["bwd"] / K, peaks, None,
