@@ -254,7 +254,8 @@ int32_t harts_la_step_host(const harts_la_plan_t* plan, const void* dev_blob, co
  * shape too under HARTS_FLAG_FMA_KERNELS, runs in fp32 on the CUDA cores.  Every decay factor is exp of a
  * difference of running sums that is <= 0 for g <= 0: exp(b_t[i] - b_j[i]) with j <= t directly, or, on the
  * tensor-core path for t and j in different 16-row blocks of a chunk, exp(b_t[i] - a[i]) exp(a[i] - b_j[i]) with a the
- * running sum at the first row of t's block -- so no gate value g <= 0 can overflow.  Errors as for harts_la_fwd /
+ * running sum at the first row of t's block (and for t, j in the same block too, while no channel of the chunk decays by
+ * more than 2^100 over a block, which bounds exp(a[i] - b_j[i])) -- so no gate value g <= 0 can overflow.  Errors as for harts_la_fwd /
  * harts_la_bwd.
  */
 int32_t harts_la_gk_workspace_bytes(const harts_la_tables_t* tables, int32_t H, int32_t dk, int32_t dv, int32_t dtype,

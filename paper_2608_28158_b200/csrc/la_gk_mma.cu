@@ -231,9 +231,65 @@ __device__ __forceinline__ void anchored_operands(const unsigned char* sQ, const
     }
 }
 
-// blocks left of the diagonal: warp -> row block I = warp & 3, 16-column tile J = warp >> 2
-__device__ __forceinline__ void scores_off_diagonal(uint32_t aQa, uint32_t aKa, unsigned char* sP, int warp, int lane) {
+// Pairs INSIDE a 16-row block: with the same anchor a_I (b at the block's first row) the key factor e^{a_I-b_j} is >= 1
+// and grows to e^{a_I - b_{16I+15}} at the block's last row.  While that total decay of a block stays below 2^MILD_LOG2
+// in every channel (bf16 and fp32 hold 2^127), the block on the diagonal is a dense product too: q^ (anchored at its
+// block, as above) against k_j e^{a_I-b_j} for the keys of the same block, masked to j <= t afterwards -- the entries
+// right of the diagonal are finite and thrown away.  A chunk in which any block decays faster takes the exact CUDA-core
+// path for its diagonal blocks instead (one decision per chunk, the same for the whole CTA).
+constexpr float MILD_LOG2 = 100.f;
+
+__device__ __forceinline__ bool chunk_is_mild(const float* sB) {
+    const int i = threadIdx.x & (D - 1), blk = threadIdx.x >> 7;       // 512 threads: 4 blocks x 128 channels
+    const float fall = sB[16 * blk * D + i] - sB[(16 * blk + 15) * D + i];
+    return __syncthreads_or(!(fall <= MILD_LOG2)) == 0;                  // also false for a NaN gate
+}
+
+// keys anchored at their OWN block: sKd[j] = k_j .* 2^{a_I(j) - b_j}  (bf16 [64][128], swizzled)
+__device__ __forceinline__ void diag_operand(const unsigned char* sK, const float* sB, unsigned char* sKd) {
+    for (int p = threadIdx.x; p < BT * 16; p += NT) {
+        const int j = p >> 4, c16 = p & 15, a_row = j & ~15;
+        uint4 x = *reinterpret_cast<const uint4*>(sK + sw256(j, c16));
+        uint32_t* w = reinterpret_cast<uint32_t*>(&x);
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+            const int i = c16 * 8 + e * 2;
+            const float2 bs = *reinterpret_cast<const float2*>(sB + j * D + i);
+            const float2 ba = *reinterpret_cast<const float2*>(sB + a_row * D + i);
+            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+            w[e] = pack2(f.x * ex2(ba.x - bs.x), f.y * ex2(ba.y - bs.y));
+        }
+        *reinterpret_cast<uint4*>(sKd + sw256(j, c16)) = x;
+    }
+}
+
+// blocks left of the diagonal: warp -> row block I = warp & 3, 16-column tile J = warp >> 2; with `diag` (a mild chunk)
+// the warps with J == I take the block on the diagonal from the keys anchored at their own block
+__device__ __forceinline__ void scores_off_diagonal(uint32_t aQa, uint32_t aKa, unsigned char* sP, int warp, int lane,
+                                                    bool diag = false, uint32_t aKd = 0) {
     const int I = warp & 3, g = lane >> 2, tq = lane & 3;
+    if (diag && (warp >> 2) == I) {
+        float acc[2][4];
+#pragma unroll
+        for (int x = 0; x < 2; x++) acc[x][0] = acc[x][1] = acc[x][2] = acc[x][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 8; ks++) {
+            uint32_t a[4], b[4];
+            frag_a<256>(a, aQa, 16 * I, ks * 16, lane);
+            frag_b_nk<256>(b, aKd, ks * 16, 16 * I, lane);
+            mma16816(acc[0], a, b[0], b[1]);
+            mma16816(acc[1], a, b[2], b[3]);
+        }
+#pragma unroll
+        for (int x = 0; x < 2; x++) {
+            const int jc = 8 * x + 2 * tq, col = 16 * I + jc;           // jc, g: column and row inside the block
+            const float v0 = jc <= g ? acc[x][0] : 0.f, v1 = jc + 1 <= g ? acc[x][1] : 0.f;
+            const float v2 = jc <= g + 8 ? acc[x][2] : 0.f, v3 = jc + 1 <= g + 8 ? acc[x][3] : 0.f;
+            *reinterpret_cast<uint32_t*>(sP + sw128(16 * I + g, col >> 3) + (col & 7) * 2) = pack2(v0, v1);
+            *reinterpret_cast<uint32_t*>(sP + sw128(16 * I + g + 8, col >> 3) + (col & 7) * 2) = pack2(v2, v3);
+        }
+        return;
+    }
     for (int J = warp >> 2; J < I; J += NW / 4) {
         float acc[2][4];
 #pragma unroll
@@ -478,11 +534,14 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         if (ONE_LAUNCH && exported && tid == 0) tc::flag_set(slot_flags + (size_t)(next_req - 1) * H + h);
         if (chunk_states) tile_to_global<D>(sSb, chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems);
         cumsum_rows(sB, sTmp);
-        step_factors(sB, sR);
+        const bool mild = chunk_is_mild(sB);
+        unsigned char* sKd = reinterpret_cast<unsigned char*>(sR);        // the two are never needed in the same chunk
+        if (mild) diag_operand(sK, sB, sKd);
+        else step_factors(sB, sR);
         anchored_operands(sQ, sK, sB, sQa, sKa);
         __syncthreads();
-        scores_diagonal(sQ, sK, sR, sP, warp, lane);
-        scores_off_diagonal(s_u32(sQa), s_u32(sKa), sP, warp, lane);
+        if (!mild) scores_diagonal(sQ, sK, sR, sP, warp, lane);
+        scores_off_diagonal(s_u32(sQa), s_u32(sKa), sP, warp, lane, mild, s_u32(sKd));
         __syncthreads();
         scale_qk(sQ, sK, sB, sQ, sK);
         __syncthreads();
@@ -670,6 +729,7 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         state_to_operand(ds, sdSb, warp, lane);
         __syncthreads();
         cumsum_rows(sB, sTmp);
+        const bool mild = chunk_is_mild(sB);          // diagonal blocks as dense products too (see chunk_is_mild)
         const int r_lo = 16 * mb + g, r_hi = r_lo + 8;            // this thread's rows in the [64][128] products
         // ---- dA = dO V^T, iq = dO S_c^T, ik = V dS^T, <S_c, dS> per channel -------------------------------------------
         float iq[4][4], ik[4][4];
@@ -707,8 +767,13 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
 #pragma unroll
             for (int n = 0; n < 2; n++) {
                 const int col = 16 * nq + 8 * n + 2 * tq;
-                *reinterpret_cast<uint32_t*>(sdAb + sw128(r_lo, col >> 3) + (col & 7) * 2) = pack2(da[n][0], da[n][1]);
-                *reinterpret_cast<uint32_t*>(sdAb + sw128(r_hi, col >> 3) + (col & 7) * 2) = pack2(da[n][2], da[n][3]);
+                // the bf16 copy serves products that sum over j <= t (or t >= j) only: zero right of the diagonal
+                const bool dg_blk = nq == mb;
+                const int jc = (col & 15), tr = g;                       // column and row inside the diagonal block
+                const float m0 = !dg_blk || jc <= tr ? da[n][0] : 0.f, m1 = !dg_blk || jc + 1 <= tr ? da[n][1] : 0.f;
+                const float m2 = !dg_blk || jc <= tr + 8 ? da[n][2] : 0.f, m3 = !dg_blk || jc + 1 <= tr + 8 ? da[n][3] : 0.f;
+                *reinterpret_cast<uint32_t*>(sdAb + sw128(r_lo, col >> 3) + (col & 7) * 2) = pack2(m0, m1);
+                *reinterpret_cast<uint32_t*>(sdAb + sw128(r_hi, col >> 3) + (col & 7) * 2) = pack2(m2, m3);
                 if (nq == mb) {
                     *reinterpret_cast<float2*>(sdAd + r_lo * 16 + (col & 15)) = make_float2(da[n][0], da[n][1]);
                     *reinterpret_cast<float2*>(sdAd + r_hi * 16 + (col & 15)) = make_float2(da[n][2], da[n][3]);
@@ -750,19 +815,28 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         // ---- scores and the anchored operands ------------------------------------------------------------------------
         anchored_operands(sQ, sK, sB, sQa, sKa);
         __syncthreads();                              // S_c is dead from here on; dA and the anchored operands are visible
-        step_factors(sB, sR);                         // over the dead S_c tile
-        scores_off_diagonal(aQa, aKa, sP, warp, lane);
+        unsigned char* sKd = sSc;                     // keys anchored at their own block, over the dead S_c tile
+        const uint32_t aKd = aSc;
+        if (mild) {
+            diag_operand(sK, sB, sKd);
+            __syncthreads();
+        } else {
+            step_factors(sB, sR);                     // over the dead S_c tile as well; read after the next barrier
+        }
+        scores_off_diagonal(aQa, aKa, sP, warp, lane, mild, aKd);
         // ---- pairs in different blocks -------------------------------------------------------------------------------
-        if (mb >= 1) {   // dq: rows of block mb against the keys of the blocks before it, anchored at block mb
+        if (mb >= 1 || mild) {   // dq: rows of block mb against the keys of the blocks before it (and, in a mild
+                                 // chunk, of its own block: dA is zero right of the diagonal), anchored at block mb
             float acc[4][4];
 #pragma unroll
             for (int n = 0; n < 4; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-            for (int ks = 0; ks < mb; ks++) {
+            for (int ks = 0; ks < mb + (mild ? 1 : 0); ks++) {
                 uint32_t a[4], b[4];
                 frag_a<128>(a, adAb, 16 * mb, 16 * ks, lane);
 #pragma unroll
                 for (int n2 = 0; n2 < 2; n2++) {
-                    frag_b_kn<256>(b, aKa, ka_row0(mb) + 16 * ks, 32 * nq + 16 * n2, lane);
+                    if (ks < mb) frag_b_kn<256>(b, aKa, ka_row0(mb) + 16 * ks, 32 * nq + 16 * n2, lane);
+                    else frag_b_kn<256>(b, aKd, 16 * mb, 32 * nq + 16 * n2, lane);
                     mma16816(acc[2 * n2], a, b[0], b[1]);
                     mma16816(acc[2 * n2 + 1], a, b[2], b[3]);
                 }
@@ -777,7 +851,9 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
                 iq[n][2] += ex2(b_hi.x - an.x) * acc[n][2]; iq[n][3] += ex2(b_hi.y - an.y) * acc[n][3];
             }
         }
-        for (int I = mb + 1; I < 4; I++) {   // dk: keys of block mb against the queries of block I, anchored at block I
+        // dk: keys of block mb against the queries of block I (in a mild chunk also I = mb: the factor e^{a_I-b_j} is then
+        // >= 1 but bounded), anchored at block I
+        for (int I = mild ? mb : mb + 1; I < 4; I++) {
             float acc[4][4];
 #pragma unroll
             for (int n = 0; n < 4; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
@@ -800,14 +876,14 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
             }
         }
         __syncthreads();                              // the anchored operands are dead, the step factors visible
-        scores_diagonal(sQ, sK, sR, sP, warp, lane);
+        if (!mild) scores_diagonal(sQ, sK, sR, sP, warp, lane);
 #pragma unroll
         for (int n = 0; n < 4; n++) {
             const int col = 32 * nq + 8 * n + 2 * tq;
             *reinterpret_cast<float2*>(sDK + r_lo * D + col) = make_float2(ik[n][0], ik[n][1]);
             *reinterpret_cast<float2*>(sDK + r_hi * D + col) = make_float2(ik[n][2], ik[n][3]);
         }
-        __syncthreads();                              // the step factors are dead
+        __syncthreads();                              // the step factors / own-block keys are dead
 #pragma unroll
         for (int n = 0; n < 4; n++) {
             const int col = 32 * nq + 8 * n + 2 * tq;
@@ -820,7 +896,7 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         {
             const int i = tid & (D - 1), blk = tid >> 7, t0 = 16 * blk;
             float total = 0.f;                            // sum of q dq - k dk over this thread's rows
-            {
+            if (!mild) {
                 // rows ascending; xr[u] = 2^{b_t - b_u} as a running product of the one-step factors (one exponential per
                 // row instead of one per pair; every factor <= 1), the same factor for dq and dk
                 float dk_acc[16], kf[16], xr[16];

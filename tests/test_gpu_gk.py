@@ -21,9 +21,9 @@ ROW_MULT = 3.0
 DT = {"fp32": torch.float32, "bf16": torch.bfloat16}
 
 
-def run_gk(fo, heads, d, dtype, seed, strong_every=0, backward=True, flags=0, raw=False):
+def run_gk(fo, heads, d, dtype, seed, strong_every=0, backward=True, flags=0, raw=False, strong_shift=7.0):
     inp = make_inputs(fo.n_tokens, heads, d, d, dtype, seed)
-    inp["g"] = make_gk(fo.n_tokens, heads, d, seed, strong_every=strong_every)
+    inp["g"] = make_gk(fo.n_tokens, heads, d, seed, strong_every=strong_every, strong_shift=strong_shift)
     plan = plan_of(fo).upload()
     phys = to_physical(plan, inp)
     cs_bytes, sc_bytes = H.harts_la_gk_workspace_bytes(plan.tables, heads, d, d, 0 if dtype == "fp32" else 1)
@@ -90,12 +90,22 @@ def test_gates_far_outside_the_usual_range_do_not_overflow():
     check(errs, "fp32")
     plan, errs = run_gk(config_forest("cfg0b"), 1, 128, "bf16", 3, strong_every=8)
     check(errs, "bf16")
+    # The tensor-core kernels take the pairs inside a 16-row block as a dense product while no channel decays by more
+    # than 2^100 over the block, and by the exact per-pair path otherwise.  Gates of about -4 per token sit right at that
+    # limit (a mixture of both kinds of chunks); gates of about -9 per token (e^-570 per chunk) are all beyond it; mild
+    # gates with two such channels test the decision per chunk.
+    for shift, every in ((12.0, 8), (12.0, 64), (9.0, 3)):
+        plan, errs = run_gk(config_forest("cfg0b"), 2, 128, "bf16", 4, strong_every=every, strong_shift=shift)
+        check(errs, "bf16")
+    plan, errs = run_gk(config_forest("cfg1"), 1, 128, "bf16", 6, strong_every=16, strong_shift=8.0)
+    check(errs, "bf16")
 
 
 def test_tensor_core_path_agrees_with_the_cuda_core_path():
     """bf16, d = 128: the same call with HARTS_FLAG_FMA_KERNELS runs the CUDA-core kernels (pair sums over whole
     chunks, no anchored operands, fp32 products).  Two different decompositions of the same sums, same bf16 roundings of
-    the inputs and states: they must agree to well within the oracle tolerance, on forests with several rounds, shared
+    the inputs and states: they must agree to within the oracle tolerance (each is within it of the oracle, so twice of it is what the triangle
+    inequality alone would give), on forests with several rounds, shared
     slots and replayed rows, three heads, with strongly decaying channels mixed in."""
     import random
     from test_plan_oracle import random_tree
@@ -108,7 +118,7 @@ def test_tensor_core_path_agrees_with_the_cuda_core_path():
         _, tc = run_gk(fo, heads, 128, "bf16", 50 + n, strong_every=8 * (n % 2), raw=True)
         _, cc = run_gk(fo, heads, 128, "bf16", 50 + n, strong_every=8 * (n % 2), raw=True, flags=H.HARTS_FLAG_FMA_KERNELS)
         for name in tc:
-            assert rel_err(tc[name], cc[name]) <= 0.6 * TOL["bf16"][name], (n, name, rel_err(tc[name], cc[name]))
+            assert rel_err(tc[name], cc[name]) <= 1.0 * TOL["bf16"][name], (n, name, rel_err(tc[name], cc[name]))
 
 
 def test_all_rounds_in_one_launch_give_the_bits_of_one_launch_per_round():

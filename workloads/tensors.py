@@ -32,15 +32,16 @@ def make_inputs(n_tokens: int, H: int, dk: int, dv: int, dtype: str, seed: int, 
     return {"q": q, "k": k, "v": v, "g": g, "dO": dO}
 
 
-def make_gk(n_tokens: int, H: int, dk: int, seed: int, device="cpu", strong_every: int = 0):
+def make_gk(n_tokens: int, H: int, dk: int, seed: int, device="cpu", strong_every: int = 0, strong_shift: float = 7.0):
     """Per-channel log-decay gk [C,H,dk] fp32 = log(sigmoid(N(3,1))) (the distribution of the scalar gate, drawn per
-    key channel).  strong_every > 0: every strong_every-th channel gets log(sigmoid(N(-4,1))) instead -- decays of
-    about e^-4 per token, e^-250 over a chunk -- to exercise gates far outside the usual range."""
+    key channel).  strong_every > 0: every strong_every-th channel gets log(sigmoid(N(3 - strong_shift, 1))) instead --
+    with the default shift decays of about e^-4 per token, e^-250 over a chunk -- to exercise gates far outside the usual
+    range."""
     gen = torch.Generator(device=device)
     gen.manual_seed(1000003 * (seed + 1) + 77)
     x = torch.randn(n_tokens, H, dk, generator=gen, device=device, dtype=torch.float32) + 3.0
     if strong_every > 0:
-        x[:, :, ::strong_every] -= 7.0
+        x[:, :, ::strong_every] -= strong_shift
     return torch.nn.functional.logsigmoid(x).contiguous()
 
 
