@@ -155,6 +155,22 @@ __device__ __forceinline__ void load_g(const float* gk, int H, int h, const int*
     }
 }
 
+// Asks the L2 for the rows of chunk c of a [rows, H, 128] tensor (the chunk after the one being worked on: its global
+// loads then find their lines in the L2 instead of waiting for HBM).  Chunks >= 1 hold own rows only, which are
+// consecutive: virtual row vr is physical row own_begin - n_replay + vr.
+template <typename T>
+__device__ __forceinline__ void prefetch_rows(const T* base, int H, int h, const SeqInfo& s, int c) {
+    constexpr int LINES = D * (int)sizeof(T) / 128;              // 128-byte lines per row and head
+    for (int p = threadIdx.x; p < BT * LINES; p += NT) {
+        const int vr = c * BT + p / LINES;
+        if (vr < s.n_virtual) {
+            const char* addr = reinterpret_cast<const char*>(base + ((size_t)(s.own_begin - s.n_replay + vr) * H + h) * D) +
+                               (p % LINES) * 128;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(addr));
+        }
+    }
+}
+
 // running sum over the rows, per channel: four threads per channel (16 rows each, scanned in registers), joined through
 // sTmp[4][128]
 __device__ __forceinline__ void cumsum_rows(float* sB, float* sTmp) {
@@ -522,6 +538,12 @@ gk_mma_fwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         load_tile_bf16(q, H, h, srow, true, sQ);
         load_tile_bf16(v, H, h, srow, false, sV);
         load_g(gk, H, h, srow, sB);
+        if (c + 1 < s.n_chunks) {
+            prefetch_rows(k, H, h, s, c + 1);
+            prefetch_rows(q, H, h, s, c + 1);
+            prefetch_rows(v, H, h, s, c + 1);
+            prefetch_rows(gk, H, h, s, c + 1);
+        }
         // start-of-chunk state: operand copy, kept for the backward, exported when the plan requests this boundary
         state_to_operand(st, sSb, warp, lane);
         const bool exported = next_req < s.req_hi && tb.slot_chunk[next_req] == c;
@@ -726,6 +748,17 @@ gk_mma_bwd_kernel(harts_la_tables_t tb, int seq_lo, int H, const __nv_bfloat16* 
         load_tile_bf16(dO, H, h, srow, true, sDO);
         load_g(gk, H, h, srow, sB);
         global_to_tile128(chunk_states + ((size_t)(s.chunk_base + c) * H + h) * state_elems, sSc);
+        if (c >= 1) {      // the next chunk of the walk (chunk 0 of a sequence with replayed rows is not consecutive)
+            if (c - 1 >= 1 || s.n_replay == 0) {
+                prefetch_rows(k, H, h, s, c - 1);
+                prefetch_rows(q, H, h, s, c - 1);
+                prefetch_rows(v, H, h, s, c - 1);
+                prefetch_rows(dO, H, h, s, c - 1);
+                prefetch_rows(gk, H, h, s, c - 1);
+            }
+            const char* st = reinterpret_cast<const char*>(chunk_states + ((size_t)(s.chunk_base + c - 1) * H + h) * state_elems);
+            for (int p = tid; p < D * D * 2 / 128; p += NT) asm volatile("prefetch.global.L2 [%0];" ::"l"(st + p * 128));
+        }
         state_to_operand(ds, sdSb, warp, lane);
         __syncthreads();
         cumsum_rows(sB, sTmp);
