@@ -72,6 +72,32 @@ __device__ __forceinline__ SeqInfo seq_info(const harts_la_tables_t& tb, int seq
     return s;
 }
 
+// Asks the L2 for what the NEXT work item of this CTA reads first: its initial state and the rows of its first chunk
+// (q, k, v).  Out of line, so that it does not weigh on the kernel's register allocation; called once per item, while
+// the item's last chunk waits for its MMAs.
+__device__ __noinline__ void prefetch_item(const harts_la_tables_t& tb, int seq_lo, int item, int H, const float* slots,
+                                           const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v) {
+    const int sp = seq_lo + item / H, h = item % H;
+    const int seq = tb.seq_order ? tb.seq_order[sp] : sp;
+    const int own_begin = tb.seq_own_begin[seq], own_len = tb.seq_own_begin[seq + 1] - own_begin;
+    const int replay_base = tb.seq_replay_ptr[seq], n_replay = tb.seq_replay_ptr[seq + 1] - replay_base;
+    const int init_slot = tb.seq_init_slot[seq];
+    const int tid = threadIdx.x;
+    if (init_slot >= 0) {
+        const char* st = reinterpret_cast<const char*>(slots + ((size_t)init_slot * H + h) * (size_t)(D * D));
+        for (int p = tid; p < D * D * 4 / 128; p += NT) asm volatile("prefetch.global.L2 [%0];" ::"l"(st + p * 128));
+    }
+    const int n_rows = min(BT, n_replay + own_len);
+    for (int p = tid; p < n_rows * 2; p += NT) {
+        const int vr = p >> 1;
+        const int r = vr < n_replay ? tb.replay_row[replay_base + vr] : own_begin + (vr - n_replay);
+        const size_t off = (((size_t)r * H + h) * D) * 2 + (p & 1) * 128;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(k) + off));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(v) + off));
+        if (vr >= n_replay) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(q) + off));
+    }
+}
+
 // out of line: the wait loop's registers (timer values, counters) must not weigh on the kernel's allocation
 __device__ __noinline__ void wait_for_slot(const int* flag, int* status, int* dead) { flag_wait(flag, status, dead); }
 
@@ -377,6 +403,13 @@ tc_fwd_kernel(const harts_la_tables_t tb, int seq_lo, int n_items, int H, const 
             for (int ks = 0; ks < 4; ks++)
                 mma_ss(tmem + COL_S, desc_mnmajor<BT>(aK, ks), desc_mnmajor<BT>(aV, ks), IDESC_S, true);
             mma_commit(&m.bar_o);
+        }
+        if constexpr (!ONE_LAUNCH) {
+            if (c == s.n_chunks - 1) {                      // the next item of this CTA (snake order), if there is one
+                const int nt = tier + 1;
+                const int nxt = (nt & 1) ? nt * G + (G - 1 - (int)blockIdx.x) : nt * G + (int)blockIdx.x;
+                if (nxt < n_items) prefetch_item(tb, seq_lo, nxt, H, slots, q, k, v);
+            }
         }
         mbar_wait(&m.bar_o, ph_o, status, &m.dead);
         ph_o ^= 1;
