@@ -923,8 +923,9 @@ class GkWorkload:
         import paper_2608_28158_b200 as H
         from workloads import CONFIGS, config_forest, make_gk, make_inputs
         self.H, self.args, self.ranks = H, args, ranks
-        self.cfg = cfg = CONFIGS[GK_CONFIG]
-        fo = config_forest(GK_CONFIG)
+        self.trees = trees = getattr(args, "gk_trees", GK_CONFIG)
+        self.cfg = cfg = CONFIGS[trees]
+        fo = config_forest(trees)
         self.plan = plan = H.harts_la_plan(fo.tree_node_ptr, fo.node_parent, fo.node_fork_off, fo.node_len, 64).upload()
         Hh, d = cfg["H"], cfg["dk"]
         self.inp = inp = make_inputs(plan.C, Hh, d, d, "bf16", 60 + ranks.rank, device="cuda")
@@ -970,13 +971,14 @@ class GkWorkload:
         fwd_bytes = th * (3 * d * 2 + 4 * d + 2 * d)
         bwd_bytes = th * (4 * d * 2 + 4 * d + 3 * d * 2 + 4 * d)
         K = plan.n_rounds
-        # what bounds the kernels by design is the exponentials of the decay-dependent sums (about 330 k per chunk-head
-        # in both passes together, 16 per clock and SM): reported beside the HBM figure
+        # beside the HBM figure: the time the special-function unit needs for the exponentials of the decayed operands
+        # (anchored q / k tiles, q~ / k~, the factors applied to the block products: about 135 k per chunk-head in both
+        # passes together when every chunk is mild, 16 per clock and SM)
         import torch
         one_launch = (not self.flags and 1 < K <= 32 and
                       plan.n_seq * Hh <= 8 * torch.cuda.get_device_properties(0).multi_processor_count)
         chunk_heads = plan.n_chunks * Hh
-        sfu_ms = chunk_heads * 330e3 / (148 * 16 * 1.965e9) * 1e3
+        sfu_ms = chunk_heads * 135e3 / (148 * 16 * 1.965e9) * 1e3
         roof = hbm_roofline("gk_mma_bwd_kernel (all rounds)", bwd_bytes / K, kernel_ms["bwd"] / K, peaks, None,
                             forward={"achieved": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9,
                                      "frac": fwd_bytes / (kernel_ms["fwd"] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
@@ -984,7 +986,7 @@ class GkWorkload:
                                         "frac_strict": (fwd_bytes + bwd_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3 / ms_step,
                                         "exponential_unit_ms": sfu_ms, "frac_exponential_unit": sfu_ms / ms_step})
         return {"dtype": "bf16",
-                "config": {"workload": "gk", "trees": GK_CONFIG, "H": Hh, "dk": d, "dv": d, "chunk": 64,
+                "config": {"workload": "gk", "trees": self.trees, "H": Hh, "dk": d, "dv": d, "chunk": 64,
                            "compact_tokens": plan.C, "rounds": K, "sequences": plan.n_seq, "chunks": plan.n_chunks,
                            "inputs": "bf16 q, k, v, dO; fp32 per-channel log-decay; dense products on the tensor cores "
                                      "(mma.sync, bf16 operands, fp32 accumulation), in-block pair sums in fp32 on the CUDA cores",
@@ -1165,6 +1167,7 @@ def main(argv=None):
     ap.add_argument("--logp-rows", type=int, default=LOGP_ROWS, help="compact-row capacity of the logp workload")
     ap.add_argument("--conv-trees", default="cfg3", help="forest of the conv workload (cfg2: a small case for captures)")
     ap.add_argument("--attn-trees", default="cfg2", help="forest of the attn workload (cfg1: a small case for captures)")
+    ap.add_argument("--gk-trees", default=GK_CONFIG, help="forest (and head count) of the gk workload: cfg1, cfg2 or cfg3")
     ap.add_argument("--attn-kv-heads", type=int, default=ATTN_H, help="kv heads of the attn workload (16 = MHA)")
     ap.add_argument("--per-config", action="store_true", help="also print a table over all configurations to stderr")
     args = ap.parse_args(argv)
