@@ -117,7 +117,11 @@ attn_dq_kernel(Index ix, int Hq, int G, float scale, const __grid_constant__ CUt
     uint32_t ph_q = 0, ph_k[KST] = {}, ph_v[2] = {0, 0}, ph_kfree[KST] = {}, ph_vfree[2] = {0, 0}, ph_s = 0, ph_p[2] = {0, 0},
              ph_dpfree = 0, ph_o = 0;
     const int n_work = ix.n_q_items * Hq;
-    for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
+    // work items come most work first; dealt in a snake pattern (tier by tier, every second tier in reverse), so that no
+    // CTA gets the largest item of every tier
+    for (int tier = 0; tier * (int)gridDim.x < n_work; tier++) {
+        const int w = tier * (int)gridDim.x + ((tier & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x);
+        if (w >= n_work) continue;
         const int item = w / Hq, h = w % Hq, hk = h / G;
         const int piece = ix.q_item[2 * item], qt = ix.q_item[2 * item + 1];
         const int q_row0 = ix.piece_row0[piece] + qt * BQ;

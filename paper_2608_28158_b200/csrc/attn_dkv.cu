@@ -81,7 +81,11 @@ attn_dkv_kernel(Index ix, int Hq, int Hkv, int G, float scale, const __grid_cons
 
     uint32_t ph_kv = 0, ph_q[STAGES] = {}, ph_free[STAGES] = {}, ph_s[2] = {0, 0}, ph_p[2] = {0, 0}, ph_o = 0;
     const int n_work = ix.n_kv_items * Hkv;
-    for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
+    // work items come most work first; dealt in a snake pattern (tier by tier, every second tier in reverse), so that no
+    // CTA gets the largest item of every tier
+    for (int tier = 0; tier * (int)gridDim.x < n_work; tier++) {
+        const int w = tier * (int)gridDim.x + ((tier & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x);
+        if (w >= n_work) continue;
         const int item = w / Hkv, hk = w % Hkv;
         const int piece = ix.kv_item[2 * item], kt = ix.kv_item[2 * item + 1];
         const int kv_row0 = ix.piece_row0[piece] + kt * BKV;
