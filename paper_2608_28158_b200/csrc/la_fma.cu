@@ -413,28 +413,56 @@ __global__ void __launch_bounds__(NT) fma_bwd_kernel(harts_la_tables_t tb, int s
     }
 }
 
-// dk/dv/dg of a replayed row += the contributions of every sequence that replayed it.
+// dk/dv/dg of a replayed row += the contributions of every sequence that replayed it (summed in table order).  A group
+// of (DK + DV) / 4 threads serves one (row, head): every thread owns four consecutive channels of dk or dv (16-byte
+// loads of the fp32 contributions), the group's first thread the scalar dg as well.
+template <typename T>
+__device__ __forceinline__ void add4(T* p, const float4& a);
+template <>
+__device__ __forceinline__ void add4<float>(float* p, const float4& a) {
+    float4 x = *reinterpret_cast<float4*>(p);
+    x.x += a.x; x.y += a.y; x.z += a.z; x.w += a.w;
+    *reinterpret_cast<float4*>(p) = x;
+}
+template <>
+__device__ __forceinline__ void add4<__nv_bfloat16>(__nv_bfloat16* p, const float4& a) {
+    uint2 raw = *reinterpret_cast<uint2*>(p);
+    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
+    float2 lo = __bfloat1622float2(h2[0]), hi = __bfloat1622float2(h2[1]);
+    h2[0] = __floats2bfloat162_rn(lo.x + a.x, lo.y + a.y);
+    h2[1] = __floats2bfloat162_rn(hi.x + a.z, hi.y + a.w);
+    *reinterpret_cast<uint2*>(p) = raw;
+}
+
 template <typename T>
 __global__ void replay_reduce_kernel(harts_la_tables_t tb, int H, int DK, int DV, T* dk_, T* dv_, float* dg,
-                                     const float* rk, const float* rv, const float* rg) {
-    const int m = blockIdx.x / H, h = blockIdx.x % H;
+                                     const float* rk, const float* rv, const float* rg, int n_items) {
+    const int per = (DK + DV) / 4;
+    const int item = blockIdx.x * (blockDim.x / per) + threadIdx.x / per, part = threadIdx.x % per;
+    if (item >= n_items) return;
+    const int m = item / H, h = item % H;
     const int row = tb.rg_row[m];
     const int lo = tb.rg_ptr[m], hi = tb.rg_ptr[m + 1];
-    for (int i = threadIdx.x; i < DK + DV + 1; i += blockDim.x) {
-        float acc = 0.f;
-        if (i < DK) {
-            for (int e = lo; e < hi; e++) acc += rk[((size_t)tb.rg_entry[e] * H + h) * DK + i];
-            T* p = dk_ + ((size_t)row * H + h) * DK + i;
-            *p = from_f<T>(to_f(*p) + acc);
-        } else if (i < DK + DV) {
-            int j = i - DK;
-            for (int e = lo; e < hi; e++) acc += rv[((size_t)tb.rg_entry[e] * H + h) * DV + j];
-            T* p = dv_ + ((size_t)row * H + h) * DV + j;
-            *p = from_f<T>(to_f(*p) + acc);
-        } else {
-            for (int e = lo; e < hi; e++) acc += rg[(size_t)tb.rg_entry[e] * H + h];
-            dg[(size_t)row * H + h] += acc;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (part * 4 < DK) {
+        const int i = part * 4;
+        for (int e = lo; e < hi; e++) {
+            const float4 x = *reinterpret_cast<const float4*>(rk + ((size_t)tb.rg_entry[e] * H + h) * DK + i);
+            acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
         }
+        add4<T>(dk_ + ((size_t)row * H + h) * DK + i, acc);
+    } else {
+        const int j = part * 4 - DK;
+        for (int e = lo; e < hi; e++) {
+            const float4 x = *reinterpret_cast<const float4*>(rv + ((size_t)tb.rg_entry[e] * H + h) * DV + j);
+            acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+        }
+        add4<T>(dv_ + ((size_t)row * H + h) * DV + j, acc);
+    }
+    if (part == 0) {
+        float g = 0.f;
+        for (int e = lo; e < hi; e++) g += rg[(size_t)tb.rg_entry[e] * H + h];
+        dg[(size_t)row * H + h] += g;
     }
 }
 
@@ -555,12 +583,14 @@ int32_t replay_reduce(const harts_la_tables_t& tb, void* dk_, void* dv_, float* 
     const float* rk = (const float*)(base + sl.rk);
     const float* rv = (const float*)(base + sl.rv);
     const float* rg = (const float*)(base + sl.rg);
-    int n = tb.n_rg_rows * H;
+    const int n = tb.n_rg_rows * H, per = (dk + dv) / 4, threads = 256;
+    if ((dk + dv) % 4 != 0 || dk % 4 != 0 || threads % per != 0) return HARTS_EUNSUPPORTED;
+    const int blocks = (n + threads / per - 1) / (threads / per);
     if (dtype == HARTS_FP32)
-        replay_reduce_kernel<float><<<n, 128, 0, stream>>>(tb, H, dk, dv, (float*)dk_, (float*)dv_, dg, rk, rv, rg);
+        replay_reduce_kernel<float><<<blocks, threads, 0, stream>>>(tb, H, dk, dv, (float*)dk_, (float*)dv_, dg, rk, rv, rg, n);
     else
-        replay_reduce_kernel<__nv_bfloat16><<<n, 128, 0, stream>>>(tb, H, dk, dv, (__nv_bfloat16*)dk_,
-                                                                   (__nv_bfloat16*)dv_, dg, rk, rv, rg);
+        replay_reduce_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(tb, H, dk, dv, (__nv_bfloat16*)dk_,
+                                                                            (__nv_bfloat16*)dv_, dg, rk, rv, rg, n);
     return cudaGetLastError() == cudaSuccess ? HARTS_OK : HARTS_ECUDA;
 }
 
