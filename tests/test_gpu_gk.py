@@ -101,6 +101,44 @@ def test_gates_far_outside_the_usual_range_do_not_overflow():
     check(errs, "bf16")
 
 
+def test_bench_size_sampled_parity():
+    """The benchmark's workload for this path -- cfg2's forest, 16 heads, d = 128, bf16, all rounds in one launch per
+    pass, every chunk on the dense-diagonal path -- with the oracle on two whole trees x three heads."""
+    from workloads import CONFIGS
+    fo = config_forest("cfg2")
+    heads, d = CONFIGS["cfg2"]["H"], 128
+    inp = make_inputs(fo.n_tokens, heads, d, d, "bf16", 21, device="cuda")
+    inp["g"] = make_gk(fo.n_tokens, heads, d, 21, device="cuda")
+    plan = plan_of(fo).upload()
+    phys = to_physical(plan, inp)
+    cs_bytes, sc_bytes = H.harts_la_gk_workspace_bytes(plan.tables, heads, d, d, 1)
+    slots = torch.full((max(plan.n_slots, 1) * heads * d * d,), float("nan"), device="cuda")
+    cs = torch.empty(cs_bytes, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(sc_bytes, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    out = {n: torch.full_like(phys[m], float("nan")) for n, m in (("o", "v"), ("dq", "q"), ("dk", "k"), ("dv", "v"), ("dg", "g"))}
+    H.harts_la_gk_fwd(plan, 0, phys["q"], phys["k"], phys["v"], phys["g"], out["o"], slots, cs, dev_status=status)
+    H.harts_la_gk_bwd(plan, 0, phys["q"], phys["k"], phys["v"], phys["g"], phys["dO"], out["dq"], out["dk"], out["dv"],
+                      out["dg"], cs, scratch, dev_status=status)
+    H.harts_la_check(status)
+    rows = torch.as_tensor(plan.row_of_token.astype(np.int64), device="cuda")
+    trees, hs = [1, 6], [0, heads // 2, heads - 1]
+    base = fo.token_base()
+    tok = np.concatenate([np.arange(base[fo.tree_node_ptr[t]], base[fo.tree_node_ptr[t + 1]]) for t in trees])
+    sub = fo.subset(trees)
+    ti, hi = torch.as_tensor(tok, device="cuda"), torch.as_tensor(hs, device="cuda")
+    pick = {n: x[ti][:, hi].cpu() for n, x in inp.items()}
+    ref = go.forest_eval(sub, pick["q"], pick["k"], pick["v"], pick["g"], pick["dO"])
+    errs = {}
+    for n, x in out.items():
+        assert torch.isfinite(x.float()).all(), n
+        got = x[rows][ti][:, hi].float().cpu().numpy()
+        errs[n] = rel_err(got, ref[n])
+        errs[n + ".row"] = row_err(got, ref[n])
+    print("cfg2 gk", errs)
+    check(errs, "bf16")
+
+
 def test_tensor_core_path_agrees_with_the_cuda_core_path():
     """bf16, d = 128: the same call with HARTS_FLAG_FMA_KERNELS runs the CUDA-core kernels (pair sums over whole
     chunks, no anchored operands, fp32 products).  Two different decompositions of the same sums, same bf16 roundings of
